@@ -1,0 +1,15 @@
+"""Reference oracle: a plain, slow, float64 CPU statement of what the training path computes.
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product package imports, calls or links this
+code; only the tests, the smoke check and the benchmark's CPU-baseline leg use it.  It
+shares no code with the CUDA library.
+
+Pin status (see tests/test_oracle_*.py):
+  ops forward/backward, loss, SGD, stage split, capacity estimate, partition optimiser,
+  redistribution without failure, snapshot, schedules ........ pinned
+  redistribution with a failed index (Algorithm 1, I_fail >= 0) ... parity unpinned beyond
+  the invariants and the two prose rules of Sec. III-F (the worked figures are not available)
+"""
+from .ops import *          # noqa: F401,F403
+from .model import OracleModel   # noqa: F401
+from .partition import *    # noqa: F401,F403

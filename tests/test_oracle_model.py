@@ -1,0 +1,165 @@
+"""Pins for the oracle's model driver: whole-network finite differences, stage split equals the
+unsplit run, SGD closed forms, an independent float64 autograd cross-check, snapshot layout."""
+import numpy as np
+import pytest
+
+import oracle
+import synth
+
+
+def build(net, idx=9, **kw):
+    ls, cfg = net(**kw)
+    return ls, cfg, oracle.OracleModel(ls, cfg, synth.init_params(idx, ls), synth.init_state(ls))
+
+
+def loss_of(m, x, y):
+    keep = [[a.copy() for a in s] for s in m.s]
+    v = m.forward(0, m.L, x, y)
+    m.s = keep
+    return float(v)
+
+
+@pytest.mark.parametrize("net", [synth.tiny_mbv2, synth.tiny_vgg, lambda: synth.har_cnn(3, 2, 12, 4, 3)])
+def test_whole_network_gradients_by_finite_differences(net):
+    ls, cfg, m = build(net)
+    rng = np.random.default_rng(3)
+    for arrs in m.p:                       # move off the symmetric init (beta 0, bias 0)
+        for a in arrs:
+            a += 0.1 * rng.standard_normal(a.shape)
+    x, y = synth.make_batch(9, cfg)
+    x = x.astype(np.float64)
+    m.forward(0, m.L, x, y)
+    m.backward(0, m.L)
+    h, checked = 1e-6, 0
+    for i, arrs in enumerate(m.p):
+        for k, a in enumerate(arrs):
+            flat = a.reshape(-1)
+            for j in rng.choice(flat.size, size=min(3, flat.size), replace=False):
+                old = flat[j]
+                flat[j] = old + h
+                fp = loss_of(m, x, y)
+                flat[j] = old - h
+                fm = loss_of(m, x, y)
+                flat[j] = old
+                num = (fp - fm) / (2 * h)
+                ana = m.g[i][k].reshape(-1)[j]
+                assert abs(num - ana) <= 1e-6 + 1e-4 * abs(ana), (i, k, j, num, ana)
+                checked += 1
+    assert checked > 20
+
+
+@pytest.mark.parametrize("net", [synth.tiny_mbv2, synth.tiny_vgg, synth.har_cnn])
+def test_split_equals_unsplit_exactly(net):
+    ls, cfg, ref = build(net)
+    x, y = synth.make_batch(9, cfg)
+    L = ref.L
+    ref.step([0, L], x, y)
+    ref.step([0, L], x, y)
+    for pts in ([0, 1, L], [0, 2, L], [0, L - 1, L], [0, 1, 2, L], list(range(L + 1))):
+        _, _, m = build(net)
+        m.step(pts, x, y)
+        m.step(pts, x, y)
+        assert m.loss == ref.loss
+        for u in range(L):
+            assert np.array_equal(m.unit_params(u), ref.unit_params(u))
+            assert np.array_equal(m.unit_grads(u), ref.unit_grads(u))
+            assert np.array_equal(m.unit_state(u), ref.unit_state(u))
+
+
+def test_boundary_tensors_of_a_split_run():
+    ls, cfg, m = build(synth.tiny_mbv2)
+    x, y = synth.make_batch(9, cfg)
+    act = m.forward(0, 3, x)
+    assert act.shape[0] == cfg["batch"] and act.ndim == 4
+    m.forward(3, m.L, act, y)
+    g = m.backward(3, m.L)
+    assert g.shape == act.shape                 # boundary gradient is shaped like the boundary activation
+    assert m.backward(0, 3, g).shape == x.shape
+
+
+def test_sgd_closed_forms():
+    ls, cfg = synth.har_cnn(2, 1, 4, 1, 2)
+    cfg.update(lr=0.5, momentum=0.9, weight_decay=0.1)
+    m = oracle.OracleModel(ls, cfg, synth.init_params(1, ls), synth.init_state(ls))
+    w0 = m.p[0][0].copy()
+    g = np.full_like(w0, 2.0)
+    m.g[0][0] = g.copy()
+    m.sgd(0, 1)                                  # first step: buffer = g + wd*w
+    m1 = g + 0.1 * w0
+    w1 = w0 - 0.5 * m1
+    assert np.allclose(m.p[0][0], w1)
+    m.g[0][0] = g.copy()
+    m.sgd(0, 1)
+    m2 = 0.9 * m1 + (g + 0.1 * w1)
+    assert np.allclose(m.p[0][0], w1 - 0.5 * m2)
+    cfg.update(momentum=0.0, weight_decay=0.0)   # reduces to w - lr*g
+    m = oracle.OracleModel(ls, cfg, synth.init_params(1, ls), synth.init_state(ls))
+    m.g[0][0] = g.copy()
+    m.sgd(0, 1, lr=0.25)
+    assert np.allclose(m.p[0][0], w0 - 0.25 * g)
+    assert np.array_equal(m.p[1][0], synth.init_params(1, ls)[1][0])   # units outside [a,b) untouched
+
+
+def _torch_reference(ls, cfg, params, x, y):
+    """The same network through torch's float64 CPU autograd: a library cross-check."""
+    import torch
+    import torch.nn.functional as F
+    K = synth.KIND
+    ps = [[torch.tensor(np.asarray(a, np.float64), requires_grad=True) for a in arrs] for arrs in params]
+    outs = {-1: torch.tensor(x.astype(np.float64)).permute(0, 3, 1, 2)}
+    for i, l in enumerate(ls):
+        t = outs[i - 1]
+        if l.kind in (K["CONV1D"], K["CONV2D"], K["FC"]):
+            w = ps[i][0].permute(3, 2, 0, 1)
+            pad = (0, l.pad) if l.kind == K["CONV1D"] else (l.pad, l.pad)
+            t = F.conv2d(t, w, ps[i][1] if l.has_bias else None, stride=l.stride, padding=pad)
+        elif l.kind == K["DWCONV3x3"]:
+            t = F.conv2d(t, ps[i][0].permute(2, 0, 1).unsqueeze(1), None, stride=l.stride, padding=1, groups=l.cin)
+        elif l.kind == K["BN"]:
+            t = F.batch_norm(t, None, None, ps[i][0], ps[i][1], training=True, eps=cfg["bn_eps"])
+        elif l.kind == K["ADD_RESIDUAL"]:
+            t = t + outs[l.residual_src]
+        elif l.kind == K["MAXPOOL2"]:
+            t = F.max_pool2d(t, 2)
+        elif l.kind == K["GAP"]:
+            t = t.mean((2, 3), keepdim=True)
+        elif l.kind == K["SOFTMAX_CE"]:
+            t = F.cross_entropy(t.flatten(1), torch.tensor(y, dtype=torch.long))
+        if l.kind != K["SOFTMAX_CE"]:
+            t = F.relu(t) if l.act == 1 else (F.relu6(t) if l.act == 2 else t)
+        outs[i] = t
+    outs[len(ls) - 1].backward()
+    return float(outs[len(ls) - 1].detach()), [[p.grad.numpy() for p in arrs] for arrs in ps]
+
+
+@pytest.mark.parametrize("net", [synth.tiny_mbv2, synth.tiny_vgg, synth.har_cnn])
+def test_against_float64_autograd(net):
+    ls, cfg, m = build(net)
+    x, y = synth.make_batch(9, cfg)
+    m.forward(0, m.L, x, y)
+    m.backward(0, m.L)
+    loss, grads = _torch_reference(ls, cfg, synth.init_params(9, ls), x, y)
+    assert abs(loss - m.loss) < 1e-12
+    for i, arrs in enumerate(grads):
+        for k, g in enumerate(arrs):
+            assert np.allclose(m.g[i][k], g, rtol=1e-9, atol=1e-12), (i, k)
+
+
+def test_bn_running_statistics_use_unbiased_variance():
+    ls, cfg, m = build(synth.tiny_vgg)
+    x, y = synth.make_batch(9, cfg)
+    m.forward(0, 1, x)
+    conv = m.out[0].reshape(-1, 8)
+    assert np.allclose(m.s[1][0], 0.1 * conv.mean(0))
+    assert np.allclose(m.s[1][1], 0.9 + 0.1 * conv.var(0, ddof=1))
+
+
+def test_snapshot_layout():
+    ls, cfg, m = build(synth.tiny_vgg)
+    snap = m.snapshot(0, m.L)
+    n_par = sum(int(np.prod(s)) for l in ls for s in synth.param_shapes(l))
+    n_st = sum(int(np.prod(s)) for l in ls for s in synth.state_shapes(l))
+    assert snap.dtype == np.float32 and snap.size == n_par + n_st
+    u0 = synth.flat_unit_params(ls, synth.init_params(9, ls), 0)
+    assert np.array_equal(snap[:u0.size], u0)
+    assert np.array_equal(np.concatenate([m.snapshot(0, 1), m.snapshot(1, m.L)]), snap)

@@ -1,0 +1,130 @@
+"""Pins for capacity estimate (Eq. 1-3), partition optimiser (Eq. 4-7), Algorithm 1 and schedules."""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+
+RNG = np.random.default_rng(11)
+
+
+def exact_inputs(L, N, comm):
+    """Integer times and dyadic capacities: every sum and product is exact in float64."""
+    t = [float(v) for v in RNG.integers(1, 40, size=L)]
+    c = [float(v) for v in RNG.choice([0.5, 1.0, 2.0, 4.0, 8.0, 1.5], size=N)]
+    if not comm:
+        return t, c, None, None
+    d = [float(v) for v in RNG.integers(1, 64, size=L)]
+    bw = [float(v) for v in RNG.choice([1.0, 2.0, 4.0], size=N - 1)]
+    return t, c, d, bw
+
+
+@pytest.mark.parametrize("comm", [False, True])
+def test_dp_equals_brute_force_every_cell(comm):
+    for L, N in [(1, 1), (2, 2), (5, 1), (6, 3), (7, 4), (9, 5), (8, 8)]:
+        for _ in range(6):
+            t, c, d, bw = exact_inputs(L, N, comm)
+            A, cut = oracle.partition_table(t, c, d, bw)
+            for n in range(1, N + 1):
+                for j in range(n - 1, L):       # every prefix problem
+                    _, best = oracle.brute_force_partition(t[:j + 1], c[:n], None if d is None else d[:j + 1],
+                                                           None if bw is None else bw[:n - 1])
+                    assert A[n][j] == best
+            pts, bott = oracle.choose_partition(t, c, d, bw)
+            _, best = oracle.brute_force_partition(t, c, d, bw)
+            assert bott == best == oracle.stage_cost(pts, t, c, d, bw)
+            assert pts[0] == 0 and pts[-1] == L and all(a < b for a, b in zip(pts, pts[1:]))
+            # canonical tie rule: last cut = smallest l reaching the optimum, recursively
+            j, n = L - 1, N
+            for p in reversed(pts[1:-1]):
+                cands = [l for l in range(n - 2, j)
+                         if max(A[n - 1][l], 0.0 if d is None else 2.0 * (d[l] / bw[n - 2]),
+                                c[n - 1] * (sum(t[:j + 1]) - sum(t[:l + 1]))) == A[n][j]]
+                assert p - 1 == min(cands)
+                j, n = p - 1, n - 1
+
+
+def test_dp_special_cases():
+    assert oracle.choose_partition([3.0, 1.0, 2.0], [1.0]) == ([0, 3], 6.0)
+    assert oracle.choose_partition([1.0] * 12, [1.0] * 4) == ([0, 3, 6, 9, 12], 3.0)
+    t = [float(v) for v in RNG.integers(1, 9, size=10)]
+    c = [1.0, 2.0, 4.0]
+    p1, b1 = oracle.choose_partition(t, c)
+    p2, b2 = oracle.choose_partition(t, [4.0 * v for v in c])      # common scale: same points
+    assert p1 == p2 and b2 == 4.0 * b1
+    # a 10x slower last stage gets fewer units than a fast one
+    fast, _ = oracle.choose_partition([1.0] * 20, [1.0, 1.0, 1.0])
+    slow, _ = oracle.choose_partition([1.0] * 20, [1.0, 1.0, 10.0])
+    assert slow[-1] - slow[-2] < fast[-1] - fast[-2]
+    # an expensive link moves the cut to the small boundary
+    pts, _ = oracle.choose_partition([1.0] * 4, [1.0, 1.0], [100.0, 100.0, 1.0, 100.0], [10.0])
+    assert pts == [0, 3, 4]
+    with pytest.raises(ValueError):
+        oracle.choose_partition([1.0, 1.0], [1.0, 1.0, 1.0])
+
+
+def test_capacity_estimate_recovers_slowdown_factors():
+    t = [float(v) for v in RNG.integers(1, 9, size=9)]
+    pts = [0, 2, 5, 9]
+    f = [1.0, 2.5, 10.0]
+    stage = [f[i] * sum(t[a:b]) for i, (a, b) in enumerate(zip(pts, pts[1:]))]
+    assert np.allclose(oracle.estimate_capacity(t, pts, stage), f)
+    stage[0] *= 3.0                                   # C_0 is 1.0 by definition whatever stage 0 reports
+    assert oracle.estimate_capacity(t, pts, stage)[0] == 1.0
+
+
+def all_partitions(L, N):
+    for cuts in itertools.combinations(range(1, L), N - 1):
+        yield [0] + list(cuts) + [L]
+
+
+def test_redistribution_without_failure_invariants():
+    L, N = 7, 3
+    for p_cur in all_partitions(L, N):
+        for p_new in all_partitions(L, N):
+            for i in range(N):
+                need, local = oracle.redistribution_plan(p_new, p_cur, i, i)
+                got = sorted(local + [l for v in need.values() for l in v])
+                assert got == list(range(p_new[i], p_new[i + 1]))           # covers the new range once
+                assert all(p_cur[i] <= l < p_cur[i + 1] for l in local)     # local = already held
+                for owner, units in need.items():
+                    assert owner != i
+                    assert all(p_cur[owner] <= l < p_cur[owner + 1] for l in units)
+                if p_new == p_cur:
+                    assert need == {} and local == list(range(p_cur[i], p_cur[i + 1]))
+
+
+def test_redistribution_failure_rules_from_the_prose():
+    # Sec. III-F: 4 workers, worker 1 fails; survivors 0,2,3 become 0,1,2.
+    p_cur, p_new = [0, 2, 4, 6, 8], [0, 3, 6, 8]
+    assert oracle.renew_worker_list([0, 1, 2, 3], [1]) == [0, 2, 3]
+    # old worker 2 (new index 1) needs units 3..5: unit 3 was the failed worker's -> its replica sits
+    # on failed+1, whose new index equals the failed index (target unchanged); 4,5 are its own.
+    need, local = oracle.redistribution_plan(p_new, p_cur, 2, 1, i_fail=1)
+    assert local == [4, 5] and need == {1: [3]}
+    # old worker 0 needs unit 2 (failed worker's) -> index 1 as well
+    need, local = oracle.redistribution_plan(p_new, p_cur, 0, 0, i_fail=1)
+    assert local == [0, 1] and need == {1: [2]}
+    # old worker 3 (new 2): target above the failed index moves down by one
+    need, local = oracle.redistribution_plan([0, 2, 5, 8], p_cur, 3, 2, i_fail=1)
+    assert local == [6, 7] and need == {1: [5]}      # unit 5 lived on old worker 2 -> new index 1
+    # last stage fails: its replica is on the central node, index 0
+    need, local = oracle.redistribution_plan([0, 3, 6, 8], p_cur, 2, 2, i_fail=3)
+    assert local == [] or all(4 <= l < 6 for l in local)
+    assert need.get(0) == [6, 7]
+
+
+def test_schedules_match_the_paper(golden_dir):
+    facts = {}
+    for line in open(golden_dir + "/schedule_ticks.txt"):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            facts[k] = int(v)
+    first, period = facts["repartition_first_batches"], facts["repartition_period"]
+    hits = [it + 1 for it in range(450) if oracle.is_repartition_iter(it)]
+    assert hits == [first, period, 2 * period, 3 * period, 4 * period]
+    chain = [it + 1 for it in range(210) if oracle.is_replication_iter(it, facts["chain_period"])]
+    glob = [it + 1 for it in range(210) if oracle.is_replication_iter(it, facts["global_period"])]
+    assert chain == [50, 100, 150, 200] and glob == [100, 200]
+    assert facts["both_replications_after_batch"] in chain and facts["both_replications_after_batch"] in glob
