@@ -1,0 +1,238 @@
+/*
+ * ftpipe.h -- C ABI of the per-stage training library (single B200, sm_100a).
+ *
+ * The calls follow the problem statement of FTPipeHD (Chen et al., arXiv 2110.02781):
+ * a DNN is cut into contiguous ranges of layers ("stages", Sec. III-B); every stage runs
+ * the forward pass, the backward pass and the SGD update of its range (Sec. III-C, IV-B);
+ * a per-layer time profile (Sec. III-B "model profiling") feeds the capacity estimate
+ * (Eq. 1-3) and the partition optimiser (Eq. 4-7); after a new partition the weights are
+ * re-homed (Sec. III-D, Algorithm 1) and on a schedule they are replicated to the next
+ * stage and to the central node (Sec. III-E).
+ *
+ * Conventions
+ *   - A "unit" is the paper's layer: what the profile, the optimiser and run_stage index.
+ *     Units are 0-indexed; a partition is N+1 boundaries 0 = p_0 < ... < p_N = L and stage i
+ *     owns units [p_i, p_{i+1}).
+ *   - Activations are channels-last (N, H, W, C); a 1-D signal has H == 1.  Element type is
+ *     float (precision 0) or bfloat16 (precision 1; master weights, gradients, statistics and
+ *     the loss stay float).
+ *   - Canonical parameter order of a unit: its ops in order; per op
+ *       CONV1D/CONV2D/FC : W[kh][kw][cin][cout] then bias[cout] if has_bias
+ *       DWCONV3x3        : W[3][3][c]
+ *       BN               : gamma[c], beta[c]      (state: running_mean[c], running_var[c])
+ *   - Ownership: the CALLER allocates every device and pinned-host buffer, including the
+ *     workspace the model lives in, and supplies the stream (a cudaStream_t passed as void*).
+ *     The library owns only the small host-side ftp_model object.  No call allocates device
+ *     memory.  Pointers marked "device" must be device addresses, "host" host addresses.
+ *   - All GPU work is asynchronous on the given stream unless stated otherwise.
+ *   - Errors: every call returns an ftp_status; arguments are validated before any launch
+ *     and a failed call launches nothing.  ftp_last_error() gives the text for this thread.
+ *     Kernels never trap or assert.
+ */
+#ifndef FTPIPE_H
+#define FTPIPE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ftp_model ftp_model; /* opaque, library-owned */
+
+typedef enum {
+    FTP_OK = 0,
+    FTP_EINVAL = 1,   /* bad argument (null pointer, bad kind, a >= b, N > L, ...) */
+    FTP_ERANGE = 2,   /* index or size out of range, buffer too small or misaligned */
+    FTP_ENOMEM = 3,   /* host allocation failed or workspace too small */
+    FTP_ECUDA = 4,    /* a CUDA runtime call or a launch failed */
+    FTP_ESTATE = 5,   /* call order violated (backward without forward, ...) */
+    FTP_ETIMEOUT = 6, /* a bounded device-side wait ran out */
+    FTP_EUNSUPPORTED = 7
+} ftp_status;
+
+enum { FTP_CONV1D = 0, FTP_CONV2D = 1, FTP_DWCONV3x3 = 2, FTP_BN = 3, FTP_ACT = 4, FTP_ADD_RESIDUAL = 5,
+       FTP_MAXPOOL2 = 6, FTP_GAP = 7, FTP_FC = 8, FTP_SOFTMAX_CE = 9 };
+enum { FTP_ACT_NONE = 0, FTP_ACT_RELU = 1, FTP_ACT_RELU6 = 2 };
+enum { FTP_FP32 = 0, FTP_BF16 = 1 };
+/* selector of ftp_get_tensor / ftp_set_tensor */
+enum { FTP_T_WEIGHTS = 0, FTP_T_GRADS = 1, FTP_T_MOMENTUM = 2, FTP_T_STATE = 3 };
+
+typedef struct {
+    int32_t unit;         /* partition unit of this op; non-decreasing along the list */
+    int32_t kind;         /* FTP_CONV1D ... FTP_SOFTMAX_CE */
+    int32_t cin, cout;    /* channels in / out (BN, pools, ADD: cin == cout) */
+    int32_t k;            /* kernel size (CONV1D: 1 x k; CONV2D: k x k; DW: 3; FC: 1) */
+    int32_t stride, pad;
+    int32_t act;          /* activation applied to this op's output (CONV*, FC, BN, ACT) */
+    int32_t has_bias;
+    int32_t residual_src; /* ADD_RESIDUAL: index of the op whose output is added; -1 otherwise */
+} ftp_layer_desc;
+
+typedef struct {
+    int32_t batch, in_c, in_h, in_w, n_classes;
+    int32_t precision;    /* FTP_FP32 or FTP_BF16 */
+    int32_t max_stages;   /* upper bound on the number of stages (each gets a weight arena) */
+    float lr, momentum, weight_decay, bn_eps, bn_momentum;
+} ftp_model_cfg;
+
+/* One record of the kernel trace (see ftp_trace_enable). */
+typedef struct {
+    int32_t kernel;       /* kernel class id, see ftp_kernel_name */
+    int32_t unit;         /* unit the launch belongs to, -1 if none */
+    int32_t op;           /* op index, -1 if none */
+    int32_t backward;     /* 0 forward, 1 backward, 2 optimiser / copies */
+    float ms;             /* device time of the launch (CUDA events on the launching stream) */
+    double bytes;         /* algorithmic bytes: each input read once, each output written once */
+    double flops;         /* algorithmic floating-point operations */
+} ftp_trace_rec;
+
+/* ---- build_model(layers): Sec. III-B (the central node loads the whole model; a worker
+ * holds the sub-model of its range).  ------------------------------------------------------ */
+
+/* Sizes of the device workspace and of the pinned-host workspace the model needs.
+ * layers: host array of n descriptors.  Pure host arithmetic. */
+ftp_status ftp_workspace_bytes(const ftp_layer_desc* layers, int32_t n, const ftp_model_cfg* cfg,
+                               size_t* dev_bytes, size_t* pinned_bytes);
+
+/* Build the unit table, the per-stage weight arenas (float master weights, momentum, BN
+ * running statistics, bf16 shadow), the gradient arena, the activation stash and the
+ * scratch space inside dev_ws (device, 256-byte aligned, >= dev_bytes) and pinned_ws
+ * (pinned host memory registered for device access, >= pinned_bytes).  The initial partition
+ * is one stage owning every unit.  Arena contents are undefined until ftp_set_tensor.
+ * The workspaces must outlive the model.  Validates the layer list (shapes must chain). */
+ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, const ftp_model_cfg* cfg, void* dev_ws,
+                           size_t dev_bytes, void* pinned_ws, size_t pinned_bytes, ftp_model** out);
+void ftp_destroy_model(ftp_model* m);
+
+ftp_status ftp_num_units(const ftp_model* m, int32_t* L);
+/* Offset and count (in floats) of a unit's trainable parameters / BN running statistics in
+ * the canonical whole-model order. */
+ftp_status ftp_unit_param_span(const ftp_model* m, int32_t unit, int64_t* offset, int64_t* count);
+ftp_status ftp_unit_state_span(const ftp_model* m, int32_t unit, int64_t* offset, int64_t* count);
+/* Shape (N, H, W, C) and byte size of the boundary activation leaving a unit: the D_j of
+ * Eq. 5 (Sec. III-B "size of the output data of each layer"). */
+ftp_status ftp_unit_output_shape(const ftp_model* m, int32_t unit, int32_t shape[4], int64_t* bytes);
+
+/* Copy `count` floats of one unit's tensor (which = FTP_T_*) from / to a host or device
+ * buffer.  Setting the weights also refreshes the bf16 shadow and marks the momentum buffer
+ * of the unit as not yet initialised.  Host copies use pageable-safe synchronous semantics:
+ * when the other side is a host pointer the call returns after the copy has completed. */
+ftp_status ftp_set_tensor(ftp_model* m, int32_t which, int32_t unit, const float* src, int64_t count,
+                          int32_t src_is_device, void* stream);
+ftp_status ftp_get_tensor(const ftp_model* m, int32_t which, int32_t unit, float* dst, int64_t count,
+                          int32_t dst_is_device, void* stream);
+
+/* ---- run_stage(a, b, micro_batch): Sec. III-B / III-C.  -------------------------------- */
+
+/* Forward of units [a, b) on one micro-batch.
+ *   act_in  : device; the input batch (a == 0) or the boundary activation leaving unit a-1.
+ *   act_out : device; receives the boundary activation leaving unit b-1; must be NULL when
+ *             b == L (the last unit ends in the loss).
+ *   labels  : device int32[batch], required iff b == L.
+ *   loss_out: device float[1], required iff b == L; mean softmax cross-entropy.
+ * act_in and act_out must stay valid and unmodified until the backward pass of the same
+ * range has completed (they are read again there; nothing is copied).  Updates the BN
+ * running statistics of the range. */
+ftp_status ftp_run_stage_forward(ftp_model* m, int32_t a, int32_t b, const void* act_in, void* act_out,
+                                 const int32_t* labels, float* loss_out, void* stream);
+
+/* Backward of units [a, b) using the values stashed by the last forward of the same range.
+ *   grad_out: device; gradient of the loss w.r.t. the boundary activation leaving unit b-1
+ *             (same shape and type); must be NULL when b == L.
+ *   grad_in : device; receives the gradient w.r.t. act_in; may be NULL when a == 0.
+ * Leaves the weight gradients of the range in the gradient arena (float).  Every reduction
+ * has a fixed order: results do not depend on how the units are grouped into stages. */
+ftp_status ftp_run_stage_backward(ftp_model* m, int32_t a, int32_t b, const void* grad_out, void* grad_in,
+                                  void* stream);
+
+/* Device copy of the logits (float[batch * n_classes]) of the last forward that reached L. */
+ftp_status ftp_get_logits(const ftp_model* m, float* dst, int32_t dst_is_device, void* stream);
+
+/* SGD with momentum and weight decay on units [a, b) (Sec. IV-B):
+ *   g <- g + wd*w ;  m <- g on a unit's first update, else mu*m + g ;  w <- w - lr*m
+ * for every trainable parameter, refreshing the bf16 shadow.  When snap_dev / snap_host are
+ * non-NULL the same kernel also stores the updated weights there (device buffer / pinned
+ * host buffer mapped into the device address space), laid out as the trainable spans of
+ * units a..b-1 back to back (the fused half of a replication tick, Sec. III-E). */
+ftp_status ftp_sgd_step(ftp_model* m, int32_t a, int32_t b, float lr, float* snap_dev, float* snap_host,
+                        void* stream);
+
+/* One synchronous training step over the current partition: forward through every stage,
+ * backward through every stage, SGD on every stage; internal boundary buffers.
+ *   x, labels   : the input batch and int32 labels; host (pinned or pageable) when
+ *                 inputs_on_host != 0 -- they are then copied to the device inside the call --
+ *                 else device.
+ *   loss_host   : if non-NULL (host float[1]) the loss is copied back and the call returns
+ *                 after the step has completed; if NULL the call is fully asynchronous. */
+ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, int32_t inputs_on_host, float lr,
+                          float* loss_host, void* stream);
+
+/* ---- profile_layers(): Sec. III-B "model profiling" and Sec. III-D "execution profiling". */
+
+/* Runs `reps` forward+backward passes of the whole model on the sample batch (device
+ * pointers) and returns, per unit, the mean forward and backward device time in seconds and
+ * the size in bytes of its output (host arrays of L entries).  Weight values are left
+ * unchanged (no optimiser step) but BN running statistics are restored afterwards.
+ * Synchronises the stream. */
+ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void* sample_in, const int32_t* labels,
+                              double* fwd_s, double* bwd_s, int64_t* out_bytes, void* stream);
+
+/* Eq. 1-3: capacities[i] = stage_times[i] / sum of layer_times over stage i; [0] = 1.0. */
+ftp_status ftp_estimate_capacity(const double* layer_times, int32_t L, const int32_t* points, int32_t N,
+                                 const double* stage_times, double* capacities);
+
+/* ---- choose_partition(layer_times, capacities): Eq. 4-7.  Pure host function.
+ *   layer_times[L] : T^0_{e,j}; capacities[N] : C_i (a slowdown multiplier).
+ *   out_bytes[L], bandwidth[N-1] : D_j and B_{i,i+1}; both NULL drops the 2*T_c term.
+ *   points_out[N+1], bottleneck_out : the optimal boundaries and A(L-1, N).
+ * Every stage is non-empty (N > L is FTP_EINVAL).  Among optimal partitions the one returned
+ * takes, from the last cut backwards, the smallest cut index reaching the optimum. */
+ftp_status ftp_choose_partition(const double* layer_times, int32_t L, const double* capacities, int32_t N,
+                                const double* out_bytes, const double* bandwidth, int32_t* points_out,
+                                double* bottleneck_out);
+
+/* Algorithm 1 for one worker.  p_cur has n_cur+1 entries (old worker list), p_new n_new+1.
+ * i_cur: the worker's old index (-1 if it held nothing), i_new: its new index, i_fail: the
+ * failed old index or -1.  owner_of_needed[k] (k over the new range p_new[i_new] ..) is the
+ * index, in the NEW worker list, to fetch unit p_new[i_new]+k from, or -1 if it is held
+ * locally; *n_local counts the local ones. */
+ftp_status ftp_redistribution_plan(const int32_t* p_new, int32_t n_new, const int32_t* p_cur, int32_t n_cur,
+                                   int32_t i_fail, int32_t i_cur, int32_t i_new, int32_t* owner_of_needed,
+                                   int32_t* n_local);
+
+/* Install a new partition (Sec. III-D "weight redistribution"): every stage computes its
+ * Algorithm-1 plan, the spans of the units that change owner (weights, momentum, running
+ * statistics, shadow) are copied between stage arenas on the stream, and only after all
+ * copies are enqueued does the owner table switch (the commit).  moved_units (nullable)
+ * receives how many units changed owner. */
+ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int32_t n_stages, int32_t* moved_units,
+                             void* stream);
+ftp_status ftp_get_partition(const ftp_model* m, int32_t* points /* max_stages+1 */, int32_t* n_stages);
+
+/* ---- snapshot_weights(stage, dst): Sec. III-E chain / global replication. ----------------- */
+
+/* Copy stage's replica -- per unit of the stage, in order: trainable weights then BN running
+ * statistics, float -- to dst (device, or host when dst_is_host).  *written = bytes copied.
+ * Asynchronous for device and pinned-host destinations. */
+ftp_status ftp_snapshot_weights(const ftp_model* m, int32_t stage, void* dst, size_t dst_bytes,
+                                int32_t dst_is_host, size_t* written, void* stream);
+
+/* ---- measurement aids ---------------------------------------------------------------------- */
+
+/* While enabled, every kernel launch is bracketed by CUDA events on its stream and recorded.
+ * ftp_trace_read synchronises, copies up to max records (in launch order) and clears the
+ * log; *total is the number that were logged. */
+ftp_status ftp_trace_enable(ftp_model* m, int32_t on);
+ftp_status ftp_trace_read(ftp_model* m, ftp_trace_rec* out, int32_t max, int32_t* total);
+const char* ftp_kernel_name(int32_t kernel);
+/* Number of kernel launches issued by this model since it was built. */
+ftp_status ftp_launch_count(const ftp_model* m, int64_t* launches);
+
+const char* ftp_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FTPIPE_H */

@@ -1,0 +1,848 @@
+// Streaming (HBM-bound) kernels: batch-norm statistics / apply / backward, activation and bias
+// backward, depthwise 3x3 convolution, pooling, softmax cross-entropy and the fused SGD update.
+// Every tensor is read and written with 16-byte accesses along the channel axis; every
+// reduction runs in a fixed order (per-thread run, shared-memory column sum, then a second pass
+// over the per-block partials) so results do not depend on scheduling.
+#include <cfloat>
+#include "kernels.h"
+
+namespace ftp {
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+namespace {
+
+// ---- 16-byte vector access with conversion to float ------------------------------------------
+template <typename T> struct VecOf;
+template <> struct VecOf<float> { static constexpr int N = 4; };
+template <> struct VecOf<__nv_bfloat16> { static constexpr int N = 8; };
+
+template <int V> __device__ __forceinline__ void ldv(const float* p, float (&o)[V]) {
+    if constexpr (V == 4) { const float4 v = __ldg(reinterpret_cast<const float4*>(p)); o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w; }
+    else { o[0] = __ldg(p); }
+}
+template <int V> __device__ __forceinline__ void ldv(const __nv_bfloat16* p, float (&o)[V]) {
+    if constexpr (V == 8) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+        const unsigned u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(u[i] << 16); o[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
+    } else { o[0] = __bfloat162float(*p); }
+}
+template <int V> __device__ __forceinline__ void stv(float* p, const float (&v)[V]) {
+    if constexpr (V == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    else p[0] = v[0];
+}
+template <int V> __device__ __forceinline__ void stv(__nv_bfloat16* p, const float (&v)[V]) {
+    if constexpr (V == 8) {
+        unsigned u[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            u[i] = *reinterpret_cast<const unsigned*>(&h);
+        }
+        *reinterpret_cast<uint4*>(p) = make_uint4(u[0], u[1], u[2], u[3]);
+    } else { p[0] = __float2bfloat16_rn(v[0]); }
+}
+// V consecutive floats of a per-channel table (V is 1, 4 or 8; the address is 16-byte aligned for V >= 4)
+template <int V> __device__ __forceinline__ void ldtab(const float* p, float (&o)[V]) {
+    if constexpr (V == 1) o[0] = __ldg(p);
+    else {
+#pragma unroll
+        for (int i = 0; i < V / 4; ++i) { const float4 v = __ldg(reinterpret_cast<const float4*>(p) + i); o[4 * i] = v.x; o[4 * i + 1] = v.y; o[4 * i + 2] = v.z; o[4 * i + 3] = v.w; }
+    }
+}
+
+__device__ __forceinline__ float act_f(float v, int act) {
+    if (act == 1) return fmaxf(v, 0.f);
+    if (act == 2) return fminf(fmaxf(v, 0.f), 6.f);
+    return v;
+}
+__device__ __forceinline__ bool act_pass(float z, int act) {      // derivative is 1 strictly inside the linear range
+    if (act == 1) return z > 0.f;
+    if (act == 2) return z > 0.f && z < 6.f;
+    return true;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline unsigned flat_blocks(long long work, int threads) {
+    long long b = (work + threads - 1) / threads;
+    const long long cap = (long long)sm_count() * 16;
+    if (b > cap) b = cap;
+    if (b < 1) b = 1;
+    return (unsigned)b;
+}
+
+// ---- folded column reductions --------------------------------------------------------------
+// grid (column tiles of 32*V, row chunks); block (32, 8).  NS sums per column.
+template <typename T, int V, int NS, typename F>
+__device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chunk, double* partial, F body) {
+    __shared__ float sh[NS][8][32 * V];
+    const int col = (blockIdx.x * 32 + threadIdx.x) * V;
+    const int r0 = blockIdx.y * rows_per_chunk, r1 = min(rows, r0 + rows_per_chunk);
+    float s[NS][V];
+#pragma unroll
+    for (int a = 0; a < NS; ++a)
+#pragma unroll
+        for (int e = 0; e < V; ++e) s[a][e] = 0.f;
+    if (col < cols)
+        for (int r = r0 + threadIdx.y; r < r1; r += 8) body((long long)r * cols + col, col, s);
+#pragma unroll
+    for (int a = 0; a < NS; ++a)
+#pragma unroll
+        for (int e = 0; e < V; ++e) sh[a][threadIdx.y][threadIdx.x * V + e] = s[a][e];
+    __syncthreads();
+    // 256 threads sum the 8 rows of NS * 32 * V columns in a fixed order
+    for (int q = threadIdx.y * 32 + threadIdx.x; q < NS * 32 * V; q += 256) {
+        const int a = q / (32 * V), c = q % (32 * V);
+        const int gc = blockIdx.x * 32 * V + c;
+        if (gc < cols) {
+            double t = 0.0;
+#pragma unroll
+            for (int y = 0; y < 8; ++y) t += (double)sh[a][y][c];
+            partial[((long long)blockIdx.y * NS + a) * cols + gc] = t;
+        }
+    }
+}
+
+// Sum over chunks and folded copies for channel c, by one warp, fixed order.  Result valid in lane 0.
+__device__ __forceinline__ double warp_fold_sum(const double* partial, int which, int ns, int chunks, int f, int C, int cols, int c) {
+    const int lane = threadIdx.x & 31;
+    double t = 0.0;
+    const int total = chunks * f;
+    for (int e = lane; e < total; e += 32) {
+        const int ch = e / f, k = e - ch * f;
+        t += partial[((long long)ch * ns + which) * cols + k * C + c];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
+    return t;
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, int rows, int cols, int rpc, double* __restrict__ partial) {
+    fold_reduce<T, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
+        float v[V];
+        ldv<V>(y + off, v);
+#pragma unroll
+        for (int e = 0; e < V; ++e) { s[0][e] += v[e]; s[1][e] = fmaf(v[e], v[e], s[1][e]); }
+    });
+}
+
+__global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
+                                   const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
+                                   float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* rstd) {
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (c >= C) return;
+    const double s1 = warp_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
+    const double s2 = warp_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
+    if ((threadIdx.x & 31) == 0) {
+        const double mu = s1 / M;
+        double var = s2 / M - mu * mu;
+        if (var < 0.0) var = 0.0;
+        const double rs = 1.0 / sqrt(var + (double)eps);
+        const float sc = (float)((double)gamma[c] * rs);
+        scale[c] = sc;
+        shift[c] = (float)((double)beta[c] - mu * (double)gamma[c] * rs);
+        mean[c] = (float)mu;
+        rstd[c] = (float)rs;
+        const double unb = M > 1.0 ? var * M / (M - 1.0) : var;
+        run_mean[c] = (float)((1.0 - (double)mom) * (double)run_mean[c] + (double)mom * mu);
+        run_var[c] = (float)((1.0 - (double)mom) * (double)run_var[c] + (double)mom * unb);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ y, const T* __restrict__ res, T* __restrict__ z,
+                                                       long long nvec, int C, const float* __restrict__ scale,
+                                                       const float* __restrict__ shift, int act) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)((i * V) % C);
+        float v[V], sc[V], sh[V];
+        ldv<V>(y + i * V, v);
+        ldtab<V>(scale + c, sc);
+        ldtab<V>(shift + c, sh);
+#pragma unroll
+        for (int e = 0; e < V; ++e) v[e] = act_f(fmaf(v[e], sc[e], sh[e]), act);
+        if (res) {
+            float r[V];
+            ldv<V>(res + i * V, r);
+#pragma unroll
+            for (int e = 0; e < V; ++e) v[e] += r[e];
+        }
+        stv<V>(z + i * V, v);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict__ dz, const T* __restrict__ y, int rows, int cols, int rpc, int C,
+                                                            const float* __restrict__ scale, const float* __restrict__ shift,
+                                                            const float* __restrict__ mean, const float* __restrict__ rstd, int act,
+                                                            double* __restrict__ partial) {
+    const int col = (blockIdx.x * 32 + threadIdx.x) * V;
+    float sc[V], sh[V], mu[V], rs[V];
+    if (col < cols) { const int c = col % C; ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(rstd + c, rs); }
+    fold_reduce<T, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
+        float d[V], v[V];
+        ldv<V>(dz + off, d);
+        ldv<V>(y + off, v);
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            const float g = act_pass(fmaf(v[e], sc[e], sh[e]), act) ? d[e] : 0.f;
+            s[0][e] += g;
+            s[1][e] = fmaf(g, (v[e] - mu[e]) * rs[e], s[1][e]);
+        }
+    });
+}
+
+__global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
+                                       const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
+                                       float* dbeta, float* coef) {
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (c >= C) return;
+    const double s1 = warp_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
+    const double s2 = warp_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
+    if ((threadIdx.x & 31) == 0) {
+        dbeta[c] = (float)s1;
+        dgamma[c] = (float)s2;
+        coef[c] = gamma[c] * rstd[c];
+        coef[C + c] = (float)(s1 / M);
+        coef[2 * C + c] = (float)(s2 / M);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dz, const T* __restrict__ y, const T* __restrict__ addend,
+                                                           T* __restrict__ dy, long long nvec, int C, const float* __restrict__ scale,
+                                                           const float* __restrict__ shift, const float* __restrict__ mean,
+                                                           const float* __restrict__ rstd, const float* __restrict__ coef, int act) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)((i * V) % C);
+        float d[V], v[V], sc[V], sh[V], mu[V], rs[V], ca[V], cb[V], cc[V], o[V];
+        ldv<V>(dz + i * V, d);
+        ldv<V>(y + i * V, v);
+        ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(rstd + c, rs);
+        ldtab<V>(coef + c, ca); ldtab<V>(coef + C + c, cb); ldtab<V>(coef + 2 * C + c, cc);
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            const float g = act_pass(fmaf(v[e], sc[e], sh[e]), act) ? d[e] : 0.f;
+            o[e] = ca[e] * (g - cb[e] - (v[e] - mu[e]) * rs[e] * cc[e]);
+        }
+        if (addend) {
+            float a[V];
+            ldv<V>(addend + i * V, a);
+#pragma unroll
+            for (int e = 0; e < V; ++e) o[e] += a[e];
+        }
+        stv<V>(dy + i * V, o);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) act_bias_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ out, T* __restrict__ dpre,
+                                                           int rows, int cols, int rpc, int act, double* __restrict__ partial) {
+    fold_reduce<T, V, 1>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[1][V]) {
+        float d[V];
+        ldv<V>(dout + off, d);
+        if (act != 0) {
+            float o[V];
+            ldv<V>(out + off, o);
+#pragma unroll
+            for (int e = 0; e < V; ++e) d[e] = act_pass(o[e], act) ? d[e] : 0.f;
+        }
+        if (dpre) stv<V>(dpre + off, d);
+#pragma unroll
+        for (int e = 0; e < V; ++e) s[0][e] += d[e];
+    });
+}
+
+__global__ void colsum_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, float* out) {
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (c >= C) return;
+    const double s = warp_fold_sum(partial, 0, 1, chunks, f, C, cols, c);
+    if ((threadIdx.x & 31) == 0) out[c] = (float)s;
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) act_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, long long nvec, int act) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        float v[V];
+        ldv<V>(x + i * V, v);
+#pragma unroll
+        for (int e = 0; e < V; ++e) v[e] = act_f(v[e], act);
+        stv<V>(y + i * V, v);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) act_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ x, const T* __restrict__ addend,
+                                                      T* __restrict__ dx, long long nvec, int act) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        float d[V], v[V];
+        ldv<V>(dout + i * V, d);
+        ldv<V>(x + i * V, v);
+#pragma unroll
+        for (int e = 0; e < V; ++e) d[e] = act_pass(v[e], act) ? d[e] : 0.f;
+        if (addend) {
+            float a[V];
+            ldv<V>(addend + i * V, a);
+#pragma unroll
+            for (int e = 0; e < V; ++e) d[e] += a[e];
+        }
+        stv<V>(dx + i * V, d);
+    }
+}
+
+// ---- depthwise 3x3 ------------------------------------------------------------------------------
+template <typename T, int V>
+__global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, ConvGeom g, long long total) {
+    const int CV = g.Cin / V;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % CV) * V;
+        long long pix = i / CV;
+        const int wo = (int)(pix % g.Wo); pix /= g.Wo;
+        const int ho = (int)(pix % g.Ho);
+        const int n = (int)(pix / g.Ho);
+        float acc[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const int hi = ho * g.stride - g.ph + r;
+            if (hi < 0 || hi >= g.H) continue;
+#pragma unroll
+            for (int s = 0; s < 3; ++s) {
+                const int wi = wo * g.stride - g.pw + s;
+                if (wi < 0 || wi >= g.W) continue;
+                float v[V], k[V];
+                ldv<V>(x + ((long long)(n * g.H + hi) * g.W + wi) * g.Cin + c, v);
+                ldtab<V>(w + (r * 3 + s) * g.Cin + c, k);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = fmaf(v[e], k[e], acc[e]);
+            }
+        }
+        stv<V>(y + i * V, acc);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy, const float* __restrict__ w, const T* __restrict__ addend,
+                                                       T* __restrict__ dx, ConvGeom g, long long total) {
+    const int CV = g.Cin / V;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % CV) * V;
+        long long pix = i / CV;
+        const int wi = (int)(pix % g.W); pix /= g.W;
+        const int hi = (int)(pix % g.H);
+        const int n = (int)(pix / g.H);
+        float acc[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const int th = hi + g.ph - r;
+            if (th < 0) continue;
+            const int ho = th / g.stride;
+            if (ho * g.stride != th || ho >= g.Ho) continue;
+#pragma unroll
+            for (int s = 0; s < 3; ++s) {
+                const int tw = wi + g.pw - s;
+                if (tw < 0) continue;
+                const int wo = tw / g.stride;
+                if (wo * g.stride != tw || wo >= g.Wo) continue;
+                float v[V], k[V];
+                ldv<V>(dy + ((long long)(n * g.Ho + ho) * g.Wo + wo) * g.Cin + c, v);
+                ldtab<V>(w + (r * 3 + s) * g.Cin + c, k);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = fmaf(v[e], k[e], acc[e]);
+            }
+        }
+        if (addend) {
+            float a[V];
+            ldv<V>(addend + i * V, a);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[e] += a[e];
+        }
+        stv<V>(dx + i * V, acc);
+    }
+}
+
+// grid (column tiles, pixel chunks), 256 threads: lane group = channel vector, the rest of the block
+// spreads over pixels.  Writes partial[chunk][9][C].
+template <typename T, int V>
+__global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, ConvGeom g,
+                                                       long long npix, int ppc, int cvt) {
+    __shared__ float sh[256][V];
+    const int CV = g.Cin / V;
+    const int cv0 = blockIdx.x * cvt;
+    const int lanes = min(cvt, CV - cv0);            // channel vectors handled by this block
+    const int G = 256 / lanes;                       // pixel groups
+    const int cl = threadIdx.x % lanes, pg = threadIdx.x / lanes;
+    const bool active = pg < G;
+    const int c = (cv0 + cl) * V;
+    const long long p0 = (long long)blockIdx.y * ppc, p1 = min(npix, p0 + ppc);
+    float acc[9][V];
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
+    if (active) {
+        for (long long pix = p0 + pg; pix < p1; pix += G) {
+            const int wo = (int)(pix % g.Wo);
+            const long long q = pix / g.Wo;
+            const int ho = (int)(q % g.Ho), n = (int)(q / g.Ho);
+            float d[V];
+            ldv<V>(dy + pix * g.Cin + c, d);
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                const int hi = ho * g.stride - g.ph + r;
+                if (hi < 0 || hi >= g.H) continue;
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    const int wi = wo * g.stride - g.pw + s;
+                    if (wi < 0 || wi >= g.W) continue;
+                    float v[V];
+                    ldv<V>(x + ((long long)(n * g.H + hi) * g.W + wi) * g.Cin + c, v);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[r * 3 + s][e] = fmaf(v[e], d[e], acc[r * 3 + s][e]);
+                }
+            }
+        }
+    }
+    float* out = partial + (long long)blockIdx.y * 9 * g.Cin;
+#pragma unroll
+    for (int t = 0; t < 9; ++t) {
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < V; ++e) sh[threadIdx.x][e] = acc[t][e];
+        __syncthreads();
+        if (threadIdx.x < lanes) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+                float s = 0.f;
+                for (int q = 0; q < G; ++q) s += sh[q * lanes + threadIdx.x][e];
+                out[t * g.Cin + c + e] = s;
+            }
+        }
+    }
+}
+
+__global__ void split_sum_kernel(const float* __restrict__ partial, int S, long long count, float* __restrict__ out) {
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count) return;
+    float s = 0.f;
+    for (int z = 0; z < S; ++z) s += partial[(long long)z * count + e];
+    out[e] = s;
+}
+
+// ---- pooling --------------------------------------------------------------------------------------
+template <typename T, int V>
+__global__ void __launch_bounds__(256) maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int H, int W, int C, long long total) {
+    const int CV = C / V, Ho = H / 2, Wo = W / 2;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % CV) * V;
+        long long pix = i / CV;
+        const int wo = (int)(pix % Wo); pix /= Wo;
+        const int ho = (int)(pix % Ho);
+        const int n = (int)(pix / Ho);
+        float m[V];
+        ldv<V>(x + ((long long)(n * H + 2 * ho) * W + 2 * wo) * C + c, m);
+#pragma unroll
+        for (int q = 1; q < 4; ++q) {
+            float v[V];
+            ldv<V>(x + ((long long)(n * H + 2 * ho + (q >> 1)) * W + 2 * wo + (q & 1)) * C + c, v);
+#pragma unroll
+            for (int e = 0; e < V; ++e) m[e] = v[e] > m[e] ? v[e] : m[e];
+        }
+        stv<V>(y + i * V, m);
+    }
+}
+
+// one thread per output pixel / channel vector writes its four inputs: the gradient goes to the first
+// maximum in row-major window order, zero elsewhere (rows/columns beyond 2*floor(H/2) get zero too)
+template <typename T, int V>
+__global__ void __launch_bounds__(256) maxpool_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ x, T* __restrict__ dx, int H, int W, int C, long long total) {
+    const int CV = C / V, Ho = H / 2, Wo = W / 2;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % CV) * V;
+        long long pix = i / CV;
+        const int wo = (int)(pix % Wo); pix /= Wo;
+        const int ho = (int)(pix % Ho);
+        const int n = (int)(pix / Ho);
+        float v[4][V], d[V];
+        int arg[V];
+        ldv<V>(dy + i * V, d);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) ldv<V>(x + ((long long)(n * H + 2 * ho + (q >> 1)) * W + 2 * wo + (q & 1)) * C + c, v[q]);
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            arg[e] = 0;
+            float m = v[0][e];
+#pragma unroll
+            for (int q = 1; q < 4; ++q) if (v[q][e] > m) { m = v[q][e]; arg[e] = q; }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float o[V];
+#pragma unroll
+            for (int e = 0; e < V; ++e) o[e] = arg[e] == q ? d[e] : 0.f;
+            stv<V>(dx + ((long long)(n * H + 2 * ho + (q >> 1)) * W + 2 * wo + (q & 1)) * C + c, o);
+        }
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) gap_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int HW, int C, long long total) {
+    const int CV = C / V;
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int c = (int)(i % CV) * V;
+    const long long n = i / CV;
+    float s[V];
+#pragma unroll
+    for (int e = 0; e < V; ++e) s[e] = 0.f;
+    for (int p = 0; p < HW; ++p) {
+        float v[V];
+        ldv<V>(x + (n * HW + p) * C + c, v);
+#pragma unroll
+        for (int e = 0; e < V; ++e) s[e] += v[e];
+    }
+    const float inv = 1.f / (float)HW;
+#pragma unroll
+    for (int e = 0; e < V; ++e) s[e] *= inv;
+    stv<V>(y + i * V, s);
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256) gap_bwd_kernel(const T* __restrict__ dy, T* __restrict__ dx, int HW, int C, long long total) {
+    const int CV = C / V;
+    const float inv = 1.f / (float)HW;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int cv = (int)(i % CV);
+        const long long n = i / CV / HW;
+        float v[V];
+        ldv<V>(dy + (n * CV + cv) * V, v);
+#pragma unroll
+        for (int e = 0; e < V; ++e) v[e] *= inv;
+        stv<V>(dx + i * V, v);
+    }
+}
+
+// ---- softmax cross-entropy: one block per sample ---------------------------------------------------
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { const float u = __shfl_xor_sync(0xffffffffu, v, o); v = is_max ? fmaxf(v, u) : v + u; }
+    __syncthreads();
+    if (lane == 0) sh[wid] = v;
+    __syncthreads();
+    float r = sh[0];
+    for (int i = 1; i < nw; ++i) r = is_max ? fmaxf(r, sh[i]) : r + sh[i];
+    return r;
+}
+
+__global__ void __launch_bounds__(128) softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int N, int K,
+                                                         float* __restrict__ per_sample, float* __restrict__ dlogits) {
+    __shared__ float sh[4];
+    const int n = blockIdx.x;
+    const float* z = logits + (long long)n * K;
+    float mx = -FLT_MAX;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) mx = fmaxf(mx, z[k]);
+    mx = block_reduce(mx, true, sh);
+    float se = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) se += expf(z[k] - mx);
+    se = block_reduce(se, false, sh);
+    int lab = labels[n];
+    lab = lab < 0 ? 0 : (lab >= K ? K - 1 : lab);
+    const float lse = logf(se);
+    const float invn = 1.f / (float)N;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        const float p = expf(z[k] - mx - lse);
+        dlogits[(long long)n * K + k] = (p - (k == lab ? 1.f : 0.f)) * invn;
+    }
+    if (threadIdx.x == 0) per_sample[n] = -(z[lab] - mx - lse);
+}
+
+__global__ void loss_mean_kernel(const float* __restrict__ per_sample, int N, float* loss) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double s = 0.0;
+        for (int i = 0; i < N; ++i) s += (double)per_sample[i];
+        *loss = (float)(s / (double)N);
+    }
+}
+
+// ---- SGD ------------------------------------------------------------------------------------------------
+template <int V>
+__global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, long long nvec, float lr,
+                                                  float mu, float wd, int first, __nv_bfloat16* __restrict__ shadow,
+                                                  float* __restrict__ snap_dev, float* __restrict__ snap_host) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        float wv[V], gv[V], mv[V];
+        ldv<V>(w + i * V, wv);
+        ldv<V>(g + i * V, gv);
+#pragma unroll
+        for (int e = 0; e < V; ++e) gv[e] = fmaf(wd, wv[e], gv[e]);
+        if (m) {
+            if (!first) {
+                ldv<V>(m + i * V, mv);
+#pragma unroll
+                for (int e = 0; e < V; ++e) gv[e] = fmaf(mu, mv[e], gv[e]);
+            }
+            stv<V>(m + i * V, gv);
+        }
+#pragma unroll
+        for (int e = 0; e < V; ++e) wv[e] = fmaf(-lr, gv[e], wv[e]);
+        stv<V>(w + i * V, wv);
+        if (snap_dev) stv<V>(snap_dev + i * V, wv);
+        if (snap_host) stv<V>(snap_host + i * V, wv);
+        if (shadow) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) shadow[i * V + e] = __float2bfloat16_rn(wv[e]);
+        }
+    }
+}
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ s, __nv_bfloat16* __restrict__ d, long long n) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        d[i] = __float2bfloat16_rn(s[i]);
+}
+
+template <typename T> inline bool can_vec(int C, const void* a, const void* b = nullptr, const void* c = nullptr, const void* d = nullptr) {
+    return C % VecOf<T>::N == 0 && aligned16(a) && aligned16(b) && aligned16(c) && aligned16(d);
+}
+
+}  // namespace
+
+// ---- host side ---------------------------------------------------------------------------------------------
+FoldPlan make_fold(long long M, int C, int elem_bytes) {
+    FoldPlan fp;
+    const int V = 16 / elem_bytes;
+    fp.vec = (C % V == 0) ? V : 1;
+    fp.f = 1;
+    if (fp.vec > 1) {
+        const int tile = 32 * V;
+        for (int f = 1; f <= 64; f *= 2)
+            if (((long long)C * f) % tile == 0 && M % f == 0) { fp.f = f; break; }
+    }
+    fp.cols = C * fp.f;
+    fp.rows = (int)(M / fp.f);
+    const int coltiles = (fp.cols + 32 * fp.vec - 1) / (32 * fp.vec);
+    long long chunks = (4LL * sm_count() + coltiles - 1) / coltiles;
+    const long long maxc = (fp.rows + 15) / 16;
+    if (chunks > maxc) chunks = maxc;
+    if (chunks < 1) chunks = 1;
+    const int rpc = (int)((fp.rows + chunks - 1) / chunks);
+    fp.chunks = (fp.rows + rpc - 1) / rpc;
+    return fp;
+}
+
+size_t fold_partial_doubles(const FoldPlan& fp) { return (size_t)fp.chunks * 2 * fp.cols; }
+
+static inline int fold_rpc(const FoldPlan& fp) { return (fp.rows + fp.chunks - 1) / fp.chunks; }
+static inline dim3 fold_grid(const FoldPlan& fp) { return dim3((fp.cols + 32 * fp.vec - 1) / (32 * fp.vec), fp.chunks); }
+
+template <typename T>
+void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (fp.vec == V && aligned16(y)) bn_stats_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(y, fp.rows, fp.cols, fold_rpc(fp), partial);
+    else bn_stats_kernel<T, 1><<<fold_grid(fp), dim3(32, 8), 0, st>>>(y, fp.rows, fp.cols, fold_rpc(fp), partial);
+}
+
+void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
+                 float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
+                 float* rstd, cudaStream_t st) {
+    bn_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
+                                                             run_mean, run_var, scale, shift, mean, rstd);
+}
+
+template <typename T>
+void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift, int act,
+              cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const long long n = M * C;
+    if (can_vec<T>(C, y, residual, z) && aligned16(scale) && aligned16(shift))
+        bn_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(y, residual, z, n / V, C, scale, shift, act);
+    else
+        bn_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(y, residual, z, n, C, scale, shift, act);
+}
+
+template <typename T>
+void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
+                   const float* mean, const float* rstd, int act, double* partial, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(rstd))
+        bn_bwd_reduce_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, rstd, act, partial);
+    else {
+        FoldPlan s = fp;                       // scalar fallback keeps the same partial layout
+        bn_bwd_reduce_kernel<T, 1><<<dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st>>>(dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, rstd, act, partial);
+    }
+}
+
+void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
+                     float* dgamma, float* dbeta, float* coef, cudaStream_t st) {
+    bn_bwd_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef);
+}
+
+template <typename T>
+void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale, const float* shift,
+                  const float* mean, const float* rstd, const float* coef, int act, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const long long n = M * C;
+    if (can_vec<T>(C, dz, y, addend, dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(rstd) && aligned16(coef))
+        bn_bwd_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(dz, y, addend, dy, n / V, C, scale, shift, mean, rstd, coef, act);
+    else
+        bn_bwd_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(dz, y, addend, dy, n, C, scale, shift, mean, rstd, coef, act);
+}
+
+template <typename T>
+void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int act, const FoldPlan& fp, double* partial,
+                  float* dbias, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (fp.vec == V && aligned16(dout) && aligned16(out) && aligned16(dpre))
+        act_bias_bwd_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
+    else
+        act_bias_bwd_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
+    if (dbias) colsum_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias);
+}
+
+template <typename T>
+void act_fwd(const T* x, T* y, long long n, int act, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (n % V == 0 && aligned16(x) && aligned16(y)) act_fwd_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(x, y, n / V, act);
+    else act_fwd_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(x, y, n, act);
+}
+
+template <typename T>
+void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int act, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (n % V == 0 && aligned16(dout) && aligned16(x) && aligned16(addend) && aligned16(dx))
+        act_bwd_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(dout, x, addend, dx, n / V, act);
+    else act_bwd_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(dout, x, addend, dx, n, act);
+}
+
+template <typename T>
+void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const long long pix = (long long)g.N * g.Ho * g.Wo;
+    if (can_vec<T>(g.Cin, x, y) && aligned16(w)) dw_fwd_kernel<T, V><<<flat_blocks(pix * (g.Cin / V), 256), 256, 0, st>>>(x, w, y, g, pix * (g.Cin / V));
+    else dw_fwd_kernel<T, 1><<<flat_blocks(pix * g.Cin, 256), 256, 0, st>>>(x, w, y, g, pix * g.Cin);
+}
+
+template <typename T>
+void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const ConvGeom& g, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const long long pix = (long long)g.N * g.H * g.W;
+    if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) dw_dgrad_kernel<T, V><<<flat_blocks(pix * (g.Cin / V), 256), 256, 0, st>>>(dy, w, addend, dx, g, pix * (g.Cin / V));
+    else dw_dgrad_kernel<T, 1><<<flat_blocks(pix * g.Cin, 256), 256, 0, st>>>(dy, w, addend, dx, g, pix * g.Cin);
+}
+
+struct DwWgPlan { int chunks, ppc; };
+static DwWgPlan plan_dw_wgrad(const ConvGeom& g) {
+    const long long npix = (long long)g.N * g.Ho * g.Wo;
+    long long chunks = 4LL * sm_count();
+    const long long maxc = (npix + 63) / 64;
+    if (chunks > maxc) chunks = maxc;
+    if (chunks < 1) chunks = 1;
+    DwWgPlan p;
+    p.ppc = (int)((npix + chunks - 1) / chunks);
+    p.chunks = (int)((npix + p.ppc - 1) / p.ppc);
+    return p;
+}
+
+size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) { return (size_t)plan_dw_wgrad(g).chunks * 9 * g.Cin; }
+
+template <typename T>
+void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const DwWgPlan p = plan_dw_wgrad(g);
+    const long long npix = (long long)g.N * g.Ho * g.Wo;
+    if (can_vec<T>(g.Cin, x, dy)) {
+        const int CV = g.Cin / V, cvt = CV < 256 ? CV : 256;
+        dw_wgrad_kernel<T, V><<<dim3((CV + cvt - 1) / cvt, p.chunks), 256, 0, st>>>(x, dy, scratch, g, npix, p.ppc, cvt);
+    } else {
+        const int CV = g.Cin, cvt = CV < 256 ? CV : 256;
+        dw_wgrad_kernel<T, 1><<<dim3((CV + cvt - 1) / cvt, p.chunks), 256, 0, st>>>(x, dy, scratch, g, npix, p.ppc, cvt);
+    }
+    const long long count = 9LL * g.Cin;
+    split_sum_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, p.chunks, count, dw);
+}
+
+template <typename T>
+void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const long long pix = (long long)N * (H / 2) * (W / 2);
+    if (can_vec<T>(C, x, y)) maxpool_fwd_kernel<T, V><<<flat_blocks(pix * (C / V), 256), 256, 0, st>>>(x, y, H, W, C, pix * (C / V));
+    else maxpool_fwd_kernel<T, 1><<<flat_blocks(pix * C, 256), 256, 0, st>>>(x, y, H, W, C, pix * C);
+}
+
+template <typename T>
+void maxpool_bwd(const T* dy, const T* x, T* dx, int N, int H, int W, int C, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    const long long pix = (long long)N * (H / 2) * (W / 2);
+    if ((H & 1) || (W & 1)) cudaMemsetAsync(dx, 0, (size_t)N * H * W * C * sizeof(T), st);   // odd edge gets no gradient
+    if (can_vec<T>(C, dy, x, dx)) maxpool_bwd_kernel<T, V><<<flat_blocks(pix * (C / V), 256), 256, 0, st>>>(dy, x, dx, H, W, C, pix * (C / V));
+    else maxpool_bwd_kernel<T, 1><<<flat_blocks(pix * C, 256), 256, 0, st>>>(dy, x, dx, H, W, C, pix * C);
+}
+
+template <typename T>
+void gap_fwd(const T* x, T* y, int N, int HW, int C, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (can_vec<T>(C, x, y)) { const long long t = (long long)N * (C / V); gap_fwd_kernel<T, V><<<(unsigned)((t + 255) / 256), 256, 0, st>>>(x, y, HW, C, t); }
+    else { const long long t = (long long)N * C; gap_fwd_kernel<T, 1><<<(unsigned)((t + 255) / 256), 256, 0, st>>>(x, y, HW, C, t); }
+}
+
+template <typename T>
+void gap_bwd(const T* dy, T* dx, int N, int HW, int C, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (can_vec<T>(C, dy, dx)) { const long long t = (long long)N * HW * (C / V); gap_bwd_kernel<T, V><<<flat_blocks(t, 256), 256, 0, st>>>(dy, dx, HW, C, t); }
+    else { const long long t = (long long)N * HW * C; gap_bwd_kernel<T, 1><<<flat_blocks(t, 256), 256, 0, st>>>(dy, dx, HW, C, t); }
+}
+
+void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, float* per_sample, float* dlogits,
+                float* loss, cudaStream_t st) {
+    softmax_ce_kernel<<<N, 128, 0, st>>>(logits, labels, N, classes, per_sample, dlogits);
+    loss_mean_kernel<<<1, 32, 0, st>>>(per_sample, N, loss);
+}
+
+void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
+                __nv_bfloat16* shadow, float* snap_dev, float* snap_host, cudaStream_t st) {
+    const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(snap_dev) && aligned16(snap_host);
+    if (v) sgd_kernel<4><<<flat_blocks(n / 4, 256), 256, 0, st>>>(w, g, m, n / 4, lr, mu, wd, first, shadow, snap_dev, snap_host);
+    else sgd_kernel<1><<<flat_blocks(n, 256), 256, 0, st>>>(w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
+}
+
+void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st) {
+    f32_to_bf16_kernel<<<flat_blocks(n, 256), 256, 0, st>>>(src, dst, n);
+}
+
+#define FTP_INSTANTIATE(T)                                                                                              \
+    template void bn_stats<T>(const T*, long long, int, const FoldPlan&, double*, cudaStream_t);                          \
+    template void bn_apply<T>(const T*, const T*, T*, long long, int, const float*, const float*, int, cudaStream_t);       \
+    template void bn_bwd_reduce<T>(const T*, const T*, long long, int, const FoldPlan&, const float*, const float*,         \
+                                   const float*, const float*, int, double*, cudaStream_t);                                \
+    template void bn_bwd_apply<T>(const T*, const T*, const T*, T*, long long, int, const float*, const float*,             \
+                                  const float*, const float*, const float*, int, cudaStream_t);                            \
+    template void act_bias_bwd<T>(const T*, const T*, T*, long long, int, int, const FoldPlan&, double*, float*,            \
+                                  cudaStream_t);                                                                           \
+    template void act_fwd<T>(const T*, T*, long long, int, cudaStream_t);                                                   \
+    template void act_bwd<T>(const T*, const T*, const T*, T*, long long, int, cudaStream_t);                               \
+    template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t);                                 \
+    template void dwconv_dgrad<T>(const T*, const float*, const T*, T*, const ConvGeom&, cudaStream_t);                     \
+    template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, cudaStream_t);                       \
+    template void maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);                                           \
+    template void maxpool_bwd<T>(const T*, const T*, T*, int, int, int, int, cudaStream_t);                                 \
+    template void gap_fwd<T>(const T*, T*, int, int, int, cudaStream_t);                                                    \
+    template void gap_bwd<T>(const T*, T*, int, int, int, cudaStream_t);
+
+FTP_INSTANTIATE(float)
+FTP_INSTANTIATE(__nv_bfloat16)
+
+}  // namespace ftp

@@ -1,0 +1,103 @@
+// Launchers of the device kernels.  Plain pointers and sizes; every launcher enqueues on the
+// given stream and returns nothing: the caller checks cudaGetLastError().
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace ftp {
+
+// Geometry of a (dense or depthwise) convolution.  Activations are (N, H, W, C).
+struct ConvGeom {
+    int N, H, W, Cin;     // input
+    int Ho, Wo, Cout;     // output
+    int kh, kw, stride, ph, pw;
+};
+
+// ---- fp32 SIMT contraction (gemm_f32.cu) ---------------------------------------------------
+// y = act(conv(x, w) + bias) (+ addend): implicit GEMM, M = N*Ho*Wo, K = kh*kw*Cin.
+void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, const ConvGeom& g, int act,
+                  cudaStream_t st);
+// dx = conv^T(dy, w) (+ addend): implicit GEMM over the input pixels, K = kh*kw*Cout.
+void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, const ConvGeom& g,
+                    cudaStream_t st);
+// dw[kh][kw][cin][cout] = sum over output pixels; split over M with a fixed-order second pass.
+// scratch must hold conv_wgrad_scratch_floats(g) floats.
+size_t conv_wgrad_scratch_floats(const ConvGeom& g);
+void conv_wgrad_f32(const float* x, const float* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st);
+
+// ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
+// Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole
+// 128-byte lines; `fold` picks f.  Partials are doubles: [chunks][2][C*f].
+struct FoldPlan {
+    int f;          // rows folded into one
+    int cols;       // C * f
+    int rows;       // M / f
+    int chunks;     // row chunks (grid.y)
+    int vec;        // elements per thread per row (16 bytes worth, or 1)
+};
+FoldPlan make_fold(long long M, int C, int elem_bytes);
+size_t fold_partial_doubles(const FoldPlan& fp);     // doubles needed for the partial sums
+
+template <typename T>
+void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st);
+// mean/var -> scale, shift, saved mean, rstd; running statistics update (momentum, unbiased variance)
+void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
+                 const float* beta, float eps, float momentum, float* run_mean, float* run_var, float* scale,
+                 float* shift, float* mean, float* rstd, cudaStream_t st);
+template <typename T>
+void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift,
+              int act, cudaStream_t st);
+// pass 1 of BN backward: sums of dz' and dz'*xhat with dz' = dz masked by the activation
+template <typename T>
+void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale,
+                   const float* shift, const float* mean, const float* rstd, int act, double* partial,
+                   cudaStream_t st);
+// -> dgamma, dbeta and the per-channel coefficients (a = gamma*rstd, b = dbeta/M, c = dgamma/M)
+void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
+                     const float* rstd, float* dgamma, float* dbeta, float* coef, cudaStream_t st);
+template <typename T>
+void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale,
+                  const float* shift, const float* mean, const float* rstd, const float* coef, int act,
+                  cudaStream_t st);
+
+// Backward of "act(pre + bias)": dpre = dout masked by the stored output; dbias = column sums.
+// dpre may be NULL when act == 0 (then dpre == dout); dbias may be NULL.
+template <typename T>
+void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int act, const FoldPlan& fp,
+                  double* partial, float* dbias, cudaStream_t st);
+template <typename T>
+void act_fwd(const T* x, T* y, long long n, int act, cudaStream_t st);
+template <typename T>
+void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int act, cudaStream_t st);
+
+template <typename T>
+void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st);
+template <typename T>
+void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const ConvGeom& g, cudaStream_t st);
+size_t dwconv_wgrad_scratch_floats(const ConvGeom& g);
+template <typename T>
+void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st);
+
+template <typename T>
+void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);
+template <typename T>
+void maxpool_bwd(const T* dy, const T* x, T* dx, int N, int H, int W, int C, cudaStream_t st);
+template <typename T>
+void gap_fwd(const T* x, T* y, int N, int HW, int C, cudaStream_t st);
+template <typename T>
+void gap_bwd(const T* dy, T* dx, int N, int HW, int C, cudaStream_t st);
+
+// loss = mean_n -log softmax(logits_n)[label_n]; dlogits = (softmax - onehot) / N.
+// per_sample: float[N] scratch.  Labels outside [0, classes) contribute as if clamped.
+void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, float* per_sample,
+                float* dlogits, float* loss, cudaStream_t st);
+
+// Fused SGD: g += wd*w; m = first ? g : mu*m + g; w -= lr*m; optional bf16 shadow and snapshot stores.
+void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
+                __nv_bfloat16* shadow, float* snap_dev, float* snap_host, cudaStream_t st);
+void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st);
+
+int sm_count();
+
+}  // namespace ftp

@@ -1,0 +1,824 @@
+// Model object and the C ABI around it: validation, memory layout inside the caller's workspace,
+// stage forward / backward / SGD, re-homing of weights after a new partition, snapshots, the
+// per-unit profile and the kernel trace.
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include "model.h"
+
+using namespace ftp;
+
+namespace {
+
+static long long g_launches = 0;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Bump {
+    char* base;
+    size_t off;
+    void* take(size_t bytes) {
+        off = align_up(off, 256);
+        void* p = base ? base + off : reinterpret_cast<void*>(off + 256);   // dry run: fake, never dereferenced
+        off += bytes;
+        return p;
+    }
+};
+
+const char* kKernelNames[K_COUNT] = {
+    "conv_fwd_f32", "conv_dgrad_f32", "conv_wgrad_f32", "bn_stats", "bn_finalize", "bn_apply", "bn_bwd_reduce",
+    "bn_bwd_finalize", "bn_bwd_apply", "act_bias_bwd", "dw_fwd", "dw_dgrad", "dw_wgrad", "maxpool_fwd", "maxpool_bwd",
+    "gap_fwd", "gap_bwd", "softmax_ce", "sgd", "act_fwd", "act_bwd", "copy", "gemm_bf16_fwd", "gemm_bf16_dgrad",
+    "gemm_bf16_wgrad"};
+
+// Brackets one launcher call with events when tracing is on.
+struct Scope {
+    ftp_model* m;
+    cudaStream_t st;
+    TraceSlot* slot;
+    Scope(ftp_model* m_, cudaStream_t st_, int kernel, int unit, int op, int bwd, double bytes, double flops, int nk = 1)
+        : m(m_), st(st_), slot(nullptr) {
+        g_launches += nk;
+        if (!m->trace) return;
+        if (m->tr_used == m->tr.size()) {
+            TraceSlot s{};
+            if (cudaEventCreate(&s.e0) != cudaSuccess || cudaEventCreate(&s.e1) != cudaSuccess) return;
+            m->tr.push_back(s);
+        }
+        slot = &m->tr[m->tr_used++];
+        slot->rec = ftp_trace_rec{kernel, unit, op, bwd, 0.f, bytes, flops};
+        cudaEventRecord(slot->e0, st);
+    }
+    ~Scope() { if (slot) cudaEventRecord(slot->e1, st); }
+};
+
+bool is_contraction(int kind) { return kind == FTP_CONV1D || kind == FTP_CONV2D || kind == FTP_FC; }
+
+// ---- shapes, parameter offsets, validation ------------------------------------------------------
+ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cfg, ftp_model& m) {
+    FTP_REQUIRE(layers && cfg, FTP_EINVAL, "build_model: null argument");
+    FTP_REQUIRE(n >= 1, FTP_EINVAL, "build_model: empty layer list");
+    FTP_REQUIRE(cfg->batch >= 1 && cfg->in_c >= 1 && cfg->in_h >= 1 && cfg->in_w >= 1 && cfg->n_classes >= 1, FTP_EINVAL,
+                "build_model: batch, input shape and class count must be positive");
+    FTP_REQUIRE(cfg->precision == FTP_FP32 || cfg->precision == FTP_BF16, FTP_EINVAL, "build_model: unknown precision %d", cfg->precision);
+    FTP_REQUIRE(cfg->max_stages >= 1 && cfg->max_stages <= 64, FTP_EINVAL, "build_model: max_stages must be in 1..64");
+    FTP_REQUIRE(layers[0].unit == 0, FTP_EINVAL, "build_model: the first op must belong to unit 0");
+    FTP_REQUIRE(layers[n - 1].kind == FTP_SOFTMAX_CE, FTP_EINVAL, "build_model: the last op must be SOFTMAX_CE");
+    m.cfg = *cfg;
+    m.esize = cfg->precision == FTP_BF16 ? 2 : 4;
+    m.ops.assign(n, Op{});
+    int H = cfg->in_h, W = cfg->in_w, C = cfg->in_c;
+    const int N = cfg->batch;
+    long long poff = 0, soff = 0;
+    m.unit_first.clear(); m.unit_last.clear();
+    for (int i = 0; i < n; ++i) {
+        const ftp_layer_desc& d = layers[i];
+        Op& o = m.ops[i];
+        o.d = d;
+        FTP_REQUIRE(i == 0 || d.unit == layers[i - 1].unit || d.unit == layers[i - 1].unit + 1, FTP_EINVAL,
+                    "build_model: op %d: unit ids must be non-decreasing without gaps", i);
+        if (i == 0 || d.unit != layers[i - 1].unit) { m.unit_first.push_back(i); m.unit_last.push_back(i); }
+        else m.unit_last.back() = i;
+        o.N = N; o.H = H; o.W = W; o.C = C;
+        o.w_off = o.b_off = o.rm_off = o.rv_off = -1;
+        o.w_cnt = o.b_cnt = 0;
+        o.gslot = -1; o.galias = i; o.addend_of = -1;
+        o.Ho = H; o.Wo = W; o.Co = C;
+        FTP_REQUIRE(d.act >= 0 && d.act <= 2, FTP_EINVAL, "build_model: op %d: unknown activation %d", i, d.act);
+        switch (d.kind) {
+            case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
+                FTP_REQUIRE(d.cin == C && d.cout >= 1, FTP_EINVAL, "build_model: op %d: cin %d does not match the incoming %d channels", i, d.cin, C);
+                int kh = 1, kw = 1, st = 1, ph = 0, pw = 0;
+                if (d.kind == FTP_CONV1D) { FTP_REQUIRE(H == 1, FTP_EINVAL, "build_model: op %d: CONV1D needs H == 1", i); kw = d.k; st = d.stride; pw = d.pad; }
+                else if (d.kind == FTP_CONV2D) { kh = kw = d.k; st = d.stride; ph = pw = d.pad; }
+                else FTP_REQUIRE(H == 1 && W == 1, FTP_EINVAL, "build_model: op %d: FC needs a 1x1 input (pool first)", i);
+                FTP_REQUIRE(kw >= 1 && st >= 1 && pw >= 0, FTP_EINVAL, "build_model: op %d: bad kernel geometry", i);
+                o.Ho = (H + 2 * ph - kh) / st + 1; o.Wo = (W + 2 * pw - kw) / st + 1; o.Co = d.cout;
+                FTP_REQUIRE(H + 2 * ph >= kh && W + 2 * pw >= kw, FTP_EINVAL, "build_model: op %d: kernel larger than the padded input", i);
+                o.g = ConvGeom{N, H, W, C, o.Ho, o.Wo, o.Co, kh, kw, st, ph, pw};
+                o.w_off = poff; o.w_cnt = (long long)kh * kw * C * d.cout; poff += o.w_cnt;
+                if (d.has_bias) { o.b_off = poff; o.b_cnt = d.cout; poff += o.b_cnt; }
+                break;
+            }
+            case FTP_DWCONV3x3:
+                FTP_REQUIRE(d.cin == C && d.cout == C && d.k == 3 && d.pad == 1 && d.stride >= 1, FTP_EINVAL,
+                            "build_model: op %d: depthwise needs cin == cout == incoming channels, k 3, pad 1", i);
+                o.Ho = (H + 2 - 3) / d.stride + 1; o.Wo = (W + 2 - 3) / d.stride + 1;
+                o.g = ConvGeom{N, H, W, C, o.Ho, o.Wo, C, 3, 3, d.stride, 1, 1};
+                o.w_off = poff; o.w_cnt = 9LL * C; poff += o.w_cnt;
+                break;
+            case FTP_BN:
+                FTP_REQUIRE(d.cin == C, FTP_EINVAL, "build_model: op %d: BN over %d channels but %d arrive", i, d.cin, C);
+                o.w_off = poff; o.w_cnt = C; poff += C;
+                o.b_off = poff; o.b_cnt = C; poff += C;
+                o.rm_off = soff; soff += C; o.rv_off = soff; soff += C;
+                break;
+            case FTP_ACT: break;
+            case FTP_ADD_RESIDUAL: {
+                const int s = d.residual_src;
+                FTP_REQUIRE(s >= -1 && s < i - 1, FTP_EINVAL, "build_model: op %d: residual_src %d out of range", i, s);
+                FTP_REQUIRE(s >= m.unit_first.back() - 1, FTP_EINVAL, "build_model: op %d: a residual connection may not cross a unit edge", i);
+                const int sh = s < 0 ? cfg->in_h : m.ops[s].Ho, sw = s < 0 ? cfg->in_w : m.ops[s].Wo, sc = s < 0 ? cfg->in_c : m.ops[s].Co;
+                FTP_REQUIRE(sh == H && sw == W && sc == C, FTP_EINVAL, "build_model: op %d: residual shapes differ", i);
+                FTP_REQUIRE(i >= 1 && layers[i - 1].kind == FTP_BN && layers[i - 1].act == FTP_ACT_NONE && layers[i - 1].unit == d.unit,
+                            FTP_EUNSUPPORTED, "build_model: op %d: a residual add must follow a BN without activation", i);
+                break;
+            }
+            case FTP_MAXPOOL2:
+                FTP_REQUIRE(H >= 2 && W >= 2, FTP_EINVAL, "build_model: op %d: max-pool input smaller than 2x2", i);
+                o.Ho = H / 2; o.Wo = W / 2;
+                break;
+            case FTP_GAP: o.Ho = 1; o.Wo = 1; break;
+            case FTP_SOFTMAX_CE:
+                FTP_REQUIRE(i == n - 1, FTP_EINVAL, "build_model: op %d: SOFTMAX_CE must be the last op", i);
+                FTP_REQUIRE(H == 1 && W == 1 && C == cfg->n_classes, FTP_EINVAL, "build_model: the loss expects %d logits, got %dx%dx%d", cfg->n_classes, H, W, C);
+                FTP_REQUIRE(i >= 1 && layers[i - 1].kind == FTP_FC && layers[i - 1].act == FTP_ACT_NONE && layers[i - 1].unit == d.unit,
+                            FTP_EUNSUPPORTED, "build_model: SOFTMAX_CE must directly follow an FC op of the same unit");
+                o.Ho = o.Wo = o.Co = 1;
+                break;
+            default: return fail(FTP_EINVAL, "build_model: op %d: unknown kind %d", i, d.kind);
+        }
+        o.in_elems = (long long)N * H * W * C;
+        o.out_elems = d.kind == FTP_SOFTMAX_CE ? 1 : (long long)N * o.Ho * o.Wo * o.Co;
+        FTP_REQUIRE(o.in_elems < (1LL << 31) && o.out_elems < (1LL << 31), FTP_ERANGE, "build_model: op %d: tensor too large", i);
+        o.out_f32 = d.kind == FTP_SOFTMAX_CE || (d.kind == FTP_FC && i + 1 < n && layers[i + 1].kind == FTP_SOFTMAX_CE);
+        H = o.Ho; W = o.Wo; C = o.Co;
+    }
+    m.L = (int)m.unit_first.size();
+    m.P = poff; m.R = soff;
+    m.unit_p_off.assign(m.L, 0); m.unit_p_cnt.assign(m.L, 0); m.unit_s_off.assign(m.L, 0); m.unit_s_cnt.assign(m.L, 0);
+    for (int u = 0; u < m.L; ++u) {
+        long long p0 = -1, p1 = 0, s0 = -1, s1 = 0;
+        for (int i = m.unit_first[u]; i <= m.unit_last[u]; ++i) {
+            const Op& o = m.ops[i];
+            if (o.w_off >= 0) { if (p0 < 0) p0 = o.w_off; p1 = o.w_off + o.w_cnt; }
+            if (o.b_off >= 0) p1 = o.b_off + o.b_cnt;
+            if (o.rm_off >= 0) { if (s0 < 0) s0 = o.rm_off; s1 = o.rv_off + o.C; }
+        }
+        m.unit_p_off[u] = p0 < 0 ? (u ? m.unit_p_off[u - 1] + m.unit_p_cnt[u - 1] : 0) : p0;
+        m.unit_p_cnt[u] = p0 < 0 ? 0 : p1 - p0;
+        m.unit_s_off[u] = s0 < 0 ? (u ? m.unit_s_off[u - 1] + m.unit_s_cnt[u - 1] : 0) : s0;
+        m.unit_s_cnt[u] = s0 < 0 ? 0 : s1 - s0;
+    }
+    // fuse "BN (no activation) -> residual add"
+    for (int i = 0; i + 1 < n; ++i)
+        if (m.ops[i + 1].d.kind == FTP_ADD_RESIDUAL) { m.ops[i].fused_add = true; m.ops[i + 1].skip = true; }
+    return FTP_OK;
+}
+
+// ---- gradient-buffer plan: which slot holds the gradient of each op's output ------------------------
+ftp_status plan_gradients(ftp_model& m, int* n_slots) {
+    const int n = (int)m.ops.size();
+    std::vector<int> refc;               // per slot: readers still to come
+    std::vector<int> freel;
+    std::vector<int> pending(n + 1, -1); // pending[j+1]: op whose output-gradient buffer must be added into grad(out[j])
+    auto alloc = [&]() { if (!freel.empty()) { int s = freel.back(); freel.pop_back(); refc[s] = 1; return s; } refc.push_back(1); return (int)refc.size() - 1; };
+    auto release = [&](int s) { if (s >= 0 && --refc[s] == 0) freel.push_back(s); };
+    for (int i = n - 1; i >= 0; --i) {
+        Op& o = m.ops[i];
+        if (o.d.kind == FTP_SOFTMAX_CE) { m.ops[i - 1].gslot = -2; continue; }
+        const int k = o.galias;                         // buffer this op reads its output gradient from
+        const int s = m.ops[k].gslot;
+        FTP_REQUIRE(s != -1, FTP_ESTATE, "build_model: op %d has no consumer for its output", i);
+        if (o.d.kind == FTP_ADD_RESIDUAL) {
+            m.ops[i - 1].galias = k; m.ops[i - 1].gslot = s;
+            const int src = o.d.residual_src;
+            FTP_REQUIRE(pending[src + 1] < 0, FTP_EUNSUPPORTED, "build_model: op %d: two residual adds share one source", i);
+            pending[src + 1] = k;
+            if (s >= 0) refc[s] += 1;                   // readers: op i-1 (already counted as op i's read) and the addend user
+            continue;
+        }
+        if (i > 0) {
+            m.ops[i - 1].gslot = alloc();
+            if (pending[i] >= 0) o.addend_of = pending[i];
+        }
+        // after op i has run: its own output gradient is consumed, and so is the addend it folded in
+        if (s >= 0) release(s);
+        if (o.addend_of >= 0) release(m.ops[o.addend_of].gslot);
+    }
+    *n_slots = (int)refc.size();
+    return FTP_OK;
+}
+
+// ---- memory layout inside the workspace --------------------------------------------------------------
+ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinned_total) {
+    Bump bp{dev_base, 0};
+    const int n = (int)m.ops.size();
+    const size_t es = (size_t)m.esize;
+    m.arena.assign(m.cfg.max_stages, Arena{});
+    for (auto& a : m.arena) {
+        a.w = (float*)bp.take((size_t)m.P * 4);
+        a.m = (float*)bp.take((size_t)m.P * 4);
+        a.run = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
+        a.wb = m.cfg.precision == FTP_BF16 ? (__nv_bfloat16*)bp.take((size_t)m.P * 2) : nullptr;
+    }
+    m.grad = (float*)bp.take((size_t)m.P * 4);
+    m.state_backup = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
+    size_t max_act = 0, red = 0, foldd = 0, dpre = 0;
+    for (int i = 0; i < n; ++i) {
+        Op& o = m.ops[i];
+        const size_t obytes = (size_t)o.out_elems * (o.out_f32 ? 4 : es);
+        o.out = (o.fused_add) ? nullptr : bp.take(obytes);            // a fused BN writes into the add's buffer
+        if (!o.out_f32 && i + 1 < n) max_act = std::max(max_act, obytes);
+        const long long Mout = (long long)o.N * o.Ho * o.Wo;
+        if (o.d.kind == FTP_BN) {
+            float* t = (float*)bp.take((size_t)o.C * 7 * 4 + 256 * 7);
+            const size_t stride = align_up((size_t)o.C * 4, 256) / 4;
+            o.scale = t; o.shift = t + stride; o.mean = t + 2 * stride; o.rstd = t + 3 * stride; o.coef = t + 4 * stride;
+            o.fold = make_fold(Mout, o.C, m.esize);
+            foldd = std::max(foldd, fold_partial_doubles(o.fold));
+        } else if (is_contraction(o.d.kind)) {
+            red = std::max(red, conv_wgrad_scratch_floats(o.g));
+            o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
+            if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
+            if (o.d.act != FTP_ACT_NONE) dpre = std::max(dpre, obytes);
+        } else if (o.d.kind == FTP_DWCONV3x3) {
+            red = std::max(red, dwconv_wgrad_scratch_floats(o.g));
+        }
+    }
+    int n_slots = 0;
+    ftp_status s = plan_gradients(m, &n_slots);
+    if (s != FTP_OK) return s;
+    m.slot_bytes = align_up(std::max<size_t>(max_act, 256), 256);
+    m.slots.assign(n_slots, nullptr);
+    for (auto& p : m.slots) p = bp.take(m.slot_bytes);
+    m.red_floats = std::max<size_t>(red, 64); m.red_scratch = (float*)bp.take(m.red_floats * 4);
+    m.fold_doubles = std::max<size_t>(foldd, 64); m.fold_scratch = (double*)bp.take(m.fold_doubles * 8);
+    m.dpre_bytes = std::max<size_t>(dpre, 256); m.dpre = bp.take(m.dpre_bytes);
+    m.dlogits = (float*)bp.take((size_t)m.cfg.batch * m.cfg.n_classes * 4);
+    m.per_sample = (float*)bp.take((size_t)m.cfg.batch * 4);
+    m.loss_dev = (float*)bp.take(256);
+    m.labels_dev = (int32_t*)bp.take((size_t)m.cfg.batch * 4);
+    m.input_dev = bp.take((size_t)m.cfg.batch * m.cfg.in_h * m.cfg.in_w * m.cfg.in_c * es);
+    *dev_total = align_up(bp.off, 256);
+    *pinned_total = 256;
+    return FTP_OK;
+}
+
+#define CUDA_OK(call)                                                                      \
+    do {                                                                                   \
+        cudaError_t e_ = (call);                                                           \
+        if (e_ != cudaSuccess) return fail(FTP_ECUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+ftp_status check_launches(const char* where) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(FTP_ECUDA, "%s: %s", where, cudaGetErrorString(e));
+    return FTP_OK;
+}
+
+inline bool a16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+
+// ---- forward of a unit range ------------------------------------------------------------------------------
+template <typename T>
+ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_out, const int32_t* labels, float* loss_out,
+                     cudaStream_t st) {
+    const int first = m->unit_first[a], last = m->unit_last[b - 1];
+    const double es = (double)m->esize;
+    m->stage_in[first] = act_in;
+    for (int i = first; i <= last; ++i) {
+        Op& o = m->ops[i];
+        const int u = o.d.unit;
+        if (m->unit_events && i == m->unit_first[u]) cudaEventRecord(m->ev_f[u], st);
+        const void* in = (i == first) ? act_in : m->cur_out[i - 1];
+        void* out = (i == last && act_out) ? act_out : o.out;
+        if (o.fused_add) out = (i + 1 == last && act_out) ? act_out : m->ops[i + 1].out;
+        const Arena& ar = m->arena[m->owner[u]];
+        const long long Mout = (long long)o.N * o.Ho * o.Wo;
+        switch (o.d.kind) {
+            case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
+                const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
+                if (m->cfg.precision == FTP_FP32) {
+                    Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
+                    conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, o.g, o.d.act, st);
+                } else {
+                    return fail(FTP_EUNSUPPORTED, "bf16 contractions are not built yet");
+                }
+                break;
+            }
+            case FTP_DWCONV3x3: {
+                Scope sc(m, st, K_DW_FWD, u, i, 0, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
+                dwconv_fwd<T>((const T*)in, ar.w + o.w_off, (T*)out, o.g, st);
+                break;
+            }
+            case FTP_BN: {
+                const long long Mr = (long long)o.N * o.H * o.W;
+                { Scope sc(m, st, K_BN_STATS, u, i, 0, o.in_elems * es, 3.0 * o.in_elems);
+                  bn_stats<T>((const T*)in, Mr, o.C, o.fold, m->fold_scratch, st); }
+                { Scope sc(m, st, K_BN_FINALIZE, u, i, 0, fold_partial_doubles(o.fold) * 8.0, 0.0);
+                  bn_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, ar.w + o.b_off, m->cfg.bn_eps, m->cfg.bn_momentum,
+                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.rstd, st); }
+                const void* res = nullptr;
+                if (o.fused_add) { const int s = m->ops[i + 1].d.residual_src; res = s < first ? act_in : m->cur_out[s]; }
+                { Scope sc(m, st, K_BN_APPLY, u, i, 0, (o.in_elems * (res ? 3.0 : 2.0)) * es, 2.0 * o.in_elems);
+                  bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.scale, o.shift, o.d.act, st); }
+                break;
+            }
+            case FTP_ACT: {
+                Scope sc(m, st, K_ACT_FWD, u, i, 0, 2.0 * o.in_elems * es, (double)o.in_elems);
+                act_fwd<T>((const T*)in, (T*)out, o.in_elems, o.d.act, st);
+                break;
+            }
+            case FTP_ADD_RESIDUAL: break;            // folded into the preceding BN
+            case FTP_MAXPOOL2: {
+                Scope sc(m, st, K_MAXPOOL_FWD, u, i, 0, (o.in_elems + o.out_elems) * es, 3.0 * o.out_elems);
+                maxpool_fwd<T>((const T*)in, (T*)out, o.N, o.H, o.W, o.C, st);
+                break;
+            }
+            case FTP_GAP: {
+                Scope sc(m, st, K_GAP_FWD, u, i, 0, (o.in_elems + o.out_elems) * es, (double)o.in_elems);
+                gap_fwd<T>((const T*)in, (T*)out, o.N, o.H * o.W, o.C, st);
+                break;
+            }
+            case FTP_SOFTMAX_CE: {
+                Scope sc(m, st, K_SOFTMAX_CE, u, i, 0, 3.0 * o.in_elems * 4.0, 4.0 * o.in_elems, 2);
+                softmax_ce((const float*)in, labels, o.N, o.C, m->per_sample, m->dlogits, loss_out, st);
+                out = loss_out;
+                break;
+            }
+        }
+        m->cur_out[i] = out;
+        if (o.fused_add) m->cur_out[i + 1] = out;
+        m->fwd_done[i] = 1;
+    }
+    if (m->unit_events) cudaEventRecord(m->ev_f[b], st);
+    return check_launches("forward");
+}
+
+// ---- backward of a unit range -----------------------------------------------------------------------------
+template <typename T>
+ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* grad_in, bool internal, cudaStream_t st) {
+    const int first = m->unit_first[a], last = m->unit_last[b - 1];
+    const double es = (double)m->esize;
+    for (int i = first; i <= last; ++i)
+        FTP_REQUIRE(m->fwd_done[i], FTP_ESTATE, "run_stage_backward: units [%d,%d) have not been run forward", a, b);
+    const void* act_in = m->stage_in[first];
+    FTP_REQUIRE(act_in, FTP_ESTATE, "run_stage_backward: the last forward did not start at unit %d", a);
+    auto gptr = [&](int j) -> void* {
+        const int k = m->ops[j].galias;
+        if (k == last && grad_out) return const_cast<void*>(grad_out);
+        const int s = m->ops[k].gslot;
+        return s == -2 ? (void*)m->dlogits : m->slots[s];
+    };
+    for (int i = last; i >= first; --i) {
+        Op& o = m->ops[i];
+        const int u = o.d.unit;
+        if (m->unit_events && i == m->unit_last[u]) cudaEventRecord(m->ev_b[u + 1], st);
+        if (o.d.kind == FTP_SOFTMAX_CE || o.d.kind == FTP_ADD_RESIDUAL) continue;   // dlogits were written by the forward
+        const void* in = (i == first) ? act_in : m->cur_out[i - 1];
+        const void* go = gptr(i);
+        void* gi = nullptr;
+        if (i == first) gi = grad_in ? grad_in : ((internal && first > 0) ? m->slots[m->ops[first - 1].gslot] : nullptr);
+        else gi = gptr(i - 1);
+        const void* addend = o.addend_of >= 0 ? gptr(o.addend_of) : nullptr;
+        const Arena& ar = m->arena[m->owner[u]];
+        float* gr = m->grad;
+        const long long Mout = (long long)o.N * o.Ho * o.Wo;
+        switch (o.d.kind) {
+            case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
+                const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
+                if (m->cfg.precision != FTP_FP32) return fail(FTP_EUNSUPPORTED, "bf16 contractions are not built yet");
+                const float* d = (const float*)go;
+                if (o.d.act != FTP_ACT_NONE || o.b_off >= 0) {
+                    float* dpre = o.d.act != FTP_ACT_NONE ? (float*)m->dpre : nullptr;
+                    Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 4.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
+                    act_bias_bwd<float>(d, (const float*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
+                                        o.b_off >= 0 ? gr + o.b_off : nullptr, st);
+                    if (dpre) d = dpre;
+                }
+                { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
+                  conv_wgrad_f32((const float*)in, d, gr + o.w_off, m->red_scratch, o.g, st); }
+                if (gi) {
+                    Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl);
+                    conv_dgrad_f32(d, ar.w + o.w_off, (const float*)addend, (float*)gi, o.g, st);
+                }
+                break;
+            }
+            case FTP_DWCONV3x3: {
+                { Scope sc(m, st, K_DW_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems, 2);
+                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, m->red_scratch, o.g, st); }
+                if (gi) {
+                    Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
+                    dwconv_dgrad<T>((const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, o.g, st);
+                }
+                break;
+            }
+            case FTP_BN: {
+                const long long Mr = (long long)o.N * o.H * o.W;
+                { Scope sc(m, st, K_BN_BWD_REDUCE, u, i, 1, 2.0 * o.in_elems * es, 8.0 * o.in_elems);
+                  bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.rstd, o.d.act, m->fold_scratch, st); }
+                { Scope sc(m, st, K_BN_BWD_FINALIZE, u, i, 1, fold_partial_doubles(o.fold) * 8.0, 0.0);
+                  bn_bwd_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, st); }
+                if (gi) {
+                    Scope sc(m, st, K_BN_BWD_APPLY, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, 8.0 * o.in_elems);
+                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.scale, o.shift, o.mean, o.rstd, o.coef, o.d.act, st);
+                }
+                break;
+            }
+            case FTP_ACT:
+                if (gi) {
+                    Scope sc(m, st, K_ACT_BWD, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, (double)o.in_elems);
+                    act_bwd<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, o.in_elems, o.d.act, st);
+                }
+                break;
+            case FTP_MAXPOOL2:
+                FTP_REQUIRE(!addend, FTP_EUNSUPPORTED, "a residual source feeding a max-pool is not supported");
+                if (gi) {
+                    Scope sc(m, st, K_MAXPOOL_BWD, u, i, 1, (2.0 * o.in_elems + o.out_elems) * es, 4.0 * o.out_elems);
+                    maxpool_bwd<T>((const T*)go, (const T*)in, (T*)gi, o.N, o.H, o.W, o.C, st);
+                }
+                break;
+            case FTP_GAP:
+                FTP_REQUIRE(!addend, FTP_EUNSUPPORTED, "a residual source feeding a global pool is not supported");
+                if (gi) {
+                    Scope sc(m, st, K_GAP_BWD, u, i, 1, (o.in_elems + o.out_elems) * es, (double)o.in_elems);
+                    gap_bwd<T>((const T*)go, (T*)gi, o.N, o.H * o.W, o.C, st);
+                }
+                break;
+        }
+    }
+    if (m->unit_events) cudaEventRecord(m->ev_b[a], st);
+    return check_launches("backward");
+}
+
+ftp_status check_range(const ftp_model* m, int a, int b, const char* who) {
+    FTP_REQUIRE(m, FTP_EINVAL, "%s: null model", who);
+    FTP_REQUIRE(a >= 0 && b <= m->L && a < b, FTP_EINVAL, "%s: need 0 <= a < b <= L (a=%d, b=%d, L=%d)", who, a, b, m->L);
+    return FTP_OK;
+}
+
+ftp_status sgd_range(ftp_model* m, int a, int b, float lr, float* snap_dev, float* snap_host, cudaStream_t st) {
+    const float mu = m->cfg.momentum, wd = m->cfg.weight_decay;
+    int u = a;
+    while (u < b) {
+        int v = u + 1;
+        while (v < b && m->owner[v] == m->owner[u] && m->mom_init[v] == m->mom_init[u]) ++v;
+        const long long off = m->unit_p_off[u];
+        const long long cnt = m->unit_p_off[v - 1] + m->unit_p_cnt[v - 1] - off;
+        if (cnt > 0) {
+            const Arena& ar = m->arena[m->owner[u]];
+            const long long rel = off - m->unit_p_off[a];
+            Scope sc(m, st, K_SGD, u, -1, 2, cnt * (mu != 0.f ? (m->mom_init[u] ? 20.0 : 16.0) : 12.0) + (ar.wb ? 2.0 * cnt : 0.0) +
+                     (snap_dev ? 4.0 * cnt : 0.0) + (snap_host ? 4.0 * cnt : 0.0), 6.0 * cnt);
+            sgd_update(ar.w + off, m->grad + off, mu != 0.f ? ar.m + off : nullptr, cnt, lr, mu, wd, m->mom_init[u] ? 0 : 1,
+                       ar.wb ? ar.wb + off : nullptr, snap_dev ? snap_dev + rel : nullptr, snap_host ? snap_host + rel : nullptr, st);
+        }
+        for (int k = u; k < v; ++k) m->mom_init[k] = 1;
+        u = v;
+    }
+    return check_launches("sgd_step");
+}
+
+template <typename T>
+ftp_status train_step_t(ftp_model* m, const void* x, const int32_t* labels, float lr, cudaStream_t st) {
+    const void* act = x;
+    for (int s = 0; s < m->n_stages; ++s) {
+        const int a = m->points[s], b = m->points[s + 1];
+        ftp_status r = fwd_range<T>(m, a, b, act, nullptr, b == m->L ? labels : nullptr, b == m->L ? m->loss_dev : nullptr, st);
+        if (r != FTP_OK) return r;
+        act = m->cur_out[m->unit_last[b - 1]];
+    }
+    for (int s = m->n_stages - 1; s >= 0; --s) {
+        ftp_status r = bwd_range<T>(m, m->points[s], m->points[s + 1], nullptr, nullptr, true, st);
+        if (r != FTP_OK) return r;
+    }
+    for (int s = 0; s < m->n_stages; ++s) {
+        ftp_status r = sgd_range(m, m->points[s], m->points[s + 1], lr, nullptr, nullptr, st);
+        if (r != FTP_OK) return r;
+    }
+    return FTP_OK;
+}
+
+}  // namespace
+
+// ================================== C ABI ===========================================================
+
+extern "C" ftp_status ftp_workspace_bytes(const ftp_layer_desc* layers, int32_t n, const ftp_model_cfg* cfg, size_t* dev_bytes,
+                                          size_t* pinned_bytes) {
+    FTP_REQUIRE(dev_bytes && pinned_bytes, FTP_EINVAL, "workspace_bytes: null output");
+    ftp_model m{};
+    ftp_status s = plan_ops(layers, n, cfg, m);
+    if (s != FTP_OK) return s;
+    return layout(m, nullptr, dev_bytes, pinned_bytes);
+}
+
+extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, const ftp_model_cfg* cfg, void* dev_ws, size_t dev_bytes,
+                                      void* pinned_ws, size_t pinned_bytes, ftp_model** out) {
+    FTP_REQUIRE(out && dev_ws && pinned_ws, FTP_EINVAL, "build_model: null argument");
+    FTP_REQUIRE((reinterpret_cast<uintptr_t>(dev_ws) & 255) == 0, FTP_ERANGE, "build_model: the device workspace must be 256-byte aligned");
+    ftp_model* m = new (std::nothrow) ftp_model{};
+    FTP_REQUIRE(m, FTP_ENOMEM, "build_model: out of host memory");
+    ftp_status s = plan_ops(layers, n, cfg, *m);
+    size_t need = 0, pneed = 0;
+    if (s == FTP_OK) s = layout(*m, (char*)dev_ws, &need, &pneed);
+    if (s == FTP_OK && (need > dev_bytes || pneed > pinned_bytes))
+        s = fail(FTP_ENOMEM, "build_model: workspace too small (need %zu device and %zu pinned bytes)", need, pneed);
+    if (s != FTP_OK) { delete m; return s; }
+    m->pinned = (float*)pinned_ws; m->pinned_bytes = pinned_bytes;
+    m->owner.assign(m->L, 0);
+    m->points = {0, m->L};
+    m->n_stages = 1;
+    m->mom_init.assign(m->L, 0);
+    m->stage_in.assign(m->ops.size(), nullptr);
+    m->cur_out.assign(m->ops.size(), nullptr);
+    m->fwd_done.assign(m->ops.size(), 0);
+    m->trace = false; m->tr_used = 0; m->unit_events = false;
+    *out = m;
+    return FTP_OK;
+}
+
+extern "C" void ftp_destroy_model(ftp_model* m) {
+    if (!m) return;
+    for (auto& t : m->tr) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
+    for (auto e : m->ev_f) cudaEventDestroy(e);
+    for (auto e : m->ev_b) cudaEventDestroy(e);
+    delete m;
+}
+
+extern "C" ftp_status ftp_num_units(const ftp_model* m, int32_t* L) {
+    FTP_REQUIRE(m && L, FTP_EINVAL, "num_units: null argument");
+    *L = m->L;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_unit_param_span(const ftp_model* m, int32_t unit, int64_t* offset, int64_t* count) {
+    FTP_REQUIRE(m && offset && count, FTP_EINVAL, "unit_param_span: null argument");
+    FTP_REQUIRE(unit >= 0 && unit < m->L, FTP_ERANGE, "unit_param_span: unit %d out of range", unit);
+    *offset = m->unit_p_off[unit]; *count = m->unit_p_cnt[unit];
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_unit_state_span(const ftp_model* m, int32_t unit, int64_t* offset, int64_t* count) {
+    FTP_REQUIRE(m && offset && count, FTP_EINVAL, "unit_state_span: null argument");
+    FTP_REQUIRE(unit >= 0 && unit < m->L, FTP_ERANGE, "unit_state_span: unit %d out of range", unit);
+    *offset = m->unit_s_off[unit]; *count = m->unit_s_cnt[unit];
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_unit_output_shape(const ftp_model* m, int32_t unit, int32_t shape[4], int64_t* bytes) {
+    FTP_REQUIRE(m && shape && bytes, FTP_EINVAL, "unit_output_shape: null argument");
+    FTP_REQUIRE(unit >= 0 && unit < m->L, FTP_ERANGE, "unit_output_shape: unit %d out of range", unit);
+    const Op& o = m->ops[m->unit_last[unit]];
+    if (o.d.kind == FTP_SOFTMAX_CE) { shape[0] = shape[1] = shape[2] = shape[3] = 1; *bytes = 4; return FTP_OK; }
+    shape[0] = o.N; shape[1] = o.Ho; shape[2] = o.Wo; shape[3] = o.Co;
+    *bytes = o.out_elems * (o.out_f32 ? 4 : m->esize);
+    return FTP_OK;
+}
+
+static ftp_status tensor_ptr(const ftp_model* m, int which, int unit, int64_t count, float** p, const char* who) {
+    FTP_REQUIRE(m, FTP_EINVAL, "%s: null model", who);
+    FTP_REQUIRE(unit >= 0 && unit < m->L, FTP_ERANGE, "%s: unit %d out of range", who, unit);
+    const Arena& ar = m->arena[m->owner[unit]];
+    long long want = m->unit_p_cnt[unit];
+    switch (which) {
+        case FTP_T_WEIGHTS: *p = ar.w + m->unit_p_off[unit]; break;
+        case FTP_T_GRADS: *p = m->grad + m->unit_p_off[unit]; break;
+        case FTP_T_MOMENTUM: *p = ar.m + m->unit_p_off[unit]; break;
+        case FTP_T_STATE: *p = ar.run + m->unit_s_off[unit]; want = m->unit_s_cnt[unit]; break;
+        default: return fail(FTP_EINVAL, "%s: unknown tensor selector %d", who, which);
+    }
+    FTP_REQUIRE(count == want, FTP_ERANGE, "%s: unit %d holds %lld floats, caller passed %lld", who, unit, want, (long long)count);
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_set_tensor(ftp_model* m, int32_t which, int32_t unit, const float* src, int64_t count, int32_t src_is_device,
+                                     void* stream) {
+    float* dst = nullptr;
+    ftp_status s = tensor_ptr(m, which, unit, count, &dst, "set_tensor");
+    if (s != FTP_OK) return s;
+    if (count == 0) return FTP_OK;
+    FTP_REQUIRE(src, FTP_EINVAL, "set_tensor: null source");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaMemcpyAsync(dst, src, (size_t)count * 4, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+    if (which == FTP_T_WEIGHTS) {
+        const Arena& ar = m->arena[m->owner[unit]];
+        if (ar.wb) { Scope sc(m, st, K_COPY, unit, -1, 2, 6.0 * count, 0.0); f32_to_bf16(dst, ar.wb + m->unit_p_off[unit], count, st); }
+        m->mom_init[unit] = 0;
+    } else if (which == FTP_T_MOMENTUM) m->mom_init[unit] = 1;
+    if (!src_is_device) CUDA_OK(cudaStreamSynchronize(st));
+    return check_launches("set_tensor");
+}
+
+extern "C" ftp_status ftp_get_tensor(const ftp_model* m, int32_t which, int32_t unit, float* dst, int64_t count, int32_t dst_is_device,
+                                     void* stream) {
+    float* src = nullptr;
+    ftp_status s = tensor_ptr(m, which, unit, count, &src, "get_tensor");
+    if (s != FTP_OK) return s;
+    if (count == 0) return FTP_OK;
+    FTP_REQUIRE(dst, FTP_EINVAL, "get_tensor: null destination");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaMemcpyAsync(dst, src, (size_t)count * 4, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    if (!dst_is_device) CUDA_OK(cudaStreamSynchronize(st));
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_run_stage_forward(ftp_model* m, int32_t a, int32_t b, const void* act_in, void* act_out, const int32_t* labels,
+                                            float* loss_out, void* stream) {
+    ftp_status s = check_range(m, a, b, "run_stage_forward");
+    if (s != FTP_OK) return s;
+    FTP_REQUIRE(act_in, FTP_EINVAL, "run_stage_forward: null act_in");
+    FTP_REQUIRE(a16(act_in) && a16(act_out), FTP_ERANGE, "run_stage_forward: activation buffers must be 16-byte aligned");
+    if (b == m->L) FTP_REQUIRE(labels && loss_out && !act_out, FTP_EINVAL, "run_stage_forward: the last stage needs labels and loss_out, and no act_out");
+    else FTP_REQUIRE(act_out && !labels && !loss_out, FTP_EINVAL, "run_stage_forward: an inner stage needs act_out and takes no labels");
+    cudaStream_t st = (cudaStream_t)stream;
+    return m->cfg.precision == FTP_FP32 ? fwd_range<float>(m, a, b, act_in, act_out, labels, loss_out, st)
+                                        : fwd_range<__nv_bfloat16>(m, a, b, act_in, act_out, labels, loss_out, st);
+}
+
+extern "C" ftp_status ftp_run_stage_backward(ftp_model* m, int32_t a, int32_t b, const void* grad_out, void* grad_in, void* stream) {
+    ftp_status s = check_range(m, a, b, "run_stage_backward");
+    if (s != FTP_OK) return s;
+    if (b == m->L) FTP_REQUIRE(!grad_out, FTP_EINVAL, "run_stage_backward: the last stage takes no grad_out");
+    else FTP_REQUIRE(grad_out, FTP_EINVAL, "run_stage_backward: an inner stage needs grad_out");
+    FTP_REQUIRE(a == 0 || grad_in, FTP_EINVAL, "run_stage_backward: grad_in is required when a > 0");
+    FTP_REQUIRE(a16(grad_out) && a16(grad_in), FTP_ERANGE, "run_stage_backward: gradient buffers must be 16-byte aligned");
+    cudaStream_t st = (cudaStream_t)stream;
+    return m->cfg.precision == FTP_FP32 ? bwd_range<float>(m, a, b, grad_out, grad_in, false, st)
+                                        : bwd_range<__nv_bfloat16>(m, a, b, grad_out, grad_in, false, st);
+}
+
+extern "C" ftp_status ftp_get_logits(const ftp_model* m, float* dst, int32_t dst_is_device, void* stream) {
+    FTP_REQUIRE(m && dst, FTP_EINVAL, "get_logits: null argument");
+    const int fc = (int)m->ops.size() - 2;
+    FTP_REQUIRE(m->fwd_done[fc] && m->cur_out[fc], FTP_ESTATE, "get_logits: no forward has reached the last unit yet");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaMemcpyAsync(dst, m->cur_out[fc], (size_t)m->cfg.batch * m->cfg.n_classes * 4,
+                            dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    if (!dst_is_device) CUDA_OK(cudaStreamSynchronize(st));
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_sgd_step(ftp_model* m, int32_t a, int32_t b, float lr, float* snap_dev, float* snap_host, void* stream) {
+    ftp_status s = check_range(m, a, b, "sgd_step");
+    if (s != FTP_OK) return s;
+    return sgd_range(m, a, b, lr, snap_dev, snap_host, (cudaStream_t)stream);
+}
+
+extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, int32_t inputs_on_host, float lr, float* loss_host,
+                                     void* stream) {
+    FTP_REQUIRE(m && x && labels, FTP_EINVAL, "train_step: null argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    const void* xin = x;
+    const int32_t* lab = labels;
+    if (inputs_on_host) {
+        const size_t in_bytes = (size_t)m->cfg.batch * m->cfg.in_h * m->cfg.in_w * m->cfg.in_c * m->esize;
+        CUDA_OK(cudaMemcpyAsync(m->input_dev, x, in_bytes, cudaMemcpyHostToDevice, st));
+        CUDA_OK(cudaMemcpyAsync(m->labels_dev, labels, (size_t)m->cfg.batch * 4, cudaMemcpyHostToDevice, st));
+        xin = m->input_dev; lab = m->labels_dev;
+    } else FTP_REQUIRE(a16(x), FTP_ERANGE, "train_step: the input batch must be 16-byte aligned");
+    ftp_status s = m->cfg.precision == FTP_FP32 ? train_step_t<float>(m, xin, lab, lr, st) : train_step_t<__nv_bfloat16>(m, xin, lab, lr, st);
+    if (s != FTP_OK) return s;
+    if (loss_host) {
+        CUDA_OK(cudaMemcpyAsync(m->pinned, m->loss_dev, 4, cudaMemcpyDeviceToHost, st));
+        CUDA_OK(cudaStreamSynchronize(st));
+        *loss_host = m->pinned[0];
+    }
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void* sample_in, const int32_t* labels, double* fwd_s,
+                                         double* bwd_s, int64_t* out_bytes, void* stream) {
+    FTP_REQUIRE(m && sample_in && labels && fwd_s && bwd_s && out_bytes, FTP_EINVAL, "profile_layers: null argument");
+    FTP_REQUIRE(reps >= 1 && reps <= 1000, FTP_EINVAL, "profile_layers: reps must be in 1..1000");
+    FTP_REQUIRE(a16(sample_in), FTP_ERANGE, "profile_layers: the sample batch must be 16-byte aligned");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int L = m->L;
+    while ((int)m->ev_f.size() < L + 1) { cudaEvent_t e; CUDA_OK(cudaEventCreate(&e)); m->ev_f.push_back(e); }
+    while ((int)m->ev_b.size() < L + 1) { cudaEvent_t e; CUDA_OK(cudaEventCreate(&e)); m->ev_b.push_back(e); }
+    // keep the BN running statistics: profiling is not training
+    for (int u = 0; u < L; ++u)
+        if (m->unit_s_cnt[u])
+            CUDA_OK(cudaMemcpyAsync(m->state_backup + m->unit_s_off[u], m->arena[m->owner[u]].run + m->unit_s_off[u],
+                                    (size_t)m->unit_s_cnt[u] * 4, cudaMemcpyDeviceToDevice, st));
+    std::vector<double> f(L, 0.0), bk(L, 0.0);
+    ftp_status s = FTP_OK;
+    const bool was_tracing = m->trace;
+    m->trace = false;
+    for (int r = -1; r < reps && s == FTP_OK; ++r) {            // r == -1: untimed warm-up pass
+        m->unit_events = r >= 0;
+        s = m->cfg.precision == FTP_FP32 ? fwd_range<float>(m, 0, L, sample_in, nullptr, labels, m->loss_dev, st)
+                                         : fwd_range<__nv_bfloat16>(m, 0, L, sample_in, nullptr, labels, m->loss_dev, st);
+        if (s == FTP_OK)
+            s = m->cfg.precision == FTP_FP32 ? bwd_range<float>(m, 0, L, nullptr, nullptr, true, st)
+                                             : bwd_range<__nv_bfloat16>(m, 0, L, nullptr, nullptr, true, st);
+        if (s != FTP_OK) break;
+        if (cudaStreamSynchronize(st) != cudaSuccess) { s = fail(FTP_ECUDA, "profile_layers: stream synchronisation failed"); break; }
+        if (r < 0) continue;
+        for (int u = 0; u < L; ++u) {
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, m->ev_f[u], m->ev_f[u + 1]); f[u] += ms * 1e-3;
+            cudaEventElapsedTime(&ms, m->ev_b[u + 1], m->ev_b[u]); bk[u] += ms * 1e-3;
+        }
+    }
+    m->unit_events = false;
+    m->trace = was_tracing;
+    for (int u = 0; u < L; ++u)
+        if (m->unit_s_cnt[u])
+            cudaMemcpyAsync(m->arena[m->owner[u]].run + m->unit_s_off[u], m->state_backup + m->unit_s_off[u], (size_t)m->unit_s_cnt[u] * 4,
+                            cudaMemcpyDeviceToDevice, st);
+    cudaStreamSynchronize(st);
+    if (s != FTP_OK) return s;
+    for (int u = 0; u < L; ++u) {
+        fwd_s[u] = f[u] / reps; bwd_s[u] = bk[u] / reps;
+        int32_t shp[4];
+        ftp_unit_output_shape(m, u, shp, &out_bytes[u]);
+    }
+    return check_launches("profile_layers");
+}
+
+extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int32_t n_stages, int32_t* moved_units, void* stream) {
+    FTP_REQUIRE(m && points, FTP_EINVAL, "set_partition: null argument");
+    FTP_REQUIRE(n_stages >= 1 && n_stages <= m->cfg.max_stages && n_stages <= m->L, FTP_EINVAL,
+                "set_partition: %d stages not in 1..min(max_stages=%d, L=%d)", n_stages, m->cfg.max_stages, m->L);
+    FTP_REQUIRE(points[0] == 0 && points[n_stages] == m->L, FTP_EINVAL, "set_partition: points must run from 0 to L");
+    for (int i = 0; i < n_stages; ++i) FTP_REQUIRE(points[i] < points[i + 1], FTP_EINVAL, "set_partition: stage %d is empty", i);
+    cudaStream_t st = (cudaStream_t)stream;
+    int moved = 0;
+    std::vector<int32_t> plan(m->L);
+    // Phase 1: every stage fetches what Algorithm 1 says it is missing, from the current owner's arena.
+    for (int i = 0; i < n_stages; ++i) {
+        int32_t n_local = 0;
+        ftp_status s = ftp_redistribution_plan(points, n_stages, m->points.data(), m->n_stages, -1, i < m->n_stages ? i : -1, i, plan.data(), &n_local);
+        if (s != FTP_OK) return s;
+        for (int u = points[i]; u < points[i + 1]; ++u) {
+            const int src = plan[u - points[i]];
+            if (src < 0) continue;                                   // already local
+            ++moved;
+            const Arena& from = m->arena[src];
+            const Arena& to = m->arena[i];
+            const long long po = m->unit_p_off[u], pc = m->unit_p_cnt[u], so = m->unit_s_off[u], sc_ = m->unit_s_cnt[u];
+            Scope sc(m, st, K_COPY, u, -1, 2, (pc * 2 + sc_) * 8.0, 0.0, 0);
+            if (pc) {
+                CUDA_OK(cudaMemcpyAsync(to.w + po, from.w + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+                CUDA_OK(cudaMemcpyAsync(to.m + po, from.m + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+                if (to.wb) CUDA_OK(cudaMemcpyAsync(to.wb + po, from.wb + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
+            }
+            if (sc_) CUDA_OK(cudaMemcpyAsync(to.run + so, from.run + so, (size_t)sc_ * 4, cudaMemcpyDeviceToDevice, st));
+        }
+    }
+    // Phase 2 (commit): only now does the owner table switch; later launches are stream-ordered after the copies.
+    for (int i = 0; i < n_stages; ++i)
+        for (int u = points[i]; u < points[i + 1]; ++u) m->owner[u] = i;
+    m->points.assign(points, points + n_stages + 1);
+    m->n_stages = n_stages;
+    std::fill(m->fwd_done.begin(), m->fwd_done.end(), 0);
+    if (moved_units) *moved_units = moved;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_get_partition(const ftp_model* m, int32_t* points, int32_t* n_stages) {
+    FTP_REQUIRE(m && points && n_stages, FTP_EINVAL, "get_partition: null argument");
+    for (int i = 0; i <= m->n_stages; ++i) points[i] = m->points[i];
+    *n_stages = m->n_stages;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_snapshot_weights(const ftp_model* m, int32_t stage, void* dst, size_t dst_bytes, int32_t dst_is_host, size_t* written,
+                                           void* stream) {
+    FTP_REQUIRE(m && dst, FTP_EINVAL, "snapshot_weights: null argument");
+    FTP_REQUIRE(stage >= 0 && stage < m->n_stages, FTP_ERANGE, "snapshot_weights: stage %d out of range (%d stages)", stage, m->n_stages);
+    const int a = m->points[stage], b = m->points[stage + 1];
+    size_t need = 0;
+    for (int u = a; u < b; ++u) need += (size_t)(m->unit_p_cnt[u] + m->unit_s_cnt[u]) * 4;
+    FTP_REQUIRE(need <= dst_bytes, FTP_ERANGE, "snapshot_weights: stage %d needs %zu bytes, buffer has %zu", stage, need, dst_bytes);
+    cudaStream_t st = (cudaStream_t)stream;
+    const cudaMemcpyKind kind = dst_is_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
+    char* p = (char*)dst;
+    const Arena& ar = m->arena[stage];
+    Scope sc(const_cast<ftp_model*>(m), st, K_COPY, a, -1, 2, 2.0 * need, 0.0, 0);
+    for (int u = a; u < b; ++u) {
+        if (m->unit_p_cnt[u]) { CUDA_OK(cudaMemcpyAsync(p, ar.w + m->unit_p_off[u], (size_t)m->unit_p_cnt[u] * 4, kind, st)); p += m->unit_p_cnt[u] * 4; }
+        if (m->unit_s_cnt[u]) { CUDA_OK(cudaMemcpyAsync(p, ar.run + m->unit_s_off[u], (size_t)m->unit_s_cnt[u] * 4, kind, st)); p += m->unit_s_cnt[u] * 4; }
+    }
+    if (written) *written = need;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_trace_enable(ftp_model* m, int32_t on) {
+    FTP_REQUIRE(m, FTP_EINVAL, "trace_enable: null model");
+    m->trace = on != 0;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_trace_read(ftp_model* m, ftp_trace_rec* out, int32_t max, int32_t* total) {
+    FTP_REQUIRE(m && total && (out || max == 0), FTP_EINVAL, "trace_read: null argument");
+    CUDA_OK(cudaDeviceSynchronize());
+    *total = (int32_t)m->tr_used;
+    for (size_t i = 0; i < m->tr_used; ++i) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, m->tr[i].e0, m->tr[i].e1);
+        m->tr[i].rec.ms = ms;
+        if ((int32_t)i < max) out[i] = m->tr[i].rec;
+    }
+    m->tr_used = 0;
+    return FTP_OK;
+}
+
+extern "C" const char* ftp_kernel_name(int32_t kernel) { return kernel >= 0 && kernel < K_COUNT ? kKernelNames[kernel] : "?"; }
+
+extern "C" ftp_status ftp_launch_count(const ftp_model* m, int64_t* launches) {
+    FTP_REQUIRE(m && launches, FTP_EINVAL, "launch_count: null argument");
+    *launches = g_launches;
+    return FTP_OK;
+}

@@ -1,0 +1,82 @@
+// Host-side model object: unit table, arena layout, execution and gradient-buffer plan.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <vector>
+#include "common.h"
+#include "kernels.h"
+
+namespace ftp {
+
+enum KernelId {
+    K_CONV_FWD_F32 = 0, K_CONV_DGRAD_F32, K_CONV_WGRAD_F32, K_BN_STATS, K_BN_FINALIZE, K_BN_APPLY, K_BN_BWD_REDUCE,
+    K_BN_BWD_FINALIZE, K_BN_BWD_APPLY, K_ACT_BIAS_BWD, K_DW_FWD, K_DW_DGRAD, K_DW_WGRAD, K_MAXPOOL_FWD,
+    K_MAXPOOL_BWD, K_GAP_FWD, K_GAP_BWD, K_SOFTMAX_CE, K_SGD, K_ACT_FWD, K_ACT_BWD, K_COPY, K_GEMM_BF16_FWD,
+    K_GEMM_BF16_DGRAD, K_GEMM_BF16_WGRAD, K_COUNT
+};
+
+struct Op {
+    ftp_layer_desc d;
+    int N, H, W, C;          // input shape
+    int Ho, Wo, Co;          // output shape
+    long long in_elems, out_elems;
+    ConvGeom g;
+    long long w_off, w_cnt;  // first trainable array (conv / dw weights, BN gamma), floats, canonical order
+    long long b_off, b_cnt;  // second trainable array (bias, BN beta)
+    long long rm_off, rv_off;  // BN running mean / variance in the state arena
+    void* out;               // internal output buffer
+    bool out_f32;            // output kept in float whatever the precision (logits, loss)
+    float *scale, *shift, *mean, *rstd, *coef;   // BN per-channel tables
+    FoldPlan fold;
+    bool fused_add;          // BN whose normalised output goes straight through the following residual add
+    bool skip;               // residual add folded into the preceding BN
+    int gslot;               // slot holding the gradient w.r.t. this op's output (-1 none, -2 dlogits)
+    int galias;              // op whose output-gradient buffer this op's output gradient shares
+    int addend_of;           // when writing the gradient of this op's input, add the gradient buffer of that op's output
+};
+
+struct Arena {
+    float* w;
+    float* m;
+    float* run;
+    __nv_bfloat16* wb;
+};
+
+struct TraceSlot { cudaEvent_t e0, e1; ftp_trace_rec rec; };
+
+}  // namespace ftp
+
+struct ftp_model {
+    ftp_model_cfg cfg;
+    std::vector<ftp::Op> ops;
+    int L;
+    int esize;                                    // bytes per activation element
+    std::vector<int> unit_first, unit_last;       // op index range of each unit
+    std::vector<long long> unit_p_off, unit_p_cnt, unit_s_off, unit_s_cnt;
+    long long P, R;
+    std::vector<ftp::Arena> arena;
+    float* grad;
+    std::vector<int> owner;                       // unit -> stage
+    std::vector<int> points;
+    int n_stages;
+    std::vector<char> mom_init;                   // per unit: momentum buffer holds a value
+    std::vector<void*> slots;
+    size_t slot_bytes;
+    float* red_scratch; size_t red_floats;
+    double* fold_scratch; size_t fold_doubles;
+    void* dpre; size_t dpre_bytes;
+    float* dlogits; float* per_sample; float* loss_dev; int32_t* labels_dev; void* input_dev; float* state_backup;
+    float* pinned; size_t pinned_bytes;
+    // run-time state of the last forward of each range
+    std::vector<const void*> stage_in;            // act_in of the range starting at op i
+    std::vector<void*> cur_out;                   // resolved output pointer of op i
+    std::vector<char> fwd_done;
+    const int32_t* cur_labels;
+    // trace
+    bool trace;
+    std::vector<ftp::TraceSlot> tr;
+    size_t tr_used;
+    // per-unit profiling events
+    bool unit_events;
+    std::vector<cudaEvent_t> ev_f, ev_b;
+};

@@ -1,0 +1,117 @@
+// Host-side scheduling arithmetic: capacity estimate (Eq. 1-3), partition optimiser (Eq. 4-7)
+// and the weight-redistribution plan (Algorithm 1).  No GPU involved.
+#include <cstring>
+#include <limits>
+#include <vector>
+#include "common.h"
+
+namespace ftp {
+
+static thread_local char g_err[512];
+char* last_error_buf() { return g_err; }
+
+ftp_status fail(ftp_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+static bool valid_points(const int32_t* p, int32_t n, int32_t L) {
+    if (n < 1 || p[0] != 0) return false;
+    for (int32_t i = 0; i < n; ++i)
+        if (p[i] >= p[i + 1]) return false;
+    return L < 0 || p[n] == L;
+}
+
+}  // namespace ftp
+
+using namespace ftp;
+
+extern "C" const char* ftp_last_error(void) { return last_error_buf(); }
+
+extern "C" ftp_status ftp_estimate_capacity(const double* layer_times, int32_t L, const int32_t* points, int32_t N,
+                                            const double* stage_times, double* capacities) {
+    FTP_REQUIRE(layer_times && points && stage_times && capacities, FTP_EINVAL, "estimate_capacity: null argument");
+    FTP_REQUIRE(L >= 1 && N >= 1 && N <= L, FTP_EINVAL, "estimate_capacity: need 1 <= N <= L (N=%d, L=%d)", N, L);
+    FTP_REQUIRE(valid_points(points, N, L), FTP_EINVAL, "estimate_capacity: points must rise from 0 to L");
+    for (int32_t i = 0; i < N; ++i) {
+        double t0 = 0.0;                                   // Eq. 2: central node's time for stage i's layers
+        for (int32_t j = points[i]; j < points[i + 1]; ++j) t0 = t0 + layer_times[j];
+        FTP_REQUIRE(t0 > 0.0, FTP_ERANGE, "estimate_capacity: stage %d has zero profiled time", i);
+        capacities[i] = stage_times[i] / t0;               // Eq. 1
+    }
+    capacities[0] = 1.0;                                   // the central node is the unit of capacity
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_choose_partition(const double* layer_times, int32_t L, const double* capacities, int32_t N,
+                                           const double* out_bytes, const double* bandwidth, int32_t* points_out,
+                                           double* bottleneck_out) {
+    FTP_REQUIRE(layer_times && capacities && points_out, FTP_EINVAL, "choose_partition: null argument");
+    FTP_REQUIRE(L >= 1 && N >= 1, FTP_EINVAL, "choose_partition: L and N must be positive");
+    FTP_REQUIRE(N <= L, FTP_EINVAL, "choose_partition: %d stages cannot all be non-empty with %d units", N, L);
+    FTP_REQUIRE((out_bytes == nullptr) == (bandwidth == nullptr), FTP_EINVAL,
+                "choose_partition: out_bytes and bandwidth must be given together");
+    const bool comm = out_bytes != nullptr;
+    const double inf = std::numeric_limits<double>::infinity();
+    std::vector<double> S(L + 1, 0.0);                     // running sums of the per-layer times
+    for (int32_t j = 0; j < L; ++j) S[j + 1] = S[j] + layer_times[j];
+    // A[n][j]: least slowest-part time of units 0..j on the first n stages; cut[n][j]: the last cut
+    std::vector<double> A((size_t)(N + 1) * L, inf);
+    std::vector<int32_t> cut((size_t)(N + 1) * L, -1);
+    for (int32_t j = 0; j < L; ++j) A[(size_t)1 * L + j] = capacities[0] * (S[j + 1] - S[0]);   // Eq. 4 base case
+    for (int32_t n = 2; n <= N; ++n) {
+        for (int32_t j = n - 1; j < L; ++j) {
+            double best = inf;
+            int32_t arg = -1;
+            for (int32_t l = n - 2; l <= j - 1; ++l) {
+                const double sub = A[(size_t)(n - 1) * L + l];
+                const double link = comm ? 2.0 * (out_bytes[l] / bandwidth[n - 2]) : 0.0;   // 2 * T_c, Eq. 5
+                const double last = capacities[n - 1] * (S[j + 1] - S[l + 1]);              // Eq. 6 with Eq. 3
+                double v = sub > link ? sub : link;
+                v = v > last ? v : last;
+                if (v < best) { best = v; arg = l; }       // strict: the smallest optimal cut wins
+            }
+            A[(size_t)n * L + j] = best;
+            cut[(size_t)n * L + j] = arg;
+        }
+    }
+    points_out[N] = L;
+    int32_t j = L - 1;
+    for (int32_t n = N; n >= 2; --n) {
+        const int32_t l = cut[(size_t)n * L + j];
+        points_out[n - 1] = l + 1;
+        j = l;
+    }
+    points_out[0] = 0;
+    if (bottleneck_out) *bottleneck_out = A[(size_t)N * L + (L - 1)];
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_redistribution_plan(const int32_t* p_new, int32_t n_new, const int32_t* p_cur, int32_t n_cur,
+                                              int32_t i_fail, int32_t i_cur, int32_t i_new, int32_t* owner_of_needed,
+                                              int32_t* n_local) {
+    FTP_REQUIRE(p_new && p_cur && owner_of_needed, FTP_EINVAL, "redistribution_plan: null argument");
+    FTP_REQUIRE(n_new >= 1 && n_cur >= 1, FTP_EINVAL, "redistribution_plan: empty worker list");
+    FTP_REQUIRE(valid_points(p_new, n_new, -1) && valid_points(p_cur, n_cur, p_new[n_new]), FTP_EINVAL,
+                "redistribution_plan: both partitions must rise from 0 to the same L");
+    FTP_REQUIRE(i_new >= 0 && i_new < n_new && i_cur >= -1 && i_cur < n_cur && i_fail >= -1 && i_fail < n_cur,
+                FTP_ERANGE, "redistribution_plan: worker index out of range");
+    const int32_t held_lo = i_cur >= 0 ? p_cur[i_cur] : 0, held_hi = i_cur >= 0 ? p_cur[i_cur + 1] : 0;
+    int32_t local = 0;
+    for (int32_t l = p_new[i_new]; l < p_new[i_new + 1]; ++l) {
+        int32_t& out = owner_of_needed[l - p_new[i_new]];
+        if (l >= held_lo && l < held_hi) { out = -1; ++local; continue; }     // needed and not missing
+        int32_t target = 0;                                                    // holder under p_cur
+        while (!(p_cur[target] <= l && l < p_cur[target + 1])) ++target;
+        if (i_fail >= 0) {
+            if (target > i_fail) target -= 1;                                  // list was renumbered
+            else if (target == i_fail && i_fail == n_cur - 1) target = 0;      // last stage's replica: central node
+        }
+        out = target;
+    }
+    if (n_local) *n_local = local;
+    return FTP_OK;
+}

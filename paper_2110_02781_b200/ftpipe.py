@@ -1,0 +1,312 @@
+"""ctypes binding of libftpipe.so: argument marshalling only, one function per C entry point,
+same names.  Device buffers are torch tensors (torch provides device memory and streams);
+every step of the path runs inside the library's kernels.
+
+There is no fallback: importing this module without the built library raises.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libftpipe.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2110_02781_b200.build`")
+lib = C.CDLL(LIB_PATH)
+
+OK = 0
+STATUS = {0: "FTP_OK", 1: "FTP_EINVAL", 2: "FTP_ERANGE", 3: "FTP_ENOMEM", 4: "FTP_ECUDA", 5: "FTP_ESTATE",
+          6: "FTP_ETIMEOUT", 7: "FTP_EUNSUPPORTED"}
+T_WEIGHTS, T_GRADS, T_MOMENTUM, T_STATE = 0, 1, 2, 3
+FP32, BF16 = 0, 1
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("unit", "kind", "cin", "cout", "k", "stride", "pad", "act", "has_bias",
+                                          "residual_src")]
+
+
+class ModelCfg(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("batch", "in_c", "in_h", "in_w", "n_classes", "precision", "max_stages")] + \
+               [(n, C.c_float) for n in ("lr", "momentum", "weight_decay", "bn_eps", "bn_momentum")]
+
+
+class TraceRec(C.Structure):
+    _fields_ = [("kernel", C.c_int32), ("unit", C.c_int32), ("op", C.c_int32), ("backward", C.c_int32),
+                ("ms", C.c_float), ("bytes", C.c_double), ("flops", C.c_double)]
+
+
+class FtpError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__(f"{STATUS.get(status, status)}: {text}")
+        self.status = status
+
+
+_vp, _i32, _i64, _sz, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t, C.c_float
+_P = C.POINTER
+_SIGS = {
+    "ftp_workspace_bytes": [_P(LayerDesc), _i32, _P(ModelCfg), _P(_sz), _P(_sz)],
+    "ftp_build_model": [_P(LayerDesc), _i32, _P(ModelCfg), _vp, _sz, _vp, _sz, _P(_vp)],
+    "ftp_num_units": [_vp, _P(_i32)],
+    "ftp_unit_param_span": [_vp, _i32, _P(_i64), _P(_i64)],
+    "ftp_unit_state_span": [_vp, _i32, _P(_i64), _P(_i64)],
+    "ftp_unit_output_shape": [_vp, _i32, _P(_i32), _P(_i64)],
+    "ftp_set_tensor": [_vp, _i32, _i32, _vp, _i64, _i32, _vp],
+    "ftp_get_tensor": [_vp, _i32, _i32, _vp, _i64, _i32, _vp],
+    "ftp_run_stage_forward": [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp],
+    "ftp_run_stage_backward": [_vp, _i32, _i32, _vp, _vp, _vp],
+    "ftp_get_logits": [_vp, _vp, _i32, _vp],
+    "ftp_sgd_step": [_vp, _i32, _i32, _f32, _vp, _vp, _vp],
+    "ftp_train_step": [_vp, _vp, _vp, _i32, _f32, _P(_f32), _vp],
+    "ftp_profile_layers": [_vp, _i32, _vp, _vp, _P(C.c_double), _P(C.c_double), _P(_i64), _vp],
+    "ftp_estimate_capacity": [_P(C.c_double), _i32, _P(_i32), _i32, _P(C.c_double), _P(C.c_double)],
+    "ftp_choose_partition": [_P(C.c_double), _i32, _P(C.c_double), _i32, _P(C.c_double), _P(C.c_double), _P(_i32),
+                             _P(C.c_double)],
+    "ftp_redistribution_plan": [_P(_i32), _i32, _P(_i32), _i32, _i32, _i32, _i32, _P(_i32), _P(_i32)],
+    "ftp_set_partition": [_vp, _P(_i32), _i32, _P(_i32), _vp],
+    "ftp_get_partition": [_vp, _P(_i32), _P(_i32)],
+    "ftp_snapshot_weights": [_vp, _i32, _vp, _sz, _i32, _P(_sz), _vp],
+    "ftp_trace_enable": [_vp, _i32],
+    "ftp_trace_read": [_vp, _P(TraceRec), _i32, _P(_i32)],
+    "ftp_launch_count": [_vp, _P(_i64)],
+}
+for _name, _args in _SIGS.items():
+    _f = getattr(lib, _name)
+    _f.argtypes, _f.restype = _args, C.c_int
+lib.ftp_destroy_model.argtypes, lib.ftp_destroy_model.restype = [_vp], None
+lib.ftp_last_error.argtypes, lib.ftp_last_error.restype = [], C.c_char_p
+lib.ftp_kernel_name.argtypes, lib.ftp_kernel_name.restype = [_i32], C.c_char_p
+
+
+def _check(status):
+    if status != OK:
+        raise FtpError(status, lib.ftp_last_error().decode())
+
+
+def _ptr(t):
+    """Address of a torch tensor / numpy array / raw int, or NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _dbl(a):
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    return a, a.ctypes.data_as(_P(C.c_double))
+
+
+def _i32arr(a):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data_as(_P(_i32))
+
+
+def layer_array(layers):
+    arr = (LayerDesc * len(layers))()
+    for i, l in enumerate(layers):
+        arr[i] = LayerDesc(*[int(v) for v in l])
+    return arr
+
+
+def model_cfg(cfg):
+    return ModelCfg(cfg["batch"], cfg["in_c"], cfg["in_h"], cfg["in_w"], cfg["n_classes"], cfg["precision"],
+                    cfg["max_stages"], cfg["lr"], cfg["momentum"], cfg["weight_decay"], cfg["bn_eps"], cfg["bn_momentum"])
+
+
+# ---- pure host functions (usable without a GPU) ------------------------------------------------
+def ftp_estimate_capacity(layer_times, points, stage_times):
+    lt, plt = _dbl(layer_times)
+    pts, ppts = _i32arr(points)
+    stt, pst = _dbl(stage_times)
+    out = np.zeros(len(pts) - 1, np.float64)
+    _check(lib.ftp_estimate_capacity(plt, len(lt), ppts, len(pts) - 1, pst, out.ctypes.data_as(_P(C.c_double))))
+    return out.tolist()
+
+
+def ftp_choose_partition(layer_times, capacities, out_bytes=None, bandwidth=None):
+    lt, plt = _dbl(layer_times)
+    cp, pcp = _dbl(capacities)
+    ob = bw = pob = pbw = None
+    if out_bytes is not None:
+        ob, pob = _dbl(out_bytes)
+    if bandwidth is not None:
+        bw, pbw = _dbl(bandwidth)
+    pts = np.zeros(len(cp) + 1, np.int32)
+    bott = C.c_double()
+    _check(lib.ftp_choose_partition(plt, len(lt), pcp, len(cp), pob, pbw, pts.ctypes.data_as(_P(_i32)), C.byref(bott)))
+    return pts.tolist(), bott.value
+
+
+def ftp_redistribution_plan(p_new, p_cur, i_cur, i_new, i_fail=-1):
+    pn, ppn = _i32arr(p_new)
+    pc, ppc = _i32arr(p_cur)
+    if not (0 <= i_new < len(pn) - 1):
+        raise FtpError(2, "i_new out of range")
+    owners = np.full(max(int(pn[i_new + 1] - pn[i_new]), 1), -7, np.int32)
+    nloc = _i32()
+    _check(lib.ftp_redistribution_plan(ppn, len(pn) - 1, ppc, len(pc) - 1, i_fail, i_cur, i_new,
+                                       owners.ctypes.data_as(_P(_i32)), C.byref(nloc)))
+    return owners[:int(pn[i_new + 1] - pn[i_new])].tolist(), nloc.value
+
+
+def ftp_workspace_bytes(layers, cfg):
+    d, p = _sz(), _sz()
+    _check(lib.ftp_workspace_bytes(layer_array(layers), len(layers), C.byref(model_cfg(cfg)), C.byref(d), C.byref(p)))
+    return d.value, p.value
+
+
+def ftp_kernel_name(k):
+    return lib.ftp_kernel_name(k).decode()
+
+
+# ---- the model -----------------------------------------------------------------------------------
+class Model:
+    """Owns the workspaces (torch device memory + pinned host memory) and the ftp_model handle.
+    Methods are the C entry points with the handle bound."""
+
+    def __init__(self, layers, cfg, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.layers, self.cfg = list(layers), dict(cfg)
+        self.device = torch.device(device)
+        dev_bytes, pin_bytes = ftp_workspace_bytes(layers, cfg)
+        self.dev_ws = torch.empty(dev_bytes + 256, dtype=torch.uint8, device=self.device)
+        self.pin_ws = torch.empty(max(pin_bytes, 256), dtype=torch.uint8).pin_memory()
+        base = (self.dev_ws.data_ptr() + 255) // 256 * 256
+        h = _vp()
+        with torch.cuda.device(self.device):
+            _check(lib.ftp_build_model(layer_array(layers), len(layers), C.byref(model_cfg(cfg)), base, dev_bytes,
+                                       self.pin_ws.data_ptr(), self.pin_ws.numel(), C.byref(h)))
+        self.h = h
+        n = _i32()
+        _check(lib.ftp_num_units(self.h, C.byref(n)))
+        self.L = n.value
+        self.act_dtype = torch.bfloat16 if cfg["precision"] == BF16 else torch.float32
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.ftp_destroy_model(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def ftp_unit_param_span(self, unit):
+        o, c = _i64(), _i64()
+        _check(lib.ftp_unit_param_span(self.h, unit, C.byref(o), C.byref(c)))
+        return o.value, c.value
+
+    def ftp_unit_state_span(self, unit):
+        o, c = _i64(), _i64()
+        _check(lib.ftp_unit_state_span(self.h, unit, C.byref(o), C.byref(c)))
+        return o.value, c.value
+
+    def ftp_unit_output_shape(self, unit):
+        shp = (_i32 * 4)()
+        b = _i64()
+        _check(lib.ftp_unit_output_shape(self.h, unit, shp, C.byref(b)))
+        return tuple(shp), b.value
+
+    def ftp_set_tensor(self, which, unit, src, stream=None):
+        """src: float32 numpy array (host) or torch CUDA tensor (device)."""
+        dev = not isinstance(src, np.ndarray)
+        if not dev:
+            src = np.ascontiguousarray(src, dtype=np.float32)
+        n = src.size if not dev else src.numel()
+        _check(lib.ftp_set_tensor(self.h, which, unit, _ptr(src), n, int(dev), _stream(stream)))
+
+    def ftp_get_tensor(self, which, unit, stream=None):
+        """Returns a float32 numpy array (host copy)."""
+        n = self.ftp_unit_state_span(unit)[1] if which == T_STATE else self.ftp_unit_param_span(unit)[1]
+        out = np.empty(n, np.float32)
+        _check(lib.ftp_get_tensor(self.h, which, unit, _ptr(out), n, 0, _stream(stream)))
+        return out
+
+    def ftp_run_stage_forward(self, a, b, act_in, act_out=None, labels=None, loss_out=None, stream=None):
+        _check(lib.ftp_run_stage_forward(self.h, a, b, _ptr(act_in), _ptr(act_out), _ptr(labels), _ptr(loss_out),
+                                         _stream(stream)))
+
+    def ftp_run_stage_backward(self, a, b, grad_out=None, grad_in=None, stream=None):
+        _check(lib.ftp_run_stage_backward(self.h, a, b, _ptr(grad_out), _ptr(grad_in), _stream(stream)))
+
+    def ftp_get_logits(self, stream=None):
+        out = np.empty((self.cfg["batch"], self.cfg["n_classes"]), np.float32)
+        _check(lib.ftp_get_logits(self.h, _ptr(out), 0, _stream(stream)))
+        return out
+
+    def ftp_sgd_step(self, a, b, lr, snap_dev=None, snap_host=None, stream=None):
+        _check(lib.ftp_sgd_step(self.h, a, b, lr, _ptr(snap_dev), _ptr(snap_host), _stream(stream)))
+
+    def ftp_train_step(self, x, labels, lr, inputs_on_host=False, want_loss=True, stream=None):
+        loss = _f32()
+        _check(lib.ftp_train_step(self.h, _ptr(x), _ptr(labels), int(inputs_on_host), lr,
+                                  C.byref(loss) if want_loss else None, _stream(stream)))
+        return loss.value if want_loss else None
+
+    def ftp_profile_layers(self, reps, sample_in, labels, stream=None):
+        f, b = np.zeros(self.L), np.zeros(self.L)
+        ob = np.zeros(self.L, np.int64)
+        _check(lib.ftp_profile_layers(self.h, reps, _ptr(sample_in), _ptr(labels), f.ctypes.data_as(_P(C.c_double)),
+                                      b.ctypes.data_as(_P(C.c_double)), ob.ctypes.data_as(_P(_i64)), _stream(stream)))
+        return f, b, ob
+
+    def ftp_set_partition(self, points, stream=None):
+        pts, pp = _i32arr(points)
+        moved = _i32()
+        _check(lib.ftp_set_partition(self.h, pp, len(pts) - 1, C.byref(moved), _stream(stream)))
+        return moved.value
+
+    def ftp_get_partition(self):
+        pts = (_i32 * (self.cfg["max_stages"] + 1))()
+        n = _i32()
+        _check(lib.ftp_get_partition(self.h, pts, C.byref(n)))
+        return list(pts[:n.value + 1])
+
+    def ftp_snapshot_weights(self, stage, dst, stream=None):
+        """dst: torch tensor, device or pinned host (float32)."""
+        w = _sz()
+        _check(lib.ftp_snapshot_weights(self.h, stage, _ptr(dst), dst.numel() * dst.element_size(),
+                                        int(not dst.is_cuda), C.byref(w), _stream(stream)))
+        return w.value
+
+    def ftp_trace_enable(self, on):
+        _check(lib.ftp_trace_enable(self.h, int(on)))
+
+    def ftp_trace_read(self, max_records=65536):
+        buf = (TraceRec * max_records)()
+        n = _i32()
+        _check(lib.ftp_trace_read(self.h, buf, max_records, C.byref(n)))
+        return [dict(kernel=ftp_kernel_name(r.kernel), unit=r.unit, op=r.op, backward=r.backward, ms=r.ms,
+                     bytes=r.bytes, flops=r.flops) for r in buf[:min(n.value, max_records)]]
+
+    def ftp_launch_count(self):
+        n = _i64()
+        _check(lib.ftp_launch_count(self.h, C.byref(n)))
+        return n.value
+
+    # -- marshalling helpers (no arithmetic) --
+    def load_params(self, per_op_params, per_op_state=None):
+        """Scatter per-op float32 arrays (canonical order) into the unit tensors."""
+        for u in range(self.L):
+            parts = [a.reshape(-1) for l, arrs in zip(self.layers, per_op_params) if l.unit == u for a in arrs]
+            if parts:
+                self.ftp_set_tensor(T_WEIGHTS, u, np.concatenate(parts).astype(np.float32))
+            if per_op_state is not None:
+                parts = [a.reshape(-1) for l, arrs in zip(self.layers, per_op_state) if l.unit == u for a in arrs]
+                if parts:
+                    self.ftp_set_tensor(T_STATE, u, np.concatenate(parts).astype(np.float32))
+
+
+__all__ = ["Model", "FtpError", "LayerDesc", "ModelCfg", "TraceRec", "ftp_estimate_capacity", "ftp_choose_partition",
+           "ftp_redistribution_plan", "ftp_workspace_bytes", "ftp_kernel_name", "layer_array", "model_cfg", "lib",
+           "T_WEIGHTS", "T_GRADS", "T_MOMENTUM", "T_STATE", "FP32", "BF16", "LIB_PATH"]

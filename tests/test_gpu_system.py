@@ -1,0 +1,156 @@
+"""GPU tests of the scheduling side of the path: profile -> capacity -> partition, re-homing of
+weights (Algorithm 1 + commit), snapshots (bit-exact), the fused SGD+snapshot, error returns."""
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from helpers import gpu_step_split, make_gpu, make_oracle, rel_err, to_dev, TOL_FP32
+
+pytestmark = pytest.mark.gpu
+F = pytest.importorskip("paper_2110_02781_b200")
+
+
+def test_profile_then_partition_matches_oracle_choice():
+    import torch
+    ls, cfg = synth.mobilenetv2(16, 32, 10, 0, True)
+    gm = make_gpu(ls, cfg, 30)
+    x, y = synth.make_batch(30, cfg)
+    state0 = [gm.ftp_get_tensor(F.T_STATE, u) for u in range(gm.L)]
+    w0 = [gm.ftp_get_tensor(F.T_WEIGHTS, u) for u in range(gm.L)]
+    f, b, ob = gm.ftp_profile_layers(10, to_dev(x), to_dev(y))           # ten runs averaged (Sec. III-B)
+    assert np.all(f > 0) and np.all(b > 0)
+    for u in range(gm.L):                                                # profiling trains nothing
+        assert np.array_equal(state0[u], gm.ftp_get_tensor(F.T_STATE, u))
+        assert np.array_equal(w0[u], gm.ftp_get_tensor(F.T_WEIGHTS, u))
+        shp, nbytes = gm.ftp_unit_output_shape(u)
+        assert ob[u] == nbytes == (4 if u == gm.L - 1 else int(np.prod(shp)) * 4)
+    t = (f + b).tolist()
+    for caps in ([1.0, 1.0, 1.0], [1.0, 2.0, 5.0, 10.0]):
+        pts, bott = F.ftp_choose_partition(t, caps)
+        assert (pts, bott) == oracle.choose_partition(t, caps)           # same times in -> same points, exactly
+        # simulated devices: stage time = measured layer time x slowdown; Eq. 1-3 recovers the factors
+        stage = [caps[i] * sum(t[a:bb]) for i, (a, bb) in enumerate(zip(pts, pts[1:]))]
+        est = F.ftp_estimate_capacity(t, pts, stage)
+        assert est == oracle.estimate_capacity(t, pts, stage)
+        assert np.allclose(est[1:], caps[1:], rtol=1e-12)
+    gm.close()
+
+
+def test_repartition_moves_weights_and_training_continues_identically():
+    ls, cfg = synth.mobilenetv2(4, 16, 10, 0, True)
+    a, b = make_gpu(ls, cfg, 31), make_gpu(ls, cfg, 31)
+    x, y = synth.make_batch(31, cfg)
+    xd, yd = to_dev(x), to_dev(y)
+    b.ftp_set_partition([0, 5, 12, 20])
+    for m in (a, b):
+        m.ftp_train_step(xd, yd, 0.01)
+    cur, new = [0, 5, 12, 20], [0, 2, 15, 18, 20]
+    moved = b.ftp_set_partition(new)
+    # Algorithm 1: units whose owner changes = union of every stage's missing set
+    expect = 0
+    for i in range(len(new) - 1):
+        need, _ = oracle.redistribution_plan(new, cur, i if i < len(cur) - 1 else None, i)
+        expect += sum(len(v) for v in need.values())
+    assert moved == expect and b.ftp_get_partition() == new
+    for m in (a, b):
+        m.ftp_train_step(xd, yd, 0.01)
+    for u in range(a.L):
+        for which in (F.T_WEIGHTS, F.T_MOMENTUM, F.T_STATE):
+            assert np.array_equal(a.ftp_get_tensor(which, u), b.ftp_get_tensor(which, u))
+
+
+def test_snapshots_are_bit_exact_and_laid_out_like_the_oracle():
+    import torch
+    ls, cfg = synth.tiny_mbv2()
+    gm, om = make_gpu(ls, cfg, 32), make_oracle(ls, cfg, 32)
+    pts = [0, 2, 5, gm.L]
+    gm.ftp_set_partition(pts)
+    x, y = synth.make_batch(32, cfg)
+    gm.ftp_train_step(to_dev(x), to_dev(y), 0.01)
+    om.step(pts, x, y)
+    total = sum(gm.ftp_unit_param_span(u)[1] + gm.ftp_unit_state_span(u)[1] for u in range(gm.L))
+    central = torch.zeros(total, dtype=torch.float32).pin_memory()          # global replication target
+    off = 0
+    for s in range(3):
+        a, b = pts[s], pts[s + 1]
+        n = sum(gm.ftp_unit_param_span(u)[1] + gm.ftp_unit_state_span(u)[1] for u in range(a, b))
+        replica = torch.full((n + 8,), -7.0, device="cuda")                  # chain replication target
+        assert gm.ftp_snapshot_weights(s, replica) == 4 * n
+        assert gm.ftp_snapshot_weights(s, central[off:off + n]) == 4 * n
+        torch.cuda.synchronize()
+        live = np.concatenate([np.concatenate([gm.ftp_get_tensor(F.T_WEIGHTS, u), gm.ftp_get_tensor(F.T_STATE, u)])
+                               for u in range(a, b)])
+        got = replica.cpu().numpy()
+        assert np.array_equal(got[:n], live) and np.all(got[n:] == -7.0)     # bytes equal, nothing past the end
+        assert np.array_equal(central[off:off + n].numpy(), live)
+        assert rel_err(got[:n], om.snapshot(a, b)) <= TOL_FP32               # same layout as the oracle's replica
+        off += n
+    with pytest.raises(F.FtpError):
+        gm.ftp_snapshot_weights(0, torch.zeros(3, device="cuda"))            # too small: refused, nothing written
+    with pytest.raises(F.FtpError):
+        gm.ftp_snapshot_weights(3, central)
+
+
+def test_fused_sgd_snapshot_equals_separate_copy():
+    import torch
+    ls, cfg = synth.tiny_mbv2()
+    a, b = make_gpu(ls, cfg, 33), make_gpu(ls, cfg, 33)
+    x, y = synth.make_batch(33, cfg)
+    xd, yd = to_dev(x), to_dev(y)
+    L = a.L
+    n = sum(a.ftp_unit_param_span(u)[1] for u in range(L))
+    snap_dev = torch.zeros(n, device="cuda")
+    snap_host = torch.zeros(n).pin_memory()
+    for m in (a, b):
+        loss = torch.zeros(1, device="cuda")
+        m.ftp_run_stage_forward(0, L, xd, None, yd, loss)
+        m.ftp_run_stage_backward(0, L)
+    a.ftp_sgd_step(0, L, 0.01)
+    b.ftp_sgd_step(0, L, 0.01, snap_dev, snap_host)
+    torch.cuda.synchronize()
+    live = np.concatenate([a.ftp_get_tensor(F.T_WEIGHTS, u) for u in range(L)])
+    assert np.array_equal(live, np.concatenate([b.ftp_get_tensor(F.T_WEIGHTS, u) for u in range(L)]))
+    assert np.array_equal(snap_dev.cpu().numpy(), live) and np.array_equal(snap_host.numpy(), live)
+
+
+def test_errors_are_returned_before_any_launch():
+    import torch
+    ls, cfg = synth.tiny_mbv2()
+    gm = make_gpu(ls, cfg, 34)
+    x, y = synth.make_batch(34, cfg)
+    xd, yd = to_dev(x), to_dev(y)
+    loss = torch.zeros(1, device="cuda")
+    before = gm.ftp_launch_count()
+    for call in (lambda: gm.ftp_run_stage_forward(3, 3, xd, None, yd, loss),            # empty range
+                 lambda: gm.ftp_run_stage_forward(0, gm.L + 1, xd, None, yd, loss),
+                 lambda: gm.ftp_run_stage_forward(0, gm.L, xd, None, None, loss),       # labels missing
+                 lambda: gm.ftp_run_stage_forward(0, 2, xd, None),                      # act_out missing
+                 lambda: gm.ftp_run_stage_backward(0, gm.L),                            # backward before forward
+                 lambda: gm.ftp_set_partition([0, 3, 3, gm.L]),                         # empty stage
+                 lambda: gm.ftp_set_partition(list(range(gm.L + 1)) ),                  # more stages than max_stages
+                 lambda: gm.ftp_set_tensor(F.T_WEIGHTS, 0, np.zeros(3, np.float32)),    # wrong size
+                 lambda: gm.ftp_get_tensor(F.T_WEIGHTS, gm.L)):
+        with pytest.raises(F.FtpError):
+            call()
+    assert gm.ftp_launch_count() == before
+    gm.ftp_run_stage_forward(0, gm.L, xd, None, yd, loss)                               # and the model still works
+    gm.ftp_run_stage_backward(0, gm.L)
+    torch.cuda.synchronize()
+    assert np.isfinite(loss.item())
+
+
+def test_trace_records_every_launch_with_its_algorithmic_work():
+    ls, cfg = synth.tiny_mbv2()
+    gm = make_gpu(ls, cfg, 35)
+    x, y = synth.make_batch(35, cfg)
+    gm.ftp_trace_enable(True)
+    n0 = gm.ftp_launch_count()
+    gm.ftp_train_step(to_dev(x), to_dev(y), 0.01)
+    recs = gm.ftp_trace_read()
+    gm.ftp_trace_enable(False)
+    assert len(recs) > 50 and all(r["ms"] > 0 for r in recs if r["kernel"] != "copy")
+    names = {r["kernel"] for r in recs}
+    assert {"conv_fwd_f32", "conv_dgrad_f32", "conv_wgrad_f32", "bn_stats", "bn_apply", "bn_bwd_reduce", "bn_bwd_apply",
+            "dw_fwd", "dw_dgrad", "dw_wgrad", "gap_fwd", "softmax_ce", "sgd"} <= names
+    assert gm.ftp_launch_count() - n0 >= len(recs)
