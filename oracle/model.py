@@ -125,6 +125,65 @@ class OracleModel:
                 acc(i - 1, ops.gap_bwd(d, x.shape))
         return grad.get(idx[0] - 1)
 
+    # ---- how close the last forward came to a discrete decision ---------------------------------
+    def decision_margin(self, a=0, b=None, per_op=False):
+        """Smallest gap, over units [a, b) of the last forward, between a value and a point where
+        the path takes a discrete decision: an activation kink (0, and 6 for ReLU6) or a tie
+        between the two largest entries of a max-pool window.  Each gap is relative to the
+        largest magnitude in its tensor.  At such a point float32 and float64 arithmetic may
+        decide differently and the gradient jumps, so parity inputs are drawn with this margin
+        above the float32 rounding noise; what is compared is then unique."""
+        worst = np.inf
+        each = []
+        for i in self.ops_of(a, self.L if b is None else b):
+            l = self.layers[i]
+            if l.kind == MAXPOOL:
+                x = self.out[i - 1]
+                n, h, w, c = x.shape
+                ho, wo = h // 2, w // 2
+                win = np.sort(np.stack([x[:, p:2 * ho:2, q:2 * wo:2] for p in (0, 1) for q in (0, 1)]), axis=0)
+                gap = win[3] - win[2]
+                # a tie between values clamped by the preceding activation routes no gradient either way
+                prev = self.layers[i - 1].act if i > 0 else 0
+                harmless = (gap == 0) & ((win[3] == 0.0) if prev else False)
+                if prev == 2:
+                    harmless |= (gap == 0) & (win[3] == 6.0)
+                gap = np.where(harmless, np.inf, gap)
+                each.append((i, float(gap.min() / max(np.abs(x).max(), 1e-300))))
+                worst = min(worst, each[-1][1])
+                continue
+            if l.act == 0 or l.kind == CE:
+                continue
+            if l.kind in (CONV1D, CONV2D, FC):
+                z = self.saved[i]
+            elif l.kind == BN:
+                z = self.saved[i][0]
+            else:
+                z = self.out[i - 1]
+            gap = np.abs(z).min()
+            if l.act == 2:
+                gap = min(gap, np.abs(z - 6.0).min())
+            each.append((i, float(gap / max(np.abs(z).max(), 1e-300))))
+            worst = min(worst, each[-1][1])
+        return each if per_op else worst
+
+    def ambiguous_outputs(self, i, margin):
+        """Boolean mask over op i's output: True where its own discrete decision (activation kink,
+        max-pool tie) lies within `margin` (relative to the tensor's largest magnitude)."""
+        l = self.layers[i]
+        if l.kind == MAXPOOL:
+            x = self.out[i - 1]
+            ho, wo = x.shape[1] // 2, x.shape[2] // 2
+            win = np.sort(np.stack([x[:, p:2 * ho:2, q:2 * wo:2] for p in (0, 1) for q in (0, 1)]), axis=0)
+            return (win[3] - win[2]) <= margin * np.abs(x).max()
+        z = self.saved[i] if l.kind in (CONV1D, CONV2D, FC) else (self.saved[i][0] if l.kind == BN else self.out[i - 1])
+        if l.act == 0:
+            return np.zeros(z.shape, bool)
+        near = np.abs(z) <= margin * np.abs(z).max()
+        if l.act == 2:
+            near |= np.abs(z - 6.0) <= margin * np.abs(z).max()
+        return near
+
     # ---- SGD on units [a, b) (Sec. IV-B: momentum 0.9, weight decay 4e-5) --------------------
     def sgd(self, a, b, lr=None):
         """g <- g + wd*w ; m <- g on the first update, else mu*m + g ; w <- w - lr*m."""

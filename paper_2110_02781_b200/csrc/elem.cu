@@ -72,6 +72,12 @@ __device__ __forceinline__ bool act_pass(float z, int act) {      // derivative 
     return true;
 }
 
+// Normalised value: the mean is a two-float sum and is subtracted first, so that the result keeps
+// float accuracy relative to its own size even when the mean dwarfs the spread.
+__device__ __forceinline__ float bn_z(float y, float mh, float ml, float scale, float beta) {
+    return fmaf((y - mh) - ml, scale, beta);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline unsigned flat_blocks(long long work, int threads) {
     long long b = (work + threads - 1) / threads;
@@ -139,7 +145,7 @@ __global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, 
 
 __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
-                                   float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* rstd) {
+                                   float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd) {
     const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (c >= C) return;
     const double s1 = warp_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
@@ -151,8 +157,10 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
         const double rs = 1.0 / sqrt(var + (double)eps);
         const float sc = (float)((double)gamma[c] * rs);
         scale[c] = sc;
-        shift[c] = (float)((double)beta[c] - mu * (double)gamma[c] * rs);
-        mean[c] = (float)mu;
+        shift[c] = beta[c];                       // z = (y - mean) * scale + beta, the mean kept as a two-float sum
+        const float mh = (float)mu;
+        mean[c] = mh;
+        mean_lo[c] = (float)(mu - (double)mh);
         rstd[c] = (float)rs;
         const double unb = M > 1.0 ? var * M / (M - 1.0) : var;
         run_mean[c] = (float)((1.0 - (double)mom) * (double)run_mean[c] + (double)mom * mu);
@@ -163,15 +171,18 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
 template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ y, const T* __restrict__ res, T* __restrict__ z,
                                                        long long nvec, int C, const float* __restrict__ scale,
-                                                       const float* __restrict__ shift, int act) {
+                                                       const float* __restrict__ shift, const float* __restrict__ mean,
+                                                       const float* __restrict__ mean_lo, int act) {
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)((i * V) % C);
-        float v[V], sc[V], sh[V];
+        float v[V], sc[V], sh[V], mu[V], ml[V];
         ldv<V>(y + i * V, v);
         ldtab<V>(scale + c, sc);
         ldtab<V>(shift + c, sh);
+        ldtab<V>(mean + c, mu);
+        ldtab<V>(mean_lo + c, ml);
 #pragma unroll
-        for (int e = 0; e < V; ++e) v[e] = act_f(fmaf(v[e], sc[e], sh[e]), act);
+        for (int e = 0; e < V; ++e) v[e] = act_f(bn_z(v[e], mu[e], ml[e], sc[e], sh[e]), act);
         if (res) {
             float r[V];
             ldv<V>(res + i * V, r);
@@ -185,20 +196,20 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ y, 
 template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict__ dz, const T* __restrict__ y, int rows, int cols, int rpc, int C,
                                                             const float* __restrict__ scale, const float* __restrict__ shift,
-                                                            const float* __restrict__ mean, const float* __restrict__ rstd, int act,
-                                                            double* __restrict__ partial) {
+                                                            const float* __restrict__ mean, const float* __restrict__ mean_lo,
+                                                            const float* __restrict__ rstd, int act, double* __restrict__ partial) {
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
-    float sc[V], sh[V], mu[V], rs[V];
-    if (col < cols) { const int c = col % C; ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(rstd + c, rs); }
+    float sc[V], sh[V], mu[V], ml[V], rs[V];
+    if (col < cols) { const int c = col % C; ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml); ldtab<V>(rstd + c, rs); }
     fold_reduce<T, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
         float d[V], v[V];
         ldv<V>(dz + off, d);
         ldv<V>(y + off, v);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
-            const float g = act_pass(fmaf(v[e], sc[e], sh[e]), act) ? d[e] : 0.f;
+            const float g = act_pass(bn_z(v[e], mu[e], ml[e], sc[e], sh[e]), act) ? d[e] : 0.f;
             s[0][e] += g;
-            s[1][e] = fmaf(g, (v[e] - mu[e]) * rs[e], s[1][e]);
+            s[1][e] = fmaf(g, ((v[e] - mu[e]) - ml[e]) * rs[e], s[1][e]);
         }
     });
 }
@@ -214,8 +225,10 @@ __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int c
         dbeta[c] = (float)s1;
         dgamma[c] = (float)s2;
         coef[c] = gamma[c] * rstd[c];
-        coef[C + c] = (float)(s1 / M);
-        coef[2 * C + c] = (float)(s2 / M);
+        const double b = s1 / M, cc = s2 / M;      // kept as two-float sums: they are subtracted from values of their own size
+        const float bh = (float)b, ch = (float)cc;
+        coef[C + c] = bh; coef[2 * C + c] = (float)(b - (double)bh);
+        coef[3 * C + c] = ch; coef[4 * C + c] = (float)(cc - (double)ch);
     }
 }
 
@@ -223,18 +236,25 @@ template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dz, const T* __restrict__ y, const T* __restrict__ addend,
                                                            T* __restrict__ dy, long long nvec, int C, const float* __restrict__ scale,
                                                            const float* __restrict__ shift, const float* __restrict__ mean,
-                                                           const float* __restrict__ rstd, const float* __restrict__ coef, int act) {
+                                                           const float* __restrict__ mean_lo, const float* __restrict__ rstd,
+                                                           const float* __restrict__ coef, int act) {
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)((i * V) % C);
-        float d[V], v[V], sc[V], sh[V], mu[V], rs[V], ca[V], cb[V], cc[V], o[V];
+        float d[V], v[V], sc[V], sh[V], mu[V], ml[V], rs[V], ca[V], bh[V], bl[V], ch[V], cl[V], o[V];
         ldv<V>(dz + i * V, d);
         ldv<V>(y + i * V, v);
-        ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(rstd + c, rs);
-        ldtab<V>(coef + c, ca); ldtab<V>(coef + C + c, cb); ldtab<V>(coef + 2 * C + c, cc);
+        ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml); ldtab<V>(rstd + c, rs);
+        ldtab<V>(coef + c, ca); ldtab<V>(coef + C + c, bh); ldtab<V>(coef + 2 * C + c, bl);
+        ldtab<V>(coef + 3 * C + c, ch); ldtab<V>(coef + 4 * C + c, cl);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
-            const float g = act_pass(fmaf(v[e], sc[e], sh[e]), act) ? d[e] : 0.f;
-            o[e] = ca[e] * (g - cb[e] - (v[e] - mu[e]) * rs[e] * cc[e]);
+            const float cen = (v[e] - mu[e]) - ml[e];
+            const float g = act_pass(fmaf(cen, sc[e], sh[e]), act) ? d[e] : 0.f;
+            const float xh = cen * rs[e];
+            float t = (g - bh[e]) - bl[e];
+            t = fmaf(-xh, ch[e], t);
+            t = fmaf(-xh, cl[e], t);
+            o[e] = ca[e] * t;
         }
         if (addend) {
             float a[V];
@@ -658,31 +678,31 @@ void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partia
 
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
-                 float* rstd, cudaStream_t st) {
+                 float* mean_lo, float* rstd, cudaStream_t st) {
     bn_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
-                                                             run_mean, run_var, scale, shift, mean, rstd);
+                                                             run_mean, run_var, scale, shift, mean, mean_lo, rstd);
 }
 
 template <typename T>
-void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift, int act,
-              cudaStream_t st) {
+void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift,
+              const float* mean, const float* mean_lo, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     const long long n = M * C;
-    if (can_vec<T>(C, y, residual, z) && aligned16(scale) && aligned16(shift))
-        bn_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(y, residual, z, n / V, C, scale, shift, act);
+    if (can_vec<T>(C, y, residual, z) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo))
+        bn_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(y, residual, z, n / V, C, scale, shift, mean, mean_lo, act);
     else
-        bn_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(y, residual, z, n, C, scale, shift, act);
+        bn_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(y, residual, z, n, C, scale, shift, mean, mean_lo, act);
 }
 
 template <typename T>
 void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
-                   const float* mean, const float* rstd, int act, double* partial, cudaStream_t st) {
+                   const float* mean, const float* mean_lo, const float* rstd, int act, double* partial, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(rstd))
-        bn_bwd_reduce_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, rstd, act, partial);
+    if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd))
+        bn_bwd_reduce_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial);
     else {
         FoldPlan s = fp;                       // scalar fallback keeps the same partial layout
-        bn_bwd_reduce_kernel<T, 1><<<dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st>>>(dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, rstd, act, partial);
+        bn_bwd_reduce_kernel<T, 1><<<dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st>>>(dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, mean_lo, rstd, act, partial);
     }
 }
 
@@ -693,13 +713,13 @@ void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int
 
 template <typename T>
 void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale, const float* shift,
-                  const float* mean, const float* rstd, const float* coef, int act, cudaStream_t st) {
+                  const float* mean, const float* mean_lo, const float* rstd, const float* coef, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     const long long n = M * C;
-    if (can_vec<T>(C, dz, y, addend, dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(rstd) && aligned16(coef))
-        bn_bwd_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(dz, y, addend, dy, n / V, C, scale, shift, mean, rstd, coef, act);
+    if (can_vec<T>(C, dz, y, addend, dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd) && aligned16(coef))
+        bn_bwd_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(dz, y, addend, dy, n / V, C, scale, shift, mean, mean_lo, rstd, coef, act);
     else
-        bn_bwd_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(dz, y, addend, dy, n, C, scale, shift, mean, rstd, coef, act);
+        bn_bwd_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(dz, y, addend, dy, n, C, scale, shift, mean, mean_lo, rstd, coef, act);
 }
 
 template <typename T>
@@ -825,11 +845,12 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
 
 #define FTP_INSTANTIATE(T)                                                                                              \
     template void bn_stats<T>(const T*, long long, int, const FoldPlan&, double*, cudaStream_t);                          \
-    template void bn_apply<T>(const T*, const T*, T*, long long, int, const float*, const float*, int, cudaStream_t);       \
+    template void bn_apply<T>(const T*, const T*, T*, long long, int, const float*, const float*, const float*,             \
+                              const float*, int, cudaStream_t);                                                            \
     template void bn_bwd_reduce<T>(const T*, const T*, long long, int, const FoldPlan&, const float*, const float*,         \
-                                   const float*, const float*, int, double*, cudaStream_t);                                \
+                                   const float*, const float*, const float*, int, double*, cudaStream_t);                  \
     template void bn_bwd_apply<T>(const T*, const T*, const T*, T*, long long, int, const float*, const float*,             \
-                                  const float*, const float*, const float*, int, cudaStream_t);                            \
+                                  const float*, const float*, const float*, const float*, int, cudaStream_t);              \
     template void act_bias_bwd<T>(const T*, const T*, T*, long long, int, int, const FoldPlan&, double*, float*,            \
                                   cudaStream_t);                                                                           \
     template void act_fwd<T>(const T*, T*, long long, int, cudaStream_t);                                                   \

@@ -41,25 +41,27 @@ size_t fold_partial_doubles(const FoldPlan& fp);     // doubles needed for the p
 
 template <typename T>
 void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st);
-// mean/var -> scale, shift, saved mean, rstd; running statistics update (momentum, unbiased variance)
+// mean/var -> scale (gamma * rstd), shift (a copy of beta), the mean as a two-float sum (mean + mean_lo),
+// rstd; running statistics update (momentum, unbiased variance).  z = ((y - mean) - mean_lo) * scale + shift.
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
                  const float* beta, float eps, float momentum, float* run_mean, float* run_var, float* scale,
-                 float* shift, float* mean, float* rstd, cudaStream_t st);
+                 float* shift, float* mean, float* mean_lo, float* rstd, cudaStream_t st);
 template <typename T>
 void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift,
-              int act, cudaStream_t st);
+              const float* mean, const float* mean_lo, int act, cudaStream_t st);
 // pass 1 of BN backward: sums of dz' and dz'*xhat with dz' = dz masked by the activation
 template <typename T>
 void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale,
-                   const float* shift, const float* mean, const float* rstd, int act, double* partial,
-                   cudaStream_t st);
-// -> dgamma, dbeta and the per-channel coefficients (a = gamma*rstd, b = dbeta/M, c = dgamma/M)
+                   const float* shift, const float* mean, const float* mean_lo, const float* rstd, int act,
+                   double* partial, cudaStream_t st);
+// -> dgamma, dbeta and the per-channel coefficients coef[5][C]: a = gamma*rstd, then b = dbeta/M and
+// c = dgamma/M each as a two-float sum (hi, lo)
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
                      const float* rstd, float* dgamma, float* dbeta, float* coef, cudaStream_t st);
 template <typename T>
 void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale,
-                  const float* shift, const float* mean, const float* rstd, const float* coef, int act,
-                  cudaStream_t st);
+                  const float* shift, const float* mean, const float* mean_lo, const float* rstd, const float* coef,
+                  int act, cudaStream_t st);
 
 // Backward of "act(pre + bias)": dpre = dout masked by the stored output; dbias = column sums.
 // dpre may be NULL when act == 0 (then dpre == dout); dbias may be NULL.

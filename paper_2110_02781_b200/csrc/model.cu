@@ -222,9 +222,10 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         if (!o.out_f32 && i + 1 < n) max_act = std::max(max_act, obytes);
         const long long Mout = (long long)o.N * o.Ho * o.Wo;
         if (o.d.kind == FTP_BN) {
-            float* t = (float*)bp.take((size_t)o.C * 7 * 4 + 256 * 7);
             const size_t stride = align_up((size_t)o.C * 4, 256) / 4;
-            o.scale = t; o.shift = t + stride; o.mean = t + 2 * stride; o.rstd = t + 3 * stride; o.coef = t + 4 * stride;
+            float* t = (float*)bp.take((5 * stride + 5 * (size_t)o.C) * 4);
+            o.scale = t; o.shift = t + stride; o.mean = t + 2 * stride; o.mean_lo = t + 3 * stride; o.rstd = t + 4 * stride;
+            o.coef = t + 5 * stride;
             o.fold = make_fold(Mout, o.C, m.esize);
             foldd = std::max(foldd, fold_partial_doubles(o.fold));
         } else if (is_contraction(o.d.kind)) {
@@ -308,11 +309,11 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                   bn_stats<T>((const T*)in, Mr, o.C, o.fold, m->fold_scratch, st); }
                 { Scope sc(m, st, K_BN_FINALIZE, u, i, 0, fold_partial_doubles(o.fold) * 8.0, 0.0);
                   bn_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, ar.w + o.b_off, m->cfg.bn_eps, m->cfg.bn_momentum,
-                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.rstd, st); }
+                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, st); }
                 const void* res = nullptr;
                 if (o.fused_add) { const int s = m->ops[i + 1].d.residual_src; res = s < first ? act_in : m->cur_out[s]; }
                 { Scope sc(m, st, K_BN_APPLY, u, i, 0, (o.in_elems * (res ? 3.0 : 2.0)) * es, 2.0 * o.in_elems);
-                  bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.scale, o.shift, o.d.act, st); }
+                  bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.scale, o.shift, o.mean, o.mean_lo, o.d.act, st); }
                 break;
             }
             case FTP_ACT: {
@@ -407,12 +408,12 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
             case FTP_BN: {
                 const long long Mr = (long long)o.N * o.H * o.W;
                 { Scope sc(m, st, K_BN_BWD_REDUCE, u, i, 1, 2.0 * o.in_elems * es, 8.0 * o.in_elems);
-                  bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.rstd, o.d.act, m->fold_scratch, st); }
+                  bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.d.act, m->fold_scratch, st); }
                 { Scope sc(m, st, K_BN_BWD_FINALIZE, u, i, 1, fold_partial_doubles(o.fold) * 8.0, 0.0);
                   bn_bwd_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, st); }
                 if (gi) {
                     Scope sc(m, st, K_BN_BWD_APPLY, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, 8.0 * o.in_elems);
-                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.scale, o.shift, o.mean, o.rstd, o.coef, o.d.act, st);
+                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef, o.d.act, st);
                 }
                 break;
             }

