@@ -230,6 +230,29 @@ const char* ftp_kernel_name(int32_t kernel);
 /* Number of kernel launches issued by this model since it was built. */
 ftp_status ftp_launch_count(const ftp_model* m, int64_t* launches);
 
+/* ---- for callers that cannot allocate ------------------------------------------------------------
+ * (The paper has no counterpart: this is a packaging variant of the weight-gradient step of
+ * run_stage's backward pass.)
+ *
+ * dw[k][k][cin][cout] = sum over output pixels of x (shifted by the tap) times dy, for a dense
+ * k x k convolution with the given stride and padding on float tensors x (n, h, w, cin) and
+ * dy (n, ho, wo, cout), all device pointers, 16-byte alignment recommended.
+ *
+ * Unlike every other call, this one takes no workspace: the partial sums of its split reduction go
+ * to an 8 MiB array that is part of the library's device image (each GPU that loads the library
+ * holds it until the process exits).  It is meant for callers that get input and output buffers
+ * and may not call cudaMalloc themselves: a stage running inside a stream-ordered region where an
+ * allocation would stall the device, or a host framework that owns all device memory.  The call
+ * itself allocates nothing, on the host or on the device.
+ *   - Shapes whose partials exceed the array are refused with FTP_ERANGE (use the model API).
+ *   - The first call on a device looks the array's address up (the device must be current); make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the array: calls whose kernels may overlap on the GPU (different
+ *     streams) race on it.  Nothing needs clearing between calls.
+ * Asynchronous on the stream. */
+ftp_status ftp_conv_wgrad_static(const float* x, const float* dy, float* dw, int32_t n, int32_t h, int32_t w,
+                                 int32_t cin, int32_t cout, int32_t k, int32_t stride, int32_t pad, void* stream);
+
 const char* ftp_last_error(void);
 
 #ifdef __cplusplus

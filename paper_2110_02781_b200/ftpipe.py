@@ -70,6 +70,7 @@ _SIGS = {
     "ftp_trace_enable": [_vp, _i32],
     "ftp_trace_read": [_vp, _P(TraceRec), _i32, _P(_i32)],
     "ftp_launch_count": [_vp, _P(_i64)],
+    "ftp_conv_wgrad_static": [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _vp],
 }
 for _name, _args in _SIGS.items():
     _f = getattr(lib, _name)
@@ -164,6 +165,15 @@ def ftp_workspace_bytes(layers, cfg):
     d, p = _sz(), _sz()
     _check(lib.ftp_workspace_bytes(layer_array(layers), len(layers), C.byref(model_cfg(cfg)), C.byref(d), C.byref(p)))
     return d.value, p.value
+
+
+def ftp_conv_wgrad_static(x, dy, dw, k, stride, pad, stream=None):
+    """Weight gradient of a dense k x k convolution without any workspace argument, for callers that
+    may not allocate device memory: x (n, h, w, cin), dy (n, ho, wo, cout) and dw (k, k, cin, cout)
+    are float32 CUDA tensors the caller already owns.  See include/ftpipe.h for the limits."""
+    n, h, w, cin = x.shape
+    _check(lib.ftp_conv_wgrad_static(_ptr(x), _ptr(dy), _ptr(dw), n, h, w, cin, dy.shape[3], k, stride, pad,
+                                     _stream(stream)))
 
 
 def ftp_kernel_name(k):
@@ -308,5 +318,5 @@ class Model:
 
 
 __all__ = ["Model", "FtpError", "LayerDesc", "ModelCfg", "TraceRec", "ftp_estimate_capacity", "ftp_choose_partition",
-           "ftp_redistribution_plan", "ftp_workspace_bytes", "ftp_kernel_name", "layer_array", "model_cfg", "lib",
+           "ftp_redistribution_plan", "ftp_workspace_bytes", "ftp_kernel_name", "ftp_conv_wgrad_static", "layer_array", "model_cfg", "lib",
            "T_WEIGHTS", "T_GRADS", "T_MOMENTUM", "T_STATE", "FP32", "BF16", "LIB_PATH"]
