@@ -26,14 +26,14 @@ FP32_ALU_PEAK_TFLOPS = 2 * 128 * 148 * 1.965e9 / 1e12      # FMA lanes x SMs x m
 FALLBACK_HBM_GBS = 6650.0
 
 
-def workload(name):
+def workload(name, batch=None):
     import synth
     if name == "cfg1":
         ls, cfg = synth.har_cnn()
         return dict(index=0, name="config 1: HAR 1D-CNN 32x9x128 fp32, 2 stages split after layer 2", layers=ls, cfg=cfg,
                     caps=None, points=[0, 2, 5])
-    ls, cfg = synth.mobilenetv2(128, 32, 10, 0, True)
-    return dict(index=1, name="config 2: MobileNetV2 32x32x3 batch 128 fp32, 3 stages at equal capacity", layers=ls,
+    ls, cfg = synth.mobilenetv2(batch or 128, 32, 10, 0, True)
+    return dict(index=1, name=f"config 2: MobileNetV2 32x32x3 batch {batch or 128} fp32, 3 stages at equal capacity", layers=ls,
                 cfg=cfg, caps=[1.0, 1.0, 1.0], points=None)
 
 
@@ -125,11 +125,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    wl = workload(args.workload)
+    wl = workload(args.workload, args.batch)
 
     if args.impl == "reference":
         if rank != 0:

@@ -119,18 +119,26 @@ __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chu
     }
 }
 
-// Sum over chunks and folded copies for channel c, by one warp, fixed order.  Result valid in lane 0.
-__device__ __forceinline__ double warp_fold_sum(const double* partial, int which, int ns, int chunks, int f, int C, int cols, int c) {
-    const int lane = threadIdx.x & 31;
+// Sum over chunks and folded copies for channel c, by one block of FIN_T threads, in a fixed order:
+// strided per-thread runs, then a shared-memory tree.  The result is valid in thread 0.
+constexpr int FIN_T = 128;
+__device__ __forceinline__ double block_fold_sum(const double* partial, int which, int ns, int chunks, int f, int C, int cols, int c) {
+    __shared__ double red[FIN_T];
     double t = 0.0;
     const int total = chunks * f;
-    for (int e = lane; e < total; e += 32) {
+    for (int e = threadIdx.x; e < total; e += FIN_T) {
         const int ch = e / f, k = e - ch * f;
         t += partial[((long long)ch * ns + which) * cols + k * C + c];
     }
+    __syncthreads();
+    red[threadIdx.x] = t;
+    __syncthreads();
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
-    return t;
+    for (int o = FIN_T / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    return red[0];
 }
 
 template <typename T, int V>
@@ -146,11 +154,10 @@ __global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, 
 __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
                                    float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd) {
-    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (c >= C) return;
-    const double s1 = warp_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
-    const double s2 = warp_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
-    if ((threadIdx.x & 31) == 0) {
+    const int c = blockIdx.x;
+    const double s1 = block_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
+    const double s2 = block_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
+    if (threadIdx.x == 0) {
         const double mu = s1 / M;
         double var = s2 / M - mu * mu;
         if (var < 0.0) var = 0.0;
@@ -217,11 +224,10 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
 __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                        const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
                                        float* dbeta, float* coef) {
-    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (c >= C) return;
-    const double s1 = warp_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
-    const double s2 = warp_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
-    if ((threadIdx.x & 31) == 0) {
+    const int c = blockIdx.x;
+    const double s1 = block_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
+    const double s2 = block_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
+    if (threadIdx.x == 0) {
         dbeta[c] = (float)s1;
         dgamma[c] = (float)s2;
         coef[c] = gamma[c] * rstd[c];
@@ -285,10 +291,9 @@ __global__ void __launch_bounds__(256) act_bias_bwd_kernel(const T* __restrict__
 }
 
 __global__ void colsum_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, float* out) {
-    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (c >= C) return;
-    const double s = warp_fold_sum(partial, 0, 1, chunks, f, C, cols, c);
-    if ((threadIdx.x & 31) == 0) out[c] = (float)s;
+    const int c = blockIdx.x;
+    const double s = block_fold_sum(partial, 0, 1, chunks, f, C, cols, c);
+    if (threadIdx.x == 0) out[c] = (float)s;
 }
 
 template <typename T, int V>
@@ -679,7 +684,7 @@ void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partia
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
                  float* mean_lo, float* rstd, cudaStream_t st) {
-    bn_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
+    bn_finalize_kernel<<<C, FIN_T, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
                                                              run_mean, run_var, scale, shift, mean, mean_lo, rstd);
 }
 
@@ -708,7 +713,7 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
 
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
                      float* dgamma, float* dbeta, float* coef, cudaStream_t st) {
-    bn_bwd_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef);
+    bn_bwd_finalize_kernel<<<C, FIN_T, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef);
 }
 
 template <typename T>
@@ -730,7 +735,7 @@ void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int 
         act_bias_bwd_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
     else
         act_bias_bwd_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
-    if (dbias) colsum_finalize_kernel<<<(C * 32 + 255) / 256, 256, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias);
+    if (dbias) colsum_finalize_kernel<<<C, FIN_T, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias);
 }
 
 template <typename T>

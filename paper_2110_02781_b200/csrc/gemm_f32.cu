@@ -13,7 +13,7 @@
 namespace ftp {
 namespace {
 
-constexpr int BM = 128, BK = 16, NT = 256;
+constexpr int BK = 16, NT = 256;
 
 struct GemmP {
     const float* A;        // gathered operand: x (forward) or dy (data gradient)
@@ -68,9 +68,11 @@ __device__ __forceinline__ float apply_act(float v, int act) {
     return v;
 }
 
-template <int BN, int MODE>
+template <int BM, int BN, int MODE>
 __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
-    constexpr int TN = BN / 16;
+    constexpr int TM = BM / 16, TN = BN / 16;
+    constexpr int ITA = BM / 64;                   // float4 loads of A per thread (vector path)
+    static_assert(BM == 128 || BM == 64, "row tile");
     constexpr int LDA = BM + 4, LDB = BN + 4;
     constexpr int NB4 = BK * BN / 4;               // float4 slots of a B tile
     constexpr int ITB = (NB4 + NT - 1) / NT;
@@ -80,9 +82,9 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     const int m0 = blockIdx.x * BM, j0 = blockIdx.y * BN;
 
-    RowInfo ri[2];
-    ri[0] = make_row<MODE>(p, m0 + (tid >> 2));
-    ri[1] = make_row<MODE>(p, m0 + (tid >> 2) + 64);
+    RowInfo ri[ITA];
+#pragma unroll
+    for (int i = 0; i < ITA; ++i) ri[i] = make_row<MODE>(p, m0 + (tid >> 2) + 64 * i);
 
     float ra[8], rb[ITB * 4];
 
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
             int r = 0, s = 0, c = k;
             if (!p.pointwise) { const int rs = k / p.Cs; c = k - rs * p.Cs; r = rs / p.kw; s = rs - r * p.kw; }
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
+            for (int i = 0; i < ITA; ++i) {
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (ri[i].ok && k < p.Kg) {
                     long long off;
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
             const int k = k0 + (tid & 15);
             const int rs = k / p.Cs, c = k - rs * p.Cs, r = rs / p.kw, s = rs - r * p.kw;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < TM; ++i) {
                 float v = 0.f;
                 const int m = m0 + (tid >> 4) + 16 * i;
                 if (m < p.M && k < p.Kg) {
@@ -122,13 +124,13 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
         if (p.vecA) {
             const int kk = (tid & 3) * 4, row = tid >> 2;
 #pragma unroll
-            for (int i = 0; i < 2; ++i)
+            for (int i = 0; i < ITA; ++i)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) As[buf][kk + e][row + 64 * i] = ra[4 * i + e];
         } else {
             const int kk = tid & 15;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) As[buf][kk][(tid >> 4) + 16 * i] = ra[i];
+            for (int i = 0; i < TM; ++i) As[buf][kk][(tid >> 4) + 16 * i] = ra[i];
         }
     };
     auto loadB = [&](int k0) {
@@ -188,9 +190,9 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
         }
     };
 
-    float acc[8][TN];
+    float acc[TM][TN];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
 
@@ -203,10 +205,13 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
         if (kt + 1 < ktiles) { loadA((kt + 1) * BK); loadB((kt + 1) * BK); }
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
-            float a[8], b[TN];
+            float a[TM], b[TN];
             const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * 4]);
-            const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][kk][64 + ty * 4]);
-            a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+            a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w;
+            if constexpr (TM == 8) {
+                const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][kk][64 + ty * 4]);
+                a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+            }
             if constexpr (TN == 8) {
                 const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tx * 4]);
                 const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][64 + tx * 4]);
@@ -219,7 +224,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
                 b[0] = b0.x; b[1] = b0.y;
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < TM; ++i)
 #pragma unroll
                 for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
@@ -234,7 +239,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
     constexpr int NG = TN / GW;
     const bool vecD = p.alignD && (p.Cd % GW) == 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < TM; ++i) {
         const int m = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
         if (m >= p.M) continue;
 #pragma unroll
@@ -436,12 +441,34 @@ WgPlan plan_wgrad(const ConvGeom& g) {
     return w;
 }
 
+// Tile shapes: (rows, columns, relative efficiency of the register micro-tile, resident blocks per SM).
+struct TileOpt { int bm, bn; float eff; int slots; };
+constexpr TileOpt kTiles[] = {{128, 128, 1.00f, 2}, {128, 64, 0.85f, 3}, {64, 128, 0.85f, 3}, {64, 64, 0.65f, 4},
+                              {128, 32, 0.55f, 4}, {64, 32, 0.45f, 6}};
+
+// Estimated cost of covering an M x N output: full waves of resident blocks, each block slowed by its
+// co-residents, padding included through the tile counts.
+inline int pick_tile(long long M, int N) {
+    const long long sms = sm_count();
+    int best = 0;
+    double best_t = 1e300;
+    for (int i = 0; i < (int)(sizeof(kTiles) / sizeof(kTiles[0])); ++i) {
+        const TileOpt& t = kTiles[i];
+        const long long tiles = ((M + t.bm - 1) / t.bm) * ((N + t.bn - 1) / t.bn);
+        const long long waves = (tiles + sms * t.slots - 1) / (sms * t.slots);
+        const double cost = (double)waves * t.slots * t.bm * t.bn / t.eff;
+        if (cost < best_t) { best_t = cost; best = i; }
+    }
+    return best;
+}
+
 template <int MODE>
 void launch_conv_gemm(const GemmP& p, cudaStream_t st) {
-    const int mt = (p.M + BM - 1) / BM;
-    if (p.Cd > 64) conv_gemm_kernel<128, MODE><<<dim3(mt, (p.Cd + 127) / 128), NT, 0, st>>>(p);
-    else if (p.Cd > 32) conv_gemm_kernel<64, MODE><<<dim3(mt, 1), NT, 0, st>>>(p);
-    else conv_gemm_kernel<32, MODE><<<dim3(mt, 1), NT, 0, st>>>(p);
+    const TileOpt t = kTiles[pick_tile(p.M, p.Cd)];
+    const dim3 grid((p.M + t.bm - 1) / t.bm, (p.Cd + t.bn - 1) / t.bn);
+#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) { conv_gemm_kernel<BM_, BN_, MODE><<<grid, NT, 0, st>>>(p); return; }
+    FTP_LAUNCH(128, 128) FTP_LAUNCH(128, 64) FTP_LAUNCH(64, 128) FTP_LAUNCH(64, 64) FTP_LAUNCH(128, 32) FTP_LAUNCH(64, 32)
+#undef FTP_LAUNCH
 }
 
 inline bool a16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; }
