@@ -126,6 +126,9 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
+    ap.add_argument("--points", default=None, help="comma-separated partition points; skips the profile-and-optimise step")
+    ap.add_argument("--graph", type=int, default=1, help="1: time CUDA-graph replays of the step (default); 0: eager launches")
+    ap.add_argument("--lean", action="store_true", help="timed region only: no end-to-end leg, no kernel trace (profiling captures)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -161,7 +164,10 @@ def main():
     lr = cfg["lr"]
 
     # partition: profile -> equal capacities -> optimiser (or the split the workload fixes)
-    fwd_s, bwd_s, out_bytes = m.ftp_profile_layers(10, xd, yd)
+    if args.points:
+        wl["points"] = [int(v) for v in args.points.split(",")]
+    else:
+        fwd_s, bwd_s, out_bytes = m.ftp_profile_layers(10, xd, yd)
     if wl["points"] is None:
         points, bottleneck = F.ftp_choose_partition((fwd_s + bwd_s).tolist(), wl["caps"])
     else:
@@ -188,7 +194,20 @@ def main():
             ms = float(t.item())
         return ms
 
-    step_dev = lambda: m.ftp_train_step(xd, yd, lr, inputs_on_host=False, want_loss=False)
+    step_eager = lambda: m.ftp_train_step(xd, yd, lr, inputs_on_host=False, want_loss=False)
+    step_dev = step_eager
+    if args.graph:
+        # the launches of one step captured once on a side stream and replayed: same kernels, no per-launch CPU cost
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(2):
+                step_eager()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step_eager()
+        step_dev = graph.replay
     step_e2e = lambda: m.ftp_train_step(xh, yh, lr, inputs_on_host=True, want_loss=True)
     for _ in range(args.warmup):
         step_dev()
@@ -196,6 +215,13 @@ def main():
     with ClockSampler(local_rank) as clk:
         ms = timed(step_dev, args.steps)
     launches = m.ftp_launch_count() - n0
+    if args.graph:                      # a replay re-issues the captured launches without passing through the counter
+        c0 = m.ftp_launch_count()
+        step_eager()
+        launches = (m.ftp_launch_count() - c0) * args.steps
+    if args.lean:
+        print(json.dumps({"lean": True, "ms_per_step": ms / args.steps, "gpu_launches": int(launches)}), flush=True)
+        return 0
     for _ in range(3):
         step_e2e()
     ms_e2e = timed(step_e2e, args.steps)
@@ -206,7 +232,7 @@ def main():
     # per-kernel roofline: one more step with every launch bracketed by events
     m.ftp_trace_enable(True)
     for _ in range(3):
-        step_dev()
+        step_eager()
     recs = m.ftp_trace_read()
     m.ftp_trace_enable(False)
     by = {}
@@ -238,7 +264,8 @@ def main():
            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
            "config": {"workload": wl["name"], "points": points, "stages": len(points) - 1, "batch": batch,
                       "parallelism": "replicas only" if world > 1 else "1 GPU, all stages resident",
-                      "cache": "step touches >1.5 GB of activations, far larger than the 126 MB L2"},
+                      "cache": "step touches >1.5 GB of activations, far larger than the 126 MB L2",
+                      "launch": "cuda graph replay of ftp_train_step" if args.graph else "eager"},
            "clocks": clk.summary(), "gpu_launches": int(launches),
            "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(xh.numel() * 4 + yh.numel() * 4),
                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / args.steps},

@@ -119,26 +119,44 @@ __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chu
     }
 }
 
-// Sum over chunks and folded copies for channel c, by one block of FIN_T threads, in a fixed order:
-// strided per-thread runs, then a shared-memory tree.  The result is valid in thread 0.
-constexpr int FIN_T = 128;
-__device__ __forceinline__ double block_fold_sum(const double* partial, int which, int ns, int chunks, int f, int C, int cols, int c) {
-    __shared__ double red[FIN_T];
-    double t = 0.0;
+// Sums over chunks and folded copies for one channel per x-lane: block (32, FIN_Y), x -> channel of a group
+// of 32 (loads coalesced across channels), y -> strided runs over the (chunk, copy) pairs with four
+// independent accumulators (loads stay in flight), then a fixed-order sum over y in shared memory.
+// NS consecutive sums starting at `first` are produced at once; results are valid in the threads with y == 0.
+constexpr int FIN_Y = 32;
+template <typename PT, int NS>
+__device__ __forceinline__ void col_fold_sums(const PT* partial, int first, int ns, int chunks, int f, int C, int cols, int c, double (&out)[NS]) {
+    __shared__ double red[NS][FIN_Y][33];
+    double t[NS][4];
+#pragma unroll
+    for (int a = 0; a < NS; ++a)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) t[a][u] = 0.0;
     const int total = chunks * f;
-    for (int e = threadIdx.x; e < total; e += FIN_T) {
-        const int ch = e / f, k = e - ch * f;
-        t += partial[((long long)ch * ns + which) * cols + k * C + c];
-    }
-    __syncthreads();
-    red[threadIdx.x] = t;
+    if (c < C)
+        for (int e = threadIdx.y; e < total; e += 4 * FIN_Y) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int ee = e + u * FIN_Y;
+                if (ee < total) {
+                    const int ch = ee / f, k = ee - ch * f;
+#pragma unroll
+                    for (int a = 0; a < NS; ++a) t[a][u] += (double)partial[((long long)ch * ns + first + a) * cols + k * C + c];
+                }
+            }
+        }
     __syncthreads();
 #pragma unroll
-    for (int o = FIN_T / 2; o > 0; o >>= 1) {
-        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
-        __syncthreads();
+    for (int a = 0; a < NS; ++a) red[a][threadIdx.y][threadIdx.x] = (t[a][0] + t[a][1]) + (t[a][2] + t[a][3]);
+    __syncthreads();
+#pragma unroll
+    for (int a = 0; a < NS; ++a) {
+        double r = 0.0;
+        if (threadIdx.y == 0)
+#pragma unroll 8
+            for (int y = 0; y < FIN_Y; ++y) r += red[a][y][threadIdx.x];
+        out[a] = r;
     }
-    return red[0];
 }
 
 template <typename T, int V>
@@ -154,10 +172,11 @@ __global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, 
 __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
                                    float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd) {
-    const int c = blockIdx.x;
-    const double s1 = block_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
-    const double s2 = block_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
-    if (threadIdx.x == 0) {
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    double ss[2];
+    col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, ss);
+    const double s1 = ss[0], s2 = ss[1];
+    if (threadIdx.y == 0 && c < C) {
         const double mu = s1 / M;
         double var = s2 / M - mu * mu;
         if (var < 0.0) var = 0.0;
@@ -224,10 +243,11 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
 __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                        const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
                                        float* dbeta, float* coef) {
-    const int c = blockIdx.x;
-    const double s1 = block_fold_sum(partial, 0, 2, chunks, f, C, cols, c);
-    const double s2 = block_fold_sum(partial, 1, 2, chunks, f, C, cols, c);
-    if (threadIdx.x == 0) {
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    double ss[2];
+    col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, ss);
+    const double s1 = ss[0], s2 = ss[1];
+    if (threadIdx.y == 0 && c < C) {
         dbeta[c] = (float)s1;
         dgamma[c] = (float)s2;
         coef[c] = gamma[c] * rstd[c];
@@ -291,9 +311,10 @@ __global__ void __launch_bounds__(256) act_bias_bwd_kernel(const T* __restrict__
 }
 
 __global__ void colsum_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, float* out) {
-    const int c = blockIdx.x;
-    const double s = block_fold_sum(partial, 0, 1, chunks, f, C, cols, c);
-    if (threadIdx.x == 0) out[c] = (float)s;
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    double ss[1];
+    col_fold_sums<double, 1>(partial, 0, 1, chunks, f, C, cols, c, ss);
+    if (threadIdx.y == 0 && c < C) out[c] = (float)ss[0];
 }
 
 template <typename T, int V>
@@ -400,72 +421,73 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
     }
 }
 
-// grid (column tiles, pixel chunks), 256 threads: lane group = channel vector, the rest of the block
-// spreads over pixels.  Writes partial[chunk][9][C].
+// Depthwise weight gradient on the folded view: grid (column tiles of 32*V, pixel-row chunks), block (32, 8).
+// A thread owns V folded columns (a fixed channel vector and a fixed pixel offset within each folded row)
+// and walks the rows of its chunk; the 9 taps are reduced over y three at a time through shared memory.
+// partial[chunk][9][cols] (float).
 template <typename T, int V>
 __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, ConvGeom g,
-                                                       long long npix, int ppc, int cvt) {
-    __shared__ float sh[256][V];
-    const int CV = g.Cin / V;
-    const int cv0 = blockIdx.x * cvt;
-    const int lanes = min(cvt, CV - cv0);            // channel vectors handled by this block
-    const int G = 256 / lanes;                       // pixel groups
-    const int cl = threadIdx.x % lanes, pg = threadIdx.x / lanes;
-    const bool active = pg < G;
-    const int c = (cv0 + cl) * V;
-    const long long p0 = (long long)blockIdx.y * ppc, p1 = min(npix, p0 + ppc);
+                                                       int rows, int cols, int f, int rpc) {
+    __shared__ float sh[3][8][32 * V];
+    const int col = (blockIdx.x * 32 + threadIdx.x) * V;
+    const int r0 = blockIdx.y * rpc, r1 = min(rows, r0 + rpc);
     float acc[9][V];
 #pragma unroll
     for (int t = 0; t < 9; ++t)
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
-    if (active) {
-        for (long long pix = p0 + pg; pix < p1; pix += G) {
+    if (col < cols) {
+        const int kf = col / g.Cin, c = col - kf * g.Cin;        // pixel offset inside a folded row, channel
+        for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+            const long long pix = (long long)r * f + kf;
             const int wo = (int)(pix % g.Wo);
             const long long q = pix / g.Wo;
             const int ho = (int)(q % g.Ho), n = (int)(q / g.Ho);
             float d[V];
             ldv<V>(dy + pix * g.Cin + c, d);
 #pragma unroll
-            for (int r = 0; r < 3; ++r) {
-                const int hi = ho * g.stride - g.ph + r;
+            for (int rr = 0; rr < 3; ++rr) {
+                const int hi = ho * g.stride - g.ph + rr;
                 if (hi < 0 || hi >= g.H) continue;
 #pragma unroll
-                for (int s = 0; s < 3; ++s) {
-                    const int wi = wo * g.stride - g.pw + s;
+                for (int ss = 0; ss < 3; ++ss) {
+                    const int wi = wo * g.stride - g.pw + ss;
                     if (wi < 0 || wi >= g.W) continue;
                     float v[V];
                     ldv<V>(x + ((long long)(n * g.H + hi) * g.W + wi) * g.Cin + c, v);
 #pragma unroll
-                    for (int e = 0; e < V; ++e) acc[r * 3 + s][e] = fmaf(v[e], d[e], acc[r * 3 + s][e]);
+                    for (int e = 0; e < V; ++e) acc[rr * 3 + ss][e] = fmaf(v[e], d[e], acc[rr * 3 + ss][e]);
                 }
             }
         }
     }
-    float* out = partial + (long long)blockIdx.y * 9 * g.Cin;
 #pragma unroll
-    for (int t = 0; t < 9; ++t) {
+    for (int gq = 0; gq < 3; ++gq) {
         __syncthreads();
 #pragma unroll
-        for (int e = 0; e < V; ++e) sh[threadIdx.x][e] = acc[t][e];
-        __syncthreads();
-        if (threadIdx.x < lanes) {
+        for (int t = 0; t < 3; ++t)
 #pragma unroll
-            for (int e = 0; e < V; ++e) {
-                float s = 0.f;
-                for (int q = 0; q < G; ++q) s += sh[q * lanes + threadIdx.x][e];
-                out[t * g.Cin + c + e] = s;
+            for (int e = 0; e < V; ++e) sh[t][threadIdx.y][threadIdx.x * V + e] = acc[gq * 3 + t][e];
+        __syncthreads();
+        for (int q = threadIdx.y * 32 + threadIdx.x; q < 3 * 32 * V; q += 256) {
+            const int t = q / (32 * V), cc = q % (32 * V);
+            const int gc = blockIdx.x * 32 * V + cc;
+            if (gc < cols) {
+                float sum = 0.f;
+#pragma unroll
+                for (int y = 0; y < 8; ++y) sum += sh[t][y][cc];
+                partial[((long long)blockIdx.y * 9 + gq * 3 + t) * cols + gc] = sum;
             }
         }
     }
 }
 
-__global__ void split_sum_kernel(const float* __restrict__ partial, int S, long long count, float* __restrict__ out) {
-    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= count) return;
-    float s = 0.f;
-    for (int z = 0; z < S; ++z) s += partial[(long long)z * count + e];
-    out[e] = s;
+// dw[t][c] = sum over chunks and folded copies of partial[chunk][t][copy * C + c]; grid (ceil(C/32), 9)
+__global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols, float* __restrict__ dw) {
+    const int c = blockIdx.x * 32 + threadIdx.x;
+    double ss[1];
+    col_fold_sums<float, 1>(partial, (int)blockIdx.y, 9, chunks, f, C, cols, c, ss);
+    if (threadIdx.y == 0 && c < C) dw[blockIdx.y * C + c] = (float)ss[0];
 }
 
 // ---- pooling --------------------------------------------------------------------------------------
@@ -684,7 +706,7 @@ void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partia
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
                  float* mean_lo, float* rstd, cudaStream_t st) {
-    bn_finalize_kernel<<<C, FIN_T, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
+    bn_finalize_kernel<<<(C + 31) / 32, dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
                                                              run_mean, run_var, scale, shift, mean, mean_lo, rstd);
 }
 
@@ -713,7 +735,7 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
 
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
                      float* dgamma, float* dbeta, float* coef, cudaStream_t st) {
-    bn_bwd_finalize_kernel<<<C, FIN_T, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef);
+    bn_bwd_finalize_kernel<<<(C + 31) / 32, dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef);
 }
 
 template <typename T>
@@ -735,7 +757,7 @@ void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int 
         act_bias_bwd_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
     else
         act_bias_bwd_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
-    if (dbias) colsum_finalize_kernel<<<C, FIN_T, 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias);
+    if (dbias) colsum_finalize_kernel<<<(C + 31) / 32, dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias);
 }
 
 template <typename T>
@@ -769,35 +791,26 @@ void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const Con
     else dw_dgrad_kernel<T, 1><<<flat_blocks(pix * g.Cin, 256), 256, 0, st>>>(dy, w, addend, dx, g, pix * g.Cin);
 }
 
-struct DwWgPlan { int chunks, ppc; };
-static DwWgPlan plan_dw_wgrad(const ConvGeom& g) {
-    const long long npix = (long long)g.N * g.Ho * g.Wo;
-    long long chunks = 4LL * sm_count();
-    const long long maxc = (npix + 63) / 64;
-    if (chunks > maxc) chunks = maxc;
-    if (chunks < 1) chunks = 1;
-    DwWgPlan p;
-    p.ppc = (int)((npix + chunks - 1) / chunks);
-    p.chunks = (int)((npix + p.ppc - 1) / p.ppc);
-    return p;
+static FoldPlan plan_dw_wgrad(const ConvGeom& g, int elem_bytes) {
+    return make_fold((long long)g.N * g.Ho * g.Wo, g.Cin, elem_bytes);
 }
 
-size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) { return (size_t)plan_dw_wgrad(g).chunks * 9 * g.Cin; }
+size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
+    const FoldPlan a = plan_dw_wgrad(g, 4), b = plan_dw_wgrad(g, 2);
+    const size_t na = (size_t)a.chunks * 9 * a.cols, nb = (size_t)b.chunks * 9 * b.cols;
+    return na > nb ? na : nb;
+}
 
 template <typename T>
 void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    const DwWgPlan p = plan_dw_wgrad(g);
-    const long long npix = (long long)g.N * g.Ho * g.Wo;
-    if (can_vec<T>(g.Cin, x, dy)) {
-        const int CV = g.Cin / V, cvt = CV < 256 ? CV : 256;
-        dw_wgrad_kernel<T, V><<<dim3((CV + cvt - 1) / cvt, p.chunks), 256, 0, st>>>(x, dy, scratch, g, npix, p.ppc, cvt);
-    } else {
-        const int CV = g.Cin, cvt = CV < 256 ? CV : 256;
-        dw_wgrad_kernel<T, 1><<<dim3((CV + cvt - 1) / cvt, p.chunks), 256, 0, st>>>(x, dy, scratch, g, npix, p.ppc, cvt);
-    }
-    const long long count = 9LL * g.Cin;
-    split_sum_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, p.chunks, count, dw);
+    FoldPlan fp = plan_dw_wgrad(g, (int)sizeof(T));
+    const int rpc = fold_rpc(fp);
+    if (fp.vec == V && aligned16(x) && aligned16(dy))
+        dw_wgrad_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
+    else
+        dw_wgrad_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
+    dw_wgrad_finalize_kernel<<<dim3((g.Cin + 31) / 32, 9), dim3(32, FIN_Y), 0, st>>>(scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw);
 }
 
 template <typename T>
