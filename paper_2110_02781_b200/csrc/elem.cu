@@ -119,26 +119,32 @@ __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chu
     }
 }
 
-// Sums over chunks and folded copies for one channel per x-lane: block (32, FIN_Y), x -> channel of a group
-// of 32 (loads coalesced across channels), y -> strided runs over the (chunk, copy) pairs with four
-// independent accumulators (loads stay in flight), then a fixed-order sum over y in shared memory.
-// NS consecutive sums starting at `first` are produced at once; results are valid in the threads with y == 0.
+// Second pass of every folded column reduction: sums over chunks and folded copies, one channel per x-lane.
+// Grid (channel groups of 32, G slices of the (chunk, copy) pairs, extra); block (32, FIN_Y).  Inside a block,
+// y -> strided runs with four independent accumulators, then a fixed-order sum over y in shared memory.  With
+// G > 1 every block parks its slice sums in fin.part and takes a ticket; the block that draws the last ticket
+// adds the G slice sums in slice order, so the result does not depend on which block that is.  Returns true in
+// the block that holds the final sums (valid in its threads with y == 0).  NS consecutive sums from `first`.
 constexpr int FIN_Y = 32;
+constexpr int FIN_GMAX = 16;
 template <typename PT, int NS>
-__device__ __forceinline__ void col_fold_sums(const PT* partial, int first, int ns, int chunks, int f, int C, int cols, int c, double (&out)[NS]) {
+__device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int ns, int chunks, int f, int C, int cols, int c,
+                                              const FinScratch fin, double (&out)[NS]) {
     __shared__ double red[NS][FIN_Y][33];
+    __shared__ unsigned ticket;
     double t[NS][4];
 #pragma unroll
     for (int a = 0; a < NS; ++a)
 #pragma unroll
         for (int u = 0; u < 4; ++u) t[a][u] = 0.0;
-    const int total = chunks * f;
+    const int total = chunks * f, G = gridDim.y;
+    const int per = (total + G - 1) / G, e0 = blockIdx.y * per, e1 = min(total, e0 + per);
     if (c < C)
-        for (int e = threadIdx.y; e < total; e += 4 * FIN_Y) {
+        for (int e = e0 + threadIdx.y; e < e1; e += 4 * FIN_Y) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int ee = e + u * FIN_Y;
-                if (ee < total) {
+                if (ee < e1) {
                     const int ch = ee / f, k = ee - ch * f;
 #pragma unroll
                     for (int a = 0; a < NS; ++a) t[a][u] += (double)partial[((long long)ch * ns + first + a) * cols + k * C + c];
@@ -157,6 +163,28 @@ __device__ __forceinline__ void col_fold_sums(const PT* partial, int first, int 
             for (int y = 0; y < FIN_Y; ++y) r += red[a][y][threadIdx.x];
         out[a] = r;
     }
+    if (G == 1) return true;
+    const int slot = blockIdx.z * gridDim.x + blockIdx.x;
+    double* mine = fin.part + ((long long)slot * FIN_GMAX + blockIdx.y) * NS * 32;
+    if (threadIdx.y == 0)
+#pragma unroll
+        for (int a = 0; a < NS; ++a) mine[a * 32 + threadIdx.x] = out[a];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0 && threadIdx.y == 0) ticket = atomicAdd(fin.counters + slot, 1u);
+    __syncthreads();
+    if (ticket != (unsigned)(G - 1)) return false;
+    __threadfence();
+    if (threadIdx.y == 0) {
+#pragma unroll
+        for (int a = 0; a < NS; ++a) {
+            double r = 0.0;
+            for (int g = 0; g < G; ++g) r += __ldcg(fin.part + ((long long)slot * FIN_GMAX + g) * NS * 32 + a * 32 + threadIdx.x);
+            out[a] = r;
+        }
+        if (threadIdx.x == 0) fin.counters[slot] = 0u;       // ready for the next launch on this stream
+    }
+    return true;
 }
 
 template <typename T, int V>
@@ -171,10 +199,11 @@ __global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, 
 
 __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
-                                   float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd) {
+                                   float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd,
+                                   const FinScratch fin) {
     const int c = blockIdx.x * 32 + threadIdx.x;
     double ss[2];
-    col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, ss);
+    if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
     if (threadIdx.y == 0 && c < C) {
         const double mu = s1 / M;
@@ -242,10 +271,10 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
 
 __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                        const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
-                                       float* dbeta, float* coef) {
+                                       float* dbeta, float* coef, const FinScratch fin) {
     const int c = blockIdx.x * 32 + threadIdx.x;
     double ss[2];
-    col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, ss);
+    if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
     if (threadIdx.y == 0 && c < C) {
         dbeta[c] = (float)s1;
@@ -310,10 +339,10 @@ __global__ void __launch_bounds__(256) act_bias_bwd_kernel(const T* __restrict__
     });
 }
 
-__global__ void colsum_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, float* out) {
+__global__ void colsum_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, float* out, const FinScratch fin) {
     const int c = blockIdx.x * 32 + threadIdx.x;
     double ss[1];
-    col_fold_sums<double, 1>(partial, 0, 1, chunks, f, C, cols, c, ss);
+    if (!col_fold_sums<double, 1>(partial, 0, 1, chunks, f, C, cols, c, fin, ss)) return;
     if (threadIdx.y == 0 && c < C) out[c] = (float)ss[0];
 }
 
@@ -482,12 +511,13 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, 
     }
 }
 
-// dw[t][c] = sum over chunks and folded copies of partial[chunk][t][copy * C + c]; grid (ceil(C/32), 9)
-__global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols, float* __restrict__ dw) {
+// dw[t][c] = sum over chunks and folded copies of partial[chunk][t][copy * C + c]; grid (ceil(C/32), G, 9)
+__global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols, float* __restrict__ dw,
+                                         const FinScratch fin) {
     const int c = blockIdx.x * 32 + threadIdx.x;
     double ss[1];
-    col_fold_sums<float, 1>(partial, (int)blockIdx.y, 9, chunks, f, C, cols, c, ss);
-    if (threadIdx.y == 0 && c < C) dw[blockIdx.y * C + c] = (float)ss[0];
+    if (!col_fold_sums<float, 1>(partial, (int)blockIdx.z, 9, chunks, f, C, cols, c, fin, ss)) return;
+    if (threadIdx.y == 0 && c < C) dw[blockIdx.z * C + c] = (float)ss[0];
 }
 
 // ---- pooling --------------------------------------------------------------------------------------
@@ -693,6 +723,13 @@ FoldPlan make_fold(long long M, int C, int elem_bytes) {
 
 size_t fold_partial_doubles(const FoldPlan& fp) { return (size_t)fp.chunks * 2 * fp.cols; }
 
+size_t fin_part_doubles(int C, int extra) { return (size_t)((C + 31) / 32) * extra * FIN_GMAX * 2 * 32; }
+size_t fin_counter_count(int C, int extra) { return (size_t)((C + 31) / 32) * extra; }
+static inline int fin_slices(const FoldPlan& fp) {
+    const int g = fp.chunks * fp.f / 256;
+    return g < 1 ? 1 : (g > FIN_GMAX ? FIN_GMAX : g);
+}
+
 static inline int fold_rpc(const FoldPlan& fp) { return (fp.rows + fp.chunks - 1) / fp.chunks; }
 static inline dim3 fold_grid(const FoldPlan& fp) { return dim3((fp.cols + 32 * fp.vec - 1) / (32 * fp.vec), fp.chunks); }
 
@@ -705,9 +742,9 @@ void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partia
 
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
-                 float* mean_lo, float* rstd, cudaStream_t st) {
-    bn_finalize_kernel<<<(C + 31) / 32, dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
-                                                             run_mean, run_var, scale, shift, mean, mean_lo, rstd);
+                 float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st) {
+    bn_finalize_kernel<<<dim3((C + 31) / 32, fin_slices(fp)), dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
+                                                             run_mean, run_var, scale, shift, mean, mean_lo, rstd, fin);
 }
 
 template <typename T>
@@ -734,8 +771,8 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
 }
 
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
-                     float* dgamma, float* dbeta, float* coef, cudaStream_t st) {
-    bn_bwd_finalize_kernel<<<(C + 31) / 32, dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef);
+                     float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st) {
+    bn_bwd_finalize_kernel<<<dim3((C + 31) / 32, fin_slices(fp)), dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
 }
 
 template <typename T>
@@ -751,13 +788,13 @@ void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, 
 
 template <typename T>
 void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int act, const FoldPlan& fp, double* partial,
-                  float* dbias, cudaStream_t st) {
+                  float* dbias, const FinScratch& fin, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     if (fp.vec == V && aligned16(dout) && aligned16(out) && aligned16(dpre))
         act_bias_bwd_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
     else
         act_bias_bwd_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
-    if (dbias) colsum_finalize_kernel<<<(C + 31) / 32, dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias);
+    if (dbias) colsum_finalize_kernel<<<dim3((C + 31) / 32, fin_slices(fp)), dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias, fin);
 }
 
 template <typename T>
@@ -802,7 +839,7 @@ size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
 }
 
 template <typename T>
-void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st) {
+void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     FoldPlan fp = plan_dw_wgrad(g, (int)sizeof(T));
     const int rpc = fold_rpc(fp);
@@ -810,7 +847,7 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
         dw_wgrad_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
     else
         dw_wgrad_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
-    dw_wgrad_finalize_kernel<<<dim3((g.Cin + 31) / 32, 9), dim3(32, FIN_Y), 0, st>>>(scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw);
+    dw_wgrad_finalize_kernel<<<dim3((g.Cin + 31) / 32, fin_slices(fp), 9), dim3(32, FIN_Y), 0, st>>>(scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
 }
 
 template <typename T>
@@ -870,12 +907,12 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
     template void bn_bwd_apply<T>(const T*, const T*, const T*, T*, long long, int, const float*, const float*,             \
                                   const float*, const float*, const float*, const float*, int, cudaStream_t);              \
     template void act_bias_bwd<T>(const T*, const T*, T*, long long, int, int, const FoldPlan&, double*, float*,            \
-                                  cudaStream_t);                                                                           \
+                                  const FinScratch&, cudaStream_t);                                                                           \
     template void act_fwd<T>(const T*, T*, long long, int, cudaStream_t);                                                   \
     template void act_bwd<T>(const T*, const T*, const T*, T*, long long, int, cudaStream_t);                               \
     template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t);                                 \
     template void dwconv_dgrad<T>(const T*, const float*, const T*, T*, const ConvGeom&, cudaStream_t);                     \
-    template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, cudaStream_t);                       \
+    template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t);                       \
     template void maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);                                           \
     template void maxpool_bwd<T>(const T*, const T*, T*, int, int, int, int, cudaStream_t);                                 \
     template void gap_fwd<T>(const T*, T*, int, int, int, cudaStream_t);                                                    \

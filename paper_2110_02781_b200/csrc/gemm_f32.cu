@@ -26,6 +26,7 @@ struct GemmP {
     int Hd, Wd;            // destination tensor spatial dims
     int kh, kw, stride, ph, pw;
     int act, vecA, vecB, alignD, pointwise;
+    int kt_per;            // reduction tiles per z-slice (split over K: slice z writes its partial at D + z*M*Cd)
 };
 
 struct RowInfo {
@@ -196,12 +197,13 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
 #pragma unroll
         for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
 
-    const int ktiles = (p.Kg + BK - 1) / BK;
-    loadA(0); loadB(0);
+    const int kt0 = blockIdx.z * p.kt_per;
+    const int ktiles = min((p.Kg + BK - 1) / BK, kt0 + p.kt_per);
+    loadA(kt0 * BK); loadB(kt0 * BK);
     storeA(0); storeB(0);
     __syncthreads();
-    for (int kt = 0; kt < ktiles; ++kt) {
-        const int buf = kt & 1;
+    for (int kt = kt0; kt < ktiles; ++kt) {
+        const int buf = (kt - kt0) & 1;
         if (kt + 1 < ktiles) { loadA((kt + 1) * BK); loadB((kt + 1) * BK); }
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
@@ -235,6 +237,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
     }
 
     // epilogue: bias, activation, residual-gradient addend, store (16-byte stores when aligned)
+    float* const Dz = p.D + (long long)blockIdx.z * p.M * p.Cd;
     constexpr int GW = TN >= 4 ? 4 : 2;            // columns per contiguous group
     constexpr int NG = TN / GW;
     const bool vecD = p.alignD && (p.Cd % GW) == 0;
@@ -257,15 +260,15 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
             if (vecD) {
                 if constexpr (GW == 4) {
                     if (p.addend) { const float4 a = __ldg(reinterpret_cast<const float4*>(p.addend + o)); v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w; }
-                    *reinterpret_cast<float4*>(p.D + o) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4*>(Dz + o) = make_float4(v[0], v[1], v[2], v[3]);
                 } else {
                     if (p.addend) { const float2 a = __ldg(reinterpret_cast<const float2*>(p.addend + o)); v[0] += a.x; v[1] += a.y; }
-                    *reinterpret_cast<float2*>(p.D + o) = make_float2(v[0], v[1]);
+                    *reinterpret_cast<float2*>(Dz + o) = make_float2(v[0], v[1]);
                 }
             } else {
 #pragma unroll
                 for (int e = 0; e < GW; ++e)
-                    if (jc + e < p.Cd) p.D[o + e] = v[e] + (p.addend ? __ldg(p.addend + o + e) : 0.f);
+                    if (jc + e < p.Cd) Dz[o + e] = v[e] + (p.addend ? __ldg(p.addend + o + e) : 0.f);
             }
         }
     }
@@ -422,6 +425,24 @@ __global__ void split_reduce_kernel(const float* __restrict__ partial, int S, lo
     out[e] = s;
 }
 
+// out[e] = sum_z partial[z][e] (+ bias[column]) (+ addend[e]), z ascending
+__global__ void split_reduce_add_kernel(const float* __restrict__ partial, int S, long long count4, const float* __restrict__ addend,
+                                        const float* __restrict__ bias, int Cd, float* __restrict__ out) {
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count4) return;
+    float4 s = __ldg(reinterpret_cast<const float4*>(partial) + e);
+    for (int z = 1; z < S; ++z) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(partial) + (long long)z * count4 + e);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    if (bias) {
+        const int c = (int)((e * 4) % Cd);
+        s.x += __ldg(bias + c); s.y += __ldg(bias + (c + 1) % Cd); s.z += __ldg(bias + (c + 2) % Cd); s.w += __ldg(bias + (c + 3) % Cd);
+    }
+    if (addend) { const float4 a = __ldg(reinterpret_cast<const float4*>(addend) + e); s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w; }
+    reinterpret_cast<float4*>(out)[e] = s;
+}
+
 struct WgPlan { int BI, S, chunk; };
 
 WgPlan plan_wgrad(const ConvGeom& g) {
@@ -430,8 +451,10 @@ WgPlan plan_wgrad(const ConvGeom& g) {
     WgPlan w;
     w.BI = Kg > 64 ? 128 : 64;
     const int tiles = ((Kg + w.BI - 1) / w.BI) * ((g.Cout + 63) / 64);
-    long long S = (2LL * sm_count() + tiles - 1) / tiles;
-    const long long maxS = (M + 255) / 256;
+    long long S = (4LL * sm_count() + tiles - 1) / tiles;          // ~4 resident blocks per SM hide the load latency
+    long long maxS = (M + 255) / 256;
+    const long long cap = (4LL << 20) / ((long long)Kg * g.Cout);  // keep the partials within 4 Mi floats
+    if (maxS > cap) maxS = cap;
     if (S > maxS) S = maxS;
     if (S < 1) S = 1;
     long long chunk = (M + S - 1) / S;
@@ -462,13 +485,46 @@ inline int pick_tile(long long M, int N) {
     return best;
 }
 
+// Split of the reduction dimension for outputs too small to fill the GPU (late layers: few pixels, many
+// channels).  Only plain products qualify (no bias, no activation); the addend joins in the second pass.
+struct GemmPlan { int tile, S, kt_per; };
+inline GemmPlan plan_gemm(long long M, int N, int Kg, bool plain) {
+    GemmPlan gp;
+    gp.tile = pick_tile(M, N);
+    const TileOpt& t = kTiles[gp.tile];
+    const long long tiles = ((M + t.bm - 1) / t.bm) * ((N + t.bn - 1) / t.bn);
+    const int ktiles = (Kg + BK - 1) / BK;
+    long long S = 1;
+    if (plain && tiles < 2LL * sm_count() && ktiles >= 8 && (M * N) % 4 == 0) {
+        S = (3LL * sm_count() + tiles - 1) / tiles;
+        if (S > ktiles / 4) S = ktiles / 4;
+        if (S > 16) S = 16;
+        if (S < 1) S = 1;
+    }
+    gp.kt_per = (int)((ktiles + S - 1) / S);
+    gp.S = (ktiles + gp.kt_per - 1) / gp.kt_per;
+    return gp;
+}
+
 template <int MODE>
-void launch_conv_gemm(const GemmP& p, cudaStream_t st) {
-    const TileOpt t = kTiles[pick_tile(p.M, p.Cd)];
-    const dim3 grid((p.M + t.bm - 1) / t.bm, (p.Cd + t.bn - 1) / t.bn);
-#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) { conv_gemm_kernel<BM_, BN_, MODE><<<grid, NT, 0, st>>>(p); return; }
+void launch_conv_gemm(GemmP p, float* scratch, cudaStream_t st) {
+    const bool plain = p.act == 0 && scratch != nullptr && (reinterpret_cast<uintptr_t>(p.D) & 15) == 0 &&
+                       (reinterpret_cast<uintptr_t>(p.addend) & 15) == 0;
+    const GemmPlan gp = plan_gemm(p.M, p.Cd, p.Kg, plain);
+    const TileOpt t = kTiles[gp.tile];
+    const dim3 grid((p.M + t.bm - 1) / t.bm, (p.Cd + t.bn - 1) / t.bn, gp.S);
+    float* const out = p.D;
+    const float* const addend = p.addend;
+    const float* const bias = p.bias;
+    p.kt_per = gp.kt_per;
+    if (gp.S > 1) { p.D = scratch; p.addend = nullptr; p.bias = nullptr; p.alignD = 1; }
+#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) conv_gemm_kernel<BM_, BN_, MODE><<<grid, NT, 0, st>>>(p);
     FTP_LAUNCH(128, 128) FTP_LAUNCH(128, 64) FTP_LAUNCH(64, 128) FTP_LAUNCH(64, 64) FTP_LAUNCH(128, 32) FTP_LAUNCH(64, 32)
 #undef FTP_LAUNCH
+    if (gp.S > 1) {
+        const long long count4 = (long long)p.M * p.Cd / 4;
+        split_reduce_add_kernel<<<(unsigned)((count4 + 255) / 256), 256, 0, st>>>(scratch, gp.S, count4, addend, bias, p.Cd, out);
+    }
 }
 
 inline bool a16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; }
@@ -476,7 +532,14 @@ inline bool is_pointwise(const ConvGeom& g) { return g.kh == 1 && g.kw == 1 && g
 
 }  // namespace
 
-void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, const ConvGeom& g, int act,
+size_t conv_gemm_scratch_floats(const ConvGeom& g) {
+    const long long Mf = (long long)g.N * g.Ho * g.Wo, Mb = (long long)g.N * g.H * g.W;
+    const GemmPlan f = plan_gemm(Mf, g.Cout, g.kh * g.kw * g.Cin, true), b = plan_gemm(Mb, g.Cin, g.kh * g.kw * g.Cout, true);
+    const size_t nf = f.S > 1 ? (size_t)f.S * Mf * g.Cout : 0, nb = b.S > 1 ? (size_t)b.S * Mb * g.Cin : 0;
+    return nf > nb ? nf : nb;
+}
+
+void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, float* scratch, const ConvGeom& g, int act,
                   cudaStream_t st) {
     GemmP p{};
     p.A = x; p.B = w; p.bias = bias; p.addend = nullptr; p.D = y;
@@ -485,10 +548,10 @@ void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, c
     p.kh = g.kh; p.kw = g.kw; p.stride = g.stride; p.ph = g.ph; p.pw = g.pw;
     p.act = act; p.vecA = (g.Cin % 4 == 0) && a16(x); p.vecB = (g.Cout % 4 == 0) && a16(w); p.alignD = a16(y);
     p.pointwise = is_pointwise(g);
-    launch_conv_gemm<0>(p, st);
+    launch_conv_gemm<0>(p, scratch, st);
 }
 
-void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, const ConvGeom& g,
+void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, float* scratch, const ConvGeom& g,
                     cudaStream_t st) {
     GemmP p{};
     p.A = dy; p.B = w; p.bias = nullptr; p.addend = addend; p.D = dx;
@@ -497,7 +560,7 @@ void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float*
     p.kh = g.kh; p.kw = g.kw; p.stride = g.stride; p.ph = g.ph; p.pw = g.pw;
     p.act = 0; p.vecA = (g.Cout % 4 == 0) && a16(dy); p.vecB = (g.Cout % 4 == 0) && a16(w); p.alignD = a16(dx) && a16(addend);
     p.pointwise = is_pointwise(g);
-    launch_conv_gemm<1>(p, st);
+    launch_conv_gemm<1>(p, scratch, st);
 }
 
 size_t conv_wgrad_scratch_floats(const ConvGeom& g) {

@@ -16,10 +16,12 @@ struct ConvGeom {
 
 // ---- fp32 SIMT contraction (gemm_f32.cu) ---------------------------------------------------
 // y = act(conv(x, w) + bias) (+ addend): implicit GEMM, M = N*Ho*Wo, K = kh*kw*Cin.
-void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, const ConvGeom& g, int act,
+// scratch (nullable): conv_gemm_scratch_floats(g) floats; lets small outputs split the reduction over blocks.
+size_t conv_gemm_scratch_floats(const ConvGeom& g);
+void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, float* scratch, const ConvGeom& g, int act,
                   cudaStream_t st);
 // dx = conv^T(dy, w) (+ addend): implicit GEMM over the input pixels, K = kh*kw*Cout.
-void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, const ConvGeom& g,
+void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, float* scratch, const ConvGeom& g,
                     cudaStream_t st);
 // dw[kh][kw][cin][cout] = sum over output pixels; split over M with a fixed-order second pass.
 // scratch must hold conv_wgrad_scratch_floats(g) floats.
@@ -37,6 +39,15 @@ struct FoldPlan {
     int vec;        // elements per thread per row (16 bytes worth, or 1)
 };
 FoldPlan make_fold(long long M, int C, int elem_bytes);
+// Scratch of the second pass: slice sums parked by its blocks and one ticket counter per channel group
+// (and per tap for the depthwise gradient).  The counters must be zero before the first launch; every
+// launch leaves them zero.  Launches sharing one FinScratch must be ordered on a stream.
+struct FinScratch {
+    double* part;
+    unsigned* counters;
+};
+size_t fin_part_doubles(int C, int extra);      // extra = 9 for the depthwise weight gradient, else 1
+size_t fin_counter_count(int C, int extra);
 size_t fold_partial_doubles(const FoldPlan& fp);     // doubles needed for the partial sums
 
 template <typename T>
@@ -45,7 +56,7 @@ void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partia
 // rstd; running statistics update (momentum, unbiased variance).  z = ((y - mean) - mean_lo) * scale + shift.
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
                  const float* beta, float eps, float momentum, float* run_mean, float* run_var, float* scale,
-                 float* shift, float* mean, float* mean_lo, float* rstd, cudaStream_t st);
+                 float* shift, float* mean, float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st);
 template <typename T>
 void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift,
               const float* mean, const float* mean_lo, int act, cudaStream_t st);
@@ -57,7 +68,7 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
 // -> dgamma, dbeta and the per-channel coefficients coef[5][C]: a = gamma*rstd, then b = dbeta/M and
 // c = dgamma/M each as a two-float sum (hi, lo)
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
-                     const float* rstd, float* dgamma, float* dbeta, float* coef, cudaStream_t st);
+                     const float* rstd, float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st);
 template <typename T>
 void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale,
                   const float* shift, const float* mean, const float* mean_lo, const float* rstd, const float* coef,
@@ -67,7 +78,7 @@ void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, 
 // dpre may be NULL when act == 0 (then dpre == dout); dbias may be NULL.
 template <typename T>
 void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int act, const FoldPlan& fp,
-                  double* partial, float* dbias, cudaStream_t st);
+                  double* partial, float* dbias, const FinScratch& fin, cudaStream_t st);
 template <typename T>
 void act_fwd(const T* x, T* y, long long n, int act, cudaStream_t st);
 template <typename T>
@@ -79,7 +90,7 @@ template <typename T>
 void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const ConvGeom& g, cudaStream_t st);
 size_t dwconv_wgrad_scratch_floats(const ConvGeom& g);
 template <typename T>
-void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st);
+void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st);
 
 template <typename T>
 void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);

@@ -214,7 +214,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     }
     m.grad = (float*)bp.take((size_t)m.P * 4);
     m.state_backup = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
-    size_t max_act = 0, red = 0, foldd = 0, dpre = 0;
+    size_t max_act = 0, red = 0, foldd = 0, dpre = 0, finp = 64, finc = 1;
     for (int i = 0; i < n; ++i) {
         Op& o = m.ops[i];
         const size_t obytes = (size_t)o.out_elems * (o.out_f32 ? 4 : es);
@@ -228,13 +228,16 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             o.coef = t + 5 * stride;
             o.fold = make_fold(Mout, o.C, m.esize);
             foldd = std::max(foldd, fold_partial_doubles(o.fold));
+            finp = std::max(finp, fin_part_doubles(o.C, 1)); finc = std::max(finc, fin_counter_count(o.C, 1));
         } else if (is_contraction(o.d.kind)) {
-            red = std::max(red, conv_wgrad_scratch_floats(o.g));
+            finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
+            red = std::max(red, std::max(conv_wgrad_scratch_floats(o.g), conv_gemm_scratch_floats(o.g)));
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
             if (o.d.act != FTP_ACT_NONE) dpre = std::max(dpre, obytes);
         } else if (o.d.kind == FTP_DWCONV3x3) {
             red = std::max(red, dwconv_wgrad_scratch_floats(o.g));
+            finp = std::max(finp, fin_part_doubles(o.C, 9)); finc = std::max(finc, fin_counter_count(o.C, 9));
         }
     }
     int n_slots = 0;
@@ -246,6 +249,8 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     m.red_floats = std::max<size_t>(red, 64); m.red_scratch = (float*)bp.take(m.red_floats * 4);
     m.fold_doubles = std::max<size_t>(foldd, 64); m.fold_scratch = (double*)bp.take(m.fold_doubles * 8);
     m.dpre_bytes = std::max<size_t>(dpre, 256); m.dpre = bp.take(m.dpre_bytes);
+    m.fin.part = (double*)bp.take(finp * 8);
+    m.fin_counter_bytes = finc * 4; m.fin.counters = (unsigned*)bp.take(m.fin_counter_bytes);
     m.dlogits = (float*)bp.take((size_t)m.cfg.batch * m.cfg.n_classes * 4);
     m.per_sample = (float*)bp.take((size_t)m.cfg.batch * 4);
     m.loss_dev = (float*)bp.take(256);
@@ -292,7 +297,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
                 if (m->cfg.precision == FTP_FP32) {
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
-                    conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, o.g, o.d.act, st);
+                    conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                 } else {
                     return fail(FTP_EUNSUPPORTED, "bf16 contractions are not built yet");
                 }
@@ -309,7 +314,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                   bn_stats<T>((const T*)in, Mr, o.C, o.fold, m->fold_scratch, st); }
                 { Scope sc(m, st, K_BN_FINALIZE, u, i, 0, fold_partial_doubles(o.fold) * 8.0, 0.0);
                   bn_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, ar.w + o.b_off, m->cfg.bn_eps, m->cfg.bn_momentum,
-                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, st); }
+                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, m->fin, st); }
                 const void* res = nullptr;
                 if (o.fused_add) { const int s = m->ops[i + 1].d.residual_src; res = s < first ? act_in : m->cur_out[s]; }
                 { Scope sc(m, st, K_BN_APPLY, u, i, 0, (o.in_elems * (res ? 3.0 : 2.0)) * es, 2.0 * o.in_elems);
@@ -385,20 +390,20 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                     float* dpre = o.d.act != FTP_ACT_NONE ? (float*)m->dpre : nullptr;
                     Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 4.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
                     act_bias_bwd<float>(d, (const float*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
-                                        o.b_off >= 0 ? gr + o.b_off : nullptr, st);
+                                        o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                     if (dpre) d = dpre;
                 }
                 { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
                   conv_wgrad_f32((const float*)in, d, gr + o.w_off, m->red_scratch, o.g, st); }
                 if (gi) {
                     Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl);
-                    conv_dgrad_f32(d, ar.w + o.w_off, (const float*)addend, (float*)gi, o.g, st);
+                    conv_dgrad_f32(d, ar.w + o.w_off, (const float*)addend, (float*)gi, m->red_scratch, o.g, st);
                 }
                 break;
             }
             case FTP_DWCONV3x3: {
                 { Scope sc(m, st, K_DW_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems, 2);
-                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, m->red_scratch, o.g, st); }
+                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, m->red_scratch, o.g, m->fin, st); }
                 if (gi) {
                     Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
                     dwconv_dgrad<T>((const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, o.g, st);
@@ -410,7 +415,7 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                 { Scope sc(m, st, K_BN_BWD_REDUCE, u, i, 1, 2.0 * o.in_elems * es, 8.0 * o.in_elems);
                   bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.d.act, m->fold_scratch, st); }
                 { Scope sc(m, st, K_BN_BWD_FINALIZE, u, i, 1, fold_partial_doubles(o.fold) * 8.0, 0.0);
-                  bn_bwd_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, st); }
+                  bn_bwd_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, m->fin, st); }
                 if (gi) {
                     Scope sc(m, st, K_BN_BWD_APPLY, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, 8.0 * o.in_elems);
                     bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef, o.d.act, st);
@@ -517,6 +522,11 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         s = fail(FTP_ENOMEM, "build_model: workspace too small (need %zu device and %zu pinned bytes)", need, pneed);
     if (s != FTP_OK) { delete m; return s; }
     m->pinned = (float*)pinned_ws; m->pinned_bytes = pinned_bytes;
+    if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess) {     // ticket counters start at zero
+        const ftp_status e = fail(FTP_ECUDA, "build_model: clearing the ticket counters failed: %s", cudaGetErrorString(cudaGetLastError()));
+        delete m;
+        return e;
+    }
     m->owner.assign(m->L, 0);
     m->points = {0, m->L};
     m->n_stages = 1;

@@ -64,6 +64,7 @@ struct ftp_model {
     size_t slot_bytes;
     float* red_scratch; size_t red_floats;
     double* fold_scratch; size_t fold_doubles;
+    ftp::FinScratch fin; size_t fin_counter_bytes;
     void* dpre; size_t dpre_bytes;
     float* dlogits; float* per_sample; float* loss_dev; int32_t* labels_dev; void* input_dev; float* state_backup;
     float* pinned; size_t pinned_bytes;
