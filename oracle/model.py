@@ -12,9 +12,28 @@ from . import ops
 CONV1D, CONV2D, DW, BN, ACT, ADD, MAXPOOL, GAP, FC, CE = range(10)
 
 
+def round_bf16(x):
+    """Round to the nearest bfloat16 (ties to even), returned as float64."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
 class OracleModel:
-    def __init__(self, layers, cfg, params, state):
-        """`params` / `state`: per op a list of arrays in canonical order (copied to float64)."""
+    def __init__(self, layers, cfg, params, state, storage=None):
+        """`params` / `state`: per op a list of arrays in canonical order (copied to float64).
+
+        storage: None -> everything float64.  "bf16" -> the precision the bf16 configurations fix:
+        activations and the gradients handed from op to op are stored as bfloat16, dense-convolution
+        weights are used as bfloat16, accumulation is exact (float64 here, float32 on the device);
+        master weights, depthwise / BN / classifier parameters, statistics, logits and the loss are
+        not rounded.  A value is rounded where it is stored: a BN whose result goes straight into a
+        residual add is rounded once, after the add; a gradient with two contributions is rounded
+        once, after they are summed.  Activation decisions are taken on the stored values for
+        convolutions with a fused activation and on the unrounded normalised value for BN."""
+        self.q = round_bf16 if (storage if storage is not None else ("bf16" if cfg.get("precision") == 1 else None)) == "bf16" \
+            else (lambda v: v)
+        self.quantised = self.q is round_bf16
         self.layers = list(layers)
         self.cfg = dict(cfg)
         self.L = self.layers[-1].unit + 1
@@ -45,11 +64,14 @@ class OracleModel:
             if l.kind in (CONV1D, CONV2D, FC):
                 ph, pw = self._pads(l)
                 bias = self.p[i][1] if l.has_bias else None
-                pre = ops.conv_fwd(x, self.p[i][0], bias, l.stride, ph, pw)
+                w = self.q(self.p[i][0]) if l.kind != FC else self.p[i][0]
+                pre = ops.conv_fwd(x, w, bias, l.stride, ph, pw)
+                if l.kind != FC:
+                    pre = self.q(pre)
                 self.saved[i] = pre
                 y = ops.act_fwd(pre, l.act)
             elif l.kind == DW:
-                y = ops.dwconv_fwd(x, self.p[i][0], l.stride, l.pad)
+                y = self.q(ops.dwconv_fwd(x, self.p[i][0], l.stride, l.pad))
             elif l.kind == BN:
                 z, mu, var, xhat = ops.bn_fwd(x, self.p[i][0], self.p[i][1], self.cfg["bn_eps"])
                 self.saved[i] = (z, var, xhat)
@@ -59,15 +81,17 @@ class OracleModel:
                 self.s[i][0] = (1 - mom) * self.s[i][0] + mom * mu
                 self.s[i][1] = (1 - mom) * self.s[i][1] + mom * unbiased
                 y = ops.act_fwd(z, l.act)
+                if not (i + 1 < len(self.layers) and self.layers[i + 1].kind == ADD):
+                    y = self.q(y)
             elif l.kind == ACT:
                 y = ops.act_fwd(x, l.act)
             elif l.kind == ADD:
-                y = x + self.out[l.residual_src]
+                y = self.q(x + self.out[l.residual_src])
             elif l.kind == MAXPOOL:
                 y, arg = ops.maxpool_fwd(x)
                 self.saved[i] = arg
             elif l.kind == GAP:
-                y = ops.gap_fwd(x)
+                y = self.q(ops.gap_fwd(x))
             elif l.kind == CE:
                 self.labels = np.asarray(labels)
                 self.logits = x.reshape(x.shape[0], -1).copy()
@@ -96,10 +120,13 @@ class OracleModel:
                 acc(i - 1, ops.softmax_ce_bwd(self.saved[i], self.labels, x.shape))
                 continue
             d = grad.pop(i)
+            if l.kind != FC:
+                d = self.q(d)                    # the gradient as it was stored for this op to read
             if l.kind in (CONV1D, CONV2D, FC):
                 ph, pw = self._pads(l)
                 d = ops.act_bwd(self.saved[i], d, l.act)
-                dx, dw, db = ops.conv_bwd(x, self.p[i][0], d, l.stride, ph, pw, l.has_bias)
+                w = self.q(self.p[i][0]) if l.kind != FC else self.p[i][0]
+                dx, dw, db = ops.conv_bwd(x, w, d, l.stride, ph, pw, l.has_bias)
                 self.g[i][0] = dw
                 if l.has_bias:
                     self.g[i][1] = db
@@ -123,7 +150,8 @@ class OracleModel:
                 acc(i - 1, ops.maxpool_bwd(d, self.saved[i], x.shape))
             elif l.kind == GAP:
                 acc(i - 1, ops.gap_bwd(d, x.shape))
-        return grad.get(idx[0] - 1)
+        g = grad.get(idx[0] - 1)
+        return None if g is None else self.q(g)
 
     # ---- how close the last forward came to a discrete decision ---------------------------------
     def decision_margin(self, a=0, b=None, per_op=False):

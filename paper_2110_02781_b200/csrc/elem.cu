@@ -692,6 +692,11 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ s, __nv_bfloat16* _
         d[i] = __float2bfloat16_rn(s[i]);
 }
 
+__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ s, float* __restrict__ d, long long n) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        d[i] = __bfloat162float(s[i]);
+}
+
 template <typename T> inline bool can_vec(int C, const void* a, const void* b = nullptr, const void* c = nullptr, const void* d = nullptr) {
     return C % VecOf<T>::N == 0 && aligned16(a) && aligned16(b) && aligned16(c) && aligned16(d);
 }
@@ -892,6 +897,10 @@ void sgd_update(float* w, const float* g, float* m, long long n, float lr, float
     const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(snap_dev) && aligned16(snap_host);
     if (v) sgd_kernel<4><<<flat_blocks(n / 4, 256), 256, 0, st>>>(w, g, m, n / 4, lr, mu, wd, first, shadow, snap_dev, snap_host);
     else sgd_kernel<1><<<flat_blocks(n, 256), 256, 0, st>>>(w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
+}
+
+void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st) {
+    bf16_to_f32_kernel<<<flat_blocks(n, 256), 256, 0, st>>>(src, dst, n);
 }
 
 void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st) {

@@ -1,6 +1,8 @@
-// fp32 SIMT contractions: dense convolution (incl. 1x1 / FC / conv1d) forward, data gradient and
-// weight gradient as implicit GEMMs.  The fp32 path has to stay within 1e-4 of a float64
-// reference, which rules tensor cores (tf32 / bf16 inputs) out for it.
+// SIMT contractions: dense convolution (incl. 1x1 / FC / conv1d) forward, data gradient and
+// weight gradient as implicit GEMMs with float accumulation.  The fp32 path has to stay within 1e-4
+// of a float64 reference, which rules tensor cores (tf32 / bf16 inputs) out for it.  The same kernels
+// are instantiated for bfloat16 tensors: they serve the shapes the tensor-core kernels do not take
+// (3 input channels, ragged channel counts).
 //
 // Tiling: 256 threads compute a 128 x BN tile of the output with an 8 x (BN/16) register
 // micro-tile per thread; the reduction dimension is walked 16 at a time through two
@@ -15,12 +17,31 @@ namespace {
 
 constexpr int BK = 16, NT = 256;
 
+// four / one consecutive elements as floats
+__device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 ldg4(const __nv_bfloat16* p) {
+    const uint2 u = __ldg(reinterpret_cast<const uint2*>(p));
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+}
+__device__ __forceinline__ float ldg1(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ldg1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void st4(float* p, float a, float b, float c, float d) { *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d); }
+__device__ __forceinline__ void st4(__nv_bfloat16* p, float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const unsigned*>(&lo), *reinterpret_cast<const unsigned*>(&hi));
+}
+__device__ __forceinline__ void st2(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
+__device__ __forceinline__ void st2(__nv_bfloat16* p, float a, float b) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b); }
+__device__ __forceinline__ void st1(float* p, float a) { *p = a; }
+__device__ __forceinline__ void st1(__nv_bfloat16* p, float a) { *p = __float2bfloat16_rn(a); }
+
+template <typename T>
 struct GemmP {
-    const float* A;        // gathered operand: x (forward) or dy (data gradient)
-    const float* B;        // weights [kh*kw][Cin][Cout]
+    const T* A;            // gathered operand: x (forward) or dy (data gradient)
+    const T* B;            // weights [kh*kw][Cin][Cout]
     const float* bias;     // forward only, nullable
-    const float* addend;   // nullable, shaped like D
-    float* D;
+    const T* addend;       // nullable, shaped like D
+    T* D;
     int M, Kg, Cd;         // GEMM rows, reduction length, output columns
     int Hs, Ws, Cs;        // source tensor: spatial dims and channels
     int Hd, Wd;            // destination tensor spatial dims
@@ -34,8 +55,8 @@ struct RowInfo {
     bool ok;
 };
 
-template <int MODE>
-__device__ __forceinline__ RowInfo make_row(const GemmP& p, int m) {
+template <int MODE, typename T>
+__device__ __forceinline__ RowInfo make_row(const GemmP<T>& p, int m) {
     RowInfo r;
     r.ok = m < p.M;
     const int hw = p.Hd * p.Wd;
@@ -48,8 +69,8 @@ __device__ __forceinline__ RowInfo make_row(const GemmP& p, int m) {
 }
 
 // Offset (in floats) of source element for row `ri` and tap (r, s), channel c; -1 if it is padding.
-template <int MODE>
-__device__ __forceinline__ long long src_offset(const GemmP& p, const RowInfo& ri, int r, int s, int c) {
+template <int MODE, typename T>
+__device__ __forceinline__ long long src_offset(const GemmP<T>& p, const RowInfo& ri, int r, int s, int c) {
     int hs, ws;
     if (MODE == 0) {
         hs = ri.hb + r; ws = ri.wb + s;
@@ -69,8 +90,8 @@ __device__ __forceinline__ float apply_act(float v, int act) {
     return v;
 }
 
-template <int BM, int BN, int MODE>
-__global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
+template <int BM, int BN, int MODE, typename T>
+__global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP<T> p) {
     constexpr int TM = BM / 16, TN = BN / 16;
     constexpr int ITA = BM / 64;                   // float4 loads of A per thread (vector path)
     static_assert(BM == 128 || BM == 64, "row tile");
@@ -101,7 +122,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
                     long long off;
                     if (p.pointwise) off = (long long)(m0 + (tid >> 2) + 64 * i) * p.Cs + k;
                     else off = src_offset<MODE>(p, ri[i], r, s, c);
-                    if (off >= 0) v = __ldg(reinterpret_cast<const float4*>(p.A + off));
+                    if (off >= 0) v = ldg4(p.A + off);
                 }
                 ra[4 * i + 0] = v.x; ra[4 * i + 1] = v.y; ra[4 * i + 2] = v.z; ra[4 * i + 3] = v.w;
             }
@@ -115,7 +136,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
                 if (m < p.M && k < p.Kg) {
                     const RowInfo q = make_row<MODE>(p, m);
                     const long long off = src_offset<MODE>(p, q, r, s, c);
-                    if (off >= 0) v = __ldg(p.A + off);
+                    if (off >= 0) v = ldg1(p.A + off);
                 }
                 ra[i] = v;
             }
@@ -143,12 +164,12 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
                 if (MODE == 0) {                     // B[k][j] = W[k*Cd + j]
                     const int kk = q / (BN / 4), j = j0 + (q % (BN / 4)) * 4, k = k0 + kk;
                     if (k < p.Kg) {
-                        const float* src = p.B + (long long)k * p.Cd + j;
+                        const T* src = p.B + (long long)k * p.Cd + j;
                         if (p.vecB) {
-                            if (j < p.Cd) { const float4 w = __ldg(reinterpret_cast<const float4*>(src)); v[0] = w.x; v[1] = w.y; v[2] = w.z; v[3] = w.w; }
+                            if (j < p.Cd) { const float4 w = ldg4(src); v[0] = w.x; v[1] = w.y; v[2] = w.z; v[3] = w.w; }
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) if (j + e < p.Cd) v[e] = __ldg(src + e);
+                            for (int e = 0; e < 4; ++e) if (j + e < p.Cd) v[e] = ldg1(src + e);
                         }
                     }
                 } else {                             // B[k=(rs,c)][j] = W[(rs*Cd + j)*Cs + c]
@@ -157,14 +178,14 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
                         if (p.vecB) {
                             if (k < p.Kg) {
                                 const int rs = k / p.Cs, c = k - rs * p.Cs;
-                                const float4 w = __ldg(reinterpret_cast<const float4*>(p.B + ((long long)rs * p.Cd + j) * p.Cs + c));
+                                const float4 w = ldg4(p.B + ((long long)rs * p.Cd + j) * p.Cs + c);
                                 v[0] = w.x; v[1] = w.y; v[2] = w.z; v[3] = w.w;
                             }
                         } else {
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 const int ke = k + e;
-                                if (ke < p.Kg) { const int rs = ke / p.Cs, c = ke - rs * p.Cs; v[e] = __ldg(p.B + ((long long)rs * p.Cd + j) * p.Cs + c); }
+                                if (ke < p.Kg) { const int rs = ke / p.Cs, c = ke - rs * p.Cs; v[e] = ldg1(p.B + ((long long)rs * p.Cd + j) * p.Cs + c); }
                             }
                         }
                     }
@@ -237,7 +258,7 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
     }
 
     // epilogue: bias, activation, residual-gradient addend, store (16-byte stores when aligned)
-    float* const Dz = p.D + (long long)blockIdx.z * p.M * p.Cd;
+    T* const Dz = p.D + (long long)blockIdx.z * p.M * p.Cd;
     constexpr int GW = TN >= 4 ? 4 : 2;            // columns per contiguous group
     constexpr int NG = TN / GW;
     const bool vecD = p.alignD && (p.Cd % GW) == 0;
@@ -259,33 +280,34 @@ __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP p) {
             }
             if (vecD) {
                 if constexpr (GW == 4) {
-                    if (p.addend) { const float4 a = __ldg(reinterpret_cast<const float4*>(p.addend + o)); v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w; }
-                    *reinterpret_cast<float4*>(Dz + o) = make_float4(v[0], v[1], v[2], v[3]);
+                    if (p.addend) { const float4 a = ldg4(p.addend + o); v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w; }
+                    st4(Dz + o, v[0], v[1], v[2], v[3]);
                 } else {
-                    if (p.addend) { const float2 a = __ldg(reinterpret_cast<const float2*>(p.addend + o)); v[0] += a.x; v[1] += a.y; }
-                    *reinterpret_cast<float2*>(Dz + o) = make_float2(v[0], v[1]);
+                    if (p.addend) { v[0] += ldg1(p.addend + o); v[1] += ldg1(p.addend + o + 1); }
+                    st2(Dz + o, v[0], v[1]);
                 }
             } else {
 #pragma unroll
                 for (int e = 0; e < GW; ++e)
-                    if (jc + e < p.Cd) Dz[o + e] = v[e] + (p.addend ? __ldg(p.addend + o + e) : 0.f);
+                    if (jc + e < p.Cd) st1(Dz + o + e, v[e] + (p.addend ? ldg1(p.addend + o + e) : 0.f));
             }
         }
     }
 }
 
 // ---- weight gradient ---------------------------------------------------------------------------
+template <typename T>
 struct WgP {
-    const float* X;
-    const float* dY;
+    const T* X;
+    const T* dY;
     float* out;            // dW, or the split partials [S][Kg][Cout]
     int M, Kg, Cout, Cs, Hs, Ws, Ho, Wo, kh, kw, stride, ph, pw;
     int chunk;             // rows of M per split (multiple of 16)
     int vecA, vecB, vecO, pointwise;
 };
 
-template <int BI>
-__global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP p) {
+template <int BI, typename T>
+__global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP<T> p) {
     constexpr int BJ = 64, TM = BI / 16;
     constexpr int LDA = BI + 4, LDB = BJ + 4;
     constexpr int ITA = BK * BI / 4 / NT;          // float4 loads of A per thread (2 or 1)
@@ -318,7 +340,7 @@ __global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP p) {
             for (int t = 0; t < ITA; ++t) {
                 const int m = mrow0 + tid / (BI / 4) + t * (NT / (BI / 4));
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (m < mend && kA < p.Kg) { const long long off = x_offset(m); if (off >= 0) v = __ldg(reinterpret_cast<const float4*>(p.X + off)); }
+                if (m < mend && kA < p.Kg) { const long long off = x_offset(m); if (off >= 0) v = ldg4(p.X + off); }
                 ra[4 * t] = v.x; ra[4 * t + 1] = v.y; ra[4 * t + 2] = v.z; ra[4 * t + 3] = v.w;
             }
         } else {
@@ -326,7 +348,7 @@ __global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP p) {
             for (int t = 0; t < BI / 16; ++t) {
                 const int m = mrow0 + tid / BI + t * (NT / BI);
                 float v = 0.f;
-                if (m < mend && kA < p.Kg) { const long long off = x_offset(m); if (off >= 0) v = __ldg(p.X + off); }
+                if (m < mend && kA < p.Kg) { const long long off = x_offset(m); if (off >= 0) v = ldg1(p.X + off); }
                 ra[t] = v;
             }
         }
@@ -346,13 +368,13 @@ __global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP p) {
         if (p.vecB) {
             const int m = mrow0 + (tid >> 4), j = j0 + (tid & 15) * 4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (m < mend && j < p.Cout) v = __ldg(reinterpret_cast<const float4*>(p.dY + (long long)m * p.Cout + j));
+            if (m < mend && j < p.Cout) v = ldg4(p.dY + (long long)m * p.Cout + j);
             rb[0] = v.x; rb[1] = v.y; rb[2] = v.z; rb[3] = v.w;
         } else {
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 const int m = mrow0 + (tid >> 6) + t * 4, j = j0 + (tid & 63);
-                rb[t] = (m < mend && j < p.Cout) ? __ldg(p.dY + (long long)m * p.Cout + j) : 0.f;
+                rb[t] = (m < mend && j < p.Cout) ? ldg1(p.dY + (long long)m * p.Cout + j) : 0.f;
             }
         }
     };
@@ -506,24 +528,28 @@ inline GemmPlan plan_gemm(long long M, int N, int Kg, bool plain) {
     return gp;
 }
 
-template <int MODE>
-void launch_conv_gemm(GemmP p, float* scratch, cudaStream_t st) {
-    const bool plain = p.act == 0 && scratch != nullptr && (reinterpret_cast<uintptr_t>(p.D) & 15) == 0 &&
+template <int MODE, typename T>
+void launch_conv_gemm(GemmP<T> p, float* scratch, cudaStream_t st) {
+    constexpr bool kF32 = sizeof(T) == 4;
+    const bool plain = kF32 && p.act == 0 && scratch != nullptr && (reinterpret_cast<uintptr_t>(p.D) & 15) == 0 &&
                        (reinterpret_cast<uintptr_t>(p.addend) & 15) == 0;
     const GemmPlan gp = plan_gemm(p.M, p.Cd, p.Kg, plain);
     const TileOpt t = kTiles[gp.tile];
     const dim3 grid((p.M + t.bm - 1) / t.bm, (p.Cd + t.bn - 1) / t.bn, gp.S);
-    float* const out = p.D;
-    const float* const addend = p.addend;
+    T* const out = p.D;
+    const T* const addend = p.addend;
     const float* const bias = p.bias;
     p.kt_per = gp.kt_per;
-    if (gp.S > 1) { p.D = scratch; p.addend = nullptr; p.bias = nullptr; p.alignD = 1; }
-#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) conv_gemm_kernel<BM_, BN_, MODE><<<grid, NT, 0, st>>>(p);
+    if (gp.S > 1) { p.D = reinterpret_cast<T*>(scratch); p.addend = nullptr; p.bias = nullptr; p.alignD = 1; }
+#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) conv_gemm_kernel<BM_, BN_, MODE, T><<<grid, NT, 0, st>>>(p);
     FTP_LAUNCH(128, 128) FTP_LAUNCH(128, 64) FTP_LAUNCH(64, 128) FTP_LAUNCH(64, 64) FTP_LAUNCH(128, 32) FTP_LAUNCH(64, 32)
 #undef FTP_LAUNCH
-    if (gp.S > 1) {
-        const long long count4 = (long long)p.M * p.Cd / 4;
-        split_reduce_add_kernel<<<(unsigned)((count4 + 255) / 256), 256, 0, st>>>(scratch, gp.S, count4, addend, bias, p.Cd, out);
+    if constexpr (kF32) {
+        if (gp.S > 1) {
+            const long long count4 = (long long)p.M * p.Cd / 4;
+            split_reduce_add_kernel<<<(unsigned)((count4 + 255) / 256), 256, 0, st>>>(scratch, gp.S, count4, reinterpret_cast<const float*>(addend), bias, p.Cd,
+                                                                                      reinterpret_cast<float*>(out));
+        }
     }
 }
 
@@ -539,28 +565,64 @@ size_t conv_gemm_scratch_floats(const ConvGeom& g) {
     return nf > nb ? nf : nb;
 }
 
-void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, float* scratch, const ConvGeom& g, int act,
-                  cudaStream_t st) {
-    GemmP p{};
+namespace {
+constexpr int kVec = 4;     // elements per vector access in these kernels (16 bytes of float, 8 of bfloat16)
+template <typename T> inline bool avec(const void* q) { return (reinterpret_cast<uintptr_t>(q) & (kVec * sizeof(T) - 1)) == 0; }
+
+template <typename T>
+void conv_fwd_t(const T* x, const T* w, const float* bias, T* y, float* scratch, const ConvGeom& g, int act, cudaStream_t st) {
+    GemmP<T> p{};
     p.A = x; p.B = w; p.bias = bias; p.addend = nullptr; p.D = y;
     p.M = g.N * g.Ho * g.Wo; p.Kg = g.kh * g.kw * g.Cin; p.Cd = g.Cout;
     p.Hs = g.H; p.Ws = g.W; p.Cs = g.Cin; p.Hd = g.Ho; p.Wd = g.Wo;
     p.kh = g.kh; p.kw = g.kw; p.stride = g.stride; p.ph = g.ph; p.pw = g.pw;
-    p.act = act; p.vecA = (g.Cin % 4 == 0) && a16(x); p.vecB = (g.Cout % 4 == 0) && a16(w); p.alignD = a16(y);
+    p.act = act; p.vecA = (g.Cin % 4 == 0) && avec<T>(x); p.vecB = (g.Cout % 4 == 0) && avec<T>(w); p.alignD = avec<T>(y);
     p.pointwise = is_pointwise(g);
-    launch_conv_gemm<0>(p, scratch, st);
+    launch_conv_gemm<0, T>(p, scratch, st);
 }
 
-void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, float* scratch, const ConvGeom& g,
-                    cudaStream_t st) {
-    GemmP p{};
+template <typename T>
+void conv_dgrad_t(const T* dy, const T* w, const T* addend, T* dx, float* scratch, const ConvGeom& g, cudaStream_t st) {
+    GemmP<T> p{};
     p.A = dy; p.B = w; p.bias = nullptr; p.addend = addend; p.D = dx;
     p.M = g.N * g.H * g.W; p.Kg = g.kh * g.kw * g.Cout; p.Cd = g.Cin;
     p.Hs = g.Ho; p.Ws = g.Wo; p.Cs = g.Cout; p.Hd = g.H; p.Wd = g.W;
     p.kh = g.kh; p.kw = g.kw; p.stride = g.stride; p.ph = g.ph; p.pw = g.pw;
-    p.act = 0; p.vecA = (g.Cout % 4 == 0) && a16(dy); p.vecB = (g.Cout % 4 == 0) && a16(w); p.alignD = a16(dx) && a16(addend);
+    p.act = 0; p.vecA = (g.Cout % 4 == 0) && avec<T>(dy); p.vecB = (g.Cout % 4 == 0) && avec<T>(w); p.alignD = avec<T>(dx) && avec<T>(addend);
     p.pointwise = is_pointwise(g);
-    launch_conv_gemm<1>(p, scratch, st);
+    launch_conv_gemm<1, T>(p, scratch, st);
+}
+
+template <typename T>
+void conv_wgrad_t(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st) {
+    const WgPlan w = plan_wgrad(g);
+    WgP<T> p{};
+    p.X = x; p.dY = dy; p.out = w.S > 1 ? scratch : dw;
+    p.M = g.N * g.Ho * g.Wo; p.Kg = g.kh * g.kw * g.Cin; p.Cout = g.Cout; p.Cs = g.Cin; p.Hs = g.H; p.Ws = g.W;
+    p.Ho = g.Ho; p.Wo = g.Wo; p.kh = g.kh; p.kw = g.kw; p.stride = g.stride; p.ph = g.ph; p.pw = g.pw;
+    p.chunk = w.chunk; p.vecA = (g.Cin % 4 == 0) && avec<T>(x); p.vecB = (g.Cout % 4 == 0) && avec<T>(dy);
+    p.vecO = (g.Cout % 4 == 0) && a16(p.out) && ((long long)p.Kg * g.Cout) % 4 == 0; p.pointwise = is_pointwise(g);
+    const dim3 grid((p.Kg + w.BI - 1) / w.BI, (g.Cout + 63) / 64, w.S);
+    if (w.BI == 128) conv_wgrad_kernel<128, T><<<grid, NT, 0, st>>>(p);
+    else conv_wgrad_kernel<64, T><<<grid, NT, 0, st>>>(p);
+    if (w.S > 1) {
+        const long long count = (long long)p.Kg * g.Cout;
+        split_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, w.S, count, dw);
+    }
+}
+}  // namespace
+
+void conv_fwd_f32(const float* x, const float* w, const float* bias, float* y, float* scratch, const ConvGeom& g, int act, cudaStream_t st) {
+    conv_fwd_t<float>(x, w, bias, y, scratch, g, act, st);
+}
+void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float* dx, float* scratch, const ConvGeom& g, cudaStream_t st) {
+    conv_dgrad_t<float>(dy, w, addend, dx, scratch, g, st);
+}
+void conv_fwd_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, __nv_bfloat16* y, const ConvGeom& g, int act, cudaStream_t st) {
+    conv_fwd_t<__nv_bfloat16>(x, w, bias, y, nullptr, g, act, st);
+}
+void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const __nv_bfloat16* addend, __nv_bfloat16* dx, const ConvGeom& g, cudaStream_t st) {
+    conv_dgrad_t<__nv_bfloat16>(dy, w, addend, dx, nullptr, g, st);
 }
 
 size_t conv_wgrad_scratch_floats(const ConvGeom& g) {
@@ -569,20 +631,10 @@ size_t conv_wgrad_scratch_floats(const ConvGeom& g) {
 }
 
 void conv_wgrad_f32(const float* x, const float* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st) {
-    const WgPlan w = plan_wgrad(g);
-    WgP p{};
-    p.X = x; p.dY = dy; p.out = w.S > 1 ? scratch : dw;
-    p.M = g.N * g.Ho * g.Wo; p.Kg = g.kh * g.kw * g.Cin; p.Cout = g.Cout; p.Cs = g.Cin; p.Hs = g.H; p.Ws = g.W;
-    p.Ho = g.Ho; p.Wo = g.Wo; p.kh = g.kh; p.kw = g.kw; p.stride = g.stride; p.ph = g.ph; p.pw = g.pw;
-    p.chunk = w.chunk; p.vecA = (g.Cin % 4 == 0) && a16(x); p.vecB = (g.Cout % 4 == 0) && a16(dy);
-    p.vecO = (g.Cout % 4 == 0) && a16(p.out) && ((long long)p.Kg * g.Cout) % 4 == 0; p.pointwise = is_pointwise(g);
-    const dim3 grid((p.Kg + w.BI - 1) / w.BI, (g.Cout + 63) / 64, w.S);
-    if (w.BI == 128) conv_wgrad_kernel<128><<<grid, NT, 0, st>>>(p);
-    else conv_wgrad_kernel<64><<<grid, NT, 0, st>>>(p);
-    if (w.S > 1) {
-        const long long count = (long long)p.Kg * g.Cout;
-        split_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, w.S, count, dw);
-    }
+    conv_wgrad_t<float>(x, dy, dw, scratch, g, st);
+}
+void conv_wgrad_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st) {
+    conv_wgrad_t<__nv_bfloat16>(x, dy, dw, scratch, g, st);
 }
 
 }  // namespace ftp

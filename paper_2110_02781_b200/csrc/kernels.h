@@ -28,6 +28,14 @@ void conv_dgrad_f32(const float* dy, const float* w, const float* addend, float*
 size_t conv_wgrad_scratch_floats(const ConvGeom& g);
 void conv_wgrad_f32(const float* x, const float* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st);
 
+// the same kernels on bfloat16 tensors (bf16 weights, float accumulation, float weight gradient)
+void conv_fwd_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* w, const float* bias, __nv_bfloat16* y, const ConvGeom& g,
+                        int act, cudaStream_t st);
+void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const __nv_bfloat16* addend, __nv_bfloat16* dx,
+                          const ConvGeom& g, cudaStream_t st);
+void conv_wgrad_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* dy, float* dw, float* scratch, const ConvGeom& g,
+                          cudaStream_t st);
+
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
 // Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole
 // 128-byte lines; `fold` picks f.  Partials are doubles: [chunks][2][C*f].
@@ -110,6 +118,7 @@ void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, 
 void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
                 __nv_bfloat16* shadow, float* snap_dev, float* snap_host, cudaStream_t st);
 void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st);
+void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st);
 
 int sm_count();
 

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cstring>
 #include <new>
+#include <type_traits>
 #include "model.h"
 
 using namespace ftp;
@@ -214,7 +215,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     }
     m.grad = (float*)bp.take((size_t)m.P * 4);
     m.state_backup = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
-    size_t max_act = 0, red = 0, foldd = 0, dpre = 0, finp = 64, finc = 1;
+    size_t max_act = 0, red = 0, foldd = 0, dpre = 0, finp = 64, finc = 1, fcin = 64;
     for (int i = 0; i < n; ++i) {
         Op& o = m.ops[i];
         const size_t obytes = (size_t)o.out_elems * (o.out_f32 ? 4 : es);
@@ -235,6 +236,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
             if (o.d.act != FTP_ACT_NONE) dpre = std::max(dpre, obytes);
+            if (o.d.kind == FTP_FC) fcin = std::max(fcin, (size_t)o.in_elems);
         } else if (o.d.kind == FTP_DWCONV3x3) {
             red = std::max(red, dwconv_wgrad_scratch_floats(o.g));
             finp = std::max(finp, fin_part_doubles(o.C, 9)); finc = std::max(finc, fin_counter_count(o.C, 9));
@@ -249,6 +251,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     m.red_floats = std::max<size_t>(red, 64); m.red_scratch = (float*)bp.take(m.red_floats * 4);
     m.fold_doubles = std::max<size_t>(foldd, 64); m.fold_scratch = (double*)bp.take(m.fold_doubles * 8);
     m.dpre_bytes = std::max<size_t>(dpre, 256); m.dpre = bp.take(m.dpre_bytes);
+    m.fc_in = (float*)bp.take(fcin * 4); m.fc_din = (float*)bp.take(fcin * 4);
     m.fin.part = (double*)bp.take(finp * 8);
     m.fin_counter_bytes = finc * 4; m.fin.counters = (unsigned*)bp.take(m.fin_counter_bytes);
     m.dlogits = (float*)bp.take((size_t)m.cfg.batch * m.cfg.n_classes * 4);
@@ -298,8 +301,15 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 if (m->cfg.precision == FTP_FP32) {
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
                     conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
-                } else {
-                    return fail(FTP_EUNSUPPORTED, "bf16 contractions are not built yet");
+                } else if constexpr (!std::is_same<T, float>::value) {
+                    if (o.d.kind == FTP_FC) {           // the classifier runs in float on a widened copy of its input
+                        Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, o.in_elems * 2.0 + (o.out_elems + o.w_cnt) * 4.0, fl, 2);
+                        bf16_to_f32((const T*)in, m->fc_in, o.in_elems, st);
+                        conv_fwd_f32(m->fc_in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
+                    } else {
+                        Scope sc(m, st, K_GEMM_BF16_FWD, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 2.0, fl);
+                        conv_fwd_bf16_simt((const T*)in, ar.wb + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (T*)out, o.g, o.d.act, st);
+                    }
                 }
                 break;
             }
@@ -384,20 +394,40 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
-                if (m->cfg.precision != FTP_FP32) return fail(FTP_EUNSUPPORTED, "bf16 contractions are not built yet");
-                const float* d = (const float*)go;
-                if (o.d.act != FTP_ACT_NONE || o.b_off >= 0) {
-                    float* dpre = o.d.act != FTP_ACT_NONE ? (float*)m->dpre : nullptr;
-                    Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 4.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
-                    act_bias_bwd<float>(d, (const float*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
+                if (m->cfg.precision == FTP_FP32 || o.d.kind == FTP_FC) {
+                    const bool widened = m->cfg.precision != FTP_FP32;        // classifier of a bf16 model: float on widened copies
+                    FTP_REQUIRE(!(widened && addend), FTP_EUNSUPPORTED, "a residual source feeding the classifier is not supported in bf16 models");
+                    const float* x = widened ? m->fc_in : (const float*)in;
+                    const float* d = (const float*)go;
+                    if (o.d.act != FTP_ACT_NONE || o.b_off >= 0) {
+                        float* dpre = o.d.act != FTP_ACT_NONE ? (float*)m->dpre : nullptr;
+                        Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 4.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
+                        act_bias_bwd<float>(d, (const float*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
+                                            o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
+                        if (dpre) d = dpre;
+                    }
+                    { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
+                      conv_wgrad_f32(x, d, gr + o.w_off, m->red_scratch, o.g, st); }
+                    if (gi) {
+                        Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
+                        conv_dgrad_f32(d, ar.w + o.w_off, widened ? nullptr : (const float*)addend, widened ? m->fc_din : (float*)gi, m->red_scratch, o.g, st);
+                        if (widened) f32_to_bf16(m->fc_din, (__nv_bfloat16*)gi, o.in_elems, st);
+                    }
+                } else if constexpr (!std::is_same<T, float>::value) {
+                    const T* d = (const T*)go;
+                    if (o.d.act != FTP_ACT_NONE || o.b_off >= 0) {
+                        T* dpre = o.d.act != FTP_ACT_NONE ? (T*)m->dpre : nullptr;
+                        Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 2.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
+                        act_bias_bwd<T>(d, (const T*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
                                         o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
-                    if (dpre) d = dpre;
-                }
-                { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
-                  conv_wgrad_f32((const float*)in, d, gr + o.w_off, m->red_scratch, o.g, st); }
-                if (gi) {
-                    Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl);
-                    conv_dgrad_f32(d, ar.w + o.w_off, (const float*)addend, (float*)gi, m->red_scratch, o.g, st);
+                        if (dpre) d = dpre;
+                    }
+                    { Scope sc(m, st, K_GEMM_BF16_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
+                      conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, m->red_scratch, o.g, st); }
+                    if (gi) {
+                        Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
+                        conv_dgrad_bf16_simt(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.g, st);
+                    }
                 }
                 break;
             }

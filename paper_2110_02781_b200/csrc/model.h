@@ -66,6 +66,7 @@ struct ftp_model {
     double* fold_scratch; size_t fold_doubles;
     ftp::FinScratch fin; size_t fin_counter_bytes;
     void* dpre; size_t dpre_bytes;
+    float* fc_in; float* fc_din;                  // bf16 models: the classifier's input and input gradient widened to float
     float* dlogits; float* per_sample; float* loss_dev; int32_t* labels_dev; void* input_dev; float* state_backup;
     float* pinned; size_t pinned_bytes;
     // run-time state of the last forward of each range

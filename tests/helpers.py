@@ -21,7 +21,7 @@ def _depths(layers):
     return out
 
 
-def clear_batch(om, idx, cfg, first_try=0, margin=MARGIN, tries=3000):
+def clear_batch(om, idx, cfg, first_try=0, margin=MARGIN, tries=3000, transform=None):
     """Seeded rejection: the first batch (by draw index) whose oracle forward keeps every value of
     op i at least margin * depth_i (relative) away from an activation kink or a max-pool tie,
     depth_i being the number of contractions before it: float32 rounding noise grows about linearly
@@ -31,6 +31,8 @@ def clear_batch(om, idx, cfg, first_try=0, margin=MARGIN, tries=3000):
     depth = _depths(om.layers)
     for t in range(first_try, first_try + tries):
         x, y = synth.make_batch(idx, cfg, t)
+        if transform is not None:
+            x = transform(x)            # e.g. rounding to the storage type the device path reads
         keep = [[v.copy() for v in s] for s in om.s]
         om.forward(0, om.L, x, y)
         om.s = keep

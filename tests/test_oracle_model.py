@@ -163,3 +163,36 @@ def test_snapshot_layout():
     u0 = synth.flat_unit_params(ls, synth.init_params(9, ls), 0)
     assert np.array_equal(snap[:u0.size], u0)
     assert np.array_equal(np.concatenate([m.snapshot(0, 1), m.snapshot(1, m.L)]), snap)
+
+
+# ---- the bf16 storage mode of the oracle (configs 3-5 fix bf16 activations and weights) ----------------
+def test_bf16_rounding_matches_the_library_conversion():
+    import torch
+    from oracle.model import round_bf16
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal(200000) * 10.0 ** rng.uniform(-6, 6, 200000)
+    ref = torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(round_bf16(x), ref)
+    ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -1.0 - 2.0 ** -8])      # halfway cases go to even
+    assert np.array_equal(round_bf16(ties), [1.0, 1.0 + 2.0 ** -6, -1.0])
+
+
+@pytest.mark.parametrize("net", [synth.tiny_mbv2, synth.tiny_vgg])
+def test_bf16_storage_mode(net):
+    from oracle.model import round_bf16
+    ls, cfg = net(precision=1)
+    x, y = synth.make_batch(9, cfg)
+    x = round_bf16(x)
+    q = oracle.OracleModel(ls, cfg, synth.init_params(9, ls), synth.init_state(ls))
+    f = oracle.OracleModel(ls, dict(cfg, precision=0), synth.init_params(9, ls), synth.init_state(ls))
+    assert q.quantised and not f.quantised
+    lq, lf = q.step([0, q.L], x, y), f.step([0, f.L], x, y)
+    assert abs(lq - lf) < 2e-2 * abs(lf) and lq != lf              # close to, but not, the float64 run
+    for i, l in enumerate(ls):                                     # what is stored is representable in bf16
+        if l.kind not in (synth.KIND["FC"], synth.KIND["SOFTMAX_CE"]) and \
+                not (i + 1 < len(ls) and ls[i + 1].kind == synth.KIND["ADD_RESIDUAL"]):
+            assert np.array_equal(q.out[i], round_bf16(q.out[i])), i
+    s = oracle.OracleModel(ls, cfg, synth.init_params(9, ls), synth.init_state(ls))   # split == unsplit still holds
+    assert s.step([0, 1, q.L - 1, q.L], x, y) == lq
+    for u in range(q.L):
+        assert np.array_equal(s.unit_params(u), q.unit_params(u))
