@@ -697,6 +697,21 @@ __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ s, float* _
         d[i] = __bfloat162float(s[i]);
 }
 
+// wt[n][k] = bf16(w[k][n]) through a 32 x 32 shared-memory tile
+__global__ void transpose_f32_to_bf16_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ wt, int K, int N) {
+    __shared__ float tile[32][33];
+    const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const int k = k0 + r, n = n0 + threadIdx.x;
+        tile[r][threadIdx.x] = (k < K && n < N) ? w[(long long)k * N + n] : 0.f;
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const int n = n0 + r, k = k0 + threadIdx.x;
+        if (n < N && k < K) wt[(long long)n * K + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+    }
+}
+
 template <typename T> inline bool can_vec(int C, const void* a, const void* b = nullptr, const void* c = nullptr, const void* d = nullptr) {
     return C % VecOf<T>::N == 0 && aligned16(a) && aligned16(b) && aligned16(c) && aligned16(d);
 }
@@ -897,6 +912,10 @@ void sgd_update(float* w, const float* g, float* m, long long n, float lr, float
     const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(snap_dev) && aligned16(snap_host);
     if (v) sgd_kernel<4><<<flat_blocks(n / 4, 256), 256, 0, st>>>(w, g, m, n / 4, lr, mu, wd, first, shadow, snap_dev, snap_host);
     else sgd_kernel<1><<<flat_blocks(n, 256), 256, 0, st>>>(w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
+}
+
+void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, cudaStream_t st) {
+    transpose_f32_to_bf16_kernel<<<dim3((N + 31) / 32, (K + 31) / 32), dim3(32, 8), 0, st>>>(w, wt, K, N);
 }
 
 void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st) {

@@ -1,0 +1,254 @@
+// bf16 contractions on the 5th-generation tensor cores (sm_100a): D[M,N] = A[M,K] * B[N,K]^T with both
+// operands K-major in global memory, float accumulation in tensor memory, bf16 output.
+//
+// One CTA computes one 128 x BN output tile.  Warp 0 (one elected thread) streams 128 x 64 and BN x 64
+// operand tiles into a ring of shared-memory stages with TMA (128-byte swizzle, out-of-range rows and
+// columns filled with zeros, no multicast); warp 1 allocates BN columns of tensor memory and, through one
+// thread, issues tcgen05.mma (M = 128, N = BN, K = 16) four times per stage, releasing the stage with
+// tcgen05.commit; warps 2-5 wait for the last commit, read the accumulator with tcgen05.ld (each warp its
+// own 32 lanes), add the optional addend, convert and store.  Every wait on an mbarrier is bounded: when it
+// runs out the kernel records a code in an error word, lets its own copies land, frees its tensor memory
+// and returns; the host reports FTP_ETIMEOUT.
+#include <cuda.h>
+#include "kernels.h"
+
+namespace ftp {
+namespace {
+
+constexpr int TC_BM = 128, TC_BK = 64, TC_STAGES = 3, TC_THREADS = 192;
+constexpr unsigned long long TC_WAIT_NS = 2000000000ull;      // two seconds
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count)); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and an error code) when the phase did not complete in time.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
+    if (mbar_test(bar, parity)) return true;
+    const unsigned long long t0 = gtime();
+    while (true) {
+        if (mbar_test(bar, parity)) return true;
+        if (*((volatile int*)err) != 0) return false;                     // another role already gave up
+        if (gtime() - t0 > TC_WAIT_NS) { atomicCAS(err, 0, code); return false; }
+        __nanosleep(64);
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// Shared-memory operand descriptor, K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);          // start address
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused with swizzle; canonical value 1)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                          // layout: 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
+          "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+          "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct TcParams {
+    __nv_bfloat16* D;
+    const __nv_bfloat16* addend;   // nullable, shaped like D
+    int M, N, K;
+    int* err;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                                                                const TcParams p) {
+    constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = BN * TC_BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ __align__(8) unsigned long long bars[2 * TC_STAGES + 1];
+    __shared__ uint32_t tmem_base;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * TC_BM;
+    const int num_kb = (p.K + TC_BK - 1) / TC_BK;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- producer: TMA loads into the stage ring ----
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % TC_STAGES;
+                const uint32_t ph = (kb / TC_STAGES) & 1;
+                if (kb >= TC_STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 1)) break;
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
+                mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+                tma_load_2d(sa, &mapA, kb * TC_BK, m0, full0 + 8 * s);
+                tma_load_2d(sb, &mapB, kb * TC_BK, n0, full0 + 8 * s);
+                issued = kb + 1;
+            }
+            if (*((volatile int*)p.err) != 0) {
+                // error path: let the copies already issued land before the block's memory is released
+                for (int kb = max(0, issued - TC_STAGES); kb < issued; ++kb) {
+                    const unsigned long long t0 = gtime();
+                    while (!mbar_test(full0 + 8 * (kb % TC_STAGES), (kb / TC_STAGES) & 1) && gtime() - t0 < 1000000ull) __nanosleep(128);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % TC_STAGES;
+                const uint32_t ph = (kb / TC_STAGES) & 1;
+                ok = mbar_wait(full0 + 8 * s, ph, p.err, 2);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
+                const uint64_t ad = umma_desc_k_sw128(sa), bd = umma_desc_k_sw128(sb);
+#pragma unroll
+                for (int k = 0; k < TC_BK / 16; ++k)                 // 16 bf16 = 32 bytes along K inside the swizzle atom
+                    umma_bf16(tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(empty0 + 8 * s);                         // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(accum);                              // accumulator complete
+        }
+    } else {
+        // ---- epilogue: warps 2..5 own tensor-memory lanes 32*(warp%4) .. +31 ----
+        const int q = warp & 3;
+        if (mbar_wait(accum, 0, p.err, 3)) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int m = m0 + q * 32 + lane;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+                const int nb = n0 + c * 32;
+                if (m < p.M) {
+                    __nv_bfloat16* drow = p.D + (long long)m * p.N + nb;
+                    const __nv_bfloat16* arow = p.addend ? p.addend + (long long)m * p.N + nb : nullptr;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {                    // 8 columns = 16 bytes per store
+                        if (nb + g * 8 < p.N) {
+                            float v[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[g * 8 + e]);
+                            if (arow) {
+                                const uint4 a = __ldg(reinterpret_cast<const uint4*>(arow + g * 8));
+                                const unsigned au[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) { v[2 * e] += __uint_as_float(au[e] << 16); v[2 * e + 1] += __uint_as_float(au[e] & 0xffff0000u); }
+                            }
+                            unsigned o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) { const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]); o[e] = *reinterpret_cast<const unsigned*>(&h); }
+                            *reinterpret_cast<uint4*>(drow + g * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// rows x cols bf16 matrix, cols contiguous; box = 64 columns x box_rows rows, 128-byte swizzle, zero fill
+bool make_map_2d(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K, int* err,
+               cudaStream_t st) {
+    CUtensorMap ma, mb;
+    if (!make_map_2d(&ma, A, M, K, TC_BM) || !make_map_2d(&mb, B, N, K, BN)) return false;
+    constexpr int smem = TC_STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+        configured = true;
+    }
+    TcParams p{D, addend, M, N, K, err};
+    tc_gemm_tn_kernel<BN><<<dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), TC_THREADS, smem, st>>>(ma, mb, p);
+    return true;
+}
+
+}  // namespace
+
+bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend) {
+    auto a16 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+    return M >= 1 && N % 8 == 0 && K % 8 == 0 && N >= 8 && K >= 8 && a16(A) && a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
+}
+
+bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K, int* err,
+                cudaStream_t st) {
+    if (N > 64) return launch_tn<128>(A, B, addend, D, M, N, K, err, st);
+    if (N > 32) return launch_tn<64>(A, B, addend, D, M, N, K, err, st);
+    return launch_tn<32>(A, B, addend, D, M, N, K, err, st);
+}
+
+}  // namespace ftp

@@ -36,6 +36,14 @@ void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const
 void conv_wgrad_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* dy, float* dw, float* scratch, const ConvGeom& g,
                           cudaStream_t st);
 
+// ---- tensor-core contraction (gemm_tc.cu): D[M,N] = A[M,K] * B[N,K]^T (+ addend), all bf16, both operands with K
+// contiguous.  tc_gemm_supported: channel counts multiples of 8, 16-byte aligned pointers, driver entry point found.
+// err: device int, stays 0 unless a bounded wait inside the kernel ran out.  Returns false if nothing was launched.
+bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
+bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K,
+                int* err, cudaStream_t st);
+void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, cudaStream_t st);   // wt[n][k] = bf16(w[k][n])
+
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
 // Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole
 // 128-byte lines; `fold` picks f.  Partials are doubles: [chunks][2][C*f].

@@ -29,8 +29,8 @@ struct Bump {
 const char* kKernelNames[K_COUNT] = {
     "conv_fwd_f32", "conv_dgrad_f32", "conv_wgrad_f32", "bn_stats", "bn_finalize", "bn_apply", "bn_bwd_reduce",
     "bn_bwd_finalize", "bn_bwd_apply", "act_bias_bwd", "dw_fwd", "dw_dgrad", "dw_wgrad", "maxpool_fwd", "maxpool_bwd",
-    "gap_fwd", "gap_bwd", "softmax_ce", "sgd", "act_fwd", "act_bwd", "copy", "gemm_bf16_fwd", "gemm_bf16_dgrad",
-    "gemm_bf16_wgrad"};
+    "gap_fwd", "gap_bwd", "softmax_ce", "sgd", "act_fwd", "act_bwd", "copy", "tc_gemm_bf16_fwd", "tc_gemm_bf16_dgrad",
+    "tc_gemm_bf16_wgrad", "conv_fwd_bf16_simt", "conv_dgrad_bf16_simt", "conv_wgrad_bf16_simt"};
 
 // Brackets one launcher call with events when tracing is on.
 struct Scope {
@@ -212,6 +212,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         a.m = (float*)bp.take((size_t)m.P * 4);
         a.run = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
         a.wb = m.cfg.precision == FTP_BF16 ? (__nv_bfloat16*)bp.take((size_t)m.P * 2) : nullptr;
+        a.wbt = m.cfg.precision == FTP_BF16 ? (__nv_bfloat16*)bp.take((size_t)m.P * 2) : nullptr;
     }
     m.grad = (float*)bp.take((size_t)m.P * 4);
     m.state_backup = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
@@ -251,6 +252,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     m.red_floats = std::max<size_t>(red, 64); m.red_scratch = (float*)bp.take(m.red_floats * 4);
     m.fold_doubles = std::max<size_t>(foldd, 64); m.fold_scratch = (double*)bp.take(m.fold_doubles * 8);
     m.dpre_bytes = std::max<size_t>(dpre, 256); m.dpre = bp.take(m.dpre_bytes);
+    m.tc_err = (int*)bp.take(256);
     m.fc_in = (float*)bp.take(fcin * 4); m.fc_din = (float*)bp.take(fcin * 4);
     m.fin.part = (double*)bp.take(finp * 8);
     m.fin_counter_bytes = finc * 4; m.fin.counters = (unsigned*)bp.take(m.fin_counter_bytes);
@@ -269,6 +271,19 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         cudaError_t e_ = (call);                                                           \
         if (e_ != cudaSuccess) return fail(FTP_ECUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
     } while (0)
+
+bool is_pointwise_op(const Op& o) {
+    return o.d.kind == FTP_CONV2D && o.g.kh == 1 && o.g.kw == 1 && o.g.stride == 1 && o.g.ph == 0 && o.d.act == FTP_ACT_NONE && o.b_off < 0;
+}
+
+// bf16 models: rebuild the transposed bf16 copy of every 1x1 convolution of units [a, b) from the float masters
+void refresh_transposed(ftp_model* m, int a, int b, cudaStream_t st) {
+    for (int i = m->unit_first[a]; i <= m->unit_last[b - 1]; ++i) {
+        const Op& o = m->ops[i];
+        const Arena& ar = m->arena[m->owner[o.d.unit]];
+        if (ar.wbt && is_pointwise_op(o)) transpose_f32_to_bf16(ar.w + o.w_off, ar.wbt + o.w_off, o.C, o.Co, st);
+    }
+}
 
 ftp_status check_launches(const char* where) {
     const cudaError_t e = cudaGetLastError();
@@ -308,7 +323,10 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                         conv_fwd_f32(m->fc_in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                     } else {
                         Scope sc(m, st, K_GEMM_BF16_FWD, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 2.0, fl);
-                        conv_fwd_bf16_simt((const T*)in, ar.wb + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (T*)out, o.g, o.d.act, st);
+                        const bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, ar.wbt + o.w_off, out, nullptr) &&
+                                        tc_gemm_tn((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, (int)Mout, o.Co, o.C, m->tc_err, st);
+                        if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_FWD_BF16_SIMT;
+                        if (!tc) conv_fwd_bf16_simt((const T*)in, ar.wb + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (T*)out, o.g, o.d.act, st);
                     }
                 }
                 break;
@@ -422,11 +440,15 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                                         o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                         if (dpre) d = dpre;
                     }
-                    { Scope sc(m, st, K_GEMM_BF16_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
+                    { Scope sc(m, st, K_CONV_WGRAD_BF16_SIMT, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
                       conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, m->red_scratch, o.g, st); }
                     if (gi) {
                         Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
-                        conv_dgrad_bf16_simt(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.g, st);
+                        // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the canonical weight layout already has K = cout contiguous
+                        const bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.C, o.Co, d, ar.wb + o.w_off, gi, addend) &&
+                                        tc_gemm_tn(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, (int)Mout, o.C, o.Co, m->tc_err, st);
+                        if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_DGRAD_BF16_SIMT;
+                        if (!tc) conv_dgrad_bf16_simt(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.g, st);
                     }
                 }
                 break;
@@ -503,6 +525,7 @@ ftp_status sgd_range(ftp_model* m, int a, int b, float lr, float* snap_dev, floa
         for (int k = u; k < v; ++k) m->mom_init[k] = 1;
         u = v;
     }
+    if (m->cfg.precision == FTP_BF16) refresh_transposed(m, a, b, st);
     return check_launches("sgd_step");
 }
 
@@ -552,7 +575,7 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         s = fail(FTP_ENOMEM, "build_model: workspace too small (need %zu device and %zu pinned bytes)", need, pneed);
     if (s != FTP_OK) { delete m; return s; }
     m->pinned = (float*)pinned_ws; m->pinned_bytes = pinned_bytes;
-    if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess) {     // ticket counters start at zero
+    if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess || cudaMemset(m->tc_err, 0, 256) != cudaSuccess) {     // ticket counters start at zero
         const ftp_status e = fail(FTP_ECUDA, "build_model: clearing the ticket counters failed: %s", cudaGetErrorString(cudaGetLastError()));
         delete m;
         return e;
@@ -634,7 +657,11 @@ extern "C" ftp_status ftp_set_tensor(ftp_model* m, int32_t which, int32_t unit, 
     CUDA_OK(cudaMemcpyAsync(dst, src, (size_t)count * 4, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
     if (which == FTP_T_WEIGHTS) {
         const Arena& ar = m->arena[m->owner[unit]];
-        if (ar.wb) { Scope sc(m, st, K_COPY, unit, -1, 2, 6.0 * count, 0.0); f32_to_bf16(dst, ar.wb + m->unit_p_off[unit], count, st); }
+        if (ar.wb) {
+            Scope sc(m, st, K_COPY, unit, -1, 2, 6.0 * count, 0.0);
+            f32_to_bf16(dst, ar.wb + m->unit_p_off[unit], count, st);
+            refresh_transposed(m, unit, unit + 1, st);
+        }
         m->mom_init[unit] = 0;
     } else if (which == FTP_T_MOMENTUM) m->mom_init[unit] = 1;
     if (!src_is_device) CUDA_OK(cudaStreamSynchronize(st));
@@ -712,8 +739,12 @@ extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t*
     if (s != FTP_OK) return s;
     if (loss_host) {
         CUDA_OK(cudaMemcpyAsync(m->pinned, m->loss_dev, 4, cudaMemcpyDeviceToHost, st));
+        CUDA_OK(cudaMemcpyAsync(m->pinned + 1, m->tc_err, 4, cudaMemcpyDeviceToHost, st));
         CUDA_OK(cudaStreamSynchronize(st));
         *loss_host = m->pinned[0];
+        int code;
+        memcpy(&code, m->pinned + 1, 4);
+        FTP_REQUIRE(code == 0, FTP_ETIMEOUT, "train_step: a bounded wait inside a tensor-core kernel ran out (code %d)", code);
     }
     return FTP_OK;
 }
@@ -794,6 +825,7 @@ extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int
                 CUDA_OK(cudaMemcpyAsync(to.w + po, from.w + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
                 CUDA_OK(cudaMemcpyAsync(to.m + po, from.m + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
                 if (to.wb) CUDA_OK(cudaMemcpyAsync(to.wb + po, from.wb + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
+                if (to.wbt) CUDA_OK(cudaMemcpyAsync(to.wbt + po, from.wbt + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
             }
             if (sc_) CUDA_OK(cudaMemcpyAsync(to.run + so, from.run + so, (size_t)sc_ * 4, cudaMemcpyDeviceToDevice, st));
         }

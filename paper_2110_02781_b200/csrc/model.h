@@ -12,7 +12,7 @@ enum KernelId {
     K_CONV_FWD_F32 = 0, K_CONV_DGRAD_F32, K_CONV_WGRAD_F32, K_BN_STATS, K_BN_FINALIZE, K_BN_APPLY, K_BN_BWD_REDUCE,
     K_BN_BWD_FINALIZE, K_BN_BWD_APPLY, K_ACT_BIAS_BWD, K_DW_FWD, K_DW_DGRAD, K_DW_WGRAD, K_MAXPOOL_FWD,
     K_MAXPOOL_BWD, K_GAP_FWD, K_GAP_BWD, K_SOFTMAX_CE, K_SGD, K_ACT_FWD, K_ACT_BWD, K_COPY, K_GEMM_BF16_FWD,
-    K_GEMM_BF16_DGRAD, K_GEMM_BF16_WGRAD, K_COUNT
+    K_GEMM_BF16_DGRAD, K_GEMM_BF16_WGRAD, K_CONV_FWD_BF16_SIMT, K_CONV_DGRAD_BF16_SIMT, K_CONV_WGRAD_BF16_SIMT, K_COUNT
 };
 
 struct Op {
@@ -39,7 +39,8 @@ struct Arena {
     float* w;
     float* m;
     float* run;
-    __nv_bfloat16* wb;
+    __nv_bfloat16* wb;       // bf16 copy of w, same layout
+    __nv_bfloat16* wbt;      // bf16 copy with every 1x1-convolution matrix transposed ([cout][cin]): the forward's K-major B operand
 };
 
 struct TraceSlot { cudaEvent_t e0, e1; ftp_trace_rec rec; };
@@ -66,6 +67,7 @@ struct ftp_model {
     double* fold_scratch; size_t fold_doubles;
     ftp::FinScratch fin; size_t fin_counter_bytes;
     void* dpre; size_t dpre_bytes;
+    int* tc_err;                                  // device word set by a tensor-core kernel whose bounded wait ran out
     float* fc_in; float* fc_din;                  // bf16 models: the classifier's input and input gradient widened to float
     float* dlogits; float* per_sample; float* loss_dev; int32_t* labels_dev; void* input_dev; float* state_backup;
     float* pinned; size_t pinned_bytes;

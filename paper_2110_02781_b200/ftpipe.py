@@ -205,7 +205,7 @@ class Model:
         self.act_dtype = torch.bfloat16 if cfg["precision"] == BF16 else torch.float32
 
     def close(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:        # lib is None while the interpreter shuts down
             lib.ftp_destroy_model(self.h)
             self.h = None
 
