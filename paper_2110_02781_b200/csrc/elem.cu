@@ -223,28 +223,33 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
     }
 }
 
+// z = act(((y - mean) - mean_lo) * scale + shift) (+ residual) on the folded view: grid (column tiles, row chunks),
+// block (32, 8).  A thread keeps the constants of its V channels in registers and walks the rows of its chunk, so
+// the only memory traffic per element is the streamed tensors themselves.
 template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ y, const T* __restrict__ res, T* __restrict__ z,
-                                                       long long nvec, int C, const float* __restrict__ scale,
+                                                       int rows, int cols, int rpc, int C, const float* __restrict__ scale,
                                                        const float* __restrict__ shift, const float* __restrict__ mean,
                                                        const float* __restrict__ mean_lo, int act) {
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)((i * V) % C);
-        float v[V], sc[V], sh[V], mu[V], ml[V];
-        ldv<V>(y + i * V, v);
-        ldtab<V>(scale + c, sc);
-        ldtab<V>(shift + c, sh);
-        ldtab<V>(mean + c, mu);
-        ldtab<V>(mean_lo + c, ml);
+    const int col = (blockIdx.x * 32 + threadIdx.x) * V;
+    if (col >= cols) return;
+    const int c = col % C;
+    float sc[V], sh[V], mu[V], ml[V];
+    ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml);
+    const int r0 = blockIdx.y * rpc, r1 = min(rows, r0 + rpc);
+    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+        const long long off = (long long)r * cols + col;
+        float v[V];
+        ldv<V>(y + off, v);
 #pragma unroll
         for (int e = 0; e < V; ++e) v[e] = act_f(bn_z(v[e], mu[e], ml[e], sc[e], sh[e]), act);
         if (res) {
-            float r[V];
-            ldv<V>(res + i * V, r);
+            float q[V];
+            ldv<V>(res + off, q);
 #pragma unroll
-            for (int e = 0; e < V; ++e) v[e] += r[e];
+            for (int e = 0; e < V; ++e) v[e] += q[e];
         }
-        stv<V>(z + i * V, v);
+        stv<V>(z + off, v);
     }
 }
 
@@ -287,20 +292,26 @@ __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int c
     }
 }
 
+// dy = a * ((g - b) - xhat * c) (+ addend), g = dz masked by the activation; same thread layout as bn_apply_kernel
 template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__ dz, const T* __restrict__ y, const T* __restrict__ addend,
-                                                           T* __restrict__ dy, long long nvec, int C, const float* __restrict__ scale,
+                                                           T* __restrict__ dy, int rows, int cols, int rpc, int C, const float* __restrict__ scale,
                                                            const float* __restrict__ shift, const float* __restrict__ mean,
                                                            const float* __restrict__ mean_lo, const float* __restrict__ rstd,
                                                            const float* __restrict__ coef, int act) {
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)((i * V) % C);
-        float d[V], v[V], sc[V], sh[V], mu[V], ml[V], rs[V], ca[V], bh[V], bl[V], ch[V], cl[V], o[V];
-        ldv<V>(dz + i * V, d);
-        ldv<V>(y + i * V, v);
-        ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml); ldtab<V>(rstd + c, rs);
-        ldtab<V>(coef + c, ca); ldtab<V>(coef + C + c, bh); ldtab<V>(coef + 2 * C + c, bl);
-        ldtab<V>(coef + 3 * C + c, ch); ldtab<V>(coef + 4 * C + c, cl);
+    const int col = (blockIdx.x * 32 + threadIdx.x) * V;
+    if (col >= cols) return;
+    const int c = col % C;
+    float sc[V], sh[V], mu[V], ml[V], rs[V], ca[V], bh[V], bl[V], ch[V], cl[V];
+    ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml); ldtab<V>(rstd + c, rs);
+    ldtab<V>(coef + c, ca); ldtab<V>(coef + C + c, bh); ldtab<V>(coef + 2 * C + c, bl);
+    ldtab<V>(coef + 3 * C + c, ch); ldtab<V>(coef + 4 * C + c, cl);
+    const int r0 = blockIdx.y * rpc, r1 = min(rows, r0 + rpc);
+    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+        const long long off = (long long)r * cols + col;
+        float d[V], v[V], o[V];
+        ldv<V>(dz + off, d);
+        ldv<V>(y + off, v);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
             const float cen = (v[e] - mu[e]) - ml[e];
@@ -313,11 +324,11 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
         }
         if (addend) {
             float a[V];
-            ldv<V>(addend + i * V, a);
+            ldv<V>(addend + off, a);
 #pragma unroll
             for (int e = 0; e < V; ++e) o[e] += a[e];
         }
-        stv<V>(dy + i * V, o);
+        stv<V>(dy + off, o);
     }
 }
 
@@ -768,14 +779,13 @@ void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, 
 }
 
 template <typename T>
-void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift,
+void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
               const float* mean, const float* mean_lo, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    const long long n = M * C;
-    if (can_vec<T>(C, y, residual, z) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo))
-        bn_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(y, residual, z, n / V, C, scale, shift, mean, mean_lo, act);
+    if (fp.vec == V && aligned16(y) && aligned16(residual) && aligned16(z) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo))
+        bn_apply_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(y, residual, z, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, act);
     else
-        bn_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(y, residual, z, n, C, scale, shift, mean, mean_lo, act);
+        bn_apply_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(y, residual, z, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, act);
 }
 
 template <typename T>
@@ -796,14 +806,14 @@ void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int
 }
 
 template <typename T>
-void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale, const float* shift,
+void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
                   const float* mean, const float* mean_lo, const float* rstd, const float* coef, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    const long long n = M * C;
-    if (can_vec<T>(C, dz, y, addend, dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd) && aligned16(coef))
-        bn_bwd_apply_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(dz, y, addend, dy, n / V, C, scale, shift, mean, mean_lo, rstd, coef, act);
+    if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(addend) && aligned16(dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) &&
+        aligned16(mean_lo) && aligned16(rstd) && aligned16(coef))
+        bn_bwd_apply_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
     else
-        bn_bwd_apply_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(dz, y, addend, dy, n, C, scale, shift, mean, mean_lo, rstd, coef, act);
+        bn_bwd_apply_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
 }
 
 template <typename T>
@@ -928,11 +938,11 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
 
 #define FTP_INSTANTIATE(T)                                                                                              \
     template void bn_stats<T>(const T*, long long, int, const FoldPlan&, double*, cudaStream_t);                          \
-    template void bn_apply<T>(const T*, const T*, T*, long long, int, const float*, const float*, const float*,             \
+    template void bn_apply<T>(const T*, const T*, T*, long long, int, const FoldPlan&, const float*, const float*, const float*, \
                               const float*, int, cudaStream_t);                                                            \
     template void bn_bwd_reduce<T>(const T*, const T*, long long, int, const FoldPlan&, const float*, const float*,         \
                                    const float*, const float*, const float*, int, double*, cudaStream_t);                  \
-    template void bn_bwd_apply<T>(const T*, const T*, const T*, T*, long long, int, const float*, const float*,             \
+    template void bn_bwd_apply<T>(const T*, const T*, const T*, T*, long long, int, const FoldPlan&, const float*, const float*, \
                                   const float*, const float*, const float*, const float*, int, cudaStream_t);              \
     template void act_bias_bwd<T>(const T*, const T*, T*, long long, int, int, const FoldPlan&, double*, float*,            \
                                   const FinScratch&, cudaStream_t);                                                                           \

@@ -625,6 +625,10 @@ void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const
     conv_dgrad_t<__nv_bfloat16>(dy, w, addend, dx, nullptr, g, st);
 }
 
+void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st) {
+    split_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(partial, S, count, out);
+}
+
 size_t conv_wgrad_scratch_floats(const ConvGeom& g) {
     const WgPlan w = plan_wgrad(g);
     return w.S > 1 ? (size_t)w.S * g.kh * g.kw * g.Cin * g.Cout : 0;

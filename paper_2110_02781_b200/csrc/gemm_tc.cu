@@ -193,6 +193,131 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
 }
 
+// Shared-memory operand descriptor, MN-major, 128-byte swizzle: a 64 x 64 slab is 64 rows (K) of 128 bytes (64 MN
+// elements); 8-row groups are 1024 bytes apart (stride offset), the next 64 MN elements start slab_bytes further
+// (leading offset).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t slab_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((slab_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+struct TcWgParams {
+    float* out;          // partials [S][Mo][No] (or the result itself when S == 1)
+    int Mo, No;          // output rows (input channels) and columns (output channels)
+    int R;               // reduction length: rows of X and dY
+    int rows_per_split;  // multiple of 64
+    int* err;
+};
+
+// out[z][i][j] = sum over rows r of split z of X[r][i] * dY[r][j].  Both operands are read as they lie in memory
+// (channels contiguous), i.e. MN-major; a stage holds 64 reduction rows.
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+                                                              const TcWgParams p) {
+    constexpr uint32_t SLAB = 64 * 64 * 2, A_BYTES = 2 * SLAB, B_BYTES = (BN / 64) * SLAB, STAGE_BYTES = A_BYTES + B_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ __align__(8) unsigned long long bars[2 * TC_STAGES + 1];
+    __shared__ uint32_t tmem_base;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i0 = blockIdx.x * TC_BM, j0 = blockIdx.y * BN;
+    const int rbeg = blockIdx.z * p.rows_per_split, rend = min(p.R, rbeg + p.rows_per_split);
+    const int num_kb = (rend - rbeg + 63) / 64;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % TC_STAGES;
+                const uint32_t ph = (kb / TC_STAGES) & 1;
+                if (kb >= TC_STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 4)) break;
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
+                const int r = rbeg + kb * 64;
+                mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+                tma_load_2d(sa, &mapX, i0, r, full0 + 8 * s);
+                tma_load_2d(sa + SLAB, &mapX, i0 + 64, r, full0 + 8 * s);
+#pragma unroll
+                for (int t = 0; t < BN / 64; ++t) tma_load_2d(sb + t * SLAB, &mapY, j0 + 64 * t, r, full0 + 8 * s);
+                issued = kb + 1;
+            }
+            if (*((volatile int*)p.err) != 0) {
+                for (int kb = max(0, issued - TC_STAGES); kb < issued; ++kb) {
+                    const unsigned long long t0 = gtime();
+                    while (!mbar_test(full0 + 8 * (kb % TC_STAGES), (kb / TC_STAGES) & 1) && gtime() - t0 < 1000000ull) __nanosleep(128);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // both operands MN-major: bits 15 and 16
+            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % TC_STAGES;
+                const uint32_t ph = (kb / TC_STAGES) & 1;
+                ok = mbar_wait(full0 + 8 * s, ph, p.err, 5);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
+                const uint64_t ad = umma_desc_mn_sw128(sa, SLAB), bd = umma_desc_mn_sw128(sb, SLAB);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)                           // 16 reduction rows = 2048 bytes further
+                    umma_bf16(tmem, ad + (uint64_t)(k * 128), bd + (uint64_t)(k * 128), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(empty0 + 8 * s);
+            }
+            if (ok) umma_commit(accum);
+        }
+    } else {
+        const int q = warp & 3;
+        if (num_kb > 0 ? mbar_wait(accum, 0, p.err, 6) : true) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int i = i0 + q * 32 + lane;
+            float* orow = p.out + ((long long)blockIdx.z * p.Mo + i) * p.No;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                if (num_kb > 0) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+                else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
+                const int jb = j0 + c * 32;
+                if (i < p.Mo) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (jb + g * 4 < p.No)
+                            *reinterpret_cast<float4*>(orow + jb + g * 4) = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
+                                                                                      __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
@@ -207,6 +332,23 @@ EncodeTiledFn encode_fn() {
             fn = reinterpret_cast<EncodeTiledFn>(p);
     }
     return fn;
+}
+
+struct TcWgPlan { int S, rows_per_split; };
+TcWgPlan plan_tc_wgrad(long long R, int Mo, int No) {
+    const long long tiles = ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
+    long long S = (3LL * sm_count() + tiles - 1) / tiles;
+    const long long maxS = (R + 511) / 512;                                 // at least 512 rows per split
+    long long cap = (8LL << 20) / ((long long)Mo * No);                     // partials within 8 Mi floats
+    if (cap < 1) cap = 1;
+    if (S > maxS) S = maxS;
+    if (S > cap) S = cap;
+    if (S < 1) S = 1;
+    long long rps = ((R + S - 1) / S + 63) / 64 * 64;
+    TcWgPlan w;
+    w.rows_per_split = (int)rps;
+    w.S = (int)((R + rps - 1) / rps);
+    return w;
 }
 
 // rows x cols bf16 matrix, cols contiguous; box = 64 columns x box_rows rows, 128-byte swizzle, zero fill
@@ -237,7 +379,36 @@ bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat
     return true;
 }
 
+template <int BN>
+bool launch_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out, long long R, int Mo, int No, const TcWgPlan& w, int* err, cudaStream_t st) {
+    CUtensorMap mx, my;
+    if (!make_map_2d(&mx, X, R, Mo, 64) || !make_map_2d(&my, dY, R, No, 64)) return false;
+    constexpr int smem = TC_STAGES * (2 + BN / 64) * 64 * 64 * 2 + 1024;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(tc_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+        configured = true;
+    }
+    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err};
+    tc_wgrad_kernel<BN><<<dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S), TC_THREADS, smem, st>>>(mx, my, p);
+    return true;
+}
+
 }  // namespace
+
+size_t tc_wgrad_scratch_floats(long long R, int Mo, int No) {
+    const TcWgPlan w = plan_tc_wgrad(R, Mo, No);
+    return w.S > 1 ? (size_t)w.S * Mo * No : 0;
+}
+
+// dW[Mo][No] = X[R][Mo]^T * dY[R][No] (bf16 in, float out); scratch holds tc_wgrad_scratch_floats floats.
+// Returns the number of splits written to scratch (1: dW was written directly), 0 if nothing was launched.
+int tc_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st) {
+    const TcWgPlan w = plan_tc_wgrad(R, Mo, No);
+    float* out = w.S > 1 ? scratch : dW;
+    const bool ok = No > 64 ? launch_wgrad<128>(X, dY, out, R, Mo, No, w, err, st) : launch_wgrad<64>(X, dY, out, R, Mo, No, w, err, st);
+    return ok ? w.S : 0;
+}
 
 bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend) {
     auto a16 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; };

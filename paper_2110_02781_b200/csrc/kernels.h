@@ -42,6 +42,9 @@ void conv_wgrad_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* dy, float
 bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
 bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K,
                 int* err, cudaStream_t st);
+size_t tc_wgrad_scratch_floats(long long R, int Mo, int No);
+int tc_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
+void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st);   // out = sum over S partial arrays, in order
 void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, cudaStream_t st);   // wt[n][k] = bf16(w[k][n])
 
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
@@ -74,7 +77,7 @@ void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, 
                  const float* beta, float eps, float momentum, float* run_mean, float* run_var, float* scale,
                  float* shift, float* mean, float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st);
 template <typename T>
-void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const float* scale, const float* shift,
+void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
               const float* mean, const float* mean_lo, int act, cudaStream_t st);
 // pass 1 of BN backward: sums of dz' and dz'*xhat with dz' = dz masked by the activation
 template <typename T>
@@ -86,7 +89,7 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
                      const float* rstd, float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st);
 template <typename T>
-void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const float* scale,
+void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const FoldPlan& fp, const float* scale,
                   const float* shift, const float* mean, const float* mean_lo, const float* rstd, const float* coef,
                   int act, cudaStream_t st);
 

@@ -234,6 +234,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         } else if (is_contraction(o.d.kind)) {
             finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
             red = std::max(red, std::max(conv_wgrad_scratch_floats(o.g), conv_gemm_scratch_floats(o.g)));
+            if (m.cfg.precision == FTP_BF16) red = std::max(red, tc_wgrad_scratch_floats(Mout, o.C, o.Co));
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
             if (o.d.act != FTP_ACT_NONE) dpre = std::max(dpre, obytes);
@@ -346,7 +347,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 const void* res = nullptr;
                 if (o.fused_add) { const int s = m->ops[i + 1].d.residual_src; res = s < first ? act_in : m->cur_out[s]; }
                 { Scope sc(m, st, K_BN_APPLY, u, i, 0, (o.in_elems * (res ? 3.0 : 2.0)) * es, 2.0 * o.in_elems);
-                  bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.scale, o.shift, o.mean, o.mean_lo, o.d.act, st); }
+                  bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.d.act, st); }
                 break;
             }
             case FTP_ACT: {
@@ -440,8 +441,15 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                                         o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                         if (dpre) d = dpre;
                     }
-                    { Scope sc(m, st, K_CONV_WGRAD_BF16_SIMT, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
-                      conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, m->red_scratch, o.g, st); }
+                    { Scope sc(m, st, K_GEMM_BF16_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
+                      int splits = 0;
+                      if (is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, d, gr + o.w_off, nullptr))
+                          splits = tc_wgrad((const T*)in, d, gr + o.w_off, m->red_scratch, Mout, o.C, o.Co, m->tc_err, st);
+                      if (splits > 1) split_reduce_f32(m->red_scratch, splits, o.w_cnt, gr + o.w_off, st);
+                      if (splits == 0) {
+                          if (sc.slot) sc.slot->rec.kernel = K_CONV_WGRAD_BF16_SIMT;
+                          conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, m->red_scratch, o.g, st);
+                      } }
                     if (gi) {
                         Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the canonical weight layout already has K = cout contiguous
@@ -470,7 +478,7 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                   bn_bwd_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, m->fin, st); }
                 if (gi) {
                     Scope sc(m, st, K_BN_BWD_APPLY, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, 8.0 * o.in_elems);
-                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef, o.d.act, st);
+                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef, o.d.act, st);
                 }
                 break;
             }
