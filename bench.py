@@ -32,17 +32,36 @@ def workload(name, batch=None):
         ls, cfg = synth.har_cnn()
         return dict(index=0, name="config 1: HAR 1D-CNN 32x9x128 fp32, 2 stages split after layer 2", layers=ls, cfg=cfg,
                     caps=None, points=[0, 2, 5])
+    if name in ("cfg3", "cfg5"):
+        b = batch or 64
+        ls, cfg = synth.mobilenetv2(b, 224, 1000, 1, False)
+        cfg["max_stages"] = 5
+        if name == "cfg3":
+            return dict(index=2, name=f"config 3: MobileNetV2 224x224x3 batch {b} bf16, 4 stages under capacity ratios 1:2:5:10",
+                        layers=ls, cfg=cfg, caps=[1.0, 2.0, 5.0, 10.0], points=None)
+        return dict(index=4, name=f"config 5: MobileNetV2 224x224x3 batch {b} bf16, 5 stages, capacities U[1,10] redrawn and partition "
+                    "re-chosen every 50 iterations, chain + global snapshots every 20", layers=ls, cfg=cfg, caps=[1.0] * 5, points=None,
+                    dynamic=dict(repartition=50, snapshot=20))
+    if name == "cfg4":
+        b = batch or 256
+        ls, cfg = synth.vgg16(b, 32, 10, 1)
+        return dict(index=3, name=f"config 4: VGG-16-style 32x32x3 batch {b} bf16, 3 stages from the partition optimiser", layers=ls,
+                    cfg=cfg, caps=[1.0, 1.0, 1.0], points=None)
     ls, cfg = synth.mobilenetv2(batch or 128, 32, 10, 0, True)
     return dict(index=1, name=f"config 2: MobileNetV2 32x32x3 batch {batch or 128} fp32, 3 stages at equal capacity", layers=ls,
                 cfg=cfg, caps=[1.0, 1.0, 1.0], points=None)
 
 
+FALLBACK_BF16_TFLOPS = 1400.0            # sustained figure of the fallback measurement
+
+
 def peaks():
+    """(HBM GB/s, bf16 tensor TFLOP/s sustained, source).  The sustained tensor figure applies: kernels are timed inside a long step."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return float(d["hbm_gbs"]), "measured"
-    return FALLBACK_HBM_GBS, "fallback"
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", d.get("bf16_tflops", FALLBACK_BF16_TFLOPS))), "measured"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
 
 
 class ClockSampler:
@@ -123,7 +142,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
     ap.add_argument("--points", default=None, help="comma-separated partition points; skips the profile-and-optimise step")
@@ -159,8 +178,10 @@ def main():
     m = F.Model(ls, cfg, f"cuda:{local_rank}")
     m.load_params(synth.init_params(wl["index"], ls), synth.init_state(ls))
     x, y = synth.make_batch(wl["index"], cfg)
-    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
-    xh, yh = torch.from_numpy(x).pin_memory(), torch.from_numpy(y).pin_memory()
+    bf16 = cfg["precision"] == 1
+    xt = torch.from_numpy(x).to(torch.bfloat16) if bf16 else torch.from_numpy(x)
+    xd, yd = xt.cuda(), torch.from_numpy(y).cuda()
+    xh, yh = xt.pin_memory(), torch.from_numpy(y).pin_memory()
     lr = cfg["lr"]
 
     # partition: profile -> equal capacities -> optimiser (or the split the workload fixes)
@@ -240,34 +261,40 @@ def main():
         k = by.setdefault(r["kernel"], dict(ms=0.0, bytes=0.0, flops=0.0, n=0))
         k["ms"] += r["ms"]; k["bytes"] += r["bytes"]; k["flops"] += r["flops"]; k["n"] += 1
     total_ms = sum(k["ms"] for k in by.values())
-    hbm_peak, peak_src = peaks()
+    hbm_peak, tensor_peak, peak_src = peaks()
     table = {}
     for name, k in sorted(by.items(), key=lambda kv: -kv[1]["ms"]):
         gbs = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
         tf = k["flops"] / (k["ms"] * 1e-3) / 1e12 if k["ms"] > 0 else 0.0
+        math_peak = tensor_peak if name.startswith("tc_") else FP32_ALU_PEAK_TFLOPS
         table[name] = dict(share=round(k["ms"] / total_ms, 4), launches_per_step=k["n"] // 3, ms_per_step=round(k["ms"] / 3, 4),
                            gbs=round(gbs, 1), tflops=round(tf, 2), frac_hbm=round(gbs / hbm_peak, 3),
-                           frac_alu=round(tf / FP32_ALU_PEAK_TFLOPS, 3))
+                           frac_math=round(tf / math_peak, 3))
     dom = next(iter(table))
     d = table[dom]
-    alu_bound = d["frac_alu"] > d["frac_hbm"]
-    roofline = {"kernel": dom, "bound": "alu" if alu_bound else "hbm",
-                "achieved": d["tflops"] if alu_bound else d["gbs"],
-                "peak": round(FP32_ALU_PEAK_TFLOPS, 1) if alu_bound else hbm_peak,
-                "unit": "TFLOP/s" if alu_bound else "GB/s",
-                "frac": d["frac_alu"] if alu_bound else d["frac_hbm"],
-                "peak_source": "derived: 2 x 128 lanes x 148 SMs x 1.965 GHz" if alu_bound else f"{peak_src} HBM copy",
-                "traffic": None, "share_of_step": d["share"], "kernels": table}
+    math_bound = d["frac_math"] > d["frac_hbm"]
+    tensor = dom.startswith("tc_")
+    roofline = {"kernel": dom, "bound": ("tensor" if tensor else "alu") if math_bound else "hbm",
+                "achieved": d["tflops"] if math_bound else d["gbs"],
+                "peak": (tensor_peak if tensor else round(FP32_ALU_PEAK_TFLOPS, 1)) if math_bound else hbm_peak,
+                "unit": "TFLOP/s" if math_bound else "GB/s",
+                "frac": d["frac_math"] if math_bound else d["frac_hbm"],
+                "peak_source": ((f"{peak_src} bf16 matmul, sustained" if tensor else "derived: 2 x 128 lanes x 148 SMs x 1.965 GHz")
+                                if math_bound else f"{peak_src} HBM copy"),
+                "traffic": None, "share_of_step": d["share"],
+                "note": "achieved = algorithmic bytes (or flops) of all launches of the kernel in a step / their CUDA-event time",
+                "kernels": table}
 
     out = {"metric": "training samples/sec per partitioned step", "value": value, "unit": "samples/s", "n_gpus": world,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-           "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
            "config": {"workload": wl["name"], "points": points, "stages": len(points) - 1, "batch": batch,
                       "parallelism": "replicas only" if world > 1 else "1 GPU, all stages resident",
-                      "cache": "step touches >1.5 GB of activations, far larger than the 126 MB L2",
+                      "cache": "a step streams far more activation bytes than the 126 MB L2 holds",
+                      "capacities": wl["caps"],
                       "launch": "cuda graph replay of ftp_train_step" if args.graph else "eager"},
            "clocks": clk.summary(), "gpu_launches": int(launches),
-           "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(xh.numel() * 4 + yh.numel() * 4),
+           "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * 4),
                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / args.steps},
            "roofline": roofline}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -712,6 +712,8 @@ __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ s, float* _
 __global__ void transpose_f32_to_bf16_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ wt, int K, int N) {
     __shared__ float tile[32][33];
     const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+    w += (long long)blockIdx.z * K * N;
+    wt += (long long)blockIdx.z * K * N;
     for (int r = threadIdx.y; r < 32; r += 8) {
         const int k = k0 + r, n = n0 + threadIdx.x;
         tile[r][threadIdx.x] = (k < K && n < N) ? w[(long long)k * N + n] : 0.f;
@@ -924,8 +926,8 @@ void sgd_update(float* w, const float* g, float* m, long long n, float lr, float
     else sgd_kernel<1><<<flat_blocks(n, 256), 256, 0, st>>>(w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
 }
 
-void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, cudaStream_t st) {
-    transpose_f32_to_bf16_kernel<<<dim3((N + 31) / 32, (K + 31) / 32), dim3(32, 8), 0, st>>>(w, wt, K, N);
+void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st) {
+    transpose_f32_to_bf16_kernel<<<dim3((N + 31) / 32, (K + 31) / 32, batch), dim3(32, 8), 0, st>>>(w, wt, K, N);
 }
 
 void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st) {

@@ -47,6 +47,22 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(dst), "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar) : "memory");
+}
+
+// 3x3 convolution (stride 1, pad 1) as an implicit GEMM: a tile of 128 output pixels is bn images x bh rows x the
+// full width; for tap (r, s) the operand tile is the same box shifted by (r-1, s-1) (forward) or (1-r, 1-s) (data
+// gradient), with everything outside the image filled with zeros by TMA.
+struct ConvTap {
+    int enabled;      // 0: plain 2-D operand
+    int H, W;         // image size
+    int chunks;       // 64-channel chunks per tap (channels / 64)
+    int flip;         // 0 forward, 1 data gradient
+    int b_rows;       // rows of the weight matrix per tap
+};
+
 // Shared-memory operand descriptor, K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t saddr) {
     uint64_t d = 0;
@@ -78,8 +94,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 struct TcParams {
     __nv_bfloat16* D;
     const __nv_bfloat16* addend;   // nullable, shaped like D
-    int M, N, K;
+    int M, N, K;                   // K: reduction length (conv: 9 * channels)
     int* err;
+    ConvTap conv;
 };
 
 template <int BN>
@@ -120,8 +137,16 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
                 if (kb >= TC_STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 1)) break;
                 const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
                 mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-                tma_load_2d(sa, &mapA, kb * TC_BK, m0, full0 + 8 * s);
-                tma_load_2d(sb, &mapB, kb * TC_BK, n0, full0 + 8 * s);
+                if (!p.conv.enabled) {
+                    tma_load_2d(sa, &mapA, kb * TC_BK, m0, full0 + 8 * s);
+                    tma_load_2d(sb, &mapB, kb * TC_BK, n0, full0 + 8 * s);
+                } else {
+                    const int tap = kb / p.conv.chunks, cc = kb - tap * p.conv.chunks, r = tap / 3, sx = tap - 3 * r;
+                    const int hw = p.conv.H * p.conv.W, img = m0 / hw, h0 = (m0 - img * hw) / p.conv.W;
+                    const int dh = p.conv.flip ? 1 - r : r - 1, dw = p.conv.flip ? 1 - sx : sx - 1;
+                    tma_load_4d(sa, &mapA, cc * 64, dw, h0 + dh, img, full0 + 8 * s);
+                    tma_load_2d(sb, &mapB, cc * 64, tap * p.conv.b_rows + n0, full0 + 8 * s);
+                }
                 issued = kb + 1;
             }
             if (*((volatile int*)p.err) != 0) {
@@ -207,11 +232,12 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t 
 }
 
 struct TcWgParams {
-    float* out;          // partials [S][Mo][No] (or the result itself when S == 1)
+    float* out;          // partials [S][taps][Mo][No] (or the result itself when S == 1)
     int Mo, No;          // output rows (input channels) and columns (output channels)
     int R;               // reduction length: rows of X and dY
     int rows_per_split;  // multiple of 64
     int* err;
+    ConvTap conv;        // enabled: grid.z = splits * 9, X is read through a 4-D map shifted by the tap
 };
 
 // out[z][i][j] = sum over rows r of split z of X[r][i] * dY[r][j].  Both operands are read as they lie in memory
@@ -227,7 +253,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int i0 = blockIdx.x * TC_BM, j0 = blockIdx.y * BN;
-    const int rbeg = blockIdx.z * p.rows_per_split, rend = min(p.R, rbeg + p.rows_per_split);
+    const int taps = p.conv.enabled ? 9 : 1;
+    const int split = blockIdx.z / taps, tap = blockIdx.z - split * taps;
+    const int rbeg = split * p.rows_per_split, rend = min(p.R, rbeg + p.rows_per_split);
     const int num_kb = (rend - rbeg + 63) / 64;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
 
@@ -255,8 +283,15 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
                 const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
                 const int r = rbeg + kb * 64;
                 mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-                tma_load_2d(sa, &mapX, i0, r, full0 + 8 * s);
-                tma_load_2d(sa + SLAB, &mapX, i0 + 64, r, full0 + 8 * s);
+                if (!p.conv.enabled) {
+                    tma_load_2d(sa, &mapX, i0, r, full0 + 8 * s);
+                    tma_load_2d(sa + SLAB, &mapX, i0 + 64, r, full0 + 8 * s);
+                } else {
+                    const int tr = tap / 3, ts = tap - 3 * tr;
+                    const int hw = p.conv.H * p.conv.W, img = r / hw, h0 = (r - img * hw) / p.conv.W;
+                    tma_load_4d(sa, &mapX, i0, ts - 1, h0 + tr - 1, img, full0 + 8 * s);
+                    tma_load_4d(sa + SLAB, &mapX, i0 + 64, ts - 1, h0 + tr - 1, img, full0 + 8 * s);
+                }
 #pragma unroll
                 for (int t = 0; t < BN / 64; ++t) tma_load_2d(sb + t * SLAB, &mapY, j0 + 64 * t, r, full0 + 8 * s);
                 issued = kb + 1;
@@ -293,7 +328,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
         if (num_kb > 0 ? mbar_wait(accum, 0, p.err, 6) : true) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int i = i0 + q * 32 + lane;
-            float* orow = p.out + ((long long)blockIdx.z * p.Mo + i) * p.No;
+            float* orow = p.out + (((long long)split * taps + tap) * p.Mo + i) * p.No;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
@@ -363,6 +398,42 @@ bool make_map_2d(CUtensorMap* map, const void* base, long long rows, long long c
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// (N, H, W, C) bf16 activation; box = 64 channels x the full width x bh rows x bn images (pix = W*bh*bn pixels)
+bool make_map_4d(CUtensorMap* map, const void* base, int N, int H, int W, int C, int pix) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    int bh = pix / W;
+    if (bh > H) bh = H;
+    const int bn = pix / (W * bh);
+    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+    const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)W, (cuuint32_t)bh, (cuuint32_t)bn};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// an image tiles into boxes of `pix` pixels made of whole rows (and whole images when the image is smaller)
+bool conv_tiles_ok(int H, int W, int pix) {
+    if (W < 1 || W > pix || pix % W != 0) return false;
+    const int bh = pix / W;
+    if (bh <= H) return H % bh == 0;
+    return bh % H == 0;            // several whole images per box
+}
+
+template <int BN>
+bool launch_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No,
+                    int flip, int* err, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    if (!make_map_4d(&ma, A, N, H, W, Ca, TC_BM) || !make_map_2d(&mb, B, 9LL * No, Ca, BN)) return false;
+    constexpr int smem = TC_STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
+    if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    const int M = N * H * W;
+    TcParams p{D, addend, M, No, 9 * Ca, err, ConvTap{1, H, W, Ca / 64, flip, No}};
+    tc_gemm_tn_kernel<BN><<<dim3((No + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), TC_THREADS, smem, st>>>(ma, mb, p);
+    return true;
+}
+
 template <int BN>
 bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K, int* err,
                cudaStream_t st) {
@@ -374,7 +445,7 @@ bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat
         if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
         configured = true;
     }
-    TcParams p{D, addend, M, N, K, err};
+    TcParams p{D, addend, M, N, K, err, ConvTap{0, 0, 0, 0, 0, 0}};
     tc_gemm_tn_kernel<BN><<<dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), TC_THREADS, smem, st>>>(ma, mb, p);
     return true;
 }
@@ -389,12 +460,69 @@ bool launch_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out, l
         if (cudaFuncSetAttribute(tc_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
         configured = true;
     }
-    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err};
+    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{0, 0, 0, 0, 0, 0}};
     tc_wgrad_kernel<BN><<<dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S), TC_THREADS, smem, st>>>(mx, my, p);
     return true;
 }
 
+template <int BN>
+bool launch_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out, int N, int H, int W, int Mo, int No, const TcWgPlan& w, int* err,
+                     cudaStream_t st) {
+    CUtensorMap mx, my;
+    const long long R = (long long)N * H * W;
+    if (!make_map_4d(&mx, X, N, H, W, Mo, 64) || !make_map_2d(&my, dY, R, No, 64)) return false;
+    constexpr int smem = TC_STAGES * (2 + BN / 64) * 64 * 64 * 2 + 1024;
+    if (cudaFuncSetAttribute(tc_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{1, H, W, 0, 0, 0}};
+    tc_wgrad_kernel<BN><<<dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S * 9), TC_THREADS, smem, st>>>(mx, my, p);
+    return true;
+}
+
+TcWgPlan plan_tc_wgrad3x3(long long R, int Mo, int No) {
+    const long long tiles = 9LL * ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
+    long long S = (3LL * sm_count() + tiles - 1) / tiles;
+    const long long maxS = (R + 511) / 512;
+    long long cap = (8LL << 20) / (9LL * Mo * No);
+    if (cap < 1) cap = 1;
+    if (S > maxS) S = maxS;
+    if (S > cap) S = cap;
+    if (S < 1) S = 1;
+    const long long rps = ((R + S - 1) / S + 63) / 64 * 64;
+    TcWgPlan w;
+    w.rows_per_split = (int)rps;
+    w.S = (int)((R + rps - 1) / rps);
+    return w;
+}
+
 }  // namespace
+
+bool tc_conv3x3_supported(int N, int H, int W, int Ca, int No, const void* A, const void* B, const void* D, const void* addend) {
+    auto a16 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+    return Ca % 64 == 0 && No % 8 == 0 && conv_tiles_ok(H, W, TC_BM) && conv_tiles_ok(H, W, 64) && (long long)N * H * W < (1LL << 31) && a16(A) &&
+           a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
+}
+
+// 3x3, stride 1, pad 1.  Forward (flip 0): A = x (N,H,W,Ca), B = weights [9][No][Ca]; data gradient (flip 1): A = dy,
+// B = weights [9][No = cin][Ca = cout].  D (N,H,W,No) bf16.
+bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No, int flip,
+                int* err, cudaStream_t st) {
+    if (No > 64) return launch_conv3x3<128>(A, B, addend, D, N, H, W, Ca, No, flip, err, st);
+    if (No > 32) return launch_conv3x3<64>(A, B, addend, D, N, H, W, Ca, No, flip, err, st);
+    return launch_conv3x3<32>(A, B, addend, D, N, H, W, Ca, No, flip, err, st);
+}
+
+size_t tc_wgrad3x3_scratch_floats(long long R, int Mo, int No) {
+    const TcWgPlan w = plan_tc_wgrad3x3(R, Mo, No);
+    return w.S > 1 ? (size_t)w.S * 9 * Mo * No : 0;
+}
+
+// dW[9][Mo][No] of a 3x3 / stride 1 / pad 1 convolution; returns the number of splits (0: nothing launched)
+int tc_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, int N, int H, int W, int Mo, int No, int* err, cudaStream_t st) {
+    const TcWgPlan w = plan_tc_wgrad3x3((long long)N * H * W, Mo, No);
+    float* out = w.S > 1 ? scratch : dW;
+    const bool ok = No > 64 ? launch_wgrad3x3<128>(X, dY, out, N, H, W, Mo, No, w, err, st) : launch_wgrad3x3<64>(X, dY, out, N, H, W, Mo, No, w, err, st);
+    return ok ? w.S : 0;
+}
 
 size_t tc_wgrad_scratch_floats(long long R, int Mo, int No) {
     const TcWgPlan w = plan_tc_wgrad(R, Mo, No);

@@ -42,10 +42,17 @@ void conv_wgrad_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* dy, float
 bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
 bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K,
                 int* err, cudaStream_t st);
+// 3x3 / stride 1 / pad 1 convolutions on the same kernels through 4-D tensor maps (zero fill = padding).
+bool tc_conv3x3_supported(int N, int H, int W, int Ca, int No, const void* A, const void* B, const void* D, const void* addend);
+bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No,
+                int flip, int* err, cudaStream_t st);
+size_t tc_wgrad3x3_scratch_floats(long long R, int Mo, int No);
+int tc_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, int N, int H, int W, int Mo, int No, int* err,
+                cudaStream_t st);
 size_t tc_wgrad_scratch_floats(long long R, int Mo, int No);
 int tc_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
 void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st);   // out = sum over S partial arrays, in order
-void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, cudaStream_t st);   // wt[n][k] = bf16(w[k][n])
+void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st);   // per matrix: wt[n][k] = bf16(w[k][n])
 
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
 // Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole

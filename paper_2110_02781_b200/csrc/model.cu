@@ -234,7 +234,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         } else if (is_contraction(o.d.kind)) {
             finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
             red = std::max(red, std::max(conv_wgrad_scratch_floats(o.g), conv_gemm_scratch_floats(o.g)));
-            if (m.cfg.precision == FTP_BF16) red = std::max(red, tc_wgrad_scratch_floats(Mout, o.C, o.Co));
+            if (m.cfg.precision == FTP_BF16) red = std::max(red, std::max(tc_wgrad_scratch_floats(Mout, o.C, o.Co), tc_wgrad3x3_scratch_floats(Mout, o.C, o.Co)));
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
             if (o.d.act != FTP_ACT_NONE) dpre = std::max(dpre, obytes);
@@ -277,12 +277,16 @@ bool is_pointwise_op(const Op& o) {
     return o.d.kind == FTP_CONV2D && o.g.kh == 1 && o.g.kw == 1 && o.g.stride == 1 && o.g.ph == 0 && o.d.act == FTP_ACT_NONE && o.b_off < 0;
 }
 
+bool is_3x3_op(const Op& o) {
+    return o.d.kind == FTP_CONV2D && o.g.kh == 3 && o.g.kw == 3 && o.g.stride == 1 && o.g.ph == 1 && o.g.pw == 1 && o.d.act == FTP_ACT_NONE && o.b_off < 0;
+}
+
 // bf16 models: rebuild the transposed bf16 copy of every 1x1 convolution of units [a, b) from the float masters
 void refresh_transposed(ftp_model* m, int a, int b, cudaStream_t st) {
     for (int i = m->unit_first[a]; i <= m->unit_last[b - 1]; ++i) {
         const Op& o = m->ops[i];
         const Arena& ar = m->arena[m->owner[o.d.unit]];
-        if (ar.wbt && is_pointwise_op(o)) transpose_f32_to_bf16(ar.w + o.w_off, ar.wbt + o.w_off, o.C, o.Co, st);
+        if (ar.wbt && (is_pointwise_op(o) || is_3x3_op(o))) transpose_f32_to_bf16(ar.w + o.w_off, ar.wbt + o.w_off, o.C, o.Co, o.g.kh * o.g.kw, st);
     }
 }
 
@@ -324,8 +328,10 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                         conv_fwd_f32(m->fc_in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                     } else {
                         Scope sc(m, st, K_GEMM_BF16_FWD, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 2.0, fl);
-                        const bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, ar.wbt + o.w_off, out, nullptr) &&
-                                        tc_gemm_tn((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, (int)Mout, o.Co, o.C, m->tc_err, st);
+                        bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, ar.wbt + o.w_off, out, nullptr) &&
+                                  tc_gemm_tn((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, (int)Mout, o.Co, o.C, m->tc_err, st);
+                        if (!tc && is_3x3_op(o) && tc_conv3x3_supported(o.N, o.H, o.W, o.C, o.Co, in, ar.wbt + o.w_off, out, nullptr))
+                            tc = tc_conv3x3((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, o.N, o.H, o.W, o.C, o.Co, 0, m->tc_err, st);
                         if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_FWD_BF16_SIMT;
                         if (!tc) conv_fwd_bf16_simt((const T*)in, ar.wb + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (T*)out, o.g, o.d.act, st);
                     }
@@ -445,6 +451,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                       int splits = 0;
                       if (is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, d, gr + o.w_off, nullptr))
                           splits = tc_wgrad((const T*)in, d, gr + o.w_off, m->red_scratch, Mout, o.C, o.Co, m->tc_err, st);
+                      if (splits == 0 && is_3x3_op(o) && o.C % 8 == 0 && tc_conv3x3_supported(o.N, o.H, o.W, 64, o.Co, in, d, gr + o.w_off, nullptr))
+                          splits = tc_wgrad3x3((const T*)in, d, gr + o.w_off, m->red_scratch, o.N, o.H, o.W, o.C, o.Co, m->tc_err, st);
                       if (splits > 1) split_reduce_f32(m->red_scratch, splits, o.w_cnt, gr + o.w_off, st);
                       if (splits == 0) {
                           if (sc.slot) sc.slot->rec.kernel = K_CONV_WGRAD_BF16_SIMT;
@@ -453,8 +461,10 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                     if (gi) {
                         Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the canonical weight layout already has K = cout contiguous
-                        const bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.C, o.Co, d, ar.wb + o.w_off, gi, addend) &&
-                                        tc_gemm_tn(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, (int)Mout, o.C, o.Co, m->tc_err, st);
+                        bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.C, o.Co, d, ar.wb + o.w_off, gi, addend) &&
+                                  tc_gemm_tn(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, (int)Mout, o.C, o.Co, m->tc_err, st);
+                        if (!tc && is_3x3_op(o) && tc_conv3x3_supported(o.N, o.H, o.W, o.Co, o.C, d, ar.wb + o.w_off, gi, addend))
+                            tc = tc_conv3x3(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.N, o.H, o.W, o.Co, o.C, 1, m->tc_err, st);
                         if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_DGRAD_BF16_SIMT;
                         if (!tc) conv_dgrad_bf16_simt(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.g, st);
                     }
