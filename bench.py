@@ -113,7 +113,7 @@ def run_reference(args, wl):
     except Exception:
         cores = os.cpu_count() or 1
     ls, cfg = wl["layers"], dict(wl["cfg"])
-    sample_batch = min(cfg["batch"], 16 if wl["index"] == 1 else cfg["batch"])
+    sample_batch = min(cfg["batch"], {0: cfg["batch"], 1: 16, 2: 2, 3: 8, 4: 2}[wl["index"]])
     cfg["batch"] = sample_batch
     om = oracle.OracleModel(ls, cfg, synth.init_params(wl["index"], ls), synth.init_state(ls))
     L = om.L
@@ -127,7 +127,8 @@ def run_reference(args, wl):
             times.append(time.perf_counter() - t)
     tot = sum(times)
     value = sample_batch * len(times) / tot
-    sample = f"{len(times)} steps of the same network at batch {sample_batch} (of {wl['cfg']['batch']}), float64 numpy"
+    sample = (f"{len(times)} steps of the same network at batch {sample_batch} (of {wl['cfg']['batch']}), float64 numpy"
+              + (", bf16 storage mode" if cfg["precision"] == 1 else ""))
     return {"impl": "reference", "metric": "training samples/sec per partitioned step", "value": value, "unit": "samples/s",
             "n_gpus": args.gpus, "steps": len(times), "warmup": args.warmup_ref, "ms_per_step": 1e3 * tot / len(times),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -136,10 +137,58 @@ def run_reference(args, wl):
             "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
+def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host):
+    """Config 5: train `steps` iterations; after every `repartition`-th the stage capacities are redrawn from U[1,10] and the
+    partition re-chosen (Eq. 4 on the profiled layer times); after every `snapshot`-th each stage's weights are copied to
+    the next stage's replica buffer (last stage -> central) and every stage's to the central pinned-host buffer.
+    Returns (total ms, per-iteration ms list, log of partitions)."""
+    import numpy as np
+    import torch
+    import synth
+    dyn = wl["dynamic"]
+    n_st = len(wl["caps"])
+    rng = synth.rng_stream(wl["index"], "capacity")
+    L = m.L
+    sizes = [m.ftp_unit_param_span(u)[1] + m.ftp_unit_state_span(u)[1] for u in range(L)]
+    total = sum(sizes)
+    replicas = [torch.empty(total, dtype=torch.float32, device="cuda") for _ in range(n_st)]      # chain targets (device)
+    central = torch.empty(2 * total, dtype=torch.float32).pin_memory()                             # chain tail + global copy (host)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    log = []
+    torch.cuda.synchronize()
+    ev[0].record()
+    for it in range(steps):
+        if on_host:
+            m.ftp_train_step(xh, yh, lr, inputs_on_host=True, want_loss=True)
+        else:
+            m.ftp_train_step(xd, yd, lr, inputs_on_host=False, want_loss=False)
+        if (it + 1) % dyn["snapshot"] == 0:
+            pts = m.ftp_get_partition()
+            off = 0
+            for s in range(len(pts) - 1):
+                n = sum(sizes[pts[s]:pts[s + 1]])
+                if s + 1 < len(pts) - 1:
+                    m.ftp_snapshot_weights(s, replicas[s + 1][:n])                     # chain: to the next stage
+                else:
+                    m.ftp_snapshot_weights(s, central[total + off:total + off + n])    # chain: last stage to the central node
+                m.ftp_snapshot_weights(s, central[off:off + n])                        # global: every stage to the central node
+                off += n
+        if (it + 1) % dyn["repartition"] == 0:
+            caps = rng.uniform(1.0, 10.0, n_st).tolist()
+            pts, bott = F.ftp_choose_partition(layer_times, caps)
+            moved = m.ftp_set_partition(pts)
+            log.append(dict(after_iteration=it + 1, capacities=[round(c, 3) for c in caps], points=pts, moved_units=moved,
+                            virtual_bottleneck_ms=round(bott * 1e3, 4)))
+        ev[it + 1].record()
+    torch.cuda.synchronize()
+    per_it = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    return ev[0].elapsed_time(ev[steps]), per_it, log
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 50; 500 for cfg5)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
@@ -153,6 +202,8 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     wl = workload(args.workload, args.batch)
+    if args.steps is None:
+        args.steps = 500 if args.workload == "cfg5" else 50
 
     if args.impl == "reference":
         if rank != 0:
@@ -217,6 +268,9 @@ def main():
 
     step_eager = lambda: m.ftp_train_step(xd, yd, lr, inputs_on_host=False, want_loss=False)
     step_dev = step_eager
+    dynamic = wl.get("dynamic")
+    if dynamic:
+        args.graph = 0                   # the partition changes during the run: launches are issued eagerly
     if args.graph:
         # the launches of one step captured once on a side stream and replayed: same kernels, no per-launch CPU cost
         side = torch.cuda.Stream()
@@ -233,8 +287,20 @@ def main():
     for _ in range(args.warmup):
         step_dev()
     n0 = m.ftp_launch_count()
+    dyn_info = None
     with ClockSampler(local_rank) as clk:
-        ms = timed(step_dev, args.steps)
+        if dynamic:
+            lt = (fwd_s + bwd_s).tolist()
+            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, args.steps, False)
+            tick = lambda i, p: (i + 1) % p == 0
+            plain = [t for i, t in enumerate(per_it) if not tick(i, dynamic["snapshot"]) and not tick(i, dynamic["repartition"])]
+            snap = [t for i, t in enumerate(per_it) if tick(i, dynamic["snapshot"]) and not tick(i, dynamic["repartition"])]
+            rep = [t for i, t in enumerate(per_it) if tick(i, dynamic["repartition"])]
+            med = lambda v: round(statistics.median(v), 4) if v else None
+            dyn_info = dict(ms_plain_iteration=med(plain), ms_snapshot_iteration=med(snap), ms_repartition_iteration=med(rep),
+                            repartitions=plog[:10], snapshot_bytes_per_tick=int(3 * 4 * sum(m.ftp_unit_param_span(u)[1] + m.ftp_unit_state_span(u)[1] for u in range(m.L))))
+        else:
+            ms = timed(step_dev, args.steps)
     launches = m.ftp_launch_count() - n0
     if args.graph:                      # a replay re-issues the captured launches without passing through the counter
         c0 = m.ftp_launch_count()
@@ -245,10 +311,17 @@ def main():
         return 0
     for _ in range(3):
         step_e2e()
-    ms_e2e = timed(step_e2e, args.steps)
+    e2e_steps = args.steps
+    if dynamic:
+        e2e_steps = max(dynamic["repartition"] * 2, args.steps // 5)
+        m.ftp_set_partition(points)
+        ms_e2e, _, _ = run_dynamic(m, F, wl, (fwd_s + bwd_s).tolist(), xd, yd, xh, yh, lr, e2e_steps, True)
+        m.ftp_set_partition(points)
+    else:
+        ms_e2e = timed(step_e2e, args.steps)
     batch = cfg["batch"]
     value = world * batch * args.steps / (ms * 1e-3)
-    e2e = world * batch * args.steps / (ms_e2e * 1e-3)
+    e2e = world * batch * e2e_steps / (ms_e2e * 1e-3)
 
     # per-kernel roofline: one more step with every launch bracketed by events
     m.ftp_trace_enable(True)
@@ -295,8 +368,10 @@ def main():
                       "launch": "cuda graph replay of ftp_train_step" if args.graph else "eager"},
            "clocks": clk.summary(), "gpu_launches": int(launches),
            "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * 4),
-                   "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / args.steps},
+                   "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps},
            "roofline": roofline}
+    if dyn_info:
+        out["config"]["dynamic"] = dyn_info
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         a2 = argparse.Namespace(**vars(args))
         a2.warmup_ref, a2.steps = 0, 2
