@@ -1,0 +1,304 @@
+// float contractions on the tensor cores with float-level accuracy: every operand x is split into
+// hi = x with the low 13 mantissa bits cleared (exactly representable as tf32) and lo = x - hi (exact), and
+// the product is accumulated as hi*hi + hi*lo + lo*hi with tcgen05.mma kind::tf32 into a float accumulator in
+// tensor memory.  The dropped lo*lo term and the tf32 truncation of lo are below 2^-20 relative, which keeps
+// the float path within 1e-4 of a float64 reference while the math leaves the SIMT pipes.
+//
+// Same structure as the bf16 kernels: one 128 x BN tile per CTA; warp 0 streams 128 x 32 and BN x 32 float
+// tiles with TMA (128-byte swizzle, zero fill); warps 2-5 split each landed stage into a hi and a lo tile,
+// make the writes visible to the tensor-core proxy and signal warp 1, which issues the 3 x 4 MMAs (K = 8) of
+// the stage; at the end warps 2-5 read the accumulator and store floats.  The tensor cores always see
+// K-major operands: an operand that lies the other way in memory (activations in the weight gradient, the
+// weights in the forward) is transposed inside shared memory by the same pass that splits it.
+// Every wait is bounded; see gemm_tc.cu for the error protocol.
+#include "gemm_tc_common.cuh"
+
+namespace ftp {
+using namespace tc;
+namespace {
+
+constexpr int T32_BK = 32;          // floats per 128-byte row
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Transposing split.  src: nslabs slabs of [32 reduction rows][32 columns] floats as TMA wrote them (128-byte rows,
+// 16-byte chunk index XORed with row % 8).  hi / lo: K-major tiles [nslabs * 32 rows][32 reduction steps] in the
+// same swizzle.  A work item moves one output row's four consecutive reduction steps; the lanes of a warp take
+// 32 neighbouring columns of one source row, which is free of bank conflicts on both sides.
+__device__ __forceinline__ void transpose_split(const uint8_t* src, uint8_t* hi, uint8_t* lo, int nslabs, int t, int threads) {
+    for (int item = t; item < nslabs * 256; item += threads) {
+        const int mn = item & 31, kq = (item >> 5) & 7, sl = item >> 8;
+        const uint8_t* s0 = src + sl * 4096 + ((mn & 3) << 2);
+        float v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int k = kq * 4 + j;
+            v[j] = *reinterpret_cast<const float*>(s0 + k * 128 + ((((mn >> 2) ^ (k & 7))) << 4));
+        }
+        float4 h, l;
+        h.x = __uint_as_float(__float_as_uint(v[0]) & 0xffffe000u); l.x = v[0] - h.x;
+        h.y = __uint_as_float(__float_as_uint(v[1]) & 0xffffe000u); l.y = v[1] - h.y;
+        h.z = __uint_as_float(__float_as_uint(v[2]) & 0xffffe000u); l.z = v[2] - h.z;
+        h.w = __uint_as_float(__float_as_uint(v[3]) & 0xffffe000u); l.w = v[3] - h.w;
+        const int row = sl * 32 + mn;
+        const int off = row * 128 + ((kq ^ (row & 7)) << 4);
+        *reinterpret_cast<float4*>(hi + off) = h;
+        *reinterpret_cast<float4*>(lo + off) = l;
+    }
+}
+
+// hi stays where TMA put it (low mantissa bits cleared), lo goes to the buffer `lo_off` bytes further.
+// Elementwise, so the swizzled placement does not matter.  `threads` cooperating threads, `t` this thread's rank.
+__device__ __forceinline__ void split_tile(uint8_t* hi, uint32_t lo_off, int bytes, int t, int threads) {
+    for (int i = t * 16; i < bytes; i += threads * 16) {
+        float4 v = *reinterpret_cast<float4*>(hi + i);
+        float4 h, l;
+        h.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u); l.x = v.x - h.x;
+        h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u); l.y = v.y - h.y;
+        h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u); l.z = v.z - h.z;
+        h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u); l.w = v.w - h.w;
+        *reinterpret_cast<float4*>(hi + i) = h;
+        *reinterpret_cast<float4*>(hi + lo_off + i) = l;
+    }
+}
+
+struct T32Params {
+    float* D;              // gemm: output [M][N]; wgrad: partials [S][Mo][No]
+    const float* addend;   // gemm only, nullable
+    int M, N, K;           // gemm: D[M,N] = A[M,K] B[N,K]^T.  wgrad: Mo = M, No = N, K = reduction rows R
+    int rows_per_split;    // wgrad
+    int* err;
+};
+
+// MODE 0: A [M][K], B [N][K], both with K contiguous (data gradient).  MODE 1: X [R][Mo], dY [R][No], both transposed
+// in shared memory (weight gradient).  MODE 2: A [M][K] as it lies, B [K][N] (the weights) transposed (forward).
+template <int BN, int STAGES, int MODE>
+__global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                                                          const T32Params p) {
+    constexpr uint32_t A_BYTES = TC_BM * T32_BK * 4, B_BYTES = BN * T32_BK * 4;          // one precision part
+    constexpr bool TA = MODE == 1, TB = MODE != 0;                                      // operand transposed in shared memory
+    constexpr uint32_t STAGE_BYTES = 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) + (TB ? B_BYTES : 0);   // [A hi][A lo][B hi][B lo][A src][B src]
+    constexpr uint32_t SLAB = 32 * 32 * 4;                                              // transposed operands land as slabs of 32 columns x 32 rows
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ __align__(8) unsigned long long bars[3 * STAGES + 1];
+    __shared__ uint32_t tmem_base;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int m0, n0, kbeg, kend, split = 0;
+    constexpr bool WGRAD = MODE == 1;
+    if (WGRAD) {
+        m0 = blockIdx.x * TC_BM; n0 = blockIdx.y * BN; split = blockIdx.z;
+        kbeg = split * p.rows_per_split; kend = min(p.K, kbeg + p.rows_per_split);
+    } else {
+        n0 = blockIdx.x * BN; m0 = blockIdx.y * TC_BM; kbeg = 0; kend = p.K;
+    }
+    const int num_kb = (kend - kbeg + T32_BK - 1) / T32_BK;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), ready0 = smem_u32(&bars[2 * STAGES]), accum = smem_u32(&bars[3 * STAGES]);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(ready0 + 8 * s, 128); }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                if (kb >= STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 11)) break;
+                const uint32_t st0 = smem_u32(smem + s * STAGE_BYTES);
+                const uint32_t sa = TA ? st0 + 2 * (A_BYTES + B_BYTES) : st0;                                       // where A lands
+                const uint32_t sb = TB ? st0 + 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) : st0 + 2 * A_BYTES;   // where B lands
+                const int k = kbeg + kb * T32_BK;
+                mbar_expect_tx(full0 + 8 * s, A_BYTES + B_BYTES);
+                if (TA) {
+#pragma unroll
+                    for (int t = 0; t < TC_BM / 32; ++t) tma_load_2d(sa + t * SLAB, &mapA, m0 + 32 * t, k, full0 + 8 * s);
+                } else tma_load_2d(sa, &mapA, k, m0, full0 + 8 * s);
+                if (TB) {
+#pragma unroll
+                    for (int t = 0; t < BN / 32; ++t) tma_load_2d(sb + t * SLAB, &mapB, n0 + 32 * t, k, full0 + 8 * s);
+                } else tma_load_2d(sb, &mapB, k, n0, full0 + 8 * s);
+                issued = kb + 1;
+            }
+            if (*((volatile int*)p.err) != 0) {
+                for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
+                    const unsigned long long t0 = gtime();
+                    while (!mbar_test(full0 + 8 * (kb % STAGES), (kb / STAGES) & 1) && gtime() - t0 < 1000000ull) __nanosleep(128);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                ok = mbar_wait(ready0 + 8 * s, ph, p.err, 12);                   // split done and visible
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + 2 * A_BYTES;
+                const uint64_t ah = umma_desc_k_sw128(sa), al = umma_desc_k_sw128(sa + A_BYTES);
+                const uint64_t bh = umma_desc_k_sw128(sb), bl = umma_desc_k_sw128(sb + B_BYTES);
+#pragma unroll
+                for (int k = 0; k < T32_BK / 8; ++k) {                 // 8 reduction steps = 32 bytes further along the row
+                    const uint64_t o = (uint64_t)(k * 2);
+                    umma_tf32(tmem, ah + o, bh + o, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_tf32(tmem, ah + o, bl + o, idesc, 1u);
+                    umma_tf32(tmem, al + o, bh + o, idesc, 1u);
+                }
+                umma_commit(empty0 + 8 * s);
+            }
+            if (ok) umma_commit(accum);
+        }
+    } else {
+        // ---- warps 2..5: split every landed stage, then the epilogue ----
+        const int t = threadIdx.x - 64;
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int s = kb % STAGES;
+            const uint32_t ph = (kb / STAGES) & 1;
+            ok = mbar_wait(full0 + 8 * s, ph, p.err, 13);
+            if (!ok) break;
+            uint8_t* st = smem + s * STAGE_BYTES;
+            uint8_t* src = st + 2 * (A_BYTES + B_BYTES);
+            if (TA) transpose_split(src, st, st + A_BYTES, TC_BM / 32, t, 128);
+            else split_tile(st, A_BYTES, A_BYTES, t, 128);
+            if (TB) transpose_split(src + (TA ? A_BYTES : 0), st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, BN / 32, t, 128);
+            else split_tile(st + 2 * A_BYTES, B_BYTES, B_BYTES, t, 128);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
+            mbar_arrive(ready0 + 8 * s);
+        }
+        const int q = warp & 3;
+        if (ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true)) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int m = m0 + q * 32 + lane;
+            float* drow = p.D + ((long long)split * p.M + m) * p.N;
+            const float* arow = (!WGRAD && p.addend) ? p.addend + (long long)m * p.N : nullptr;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                if (num_kb > 0) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+                else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
+                const int nb = n0 + c * 32;
+                if (m < p.M) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (nb + g * 4 < p.N) {
+                            float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                            if (arow) { const float4 a = __ldg(reinterpret_cast<const float4*>(arow + nb + g * 4)); v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w; }
+                            *reinterpret_cast<float4*>(drow + nb + g * 4) = v;
+                        }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+}
+
+// rows x cols float matrix, cols contiguous; box = 32 columns x box_rows rows, 128-byte swizzle, zero fill
+bool make_map_f32(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)T32_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int STAGES, int MODE>
+bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const T32Params& p, dim3 grid, cudaStream_t st) {
+    constexpr int smem = STAGES * (2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0)) + 1024;
+    if (cudaFuncSetAttribute(tc32_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    tc32_kernel<BN, STAGES, MODE><<<grid, TC_THREADS, smem, st>>>(ma, mb, p);
+    return true;
+}
+
+struct Wg32Plan { int S, rows_per_split; };
+Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
+    const long long tiles = ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
+    long long S = (3LL * sm_count() + tiles - 1) / tiles;
+    const long long maxS = (R + 255) / 256;
+    long long cap = (8LL << 20) / ((long long)Mo * No);
+    if (cap < 1) cap = 1;
+    if (S > maxS) S = maxS;
+    if (S > cap) S = cap;
+    if (S < 1) S = 1;
+    const long long rps = ((R + S - 1) / S + 31) / 32 * 32;
+    Wg32Plan w;
+    w.rows_per_split = (int)rps;
+    w.S = (int)((R + rps - 1) / rps);
+    return w;
+}
+
+}  // namespace
+
+bool tc32_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend) {
+    auto a16 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
+    return M >= 1 && N % 4 == 0 && K % 4 == 0 && N >= 4 && K >= 4 && a16(A) && a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
+}
+
+// D[M,N] = A[M,K] * B (+ addend), float in and out, split-tf32 arithmetic.
+// b_is_kn == 0: B is [N][K] (K contiguous); b_is_kn == 1: B is [K][N] (N contiguous, as convolution weights lie).
+bool tc32_gemm(const float* A, const float* B, int b_is_kn, const float* addend, float* D, int M, int N, int K, int* err, cudaStream_t st) {
+    const int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
+    CUtensorMap ma, mb;
+    if (!make_map_f32(&ma, A, M, K, TC_BM)) return false;
+    if (!(b_is_kn ? make_map_f32(&mb, B, K, N, 32) : make_map_f32(&mb, B, N, K, BN))) return false;
+    T32Params p{D, addend, M, N, K, 0, err};
+    const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM);
+    if (b_is_kn) {
+        if (BN == 128) return launch32<128, 2, 2>(ma, mb, p, grid, st);
+        if (BN == 64) return launch32<64, 3, 2>(ma, mb, p, grid, st);
+        return launch32<32, 3, 2>(ma, mb, p, grid, st);
+    }
+    if (BN == 128) return launch32<128, 2, 0>(ma, mb, p, grid, st);
+    if (BN == 64) return launch32<64, 3, 0>(ma, mb, p, grid, st);
+    return launch32<32, 3, 0>(ma, mb, p, grid, st);
+}
+
+size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No) {
+    const Wg32Plan w = plan_wgrad32(R, Mo, No);
+    return w.S > 1 ? (size_t)w.S * Mo * No : 0;
+}
+
+// dW[Mo][No] = X[R][Mo]^T * dY[R][No]; returns the number of splits (0: nothing launched)
+int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st) {
+    const Wg32Plan w = plan_wgrad32(R, Mo, No);
+    const int BN = No > 64 ? 128 : (No > 32 ? 64 : 32);
+    CUtensorMap mx, my;
+    if (!make_map_f32(&mx, X, R, Mo, 32) || !make_map_f32(&my, dY, R, No, 32)) return 0;
+    T32Params p{w.S > 1 ? scratch : dW, nullptr, Mo, No, (int)R, w.rows_per_split, err};
+    const dim3 grid((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S);
+    bool ok;
+    if (BN == 128) ok = launch32<128, 2, 1>(mx, my, p, grid, st);
+    else if (BN == 64) ok = launch32<64, 2, 1>(mx, my, p, grid, st);
+    else ok = launch32<32, 3, 1>(mx, my, p, grid, st);
+    return ok ? w.S : 0;
+}
+
+}  // namespace ftp

@@ -54,6 +54,12 @@ int tc_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* 
 void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st);   // out = sum over S partial arrays, in order
 void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st);   // per matrix: wt[n][k] = bf16(w[k][n])
 
+// ---- float contractions on tensor cores with split-tf32 arithmetic (gemm_tc32.cu); same conventions as above ----
+bool tc32_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
+bool tc32_gemm(const float* A, const float* B, int b_is_kn, const float* addend, float* D, int M, int N, int K, int* err, cudaStream_t st);
+size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
+int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
+
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
 // Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole
 // 128-byte lines; `fold` picks f.  Partials are doubles: [chunks][2][C*f].

@@ -30,7 +30,8 @@ const char* kKernelNames[K_COUNT] = {
     "conv_fwd_f32", "conv_dgrad_f32", "conv_wgrad_f32", "bn_stats", "bn_finalize", "bn_apply", "bn_bwd_reduce",
     "bn_bwd_finalize", "bn_bwd_apply", "act_bias_bwd", "dw_fwd", "dw_dgrad", "dw_wgrad", "maxpool_fwd", "maxpool_bwd",
     "gap_fwd", "gap_bwd", "softmax_ce", "sgd", "act_fwd", "act_bwd", "copy", "tc_gemm_bf16_fwd", "tc_gemm_bf16_dgrad",
-    "tc_gemm_bf16_wgrad", "conv_fwd_bf16_simt", "conv_dgrad_bf16_simt", "conv_wgrad_bf16_simt"};
+    "tc_gemm_bf16_wgrad", "conv_fwd_bf16_simt", "conv_dgrad_bf16_simt", "conv_wgrad_bf16_simt",
+    "tc_gemm_tf32x3_fwd", "tc_gemm_tf32x3_dgrad", "tc_gemm_tf32x3_wgrad"};
 
 // Brackets one launcher call with events when tracing is on.
 struct Scope {
@@ -234,6 +235,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         } else if (is_contraction(o.d.kind)) {
             finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
             red = std::max(red, std::max(conv_wgrad_scratch_floats(o.g), conv_gemm_scratch_floats(o.g)));
+            red = std::max(red, tc32_wgrad_scratch_floats(Mout, o.C, o.Co));
             if (m.cfg.precision == FTP_BF16) red = std::max(red, std::max(tc_wgrad_scratch_floats(Mout, o.C, o.Co), tc_wgrad3x3_scratch_floats(Mout, o.C, o.Co)));
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
@@ -320,7 +322,10 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
                 if (m->cfg.precision == FTP_FP32) {
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
-                    conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
+                    const bool tc = is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, in, ar.w + o.w_off, out, nullptr) &&
+                                    tc32_gemm((const float*)in, ar.w + o.w_off, 1, nullptr, (float*)out, (int)Mout, o.Co, o.C, m->tc_err, st);
+                    if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_FWD;
+                    if (!tc) conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                 } else if constexpr (!std::is_same<T, float>::value) {
                     if (o.d.kind == FTP_FC) {           // the classifier runs in float on a widened copy of its input
                         Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, o.in_elems * 2.0 + (o.out_elems + o.w_cnt) * 4.0, fl, 2);
@@ -432,10 +437,19 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                         if (dpre) d = dpre;
                     }
                     { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
-                      conv_wgrad_f32(x, d, gr + o.w_off, m->red_scratch, o.g, st); }
+                      int splits = 0;
+                      if (is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr))
+                          splits = tc32_wgrad(x, d, gr + o.w_off, m->red_scratch, Mout, o.C, o.Co, m->tc_err, st);
+                      if (splits > 1) split_reduce_f32(m->red_scratch, splits, o.w_cnt, gr + o.w_off, st);
+                      if (splits > 0 && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
+                      if (splits == 0) conv_wgrad_f32(x, d, gr + o.w_off, m->red_scratch, o.g, st); }
                     if (gi) {
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
-                        conv_dgrad_f32(d, ar.w + o.w_off, widened ? nullptr : (const float*)addend, widened ? m->fc_din : (float*)gi, m->red_scratch, o.g, st);
+                        // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the weights as they lie are the K-major B operand
+                        const bool tc = !widened && is_pointwise_op(o) && tc32_supported((int)Mout, o.C, o.Co, d, ar.w + o.w_off, gi, addend) &&
+                                        tc32_gemm(d, ar.w + o.w_off, 0, (const float*)addend, (float*)gi, (int)Mout, o.C, o.Co, m->tc_err, st);
+                        if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_DGRAD;
+                        if (!tc) conv_dgrad_f32(d, ar.w + o.w_off, widened ? nullptr : (const float*)addend, widened ? m->fc_din : (float*)gi, m->red_scratch, o.g, st);
                         if (widened) f32_to_bf16(m->fc_din, (__nv_bfloat16*)gi, o.in_elems, st);
                     }
                 } else if constexpr (!std::is_same<T, float>::value) {

@@ -12,7 +12,7 @@ enum KernelId {
     K_CONV_FWD_F32 = 0, K_CONV_DGRAD_F32, K_CONV_WGRAD_F32, K_BN_STATS, K_BN_FINALIZE, K_BN_APPLY, K_BN_BWD_REDUCE,
     K_BN_BWD_FINALIZE, K_BN_BWD_APPLY, K_ACT_BIAS_BWD, K_DW_FWD, K_DW_DGRAD, K_DW_WGRAD, K_MAXPOOL_FWD,
     K_MAXPOOL_BWD, K_GAP_FWD, K_GAP_BWD, K_SOFTMAX_CE, K_SGD, K_ACT_FWD, K_ACT_BWD, K_COPY, K_GEMM_BF16_FWD,
-    K_GEMM_BF16_DGRAD, K_GEMM_BF16_WGRAD, K_CONV_FWD_BF16_SIMT, K_CONV_DGRAD_BF16_SIMT, K_CONV_WGRAD_BF16_SIMT, K_COUNT
+    K_GEMM_BF16_DGRAD, K_GEMM_BF16_WGRAD, K_CONV_FWD_BF16_SIMT, K_CONV_DGRAD_BF16_SIMT, K_CONV_WGRAD_BF16_SIMT, K_TC32_FWD, K_TC32_DGRAD, K_TC32_WGRAD, K_COUNT
 };
 
 struct Op {
