@@ -79,7 +79,7 @@ struct T32Params {
 // in shared memory (weight gradient).  MODE 2: A [M][K] as it lies, B [K][N] (the weights) transposed (forward).
 template <int BN, int STAGES, int MODE>
 __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                                                          const T32Params p) {
+                                                          const __grid_constant__ CUtensorMap mapD, const T32Params p) {
     constexpr uint32_t A_BYTES = TC_BM * T32_BK * 4, B_BYTES = BN * T32_BK * 4;          // one precision part
     constexpr bool TA = MODE == 1, TB = MODE != 0;                                      // operand transposed in shared memory
     constexpr uint32_t STAGE_BYTES = 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) + (TB ? B_BYTES : 0);   // [A hi][A lo][B hi][B lo][A src][B src]
@@ -99,6 +99,11 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
         n0 = blockIdx.x * BN; m0 = blockIdx.y * TC_BM; kbeg = 0; kend = p.K;
     }
     const int num_kb = (kend - kbeg + T32_BK - 1) / T32_BK;
+    // transposed operands arrive as 32-column slabs: slabs wholly beyond the matrix are neither loaded nor converted
+    // (their rows of the hi / lo tiles are cleared once)
+    const int slabsA = TA ? min(TC_BM / 32, (p.M - m0 + 31) / 32) : TC_BM / 32;
+    const int slabsB = TB ? min(BN / 32, (p.N - n0 + 31) / 32) : BN / 32;
+    const uint32_t tx_bytes = (TA ? slabsA * SLAB : A_BYTES) + (TB ? slabsB * SLAB : B_BYTES);
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), ready0 = smem_u32(&bars[2 * STAGES]), accum = smem_u32(&bars[3 * STAGES]);
 
     if (threadIdx.x == 0) {
@@ -126,14 +131,12 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
                 const uint32_t sa = TA ? st0 + 2 * (A_BYTES + B_BYTES) : st0;                                       // where A lands
                 const uint32_t sb = TB ? st0 + 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) : st0 + 2 * A_BYTES;   // where B lands
                 const int k = kbeg + kb * T32_BK;
-                mbar_expect_tx(full0 + 8 * s, A_BYTES + B_BYTES);
+                mbar_expect_tx(full0 + 8 * s, tx_bytes);
                 if (TA) {
-#pragma unroll
-                    for (int t = 0; t < TC_BM / 32; ++t) tma_load_2d(sa + t * SLAB, &mapA, m0 + 32 * t, k, full0 + 8 * s);
+                    for (int t = 0; t < slabsA; ++t) tma_load_2d(sa + t * SLAB, &mapA, m0 + 32 * t, k, full0 + 8 * s);
                 } else tma_load_2d(sa, &mapA, k, m0, full0 + 8 * s);
                 if (TB) {
-#pragma unroll
-                    for (int t = 0; t < BN / 32; ++t) tma_load_2d(sb + t * SLAB, &mapB, n0 + 32 * t, k, full0 + 8 * s);
+                    for (int t = 0; t < slabsB; ++t) tma_load_2d(sb + t * SLAB, &mapB, n0 + 32 * t, k, full0 + 8 * s);
                 } else tma_load_2d(sb, &mapB, k, n0, full0 + 8 * s);
                 issued = kb + 1;
             }
@@ -172,6 +175,15 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
         // ---- warps 2..5: split every landed stage, then the epilogue ----
         const int t = threadIdx.x - 64;
         bool ok = true;
+        if ((TA && slabsA < TC_BM / 32) || (TB && slabsB < BN / 32)) {
+            // clear the rows of the hi / lo tiles that no slab will ever fill
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s = 0; s < STAGES; ++s) {
+                uint8_t* st = smem + s * STAGE_BYTES;
+                if (TA) for (int i = slabsA * SLAB + t * 16; i < (int)A_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + i) = z; *reinterpret_cast<float4*>(st + A_BYTES + i) = z; }
+                if (TB) for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
+            }
+        }
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % STAGES;
             const uint32_t ph = (kb / STAGES) & 1;
@@ -179,19 +191,21 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
             if (!ok) break;
             uint8_t* st = smem + s * STAGE_BYTES;
             uint8_t* src = st + 2 * (A_BYTES + B_BYTES);
-            if (TA) transpose_split(src, st, st + A_BYTES, TC_BM / 32, t, 128);
+            if (TA) transpose_split(src, st, st + A_BYTES, slabsA, t, 128);
             else split_tile(st, A_BYTES, A_BYTES, t, 128);
-            if (TB) transpose_split(src + (TA ? A_BYTES : 0), st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, BN / 32, t, 128);
+            if (TB) transpose_split(src + (TA ? A_BYTES : 0), st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, t, 128);
             else split_tile(st + 2 * A_BYTES, B_BYTES, B_BYTES, t, 128);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
             mbar_arrive(ready0 + 8 * s);
         }
+        // ---- epilogue: accumulator -> shared-memory tiles of 128 rows x 32 columns (the operand stages are free
+        // now) -> one TMA store per tile, which writes whole lines and clips at the edges of the output ----
         const int q = warp & 3;
-        if (ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true)) {
+        const bool have = ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true);
+        if (have) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int m = m0 + q * 32 + lane;
-            float* drow = p.D + ((long long)split * p.M + m) * p.N;
-            const float* arow = (!WGRAD && p.addend) ? p.addend + (long long)m * p.N : nullptr;
+            const int row = q * 32 + lane, m = m0 + row;
+            const float* arow = (!WGRAD && p.addend && m < p.M) ? p.addend + (long long)m * p.N : nullptr;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
@@ -201,16 +215,25 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
                     for (int e = 0; e < 32; ++e) r[e] = 0u;
                 }
                 const int nb = n0 + c * 32;
-                if (m < p.M) {
+                uint8_t* trow = smem + c * (TC_BM * 128) + row * 128;
 #pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        if (nb + g * 4 < p.N) {
-                            float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
-                            if (arow) { const float4 a = __ldg(reinterpret_cast<const float4*>(arow + nb + g * 4)); v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w; }
-                            *reinterpret_cast<float4*>(drow + nb + g * 4) = v;
-                        }
+                for (int g = 0; g < 8; ++g) {
+                    float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                    if (arow && nb + g * 4 < p.N) { const float4 a = __ldg(reinterpret_cast<const float4*>(arow + nb + g * 4)); v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w; }
+                    *reinterpret_cast<float4*>(trow + ((g ^ (row & 7)) << 4)) = v;
                 }
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");                      // the four epilogue warps
+        if (have && threadIdx.x == 64) {
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c)
+                if (n0 + c * 32 < p.N)
+                    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                                 ::"l"(&mapD), "r"(n0 + c * 32), "r"(m0), "r"(split), "r"(smem_u32(smem + c * (TC_BM * 128))) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -230,11 +253,25 @@ bool make_map_f32(CUtensorMap* map, const void* base, long long rows, long long 
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// output [S][rows][cols] floats; box = 32 columns x 128 rows x 1, 128-byte swizzle (stores clip at the edges)
+bool make_map_out(CUtensorMap* map, const void* base, long long S, long long rows, long long cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)S};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)rows * cols * 4};
+    const cuuint32_t box[3] = {32, (cuuint32_t)TC_BM, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, int STAGES, int MODE>
-bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const T32Params& p, dim3 grid, cudaStream_t st) {
-    constexpr int smem = STAGES * (2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0)) + 1024;
+bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
+    constexpr int ring = STAGES * (2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0));
+    constexpr int stage_out = TC_BM * BN * 4;                         // the epilogue reuses the ring as its staging area
+    constexpr int smem = (ring > stage_out ? ring : stage_out) + 1024;
     if (cudaFuncSetAttribute(tc32_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    tc32_kernel<BN, STAGES, MODE><<<grid, TC_THREADS, smem, st>>>(ma, mb, p);
+    tc32_kernel<BN, STAGES, MODE><<<grid, TC_THREADS, smem, st>>>(ma, mb, md, p);
     return true;
 }
 
@@ -262,23 +299,38 @@ bool tc32_supported(int M, int N, int K, const void* A, const void* B, const voi
     return M >= 1 && N % 4 == 0 && K % 4 == 0 && N >= 4 && K >= 4 && a16(A) && a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
 }
 
+template <int BN, int MODE>
+bool launch32_stages(int num_kb, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
+    // Many tiles (memory-bound layers): one stage per CTA, so that several CTAs share an SM and hide each other's
+    // latencies.  Few tiles (late layers, long reductions): a deeper ring inside the CTA instead.
+    constexpr int MAXS = BN == 128 ? 2 : 3;
+    const long long tiles = (long long)grid.x * grid.y * grid.z;
+    int stages = tiles >= 4LL * sm_count() ? 1 : (tiles >= 2LL * sm_count() ? 2 : MAXS);
+    if (stages > num_kb) stages = num_kb < 1 ? 1 : num_kb;
+    if (stages > MAXS) stages = MAXS;
+    if (stages == 1) return launch32<BN, 1, MODE>(ma, mb, md, p, grid, st);
+    if (stages == 2) return launch32<BN, 2, MODE>(ma, mb, md, p, grid, st);
+    return launch32<BN, 3, MODE>(ma, mb, md, p, grid, st);
+}
+
 // D[M,N] = A[M,K] * B (+ addend), float in and out, split-tf32 arithmetic.
 // b_is_kn == 0: B is [N][K] (K contiguous); b_is_kn == 1: B is [K][N] (N contiguous, as convolution weights lie).
 bool tc32_gemm(const float* A, const float* B, int b_is_kn, const float* addend, float* D, int M, int N, int K, int* err, cudaStream_t st) {
     const int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
-    CUtensorMap ma, mb;
-    if (!make_map_f32(&ma, A, M, K, TC_BM)) return false;
+    CUtensorMap ma, mb, md;
+    if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, D, 1, M, N)) return false;
     if (!(b_is_kn ? make_map_f32(&mb, B, K, N, 32) : make_map_f32(&mb, B, N, K, BN))) return false;
     T32Params p{D, addend, M, N, K, 0, err};
     const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM);
+    const int nkb = (K + T32_BK - 1) / T32_BK;
     if (b_is_kn) {
-        if (BN == 128) return launch32<128, 2, 2>(ma, mb, p, grid, st);
-        if (BN == 64) return launch32<64, 3, 2>(ma, mb, p, grid, st);
-        return launch32<32, 3, 2>(ma, mb, p, grid, st);
+        if (BN == 128) return launch32_stages<128, 2>(nkb, ma, mb, md, p, grid, st);
+        if (BN == 64) return launch32_stages<64, 2>(nkb, ma, mb, md, p, grid, st);
+        return launch32_stages<32, 2>(nkb, ma, mb, md, p, grid, st);
     }
-    if (BN == 128) return launch32<128, 2, 0>(ma, mb, p, grid, st);
-    if (BN == 64) return launch32<64, 3, 0>(ma, mb, p, grid, st);
-    return launch32<32, 3, 0>(ma, mb, p, grid, st);
+    if (BN == 128) return launch32_stages<128, 0>(nkb, ma, mb, md, p, grid, st);
+    if (BN == 64) return launch32_stages<64, 0>(nkb, ma, mb, md, p, grid, st);
+    return launch32_stages<32, 0>(nkb, ma, mb, md, p, grid, st);
 }
 
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No) {
@@ -290,14 +342,16 @@ size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No) {
 int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st) {
     const Wg32Plan w = plan_wgrad32(R, Mo, No);
     const int BN = No > 64 ? 128 : (No > 32 ? 64 : 32);
-    CUtensorMap mx, my;
-    if (!make_map_f32(&mx, X, R, Mo, 32) || !make_map_f32(&my, dY, R, No, 32)) return 0;
-    T32Params p{w.S > 1 ? scratch : dW, nullptr, Mo, No, (int)R, w.rows_per_split, err};
+    CUtensorMap mx, my, md;
+    float* out = w.S > 1 ? scratch : dW;
+    if (!make_map_f32(&mx, X, R, Mo, 32) || !make_map_f32(&my, dY, R, No, 32) || !make_map_out(&md, out, w.S, Mo, No)) return 0;
+    T32Params p{out, nullptr, Mo, No, (int)R, w.rows_per_split, err};
     const dim3 grid((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S);
+    const int nkb = (w.rows_per_split + T32_BK - 1) / T32_BK;
     bool ok;
-    if (BN == 128) ok = launch32<128, 2, 1>(mx, my, p, grid, st);
-    else if (BN == 64) ok = launch32<64, 2, 1>(mx, my, p, grid, st);
-    else ok = launch32<32, 3, 1>(mx, my, p, grid, st);
+    if (BN == 128) ok = launch32_stages<128, 1>(nkb, mx, my, md, p, grid, st);
+    else if (BN == 64) ok = launch32_stages<64, 1>(nkb, mx, my, md, p, grid, st);
+    else ok = launch32_stages<32, 1>(nkb, mx, my, md, p, grid, st);
     return ok ? w.S : 0;
 }
 
