@@ -4,9 +4,21 @@
 // reduction runs in a fixed order (per-thread run, shared-memory column sum, then a second pass
 // over the per-block partials) so results do not depend on scheduling.
 #include <cfloat>
+#include <cstdlib>
+#include <cstring>
 #include "kernels.h"
+#include "launch.cuh"
 
 namespace ftp {
+
+bool pdl_enabled() {
+    static int on = -1;
+    if (on < 0) {
+        const char* e = std::getenv("FTP_PDL");
+        on = (e && std::strcmp(e, "0") == 0) ? 0 : 1;
+    }
+    return on == 1;
+}
 
 int sm_count() {
     static int n = 0;
@@ -120,55 +132,55 @@ __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chu
 }
 
 // Second pass of every folded column reduction: sums over chunks and folded copies, one channel per x-lane.
-// Grid (channel groups of 32, G slices of the (chunk, copy) pairs, extra); block (32, FIN_Y).  Inside a block,
-// y -> strided runs with four independent accumulators, then a fixed-order sum over y in shared memory.  With
+// Grid (channel groups of FIN_X, G slices of the (chunk, copy) pairs, extra); block (FIN_X, FIN_Y).  Inside a block,
+// y -> strided runs, four loads in flight at a time, then a fixed-shape tree over y in shared memory.  With
 // G > 1 every block parks its slice sums in fin.part and takes a ticket; the block that draws the last ticket
 // adds the G slice sums in slice order, so the result does not depend on which block that is.  Returns true in
 // the block that holds the final sums (valid in its threads with y == 0).  NS consecutive sums from `first`.
-constexpr int FIN_Y = 32;
+constexpr int FIN_X = 8;
+constexpr int FIN_Y = 128;
 constexpr int FIN_GMAX = 16;
 template <typename PT, int NS>
 __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int ns, int chunks, int f, int C, int cols, int c,
                                               const FinScratch fin, double (&out)[NS]) {
-    __shared__ double red[NS][FIN_Y][33];
+    __shared__ double red[NS][FIN_Y][FIN_X + 1];
     __shared__ unsigned ticket;
-    double t[NS][4];
+    double t[NS];
 #pragma unroll
-    for (int a = 0; a < NS; ++a)
-#pragma unroll
-        for (int u = 0; u < 4; ++u) t[a][u] = 0.0;
+    for (int a = 0; a < NS; ++a) t[a] = 0.0;
     const int total = chunks * f, G = gridDim.y;
     const int per = (total + G - 1) / G, e0 = blockIdx.y * per, e1 = min(total, e0 + per);
-    if (c < C)
-        for (int e = e0 + threadIdx.y; e < e1; e += 4 * FIN_Y) {
+    for (int e = e0 + threadIdx.y; e < e1; e += 4 * FIN_Y) {
+        double v[NS][4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int ee = e + u * FIN_Y;
-                if (ee < e1) {
-                    const int ch = ee / f, k = ee - ch * f;
+        for (int u = 0; u < 4; ++u) {                    // four independent loads in flight per sum
+            const int ee = e + u * FIN_Y;
+            const bool ok = ee < e1 && c < C;
+            const int ch = ok ? ee / f : 0, k = ok ? ee - ch * f : 0;
 #pragma unroll
-                    for (int a = 0; a < NS; ++a) t[a][u] += (double)partial[((long long)ch * ns + first + a) * cols + k * C + c];
-                }
-            }
+            for (int a = 0; a < NS; ++a) v[a][u] = ok ? (double)partial[((long long)ch * ns + first + a) * cols + k * C + c] : 0.0;
         }
-    __syncthreads();
 #pragma unroll
-    for (int a = 0; a < NS; ++a) red[a][threadIdx.y][threadIdx.x] = (t[a][0] + t[a][1]) + (t[a][2] + t[a][3]);
-    __syncthreads();
-#pragma unroll
-    for (int a = 0; a < NS; ++a) {
-        double r = 0.0;
-        if (threadIdx.y == 0)
-#pragma unroll 8
-            for (int y = 0; y < FIN_Y; ++y) r += red[a][y][threadIdx.x];
-        out[a] = r;
+        for (int a = 0; a < NS; ++a) t[a] += (v[a][0] + v[a][1]) + (v[a][2] + v[a][3]);
     }
+#pragma unroll
+    for (int a = 0; a < NS; ++a) red[a][threadIdx.y][threadIdx.x] = t[a];
+    __syncthreads();
+#pragma unroll 1
+    for (int s = FIN_Y / 2; s >= 1; s >>= 1) {           // fixed-shape tree over y
+        if ((int)threadIdx.y < s)
+#pragma unroll
+            for (int a = 0; a < NS; ++a) red[a][threadIdx.y][threadIdx.x] += red[a][threadIdx.y + s][threadIdx.x];
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < NS; ++a) out[a] = red[a][0][threadIdx.x];
     if (G == 1) return true;
     const int slot = blockIdx.z * gridDim.x + blockIdx.x;
-    double* mine = fin.part + ((long long)slot * FIN_GMAX + blockIdx.y) * NS * 32;
+    double* mine = fin.part + ((long long)slot * FIN_GMAX + blockIdx.y) * NS * FIN_X;
     if (threadIdx.y == 0)
 #pragma unroll
-        for (int a = 0; a < NS; ++a) mine[a * 32 + threadIdx.x] = out[a];
+        for (int a = 0; a < NS; ++a) mine[a * FIN_X + threadIdx.x] = out[a];
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0 && threadIdx.y == 0) ticket = atomicAdd(fin.counters + slot, 1u);
@@ -179,7 +191,7 @@ __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int 
 #pragma unroll
         for (int a = 0; a < NS; ++a) {
             double r = 0.0;
-            for (int g = 0; g < G; ++g) r += __ldcg(fin.part + ((long long)slot * FIN_GMAX + g) * NS * 32 + a * 32 + threadIdx.x);
+            for (int g = 0; g < G; ++g) r += __ldcg(fin.part + ((long long)slot * FIN_GMAX + g) * NS * FIN_X + a * FIN_X + threadIdx.x);
             out[a] = r;
         }
         if (threadIdx.x == 0) fin.counters[slot] = 0u;       // ready for the next launch on this stream
@@ -189,6 +201,7 @@ __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int 
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, int rows, int cols, int rpc, double* __restrict__ partial) {
+    grid_dep_sync();
     fold_reduce<T, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
         float v[V];
         ldv<V>(y + off, v);
@@ -201,7 +214,8 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
                                    float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd,
                                    const FinScratch fin) {
-    const int c = blockIdx.x * 32 + threadIdx.x;
+    grid_dep_sync();
+    const int c = blockIdx.x * FIN_X + threadIdx.x;
     double ss[2];
     if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
@@ -231,6 +245,7 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const T* __restrict__ y, 
                                                        int rows, int cols, int rpc, int C, const float* __restrict__ scale,
                                                        const float* __restrict__ shift, const float* __restrict__ mean,
                                                        const float* __restrict__ mean_lo, int act) {
+    grid_dep_sync();
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     if (col >= cols) return;
     const int c = col % C;
@@ -258,6 +273,7 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
                                                             const float* __restrict__ scale, const float* __restrict__ shift,
                                                             const float* __restrict__ mean, const float* __restrict__ mean_lo,
                                                             const float* __restrict__ rstd, int act, double* __restrict__ partial) {
+    grid_dep_sync();
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     float sc[V], sh[V], mu[V], ml[V], rs[V];
     if (col < cols) { const int c = col % C; ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml); ldtab<V>(rstd + c, rs); }
@@ -277,7 +293,8 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
 __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
                                        const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
                                        float* dbeta, float* coef, const FinScratch fin) {
-    const int c = blockIdx.x * 32 + threadIdx.x;
+    grid_dep_sync();
+    const int c = blockIdx.x * FIN_X + threadIdx.x;
     double ss[2];
     if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
@@ -299,6 +316,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
                                                            const float* __restrict__ shift, const float* __restrict__ mean,
                                                            const float* __restrict__ mean_lo, const float* __restrict__ rstd,
                                                            const float* __restrict__ coef, int act) {
+    grid_dep_sync();
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     if (col >= cols) return;
     const int c = col % C;
@@ -335,6 +353,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
 template <typename T, int V>
 __global__ void __launch_bounds__(256) act_bias_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ out, T* __restrict__ dpre,
                                                            int rows, int cols, int rpc, int act, double* __restrict__ partial) {
+    grid_dep_sync();
     fold_reduce<T, V, 1>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[1][V]) {
         float d[V];
         ldv<V>(dout + off, d);
@@ -351,7 +370,8 @@ __global__ void __launch_bounds__(256) act_bias_bwd_kernel(const T* __restrict__
 }
 
 __global__ void colsum_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, float* out, const FinScratch fin) {
-    const int c = blockIdx.x * 32 + threadIdx.x;
+    grid_dep_sync();
+    const int c = blockIdx.x * FIN_X + threadIdx.x;
     double ss[1];
     if (!col_fold_sums<double, 1>(partial, 0, 1, chunks, f, C, cols, c, fin, ss)) return;
     if (threadIdx.y == 0 && c < C) out[c] = (float)ss[0];
@@ -359,6 +379,7 @@ __global__ void colsum_finalize_kernel(const double* __restrict__ partial, int c
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256) act_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, long long nvec, int act) {
+    grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         float v[V];
         ldv<V>(x + i * V, v);
@@ -371,6 +392,7 @@ __global__ void __launch_bounds__(256) act_fwd_kernel(const T* __restrict__ x, T
 template <typename T, int V>
 __global__ void __launch_bounds__(256) act_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ x, const T* __restrict__ addend,
                                                       T* __restrict__ dx, long long nvec, int act) {
+    grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         float d[V], v[V];
         ldv<V>(dout + i * V, d);
@@ -388,15 +410,28 @@ __global__ void __launch_bounds__(256) act_bwd_kernel(const T* __restrict__ dout
 }
 
 // ---- depthwise 3x3 ------------------------------------------------------------------------------
+// The two gather kernels below map a block of 256 threads onto a tile of 64 output pixels (TW = 2^tws wide,
+// 64 / TW rows of the (image, row) index space) times 8 channel vectors, two pixels per thread, so that the
+// nine taps of neighbouring outputs hit the lines their neighbours just fetched.  grid (pixel tiles, ceil(CV / 8)).
 template <typename T, int V>
-__global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, ConvGeom g, long long total) {
+__global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, ConvGeom g, int tws) {
+    grid_dep_sync();
     const int CV = g.Cin / V;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(i % CV) * V;
-        long long pix = i / CV;
-        const int wo = (int)(pix % g.Wo); pix /= g.Wo;
-        const int ho = (int)(pix % g.Ho);
-        const int n = (int)(pix / g.Ho);
+    const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
+    if (cv >= CV) return;
+    const int c = cv * V;
+    const int slot = threadIdx.x >> 3, TW = 1 << tws, half = 32 >> tws;
+    const int tiles_w = (g.Wo + TW - 1) >> tws;
+    const int tw_i = blockIdx.x % tiles_w, tr_i = blockIdx.x / tiles_w;
+    const int wo = tw_i * TW + (slot & (TW - 1));
+    if (wo >= g.Wo) return;
+    const int rows = g.N * g.Ho;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int R = tr_i * 2 * half + (slot >> tws) + k * half;
+        if (R >= rows) break;
+        const int n = R / g.Ho, ho = R - n * g.Ho;
+        const long long i = ((long long)R * g.Wo + wo) * CV + cv;
         float acc[V];
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[e] = 0.f;
@@ -421,14 +456,24 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, co
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy, const float* __restrict__ w, const T* __restrict__ addend,
-                                                       T* __restrict__ dx, ConvGeom g, long long total) {
+                                                       T* __restrict__ dx, ConvGeom g, int tws) {
+    grid_dep_sync();
     const int CV = g.Cin / V;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(i % CV) * V;
-        long long pix = i / CV;
-        const int wi = (int)(pix % g.W); pix /= g.W;
-        const int hi = (int)(pix % g.H);
-        const int n = (int)(pix / g.H);
+    const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
+    if (cv >= CV) return;
+    const int c = cv * V;
+    const int slot = threadIdx.x >> 3, TW = 1 << tws, half = 32 >> tws;
+    const int tiles_w = (g.W + TW - 1) >> tws;
+    const int tw_i = blockIdx.x % tiles_w, tr_i = blockIdx.x / tiles_w;
+    const int wi = tw_i * TW + (slot & (TW - 1));
+    if (wi >= g.W) return;
+    const int rows = g.N * g.H;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int R = tr_i * 2 * half + (slot >> tws) + k * half;
+        if (R >= rows) break;
+        const int n = R / g.H, hi = R - n * g.H;
+        const long long i = ((long long)R * g.W + wi) * CV + cv;
         float acc[V];
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[e] = 0.f;
@@ -468,6 +513,7 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
 template <typename T, int V>
 __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, ConvGeom g,
                                                        int rows, int cols, int f, int rpc) {
+    grid_dep_sync();
     __shared__ float sh[3][8][32 * V];
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     const int r0 = blockIdx.y * rpc, r1 = min(rows, r0 + rpc);
@@ -525,7 +571,8 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, 
 // dw[t][c] = sum over chunks and folded copies of partial[chunk][t][copy * C + c]; grid (ceil(C/32), G, 9)
 __global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols, float* __restrict__ dw,
                                          const FinScratch fin) {
-    const int c = blockIdx.x * 32 + threadIdx.x;
+    grid_dep_sync();
+    const int c = blockIdx.x * FIN_X + threadIdx.x;
     double ss[1];
     if (!col_fold_sums<float, 1>(partial, (int)blockIdx.z, 9, chunks, f, C, cols, c, fin, ss)) return;
     if (threadIdx.y == 0 && c < C) dw[blockIdx.z * C + c] = (float)ss[0];
@@ -534,6 +581,7 @@ __global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int 
 // ---- pooling --------------------------------------------------------------------------------------
 template <typename T, int V>
 __global__ void __launch_bounds__(256) maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int H, int W, int C, long long total) {
+    grid_dep_sync();
     const int CV = C / V, Ho = H / 2, Wo = W / 2;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % CV) * V;
@@ -558,6 +606,7 @@ __global__ void __launch_bounds__(256) maxpool_fwd_kernel(const T* __restrict__ 
 // maximum in row-major window order, zero elsewhere (rows/columns beyond 2*floor(H/2) get zero too)
 template <typename T, int V>
 __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ x, T* __restrict__ dx, int H, int W, int C, long long total) {
+    grid_dep_sync();
     const int CV = C / V, Ho = H / 2, Wo = W / 2;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % CV) * V;
@@ -589,6 +638,7 @@ __global__ void __launch_bounds__(256) maxpool_bwd_kernel(const T* __restrict__ 
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256) gap_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int HW, int C, long long total) {
+    grid_dep_sync();
     const int CV = C / V;
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
@@ -611,6 +661,7 @@ __global__ void __launch_bounds__(256) gap_fwd_kernel(const T* __restrict__ x, T
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256) gap_bwd_kernel(const T* __restrict__ dy, T* __restrict__ dx, int HW, int C, long long total) {
+    grid_dep_sync();
     const int CV = C / V;
     const float inv = 1.f / (float)HW;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
@@ -639,6 +690,7 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
 
 __global__ void __launch_bounds__(128) softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int N, int K,
                                                          float* __restrict__ per_sample, float* __restrict__ dlogits) {
+    grid_dep_sync();
     __shared__ float sh[4];
     const int n = blockIdx.x;
     const float* z = logits + (long long)n * K;
@@ -660,6 +712,7 @@ __global__ void __launch_bounds__(128) softmax_ce_kernel(const float* __restrict
 }
 
 __global__ void loss_mean_kernel(const float* __restrict__ per_sample, int N, float* loss) {
+    grid_dep_sync();
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         double s = 0.0;
         for (int i = 0; i < N; ++i) s += (double)per_sample[i];
@@ -672,6 +725,7 @@ template <int V>
 __global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, long long nvec, float lr,
                                                   float mu, float wd, int first, __nv_bfloat16* __restrict__ shadow,
                                                   float* __restrict__ snap_dev, float* __restrict__ snap_host) {
+    grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         float wv[V], gv[V], mv[V];
         ldv<V>(w + i * V, wv);
@@ -699,17 +753,20 @@ __global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const f
 }
 
 __global__ void f32_to_bf16_kernel(const float* __restrict__ s, __nv_bfloat16* __restrict__ d, long long n) {
+    grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         d[i] = __float2bfloat16_rn(s[i]);
 }
 
 __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ s, float* __restrict__ d, long long n) {
+    grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         d[i] = __bfloat162float(s[i]);
 }
 
 // wt[n][k] = bf16(w[k][n]) through a 32 x 32 shared-memory tile
 __global__ void transpose_f32_to_bf16_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ wt, int K, int N) {
+    grid_dep_sync();
     __shared__ float tile[32][33];
     const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
     w += (long long)blockIdx.z * K * N;
@@ -756,10 +813,10 @@ FoldPlan make_fold(long long M, int C, int elem_bytes) {
 
 size_t fold_partial_doubles(const FoldPlan& fp) { return (size_t)fp.chunks * 2 * fp.cols; }
 
-size_t fin_part_doubles(int C, int extra) { return (size_t)((C + 31) / 32) * extra * FIN_GMAX * 2 * 32; }
-size_t fin_counter_count(int C, int extra) { return (size_t)((C + 31) / 32) * extra; }
+size_t fin_part_doubles(int C, int extra) { return (size_t)((C + FIN_X - 1) / FIN_X) * extra * FIN_GMAX * 2 * FIN_X; }
+size_t fin_counter_count(int C, int extra) { return (size_t)((C + FIN_X - 1) / FIN_X) * extra; }
 static inline int fin_slices(const FoldPlan& fp) {
-    const int g = fp.chunks * fp.f / 256;
+    const int g = fp.chunks * fp.f / (4 * FIN_Y);
     return g < 1 ? 1 : (g > FIN_GMAX ? FIN_GMAX : g);
 }
 
@@ -769,14 +826,14 @@ static inline dim3 fold_grid(const FoldPlan& fp) { return dim3((fp.cols + 32 * f
 template <typename T>
 void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    if (fp.vec == V && aligned16(y)) bn_stats_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(y, fp.rows, fp.cols, fold_rpc(fp), partial);
-    else bn_stats_kernel<T, 1><<<fold_grid(fp), dim3(32, 8), 0, st>>>(y, fp.rows, fp.cols, fold_rpc(fp), partial);
+    if (fp.vec == V && aligned16(y)) launch(bn_stats_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, fp.rows, fp.cols, fold_rpc(fp), partial);
+    else launch(bn_stats_kernel<T, 1>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, fp.rows, fp.cols, fold_rpc(fp), partial);
 }
 
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
                  float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st) {
-    bn_finalize_kernel<<<dim3((C + 31) / 32, fin_slices(fp)), dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
+    launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
                                                              run_mean, run_var, scale, shift, mean, mean_lo, rstd, fin);
 }
 
@@ -785,9 +842,9 @@ void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const Fol
               const float* mean, const float* mean_lo, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     if (fp.vec == V && aligned16(y) && aligned16(residual) && aligned16(z) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo))
-        bn_apply_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(y, residual, z, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, act);
+        launch(bn_apply_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, residual, z, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, act);
     else
-        bn_apply_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(y, residual, z, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, act);
+        launch(bn_apply_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, y, residual, z, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, act);
 }
 
 template <typename T>
@@ -795,16 +852,16 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
                    const float* mean, const float* mean_lo, const float* rstd, int act, double* partial, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd))
-        bn_bwd_reduce_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial);
+        launch(bn_bwd_reduce_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial);
     else {
         FoldPlan s = fp;                       // scalar fallback keeps the same partial layout
-        bn_bwd_reduce_kernel<T, 1><<<dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st>>>(dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, mean_lo, rstd, act, partial);
+        launch(bn_bwd_reduce_kernel<T, 1>, dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st, dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, mean_lo, rstd, act, partial);
     }
 }
 
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
                      float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st) {
-    bn_bwd_finalize_kernel<<<dim3((C + 31) / 32, fin_slices(fp)), dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
+    launch(bn_bwd_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
 }
 
 template <typename T>
@@ -813,9 +870,9 @@ void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, 
     constexpr int V = VecOf<T>::N;
     if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(addend) && aligned16(dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) &&
         aligned16(mean_lo) && aligned16(rstd) && aligned16(coef))
-        bn_bwd_apply_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
+        launch(bn_bwd_apply_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
     else
-        bn_bwd_apply_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
+        launch(bn_bwd_apply_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
 }
 
 template <typename T>
@@ -823,41 +880,46 @@ void act_bias_bwd(const T* dout, const T* out, T* dpre, long long M, int C, int 
                   float* dbias, const FinScratch& fin, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     if (fp.vec == V && aligned16(dout) && aligned16(out) && aligned16(dpre))
-        act_bias_bwd_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
+        launch(act_bias_bwd_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
     else
-        act_bias_bwd_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
-    if (dbias) colsum_finalize_kernel<<<dim3((C + 31) / 32, fin_slices(fp)), dim3(32, FIN_Y), 0, st>>>(partial, fp.chunks, fp.f, C, fp.cols, dbias, fin);
+        launch(act_bias_bwd_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, dout, out, dpre, fp.rows, fp.cols, fold_rpc(fp), act, partial);
+    if (dbias) launch(colsum_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, dbias, fin);
 }
 
 template <typename T>
 void act_fwd(const T* x, T* y, long long n, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    if (n % V == 0 && aligned16(x) && aligned16(y)) act_fwd_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(x, y, n / V, act);
-    else act_fwd_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(x, y, n, act);
+    if (n % V == 0 && aligned16(x) && aligned16(y)) launch(act_fwd_kernel<T, V>, dim3(flat_blocks(n / V, 256)), dim3(256), 0, st, x, y, n / V, act);
+    else launch(act_fwd_kernel<T, 1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, x, y, n, act);
 }
 
 template <typename T>
 void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     if (n % V == 0 && aligned16(dout) && aligned16(x) && aligned16(addend) && aligned16(dx))
-        act_bwd_kernel<T, V><<<flat_blocks(n / V, 256), 256, 0, st>>>(dout, x, addend, dx, n / V, act);
-    else act_bwd_kernel<T, 1><<<flat_blocks(n, 256), 256, 0, st>>>(dout, x, addend, dx, n, act);
+        launch(act_bwd_kernel<T, V>, dim3(flat_blocks(n / V, 256)), dim3(256), 0, st, dout, x, addend, dx, n / V, act);
+    else launch(act_bwd_kernel<T, 1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, dout, x, addend, dx, n, act);
 }
+
+// log2 of the tile width: the largest power of two <= min(8, width)
+static inline int dw_tile_shift(int width) { return width >= 8 ? 3 : width >= 4 ? 2 : width >= 2 ? 1 : 0; }
 
 template <typename T>
 void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    const long long pix = (long long)g.N * g.Ho * g.Wo;
-    if (can_vec<T>(g.Cin, x, y) && aligned16(w)) dw_fwd_kernel<T, V><<<flat_blocks(pix * (g.Cin / V), 256), 256, 0, st>>>(x, w, y, g, pix * (g.Cin / V));
-    else dw_fwd_kernel<T, 1><<<flat_blocks(pix * g.Cin, 256), 256, 0, st>>>(x, w, y, g, pix * g.Cin);
+    const int tws = dw_tile_shift(g.Wo);
+    const unsigned tiles = (unsigned)(((g.Wo + (1 << tws) - 1) >> tws) * (((long long)g.N * g.Ho + (64 >> tws) - 1) / (64 >> tws)));
+    if (can_vec<T>(g.Cin, x, y) && aligned16(w)) launch(dw_fwd_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
+    else launch(dw_fwd_kernel<T, 1>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
 }
 
 template <typename T>
 void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const ConvGeom& g, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    const long long pix = (long long)g.N * g.H * g.W;
-    if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) dw_dgrad_kernel<T, V><<<flat_blocks(pix * (g.Cin / V), 256), 256, 0, st>>>(dy, w, addend, dx, g, pix * (g.Cin / V));
-    else dw_dgrad_kernel<T, 1><<<flat_blocks(pix * g.Cin, 256), 256, 0, st>>>(dy, w, addend, dx, g, pix * g.Cin);
+    const int tws = dw_tile_shift(g.W);
+    const unsigned tiles = (unsigned)(((g.W + (1 << tws) - 1) >> tws) * (((long long)g.N * g.H + (64 >> tws) - 1) / (64 >> tws)));
+    if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) launch(dw_dgrad_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
+    else launch(dw_dgrad_kernel<T, 1>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
 }
 
 static FoldPlan plan_dw_wgrad(const ConvGeom& g, int elem_bytes) {
@@ -876,18 +938,18 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
     FoldPlan fp = plan_dw_wgrad(g, (int)sizeof(T));
     const int rpc = fold_rpc(fp);
     if (fp.vec == V && aligned16(x) && aligned16(dy))
-        dw_wgrad_kernel<T, V><<<fold_grid(fp), dim3(32, 8), 0, st>>>(x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
+        launch(dw_wgrad_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
     else
-        dw_wgrad_kernel<T, 1><<<dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st>>>(x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
-    dw_wgrad_finalize_kernel<<<dim3((g.Cin + 31) / 32, fin_slices(fp), 9), dim3(32, FIN_Y), 0, st>>>(scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
+        launch(dw_wgrad_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
+    launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, fin_slices(fp), 9), dim3(FIN_X, FIN_Y), 0, st, scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
 }
 
 template <typename T>
 void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     const long long pix = (long long)N * (H / 2) * (W / 2);
-    if (can_vec<T>(C, x, y)) maxpool_fwd_kernel<T, V><<<flat_blocks(pix * (C / V), 256), 256, 0, st>>>(x, y, H, W, C, pix * (C / V));
-    else maxpool_fwd_kernel<T, 1><<<flat_blocks(pix * C, 256), 256, 0, st>>>(x, y, H, W, C, pix * C);
+    if (can_vec<T>(C, x, y)) launch(maxpool_fwd_kernel<T, V>, dim3(flat_blocks(pix * (C / V), 256)), dim3(256), 0, st, x, y, H, W, C, pix * (C / V));
+    else launch(maxpool_fwd_kernel<T, 1>, dim3(flat_blocks(pix * C, 256)), dim3(256), 0, st, x, y, H, W, C, pix * C);
 }
 
 template <typename T>
@@ -895,47 +957,47 @@ void maxpool_bwd(const T* dy, const T* x, T* dx, int N, int H, int W, int C, cud
     constexpr int V = VecOf<T>::N;
     const long long pix = (long long)N * (H / 2) * (W / 2);
     if ((H & 1) || (W & 1)) cudaMemsetAsync(dx, 0, (size_t)N * H * W * C * sizeof(T), st);   // odd edge gets no gradient
-    if (can_vec<T>(C, dy, x, dx)) maxpool_bwd_kernel<T, V><<<flat_blocks(pix * (C / V), 256), 256, 0, st>>>(dy, x, dx, H, W, C, pix * (C / V));
-    else maxpool_bwd_kernel<T, 1><<<flat_blocks(pix * C, 256), 256, 0, st>>>(dy, x, dx, H, W, C, pix * C);
+    if (can_vec<T>(C, dy, x, dx)) launch(maxpool_bwd_kernel<T, V>, dim3(flat_blocks(pix * (C / V), 256)), dim3(256), 0, st, dy, x, dx, H, W, C, pix * (C / V));
+    else launch(maxpool_bwd_kernel<T, 1>, dim3(flat_blocks(pix * C, 256)), dim3(256), 0, st, dy, x, dx, H, W, C, pix * C);
 }
 
 template <typename T>
 void gap_fwd(const T* x, T* y, int N, int HW, int C, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    if (can_vec<T>(C, x, y)) { const long long t = (long long)N * (C / V); gap_fwd_kernel<T, V><<<(unsigned)((t + 255) / 256), 256, 0, st>>>(x, y, HW, C, t); }
-    else { const long long t = (long long)N * C; gap_fwd_kernel<T, 1><<<(unsigned)((t + 255) / 256), 256, 0, st>>>(x, y, HW, C, t); }
+    if (can_vec<T>(C, x, y)) { const long long t = (long long)N * (C / V); launch(gap_fwd_kernel<T, V>, dim3((unsigned)((t + 255) / 256)), dim3(256), 0, st, x, y, HW, C, t); }
+    else { const long long t = (long long)N * C; launch(gap_fwd_kernel<T, 1>, dim3((unsigned)((t + 255) / 256)), dim3(256), 0, st, x, y, HW, C, t); }
 }
 
 template <typename T>
 void gap_bwd(const T* dy, T* dx, int N, int HW, int C, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    if (can_vec<T>(C, dy, dx)) { const long long t = (long long)N * HW * (C / V); gap_bwd_kernel<T, V><<<flat_blocks(t, 256), 256, 0, st>>>(dy, dx, HW, C, t); }
-    else { const long long t = (long long)N * HW * C; gap_bwd_kernel<T, 1><<<flat_blocks(t, 256), 256, 0, st>>>(dy, dx, HW, C, t); }
+    if (can_vec<T>(C, dy, dx)) { const long long t = (long long)N * HW * (C / V); launch(gap_bwd_kernel<T, V>, dim3(flat_blocks(t, 256)), dim3(256), 0, st, dy, dx, HW, C, t); }
+    else { const long long t = (long long)N * HW * C; launch(gap_bwd_kernel<T, 1>, dim3(flat_blocks(t, 256)), dim3(256), 0, st, dy, dx, HW, C, t); }
 }
 
 void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, float* per_sample, float* dlogits,
                 float* loss, cudaStream_t st) {
-    softmax_ce_kernel<<<N, 128, 0, st>>>(logits, labels, N, classes, per_sample, dlogits);
-    loss_mean_kernel<<<1, 32, 0, st>>>(per_sample, N, loss);
+    launch(softmax_ce_kernel, dim3(N), dim3(128), 0, st, logits, labels, N, classes, per_sample, dlogits);
+    launch(loss_mean_kernel, dim3(1), dim3(32), 0, st, per_sample, N, loss);
 }
 
 void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
                 __nv_bfloat16* shadow, float* snap_dev, float* snap_host, cudaStream_t st) {
     const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(snap_dev) && aligned16(snap_host);
-    if (v) sgd_kernel<4><<<flat_blocks(n / 4, 256), 256, 0, st>>>(w, g, m, n / 4, lr, mu, wd, first, shadow, snap_dev, snap_host);
-    else sgd_kernel<1><<<flat_blocks(n, 256), 256, 0, st>>>(w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
+    if (v) launch(sgd_kernel<4>, dim3(flat_blocks(n / 4, 256)), dim3(256), 0, st, w, g, m, n / 4, lr, mu, wd, first, shadow, snap_dev, snap_host);
+    else launch(sgd_kernel<1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
 }
 
 void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st) {
-    transpose_f32_to_bf16_kernel<<<dim3((N + 31) / 32, (K + 31) / 32, batch), dim3(32, 8), 0, st>>>(w, wt, K, N);
+    launch(transpose_f32_to_bf16_kernel, dim3((N + 31) / 32, (K + 31) / 32, batch), dim3(32, 8), 0, st, w, wt, K, N);
 }
 
 void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st) {
-    bf16_to_f32_kernel<<<flat_blocks(n, 256), 256, 0, st>>>(src, dst, n);
+    launch(bf16_to_f32_kernel, dim3(flat_blocks(n, 256)), dim3(256), 0, st, src, dst, n);
 }
 
 void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st) {
-    f32_to_bf16_kernel<<<flat_blocks(n, 256), 256, 0, st>>>(src, dst, n);
+    launch(f32_to_bf16_kernel, dim3(flat_blocks(n, 256)), dim3(256), 0, st, src, dst, n);
 }
 
 #define FTP_INSTANTIATE(T)                                                                                              \

@@ -11,6 +11,7 @@
 // channel count allows; rows are output pixels (forward), input pixels (data gradient) or
 // reduction steps (weight gradient).
 #include "kernels.h"
+#include "launch.cuh"
 
 namespace ftp {
 namespace {
@@ -92,6 +93,7 @@ __device__ __forceinline__ float apply_act(float v, int act) {
 
 template <int BM, int BN, int MODE, typename T>
 __global__ void __launch_bounds__(NT) conv_gemm_kernel(const GemmP<T> p) {
+    grid_dep_sync();
     constexpr int TM = BM / 16, TN = BN / 16;
     constexpr int ITA = BM / 64;                   // float4 loads of A per thread (vector path)
     static_assert(BM == 128 || BM == 64, "row tile");
@@ -308,6 +310,7 @@ struct WgP {
 
 template <int BI, typename T>
 __global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP<T> p) {
+    grid_dep_sync();
     constexpr int BJ = 64, TM = BI / 16;
     constexpr int LDA = BI + 4, LDB = BJ + 4;
     constexpr int ITA = BK * BI / 4 / NT;          // float4 loads of A per thread (2 or 1)
@@ -440,6 +443,7 @@ __global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP<T> p) {
 
 // out[e] = sum_z partial[z][e], z ascending: the fixed-order second pass of every split reduction
 __global__ void split_reduce_kernel(const float* __restrict__ partial, int S, long long count, float* __restrict__ out) {
+    grid_dep_sync();
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= count) return;
     float s = 0.f;
@@ -450,6 +454,7 @@ __global__ void split_reduce_kernel(const float* __restrict__ partial, int S, lo
 // out[e] = sum_z partial[z][e] (+ bias[column]) (+ addend[e]), z ascending
 __global__ void split_reduce_add_kernel(const float* __restrict__ partial, int S, long long count4, const float* __restrict__ addend,
                                         const float* __restrict__ bias, int Cd, float* __restrict__ out) {
+    grid_dep_sync();
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= count4) return;
     float4 s = __ldg(reinterpret_cast<const float4*>(partial) + e);
@@ -541,13 +546,13 @@ void launch_conv_gemm(GemmP<T> p, float* scratch, cudaStream_t st) {
     const float* const bias = p.bias;
     p.kt_per = gp.kt_per;
     if (gp.S > 1) { p.D = reinterpret_cast<T*>(scratch); p.addend = nullptr; p.bias = nullptr; p.alignD = 1; }
-#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) conv_gemm_kernel<BM_, BN_, MODE, T><<<grid, NT, 0, st>>>(p);
+#define FTP_LAUNCH(BM_, BN_) if (t.bm == BM_ && t.bn == BN_) launch(conv_gemm_kernel<BM_, BN_, MODE, T>, grid, dim3(NT), 0, st, p);
     FTP_LAUNCH(128, 128) FTP_LAUNCH(128, 64) FTP_LAUNCH(64, 128) FTP_LAUNCH(64, 64) FTP_LAUNCH(128, 32) FTP_LAUNCH(64, 32)
 #undef FTP_LAUNCH
     if constexpr (kF32) {
         if (gp.S > 1) {
             const long long count4 = (long long)p.M * p.Cd / 4;
-            split_reduce_add_kernel<<<(unsigned)((count4 + 255) / 256), 256, 0, st>>>(scratch, gp.S, count4, reinterpret_cast<const float*>(addend), bias, p.Cd,
+            launch(split_reduce_add_kernel, dim3((unsigned)((count4 + 255) / 256)), dim3(256), 0, st, scratch, gp.S, count4, reinterpret_cast<const float*>(addend), bias, p.Cd,
                                                                                       reinterpret_cast<float*>(out));
         }
     }
@@ -603,11 +608,11 @@ void conv_wgrad_t(const T* x, const T* dy, float* dw, float* scratch, const Conv
     p.chunk = w.chunk; p.vecA = (g.Cin % 4 == 0) && avec<T>(x); p.vecB = (g.Cout % 4 == 0) && avec<T>(dy);
     p.vecO = (g.Cout % 4 == 0) && a16(p.out) && ((long long)p.Kg * g.Cout) % 4 == 0; p.pointwise = is_pointwise(g);
     const dim3 grid((p.Kg + w.BI - 1) / w.BI, (g.Cout + 63) / 64, w.S);
-    if (w.BI == 128) conv_wgrad_kernel<128, T><<<grid, NT, 0, st>>>(p);
-    else conv_wgrad_kernel<64, T><<<grid, NT, 0, st>>>(p);
+    if (w.BI == 128) launch(conv_wgrad_kernel<128, T>, grid, dim3(NT), 0, st, p);
+    else launch(conv_wgrad_kernel<64, T>, grid, dim3(NT), 0, st, p);
     if (w.S > 1) {
         const long long count = (long long)p.Kg * g.Cout;
-        split_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, w.S, count, dw);
+        launch(split_reduce_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, scratch, w.S, count, dw);
     }
 }
 }  // namespace
@@ -626,7 +631,7 @@ void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const
 }
 
 void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st) {
-    split_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(partial, S, count, out);
+    launch(split_reduce_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, partial, S, count, out);
 }
 
 size_t conv_wgrad_scratch_floats(const ConvGeom& g) {

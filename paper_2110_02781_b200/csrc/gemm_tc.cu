@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base;
+    grid_dep_sync();                 // everything above overlaps the tail of the preceding kernel
 
     if (warp == 0) {
         if (lane == 0) {
@@ -211,6 +212,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base;
+    grid_dep_sync();                 // everything above overlaps the tail of the preceding kernel
 
     if (warp == 0) {
         if (lane == 0) {
@@ -353,7 +355,7 @@ bool launch_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_b
     if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
     const int M = N * H * W;
     TcParams p{D, addend, M, No, 9 * Ca, err, ConvTap{1, H, W, Ca / 64, flip, No}};
-    tc_gemm_tn_kernel<BN><<<dim3((No + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), TC_THREADS, smem, st>>>(ma, mb, p);
+    launch(tc_gemm_tn_kernel<BN>, dim3((No + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, p);
     return true;
 }
 
@@ -369,7 +371,7 @@ bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat
         configured = true;
     }
     TcParams p{D, addend, M, N, K, err, ConvTap{0, 0, 0, 0, 0, 0}};
-    tc_gemm_tn_kernel<BN><<<dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), TC_THREADS, smem, st>>>(ma, mb, p);
+    launch(tc_gemm_tn_kernel<BN>, dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, p);
     return true;
 }
 
@@ -384,7 +386,7 @@ bool launch_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out, l
         configured = true;
     }
     TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{0, 0, 0, 0, 0, 0}};
-    tc_wgrad_kernel<BN><<<dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S), TC_THREADS, smem, st>>>(mx, my, p);
+    launch(tc_wgrad_kernel<BN>, dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S), dim3(TC_THREADS), smem, st, mx, my, p);
     return true;
 }
 
@@ -397,7 +399,7 @@ bool launch_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out
     constexpr int smem = TC_STAGES * (2 + BN / 64) * 64 * 64 * 2 + 1024;
     if (cudaFuncSetAttribute(tc_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
     TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{1, H, W, 0, 0, 0}};
-    tc_wgrad_kernel<BN><<<dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S * 9), TC_THREADS, smem, st>>>(mx, my, p);
+    launch(tc_wgrad_kernel<BN>, dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S * 9), dim3(TC_THREADS), smem, st, mx, my, p);
     return true;
 }
 

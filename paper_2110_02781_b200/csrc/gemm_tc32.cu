@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base;
+    grid_dep_sync();                 // everything above overlaps the tail of the preceding kernel
 
     if (warp == 0) {
         if (lane == 0) {
@@ -271,7 +272,7 @@ bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& m
     constexpr int stage_out = TC_BM * BN * 4;                         // the epilogue reuses the ring as its staging area
     constexpr int smem = (ring > stage_out ? ring : stage_out) + 1024;
     if (cudaFuncSetAttribute(tc32_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    tc32_kernel<BN, STAGES, MODE><<<grid, TC_THREADS, smem, st>>>(ma, mb, md, p);
+    launch(tc32_kernel<BN, STAGES, MODE>, grid, dim3(TC_THREADS), smem, st, ma, mb, md, p);
     return true;
 }
 
@@ -280,7 +281,7 @@ Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
     const long long tiles = ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
     long long S = (3LL * sm_count() + tiles - 1) / tiles;
     const long long maxS = (R + 255) / 256;
-    long long cap = (8LL << 20) / ((long long)Mo * No);
+    long long cap = (2LL << 20) / ((long long)Mo * No);                     // partial sums cost traffic too: at most 2 Mi floats
     if (cap < 1) cap = 1;
     if (S > maxS) S = maxS;
     if (S > cap) S = cap;

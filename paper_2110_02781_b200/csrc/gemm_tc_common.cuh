@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda.h>
 #include "kernels.h"
+#include "launch.cuh"
 
 namespace ftp {
 namespace tc {

@@ -2,6 +2,7 @@
 // stage forward / backward / SGD, re-homing of weights after a new partition, snapshots, the
 // per-unit profile and the kernel trace.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <type_traits>
@@ -253,12 +254,14 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     m.slots.assign(n_slots, nullptr);
     for (auto& p : m.slots) p = bp.take(m.slot_bytes);
     m.red_floats = std::max<size_t>(red, 64); m.red_scratch = (float*)bp.take(m.red_floats * 4);
+    m.red_side = (float*)bp.take(m.red_floats * 4);
     m.fold_doubles = std::max<size_t>(foldd, 64); m.fold_scratch = (double*)bp.take(m.fold_doubles * 8);
     m.dpre_bytes = std::max<size_t>(dpre, 256); m.dpre = bp.take(m.dpre_bytes);
     m.tc_err = (int*)bp.take(256);
     m.fc_in = (float*)bp.take(fcin * 4); m.fc_din = (float*)bp.take(fcin * 4);
     m.fin.part = (double*)bp.take(finp * 8);
     m.fin_counter_bytes = finc * 4; m.fin.counters = (unsigned*)bp.take(m.fin_counter_bytes);
+    m.fin_side.part = (double*)bp.take(finp * 8); m.fin_side.counters = (unsigned*)bp.take(m.fin_counter_bytes);
     m.dlogits = (float*)bp.take((size_t)m.cfg.batch * m.cfg.n_classes * 4);
     m.per_sample = (float*)bp.take((size_t)m.cfg.batch * 4);
     m.loss_dev = (float*)bp.take(256);
@@ -407,6 +410,34 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
         const int s = m->ops[k].gslot;
         return s == -2 ? (void*)m->dlogits : m->slots[s];
     };
+    // Weight gradients feed nothing but the update, so they leave the chain of input gradients: each runs on the second
+    // stream after the kernel that produced its output gradient, and the main stream waits for it only before it
+    // overwrites the buffer that the weight gradient reads (and once at the end).  Per-unit timing and tracing keep
+    // everything on one stream.
+    const bool side_on = m->overlap && !m->unit_events && !m->trace;
+    struct Pending { const void* buf; cudaEvent_t done; };
+    std::vector<Pending> pending;
+    struct Join {                                            // the second stream always rejoins the caller's stream
+        ftp_model* m; cudaStream_t st; bool used;
+        ~Join() { if (used && cudaEventRecord(m->ev_side.back(), m->side) == cudaSuccess) cudaStreamWaitEvent(st, m->ev_side.back(), 0); }
+    } join{m, st, false};
+    auto fork = [&](int i) -> cudaStream_t {                 // stream for the weight gradient of operation i
+        if (!side_on) return st;
+        cudaEventRecord(m->ev_fork[i], st);
+        cudaStreamWaitEvent(m->side, m->ev_fork[i], 0);
+        join.used = true;
+        return m->side;
+    };
+    auto forked = [&](int i, const void* read) {             // after the launches: remember which buffer they read
+        if (!side_on) return;
+        cudaEventRecord(m->ev_side[i], m->side);
+        pending.push_back({read, m->ev_side[i]});
+    };
+    auto before_write = [&](const void* buf) {               // main stream is about to overwrite buf
+        for (size_t k = 0; k < pending.size();)
+            if (pending[k].buf == buf) { cudaStreamWaitEvent(st, pending[k].done, 0); pending.erase(pending.begin() + k); }
+            else ++k;
+    };
     for (int i = last; i >= first; --i) {
         Op& o = m->ops[i];
         const int u = o.d.unit;
@@ -421,6 +452,7 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
         const Arena& ar = m->arena[m->owner[u]];
         float* gr = m->grad;
         const long long Mout = (long long)o.N * o.Ho * o.Wo;
+        if (gi) before_write(gi);
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
@@ -431,18 +463,22 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                     const float* d = (const float*)go;
                     if (o.d.act != FTP_ACT_NONE || o.b_off >= 0) {
                         float* dpre = o.d.act != FTP_ACT_NONE ? (float*)m->dpre : nullptr;
+                        if (dpre) before_write(dpre);
                         Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 4.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
                         act_bias_bwd<float>(d, (const float*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
                                             o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                         if (dpre) d = dpre;
                     }
                     { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
+                      const cudaStream_t ws = fork(i);
+                      float* rs = ws == st ? m->red_scratch : m->red_side;
                       int splits = 0;
                       if (is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr))
-                          splits = tc32_wgrad(x, d, gr + o.w_off, m->red_scratch, Mout, o.C, o.Co, m->tc_err, st);
-                      if (splits > 1) split_reduce_f32(m->red_scratch, splits, o.w_cnt, gr + o.w_off, st);
+                          splits = tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws);
+                      if (splits > 1) split_reduce_f32(rs, splits, o.w_cnt, gr + o.w_off, ws);
                       if (splits > 0 && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
-                      if (splits == 0) conv_wgrad_f32(x, d, gr + o.w_off, m->red_scratch, o.g, st); }
+                      if (splits == 0) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
+                      forked(i, d); }
                     if (gi) {
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the weights as they lie are the K-major B operand
@@ -456,22 +492,26 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                     const T* d = (const T*)go;
                     if (o.d.act != FTP_ACT_NONE || o.b_off >= 0) {
                         T* dpre = o.d.act != FTP_ACT_NONE ? (T*)m->dpre : nullptr;
+                        if (dpre) before_write(dpre);
                         Scope sc(m, st, K_ACT_BIAS_BWD, u, i, 1, o.out_elems * 2.0 * (dpre ? 3.0 : 1.0), (double)o.out_elems, o.b_off >= 0 ? 2 : 1);
                         act_bias_bwd<T>(d, (const T*)m->cur_out[i], dpre, Mout, o.Co, o.d.act, o.fold, m->fold_scratch,
                                         o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                         if (dpre) d = dpre;
                     }
                     { Scope sc(m, st, K_GEMM_BF16_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
+                      const cudaStream_t ws = fork(i);
+                      float* rs = ws == st ? m->red_scratch : m->red_side;
                       int splits = 0;
                       if (is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, d, gr + o.w_off, nullptr))
-                          splits = tc_wgrad((const T*)in, d, gr + o.w_off, m->red_scratch, Mout, o.C, o.Co, m->tc_err, st);
+                          splits = tc_wgrad((const T*)in, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws);
                       if (splits == 0 && is_3x3_op(o) && o.C % 8 == 0 && tc_conv3x3_supported(o.N, o.H, o.W, 64, o.Co, in, d, gr + o.w_off, nullptr))
-                          splits = tc_wgrad3x3((const T*)in, d, gr + o.w_off, m->red_scratch, o.N, o.H, o.W, o.C, o.Co, m->tc_err, st);
-                      if (splits > 1) split_reduce_f32(m->red_scratch, splits, o.w_cnt, gr + o.w_off, st);
+                          splits = tc_wgrad3x3((const T*)in, d, gr + o.w_off, rs, o.N, o.H, o.W, o.C, o.Co, m->tc_err, ws);
+                      if (splits > 1) split_reduce_f32(rs, splits, o.w_cnt, gr + o.w_off, ws);
                       if (splits == 0) {
                           if (sc.slot) sc.slot->rec.kernel = K_CONV_WGRAD_BF16_SIMT;
-                          conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, m->red_scratch, o.g, st);
-                      } }
+                          conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, rs, o.g, ws);
+                      }
+                      forked(i, d); }
                     if (gi) {
                         Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the canonical weight layout already has K = cout contiguous
@@ -487,7 +527,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
             }
             case FTP_DWCONV3x3: {
                 { Scope sc(m, st, K_DW_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems, 2);
-                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, m->red_scratch, o.g, m->fin, st); }
+                  const cudaStream_t ws = fork(i);
+                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, ws == st ? m->red_scratch : m->red_side, o.g, ws == st ? m->fin : m->fin_side, ws);
+                  forked(i, go); }
                 if (gi) {
                     Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
                     dwconv_dgrad<T>((const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, o.g, st);
@@ -607,10 +649,27 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         s = fail(FTP_ENOMEM, "build_model: workspace too small (need %zu device and %zu pinned bytes)", need, pneed);
     if (s != FTP_OK) { delete m; return s; }
     m->pinned = (float*)pinned_ws; m->pinned_bytes = pinned_bytes;
-    if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess || cudaMemset(m->tc_err, 0, 256) != cudaSuccess) {     // ticket counters start at zero
+    if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess || cudaMemset(m->fin_side.counters, 0, m->fin_counter_bytes) != cudaSuccess ||
+        cudaMemset(m->tc_err, 0, 256) != cudaSuccess) {     // ticket counters start at zero
         const ftp_status e = fail(FTP_ECUDA, "build_model: clearing the ticket counters failed: %s", cudaGetErrorString(cudaGetLastError()));
         delete m;
         return e;
+    }
+    {   // second stream and its fork / join events: one pair per operation, created here so that nothing is created inside a stream capture
+        const char* e = std::getenv("FTP_OVERLAP");
+        m->overlap = !(e && std::strcmp(e, "0") == 0);
+        bool ok = cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking) == cudaSuccess;
+        for (size_t i = 0; ok && i <= m->ops.size(); ++i) {
+            cudaEvent_t a = nullptr, b = nullptr;
+            ok = cudaEventCreateWithFlags(&a, cudaEventDisableTiming) == cudaSuccess && cudaEventCreateWithFlags(&b, cudaEventDisableTiming) == cudaSuccess;
+            if (a) m->ev_fork.push_back(a);
+            if (b) m->ev_side.push_back(b);
+        }
+        if (!ok) {
+            const ftp_status er = fail(FTP_ECUDA, "build_model: creating the second stream failed: %s", cudaGetErrorString(cudaGetLastError()));
+            ftp_destroy_model(m);
+            return er;
+        }
     }
     m->owner.assign(m->L, 0);
     m->points = {0, m->L};
@@ -629,6 +688,9 @@ extern "C" void ftp_destroy_model(ftp_model* m) {
     for (auto& t : m->tr) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
     for (auto e : m->ev_f) cudaEventDestroy(e);
     for (auto e : m->ev_b) cudaEventDestroy(e);
+    for (auto e : m->ev_fork) cudaEventDestroy(e);
+    for (auto e : m->ev_side) cudaEventDestroy(e);
+    if (m->side) cudaStreamDestroy(m->side);
     delete m;
 }
 

@@ -66,6 +66,9 @@ struct ftp_model {
     float* red_scratch; size_t red_floats;
     double* fold_scratch; size_t fold_doubles;
     ftp::FinScratch fin; size_t fin_counter_bytes;
+    // weight gradients run on a second stream beside the chain of input gradients; they have scratch of their own
+    float* red_side; ftp::FinScratch fin_side;
+    cudaStream_t side; std::vector<cudaEvent_t> ev_fork, ev_side; bool overlap;
     void* dpre; size_t dpre_bytes;
     int* tc_err;                                  // device word set by a tensor-core kernel whose bounded wait ran out
     float* fc_in; float* fc_din;                  // bf16 models: the classifier's input and input gradient widened to float
