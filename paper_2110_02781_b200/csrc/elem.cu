@@ -506,6 +506,69 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
     }
 }
 
+// Stride-1 depthwise 3x3 (padding 1), forward (FLIP = 0) or data gradient (FLIP = 1: the same sum with the
+// taps mirrored): a thread computes four neighbouring outputs of one row for one channel vector from the
+// 3 x 6 inputs they share, so every input vector is loaded once per row of taps instead of three times and
+// the six loads of a row are in flight together.  Block: 8 channel vectors x 32 strips; strips are numbered
+// row-major over (image, row, strip of 4 columns).
+template <typename T, int V, int FLIP>
+__global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, const float* __restrict__ w, const T* __restrict__ addend,
+                                                       T* __restrict__ y, int N, int H, int W, int C) {
+    grid_dep_sync();
+    const int CV = C / V;
+    const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
+    if (cv >= CV) return;
+    const int c = cv * V;
+    const int strips_w = (W + 3) >> 2;
+    const long long strip = (long long)blockIdx.x * 32 + (threadIdx.x >> 3);
+    if (strip >= (long long)N * H * strips_w) return;
+    const int w0 = (int)(strip % strips_w) * 4;
+    const long long R = strip / strips_w;                 // image * H + row
+    const int h = (int)(R % H);
+    float acc[4][V];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[j][e] = 0.f;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int hi = h - 1 + r;
+        if (hi < 0 || hi >= H) continue;
+        const T* row = x + ((R - h + hi) * W) * (long long)C + c;
+        float in[6][V];
+#pragma unroll
+        for (int j = 0; j < 6; ++j) {
+            const int wi = w0 - 1 + j;
+            if (wi >= 0 && wi < W) ldv<V>(row + (long long)wi * C, in[j]);
+            else {
+#pragma unroll
+                for (int e = 0; e < V; ++e) in[j][e] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            float k[V];
+            ldtab<V>(w + ((FLIP ? 2 - r : r) * 3 + (FLIP ? 2 - s : s)) * C + c, k);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[j][e] = fmaf(in[j + s][e], k[e], acc[j][e]);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (w0 + j >= W) break;
+        const long long o = ((R * W) + w0 + j) * (long long)C + c;
+        if (addend) {
+            float a[V];
+            ldv<V>(addend + o, a);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[j][e] += a[e];
+        }
+        stv<V>(y + o, acc[j]);
+    }
+}
+
 // Depthwise weight gradient on the folded view: grid (column tiles of 32*V, pixel-row chunks), block (32, 8).
 // A thread owns V folded columns (a fixed channel vector and a fixed pixel offset within each folded row)
 // and walks the rows of its chunk; the 9 taps are reduced over y three at a time through shared memory.
@@ -723,7 +786,7 @@ __global__ void loss_mean_kernel(const float* __restrict__ per_sample, int N, fl
 // ---- SGD ------------------------------------------------------------------------------------------------
 template <int V>
 __global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, long long nvec, float lr,
-                                                  float mu, float wd, int first, __nv_bfloat16* __restrict__ shadow,
+                                                  float mu, float wd, int first, __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo,
                                                   float* __restrict__ snap_dev, float* __restrict__ snap_host) {
     grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
@@ -743,6 +806,12 @@ __global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const f
 #pragma unroll
         for (int e = 0; e < V; ++e) wv[e] = fmaf(-lr, gv[e], wv[e]);
         stv<V>(w + i * V, wv);
+        if (lo) {
+            float lv[V];
+#pragma unroll
+            for (int e = 0; e < V; ++e) lv[e] = wv[e] - __uint_as_float(__float_as_uint(wv[e]) & 0xffffe000u);
+            stv<V>(lo + i * V, lv);
+        }
         if (snap_dev) stv<V>(snap_dev + i * V, wv);
         if (snap_host) stv<V>(snap_host + i * V, wv);
         if (shadow) {
@@ -779,6 +848,41 @@ __global__ void transpose_f32_to_bf16_kernel(const float* __restrict__ w, __nv_b
     for (int r = threadIdx.y; r < 32; r += 8) {
         const int n = n0 + r, k = k0 + threadIdx.x;
         if (n < N && k < K) wt[(long long)n * K + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+    }
+}
+
+__global__ void tf32_lo_kernel(const float* __restrict__ w, float* __restrict__ lo, long long n) {
+    grid_dep_sync();
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float v = w[i];
+        lo[i] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+    }
+}
+
+// One block per 32 x 32 tile of one of the matrices of the table: wt[n][k] = w[k][n], wtl[n][k] = its lo part.
+__global__ void transpose_split_f32_kernel(const TransposeEntryDev* __restrict__ table, int n, int tile_base, const float* __restrict__ w,
+                                           float* __restrict__ wt, float* __restrict__ wtl) {
+    grid_dep_sync();
+    __shared__ float tile[32][33];
+    const int t = tile_base + blockIdx.x;
+    int e = 0;
+    while (e + 1 < n && table[e + 1].tile0 <= t) ++e;
+    const TransposeEntryDev en = table[e];
+    const int local = t - en.tile0, tn = (en.N + 31) / 32;
+    const int k0 = (local / tn) * 32, n0 = (local % tn) * 32;
+    const float* src = w + en.w_off;
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const int k = k0 + r, c = n0 + threadIdx.x;
+        tile[r][threadIdx.x] = (k < en.K && c < en.N) ? src[(long long)k * en.N + c] : 0.f;
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const int c = n0 + r, k = k0 + threadIdx.x;
+        if (c < en.N && k < en.K) {
+            const float v = tile[threadIdx.x][r];
+            wt[en.w_off + (long long)c * en.K + k] = v;
+            wtl[en.w_off + (long long)c * en.K + k] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+        }
     }
 }
 
@@ -909,6 +1013,11 @@ void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_
     constexpr int V = VecOf<T>::N;
     const int tws = dw_tile_shift(g.Wo);
     const unsigned tiles = (unsigned)(((g.Wo + (1 << tws) - 1) >> tws) * (((long long)g.N * g.Ho + (64 >> tws) - 1) / (64 >> tws)));
+    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w)) {
+        const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
+        launch(dw_strip_kernel<T, V, 0>, dim3((unsigned)((strips + 31) / 32), (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin);
+        return;
+    }
     if (can_vec<T>(g.Cin, x, y) && aligned16(w)) launch(dw_fwd_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
     else launch(dw_fwd_kernel<T, 1>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
 }
@@ -918,6 +1027,11 @@ void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const Con
     constexpr int V = VecOf<T>::N;
     const int tws = dw_tile_shift(g.W);
     const unsigned tiles = (unsigned)(((g.W + (1 << tws) - 1) >> tws) * (((long long)g.N * g.H + (64 >> tws) - 1) / (64 >> tws)));
+    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
+        const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
+        launch(dw_strip_kernel<T, V, 1>, dim3((unsigned)((strips + 31) / 32), (g.Cin / V + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin);
+        return;
+    }
     if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) launch(dw_dgrad_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
     else launch(dw_dgrad_kernel<T, 1>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
 }
@@ -982,10 +1096,18 @@ void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, 
 }
 
 void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
-                __nv_bfloat16* shadow, float* snap_dev, float* snap_host, cudaStream_t st) {
-    const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(snap_dev) && aligned16(snap_host);
-    if (v) launch(sgd_kernel<4>, dim3(flat_blocks(n / 4, 256)), dim3(256), 0, st, w, g, m, n / 4, lr, mu, wd, first, shadow, snap_dev, snap_host);
-    else launch(sgd_kernel<1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, g, m, n, lr, mu, wd, first, shadow, snap_dev, snap_host);
+                __nv_bfloat16* shadow, float* lo, float* snap_dev, float* snap_host, cudaStream_t st) {
+    const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(lo) && aligned16(snap_dev) && aligned16(snap_host);
+    if (v) launch(sgd_kernel<4>, dim3(flat_blocks(n / 4, 256)), dim3(256), 0, st, w, g, m, n / 4, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
+    else launch(sgd_kernel<1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, g, m, n, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
+}
+
+void tf32_lo(const float* w, float* lo, long long n, cudaStream_t st) {
+    launch(tf32_lo_kernel, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, lo, n);
+}
+
+void transpose_split_f32(const TransposeEntryDev* table, int n, int tile_base, int tiles, const float* w, float* wt, float* wtl, cudaStream_t st) {
+    if (tiles > 0) launch(transpose_split_f32_kernel, dim3(tiles), dim3(32, 8), 0, st, table, n, tile_base, w, wt, wtl);
 }
 
 void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st) {

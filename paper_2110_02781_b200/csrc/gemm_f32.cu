@@ -441,14 +441,27 @@ __global__ void __launch_bounds__(NT) conv_wgrad_kernel(const WgP<T> p) {
     }
 }
 
-// out[e] = sum_z partial[z][e], z ascending: the fixed-order second pass of every split reduction
-__global__ void split_reduce_kernel(const float* __restrict__ partial, int S, long long count, float* __restrict__ out) {
+// out[e] = sum_z partial[z][e]: the fixed-order second pass of every split reduction.  Block (32, 8): eight
+// interleaved runs over z per element (two loads in flight each), combined in run order through shared memory.
+__global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restrict__ partial, int S, long long count, float* __restrict__ out) {
     grid_dep_sync();
-    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= count) return;
-    float s = 0.f;
-    for (int z = 0; z < S; ++z) s += partial[(long long)z * count + e];
-    out[e] = s;
+    __shared__ float sh[8][33];
+    const long long e = (long long)blockIdx.x * 32 + threadIdx.x;
+    float s0 = 0.f, s1 = 0.f;
+    if (e < count)
+        for (int z = threadIdx.y; z < S; z += 16) {
+            const float a = partial[(long long)z * count + e];
+            const float b = z + 8 < S ? partial[(long long)(z + 8) * count + e] : 0.f;
+            s0 += a; s1 += b;
+        }
+    sh[threadIdx.y][threadIdx.x] = s0 + s1;
+    __syncthreads();
+    if (threadIdx.y == 0 && e < count) {
+        float s = 0.f;
+#pragma unroll
+        for (int y = 0; y < 8; ++y) s += sh[y][threadIdx.x];
+        out[e] = s;
+    }
 }
 
 // out[e] = sum_z partial[z][e] (+ bias[column]) (+ addend[e]), z ascending
@@ -612,7 +625,7 @@ void conv_wgrad_t(const T* x, const T* dy, float* dw, float* scratch, const Conv
     else launch(conv_wgrad_kernel<64, T>, grid, dim3(NT), 0, st, p);
     if (w.S > 1) {
         const long long count = (long long)p.Kg * g.Cout;
-        launch(split_reduce_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, scratch, w.S, count, dw);
+        launch(split_reduce_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, scratch, w.S, count, dw);
     }
 }
 }  // namespace
@@ -631,7 +644,7 @@ void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const
 }
 
 void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st) {
-    launch(split_reduce_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, partial, S, count, out);
+    launch(split_reduce_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, partial, S, count, out);
 }
 
 size_t conv_wgrad_scratch_floats(const ConvGeom& g) {

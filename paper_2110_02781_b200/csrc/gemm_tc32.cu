@@ -52,26 +52,27 @@ __device__ __forceinline__ void transpose_split(const uint8_t* src, uint8_t* hi,
     }
 }
 
-// hi stays where TMA put it (low mantissa bits cleared), lo goes to the buffer `lo_off` bytes further.
-// Elementwise, so the swizzled placement does not matter.  `threads` cooperating threads, `t` this thread's rank.
-__device__ __forceinline__ void split_tile(uint8_t* hi, uint32_t lo_off, int bytes, int t, int threads) {
+// The tensor core reads only the upper 19 bits of a tf32 operand, so the tile as TMA delivered it already is the
+// "hi" part; the "lo" part x - trunc(x) goes to the buffer `lo_off` bytes further.  Elementwise, so the swizzled
+// placement does not matter.  `threads` cooperating threads, `t` this thread's rank.
+__device__ __forceinline__ void split_tile(const uint8_t* hi, uint8_t* lo, int bytes, int t, int threads) {
     for (int i = t * 16; i < bytes; i += threads * 16) {
-        float4 v = *reinterpret_cast<float4*>(hi + i);
-        float4 h, l;
-        h.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u); l.x = v.x - h.x;
-        h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u); l.y = v.y - h.y;
-        h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u); l.z = v.z - h.z;
-        h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u); l.w = v.w - h.w;
-        *reinterpret_cast<float4*>(hi + i) = h;
-        *reinterpret_cast<float4*>(hi + lo_off + i) = l;
+        const float4 v = *reinterpret_cast<const float4*>(hi + i);
+        float4 l;
+        l.x = v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+        l.y = v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+        l.z = v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+        l.w = v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+        *reinterpret_cast<float4*>(lo + i) = l;
     }
 }
 
 struct T32Params {
-    float* D;              // gemm: output [M][N]; wgrad: partials [S][Mo][No]
-    const float* addend;   // gemm only, nullable
+    float* D;              // output [S][M][N]: the result itself when S == 1, else partial sums over slices of the reduction
+    const float* addend;   // gemm with S == 1 only, nullable
     int M, N, K;           // gemm: D[M,N] = A[M,K] B[N,K]^T.  wgrad: Mo = M, No = N, K = reduction rows R
-    int rows_per_split;    // wgrad
+    int rows_per_split;    // reduction elements per slice (a multiple of 32)
+    int b_lo_given;        // MODE 0: the lo part of B comes from memory (mapBlo) instead of being computed per tile
     int* err;
 };
 
@@ -79,7 +80,8 @@ struct T32Params {
 // in shared memory (weight gradient).  MODE 2: A [M][K] as it lies, B [K][N] (the weights) transposed (forward).
 template <int BN, int STAGES, int MODE>
 __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                                                          const __grid_constant__ CUtensorMap mapD, const T32Params p) {
+                                                          const __grid_constant__ CUtensorMap mapBlo, const __grid_constant__ CUtensorMap mapD,
+                                                          const T32Params p) {
     constexpr uint32_t A_BYTES = TC_BM * T32_BK * 4, B_BYTES = BN * T32_BK * 4;          // one precision part
     constexpr bool TA = MODE == 1, TB = MODE != 0;                                      // operand transposed in shared memory
     constexpr uint32_t STAGE_BYTES = 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) + (TB ? B_BYTES : 0);   // [A hi][A lo][B hi][B lo][A src][B src]
@@ -96,14 +98,16 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
         m0 = blockIdx.x * TC_BM; n0 = blockIdx.y * BN; split = blockIdx.z;
         kbeg = split * p.rows_per_split; kend = min(p.K, kbeg + p.rows_per_split);
     } else {
-        n0 = blockIdx.x * BN; m0 = blockIdx.y * TC_BM; kbeg = 0; kend = p.K;
+        n0 = blockIdx.x * BN; m0 = blockIdx.y * TC_BM; split = blockIdx.z;
+        kbeg = split * p.rows_per_split; kend = min(p.K, kbeg + p.rows_per_split);
     }
     const int num_kb = (kend - kbeg + T32_BK - 1) / T32_BK;
     // transposed operands arrive as 32-column slabs: slabs wholly beyond the matrix are neither loaded nor converted
     // (their rows of the hi / lo tiles are cleared once)
     const int slabsA = TA ? min(TC_BM / 32, (p.M - m0 + 31) / 32) : TC_BM / 32;
     const int slabsB = TB ? min(BN / 32, (p.N - n0 + 31) / 32) : BN / 32;
-    const uint32_t tx_bytes = (TA ? slabsA * SLAB : A_BYTES) + (TB ? slabsB * SLAB : B_BYTES);
+    const bool b_pre = MODE == 0 && p.b_lo_given;
+    const uint32_t tx_bytes = (TA ? slabsA * SLAB : A_BYTES) + (TB ? slabsB * SLAB : B_BYTES) + (b_pre ? B_BYTES : 0);
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), ready0 = smem_u32(&bars[2 * STAGES]), accum = smem_u32(&bars[3 * STAGES]);
 
     if (threadIdx.x == 0) {
@@ -139,6 +143,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
                 if (TB) {
                     for (int t = 0; t < slabsB; ++t) tma_load_2d(sb + t * SLAB, &mapB, n0 + 32 * t, k, full0 + 8 * s);
                 } else tma_load_2d(sb, &mapB, k, n0, full0 + 8 * s);
+                if (b_pre) tma_load_2d(sb + B_BYTES, &mapBlo, k, n0, full0 + 8 * s);
                 issued = kb + 1;
             }
             if (*((volatile int*)p.err) != 0) {
@@ -193,9 +198,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
             uint8_t* st = smem + s * STAGE_BYTES;
             uint8_t* src = st + 2 * (A_BYTES + B_BYTES);
             if (TA) transpose_split(src, st, st + A_BYTES, slabsA, t, 128);
-            else split_tile(st, A_BYTES, A_BYTES, t, 128);
+            else split_tile(st, st + A_BYTES, A_BYTES, t, 128);
             if (TB) transpose_split(src + (TA ? A_BYTES : 0), st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, t, 128);
-            else split_tile(st + 2 * A_BYTES, B_BYTES, B_BYTES, t, 128);
+            else if (!b_pre) split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t, 128);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
             mbar_arrive(ready0 + 8 * s);
         }
@@ -267,12 +272,12 @@ bool make_map_out(CUtensorMap* map, const void* base, long long S, long long row
 }
 
 template <int BN, int STAGES, int MODE>
-bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
+bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
     constexpr int ring = STAGES * (2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0));
     constexpr int stage_out = TC_BM * BN * 4;                         // the epilogue reuses the ring as its staging area
     constexpr int smem = (ring > stage_out ? ring : stage_out) + 1024;
     if (cudaFuncSetAttribute(tc32_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    launch(tc32_kernel<BN, STAGES, MODE>, grid, dim3(TC_THREADS), smem, st, ma, mb, md, p);
+    launch(tc32_kernel<BN, STAGES, MODE>, grid, dim3(TC_THREADS), smem, st, ma, mb, ml, md, p);
     return true;
 }
 
@@ -300,38 +305,107 @@ bool tc32_supported(int M, int N, int K, const void* A, const void* B, const voi
     return M >= 1 && N % 4 == 0 && K % 4 == 0 && N >= 4 && K >= 4 && a16(A) && a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
 }
 
+constexpr int stage_bytes32(int BN, int MODE) {
+    return 2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0);
+}
+constexpr int max_stages32(int BN, int MODE) {
+    const int n = (226 * 1024) / stage_bytes32(BN, MODE);
+    return n > 4 ? 4 : n;
+}
+
 template <int BN, int MODE>
-bool launch32_stages(int num_kb, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
+bool launch32_stages(int num_kb, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& md, const T32Params& p, dim3 grid,
+                     cudaStream_t st) {
     // Many tiles (memory-bound layers): one stage per CTA, so that several CTAs share an SM and hide each other's
-    // latencies.  Few tiles (late layers, long reductions): a deeper ring inside the CTA instead.
-    constexpr int MAXS = BN == 128 ? 2 : 3;
+    // latencies.  Few tiles (late layers, long reductions): as deep a ring as shared memory holds instead.
+    constexpr int MAXS = max_stages32(BN, MODE);
     const long long tiles = (long long)grid.x * grid.y * grid.z;
     int stages = tiles >= 4LL * sm_count() ? 1 : (tiles >= 2LL * sm_count() ? 2 : MAXS);
     if (stages > num_kb) stages = num_kb < 1 ? 1 : num_kb;
     if (stages > MAXS) stages = MAXS;
-    if (stages == 1) return launch32<BN, 1, MODE>(ma, mb, md, p, grid, st);
-    if (stages == 2) return launch32<BN, 2, MODE>(ma, mb, md, p, grid, st);
-    return launch32<BN, 3, MODE>(ma, mb, md, p, grid, st);
+    if (stages == 1) return launch32<BN, 1, MODE>(ma, mb, ml, md, p, grid, st);
+    if (stages == 2) return launch32<BN, 2, MODE>(ma, mb, ml, md, p, grid, st);
+    if constexpr (MAXS >= 3) { if (stages == 3) return launch32<BN, 3, MODE>(ma, mb, ml, md, p, grid, st); }
+    if constexpr (MAXS >= 4) { if (stages == 4) return launch32<BN, 4, MODE>(ma, mb, ml, md, p, grid, st); }
+    return false;
+}
+
+// out = addend + sum over S slices, slice order fixed
+__global__ void __launch_bounds__(256) slice_sum_kernel(const float4* __restrict__ part, int S, long long count4, const float4* __restrict__ addend,
+                                                        float4* __restrict__ out) {
+    grid_dep_sync();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count4) return;
+    float4 a = part[i];
+    for (int s = 1; s < S; ++s) { const float4 v = part[(long long)s * count4 + i]; a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+    if (addend) { const float4 v = addend[i]; a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+    out[i] = a;
+}
+
+// Tile width and reduction slices of a product D[M,N] over K.  With fewer tiles than SMs the tiles get narrower and
+// the reduction is cut into slices (each at least four 32-wide blocks), so that the late, small layers still
+// spread over the machine; the slices are summed in order by a second kernel.
+struct G32Plan { int BN, S, rps; };
+G32Plan plan_gemm32(int M, int N, int K) {
+    const int sms = sm_count(), mt = (M + TC_BM - 1) / TC_BM;
+    int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
+    while (BN > 32 && (long long)mt * ((N + BN - 1) / BN) < sms) BN >>= 1;
+    const long long tiles = (long long)mt * ((N + BN - 1) / BN);
+    const int nkb = (K + T32_BK - 1) / T32_BK;
+    long long S = 1;
+    if (tiles < sms && nkb >= 8) {
+        S = (2LL * sms + tiles - 1) / tiles;
+        if (S > nkb / 4) S = nkb / 4;
+        if (S > 8) S = 8;
+        const long long cap = (4LL << 20) / ((long long)M * N);
+        if (S > cap) S = cap;
+        if (S < 1) S = 1;
+    }
+    G32Plan g;
+    g.BN = BN;
+    g.rps = (int)((nkb + S - 1) / S) * T32_BK;
+    g.S = (K + g.rps - 1) / g.rps;
+    return g;
 }
 
 // D[M,N] = A[M,K] * B (+ addend), float in and out, split-tf32 arithmetic.
 // b_is_kn == 0: B is [N][K] (K contiguous); b_is_kn == 1: B is [K][N] (N contiguous, as convolution weights lie).
-bool tc32_gemm(const float* A, const float* B, int b_is_kn, const float* addend, float* D, int M, int N, int K, int* err, cudaStream_t st) {
-    const int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
-    CUtensorMap ma, mb, md;
-    if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, D, 1, M, N)) return false;
+bool tc32_gemm(const float* A, const float* B, const float* B_lo, int b_is_kn, const float* addend, float* D, float* scratch, int M, int N, int K, int* err,
+               cudaStream_t st) {
+    G32Plan g = plan_gemm32(M, N, K);
+    if (g.S > 1 && !scratch) { g.S = 1; g.rps = (K + T32_BK - 1) / T32_BK * T32_BK; }
+    const int BN = g.BN;
+    float* out = g.S > 1 ? scratch : D;
+    CUtensorMap ma, mb, ml, md;
+    if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, out, g.S, M, N)) return false;
     if (!(b_is_kn ? make_map_f32(&mb, B, K, N, 32) : make_map_f32(&mb, B, N, K, BN))) return false;
-    T32Params p{D, addend, M, N, K, 0, err};
-    const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM);
-    const int nkb = (K + T32_BK - 1) / T32_BK;
+    const bool pre = !b_is_kn && B_lo != nullptr;
+    if (pre) { if (!make_map_f32(&ml, B_lo, N, K, BN)) return false; }
+    else ml = mb;
+    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, pre ? 1 : 0, err};
+    const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM, g.S);
+    const int nkb = g.rps / T32_BK;
+    bool ok;
     if (b_is_kn) {
-        if (BN == 128) return launch32_stages<128, 2>(nkb, ma, mb, md, p, grid, st);
-        if (BN == 64) return launch32_stages<64, 2>(nkb, ma, mb, md, p, grid, st);
-        return launch32_stages<32, 2>(nkb, ma, mb, md, p, grid, st);
+        if (BN == 128) ok = launch32_stages<128, 2>(nkb, ma, mb, ml, md, p, grid, st);
+        else if (BN == 64) ok = launch32_stages<64, 2>(nkb, ma, mb, ml, md, p, grid, st);
+        else ok = launch32_stages<32, 2>(nkb, ma, mb, ml, md, p, grid, st);
+    } else {
+        if (BN == 128) ok = launch32_stages<128, 0>(nkb, ma, mb, ml, md, p, grid, st);
+        else if (BN == 64) ok = launch32_stages<64, 0>(nkb, ma, mb, ml, md, p, grid, st);
+        else ok = launch32_stages<32, 0>(nkb, ma, mb, ml, md, p, grid, st);
     }
-    if (BN == 128) return launch32_stages<128, 0>(nkb, ma, mb, md, p, grid, st);
-    if (BN == 64) return launch32_stages<64, 0>(nkb, ma, mb, md, p, grid, st);
-    return launch32_stages<32, 0>(nkb, ma, mb, md, p, grid, st);
+    if (ok && g.S > 1) {
+        const long long count4 = (long long)M * N / 4;
+        launch(slice_sum_kernel, dim3((unsigned)((count4 + 255) / 256)), dim3(256), 0, st, reinterpret_cast<const float4*>(scratch), g.S, count4,
+               reinterpret_cast<const float4*>(addend), reinterpret_cast<float4*>(D));
+    }
+    return ok;
+}
+
+size_t tc32_gemm_scratch_floats(int M, int N, int K) {
+    const G32Plan g = plan_gemm32(M, N, K);
+    return g.S > 1 ? (size_t)g.S * M * N : 0;
 }
 
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No) {
@@ -346,13 +420,13 @@ int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long 
     CUtensorMap mx, my, md;
     float* out = w.S > 1 ? scratch : dW;
     if (!make_map_f32(&mx, X, R, Mo, 32) || !make_map_f32(&my, dY, R, No, 32) || !make_map_out(&md, out, w.S, Mo, No)) return 0;
-    T32Params p{out, nullptr, Mo, No, (int)R, w.rows_per_split, err};
+    T32Params p{out, nullptr, Mo, No, (int)R, w.rows_per_split, 0, err};
     const dim3 grid((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S);
     const int nkb = (w.rows_per_split + T32_BK - 1) / T32_BK;
     bool ok;
-    if (BN == 128) ok = launch32_stages<128, 1>(nkb, mx, my, md, p, grid, st);
-    else if (BN == 64) ok = launch32_stages<64, 1>(nkb, mx, my, md, p, grid, st);
-    else ok = launch32_stages<32, 1>(nkb, mx, my, md, p, grid, st);
+    if (BN == 128) ok = launch32_stages<128, 1>(nkb, mx, my, my, md, p, grid, st);
+    else if (BN == 64) ok = launch32_stages<64, 1>(nkb, mx, my, my, md, p, grid, st);
+    else ok = launch32_stages<32, 1>(nkb, mx, my, my, md, p, grid, st);
     return ok ? w.S : 0;
 }
 

@@ -56,7 +56,11 @@ void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int 
 
 // ---- float contractions on tensor cores with split-tf32 arithmetic (gemm_tc32.cu); same conventions as above ----
 bool tc32_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
-bool tc32_gemm(const float* A, const float* B, int b_is_kn, const float* addend, float* D, int M, int N, int K, int* err, cudaStream_t st);
+// scratch (nullable): tc32_gemm_scratch_floats(M, N, K) floats; lets products with few tiles cut the reduction into slices
+size_t tc32_gemm_scratch_floats(int M, int N, int K);
+// B_lo (nullable, only with b_is_kn == 0): B - trunc_tf32(B) laid out like B, saves computing it per tile
+bool tc32_gemm(const float* A, const float* B, const float* B_lo, int b_is_kn, const float* addend, float* D, float* scratch, int M, int N, int K,
+               int* err, cudaStream_t st);
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
 int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
 
@@ -139,8 +143,15 @@ void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, 
                 float* dlogits, float* loss, cudaStream_t st);
 
 // Fused SGD: g += wd*w; m = first ? g : mu*m + g; w -= lr*m; optional bf16 shadow and snapshot stores.
+// lo (nullable): receives w - trunc_tf32(w) of the updated weights.
 void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
-                __nv_bfloat16* shadow, float* snap_dev, float* snap_host, cudaStream_t st);
+                __nv_bfloat16* shadow, float* lo, float* snap_dev, float* snap_host, cudaStream_t st);
+void tf32_lo(const float* w, float* lo, long long n, cudaStream_t st);                   // lo = w - trunc_tf32(w)
+// Batched transposition of float matrices: entry e describes a [K][N] matrix at w + w_off whose transpose goes to
+// wt + w_off ([N][K]) and the lo part of the transpose to wtl + w_off.  table: n + 1 device entries (the last one
+// closes the tile range); tiles = table[n].tile0 - table[0].tile0 blocks are launched.
+struct TransposeEntryDev { long long w_off; int K, N, tile0, pad; };
+void transpose_split_f32(const TransposeEntryDev* table, int n, int tile_base, int tiles, const float* w, float* wt, float* wtl, cudaStream_t st);
 void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st);
 void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st);
 

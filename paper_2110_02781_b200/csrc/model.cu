@@ -203,6 +203,8 @@ ftp_status plan_gradients(ftp_model& m, int* n_slots) {
     return FTP_OK;
 }
 
+bool is_pointwise_op(const Op& o);
+
 // ---- memory layout inside the workspace --------------------------------------------------------------
 ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinned_total) {
     Bump bp{dev_base, 0};
@@ -215,6 +217,25 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         a.run = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
         a.wb = m.cfg.precision == FTP_BF16 ? (__nv_bfloat16*)bp.take((size_t)m.P * 2) : nullptr;
         a.wbt = m.cfg.precision == FTP_BF16 ? (__nv_bfloat16*)bp.take((size_t)m.P * 2) : nullptr;
+        const bool f32 = m.cfg.precision == FTP_FP32;
+        a.wl = f32 ? (float*)bp.take((size_t)m.P * 4) : nullptr;
+        a.wt = f32 ? (float*)bp.take((size_t)m.P * 4) : nullptr;
+        a.wtl = f32 ? (float*)bp.take((size_t)m.P * 4) : nullptr;
+    }
+    {   // table of the 1x1-convolution matrices for the batched transposition
+        m.tp_host.clear(); m.tp_first.assign(m.L + 1, 0);
+        int tile0 = 0, u_next = 0;
+        for (int i = 0; i < n; ++i) {
+            const Op& o = m.ops[i];
+            while (u_next <= o.d.unit) m.tp_first[u_next++] = (int)m.tp_host.size();
+            if (m.cfg.precision == FTP_FP32 && is_pointwise_op(o) && o.d.kind != FTP_FC) {
+                m.tp_host.push_back(TransposeEntryDev{o.w_off, o.C, o.Co, tile0, 0});
+                tile0 += ((o.C + 31) / 32) * ((o.Co + 31) / 32);
+            }
+        }
+        while (u_next <= m.L) m.tp_first[u_next++] = (int)m.tp_host.size();
+        m.tp_host.push_back(TransposeEntryDev{0, 0, 0, tile0, 0});
+        m.tp_dev = (TransposeEntryDev*)bp.take(m.tp_host.size() * sizeof(TransposeEntryDev));
     }
     m.grad = (float*)bp.take((size_t)m.P * 4);
     m.state_backup = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
@@ -237,6 +258,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
             red = std::max(red, std::max(conv_wgrad_scratch_floats(o.g), conv_gemm_scratch_floats(o.g)));
             red = std::max(red, tc32_wgrad_scratch_floats(Mout, o.C, o.Co));
+            red = std::max(red, std::max(tc32_gemm_scratch_floats((int)Mout, o.Co, o.C), tc32_gemm_scratch_floats((int)Mout, o.C, o.Co)));
             if (m.cfg.precision == FTP_BF16) red = std::max(red, std::max(tc_wgrad_scratch_floats(Mout, o.C, o.Co), tc_wgrad3x3_scratch_floats(Mout, o.C, o.Co)));
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
@@ -286,8 +308,22 @@ bool is_3x3_op(const Op& o) {
     return o.d.kind == FTP_CONV2D && o.g.kh == 3 && o.g.kw == 3 && o.g.stride == 1 && o.g.ph == 1 && o.g.pw == 1 && o.d.act == FTP_ACT_NONE && o.b_off < 0;
 }
 
-// bf16 models: rebuild the transposed bf16 copy of every 1x1 convolution of units [a, b) from the float masters
+// Rebuild the transposed copies of the 1x1-convolution matrices of units [a, b) from the float masters: bf16 models
+// one matrix at a time, float models in one batched launch per owning arena.
 void refresh_transposed(ftp_model* m, int a, int b, cudaStream_t st) {
+    if (m->cfg.precision == FTP_FP32) {
+        for (int u = a; u < b;) {
+            int v = u + 1;
+            while (v < b && m->owner[v] == m->owner[u]) ++v;
+            const Arena& ar = m->arena[m->owner[u]];
+            const int e0 = m->tp_first[u], e1 = m->tp_first[v];
+            if (e1 > e0)
+                transpose_split_f32(m->tp_dev + e0, e1 - e0, m->tp_host[e0].tile0, m->tp_host[e1].tile0 - m->tp_host[e0].tile0,
+                                    ar.w, ar.wt, ar.wtl, st);
+            u = v;
+        }
+        return;
+    }
     for (int i = m->unit_first[a]; i <= m->unit_last[b - 1]; ++i) {
         const Op& o = m->ops[i];
         const Arena& ar = m->arena[m->owner[o.d.unit]];
@@ -325,8 +361,9 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
                 if (m->cfg.precision == FTP_FP32) {
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
-                    const bool tc = is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, in, ar.w + o.w_off, out, nullptr) &&
-                                    tc32_gemm((const float*)in, ar.w + o.w_off, 1, nullptr, (float*)out, (int)Mout, o.Co, o.C, m->tc_err, st);
+                    const bool tc = is_pointwise_op(o) && o.d.kind != FTP_FC && tc32_supported((int)Mout, o.Co, o.C, in, ar.wt + o.w_off, out, nullptr) &&
+                                    tc32_gemm((const float*)in, ar.wt + o.w_off, ar.wtl + o.w_off, 0, nullptr, (float*)out, m->red_scratch, (int)Mout, o.Co, o.C,
+                                              m->tc_err, st);
                     if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_FWD;
                     if (!tc) conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                 } else if constexpr (!std::is_same<T, float>::value) {
@@ -483,7 +520,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the weights as they lie are the K-major B operand
                         const bool tc = !widened && is_pointwise_op(o) && tc32_supported((int)Mout, o.C, o.Co, d, ar.w + o.w_off, gi, addend) &&
-                                        tc32_gemm(d, ar.w + o.w_off, 0, (const float*)addend, (float*)gi, (int)Mout, o.C, o.Co, m->tc_err, st);
+                                        tc32_gemm(d, ar.w + o.w_off, ar.wl + o.w_off, 0, (const float*)addend, (float*)gi, m->red_scratch, (int)Mout, o.C, o.Co,
+                                                  m->tc_err, st);
                         if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_DGRAD;
                         if (!tc) conv_dgrad_f32(d, ar.w + o.w_off, widened ? nullptr : (const float*)addend, widened ? m->fc_din : (float*)gi, m->red_scratch, o.g, st);
                         if (widened) f32_to_bf16(m->fc_din, (__nv_bfloat16*)gi, o.in_elems, st);
@@ -594,12 +632,13 @@ ftp_status sgd_range(ftp_model* m, int a, int b, float lr, float* snap_dev, floa
             Scope sc(m, st, K_SGD, u, -1, 2, cnt * (mu != 0.f ? (m->mom_init[u] ? 20.0 : 16.0) : 12.0) + (ar.wb ? 2.0 * cnt : 0.0) +
                      (snap_dev ? 4.0 * cnt : 0.0) + (snap_host ? 4.0 * cnt : 0.0), 6.0 * cnt);
             sgd_update(ar.w + off, m->grad + off, mu != 0.f ? ar.m + off : nullptr, cnt, lr, mu, wd, m->mom_init[u] ? 0 : 1,
-                       ar.wb ? ar.wb + off : nullptr, snap_dev ? snap_dev + rel : nullptr, snap_host ? snap_host + rel : nullptr, st);
+                       ar.wb ? ar.wb + off : nullptr, ar.wl ? ar.wl + off : nullptr, snap_dev ? snap_dev + rel : nullptr,
+                       snap_host ? snap_host + rel : nullptr, st);
         }
         for (int k = u; k < v; ++k) m->mom_init[k] = 1;
         u = v;
     }
-    if (m->cfg.precision == FTP_BF16) refresh_transposed(m, a, b, st);
+    refresh_transposed(m, a, b, st);
     return check_launches("sgd_step");
 }
 
@@ -652,6 +691,11 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
     if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess || cudaMemset(m->fin_side.counters, 0, m->fin_counter_bytes) != cudaSuccess ||
         cudaMemset(m->tc_err, 0, 256) != cudaSuccess) {     // ticket counters start at zero
         const ftp_status e = fail(FTP_ECUDA, "build_model: clearing the ticket counters failed: %s", cudaGetErrorString(cudaGetLastError()));
+        delete m;
+        return e;
+    }
+    if (cudaMemcpy(m->tp_dev, m->tp_host.data(), m->tp_host.size() * sizeof(TransposeEntryDev), cudaMemcpyHostToDevice) != cudaSuccess) {
+        const ftp_status e = fail(FTP_ECUDA, "build_model: uploading the transposition table failed: %s", cudaGetErrorString(cudaGetLastError()));
         delete m;
         return e;
     }
@@ -754,6 +798,11 @@ extern "C" ftp_status ftp_set_tensor(ftp_model* m, int32_t which, int32_t unit, 
         if (ar.wb) {
             Scope sc(m, st, K_COPY, unit, -1, 2, 6.0 * count, 0.0);
             f32_to_bf16(dst, ar.wb + m->unit_p_off[unit], count, st);
+            refresh_transposed(m, unit, unit + 1, st);
+        }
+        if (ar.wl) {
+            Scope sc(m, st, K_COPY, unit, -1, 2, 16.0 * count, 0.0);
+            tf32_lo(dst, ar.wl + m->unit_p_off[unit], count, st);
             refresh_transposed(m, unit, unit + 1, st);
         }
         m->mom_init[unit] = 0;
@@ -920,6 +969,11 @@ extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int
                 CUDA_OK(cudaMemcpyAsync(to.m + po, from.m + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
                 if (to.wb) CUDA_OK(cudaMemcpyAsync(to.wb + po, from.wb + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
                 if (to.wbt) CUDA_OK(cudaMemcpyAsync(to.wbt + po, from.wbt + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
+                if (to.wl) {
+                    CUDA_OK(cudaMemcpyAsync(to.wl + po, from.wl + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+                    CUDA_OK(cudaMemcpyAsync(to.wt + po, from.wt + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+                    CUDA_OK(cudaMemcpyAsync(to.wtl + po, from.wtl + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+                }
             }
             if (sc_) CUDA_OK(cudaMemcpyAsync(to.run + so, from.run + so, (size_t)sc_ * 4, cudaMemcpyDeviceToDevice, st));
         }

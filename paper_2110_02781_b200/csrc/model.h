@@ -41,6 +41,9 @@ struct Arena {
     float* run;
     __nv_bfloat16* wb;       // bf16 copy of w, same layout
     __nv_bfloat16* wbt;      // bf16 copy with every 1x1-convolution matrix transposed ([cout][cin]): the forward's K-major B operand
+    // float models, for the split-tf32 tensor-core products: wl = w - trunc_tf32(w), same layout as w (data gradient);
+    // wt / wtl = every 1x1-convolution matrix transposed, as it is and its lo part (forward)
+    float* wl; float* wt; float* wtl;
 };
 
 struct TraceSlot { cudaEvent_t e0, e1; ftp_trace_rec rec; };
@@ -69,6 +72,8 @@ struct ftp_model {
     // weight gradients run on a second stream beside the chain of input gradients; they have scratch of their own
     float* red_side; ftp::FinScratch fin_side;
     cudaStream_t side; std::vector<cudaEvent_t> ev_fork, ev_side; bool overlap;
+    std::vector<ftp::TransposeEntryDev> tp_host; std::vector<int> tp_first;   // tp_first[u]: first entry of unit u (L + 1 values)
+    ftp::TransposeEntryDev* tp_dev;
     void* dpre; size_t dpre_bytes;
     int* tc_err;                                  // device word set by a tensor-core kernel whose bounded wait ran out
     float* fc_in; float* fc_din;                  // bf16 models: the classifier's input and input gradient widened to float
