@@ -2,14 +2,19 @@
 // hi = x with the low 13 mantissa bits cleared (exactly representable as tf32) and lo = x - hi (exact), and
 // the product is accumulated as hi*hi + hi*lo + lo*hi with tcgen05.mma kind::tf32 into a float accumulator in
 // tensor memory.  The dropped lo*lo term and the tf32 truncation of lo are below 2^-20 relative, which keeps
-// the float path within 1e-4 of a float64 reference while the math leaves the SIMT pipes.
+// the float path within 1e-4 of a float64 reference while the math leaves the SIMT pipes.  The tensor core
+// reads only the upper 19 bits of a tf32 operand, so a float tile as it lies in memory already is its hi part.
 //
-// Same structure as the bf16 kernels: one 128 x BN tile per CTA; warp 0 streams 128 x 32 and BN x 32 float
-// tiles with TMA (128-byte swizzle, zero fill); warps 2-5 split each landed stage into a hi and a lo tile,
-// make the writes visible to the tensor-core proxy and signal warp 1, which issues the 3 x 4 MMAs (K = 8) of
-// the stage; at the end warps 2-5 read the accumulator and store floats.  The tensor cores always see
-// K-major operands: an operand that lies the other way in memory (activations in the weight gradient, the
-// weights in the forward) is transposed inside shared memory by the same pass that splits it.
+// Two kernels, one 128 x BN tile (and one slice of the reduction) per CTA, warp roles as in the bf16 kernels:
+//  * tc32_kernel: both operands with the reduction contiguous (forward with pre-transposed weights, data
+//    gradient).  Warp 0 streams 128 x 32 and BN x 32 float tiles with TMA (128-byte swizzle, zero fill); warps
+//    2-5 write the lo tile of A (and of B, unless the caller keeps B's lo part in memory, as the model does for
+//    its weights), make the writes visible to the tensor-core proxy and signal warp 1, which issues the 3 x 4
+//    MMAs (K = 8) of the stage; at the end warps 2-5 read the accumulator, stage it in shared memory and store
+//    it with TMA.
+//  * tc32_wgrad_kernel: both operands have the reduction as their slow dimension (activations and output
+//    gradients of the weight gradient); they land in a ring of source buffers and are transposed and split
+//    into K-major operand buffers by warps 2-5, the loads running ahead of conversion and MMAs.
 // Every wait is bounded; see gemm_tc.cu for the error protocol.
 #include "gemm_tc_common.cuh"
 
@@ -72,42 +77,86 @@ struct T32Params {
     const float* addend;   // gemm with S == 1 only, nullable
     int M, N, K;           // gemm: D[M,N] = A[M,K] B[N,K]^T.  wgrad: Mo = M, No = N, K = reduction rows R
     int rows_per_split;    // reduction elements per slice (a multiple of 32)
-    int b_lo_given;        // MODE 0: the lo part of B comes from memory (mapBlo) instead of being computed per tile
+    int b_lo_given;        // gemm: the lo part of B comes from memory (mapBlo) instead of being computed per tile
     int* err;
 };
 
-// MODE 0: A [M][K], B [N][K], both with K contiguous (data gradient).  MODE 1: X [R][Mo], dY [R][No], both transposed
-// in shared memory (weight gradient).  MODE 2: A [M][K] as it lies, B [K][N] (the weights) transposed (forward).
-template <int BN, int STAGES, int MODE>
+// Epilogue shared by both kernels, run by warps 2..5: accumulator -> shared-memory tiles of 128 rows x 32 columns
+// (the operand buffers are free by now) -> one TMA store per tile, which writes whole lines and clips at the
+// edges of the output.  `have`: the accumulator is complete (or there was nothing to accumulate).
+template <int BN>
+__device__ __forceinline__ void epilogue32(uint8_t* smem, uint32_t tmem, const CUtensorMap* mapD, const T32Params& p, const float* addend, int m0, int n0,
+                                           int split, int num_kb, bool have) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, q = warp & 3;
+    if (have) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int row = q * 32 + lane, m = m0 + row;
+        const float* arow = (addend && m < p.M) ? addend + (long long)m * p.N : nullptr;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            uint32_t r[32];
+            if (num_kb > 0) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+            else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) r[e] = 0u;
+            }
+            const int nb = n0 + c * 32;
+            uint8_t* trow = smem + c * (TC_BM * 128) + row * 128;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                if (arow && nb + g * 4 < p.N) { const float4 a = __ldg(reinterpret_cast<const float4*>(arow + nb + g * 4)); v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w; }
+                *reinterpret_cast<float4*>(trow + ((g ^ (row & 7)) << 4)) = v;
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");                      // the four epilogue warps
+    if (have && threadIdx.x == 64) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c)
+            if (n0 + c * 32 < p.N)
+                asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                             ::"l"(mapD), "r"(n0 + c * 32), "r"(m0), "r"(split), "r"(smem_u32(smem + c * (TC_BM * 128))) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
+    }
+}
+
+// twelve tf32 MMAs per 32-wide block of the reduction: hi*hi, hi*lo, lo*hi for each of its four 8-wide steps
+template <int BN>
+__device__ __forceinline__ void mma_block32(uint32_t tmem, uint32_t a_hi, uint32_t a_lo, uint32_t b_hi, uint32_t b_lo, bool first) {
+    constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+    const uint64_t ah = umma_desc_k_sw128(a_hi), al = umma_desc_k_sw128(a_lo);
+    const uint64_t bh = umma_desc_k_sw128(b_hi), bl = umma_desc_k_sw128(b_lo);
+#pragma unroll
+    for (int k = 0; k < T32_BK / 8; ++k) {                 // 8 reduction steps = 32 bytes further along the row
+        const uint64_t o = (uint64_t)(k * 2);
+        umma_tf32(tmem, ah + o, bh + o, idesc, (!first || k > 0) ? 1u : 0u);
+        umma_tf32(tmem, ah + o, bl + o, idesc, 1u);
+        umma_tf32(tmem, al + o, bh + o, idesc, 1u);
+    }
+}
+
+// D[M,N] (one slice of the reduction per blockIdx.z) = A[M,K] B[N,K]^T, both operands with K contiguous.
+// Stage: [A as loaded = hi][A lo][B hi][B lo].
+template <int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                                                           const __grid_constant__ CUtensorMap mapBlo, const __grid_constant__ CUtensorMap mapD,
                                                           const T32Params p) {
     constexpr uint32_t A_BYTES = TC_BM * T32_BK * 4, B_BYTES = BN * T32_BK * 4;          // one precision part
-    constexpr bool TA = MODE == 1, TB = MODE != 0;                                      // operand transposed in shared memory
-    constexpr uint32_t STAGE_BYTES = 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) + (TB ? B_BYTES : 0);   // [A hi][A lo][B hi][B lo][A src][B src]
-    constexpr uint32_t SLAB = 32 * 32 * 4;                                              // transposed operands land as slabs of 32 columns x 32 rows
+    constexpr uint32_t STAGE_BYTES = 2 * (A_BYTES + B_BYTES);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ __align__(8) unsigned long long bars[3 * STAGES + 1];
     __shared__ uint32_t tmem_base;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int m0, n0, kbeg, kend, split = 0;
-    constexpr bool WGRAD = MODE == 1;
-    if (WGRAD) {
-        m0 = blockIdx.x * TC_BM; n0 = blockIdx.y * BN; split = blockIdx.z;
-        kbeg = split * p.rows_per_split; kend = min(p.K, kbeg + p.rows_per_split);
-    } else {
-        n0 = blockIdx.x * BN; m0 = blockIdx.y * TC_BM; split = blockIdx.z;
-        kbeg = split * p.rows_per_split; kend = min(p.K, kbeg + p.rows_per_split);
-    }
+    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * TC_BM, split = blockIdx.z;
+    const int kbeg = split * p.rows_per_split, kend = min(p.K, kbeg + p.rows_per_split);
     const int num_kb = (kend - kbeg + T32_BK - 1) / T32_BK;
-    // transposed operands arrive as 32-column slabs: slabs wholly beyond the matrix are neither loaded nor converted
-    // (their rows of the hi / lo tiles are cleared once)
-    const int slabsA = TA ? min(TC_BM / 32, (p.M - m0 + 31) / 32) : TC_BM / 32;
-    const int slabsB = TB ? min(BN / 32, (p.N - n0 + 31) / 32) : BN / 32;
-    const bool b_pre = MODE == 0 && p.b_lo_given;
-    const uint32_t tx_bytes = (TA ? slabsA * SLAB : A_BYTES) + (TB ? slabsB * SLAB : B_BYTES) + (b_pre ? B_BYTES : 0);
+    const bool b_pre = p.b_lo_given != 0;
+    const uint32_t tx_bytes = A_BYTES + B_BYTES + (b_pre ? B_BYTES : 0);
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), ready0 = smem_u32(&bars[2 * STAGES]), accum = smem_u32(&bars[3 * STAGES]);
 
     if (threadIdx.x == 0) {
@@ -132,17 +181,11 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
                 const int s = kb % STAGES;
                 const uint32_t ph = (kb / STAGES) & 1;
                 if (kb >= STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 11)) break;
-                const uint32_t st0 = smem_u32(smem + s * STAGE_BYTES);
-                const uint32_t sa = TA ? st0 + 2 * (A_BYTES + B_BYTES) : st0;                                       // where A lands
-                const uint32_t sb = TB ? st0 + 2 * (A_BYTES + B_BYTES) + (TA ? A_BYTES : 0) : st0 + 2 * A_BYTES;   // where B lands
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + 2 * A_BYTES;
                 const int k = kbeg + kb * T32_BK;
                 mbar_expect_tx(full0 + 8 * s, tx_bytes);
-                if (TA) {
-                    for (int t = 0; t < slabsA; ++t) tma_load_2d(sa + t * SLAB, &mapA, m0 + 32 * t, k, full0 + 8 * s);
-                } else tma_load_2d(sa, &mapA, k, m0, full0 + 8 * s);
-                if (TB) {
-                    for (int t = 0; t < slabsB; ++t) tma_load_2d(sb + t * SLAB, &mapB, n0 + 32 * t, k, full0 + 8 * s);
-                } else tma_load_2d(sb, &mapB, k, n0, full0 + 8 * s);
+                tma_load_2d(sa, &mapA, k, m0, full0 + 8 * s);
+                tma_load_2d(sb, &mapB, k, n0, full0 + 8 * s);
                 if (b_pre) tma_load_2d(sb + B_BYTES, &mapBlo, k, n0, full0 + 8 * s);
                 issued = kb + 1;
             }
@@ -155,92 +198,157 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % STAGES;
                 const uint32_t ph = (kb / STAGES) & 1;
-                ok = mbar_wait(ready0 + 8 * s, ph, p.err, 12);                   // split done and visible
+                ok = mbar_wait(ready0 + 8 * s, ph, p.err, 12);                   // lo parts written and visible
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + 2 * A_BYTES;
-                const uint64_t ah = umma_desc_k_sw128(sa), al = umma_desc_k_sw128(sa + A_BYTES);
-                const uint64_t bh = umma_desc_k_sw128(sb), bl = umma_desc_k_sw128(sb + B_BYTES);
-#pragma unroll
-                for (int k = 0; k < T32_BK / 8; ++k) {                 // 8 reduction steps = 32 bytes further along the row
-                    const uint64_t o = (uint64_t)(k * 2);
-                    umma_tf32(tmem, ah + o, bh + o, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    umma_tf32(tmem, ah + o, bl + o, idesc, 1u);
-                    umma_tf32(tmem, al + o, bh + o, idesc, 1u);
-                }
+                mma_block32<BN>(tmem, sa, sa + A_BYTES, sb, sb + B_BYTES, kb == 0);
                 umma_commit(empty0 + 8 * s);
             }
             if (ok) umma_commit(accum);
         }
     } else {
-        // ---- warps 2..5: split every landed stage, then the epilogue ----
+        // ---- warps 2..5: lo part of every landed stage, then the epilogue ----
         const int t = threadIdx.x - 64;
         bool ok = true;
-        if ((TA && slabsA < TC_BM / 32) || (TB && slabsB < BN / 32)) {
-            // clear the rows of the hi / lo tiles that no slab will ever fill
-            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int s = 0; s < STAGES; ++s) {
-                uint8_t* st = smem + s * STAGE_BYTES;
-                if (TA) for (int i = slabsA * SLAB + t * 16; i < (int)A_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + i) = z; *reinterpret_cast<float4*>(st + A_BYTES + i) = z; }
-                if (TB) for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
-            }
-        }
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % STAGES;
             const uint32_t ph = (kb / STAGES) & 1;
             ok = mbar_wait(full0 + 8 * s, ph, p.err, 13);
             if (!ok) break;
             uint8_t* st = smem + s * STAGE_BYTES;
-            uint8_t* src = st + 2 * (A_BYTES + B_BYTES);
-            if (TA) transpose_split(src, st, st + A_BYTES, slabsA, t, 128);
-            else split_tile(st, st + A_BYTES, A_BYTES, t, 128);
-            if (TB) transpose_split(src + (TA ? A_BYTES : 0), st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, t, 128);
-            else if (!b_pre) split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t, 128);
+            split_tile(st, st + A_BYTES, A_BYTES, t, 128);
+            if (!b_pre) split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t, 128);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
             mbar_arrive(ready0 + 8 * s);
         }
-        // ---- epilogue: accumulator -> shared-memory tiles of 128 rows x 32 columns (the operand stages are free
-        // now) -> one TMA store per tile, which writes whole lines and clips at the edges of the output ----
-        const int q = warp & 3;
         const bool have = ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true);
-        if (have) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int row = q * 32 + lane, m = m0 + row;
-            const float* arow = (!WGRAD && p.addend && m < p.M) ? p.addend + (long long)m * p.N : nullptr;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                if (num_kb > 0) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
-                else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) r[e] = 0u;
-                }
-                const int nb = n0 + c * 32;
-                uint8_t* trow = smem + c * (TC_BM * 128) + row * 128;
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]), __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
-                    if (arow && nb + g * 4 < p.N) { const float4 a = __ldg(reinterpret_cast<const float4*>(arow + nb + g * 4)); v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w; }
-                    *reinterpret_cast<float4*>(trow + ((g ^ (row & 7)) << 4)) = v;
+        epilogue32<BN>(smem, tmem, &mapD, p, p.addend, m0, n0, split, num_kb, have);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+}
+
+// Weight gradient: partials [slice][Mo][No] of X[R][Mo]^T dY[R][No].  Both operands have the reduction (rows) as
+// their slow dimension, so they land as slabs of 32 rows x 32 columns in a ring of source buffers; warps 2..5
+// transpose and split each source buffer into one of two operand buffers ([A hi][A lo][B hi][B lo]) and hand
+// the source buffer straight back to the loader, so that the loads run several reduction blocks ahead of the
+// conversion and the MMAs instead of waiting for them.
+template <int BN> struct Wg32Smem {
+    static constexpr uint32_t A_BYTES = TC_BM * T32_BK * 4, B_BYTES = BN * T32_BK * 4;
+    static constexpr uint32_t SRC_BYTES = A_BYTES + B_BYTES, OP_BYTES = 2 * SRC_BYTES;
+    static constexpr int NOP = 2;
+    static constexpr int NSRC_FIT = (226 * 1024 - NOP * (int)OP_BYTES) / (int)SRC_BYTES;
+    static constexpr int NSRC = NSRC_FIT > 6 ? 6 : NSRC_FIT;
+    static constexpr int TOTAL = NOP * (int)OP_BYTES + NSRC * (int)SRC_BYTES + 1024;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS) tc32_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+                                                                const __grid_constant__ CUtensorMap mapD, const T32Params p) {
+    using L = Wg32Smem<BN>;
+    constexpr uint32_t A_BYTES = L::A_BYTES, B_BYTES = L::B_BYTES, SRC_BYTES = L::SRC_BYTES, OP_BYTES = L::OP_BYTES, SLAB = 32 * 32 * 4;
+    constexpr int NOP = L::NOP, NSRC = L::NSRC;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* srcs = smem + NOP * OP_BYTES;
+    __shared__ __align__(8) unsigned long long bars[2 * NSRC + 2 * NOP + 1];
+    __shared__ uint32_t tmem_base;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * TC_BM, n0 = blockIdx.y * BN, split = blockIdx.z;
+    const int kbeg = split * p.rows_per_split, kend = min(p.K, kbeg + p.rows_per_split);
+    const int num_kb = (kend - kbeg + T32_BK - 1) / T32_BK;
+    // slabs wholly beyond the matrix are neither loaded nor converted (their rows of the hi / lo tiles are cleared once)
+    const int slabsA = min(TC_BM / 32, (p.M - m0 + 31) / 32), slabsB = min(BN / 32, (p.N - n0 + 31) / 32);
+    const uint32_t tx_bytes = (uint32_t)(slabsA + slabsB) * SLAB;
+    const uint32_t sfull0 = smem_u32(&bars[0]), sempty0 = smem_u32(&bars[NSRC]), ready0 = smem_u32(&bars[2 * NSRC]),
+                   oempty0 = smem_u32(&bars[2 * NSRC + NOP]), accum = smem_u32(&bars[2 * NSRC + 2 * NOP]);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NSRC; ++s) { mbar_init(sfull0 + 8 * s, 1); mbar_init(sempty0 + 8 * s, 128); }
+        for (int s = 0; s < NOP; ++s) { mbar_init(ready0 + 8 * s, 128); mbar_init(oempty0 + 8 * s, 1); }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base;
+    grid_dep_sync();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % NSRC;
+                const uint32_t ph = (kb / NSRC) & 1;
+                if (kb >= NSRC && !mbar_wait(sempty0 + 8 * s, ph ^ 1, p.err, 11)) break;
+                const uint32_t sa = smem_u32(srcs + s * SRC_BYTES), sb = sa + A_BYTES;
+                const int k = kbeg + kb * T32_BK;
+                mbar_expect_tx(sfull0 + 8 * s, tx_bytes);
+                for (int t = 0; t < slabsA; ++t) tma_load_2d(sa + t * SLAB, &mapX, m0 + 32 * t, k, sfull0 + 8 * s);
+                for (int t = 0; t < slabsB; ++t) tma_load_2d(sb + t * SLAB, &mapY, n0 + 32 * t, k, sfull0 + 8 * s);
+                issued = kb + 1;
+            }
+            if (*((volatile int*)p.err) != 0) {
+                for (int kb = max(0, issued - NSRC); kb < issued; ++kb) {
+                    const unsigned long long t0 = gtime();
+                    while (!mbar_test(sfull0 + 8 * (kb % NSRC), (kb / NSRC) & 1) && gtime() - t0 < 1000000ull) __nanosleep(128);
                 }
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");                      // the four epilogue warps
-        if (have && threadIdx.x == 64) {
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c)
-                if (n0 + c * 32 < p.N)
-                    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
-                                 ::"l"(&mapD), "r"(n0 + c * 32), "r"(m0), "r"(split), "r"(smem_u32(smem + c * (TC_BM * 128))) : "memory");
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % NOP;
+                const uint32_t ph = (kb / NOP) & 1;
+                ok = mbar_wait(ready0 + 8 * s, ph, p.err, 12);                   // transposed, split and visible
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = smem_u32(smem + s * OP_BYTES), sb = sa + 2 * A_BYTES;
+                mma_block32<BN>(tmem, sa, sa + A_BYTES, sb, sb + B_BYTES, kb == 0);
+                umma_commit(oempty0 + 8 * s);
+            }
+            if (ok) umma_commit(accum);
         }
+    } else {
+        const int t = threadIdx.x - 64;
+        bool ok = true;
+        if (slabsA < TC_BM / 32 || slabsB < BN / 32) {
+            // clear the rows of the hi / lo tiles that no slab will ever fill
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s = 0; s < NOP; ++s) {
+                uint8_t* st = smem + s * OP_BYTES;
+                for (int i = slabsA * SLAB + t * 16; i < (int)A_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + i) = z; *reinterpret_cast<float4*>(st + A_BYTES + i) = z; }
+                for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
+            }
+        }
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int ss = kb % NSRC, os = kb % NOP;
+            ok = mbar_wait(sfull0 + 8 * ss, (kb / NSRC) & 1, p.err, 13);
+            if (ok && kb >= NOP) ok = mbar_wait(oempty0 + 8 * os, ((kb / NOP) & 1) ^ 1, p.err, 15);   // the MMAs that read this operand buffer are done
+            if (!ok) break;
+            const uint8_t* src = srcs + ss * SRC_BYTES;
+            uint8_t* st = smem + os * OP_BYTES;
+            transpose_split(src, st, st + A_BYTES, slabsA, t, 128);
+            transpose_split(src + A_BYTES, st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, t, 128);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
+            mbar_arrive(ready0 + 8 * os);
+            mbar_arrive(sempty0 + 8 * ss);                                      // the loader may refill the source buffer
+        }
+        const bool have = ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true);
+        epilogue32<BN>(smem, tmem, &mapD, p, nullptr, m0, n0, split, num_kb, have);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -271,13 +379,22 @@ bool make_map_out(CUtensorMap* map, const void* base, long long S, long long row
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES, int MODE>
+template <int BN, int STAGES>
 bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
-    constexpr int ring = STAGES * (2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0));
+    constexpr int ring = STAGES * 2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4);
     constexpr int stage_out = TC_BM * BN * 4;                         // the epilogue reuses the ring as its staging area
     constexpr int smem = (ring > stage_out ? ring : stage_out) + 1024;
-    if (cudaFuncSetAttribute(tc32_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    launch(tc32_kernel<BN, STAGES, MODE>, grid, dim3(TC_THREADS), smem, st, ma, mb, ml, md, p);
+    if (cudaFuncSetAttribute(tc32_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    launch(tc32_kernel<BN, STAGES>, grid, dim3(TC_THREADS), smem, st, ma, mb, ml, md, p);
+    return true;
+}
+
+template <int BN>
+bool launch32_wgrad(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
+    constexpr int smem = Wg32Smem<BN>::TOTAL;
+    static_assert(Wg32Smem<BN>::NSRC >= 2 && Wg32Smem<BN>::NOP * (int)Wg32Smem<BN>::OP_BYTES >= TC_BM * BN * 4, "shared-memory plan");
+    if (cudaFuncSetAttribute(tc32_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    launch(tc32_wgrad_kernel<BN>, grid, dim3(TC_THREADS), smem, st, mx, my, md, p);
     return true;
 }
 
@@ -305,28 +422,25 @@ bool tc32_supported(int M, int N, int K, const void* A, const void* B, const voi
     return M >= 1 && N % 4 == 0 && K % 4 == 0 && N >= 4 && K >= 4 && a16(A) && a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
 }
 
-constexpr int stage_bytes32(int BN, int MODE) {
-    return 2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4) + (MODE == 1 ? TC_BM * T32_BK * 4 : 0) + (MODE != 0 ? BN * T32_BK * 4 : 0);
-}
-constexpr int max_stages32(int BN, int MODE) {
-    const int n = (226 * 1024) / stage_bytes32(BN, MODE);
+constexpr int max_stages32(int BN) {
+    const int n = (226 * 1024) / (2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4));
     return n > 4 ? 4 : n;
 }
 
-template <int BN, int MODE>
+template <int BN>
 bool launch32_stages(int num_kb, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& md, const T32Params& p, dim3 grid,
                      cudaStream_t st) {
     // Many tiles (memory-bound layers): one stage per CTA, so that several CTAs share an SM and hide each other's
     // latencies.  Few tiles (late layers, long reductions): as deep a ring as shared memory holds instead.
-    constexpr int MAXS = max_stages32(BN, MODE);
+    constexpr int MAXS = max_stages32(BN);
     const long long tiles = (long long)grid.x * grid.y * grid.z;
     int stages = tiles >= 4LL * sm_count() ? 1 : (tiles >= 2LL * sm_count() ? 2 : MAXS);
     if (stages > num_kb) stages = num_kb < 1 ? 1 : num_kb;
     if (stages > MAXS) stages = MAXS;
-    if (stages == 1) return launch32<BN, 1, MODE>(ma, mb, ml, md, p, grid, st);
-    if (stages == 2) return launch32<BN, 2, MODE>(ma, mb, ml, md, p, grid, st);
-    if constexpr (MAXS >= 3) { if (stages == 3) return launch32<BN, 3, MODE>(ma, mb, ml, md, p, grid, st); }
-    if constexpr (MAXS >= 4) { if (stages == 4) return launch32<BN, 4, MODE>(ma, mb, ml, md, p, grid, st); }
+    if (stages == 1) return launch32<BN, 1>(ma, mb, ml, md, p, grid, st);
+    if (stages == 2) return launch32<BN, 2>(ma, mb, ml, md, p, grid, st);
+    if constexpr (MAXS >= 3) { if (stages == 3) return launch32<BN, 3>(ma, mb, ml, md, p, grid, st); }
+    if constexpr (MAXS >= 4) { if (stages == 4) return launch32<BN, 4>(ma, mb, ml, md, p, grid, st); }
     return false;
 }
 
@@ -368,33 +482,23 @@ G32Plan plan_gemm32(int M, int N, int K) {
     return g;
 }
 
-// D[M,N] = A[M,K] * B (+ addend), float in and out, split-tf32 arithmetic.
-// b_is_kn == 0: B is [N][K] (K contiguous); b_is_kn == 1: B is [K][N] (N contiguous, as convolution weights lie).
-bool tc32_gemm(const float* A, const float* B, const float* B_lo, int b_is_kn, const float* addend, float* D, float* scratch, int M, int N, int K, int* err,
-               cudaStream_t st) {
+// D[M,N] = A[M,K] * B[N,K]^T (+ addend), float in and out, split-tf32 arithmetic; both operands with K contiguous.
+bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err, cudaStream_t st) {
     G32Plan g = plan_gemm32(M, N, K);
     if (g.S > 1 && !scratch) { g.S = 1; g.rps = (K + T32_BK - 1) / T32_BK * T32_BK; }
     const int BN = g.BN;
     float* out = g.S > 1 ? scratch : D;
     CUtensorMap ma, mb, ml, md;
-    if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, out, g.S, M, N)) return false;
-    if (!(b_is_kn ? make_map_f32(&mb, B, K, N, 32) : make_map_f32(&mb, B, N, K, BN))) return false;
-    const bool pre = !b_is_kn && B_lo != nullptr;
-    if (pre) { if (!make_map_f32(&ml, B_lo, N, K, BN)) return false; }
+    if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, out, g.S, M, N) || !make_map_f32(&mb, B, N, K, BN)) return false;
+    if (B_lo) { if (!make_map_f32(&ml, B_lo, N, K, BN)) return false; }
     else ml = mb;
-    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, pre ? 1 : 0, err};
+    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, B_lo ? 1 : 0, err};
     const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM, g.S);
     const int nkb = g.rps / T32_BK;
     bool ok;
-    if (b_is_kn) {
-        if (BN == 128) ok = launch32_stages<128, 2>(nkb, ma, mb, ml, md, p, grid, st);
-        else if (BN == 64) ok = launch32_stages<64, 2>(nkb, ma, mb, ml, md, p, grid, st);
-        else ok = launch32_stages<32, 2>(nkb, ma, mb, ml, md, p, grid, st);
-    } else {
-        if (BN == 128) ok = launch32_stages<128, 0>(nkb, ma, mb, ml, md, p, grid, st);
-        else if (BN == 64) ok = launch32_stages<64, 0>(nkb, ma, mb, ml, md, p, grid, st);
-        else ok = launch32_stages<32, 0>(nkb, ma, mb, ml, md, p, grid, st);
-    }
+    if (BN == 128) ok = launch32_stages<128>(nkb, ma, mb, ml, md, p, grid, st);
+    else if (BN == 64) ok = launch32_stages<64>(nkb, ma, mb, ml, md, p, grid, st);
+    else ok = launch32_stages<32>(nkb, ma, mb, ml, md, p, grid, st);
     if (ok && g.S > 1) {
         const long long count4 = (long long)M * N / 4;
         launch(slice_sum_kernel, dim3((unsigned)((count4 + 255) / 256)), dim3(256), 0, st, reinterpret_cast<const float4*>(scratch), g.S, count4,
@@ -422,11 +526,10 @@ int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long 
     if (!make_map_f32(&mx, X, R, Mo, 32) || !make_map_f32(&my, dY, R, No, 32) || !make_map_out(&md, out, w.S, Mo, No)) return 0;
     T32Params p{out, nullptr, Mo, No, (int)R, w.rows_per_split, 0, err};
     const dim3 grid((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S);
-    const int nkb = (w.rows_per_split + T32_BK - 1) / T32_BK;
     bool ok;
-    if (BN == 128) ok = launch32_stages<128, 1>(nkb, mx, my, my, md, p, grid, st);
-    else if (BN == 64) ok = launch32_stages<64, 1>(nkb, mx, my, my, md, p, grid, st);
-    else ok = launch32_stages<32, 1>(nkb, mx, my, my, md, p, grid, st);
+    if (BN == 128) ok = launch32_wgrad<128>(mx, my, md, p, grid, st);
+    else if (BN == 64) ok = launch32_wgrad<64>(mx, my, md, p, grid, st);
+    else ok = launch32_wgrad<32>(mx, my, md, p, grid, st);
     return ok ? w.S : 0;
 }
 

@@ -58,9 +58,9 @@ void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int 
 bool tc32_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
 // scratch (nullable): tc32_gemm_scratch_floats(M, N, K) floats; lets products with few tiles cut the reduction into slices
 size_t tc32_gemm_scratch_floats(int M, int N, int K);
-// B_lo (nullable, only with b_is_kn == 0): B - trunc_tf32(B) laid out like B, saves computing it per tile
-bool tc32_gemm(const float* A, const float* B, const float* B_lo, int b_is_kn, const float* addend, float* D, float* scratch, int M, int N, int K,
-               int* err, cudaStream_t st);
+// B is [N][K]; B_lo (nullable): B - trunc_tf32(B) laid out like B, saves computing it per tile
+bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err,
+               cudaStream_t st);
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
 int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
 

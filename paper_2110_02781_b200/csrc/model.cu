@@ -362,7 +362,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 if (m->cfg.precision == FTP_FP32) {
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
                     const bool tc = is_pointwise_op(o) && o.d.kind != FTP_FC && tc32_supported((int)Mout, o.Co, o.C, in, ar.wt + o.w_off, out, nullptr) &&
-                                    tc32_gemm((const float*)in, ar.wt + o.w_off, ar.wtl + o.w_off, 0, nullptr, (float*)out, m->red_scratch, (int)Mout, o.Co, o.C,
+                                    tc32_gemm((const float*)in, ar.wt + o.w_off, ar.wtl + o.w_off, nullptr, (float*)out, m->red_scratch, (int)Mout, o.Co, o.C,
                                               m->tc_err, st);
                     if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_FWD;
                     if (!tc) conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
@@ -520,7 +520,7 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the weights as they lie are the K-major B operand
                         const bool tc = !widened && is_pointwise_op(o) && tc32_supported((int)Mout, o.C, o.Co, d, ar.w + o.w_off, gi, addend) &&
-                                        tc32_gemm(d, ar.w + o.w_off, ar.wl + o.w_off, 0, (const float*)addend, (float*)gi, m->red_scratch, (int)Mout, o.C, o.Co,
+                                        tc32_gemm(d, ar.w + o.w_off, ar.wl + o.w_off, (const float*)addend, (float*)gi, m->red_scratch, (int)Mout, o.C, o.Co,
                                                   m->tc_err, st);
                         if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_DGRAD;
                         if (!tc) conv_dgrad_f32(d, ar.w + o.w_off, widened ? nullptr : (const float*)addend, widened ? m->fc_din : (float*)gi, m->red_scratch, o.g, st);
