@@ -464,6 +464,21 @@ __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restri
     }
 }
 
+// the same for few slices: one thread per element, z ascending
+__global__ void __launch_bounds__(256) split_reduce_flat_kernel(const float* __restrict__ partial, int S, long long count, float* __restrict__ out) {
+    grid_dep_sync();
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count) return;
+    float s = 0.f;
+    for (int z = 0; z < S; ++z) s += partial[(long long)z * count + e];
+    out[e] = s;
+}
+
+static inline void launch_split_reduce(const float* partial, int S, long long count, float* out, cudaStream_t st) {
+    if (S >= 16) launch(split_reduce_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, partial, S, count, out);
+    else launch(split_reduce_flat_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, partial, S, count, out);
+}
+
 // out[e] = sum_z partial[z][e] (+ bias[column]) (+ addend[e]), z ascending
 __global__ void split_reduce_add_kernel(const float* __restrict__ partial, int S, long long count4, const float* __restrict__ addend,
                                         const float* __restrict__ bias, int Cd, float* __restrict__ out) {
@@ -625,7 +640,7 @@ void conv_wgrad_t(const T* x, const T* dy, float* dw, float* scratch, const Conv
     else launch(conv_wgrad_kernel<64, T>, grid, dim3(NT), 0, st, p);
     if (w.S > 1) {
         const long long count = (long long)p.Kg * g.Cout;
-        launch(split_reduce_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, scratch, w.S, count, dw);
+        launch_split_reduce(scratch, w.S, count, dw, st);
     }
 }
 }  // namespace
@@ -644,7 +659,7 @@ void conv_dgrad_bf16_simt(const __nv_bfloat16* dy, const __nv_bfloat16* w, const
 }
 
 void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st) {
-    launch(split_reduce_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, partial, S, count, out);
+    launch_split_reduce(partial, S, count, out, st);
 }
 
 size_t conv_wgrad_scratch_floats(const ConvGeom& g) {

@@ -23,15 +23,18 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false (and an error code) when the phase did not complete in time.
+// Bounded wait: false (and an error code) when the phase did not complete in time.  try_wait itself suspends the
+// thread for a short, hardware-defined time, so the loop polls it back to back and only every 64th round looks
+// at the clock and at the error word (a global load), which would otherwise sit on every hand-off.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
     if (mbar_test(bar, parity)) return true;
     const unsigned long long t0 = gtime();
-    while (true) {
+    for (unsigned it = 1;; ++it) {
         if (mbar_test(bar, parity)) return true;
-        if (*((volatile int*)err) != 0) return false;                     // another role already gave up
-        if (gtime() - t0 > TC_WAIT_NS) { atomicCAS(err, 0, code); return false; }
-        __nanosleep(64);
+        if ((it & 63u) == 0u) {
+            if (*((volatile int*)err) != 0) return false;                 // another role already gave up
+            if (gtime() - t0 > TC_WAIT_NS) { atomicCAS(err, 0, code); return false; }
+        }
     }
 }
 
