@@ -53,6 +53,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
 
     if (threadIdx.x == 0) {
+        tma_prefetch_map(&mapA); tma_prefetch_map(&mapB);
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -200,6 +201,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
 
     if (threadIdx.x == 0) {
+        tma_prefetch_map(&mapX); tma_prefetch_map(&mapY);
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

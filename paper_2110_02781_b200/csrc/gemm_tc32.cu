@@ -160,6 +160,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), ready0 = smem_u32(&bars[2 * STAGES]), accum = smem_u32(&bars[3 * STAGES]);
 
     if (threadIdx.x == 0) {
+        tma_prefetch_map(&mapA); tma_prefetch_map(&mapB); tma_prefetch_map(&mapBlo); tma_prefetch_map(&mapD);
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(ready0 + 8 * s, 128); }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -271,6 +272,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_wgrad_kernel(const __grid_con
                    oempty0 = smem_u32(&bars[2 * NSRC + NOP]), accum = smem_u32(&bars[2 * NSRC + 2 * NOP]);
 
     if (threadIdx.x == 0) {
+        tma_prefetch_map(&mapX); tma_prefetch_map(&mapY); tma_prefetch_map(&mapD);
         for (int s = 0; s < NSRC; ++s) { mbar_init(sfull0 + 8 * s, 1); mbar_init(sempty0 + 8 * s, 128); }
         for (int s = 0; s < NOP; ++s) { mbar_init(ready0 + 8 * s, 128); mbar_init(oempty0 + 8 * s, 1); }
         mbar_init(accum, 1);
