@@ -400,9 +400,21 @@ bool launch32_wgrad(const CUtensorMap& mx, const CUtensorMap& my, const CUtensor
     return true;
 }
 
-struct Wg32Plan { int S, rows_per_split; };
+// The tensor core works on 128 x BN tiles whatever part of them is padding, so the weight gradient is computed as
+// dW or as dW^T, whichever pads less: the wider of (cin, cout) goes to the 128-row side.  A transposed result is
+// put right by the second pass, which then always runs.
+struct Wg32Plan { int S, rows_per_split, BN, swap; };
+static inline int bn_for(int n) { return n > 64 ? 128 : (n > 32 ? 64 : 32); }
+static inline long long mma_area(int m, int n) {
+    const int bn = bn_for(n);
+    return (long long)((m + TC_BM - 1) / TC_BM) * TC_BM * ((n + bn - 1) / bn) * bn;
+}
 Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
-    const long long tiles = ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
+    Wg32Plan w;
+    w.swap = mma_area(No, Mo) < mma_area(Mo, No) ? 1 : 0;
+    const int m = w.swap ? No : Mo, n = w.swap ? Mo : No;
+    w.BN = bn_for(n);
+    const long long tiles = (long long)((m + TC_BM - 1) / TC_BM) * ((n + w.BN - 1) / w.BN);
     long long S = (3LL * sm_count() + tiles - 1) / tiles;
     const long long maxS = (R + 255) / 256;
     long long cap = (2LL << 20) / ((long long)Mo * No);                     // partial sums cost traffic too: at most 2 Mi floats
@@ -411,10 +423,35 @@ Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
     if (S > cap) S = cap;
     if (S < 1) S = 1;
     const long long rps = ((R + S - 1) / S + 31) / 32 * 32;
-    Wg32Plan w;
     w.rows_per_split = (int)rps;
     w.S = (int)((R + rps - 1) / rps);
     return w;
+}
+
+// out[i][j] = sum_z partial[z][j][i] (partial slices are [cols][rows] = the transpose of out[rows][cols]); z in eight
+// interleaved runs combined in run order, as in the plain second pass
+__global__ void __launch_bounds__(256) slice_sum_transposed_kernel(const float* __restrict__ partial, int S, int rows, int cols, float* __restrict__ out) {
+    grid_dep_sync();
+    __shared__ float sh[8][33];
+    const long long count = (long long)rows * cols;
+    const long long e = (long long)blockIdx.x * 32 + threadIdx.x;
+    float s0 = 0.f, s1 = 0.f;
+    if (e < count) {
+        const long long src = (e % cols) * rows + e / cols;
+        for (int z = threadIdx.y; z < S; z += 16) {
+            const float a = partial[(long long)z * count + src];
+            const float b = z + 8 < S ? partial[(long long)(z + 8) * count + src] : 0.f;
+            s0 += a; s1 += b;
+        }
+    }
+    sh[threadIdx.y][threadIdx.x] = s0 + s1;
+    __syncthreads();
+    if (threadIdx.y == 0 && e < count) {
+        float s = 0.f;
+#pragma unroll
+        for (int y = 0; y < 8; ++y) s += sh[y][threadIdx.x];
+        out[e] = s;
+    }
 }
 
 }  // namespace
@@ -516,23 +553,31 @@ size_t tc32_gemm_scratch_floats(int M, int N, int K) {
 
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No) {
     const Wg32Plan w = plan_wgrad32(R, Mo, No);
-    return w.S > 1 ? (size_t)w.S * Mo * No : 0;
+    return (w.S > 1 || w.swap) ? (size_t)w.S * Mo * No : 0;
 }
 
-// dW[Mo][No] = X[R][Mo]^T * dY[R][No]; returns the number of splits (0: nothing launched)
-int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st) {
+// dW[Mo][No] = X[R][Mo]^T * dY[R][No], second pass included; false: nothing launched
+bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st) {
     const Wg32Plan w = plan_wgrad32(R, Mo, No);
-    const int BN = No > 64 ? 128 : (No > 32 ? 64 : 32);
+    const bool two_pass = w.S > 1 || w.swap;
+    if (two_pass && !scratch) return false;
+    const float* A = w.swap ? dY : X;
+    const float* B = w.swap ? X : dY;
+    const int m = w.swap ? No : Mo, n = w.swap ? Mo : No;
     CUtensorMap mx, my, md;
-    float* out = w.S > 1 ? scratch : dW;
-    if (!make_map_f32(&mx, X, R, Mo, 32) || !make_map_f32(&my, dY, R, No, 32) || !make_map_out(&md, out, w.S, Mo, No)) return 0;
-    T32Params p{out, nullptr, Mo, No, (int)R, w.rows_per_split, 0, err};
-    const dim3 grid((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S);
+    float* out = two_pass ? scratch : dW;
+    if (!make_map_f32(&mx, A, R, m, 32) || !make_map_f32(&my, B, R, n, 32) || !make_map_out(&md, out, w.S, m, n)) return false;
+    T32Params p{out, nullptr, m, n, (int)R, w.rows_per_split, 0, err};
+    const dim3 grid((m + TC_BM - 1) / TC_BM, (n + w.BN - 1) / w.BN, w.S);
     bool ok;
-    if (BN == 128) ok = launch32_wgrad<128>(mx, my, md, p, grid, st);
-    else if (BN == 64) ok = launch32_wgrad<64>(mx, my, md, p, grid, st);
+    if (w.BN == 128) ok = launch32_wgrad<128>(mx, my, md, p, grid, st);
+    else if (w.BN == 64) ok = launch32_wgrad<64>(mx, my, md, p, grid, st);
     else ok = launch32_wgrad<32>(mx, my, md, p, grid, st);
-    return ok ? w.S : 0;
+    if (!ok) return false;
+    const long long count = (long long)Mo * No;
+    if (w.swap) launch(slice_sum_transposed_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, (const float*)scratch, w.S, Mo, No, dW);
+    else if (w.S > 1) split_reduce_f32(scratch, w.S, count, dW, st);
+    return true;
 }
 
 }  // namespace ftp

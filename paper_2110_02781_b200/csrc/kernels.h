@@ -62,7 +62,8 @@ size_t tc32_gemm_scratch_floats(int M, int N, int K);
 bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err,
                cudaStream_t st);
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
-int tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
+// dW[Mo][No] = X[R][Mo]^T dY[R][No], the fixed-order second pass over the reduction slices included
+bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
 
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
 // Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole

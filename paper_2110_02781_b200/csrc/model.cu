@@ -509,12 +509,10 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                     { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
                       const cudaStream_t ws = fork(i);
                       float* rs = ws == st ? m->red_scratch : m->red_side;
-                      int splits = 0;
-                      if (is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr))
-                          splits = tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws);
-                      if (splits > 1) split_reduce_f32(rs, splits, o.w_cnt, gr + o.w_off, ws);
-                      if (splits > 0 && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
-                      if (splits == 0) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
+                      const bool tc = is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr) &&
+                                      tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws);
+                      if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
+                      if (!tc) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
                       forked(i, d); }
                     if (gi) {
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
