@@ -34,26 +34,36 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint6
 // Transposing split.  src: nslabs slabs of [32 reduction rows][32 columns] floats as TMA wrote them (128-byte rows,
 // 16-byte chunk index XORed with row % 8).  hi / lo: K-major tiles [nslabs * 32 rows][32 reduction steps] in the
 // same swizzle.  A work item moves one output row's four consecutive reduction steps; the lanes of a warp take
-// 32 neighbouring columns of one source row, which is free of bank conflicts on both sides.
-__device__ __forceinline__ void transpose_split(const uint8_t* src, uint8_t* hi, uint8_t* lo, int nslabs, int t, int threads) {
-    for (int item = t; item < nslabs * 256; item += threads) {
-        const int mn = item & 31, kq = (item >> 5) & 7, sl = item >> 8;
-        const uint8_t* s0 = src + sl * 4096 + ((mn & 3) << 2);
+// 32 neighbouring columns of one source row, which is free of bank conflicts on both sides.  256 threads
+// cooperate: thread t always has column t % 32 and reduction steps 4 * (t / 32) .. + 3 of whatever slab it works
+// on, so its source and destination offsets inside a slab are computed once.
+struct TsplitLane { uint32_t s[4], d; };
+__device__ __forceinline__ TsplitLane tsplit_lane(int t) {
+    const int mn = t & 31, kq = (t >> 5) & 7;
+    TsplitLane l;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int k = kq * 4 + j;
+        l.s[j] = (uint32_t)(((mn & 3) << 2) + k * 128 + (((mn >> 2) ^ (k & 7)) << 4));
+    }
+    l.d = (uint32_t)(mn * 128 + ((kq ^ (mn & 7)) << 4));
+    return l;
+}
+__device__ __forceinline__ void transpose_split256(const uint8_t* src, uint8_t* hi, uint8_t* lo, int nslabs, const TsplitLane& l) {
+#pragma unroll 2
+    for (int sl = 0; sl < nslabs; ++sl) {
+        const uint8_t* s0 = src + sl * 4096;
         float v[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int k = kq * 4 + j;
-            v[j] = *reinterpret_cast<const float*>(s0 + k * 128 + ((((mn >> 2) ^ (k & 7))) << 4));
-        }
-        float4 h, l;
-        h.x = __uint_as_float(__float_as_uint(v[0]) & 0xffffe000u); l.x = v[0] - h.x;
-        h.y = __uint_as_float(__float_as_uint(v[1]) & 0xffffe000u); l.y = v[1] - h.y;
-        h.z = __uint_as_float(__float_as_uint(v[2]) & 0xffffe000u); l.z = v[2] - h.z;
-        h.w = __uint_as_float(__float_as_uint(v[3]) & 0xffffe000u); l.w = v[3] - h.w;
-        const int row = sl * 32 + mn;
-        const int off = row * 128 + ((kq ^ (row & 7)) << 4);
+        for (int j = 0; j < 4; ++j) v[j] = *reinterpret_cast<const float*>(s0 + l.s[j]);
+        float4 h, q;
+        h.x = __uint_as_float(__float_as_uint(v[0]) & 0xffffe000u); q.x = v[0] - h.x;
+        h.y = __uint_as_float(__float_as_uint(v[1]) & 0xffffe000u); q.y = v[1] - h.y;
+        h.z = __uint_as_float(__float_as_uint(v[2]) & 0xffffe000u); q.z = v[2] - h.z;
+        h.w = __uint_as_float(__float_as_uint(v[3]) & 0xffffe000u); q.w = v[3] - h.w;
+        const uint32_t off = sl * 4096 + l.d;
         *reinterpret_cast<float4*>(hi + off) = h;
-        *reinterpret_cast<float4*>(lo + off) = l;
+        *reinterpret_cast<float4*>(lo + off) = q;
     }
 }
 
@@ -249,8 +259,12 @@ template <int BN> struct Wg32Smem {
     static constexpr int TOTAL = NOP * (int)OP_BYTES + NSRC * (int)SRC_BYTES + 1024;
 };
 
+// The conversion is the long pole of this kernel, so eight warps share it (two per scheduler hide each other's
+// shared-memory latency); four of them go on to the epilogue.
+constexpr int WG32_CONV = 256, WG32_THREADS = 64 + WG32_CONV;
+
 template <int BN>
-__global__ void __launch_bounds__(TC_THREADS) tc32_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+__global__ void __launch_bounds__(WG32_THREADS) tc32_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                                                                 const __grid_constant__ CUtensorMap mapD, const T32Params p) {
     using L = Wg32Smem<BN>;
     constexpr uint32_t A_BYTES = L::A_BYTES, B_BYTES = L::B_BYTES, SRC_BYTES = L::SRC_BYTES, OP_BYTES = L::OP_BYTES, SLAB = 32 * 32 * 4;
@@ -273,8 +287,8 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_wgrad_kernel(const __grid_con
 
     if (threadIdx.x == 0) {
         tma_prefetch_map(&mapX); tma_prefetch_map(&mapY); tma_prefetch_map(&mapD);
-        for (int s = 0; s < NSRC; ++s) { mbar_init(sfull0 + 8 * s, 1); mbar_init(sempty0 + 8 * s, 128); }
-        for (int s = 0; s < NOP; ++s) { mbar_init(ready0 + 8 * s, 128); mbar_init(oempty0 + 8 * s, 1); }
+        for (int s = 0; s < NSRC; ++s) { mbar_init(sfull0 + 8 * s, 1); mbar_init(sempty0 + 8 * s, WG32_CONV); }
+        for (int s = 0; s < NOP; ++s) { mbar_init(ready0 + 8 * s, WG32_CONV); mbar_init(oempty0 + 8 * s, 1); }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -326,14 +340,16 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_wgrad_kernel(const __grid_con
         }
     } else {
         const int t = threadIdx.x - 64;
+        static_assert(WG32_CONV == 256, "transpose_split256 assumes 256 converter threads");
+        const TsplitLane lane_off = tsplit_lane(t);
         bool ok = true;
         if (slabsA < TC_BM / 32 || slabsB < BN / 32) {
             // clear the rows of the hi / lo tiles that no slab will ever fill
             const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int s = 0; s < NOP; ++s) {
                 uint8_t* st = smem + s * OP_BYTES;
-                for (int i = slabsA * SLAB + t * 16; i < (int)A_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + i) = z; *reinterpret_cast<float4*>(st + A_BYTES + i) = z; }
-                for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += 128 * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
+                for (int i = slabsA * SLAB + t * 16; i < (int)A_BYTES; i += WG32_CONV * 16) { *reinterpret_cast<float4*>(st + i) = z; *reinterpret_cast<float4*>(st + A_BYTES + i) = z; }
+                for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += WG32_CONV * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
             }
         }
         for (int kb = 0; kb < num_kb && ok; ++kb) {
@@ -343,14 +359,16 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_wgrad_kernel(const __grid_con
             if (!ok) break;
             const uint8_t* src = srcs + ss * SRC_BYTES;
             uint8_t* st = smem + os * OP_BYTES;
-            transpose_split(src, st, st + A_BYTES, slabsA, t, 128);
-            transpose_split(src + A_BYTES, st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, t, 128);
+            transpose_split256(src, st, st + A_BYTES, slabsA, lane_off);
+            transpose_split256(src + A_BYTES, st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, lane_off);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
             mbar_arrive(ready0 + 8 * os);
             mbar_arrive(sempty0 + 8 * ss);                                      // the loader may refill the source buffer
         }
-        const bool have = ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true);
-        epilogue32<BN>(smem, tmem, &mapD, p, nullptr, m0, n0, split, num_kb, have);
+        if (warp < 6) {                                                         // warps 2..5 own the four lane quarters of tensor memory
+            const bool have = ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true);
+            epilogue32<BN>(smem, tmem, &mapD, p, nullptr, m0, n0, split, num_kb, have);
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -396,7 +414,7 @@ bool launch32_wgrad(const CUtensorMap& mx, const CUtensorMap& my, const CUtensor
     constexpr int smem = Wg32Smem<BN>::TOTAL;
     static_assert(Wg32Smem<BN>::NSRC >= 2 && Wg32Smem<BN>::NOP * (int)Wg32Smem<BN>::OP_BYTES >= TC_BM * BN * 4, "shared-memory plan");
     if (cudaFuncSetAttribute(tc32_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    launch(tc32_wgrad_kernel<BN>, grid, dim3(TC_THREADS), smem, st, mx, my, md, p);
+    launch(tc32_wgrad_kernel<BN>, grid, dim3(WG32_THREADS), smem, st, mx, my, md, p);
     return true;
 }
 
