@@ -3,6 +3,7 @@
 // Every tensor is read and written with 16-byte accesses along the channel axis; every
 // reduction runs in a fixed order (per-thread run, shared-memory column sum, then a second pass
 // over the per-block partials) so results do not depend on scheduling.
+#include <algorithm>
 #include <cfloat>
 #include <cstdlib>
 #include <cstring>
@@ -631,6 +632,83 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, 
     }
 }
 
+// Stride-1 depthwise weight gradient (padding 1) on strips of four neighbouring outputs, as dw_strip_kernel: a
+// thread loads the four output gradients and the 3 x 6 inputs of a strip once and feeds all nine taps from them;
+// it walks strips blockIdx.x * 32 + slot, + gridDim.x * 32, ... with its nine accumulators in registers, and the
+// 32 strip slots of the block are added in slot order through shared memory.  partial[blockIdx.x][9][C] (float).
+template <typename T, int V>
+__global__ void __launch_bounds__(256) dw_wgrad_strip_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, int N, int H,
+                                                             int W, int C) {
+    grid_dep_sync();
+    __shared__ float sh[3][32][8 * V];
+    const int CV = C / V, cvl = threadIdx.x & 7, cv = blockIdx.y * 8 + cvl, slot = threadIdx.x >> 3;
+    const int c = cv * V;
+    const int strips_w = (W + 3) >> 2;
+    const long long strips = (long long)N * H * strips_w;
+    float acc[9][V];
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
+    if (cv < CV) {
+        for (long long s = (long long)blockIdx.x * 32 + slot; s < strips; s += (long long)gridDim.x * 32) {
+            const int w0 = (int)(s % strips_w) * 4;
+            const long long R = s / strips_w;
+            const int h = (int)(R % H);
+            float d[4][V];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (w0 + j < W) ldv<V>(dy + ((R * W) + w0 + j) * (long long)C + c, d[j]);
+                else {
+#pragma unroll
+                    for (int e = 0; e < V; ++e) d[j][e] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int rr = 0; rr < 3; ++rr) {
+                const int hi = h - 1 + rr;
+                if (hi < 0 || hi >= H) continue;
+                const T* row = x + ((R - h + hi) * W) * (long long)C + c;
+                float in[6][V];
+#pragma unroll
+                for (int j = 0; j < 6; ++j) {
+                    const int wi = w0 - 1 + j;
+                    if (wi >= 0 && wi < W) ldv<V>(row + (long long)wi * C, in[j]);
+                    else {
+#pragma unroll
+                        for (int e = 0; e < V; ++e) in[j][e] = 0.f;
+                    }
+                }
+#pragma unroll
+                for (int ss = 0; ss < 3; ++ss)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int e = 0; e < V; ++e) acc[rr * 3 + ss][e] = fmaf(in[j + ss][e], d[j][e], acc[rr * 3 + ss][e]);
+            }
+        }
+    }
+#pragma unroll
+    for (int gq = 0; gq < 3; ++gq) {
+        __syncthreads();
+#pragma unroll
+        for (int t = 0; t < 3; ++t)
+#pragma unroll
+            for (int e = 0; e < V; ++e) sh[t][slot][cvl * V + e] = acc[gq * 3 + t][e];
+        __syncthreads();
+        for (int q = threadIdx.x; q < 3 * 8 * V; q += 256) {
+            const int t = q / (8 * V), cc = q % (8 * V);
+            const int gc = blockIdx.y * 8 * V + cc;
+            if (gc < C) {
+                float sum = 0.f;
+#pragma unroll 8
+                for (int y = 0; y < 32; ++y) sum += sh[t][y][cc];
+                partial[((long long)blockIdx.x * 9 + gq * 3 + t) * C + gc] = sum;
+            }
+        }
+    }
+}
+
 // dw[t][c] = sum over chunks and folded copies of partial[chunk][t][copy * C + c]; grid (ceil(C/32), G, 9)
 __global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols, float* __restrict__ dw,
                                          const FinScratch fin) {
@@ -1040,15 +1118,36 @@ static FoldPlan plan_dw_wgrad(const ConvGeom& g, int elem_bytes) {
     return make_fold((long long)g.N * g.Ho * g.Wo, g.Cin, elem_bytes);
 }
 
+// strip kernel: number of blocks along the strips (each block walks strips with that stride)
+static inline int dw_wgrad_strip_blocks(const ConvGeom& g, int V) {
+    const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
+    const int cgroups = (g.Cin / V + 7) / 8;
+    long long gx = (6LL * sm_count() + cgroups - 1) / cgroups;
+    const long long most = (strips + 31) / 32;
+    if (gx > most) gx = most;
+    return (int)(gx < 1 ? 1 : gx);
+}
+
 size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
     const FoldPlan a = plan_dw_wgrad(g, 4), b = plan_dw_wgrad(g, 2);
-    const size_t na = (size_t)a.chunks * 9 * a.cols, nb = (size_t)b.chunks * 9 * b.cols;
-    return na > nb ? na : nb;
+    size_t n = std::max((size_t)a.chunks * 9 * a.cols, (size_t)b.chunks * 9 * b.cols);
+    if (g.Cin % 4 == 0) n = std::max(n, (size_t)dw_wgrad_strip_blocks(g, 4) * 9 * g.Cin);
+    if (g.Cin % 8 == 0) n = std::max(n, (size_t)dw_wgrad_strip_blocks(g, 8) * 9 * g.Cin);
+    return n;
 }
 
 template <typename T>
 void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
+    // (float tensors only: with eight bf16 channels per thread the nine accumulators leave too few warps per SM)
+    if (sizeof(T) == 4 && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy)) {
+        const int gx = dw_wgrad_strip_blocks(g, V);
+        launch(dw_wgrad_strip_kernel<T, V>, dim3(gx, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
+        int slices = gx / (4 * FIN_Y);
+        slices = slices < 1 ? 1 : (slices > FIN_GMAX ? FIN_GMAX : slices);
+        launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, slices, 9), dim3(FIN_X, FIN_Y), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw, fin);
+        return;
+    }
     FoldPlan fp = plan_dw_wgrad(g, (int)sizeof(T));
     const int rpc = fold_rpc(fp);
     if (fp.vec == V && aligned16(x) && aligned16(dy))
