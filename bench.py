@@ -54,6 +54,32 @@ def workload(name, batch=None):
 
 FALLBACK_BF16_TFLOPS = 1400.0            # sustained figure of the fallback measurement
 
+# Whole-step algorithmic work per sample: bytes of every tensor pass of the separate conv / BN forward / BN backward /
+# data-gradient / weight-gradient kernels counted once ((3 I + 11 O) elements per op), and dense + depthwise flops
+# (backward counted as twice the forward).  Keys: workload name -> (bytes per sample, flop per sample).
+STEP_WORK = {"cfg2": (11.73e9 / 128, (63.1e9 + 4.5e9) / 128), "cfg3": (12.00e9 / 64, (107.5e9 + 8.0e9) / 64),
+             "cfg5": (12.00e9 / 64, (107.5e9 + 8.0e9) / 64), "cfg4": (1.84e9 / 256, 481.1e9 / 256), "cfg1": (10e6 / 32, 1.08e9 / 32)}
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of all launches of a kernel class in one step, from one ncu
+# pass (profiles/ncu_tc32_kernels_cfg2_b128.md).  Valid only for the default batch and while the kernel source is the
+# one the counters were taken on: the entry carries the sha256 of that source file.
+NCU_TRAFFIC = {("cfg2", "tc_gemm_tf32x3_wgrad"): dict(bytes_per_step=1.038e9, source="paper_2110_02781_b200/csrc/gemm_tc32.cu",
+                                                     sha256="05a5819bd7ddc8f56e2b30af64a77cba0becc68bacda04293daf7a6e1b390be8")}
+
+
+def ncu_traffic(wl_key, kernel, default_batch):
+    e = NCU_TRAFFIC.get((wl_key, kernel))
+    if not e or not default_batch:
+        return None
+    import hashlib
+    try:
+        with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), e["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != e["sha256"]:
+                return None
+    except OSError:
+        return None
+    return e["bytes_per_step"]
+
 
 def peaks():
     """(HBM GB/s, bf16 tensor TFLOP/s sustained, source).  The sustained tensor figure applies: kernels are timed inside a long step."""
@@ -220,10 +246,9 @@ def main():
 
     assert args.warmup >= 3, "at least 3 warm-up steps"
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2110_02781_b200.replicas import Replicas
+    reps = Replicas("nccl", torch.device("cuda", local_rank))
+    dist = reps.dist
 
     ls, cfg = wl["layers"], wl["cfg"]
     m = F.Model(ls, cfg, f"cuda:{local_rank}")
@@ -247,8 +272,7 @@ def main():
     m.ftp_set_partition(points)
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
+        reps.barrier()
         torch.cuda.synchronize()
 
     def timed(fn, steps):
@@ -259,12 +283,7 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return reps.max_over_ranks(e0.elapsed_time(e1))
 
     step_eager = lambda: m.ftp_train_step(xd, yd, lr, inputs_on_host=False, want_loss=False)
     step_dev = step_eager
@@ -291,7 +310,10 @@ def main():
     with ClockSampler(local_rank) as clk:
         if dynamic:
             lt = (fwd_s + bwd_s).tolist()
+            barrier()
             ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, args.steps, False)
+            barrier()
+            ms = reps.max_over_ranks(ms)
             tick = lambda i, p: (i + 1) % p == 0
             plain = [t for i, t in enumerate(per_it) if not tick(i, dynamic["snapshot"]) and not tick(i, dynamic["repartition"])]
             snap = [t for i, t in enumerate(per_it) if tick(i, dynamic["snapshot"]) and not tick(i, dynamic["repartition"])]
@@ -315,13 +337,16 @@ def main():
     if dynamic:
         e2e_steps = max(dynamic["repartition"] * 2, args.steps // 5)
         m.ftp_set_partition(points)
+        barrier()
         ms_e2e, _, _ = run_dynamic(m, F, wl, (fwd_s + bwd_s).tolist(), xd, yd, xh, yh, lr, e2e_steps, True)
+        barrier()
+        ms_e2e = reps.max_over_ranks(ms_e2e)
         m.ftp_set_partition(points)
     else:
         ms_e2e = timed(step_e2e, args.steps)
     batch = cfg["batch"]
-    value = world * batch * args.steps / (ms * 1e-3)
-    e2e = world * batch * e2e_steps / (ms_e2e * 1e-3)
+    value = reps.job_throughput(batch * args.steps, ms)
+    e2e = reps.job_throughput(batch * e2e_steps, ms_e2e)
 
     # per-kernel roofline: one more step with every launch bracketed by events
     m.ftp_trace_enable(True)
@@ -354,9 +379,17 @@ def main():
                 "frac": d["frac_math"] if math_bound else d["frac_hbm"],
                 "peak_source": ((f"{peak_src} bf16 matmul, sustained" if tensor else "derived: 2 x 128 lanes x 148 SMs x 1.965 GHz")
                                 if math_bound else f"{peak_src} HBM copy"),
-                "traffic": None, "share_of_step": d["share"],
+                "traffic": ncu_traffic(args.workload, dom, args.batch is None), "share_of_step": d["share"],
                 "note": "achieved = algorithmic bytes (or flops) of all launches of the kernel in a step / their CUDA-event time",
                 "kernels": table}
+    sw = STEP_WORK.get(args.workload)
+    if sw:
+        step_s = ms / args.steps * 1e-3
+        gbs = sw[0] * batch / step_s / 1e9
+        tfs = sw[1] * batch / step_s / 1e12
+        roofline["step"] = {"algorithmic_GB": round(sw[0] * batch / 1e9, 3), "GB/s": round(gbs, 1), "frac_hbm": round(gbs / hbm_peak, 3),
+                            "TFLOP/s": round(tfs, 2), "frac_tensor": round(tfs / tensor_peak, 3) if bf16 else None,
+                            "note": "whole step: algorithmic bytes (flops) of all kernels / device time of the timed steps"}
 
     out = {"metric": "training samples/sec per partitioned step", "value": value, "unit": "samples/s", "n_gpus": world,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -378,8 +411,7 @@ def main():
         out["cpu_baseline"] = run_reference(a2, wl)["cpu_baseline"]
     if rank == 0:
         print(json.dumps(out), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    reps.close()
     return 0
 
 

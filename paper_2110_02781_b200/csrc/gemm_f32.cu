@@ -1,8 +1,8 @@
 // SIMT contractions: dense convolution (incl. 1x1 / FC / conv1d) forward, data gradient and
-// weight gradient as implicit GEMMs with float accumulation.  The fp32 path has to stay within 1e-4
-// of a float64 reference, which rules tensor cores (tf32 / bf16 inputs) out for it.  The same kernels
-// are instantiated for bfloat16 tensors: they serve the shapes the tensor-core kernels do not take
-// (3 input channels, ragged channel counts).
+// weight gradient as implicit GEMMs with float accumulation.  They serve the shapes the tensor-core
+// kernels (split-tf32 for float tensors, bf16) do not take: spatial kernels of float models, 3 input
+// channels, ragged channel counts, bias or activation fused into the convolution, the classifier.
+// Instantiated for float and for bfloat16 tensors.
 //
 // Tiling: 256 threads compute a 128 x BN tile of the output with an 8 x (BN/16) register
 // micro-tile per thread; the reduction dimension is walked 16 at a time through two
