@@ -144,7 +144,8 @@ constexpr int FIN_GMAX = 16;
 template <typename PT, int NS>
 __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int ns, int chunks, int f, int C, int cols, int c,
                                               const FinScratch fin, double (&out)[NS]) {
-    __shared__ double red[NS][FIN_Y][FIN_X + 1];
+    static_assert(FIN_X == 8 && FIN_Y == 128, "the reduction below is written for 8 x 128 threads");
+    __shared__ double red[NS][FIN_X * FIN_Y / 32][FIN_X];
     __shared__ unsigned ticket;
     double t[NS];
 #pragma unroll
@@ -164,18 +165,31 @@ __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int 
 #pragma unroll
         for (int a = 0; a < NS; ++a) t[a] += (v[a][0] + v[a][1]) + (v[a][2] + v[a][3]);
     }
+    // fixed-shape sum over y: the four y of a warp by shuffles, the 32 warps through shared memory (eight per lane
+    // group of the first warp, in order), the four lane groups by shuffles again
+    const int lane = (threadIdx.y * FIN_X + threadIdx.x) & 31, warp = (threadIdx.y * FIN_X + threadIdx.x) >> 5;
 #pragma unroll
-    for (int a = 0; a < NS; ++a) red[a][threadIdx.y][threadIdx.x] = t[a];
-    __syncthreads();
-#pragma unroll 1
-    for (int s = FIN_Y / 2; s >= 1; s >>= 1) {           // fixed-shape tree over y
-        if ((int)threadIdx.y < s)
-#pragma unroll
-            for (int a = 0; a < NS; ++a) red[a][threadIdx.y][threadIdx.x] += red[a][threadIdx.y + s][threadIdx.x];
-        __syncthreads();
+    for (int a = 0; a < NS; ++a) {
+        double v = t[a];
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        if (lane < FIN_X) red[a][warp][lane] = v;
     }
+    __syncthreads();
 #pragma unroll
-    for (int a = 0; a < NS; ++a) out[a] = red[a][0][threadIdx.x];
+    for (int a = 0; a < NS; ++a) out[a] = 0.0;
+    if (warp == 0) {
+        const int x = lane & (FIN_X - 1), q = lane >> 3;
+#pragma unroll
+        for (int a = 0; a < NS; ++a) {
+            double v = 0.0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) v += red[a][q * 8 + w][x];
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            out[a] = v;
+        }
+    }
     if (G == 1) return true;
     const int slot = blockIdx.z * gridDim.x + blockIdx.x;
     double* mine = fin.part + ((long long)slot * FIN_GMAX + blockIdx.y) * NS * FIN_X;
@@ -211,30 +225,40 @@ __global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, 
     });
 }
 
-__global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
+// 1 / sqrt(v) in double from the float estimate and two Newton steps (the divide-and-root sequence is several
+// hundred cycles of dependent fp64 work on a kernel that is nothing but latency)
+__device__ __forceinline__ double rsqrt_f64(double v) {
+    double r = (double)rsqrtf((float)v);
+    r = r * (1.5 - 0.5 * v * r * r);
+    r = r * (1.5 - 0.5 * v * r * r);
+    return r;
+}
+
+__global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M, double inv_M, double unbias,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
                                    float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd,
                                    const FinScratch fin) {
     grid_dep_sync();
     const int c = blockIdx.x * FIN_X + threadIdx.x;
+    float ga = 0.f, be = 0.f, rm = 0.f, rv = 0.f;                    // fetched up front: their latency hides behind the sums
+    if (threadIdx.y == 0 && c < C) { ga = gamma[c]; be = beta[c]; rm = run_mean[c]; rv = run_var[c]; }
     double ss[2];
     if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
     if (threadIdx.y == 0 && c < C) {
-        const double mu = s1 / M;
-        double var = s2 / M - mu * mu;
+        const double mu = s1 * inv_M;
+        double var = s2 * inv_M - mu * mu;
         if (var < 0.0) var = 0.0;
-        const double rs = 1.0 / sqrt(var + (double)eps);
-        const float sc = (float)((double)gamma[c] * rs);
+        const double rs = rsqrt_f64(var + (double)eps);
+        const float sc = (float)((double)ga * rs);
         scale[c] = sc;
-        shift[c] = beta[c];                       // z = (y - mean) * scale + beta, the mean kept as a two-float sum
+        shift[c] = be;                            // z = (y - mean) * scale + beta, the mean kept as a two-float sum
         const float mh = (float)mu;
         mean[c] = mh;
         mean_lo[c] = (float)(mu - (double)mh);
         rstd[c] = (float)rs;
-        const double unb = M > 1.0 ? var * M / (M - 1.0) : var;
-        run_mean[c] = (float)((1.0 - (double)mom) * (double)run_mean[c] + (double)mom * mu);
-        run_var[c] = (float)((1.0 - (double)mom) * (double)run_var[c] + (double)mom * unb);
+        run_mean[c] = (float)((1.0 - (double)mom) * (double)rm + (double)mom * mu);
+        run_var[c] = (float)((1.0 - (double)mom) * (double)rv + (double)mom * (var * unbias));
     }
 }
 
@@ -291,19 +315,21 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
     });
 }
 
-__global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M,
+__global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double inv_M,
                                        const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
                                        float* dbeta, float* coef, const FinScratch fin) {
     grid_dep_sync();
     const int c = blockIdx.x * FIN_X + threadIdx.x;
+    float ga = 0.f, rs = 0.f;
+    if (threadIdx.y == 0 && c < C) { ga = gamma[c]; rs = rstd[c]; }
     double ss[2];
     if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
     if (threadIdx.y == 0 && c < C) {
         dbeta[c] = (float)s1;
         dgamma[c] = (float)s2;
-        coef[c] = gamma[c] * rstd[c];
-        const double b = s1 / M, cc = s2 / M;      // kept as two-float sums: they are subtracted from values of their own size
+        coef[c] = ga * rs;
+        const double b = s1 * inv_M, cc = s2 * inv_M;      // kept as two-float sums: they are subtracted from values of their own size
         const float bh = (float)b, ch = (float)cc;
         coef[C + c] = bh; coef[2 * C + c] = (float)(b - (double)bh);
         coef[3 * C + c] = ch; coef[4 * C + c] = (float)(cc - (double)ch);
@@ -1015,7 +1041,8 @@ void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partia
 void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
                  float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st) {
-    launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, beta, eps, momentum,
+    launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, (double)M, 1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0,
+           gamma, beta, eps, momentum,
                                                              run_mean, run_var, scale, shift, mean, mean_lo, rstd, fin);
 }
 
@@ -1043,7 +1070,7 @@ void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& 
 
 void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
                      float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st) {
-    launch(bn_bwd_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
+    launch(bn_bwd_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, 1.0 / (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
 }
 
 template <typename T>
