@@ -48,6 +48,10 @@ template <int V> __device__ __forceinline__ void ldv(const __nv_bfloat16* p, flo
         const unsigned u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(u[i] << 16); o[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
+    } else if constexpr (V == 4) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+        o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+        o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
     } else { o[0] = __bfloat162float(*p); }
 }
 template <int V> __device__ __forceinline__ void stv(float* p, const float (&v)[V]) {
@@ -63,6 +67,9 @@ template <int V> __device__ __forceinline__ void stv(__nv_bfloat16* p, const flo
             u[i] = *reinterpret_cast<const unsigned*>(&h);
         }
         *reinterpret_cast<uint4*>(p) = make_uint4(u[0], u[1], u[2], u[3]);
+    } else if constexpr (V == 4) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+        *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const unsigned*>(&a), *reinterpret_cast<const unsigned*>(&b));
     } else { p[0] = __float2bfloat16_rn(v[0]); }
 }
 // V consecutive floats of a per-channel table (V is 1, 4 or 8; the address is 16-byte aligned for V >= 4)
@@ -1030,6 +1037,8 @@ static inline int fin_slices(const FoldPlan& fp) {
 
 static inline int fold_rpc(const FoldPlan& fp) { return (fp.rows + fp.chunks - 1) / fp.chunks; }
 static inline dim3 fold_grid(const FoldPlan& fp) { return dim3((fp.cols + 32 * fp.vec - 1) / (32 * fp.vec), fp.chunks); }
+// the same row chunks walked with w columns per thread (w divides fp.vec)
+static inline dim3 fold_grid_w(const FoldPlan& fp, int w) { return dim3((fp.cols + 32 * w - 1) / (32 * w), fp.chunks); }
 
 template <typename T>
 void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st) {
@@ -1060,8 +1069,9 @@ template <typename T>
 void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
                    const float* mean, const float* mean_lo, const float* rstd, int act, double* partial, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
+    constexpr int W = 4;      // columns per thread: four keep the per-channel constants of a thread at a register count that leaves four blocks per SM
     if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd))
-        launch(bn_bwd_reduce_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial);
+        launch(bn_bwd_reduce_kernel<T, W>, dim3(fold_grid_w(fp, W)), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial);
     else {
         FoldPlan s = fp;                       // scalar fallback keeps the same partial layout
         launch(bn_bwd_reduce_kernel<T, 1>, dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st, dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, mean_lo, rstd, act, partial);
@@ -1077,9 +1087,10 @@ template <typename T>
 void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
                   const float* mean, const float* mean_lo, const float* rstd, const float* coef, int act, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
+    constexpr int W = 4;      // columns per thread: four keep the per-channel constants of a thread at a register count that leaves four blocks per SM
     if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(addend) && aligned16(dy) && aligned16(scale) && aligned16(shift) && aligned16(mean) &&
         aligned16(mean_lo) && aligned16(rstd) && aligned16(coef))
-        launch(bn_bwd_apply_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
+        launch(bn_bwd_apply_kernel<T, W>, dim3(fold_grid_w(fp, W)), dim3(32, 8), 0, st, dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
     else
         launch(bn_bwd_apply_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, dz, y, addend, dy, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, coef, act);
 }
