@@ -1131,7 +1131,8 @@ void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_
     const unsigned tiles = (unsigned)(((g.Wo + (1 << tws) - 1) >> tws) * (((long long)g.N * g.Ho + (64 >> tws) - 1) / (64 >> tws)));
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w)) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
-        launch(dw_strip_kernel<T, V, 0>, dim3((unsigned)((strips + 31) / 32), (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin);
+        // four channels per thread for either type: eight lanes of a block then cover 32 channels, which every layer has
+        launch(dw_strip_kernel<T, 4, 0>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin);
         return;
     }
     if (can_vec<T>(g.Cin, x, y) && aligned16(w)) launch(dw_fwd_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
@@ -1145,7 +1146,7 @@ void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const Con
     const unsigned tiles = (unsigned)(((g.W + (1 << tws) - 1) >> tws) * (((long long)g.N * g.H + (64 >> tws) - 1) / (64 >> tws)));
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
-        launch(dw_strip_kernel<T, V, 1>, dim3((unsigned)((strips + 31) / 32), (g.Cin / V + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin);
+        launch(dw_strip_kernel<T, 4, 1>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin);
         return;
     }
     if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) launch(dw_dgrad_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
@@ -1177,10 +1178,11 @@ size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
 template <typename T>
 void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
-    // (float tensors only: with eight bf16 channels per thread the nine accumulators leave too few warps per SM)
-    if (sizeof(T) == 4 && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy)) {
-        const int gx = dw_wgrad_strip_blocks(g, V);
-        launch(dw_wgrad_strip_kernel<T, V>, dim3(gx, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
+    // four channels per thread for either type: with eight bf16 channels the nine accumulators would leave too few warps per SM
+    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy)) {
+        constexpr int SV = 4;
+        const int gx = dw_wgrad_strip_blocks(g, SV);
+        launch(dw_wgrad_strip_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
         int slices = gx / (4 * FIN_Y);
         slices = slices < 1 ? 1 : (slices > FIN_GMAX ? FIN_GMAX : slices);
         launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, slices, 9), dim3(FIN_X, FIN_Y), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw, fin);
