@@ -7,6 +7,8 @@ import importlib
 
 
 def __getattr__(name):
+    if name in ("build", "replicas"):                      # plain submodules: never need the library
+        return importlib.import_module("." + name, __name__)
     ft = importlib.import_module(".ftpipe", __name__)      # raises if libftpipe.so is missing: there is no fallback
     try:
         return getattr(ft, name)
