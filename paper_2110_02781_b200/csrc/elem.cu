@@ -7,6 +7,7 @@
 #include <cfloat>
 #include <cstdlib>
 #include <cstring>
+#include <initializer_list>
 #include "kernels.h"
 #include "launch.cuh"
 
@@ -109,8 +110,10 @@ inline unsigned flat_blocks(long long work, int threads) {
 
 // ---- folded column reductions --------------------------------------------------------------
 // grid (column tiles of 32*V, row chunks); block (32, 8).  NS sums per column.
+// copies > 1 (then copies * C == 32 * V): the copies of a channel inside the column tile are added up as well, in copy
+// order, and the partial sums are laid out [chunk][NS][cols / copies].
 template <typename T, int V, int NS, typename F>
-__device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chunk, double* partial, F body) {
+__device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chunk, double* partial, F body, int C = 0, int copies = 1) {
     __shared__ float sh[NS][8][32 * V];
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     const int r0 = blockIdx.y * rows_per_chunk, r1 = min(rows, r0 + rows_per_chunk);
@@ -126,6 +129,18 @@ __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chu
 #pragma unroll
         for (int e = 0; e < V; ++e) sh[a][threadIdx.y][threadIdx.x * V + e] = s[a][e];
     __syncthreads();
+    if (copies > 1) {
+        const int colsP = cols / copies;
+        for (int q = threadIdx.y * 32 + threadIdx.x; q < NS * C; q += 256) {
+            const int a = q / C, c = q - a * C;
+            double t = 0.0;
+            for (int k = 0; k < copies; ++k)
+#pragma unroll
+                for (int y = 0; y < 8; ++y) t += (double)sh[a][y][k * C + c];
+            partial[((long long)blockIdx.y * NS + a) * colsP + blockIdx.x * C + c] = t;
+        }
+        return;
+    }
     // 256 threads sum the 8 rows of NS * 32 * V columns in a fixed order
     for (int q = threadIdx.y * 32 + threadIdx.x; q < NS * 32 * V; q += 256) {
         const int a = q / (32 * V), c = q % (32 * V);
@@ -222,14 +237,35 @@ __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int 
 }
 
 template <typename T, int V>
-__global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, int rows, int cols, int rpc, double* __restrict__ partial) {
+__global__ void __launch_bounds__(256) bn_stats_kernel(const T* __restrict__ y, int rows, int cols, int rpc, double* __restrict__ partial, int C, int copies) {
     grid_dep_sync();
     fold_reduce<T, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
         float v[V];
         ldv<V>(y + off, v);
 #pragma unroll
         for (int e = 0; e < V; ++e) { s[0][e] += v[e]; s[1][e] = fmaf(v[e], v[e], s[1][e]); }
-    });
+    }, C, copies);
+}
+
+// Second pass of a product whose reduction was cut into S slices, for an output that feeds a batch norm: adds the
+// slices in slice order, stores the result and reduces its statistics on the way (same layout as bn_stats_kernel).
+template <int V>
+__global__ void __launch_bounds__(256) slice_sum_stats_kernel(const float* __restrict__ part, int S, long long slice_elems, float* __restrict__ out,
+                                                              int rows, int cols, int rpc, double* __restrict__ partial, int C, int copies) {
+    grid_dep_sync();
+    fold_reduce<float, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
+        float a[V];
+        ldv<V>(part + off, a);
+        for (int z = 1; z < S; ++z) {
+            float v[V];
+            ldv<V>(part + (long long)z * slice_elems + off, v);
+#pragma unroll
+            for (int e = 0; e < V; ++e) a[e] += v[e];
+        }
+        stv<V>(out + off, a);
+#pragma unroll
+        for (int e = 0; e < V; ++e) { s[0][e] += a[e]; s[1][e] = fmaf(a[e], a[e], s[1][e]); }
+    }, C, copies);
 }
 
 // 1 / sqrt(v) in double from the float estimate and two Newton steps (the divide-and-root sequence is several
@@ -304,7 +340,7 @@ template <typename T, int V>
 __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict__ dz, const T* __restrict__ y, int rows, int cols, int rpc, int C,
                                                             const float* __restrict__ scale, const float* __restrict__ shift,
                                                             const float* __restrict__ mean, const float* __restrict__ mean_lo,
-                                                            const float* __restrict__ rstd, int act, double* __restrict__ partial) {
+                                                            const float* __restrict__ rstd, int act, double* __restrict__ partial, int copies) {
     grid_dep_sync();
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     float sc[V], sh[V], mu[V], ml[V], rs[V];
@@ -319,7 +355,7 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
             s[0][e] += g;
             s[1][e] = fmaf(g, ((v[e] - mu[e]) - ml[e]) * rs[e], s[1][e]);
         }
-    });
+    }, C, copies);
 }
 
 __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double inv_M,
@@ -488,7 +524,9 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, co
     }
 }
 
-template <typename T, int V>
+// STRIDE is a compile-time 1 or 2 (0: read g.stride): the gather divides by it once per tap, and a division by a
+// run-time value costs more than the tap's multiply-adds.
+template <typename T, int V, int STRIDE>
 __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy, const float* __restrict__ w, const T* __restrict__ addend,
                                                        T* __restrict__ dx, ConvGeom g, int tws) {
     grid_dep_sync();
@@ -502,6 +540,7 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
     const int wi = tw_i * TW + (slot & (TW - 1));
     if (wi >= g.W) return;
     const int rows = g.N * g.H;
+    const int stride = STRIDE > 0 ? STRIDE : g.stride;
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
         const int R = tr_i * 2 * half + (slot >> tws) + k * half;
@@ -515,14 +554,14 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
         for (int r = 0; r < 3; ++r) {
             const int th = hi + g.ph - r;
             if (th < 0) continue;
-            const int ho = th / g.stride;
-            if (ho * g.stride != th || ho >= g.Ho) continue;
+            const int ho = th / stride;
+            if (ho * stride != th || ho >= g.Ho) continue;
 #pragma unroll
             for (int s = 0; s < 3; ++s) {
                 const int tw = wi + g.pw - s;
                 if (tw < 0) continue;
-                const int wo = tw / g.stride;
-                if (wo * g.stride != tw || wo >= g.Wo) continue;
+                const int wo = tw / stride;
+                if (wo * stride != tw || wo >= g.Wo) continue;
                 float v[V], k[V];
                 ldv<V>(dy + ((long long)(n * g.Ho + ho) * g.Wo + wo) * g.Cin + c, v);
                 ldtab<V>(w + (r * 3 + s) * g.Cin + c, k);
@@ -545,17 +584,13 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
 // 3 x 6 inputs they share, so every input vector is loaded once per row of taps instead of three times and
 // the six loads of a row are in flight together.  Block: 8 channel vectors x 32 strips; strips are numbered
 // row-major over (image, row, strip of 4 columns).
-template <typename T, int V, int FLIP>
-__global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, const float* __restrict__ w, const T* __restrict__ addend,
-                                                       T* __restrict__ y, int N, int H, int W, int C) {
-    grid_dep_sync();
-    const int CV = C / V;
-    const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
-    if (cv >= CV) return;
-    const int c = cv * V;
-    const int strips_w = (W + 3) >> 2;
-    const long long strip = (long long)blockIdx.x * 32 + (threadIdx.x >> 3);
-    if (strip >= (long long)N * H * strips_w) return;
+template <typename T> __device__ __forceinline__ float as_stored(float v);
+template <> __device__ __forceinline__ float as_stored<float>(float v) { return v; }
+template <> __device__ __forceinline__ float as_stored<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+template <typename T, int V, int FLIP, bool STATS>
+__device__ __forceinline__ void dw_strip_body(const T* __restrict__ x, const float* __restrict__ w, const T* __restrict__ addend, T* __restrict__ y,
+                                              int H, int W, int C, int c, long long strip, int strips_w, float (&su)[V], float (&sq)[V]) {
     const int w0 = (int)(strip % strips_w) * 4;
     const long long R = strip / strips_w;                 // image * H + row
     const int h = (int)(R % H);
@@ -600,6 +635,46 @@ __global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, 
             for (int e = 0; e < V; ++e) acc[j][e] += a[e];
         }
         stv<V>(y + o, acc[j]);
+        if constexpr (STATS) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) { const float v = as_stored<T>(acc[j][e]); su[e] += v; sq[e] = fmaf(v, v, sq[e]); }
+        }
+    }
+}
+
+// STATS: the block also leaves the column sums and sums of squares of the values it stored (as stored: rounded to T)
+// in stats[blockIdx.x][2][C], for the batch norm that follows.
+template <typename T, int V, int FLIP, int STATS>
+__global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, const float* __restrict__ w, const T* __restrict__ addend,
+                                                       T* __restrict__ y, int N, int H, int W, int C, double* __restrict__ stats) {
+    grid_dep_sync();
+    const int CV = C / V;
+    const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
+    const int c = cv * V;
+    const int strips_w = (W + 3) >> 2;
+    const long long strip = (long long)blockIdx.x * 32 + (threadIdx.x >> 3);
+    const bool live = cv < CV && strip < (long long)N * H * strips_w;
+    if constexpr (STATS) {
+        __shared__ float shs[2][32][8 * V];
+        float su[V], sq[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) su[e] = sq[e] = 0.f;
+        if (live) dw_strip_body<T, V, FLIP, true>(x, w, addend, y, H, W, C, c, strip, strips_w, su, sq);
+#pragma unroll
+        for (int e = 0; e < V; ++e) { shs[0][threadIdx.x >> 3][(threadIdx.x & 7) * V + e] = su[e]; shs[1][threadIdx.x >> 3][(threadIdx.x & 7) * V + e] = sq[e]; }
+        __syncthreads();
+        if (threadIdx.x < 2 * 8 * V) {
+            const int a = threadIdx.x / (8 * V), ch = threadIdx.x % (8 * V), gc = blockIdx.y * 8 * V + ch;
+            if (gc < C) {
+                double t = 0.0;
+#pragma unroll
+                for (int k = 0; k < 32; ++k) t += (double)shs[a][k][ch];
+                stats[((long long)blockIdx.x * 2 + a) * C + gc] = t;
+            }
+        }
+    } else {
+        float su[V], sq[V];
+        if (live) dw_strip_body<T, V, FLIP, false>(x, w, addend, y, H, W, C, c, strip, strips_w, su, sq);
     }
 }
 
@@ -750,6 +825,32 @@ __global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int 
     double ss[1];
     if (!col_fold_sums<float, 1>(partial, (int)blockIdx.z, 9, chunks, f, C, cols, c, fin, ss)) return;
     if (threadIdx.y == 0 && c < C) dw[blockIdx.z * C + c] = (float)ss[0];
+}
+
+// The same sum when a channel has few partial sums (at most DW_FIN_SMALL): one block of 32 channels x 8 runs per tap
+// instead of 1024-thread blocks per eight channels.  grid (ceil(C/32), 9), block (32, 8); the runs are added in order.
+constexpr int DW_FIN_SMALL = 512;
+__global__ void __launch_bounds__(256) dw_wgrad_finalize_small_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols,
+                                                                      float* __restrict__ dw) {
+    grid_dep_sync();
+    __shared__ double sh[8][32];
+    const int c = blockIdx.x * 32 + threadIdx.x, t = blockIdx.y, total = chunks * f;
+    double a = 0.0;
+    if (c < C) {
+#pragma unroll 4
+        for (int e = threadIdx.y; e < total; e += 8) {
+            const int ch = e / f, k = e - ch * f;
+            a += (double)partial[((long long)ch * 9 + t) * cols + k * C + c];
+        }
+    }
+    sh[threadIdx.y][threadIdx.x] = a;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        double r = 0.0;
+#pragma unroll
+        for (int y = 0; y < 8; ++y) r += sh[y][threadIdx.x];
+        dw[t * C + c] = (float)r;
+    }
 }
 
 // ---- pooling --------------------------------------------------------------------------------------
@@ -1021,9 +1122,21 @@ FoldPlan make_fold(long long M, int C, int elem_bytes) {
     const long long maxc = (fp.rows + 15) / 16;
     if (chunks > maxc) chunks = maxc;
     if (chunks < 1) chunks = 1;
+    // The reducing kernels merge the folded copies that fall inside one column tile.
+    fp.fused = 0; fp.copies_fwd = fp.copies_bwd = 1;
+    if (fp.vec > 1) {
+        auto copies_in = [&](int tile) { return (tile % C == 0) ? std::min(fp.f, tile / C) : 1; };
+        fp.copies_fwd = copies_in(32 * fp.vec); fp.copies_bwd = copies_in(128);
+        fp.fused = 1;
+    }
     const int rpc = (int)((fp.rows + chunks - 1) / chunks);
     fp.chunks = (fp.rows + rpc - 1) / rpc;
     return fp;
+}
+
+static inline int fin_slices_ps(const PartialSums& ps) {
+    const int g = ps.entries / (4 * FIN_Y);
+    return g < 1 ? 1 : (g > FIN_GMAX ? FIN_GMAX : g);
 }
 
 size_t fold_partial_doubles(const FoldPlan& fp) { return (size_t)fp.chunks * 2 * fp.cols; }
@@ -1040,19 +1153,33 @@ static inline dim3 fold_grid(const FoldPlan& fp) { return dim3((fp.cols + 32 * f
 // the same row chunks walked with w columns per thread (w divides fp.vec)
 static inline dim3 fold_grid_w(const FoldPlan& fp, int w) { return dim3((fp.cols + 32 * w - 1) / (32 * w), fp.chunks); }
 
-template <typename T>
-void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st) {
-    constexpr int V = VecOf<T>::N;
-    if (fp.vec == V && aligned16(y)) launch(bn_stats_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, fp.rows, fp.cols, fold_rpc(fp), partial);
-    else launch(bn_stats_kernel<T, 1>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, fp.rows, fp.cols, fold_rpc(fp), partial);
+size_t producer_partial_doubles(long long M, int C) { return (size_t)((M + 127) / 128) * 2 * (size_t)C; }
+
+bool slice_sum_stats(const float* part, int S, float* D, long long M, int C, const FoldPlan& fp, double* partial, PartialSums* out, cudaStream_t st) {
+    if (fp.vec != 4 || !aligned16(part) || !aligned16(D) || (M * C) % 4 != 0) return false;
+    const int copies = fp.fused ? fp.copies_fwd : 1;
+    launch(slice_sum_stats_kernel<4>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, part, S, M * C, D, fp.rows, fp.cols, fold_rpc(fp), partial, C, copies);
+    *out = PartialSums{partial, fp.chunks * (fp.f / copies), fp.f / copies};
+    return true;
 }
 
-void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* beta,
+template <typename T>
+PartialSums bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st) {
+    constexpr int V = VecOf<T>::N;
+    if (fp.vec == V && aligned16(y)) {
+        const int copies = fp.fused ? fp.copies_fwd : 1;
+        launch(bn_stats_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, fp.rows, fp.cols, fold_rpc(fp), partial, C, copies);
+        return PartialSums{partial, fp.chunks * (fp.f / copies), fp.f / copies};
+    }
+    launch(bn_stats_kernel<T, 1>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, y, fp.rows, fp.cols, fold_rpc(fp), partial, C, 1);
+    return PartialSums{partial, fp.chunks * fp.f, fp.f};
+}
+
+void bn_finalize(const PartialSums& ps, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
                  float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st) {
-    launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, (double)M, 1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0,
-           gamma, beta, eps, momentum,
-                                                             run_mean, run_var, scale, shift, mean, mean_lo, rstd, fin);
+    launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp, (double)M,
+           1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0, gamma, beta, eps, momentum, run_mean, run_var, scale, shift, mean, mean_lo, rstd, fin);
 }
 
 template <typename T>
@@ -1066,21 +1193,24 @@ void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const Fol
 }
 
 template <typename T>
-void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
-                   const float* mean, const float* mean_lo, const float* rstd, int act, double* partial, cudaStream_t st) {
+PartialSums bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
+                          const float* mean, const float* mean_lo, const float* rstd, int act, double* partial, cudaStream_t st) {
     constexpr int V = VecOf<T>::N;
     constexpr int W = 4;      // columns per thread: four keep the per-channel constants of a thread at a register count that leaves four blocks per SM
-    if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd))
-        launch(bn_bwd_reduce_kernel<T, W>, dim3(fold_grid_w(fp, W)), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial);
-    else {
-        FoldPlan s = fp;                       // scalar fallback keeps the same partial layout
-        launch(bn_bwd_reduce_kernel<T, 1>, dim3((s.cols + 31) / 32, s.chunks), dim3(32, 8), 0, st, dz, y, s.rows, s.cols, fold_rpc(s), C, scale, shift, mean, mean_lo, rstd, act, partial);
+    if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd)) {
+        const int copies = fp.fused ? fp.copies_bwd : 1;
+        launch(bn_bwd_reduce_kernel<T, W>, dim3(fold_grid_w(fp, W)), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial, copies);
+        return PartialSums{partial, fp.chunks * (fp.f / copies), fp.f / copies};
     }
+    // the scalar fallback keeps the plain partial layout
+    launch(bn_bwd_reduce_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial, 1);
+    return PartialSums{partial, fp.chunks * fp.f, fp.f};
 }
 
-void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma, const float* rstd,
+void bn_bwd_finalize(const PartialSums& ps, long long M, int C, const float* gamma, const float* rstd,
                      float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st) {
-    launch(bn_bwd_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices(fp)), dim3(FIN_X, FIN_Y), 0, st, partial, fp.chunks, fp.f, C, fp.cols, 1.0 / (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
+    launch(bn_bwd_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp,
+           1.0 / (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
 }
 
 template <typename T>
@@ -1125,14 +1255,19 @@ void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int
 static inline int dw_tile_shift(int width) { return width >= 8 ? 3 : width >= 4 ? 2 : width >= 2 ? 1 : 0; }
 
 template <typename T>
-void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st) {
+void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st, const ColStatsReq* stats) {
     constexpr int V = VecOf<T>::N;
     const int tws = dw_tile_shift(g.Wo);
     const unsigned tiles = (unsigned)(((g.Wo + (1 << tws) - 1) >> tws) * (((long long)g.N * g.Ho + (64 >> tws) - 1) / (64 >> tws)));
+    if (stats) stats->out->entries = 0;
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w)) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
+        const dim3 grid((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8);
         // four channels per thread for either type: eight lanes of a block then cover 32 channels, which every layer has
-        launch(dw_strip_kernel<T, 4, 0>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin);
+        if (stats) {
+            launch(dw_strip_kernel<T, 4, 0, 1>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, stats->partial);
+            *stats->out = PartialSums{stats->partial, (int)grid.x, 1};
+        } else launch(dw_strip_kernel<T, 4, 0, 0>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, (double*)nullptr);
         return;
     }
     if (can_vec<T>(g.Cin, x, y) && aligned16(w)) launch(dw_fwd_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
@@ -1146,11 +1281,15 @@ void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const Con
     const unsigned tiles = (unsigned)(((g.W + (1 << tws) - 1) >> tws) * (((long long)g.N * g.H + (64 >> tws) - 1) / (64 >> tws)));
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
-        launch(dw_strip_kernel<T, 4, 1>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin);
+        launch(dw_strip_kernel<T, 4, 1, 0>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin, (double*)nullptr);
         return;
     }
-    if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) launch(dw_dgrad_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
-    else launch(dw_dgrad_kernel<T, 1>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
+    if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
+        const dim3 grid(tiles, (g.Cin / V + 7) / 8);
+        if (g.stride == 2) launch(dw_dgrad_kernel<T, V, 2>, grid, dim3(256), 0, st, dy, w, addend, dx, g, tws);
+        else if (g.stride == 1) launch(dw_dgrad_kernel<T, V, 1>, grid, dim3(256), 0, st, dy, w, addend, dx, g, tws);
+        else launch(dw_dgrad_kernel<T, V, 0>, grid, dim3(256), 0, st, dy, w, addend, dx, g, tws);
+    } else launch(dw_dgrad_kernel<T, 1, 0>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g, tws);
 }
 
 static FoldPlan plan_dw_wgrad(const ConvGeom& g, int elem_bytes) {
@@ -1183,6 +1322,10 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
         constexpr int SV = 4;
         const int gx = dw_wgrad_strip_blocks(g, SV);
         launch(dw_wgrad_strip_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
+        if (gx <= DW_FIN_SMALL) {
+            launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
+            return;
+        }
         int slices = gx / (4 * FIN_Y);
         slices = slices < 1 ? 1 : (slices > FIN_GMAX ? FIN_GMAX : slices);
         launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, slices, 9), dim3(FIN_X, FIN_Y), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw, fin);
@@ -1194,7 +1337,8 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
         launch(dw_wgrad_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
     else
         launch(dw_wgrad_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
-    launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, fin_slices(fp), 9), dim3(FIN_X, FIN_Y), 0, st, scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
+    if (fp.chunks * fp.f <= DW_FIN_SMALL) launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw);
+    else launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, fin_slices(fp), 9), dim3(FIN_X, FIN_Y), 0, st, scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
 }
 
 template <typename T>
@@ -1262,10 +1406,10 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
 }
 
 #define FTP_INSTANTIATE(T)                                                                                              \
-    template void bn_stats<T>(const T*, long long, int, const FoldPlan&, double*, cudaStream_t);                          \
+    template PartialSums bn_stats<T>(const T*, long long, int, const FoldPlan&, double*, cudaStream_t);                          \
     template void bn_apply<T>(const T*, const T*, T*, long long, int, const FoldPlan&, const float*, const float*, const float*, \
                               const float*, int, cudaStream_t);                                                            \
-    template void bn_bwd_reduce<T>(const T*, const T*, long long, int, const FoldPlan&, const float*, const float*,         \
+    template PartialSums bn_bwd_reduce<T>(const T*, const T*, long long, int, const FoldPlan&, const float*, const float*,         \
                                    const float*, const float*, const float*, int, double*, cudaStream_t);                  \
     template void bn_bwd_apply<T>(const T*, const T*, const T*, T*, long long, int, const FoldPlan&, const float*, const float*, \
                                   const float*, const float*, const float*, const float*, int, cudaStream_t);              \
@@ -1273,7 +1417,7 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
                                   const FinScratch&, cudaStream_t);                                                                           \
     template void act_fwd<T>(const T*, T*, long long, int, cudaStream_t);                                                   \
     template void act_bwd<T>(const T*, const T*, const T*, T*, long long, int, cudaStream_t);                               \
-    template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t);                                 \
+    template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t, const ColStatsReq*);             \
     template void dwconv_dgrad<T>(const T*, const float*, const T*, T*, const ConvGeom&, cudaStream_t);                     \
     template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t);                       \
     template void maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);                                           \

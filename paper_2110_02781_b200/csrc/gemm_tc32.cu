@@ -89,6 +89,7 @@ struct T32Params {
     int rows_per_split;    // reduction elements per slice (a multiple of 32)
     int b_lo_given;        // gemm: the lo part of B comes from memory (mapBlo) instead of being computed per tile
     int* err;
+    double* stats;         // gemm with S == 1 only, nullable: [row tiles][2][N] column sums and sums of squares of each output tile
 };
 
 // Epilogue shared by both kernels, run by warps 2..5: accumulator -> shared-memory tiles of 128 rows x 32 columns
@@ -129,8 +130,37 @@ __device__ __forceinline__ void epilogue32(uint8_t* smem, uint32_t tmem, const C
                 asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
                              ::"l"(mapD), "r"(n0 + c * 32), "r"(m0), "r"(split), "r"(smem_u32(smem + c * (TC_BM * 128))) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
     }
+    if (p.stats) {
+        // Column sums of the staged tile for the batch norm that follows: thread t takes column t % BN and the
+        // rows of group t / BN, in double; the 128 / BN groups are added in group order.  Rows past M hold zeros.
+        constexpr int G = TC_BM / BN, RPG = TC_BM / G;
+        __shared__ double red[2][TC_BM];
+        const int t = threadIdx.x - 64, col = t % BN, grp = t / BN;
+        double s = 0.0, q = 0.0;
+        if (have) {
+            const uint8_t* base = smem + (col >> 5) * (TC_BM * 128) + ((col & 3) << 2);
+            const int g = (col & 31) >> 2;
+#pragma unroll 8
+            for (int r = grp * RPG; r < (grp + 1) * RPG; ++r) {
+                const double v = (double)*reinterpret_cast<const float*>(base + r * 128 + ((g ^ (r & 7)) << 4));
+                s += v;
+                q = fma(v, v, q);
+            }
+        }
+        if (G > 1) {
+            red[0][t] = s; red[1][t] = q;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (grp == 0)
+                for (int k = 1; k < G; ++k) { s += red[0][k * BN + col]; q += red[1][k * BN + col]; }
+        }
+        if (have && grp == 0 && n0 + col < p.N) {
+            double* dst = p.stats + ((long long)blockIdx.y * 2) * p.N + n0 + col;
+            dst[0] = s;
+            dst[p.N] = q;
+        }
+    }
+    if (have && threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
 }
 
 // twelve tf32 MMAs per 32-wide block of the reduction: hi*hi, hi*lo, lo*hi for each of its four 8-wide steps
@@ -540,7 +570,11 @@ G32Plan plan_gemm32(int M, int N, int K) {
 }
 
 // D[M,N] = A[M,K] * B[N,K]^T (+ addend), float in and out, split-tf32 arithmetic; both operands with K contiguous.
-bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err, cudaStream_t st) {
+// stats (nullable): the output feeds a batch norm whose fold plan is stats->fold; the partial sums of its statistics go
+// to stats->partial, from the epilogue of the product kernel (one entry per 128-row tile) or from the kernel that adds
+// the reduction slices, and *stats->out describes them.
+bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err, cudaStream_t st,
+               const ColStatsReq* stats) {
     G32Plan g = plan_gemm32(M, N, K);
     if (g.S > 1 && !scratch) { g.S = 1; g.rps = (K + T32_BK - 1) / T32_BK * T32_BK; }
     const int BN = g.BN;
@@ -549,14 +583,17 @@ bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* a
     if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, out, g.S, M, N) || !make_map_f32(&mb, B, N, K, BN)) return false;
     if (B_lo) { if (!make_map_f32(&ml, B_lo, N, K, BN)) return false; }
     else ml = mb;
-    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, B_lo ? 1 : 0, err};
+    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, B_lo ? 1 : 0, err, (stats && g.S == 1) ? stats->partial : nullptr};
     const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM, g.S);
     const int nkb = g.rps / T32_BK;
     bool ok;
     if (BN == 128) ok = launch32_stages<128>(nkb, ma, mb, ml, md, p, grid, st);
     else if (BN == 64) ok = launch32_stages<64>(nkb, ma, mb, ml, md, p, grid, st);
     else ok = launch32_stages<32>(nkb, ma, mb, ml, md, p, grid, st);
+    if (ok && stats) *stats->out = PartialSums{stats->partial, (int)grid.y, 1};
+    if (ok && g.S > 1 && stats && !addend && slice_sum_stats(scratch, g.S, D, M, N, *stats->fold, stats->partial, stats->out, st)) return true;
     if (ok && g.S > 1) {
+        if (stats) stats->out->entries = 0;          // none were produced
         const long long count4 = (long long)M * N / 4;
         launch(slice_sum_kernel, dim3((unsigned)((count4 + 255) / 256)), dim3(256), 0, st, reinterpret_cast<const float4*>(scratch), g.S, count4,
                reinterpret_cast<const float4*>(addend), reinterpret_cast<float4*>(D));

@@ -59,8 +59,9 @@ bool tc32_supported(int M, int N, int K, const void* A, const void* B, const voi
 // scratch (nullable): tc32_gemm_scratch_floats(M, N, K) floats; lets products with few tiles cut the reduction into slices
 size_t tc32_gemm_scratch_floats(int M, int N, int K);
 // B is [N][K]; B_lo (nullable): B - trunc_tf32(B) laid out like B, saves computing it per tile
+struct ColStatsReq;
 bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err,
-               cudaStream_t st);
+               cudaStream_t st, const ColStatsReq* stats = nullptr);
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
 // dW[Mo][No] = X[R][Mo]^T dY[R][No], the fixed-order second pass over the reduction slices included
 bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
@@ -74,6 +75,11 @@ struct FoldPlan {
     int rows;       // M / f
     int chunks;     // row chunks (grid.y)
     int vec;        // elements per thread per row (16 bytes worth, or 1)
+    // The reducing kernels merge the folded copies of a channel that fall inside one column tile, so a channel has
+    // chunks * f / copies partial sums for the second pass to add.
+    int fused;      // 1: merged layout in use (vectorisable tensor)
+    int copies_fwd; // copies merged per column tile of 32 * vec columns (statistics kernel)
+    int copies_bwd; // copies merged per column tile of 128 columns (backward reduction)
 };
 FoldPlan make_fold(long long M, int C, int elem_bytes);
 // Scratch of the second pass: slice sums parked by its blocks and one ticket counter per channel group
@@ -87,11 +93,26 @@ size_t fin_part_doubles(int C, int extra);      // extra = 9 for the depthwise w
 size_t fin_counter_count(int C, int extra);
 size_t fold_partial_doubles(const FoldPlan& fp);     // doubles needed for the partial sums
 
+// Partial sums laid out [entries / fp][2][C * fp] (entry e: chunk e / fp, copy e % fp), as a reducing kernel leaves them.
+struct PartialSums {
+    const double* p;
+    int entries, fp;
+};
+// A producer is asked to leave the statistics of its output for the batch norm that follows (fold = that batch
+// norm's plan).  It stores what it wrote in *out; out->entries == 0 means it wrote none.
+struct ColStatsReq {
+    double* partial;
+    const FoldPlan* fold;
+    PartialSums* out;
+};
+size_t producer_partial_doubles(long long M, int C);      // room a producer may need: one entry per 128 rows
+// D = sum of the S slices part[s][M][C] in slice order, and the statistics of D on the way.  false: nothing launched.
+bool slice_sum_stats(const float* part, int S, float* D, long long M, int C, const FoldPlan& fp, double* partial, PartialSums* out, cudaStream_t st);
 template <typename T>
-void bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st);
+PartialSums bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double* partial, cudaStream_t st);
 // mean/var -> scale (gamma * rstd), shift (a copy of beta), the mean as a two-float sum (mean + mean_lo),
 // rstd; running statistics update (momentum, unbiased variance).  z = ((y - mean) - mean_lo) * scale + shift.
-void bn_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
+void bn_finalize(const PartialSums& ps, long long M, int C, const float* gamma,
                  const float* beta, float eps, float momentum, float* run_mean, float* run_var, float* scale,
                  float* shift, float* mean, float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st);
 template <typename T>
@@ -99,12 +120,12 @@ void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const Fol
               const float* mean, const float* mean_lo, int act, cudaStream_t st);
 // pass 1 of BN backward: sums of dz' and dz'*xhat with dz' = dz masked by the activation
 template <typename T>
-void bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale,
+PartialSums bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const FoldPlan& fp, const float* scale,
                    const float* shift, const float* mean, const float* mean_lo, const float* rstd, int act,
                    double* partial, cudaStream_t st);
 // -> dgamma, dbeta and the per-channel coefficients coef[5][C]: a = gamma*rstd, then b = dbeta/M and
 // c = dgamma/M each as a two-float sum (hi, lo)
-void bn_bwd_finalize(const double* partial, const FoldPlan& fp, long long M, int C, const float* gamma,
+void bn_bwd_finalize(const PartialSums& ps, long long M, int C, const float* gamma,
                      const float* rstd, float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st);
 template <typename T>
 void bn_bwd_apply(const T* dz, const T* y, const T* addend, T* dy, long long M, int C, const FoldPlan& fp, const float* scale,
@@ -122,7 +143,7 @@ template <typename T>
 void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int act, cudaStream_t st);
 
 template <typename T>
-void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st);
+void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st, const ColStatsReq* stats = nullptr);
 template <typename T>
 void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const ConvGeom& g, cudaStream_t st);
 size_t dwconv_wgrad_scratch_floats(const ConvGeom& g);

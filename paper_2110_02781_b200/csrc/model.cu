@@ -252,7 +252,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             o.scale = t; o.shift = t + stride; o.mean = t + 2 * stride; o.mean_lo = t + 3 * stride; o.rstd = t + 4 * stride;
             o.coef = t + 5 * stride;
             o.fold = make_fold(Mout, o.C, m.esize);
-            foldd = std::max(foldd, fold_partial_doubles(o.fold));
+            foldd = std::max(foldd, std::max(fold_partial_doubles(o.fold), producer_partial_doubles(Mout, o.C)));
             finp = std::max(finp, fin_part_doubles(o.C, 1)); finc = std::max(finc, fin_counter_count(o.C, 1));
         } else if (is_contraction(o.d.kind)) {
             finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
@@ -346,6 +346,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                      cudaStream_t st) {
     const int first = m->unit_first[a], last = m->unit_last[b - 1];
     const double es = (double)m->esize;
+    PartialSums next_ps{nullptr, 0, 1};
     m->stage_in[first] = act_in;
     for (int i = first; i <= last; ++i) {
         Op& o = m->ops[i];
@@ -356,6 +357,12 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
         if (o.fused_add) out = (i + 1 == last && act_out) ? act_out : m->ops[i + 1].out;
         const Arena& ar = m->arena[m->owner[u]];
         const long long Mout = (long long)o.N * o.Ho * o.Wo;
+        // a producer whose output goes straight into a batch norm of this range leaves the statistics as it stores
+        PartialSums have_ps = next_ps;
+        next_ps.entries = 0;
+        ColStatsReq req{m->fold_scratch, nullptr, &next_ps};
+        const ColStatsReq* stats_req = nullptr;
+        if (m->producer_stats && i + 1 <= last && m->ops[i + 1].d.kind == FTP_BN && o.d.kind != FTP_BN) { req.fold = &m->ops[i + 1].fold; stats_req = &req; }
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
@@ -363,7 +370,8 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
                     const bool tc = is_pointwise_op(o) && o.d.kind != FTP_FC && tc32_supported((int)Mout, o.Co, o.C, in, ar.wt + o.w_off, out, nullptr) &&
                                     tc32_gemm((const float*)in, ar.wt + o.w_off, ar.wtl + o.w_off, nullptr, (float*)out, m->red_scratch, (int)Mout, o.Co, o.C,
-                                              m->tc_err, st);
+                                              m->tc_err, st, stats_req);
+                    if (!tc) next_ps.entries = 0;
                     if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_FWD;
                     if (!tc) conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                 } else if constexpr (!std::is_same<T, float>::value) {
@@ -385,18 +393,21 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
             }
             case FTP_DWCONV3x3: {
                 Scope sc(m, st, K_DW_FWD, u, i, 0, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
-                dwconv_fwd<T>((const T*)in, ar.w + o.w_off, (T*)out, o.g, st);
+                dwconv_fwd<T>((const T*)in, ar.w + o.w_off, (T*)out, o.g, st, stats_req);
                 break;
             }
             case FTP_BN: {
                 const long long Mr = (long long)o.N * o.H * o.W;
-                { Scope sc(m, st, K_BN_STATS, u, i, 0, o.in_elems * es, 3.0 * o.in_elems);
-                  bn_stats<T>((const T*)in, Mr, o.C, o.fold, m->fold_scratch, st); }
-                { Scope sc(m, st, K_BN_FINALIZE, u, i, 0, fold_partial_doubles(o.fold) * 8.0, 0.0);
-                  bn_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, ar.w + o.b_off, m->cfg.bn_eps, m->cfg.bn_momentum,
-                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, m->fin, st); }
+                PartialSums ps = have_ps;
+                if (ps.entries <= 0) {
+                    Scope sc(m, st, K_BN_STATS, u, i, 0, o.in_elems * es, 3.0 * o.in_elems);
+                    ps = bn_stats<T>((const T*)in, Mr, o.C, o.fold, m->fold_scratch, st);
+                }
                 const void* res = nullptr;
                 if (o.fused_add) { const int s = m->ops[i + 1].d.residual_src; res = s < first ? act_in : m->cur_out[s]; }
+                { Scope sc(m, st, K_BN_FINALIZE, u, i, 0, ps.entries * 2.0 * o.C * 8.0, 0.0);
+                  bn_finalize(ps, Mr, o.C, ar.w + o.w_off, ar.w + o.b_off, m->cfg.bn_eps, m->cfg.bn_momentum,
+                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, m->fin, st); }
                 { Scope sc(m, st, K_BN_APPLY, u, i, 0, (o.in_elems * (res ? 3.0 : 2.0)) * es, 2.0 * o.in_elems);
                   bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.d.act, st); }
                 break;
@@ -574,10 +585,11 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
             }
             case FTP_BN: {
                 const long long Mr = (long long)o.N * o.H * o.W;
+                PartialSums ps;
                 { Scope sc(m, st, K_BN_BWD_REDUCE, u, i, 1, 2.0 * o.in_elems * es, 8.0 * o.in_elems);
-                  bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.d.act, m->fold_scratch, st); }
-                { Scope sc(m, st, K_BN_BWD_FINALIZE, u, i, 1, fold_partial_doubles(o.fold) * 8.0, 0.0);
-                  bn_bwd_finalize(m->fold_scratch, o.fold, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, m->fin, st); }
+                  ps = bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.d.act, m->fold_scratch, st); }
+                { Scope sc(m, st, K_BN_BWD_FINALIZE, u, i, 1, ps.entries * 2.0 * o.C * 8.0, 0.0);
+                  bn_bwd_finalize(ps, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, m->fin, st); }
                 if (gi) {
                     Scope sc(m, st, K_BN_BWD_APPLY, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, 8.0 * o.in_elems);
                     bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef, o.d.act, st);
@@ -700,6 +712,8 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
     {   // second stream and its fork / join events: one pair per operation, created here so that nothing is created inside a stream capture
         const char* e = std::getenv("FTP_OVERLAP");
         m->overlap = !(e && std::strcmp(e, "0") == 0);
+        const char* ps = std::getenv("FTP_PRODUCER_STATS");          // 0: batch-norm statistics always by their own kernel (A/B measurements)
+        m->producer_stats = !(ps && std::strcmp(ps, "0") == 0);
         bool ok = cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking) == cudaSuccess;
         for (size_t i = 0; ok && i <= m->ops.size(); ++i) {
             cudaEvent_t a = nullptr, b = nullptr;
