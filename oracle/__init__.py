@@ -7,8 +7,9 @@ shares no code with the CUDA library.
 Pin status (see tests/test_oracle_*.py):
   ops forward/backward, loss, SGD, stage split, capacity estimate, partition optimiser,
   redistribution without failure, snapshot, schedules ........ pinned
-  redistribution with a failed index (Algorithm 1, I_fail >= 0) ... parity unpinned beyond
-  the invariants and the two prose rules of Sec. III-F (the worked figures are not available)
+  redistribution with a failed index (Algorithm 1, I_fail >= 0) and recovery sources after
+  failures (Sec. III-F) ... parity unpinned beyond invariants, the prose rules of Sec. III-F and
+  the agreement of the prose plan with Algorithm 1 (the worked figures are not available)
 """
 from .ops import *          # noqa: F401,F403
 from .model import OracleModel   # noqa: F401

@@ -8,7 +8,7 @@ import itertools
 
 __all__ = ["estimate_capacity", "choose_partition", "partition_table", "brute_force_partition",
            "stage_cost", "redistribution_plan", "is_repartition_iter", "is_replication_iter",
-           "renew_worker_list"]
+           "renew_worker_list", "recovery_sources"]
 
 
 def estimate_capacity(layer_times, points, stage_times):
@@ -130,6 +130,41 @@ def renew_worker_list(workers, failed):
     """Sec. III-F: drop the failed workers; the survivors keep their order, so every index above
     a failed one moves down."""
     return [w for w in workers if w not in failed]
+
+
+def recovery_sources(p_cur, failed, p_new):
+    """Sec. III-F, recovery after one or several workers failed.  p_cur is indexed by the old worker
+    list, p_new by the renewed one (survivors in order).  For every new stage j the units of its new
+    range with where their weights come from:
+      ("local",)        the worker holds the unit already;
+      ("stage", i)      the live weights of surviving worker i (new index);
+      ("replica", i)    the chain replica of a failed worker, kept by the worker after it in the old
+                        list (new index i), or by the central node (i = 0) when the last worker failed;
+      ("central",)      the global replica on the central node: the failed worker's neighbour failed too.
+    Worker 0 is the central node and does not fail (Sec. III-E)."""
+    n_cur = len(p_cur) - 1
+    failed = sorted(set(failed))
+    assert failed and all(0 < f < n_cur for f in failed), "failed workers must be among 1 .. n_cur-1"
+    alive = renew_worker_list(list(range(n_cur)), failed)
+    assert len(p_new) - 1 == len(alive), "the new partition must have one stage per survivor"
+    plan = []
+    for j, old in enumerate(alive):
+        items = []
+        for u in range(p_new[j], p_new[j + 1]):
+            holder = next(i for i in range(n_cur) if p_cur[i] <= u < p_cur[i + 1])
+            if holder == old:
+                src = ("local",)
+            elif holder not in failed:
+                src = ("stage", alive.index(holder))
+            elif holder == n_cur - 1:
+                src = ("replica", 0)
+            elif holder + 1 not in failed:
+                src = ("replica", alive.index(holder + 1))
+            else:
+                src = ("central",)
+            items.append((u, src))
+        plan.append(items)
+    return plan
 
 
 def is_repartition_iter(it, first=10, period=100):

@@ -115,6 +115,65 @@ def test_redistribution_failure_rules_from_the_prose():
     assert need.get(0) == [6, 7]
 
 
+def _compositions(L, n):
+    import itertools
+    for cuts in itertools.combinations(range(1, L), n - 1):
+        yield [0, *cuts, L]
+
+
+def test_recovery_sources_single_failure_equals_algorithm_1():
+    """With one failed worker the prose of Sec. III-F and the printed Algorithm 1 must name the same
+    place for every unit: the plan built from the prose is compared with Algorithm 1 run for every
+    surviving worker, over every pair of partitions of 6 units on 4 -> 3 workers."""
+    L, n = 6, 4
+    for p_cur in _compositions(L, n):
+        for p_new in _compositions(L, n - 1):
+            for f in range(1, n):
+                alive = oracle.renew_worker_list(list(range(n)), [f])
+                plan = oracle.recovery_sources(p_cur, [f], p_new)
+                for j, old in enumerate(alive):
+                    need, local = oracle.redistribution_plan(p_new, p_cur, old, j, i_fail=f)
+                    want = {}
+                    for u, src in plan[j]:
+                        if src[0] == "local":
+                            assert u in local
+                        else:
+                            assert src[0] in ("stage", "replica")       # one failure never needs the global replica
+                            want.setdefault(src[1], []).append(u)
+                    assert want == need, (p_cur, p_new, f, j)
+
+
+def test_recovery_sources_every_source_really_holds_the_unit():
+    """A small world: worker i holds its units; worker i+1 keeps the chain replica of worker i, the
+    central node (0) that of the last worker and the global replica of everything.  After any set of
+    failures every unit of every new stage must come from a place that survived and has it, the new
+    ranges must cover all units exactly once, and the global replica is used only when a failed
+    worker's neighbour failed too."""
+    import itertools
+    L, n = 7, 5
+    for p_cur in list(_compositions(L, n))[::3]:
+        for k in (1, 2, 3):
+            for failed in itertools.combinations(range(1, n), k):
+                alive = oracle.renew_worker_list(list(range(n)), list(failed))
+                p_new = next(_compositions(L, len(alive)))
+                plan = oracle.recovery_sources(p_cur, list(failed), p_new)
+                seen = []
+                for j, items in enumerate(plan):
+                    for u, src in items:
+                        seen.append(u)
+                        holder = next(i for i in range(n) if p_cur[i] <= u < p_cur[i + 1])
+                        if src[0] == "local":
+                            assert holder == alive[j]
+                        elif src[0] == "stage":
+                            assert alive[src[1]] == holder and holder not in failed
+                        elif src[0] == "replica":
+                            keeper = 0 if holder == n - 1 else holder + 1
+                            assert holder in failed and alive[src[1]] == keeper and keeper not in failed
+                        else:
+                            assert holder in failed and holder != n - 1 and holder + 1 in failed
+                assert seen == list(range(L))
+
+
 def test_schedules_match_the_paper(golden_dir):
     facts = {}
     for line in open(golden_dir + "/schedule_ticks.txt"):
