@@ -211,6 +211,48 @@ ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int32_t n_stag
                              void* stream);
 ftp_status ftp_get_partition(const ftp_model* m, int32_t* points /* max_stages+1 */, int32_t* n_stages);
 
+/* ---- recovery from worker failures: Sec. III-F.  --------------------------------------------
+ * A failure is a host-side event here (all stages share one GPU): the caller names the stages
+ * whose memory is to be treated as lost; nothing on the device is faulted. */
+
+/* Where a unit's weights come from after failures (pure host function).  failed[n_failed]:
+ * distinct old indices in 1 .. n_cur-1 (worker 0 is the central node and does not fail); the
+ * survivors keep their order and become 0 .. n_new-1, n_new = n_cur - n_failed.  For every unit u
+ * of the model: kind[u] is FTP_SRC_LOCAL (its new owner holds it already), FTP_SRC_STAGE (the live
+ * weights of surviving worker index[u], new numbering), FTP_SRC_REPLICA (the chain replica of the
+ * failed worker that held u, kept by the worker after it, index[u] in the new numbering, 0 = the
+ * central node for the last worker) or FTP_SRC_CENTRAL (the global replica on the central node:
+ * the keeper of the chain replica failed too).  With one failure this is Algorithm 1. */
+enum { FTP_SRC_LOCAL = 0, FTP_SRC_STAGE = 1, FTP_SRC_REPLICA = 2, FTP_SRC_CENTRAL = 3 };
+ftp_status ftp_recovery_plan(const int32_t* p_cur, int32_t n_cur, const int32_t* failed, int32_t n_failed,
+                             const int32_t* p_new, int32_t n_new, int32_t* kind /* L */, int32_t* index /* L */);
+
+/* One failed stage and its chain replica: the bytes ftp_snapshot_weights(stage) wrote under the
+ * partition that is current now (device memory, or host memory for the last stage, whose replica
+ * the central node keeps).  replica may be NULL when none exists. */
+typedef struct {
+    int32_t stage;
+    int32_t replica_is_host;
+    const void* replica;
+    size_t replica_bytes;
+} ftp_failed_stage;
+
+/* Recover and re-partition (Sec. III-F): the failed stages' arenas are abandoned, the survivors
+ * are renumbered in order, and the model is spread over them at p_new (n_new = stages - n_failed
+ * boundaries + 1, normally from ftp_choose_partition).  Per unit, following ftp_recovery_plan:
+ * local units stay where they are, units of other survivors are copied between arenas with their
+ * momentum, units of a failed stage are loaded from its chain replica (weights and BN running
+ * statistics as of that replica; their momentum restarts from the next gradient) or, when the
+ * replica's keeper failed too or no replica was given, from `central`: the global replica, all
+ * units in canonical order, host memory, nullable.  A unit with no source left is FTP_ESTATE and
+ * nothing is changed.  The owner table switches only after every copy is enqueued (the commit);
+ * forward state of all units is discarded, as the paper discards the batches in flight.
+ * counts (nullable): units taken from other stages, from chain replicas, from the global replica.
+ * A replica must have been taken under the current partition (its size is checked). */
+ftp_status ftp_recover(ftp_model* m, const ftp_failed_stage* failed, int32_t n_failed, const void* central,
+                       size_t central_bytes, const int32_t* p_new, int32_t n_new, int32_t* counts /* 3 */,
+                       void* stream);
+
 /* ---- snapshot_weights(stage, dst): Sec. III-E chain / global replication. ----------------- */
 
 /* Copy stage's replica -- per unit of the stage, in order: trainable weights then BN running

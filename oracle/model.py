@@ -252,6 +252,26 @@ class OracleModel:
     def unit_state(self, unit):
         return self._flat(self.s, unit)
 
+    def set_unit(self, unit, params_flat, state_flat, reset_momentum=True):
+        """Load a unit from a replica (Sec. III-F): trainable weights and BN running statistics in
+        canonical order; the momentum of the unit starts afresh, as on a worker that just received
+        the weights (the replica of Sec. III-E holds weights only)."""
+        def scatter(store, flat):
+            off = 0
+            for i, l in enumerate(self.layers):
+                if l.unit != unit:
+                    continue
+                for k, v in enumerate(store[i]):
+                    store[i][k] = np.asarray(flat[off:off + v.size], np.float64).reshape(v.shape).copy()
+                    off += v.size
+            assert off == len(flat), "replica size does not match the unit"
+        scatter(self.p, params_flat)
+        scatter(self.s, state_flat)
+        if reset_momentum:
+            for i, l in enumerate(self.layers):
+                if l.unit == unit:
+                    self.m[i] = [None] * len(self.m[i])
+
     def unit_param_count(self, unit):
         return self.unit_params(unit).size
 

@@ -730,6 +730,7 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
     m->owner.assign(m->L, 0);
     m->points = {0, m->L};
     m->n_stages = 1;
+    m->worker.assign(1, 0);
     m->mom_init.assign(m->L, 0);
     m->stage_in.assign(m->ops.size(), nullptr);
     m->cur_out.assign(m->ops.size(), nullptr);
@@ -954,6 +955,26 @@ extern "C" ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void*
     return check_launches("profile_layers");
 }
 
+// Everything arena `from` holds of unit u (weights, momentum, running statistics and the derived copies) -> arena `to`.
+static ftp_status copy_unit(ftp_model* m, int u, int from_arena, int to_arena, cudaStream_t st) {
+    const Arena& from = m->arena[from_arena];
+    const Arena& to = m->arena[to_arena];
+    const long long po = m->unit_p_off[u], pc = m->unit_p_cnt[u], so = m->unit_s_off[u], sc_ = m->unit_s_cnt[u];
+    if (pc) {
+        CUDA_OK(cudaMemcpyAsync(to.w + po, from.w + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+        CUDA_OK(cudaMemcpyAsync(to.m + po, from.m + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+        if (to.wb) CUDA_OK(cudaMemcpyAsync(to.wb + po, from.wb + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
+        if (to.wbt) CUDA_OK(cudaMemcpyAsync(to.wbt + po, from.wbt + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
+        if (to.wl) {
+            CUDA_OK(cudaMemcpyAsync(to.wl + po, from.wl + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+            CUDA_OK(cudaMemcpyAsync(to.wt + po, from.wt + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+            CUDA_OK(cudaMemcpyAsync(to.wtl + po, from.wtl + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+        }
+    }
+    if (sc_) CUDA_OK(cudaMemcpyAsync(to.run + so, from.run + so, (size_t)sc_ * 4, cudaMemcpyDeviceToDevice, st));
+    return FTP_OK;
+}
+
 extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int32_t n_stages, int32_t* moved_units, void* stream) {
     FTP_REQUIRE(m && points, FTP_EINVAL, "set_partition: null argument");
     FTP_REQUIRE(n_stages >= 1 && n_stages <= m->cfg.max_stages && n_stages <= m->L, FTP_EINVAL,
@@ -963,6 +984,12 @@ extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int
     cudaStream_t st = (cudaStream_t)stream;
     int moved = 0;
     std::vector<int32_t> plan(m->L);
+    // stages beyond the current worker list are joined by workers whose arenas are idle (lowest first)
+    std::vector<int> worker = m->worker;
+    worker.resize(std::min<size_t>(worker.size(), (size_t)n_stages));
+    for (int a = 0; (int)worker.size() < n_stages && a < m->cfg.max_stages; ++a)
+        if (std::find(worker.begin(), worker.end(), a) == worker.end()) worker.push_back(a);
+    FTP_REQUIRE((int)worker.size() == n_stages, FTP_ESTATE, "set_partition: no idle arena left for %d stages", n_stages);
     // Phase 1: every stage fetches what Algorithm 1 says it is missing, from the current owner's arena.
     for (int i = 0; i < n_stages; ++i) {
         int32_t n_local = 0;
@@ -972,27 +999,15 @@ extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int
             const int src = plan[u - points[i]];
             if (src < 0) continue;                                   // already local
             ++moved;
-            const Arena& from = m->arena[src];
-            const Arena& to = m->arena[i];
-            const long long po = m->unit_p_off[u], pc = m->unit_p_cnt[u], so = m->unit_s_off[u], sc_ = m->unit_s_cnt[u];
-            Scope sc(m, st, K_COPY, u, -1, 2, (pc * 2 + sc_) * 8.0, 0.0, 0);
-            if (pc) {
-                CUDA_OK(cudaMemcpyAsync(to.w + po, from.w + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
-                CUDA_OK(cudaMemcpyAsync(to.m + po, from.m + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
-                if (to.wb) CUDA_OK(cudaMemcpyAsync(to.wb + po, from.wb + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
-                if (to.wbt) CUDA_OK(cudaMemcpyAsync(to.wbt + po, from.wbt + po, (size_t)pc * 2, cudaMemcpyDeviceToDevice, st));
-                if (to.wl) {
-                    CUDA_OK(cudaMemcpyAsync(to.wl + po, from.wl + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
-                    CUDA_OK(cudaMemcpyAsync(to.wt + po, from.wt + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
-                    CUDA_OK(cudaMemcpyAsync(to.wtl + po, from.wtl + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
-                }
-            }
-            if (sc_) CUDA_OK(cudaMemcpyAsync(to.run + so, from.run + so, (size_t)sc_ * 4, cudaMemcpyDeviceToDevice, st));
+            Scope sc(m, st, K_COPY, u, -1, 2, (m->unit_p_cnt[u] * 2 + m->unit_s_cnt[u]) * 8.0, 0.0, 0);
+            const ftp_status cs = copy_unit(m, u, m->worker[src], worker[i], st);
+            if (cs != FTP_OK) return cs;
         }
     }
     // Phase 2 (commit): only now does the owner table switch; later launches are stream-ordered after the copies.
     for (int i = 0; i < n_stages; ++i)
-        for (int u = points[i]; u < points[i + 1]; ++u) m->owner[u] = i;
+        for (int u = points[i]; u < points[i + 1]; ++u) m->owner[u] = worker[i];
+    m->worker = worker;
     m->points.assign(points, points + n_stages + 1);
     m->n_stages = n_stages;
     std::fill(m->fwd_done.begin(), m->fwd_done.end(), 0);
@@ -1007,6 +1022,96 @@ extern "C" ftp_status ftp_get_partition(const ftp_model* m, int32_t* points, int
     return FTP_OK;
 }
 
+extern "C" ftp_status ftp_recover(ftp_model* m, const ftp_failed_stage* failed, int32_t n_failed, const void* central, size_t central_bytes,
+                                  const int32_t* p_new, int32_t n_new, int32_t* counts, void* stream) {
+    FTP_REQUIRE(m && failed && p_new, FTP_EINVAL, "recover: null argument");
+    const int n_cur = m->n_stages, L = m->L;
+    std::vector<int32_t> fl(std::max(n_failed, 0)), kind(L), index(L);
+    for (int k = 0; k < n_failed; ++k) fl[k] = failed[k].stage;
+    ftp_status s = ftp_recovery_plan(m->points.data(), n_cur, fl.data(), n_failed, p_new, n_new, kind.data(), index.data());
+    if (s != FTP_OK) return s;
+    FTP_REQUIRE(p_new[n_new] == L, FTP_EINVAL, "recover: the new partition must end at unit %d", L);
+    // survivors in order: new stage j is the worker that was stage alive[j] and keeps its arena
+    std::vector<int> alive, worker;
+    for (int i = 0; i < n_cur; ++i)
+        if (std::find(fl.begin(), fl.end(), i) == fl.end()) { alive.push_back(i); worker.push_back(m->worker[i]); }
+    auto unit_bytes = [&](int u) { return (size_t)(m->unit_p_cnt[u] + m->unit_s_cnt[u]) * 4; };
+    size_t all_bytes = 0;
+    std::vector<size_t> central_off(L);
+    for (int u = 0; u < L; ++u) { central_off[u] = all_bytes; all_bytes += unit_bytes(u); }
+    // where each failed stage's units lie inside its chain replica; all checks before the first copy
+    std::vector<const ftp_failed_stage*> rec(n_cur, nullptr);
+    for (int k = 0; k < n_failed; ++k) {
+        const ftp_failed_stage& f = failed[k];
+        rec[f.stage] = &f;
+        if (!f.replica) continue;
+        size_t need = 0;
+        for (int u = m->points[f.stage]; u < m->points[f.stage + 1]; ++u) need += unit_bytes(u);
+        FTP_REQUIRE(f.replica_bytes == need, FTP_ESTATE, "recover: the replica of stage %d has %zu bytes, the stage's units take %zu (was it taken under another partition?)",
+                    f.stage, f.replica_bytes, need);
+    }
+    for (int u = 0; u < L; ++u) {
+        if (kind[u] != FTP_SRC_REPLICA && kind[u] != FTP_SRC_CENTRAL) continue;
+        int holder = 0;
+        while (!(m->points[holder] <= u && u < m->points[holder + 1])) ++holder;
+        if (kind[u] == FTP_SRC_REPLICA && !rec[holder]->replica) kind[u] = FTP_SRC_CENTRAL;        // no chain replica was ever taken
+        if (kind[u] == FTP_SRC_CENTRAL)
+            FTP_REQUIRE(central && central_bytes >= all_bytes, FTP_ESTATE, "recover: unit %d is lost (no chain replica survives and the global replica is %s)", u,
+                        central ? "too short" : "missing");
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    int n_stage = 0, n_replica = 0, n_central = 0;
+    std::vector<int> reloaded;
+    for (int j = 0; j < n_new; ++j)
+        for (int u = p_new[j]; u < p_new[j + 1]; ++u) {
+            if (kind[u] == FTP_SRC_LOCAL) continue;
+            Scope sc(m, st, K_COPY, u, -1, 2, 2.0 * unit_bytes(u), 0.0, 0);
+            if (kind[u] == FTP_SRC_STAGE) {
+                ++n_stage;
+                s = copy_unit(m, u, worker[index[u]], worker[j], st);
+                if (s != FTP_OK) return s;
+                continue;
+            }
+            // from a replica: weights and running statistics as they were replicated; momentum restarts
+            const char* src;
+            cudaMemcpyKind how;
+            if (kind[u] == FTP_SRC_REPLICA) {
+                int holder = 0;
+                while (!(m->points[holder] <= u && u < m->points[holder + 1])) ++holder;
+                size_t off = 0;
+                for (int v = m->points[holder]; v < u; ++v) off += unit_bytes(v);
+                src = (const char*)rec[holder]->replica + off;
+                how = rec[holder]->replica_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+                ++n_replica;
+            } else {
+                src = (const char*)central + central_off[u];
+                how = cudaMemcpyHostToDevice;
+                ++n_central;
+            }
+            const Arena& to = m->arena[worker[j]];
+            if (m->unit_p_cnt[u]) CUDA_OK(cudaMemcpyAsync(to.w + m->unit_p_off[u], src, (size_t)m->unit_p_cnt[u] * 4, how, st));
+            if (m->unit_s_cnt[u]) CUDA_OK(cudaMemcpyAsync(to.run + m->unit_s_off[u], src + (size_t)m->unit_p_cnt[u] * 4, (size_t)m->unit_s_cnt[u] * 4, how, st));
+            reloaded.push_back(u);
+        }
+    // commit: the survivors' list and the owner table switch, then the derived copies of the reloaded weights are rebuilt
+    for (int j = 0; j < n_new; ++j)
+        for (int u = p_new[j]; u < p_new[j + 1]; ++u) m->owner[u] = worker[j];
+    m->worker = worker;
+    m->points.assign(p_new, p_new + n_new + 1);
+    m->n_stages = n_new;
+    std::fill(m->fwd_done.begin(), m->fwd_done.end(), 0);
+    for (int u : reloaded) {
+        const Arena& ar = m->arena[m->owner[u]];
+        const long long po = m->unit_p_off[u], pc = m->unit_p_cnt[u];
+        m->mom_init[u] = 0;
+        if (!pc) continue;
+        if (ar.wb) { f32_to_bf16(ar.w + po, ar.wb + po, pc, st); refresh_transposed(m, u, u + 1, st); }
+        if (ar.wl) { tf32_lo(ar.w + po, ar.wl + po, pc, st); refresh_transposed(m, u, u + 1, st); }
+    }
+    if (counts) { counts[0] = n_stage; counts[1] = n_replica; counts[2] = n_central; }
+    return check_launches("recover");
+}
+
 extern "C" ftp_status ftp_snapshot_weights(const ftp_model* m, int32_t stage, void* dst, size_t dst_bytes, int32_t dst_is_host, size_t* written,
                                            void* stream) {
     FTP_REQUIRE(m && dst, FTP_EINVAL, "snapshot_weights: null argument");
@@ -1018,7 +1123,7 @@ extern "C" ftp_status ftp_snapshot_weights(const ftp_model* m, int32_t stage, vo
     cudaStream_t st = (cudaStream_t)stream;
     const cudaMemcpyKind kind = dst_is_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
     char* p = (char*)dst;
-    const Arena& ar = m->arena[stage];
+    const Arena& ar = m->arena[m->worker[stage]];
     Scope sc(const_cast<ftp_model*>(m), st, K_COPY, a, -1, 2, 2.0 * need, 0.0, 0);
     for (int u = a; u < b; ++u) {
         if (m->unit_p_cnt[u]) { CUDA_OK(cudaMemcpyAsync(p, ar.w + m->unit_p_off[u], (size_t)m->unit_p_cnt[u] * 4, kind, st)); p += m->unit_p_cnt[u] * 4; }

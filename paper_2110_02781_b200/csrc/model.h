@@ -60,7 +60,8 @@ struct ftp_model {
     long long P, R;
     std::vector<ftp::Arena> arena;
     float* grad;
-    std::vector<int> owner;                       // unit -> stage
+    std::vector<int> owner;                       // unit -> arena of the worker that holds it
+    std::vector<int> worker;                      // stage -> arena (a worker keeps its arena when failures renumber the stages)
     std::vector<int> points;
     int n_stages;
     std::vector<char> mom_init;                   // per unit: momentum buffer holds a value

@@ -115,3 +115,34 @@ extern "C" ftp_status ftp_redistribution_plan(const int32_t* p_new, int32_t n_ne
     if (n_local) *n_local = local;
     return FTP_OK;
 }
+
+extern "C" ftp_status ftp_recovery_plan(const int32_t* p_cur, int32_t n_cur, const int32_t* failed, int32_t n_failed, const int32_t* p_new,
+                                        int32_t n_new, int32_t* kind, int32_t* index) {
+    FTP_REQUIRE(p_cur && failed && p_new && kind && index, FTP_EINVAL, "recovery_plan: null argument");
+    FTP_REQUIRE(n_cur >= 2 && n_failed >= 1 && n_new == n_cur - n_failed && n_new >= 1, FTP_EINVAL,
+                "recovery_plan: %d workers minus %d failed must leave the %d stages of the new partition", n_cur, n_failed, n_new);
+    FTP_REQUIRE(valid_points(p_new, n_new, -1) && valid_points(p_cur, n_cur, p_new[n_new]), FTP_EINVAL,
+                "recovery_plan: both partitions must rise from 0 to the same L");
+    std::vector<char> dead(n_cur, 0);
+    for (int32_t k = 0; k < n_failed; ++k) {
+        FTP_REQUIRE(failed[k] >= 1 && failed[k] < n_cur, FTP_ERANGE, "recovery_plan: failed worker %d is not among 1..%d (worker 0, the central node, does not fail)",
+                    failed[k], n_cur - 1);
+        FTP_REQUIRE(!dead[failed[k]], FTP_EINVAL, "recovery_plan: worker %d is listed twice", failed[k]);
+        dead[failed[k]] = 1;
+    }
+    std::vector<int32_t> new_index(n_cur, -1), alive;
+    for (int32_t i = 0; i < n_cur; ++i)
+        if (!dead[i]) { new_index[i] = (int32_t)alive.size(); alive.push_back(i); }
+    for (int32_t j = 0; j < n_new; ++j)
+        for (int32_t u = p_new[j]; u < p_new[j + 1]; ++u) {
+            int32_t holder = 0;
+            while (!(p_cur[holder] <= u && u < p_cur[holder + 1])) ++holder;
+            if (holder == alive[j]) { kind[u] = FTP_SRC_LOCAL; index[u] = j; }
+            else if (!dead[holder]) { kind[u] = FTP_SRC_STAGE; index[u] = new_index[holder]; }
+            else if (holder == n_cur - 1) { kind[u] = FTP_SRC_REPLICA; index[u] = 0; }                       // the central node keeps the last worker's replica
+            else if (!dead[holder + 1]) { kind[u] = FTP_SRC_REPLICA; index[u] = new_index[holder + 1]; }
+            else { kind[u] = FTP_SRC_CENTRAL; index[u] = 0; }
+        }
+    return FTP_OK;
+}
+

@@ -64,6 +64,8 @@ _SIGS = {
     "ftp_choose_partition": [_P(C.c_double), _i32, _P(C.c_double), _i32, _P(C.c_double), _P(C.c_double), _P(_i32),
                              _P(C.c_double)],
     "ftp_redistribution_plan": [_P(_i32), _i32, _P(_i32), _i32, _i32, _i32, _i32, _P(_i32), _P(_i32)],
+    "ftp_recovery_plan": [_P(_i32), _i32, _P(_i32), _i32, _P(_i32), _i32, _P(_i32), _P(_i32)],
+    "ftp_recover": [_vp, _vp, _i32, _vp, _sz, _P(_i32), _i32, _P(_i32), _vp],
     "ftp_set_partition": [_vp, _P(_i32), _i32, _P(_i32), _vp],
     "ftp_get_partition": [_vp, _P(_i32), _P(_i32)],
     "ftp_snapshot_weights": [_vp, _i32, _vp, _sz, _i32, _P(_sz), _vp],
@@ -159,6 +161,25 @@ def ftp_redistribution_plan(p_new, p_cur, i_cur, i_new, i_fail=-1):
     _check(lib.ftp_redistribution_plan(ppn, len(pn) - 1, ppc, len(pc) - 1, i_fail, i_cur, i_new,
                                        owners.ctypes.data_as(_P(_i32)), C.byref(nloc)))
     return owners[:int(pn[i_new + 1] - pn[i_new])].tolist(), nloc.value
+
+
+SRC_LOCAL, SRC_STAGE, SRC_REPLICA, SRC_CENTRAL = 0, 1, 2, 3
+
+
+class FailedStage(C.Structure):
+    _fields_ = [("stage", _i32), ("replica_is_host", _i32), ("replica", _vp), ("replica_bytes", _sz)]
+
+
+def ftp_recovery_plan(p_cur, failed, p_new):
+    """Per unit: (kind, index) as ftp_recovery_plan in include/ftpipe.h defines them."""
+    pc, ppc = _i32arr(p_cur)
+    pn, ppn = _i32arr(p_new)
+    fl, pfl = _i32arr(failed)
+    L = int(pc[-1])
+    kind, index = np.full(max(L, 1), -7, np.int32), np.full(max(L, 1), -7, np.int32)
+    _check(lib.ftp_recovery_plan(ppc, len(pc) - 1, pfl, len(fl), ppn, len(pn) - 1, kind.ctypes.data_as(_P(_i32)),
+                                 index.ctypes.data_as(_P(_i32))))
+    return kind[:L].tolist(), index[:L].tolist()
 
 
 def ftp_workspace_bytes(layers, cfg):
@@ -276,6 +297,21 @@ class Model:
         _check(lib.ftp_set_partition(self.h, pp, len(pts) - 1, C.byref(moved), _stream(stream)))
         return moved.value
 
+    def ftp_recover(self, failed, p_new, central=None, stream=None):
+        """failed: {stage: chain replica tensor (device, or host for the last stage) or None}; central: the global
+        replica (host tensor, all units in canonical order) or None.  Returns (from stages, from replicas, from central)."""
+        recs = (FailedStage * max(len(failed), 1))()
+        for k, (stage, rep) in enumerate(sorted(failed.items())):
+            recs[k].stage = stage
+            recs[k].replica_is_host = int(rep is not None and not rep.is_cuda)
+            recs[k].replica = _ptr(rep)
+            recs[k].replica_bytes = 0 if rep is None else rep.numel() * rep.element_size()
+        pts, pp = _i32arr(p_new)
+        counts = (_i32 * 3)()
+        _check(lib.ftp_recover(self.h, recs, len(failed), _ptr(central), 0 if central is None else central.numel() * central.element_size(),
+                               pp, len(pts) - 1, counts, _stream(stream)))
+        return tuple(counts)
+
     def ftp_get_partition(self):
         pts = (_i32 * (self.cfg["max_stages"] + 1))()
         n = _i32()
@@ -318,5 +354,5 @@ class Model:
 
 
 __all__ = ["Model", "FtpError", "LayerDesc", "ModelCfg", "TraceRec", "ftp_estimate_capacity", "ftp_choose_partition",
-           "ftp_redistribution_plan", "ftp_workspace_bytes", "ftp_kernel_name", "ftp_conv_wgrad_static", "layer_array", "model_cfg", "lib",
+           "ftp_redistribution_plan", "ftp_recovery_plan", "FailedStage", "SRC_LOCAL", "SRC_STAGE", "SRC_REPLICA", "SRC_CENTRAL", "ftp_workspace_bytes", "ftp_kernel_name", "ftp_conv_wgrad_static", "layer_array", "model_cfg", "lib",
            "T_WEIGHTS", "T_GRADS", "T_MOMENTUM", "T_STATE", "FP32", "BF16", "LIB_PATH"]

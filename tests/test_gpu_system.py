@@ -5,7 +5,7 @@ import pytest
 
 import oracle
 import synth
-from helpers import gpu_step_split, make_gpu, make_oracle, rel_err, to_dev, TOL_FP32
+from helpers import clear_batch, gpu_step_split, make_gpu, make_oracle, perturb, rel_err, to_dev, TOL_FP32
 
 pytestmark = pytest.mark.gpu
 F = pytest.importorskip("paper_2110_02781_b200")
@@ -154,3 +154,108 @@ def test_trace_records_every_launch_with_its_algorithmic_work():
     assert {"conv_fwd_f32", "conv_dgrad_f32", "conv_wgrad_f32", "bn_stats", "bn_apply", "bn_bwd_reduce", "bn_bwd_apply",
             "dw_fwd", "dw_dgrad", "dw_wgrad", "gap_fwd", "softmax_ce", "sgd"} <= names
     assert gm.ftp_launch_count() - n0 >= len(recs)
+
+
+def _replicas(gm, sizes):
+    """Chain and global replicas as the paper keeps them: stage i's weights with stage i+1 (device), the last
+    stage's and everybody's with the central node (pinned host)."""
+    import torch
+    pts = gm.ftp_get_partition()
+    n = len(pts) - 1
+    total = sum(sizes)
+    chain = {}
+    central = torch.empty(total, dtype=torch.float32).pin_memory()
+    off = 0
+    for s in range(n):
+        cnt = sum(sizes[pts[s]:pts[s + 1]])
+        chain[s] = torch.empty(cnt, dtype=torch.float32, device="cuda") if s + 1 < n else torch.empty(cnt, dtype=torch.float32).pin_memory()
+        gm.ftp_snapshot_weights(s, chain[s])
+        gm.ftp_snapshot_weights(s, central[off:off + cnt])
+        off += cnt
+    torch.cuda.synchronize()
+    return chain, central
+
+
+@pytest.mark.parametrize("failed", [[2], [3], [1, 2], [1, 3]], ids=lambda f: "fail" + "_".join(map(str, f)))
+def test_recovery_after_stage_failures(failed):
+    """Sec. III-F on one GPU: train, replicate, train on (so the replicas are stale), then lose some stages.  After
+    ftp_recover every unit of a surviving stage must hold its live weights bit for bit, every unit of a failed stage
+    the bytes of the replica the plan names, and training must go on exactly as the oracle does from that state
+    (momentum of the reloaded units restarted)."""
+    import torch
+    ls, cfg = synth.tiny_mbv2(momentum=0.9)
+    cfg = dict(cfg, max_stages=4)
+    params, state = perturb(ls, 81), synth.init_state(ls)
+    om = oracle.OracleModel(ls, cfg, params, state)
+    gm = F.Model(ls, cfg)
+    gm.load_params(params, state)
+    L = gm.L
+    p_cur = [0, 2, 4, 5, L]
+    gm.ftp_set_partition(p_cur)
+    x, y, _ = clear_batch(om, 81, cfg)
+    xd, yd = to_dev(x), to_dev(y)
+    lr = cfg["lr"]
+    sizes = [gm.ftp_unit_param_span(u)[1] + gm.ftp_unit_state_span(u)[1] for u in range(L)]
+    for _ in range(2):
+        gm.ftp_train_step(xd, yd, lr)
+        om.step(p_cur, x, y)
+    chain, central = _replicas(gm, sizes)
+    snap_w = [om.unit_params(u).copy() for u in range(L)]
+    snap_s = [om.unit_state(u).copy() for u in range(L)]
+    gm.ftp_train_step(xd, yd, lr)                       # the replicas are one step old when the failure happens
+    om.step(p_cur, x, y)
+    live = [np.concatenate([gm.ftp_get_tensor(F.T_WEIGHTS, u), gm.ftp_get_tensor(F.T_STATE, u)]) for u in range(L)]
+    n_new = len(p_cur) - 1 - len(failed)
+    p_new = {3: [0, 3, 5, L], 2: [0, 4, L]}[n_new]
+    plan = oracle.recovery_sources(p_cur, failed, p_new)
+    # the chain replica of a failed stage is usable only if its keeper (the next stage) survived
+    counts = gm.ftp_recover({f: chain[f] for f in failed}, p_new, central)
+    torch.cuda.synchronize()
+    assert gm.ftp_get_partition() == p_new
+    want = [sum(1 for items in plan for _, s in items if s[0] == k) for k in ("stage", "replica", "central")]
+    assert list(counts) == want
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    central_np = central.numpy()
+    for items in plan:
+        for u, src in items:
+            got = np.concatenate([gm.ftp_get_tensor(F.T_WEIGHTS, u), gm.ftp_get_tensor(F.T_STATE, u)])
+            if src[0] in ("local", "stage"):
+                assert np.array_equal(got, live[u]), f"unit {u} ({src}) lost its live weights"
+            else:
+                assert np.array_equal(got, central_np[offs[u]:offs[u + 1]]), f"unit {u} ({src}) is not the replicated copy"
+                om.set_unit(u, snap_w[u], snap_s[u], reset_momentum=True)
+    # training continues identically on both sides
+    for _ in range(2):
+        loss = gm.ftp_train_step(xd, yd, lr)
+        ref = om.step(p_new, x, y)
+        assert abs(loss - ref) <= TOL_FP32 * max(abs(ref), 1.0)
+    for u in range(L):
+        assert rel_err(gm.ftp_get_tensor(F.T_WEIGHTS, u), om.unit_params(u)) <= TOL_FP32
+    # a stage can rejoin: four stages again, on whichever arenas are idle
+    gm.ftp_set_partition(p_cur)
+    loss = gm.ftp_train_step(xd, yd, lr)
+    ref = om.step(p_cur, x, y)
+    assert abs(loss - ref) <= TOL_FP32 * max(abs(ref), 1.0)
+    gm.close()
+
+
+def test_recover_refuses_what_it_cannot_restore():
+    import torch
+    ls, cfg = synth.tiny_mbv2()
+    cfg = dict(cfg, max_stages=4)
+    gm = F.Model(ls, cfg)
+    gm.load_params(synth.init_params(82, ls), synth.init_state(ls))
+    L = gm.L
+    gm.ftp_set_partition([0, 2, 4, L])
+    before = gm.ftp_get_partition()
+    with pytest.raises(F.FtpError):
+        gm.ftp_recover({0: None}, [0, 3, L])                        # the central node does not fail
+    with pytest.raises(F.FtpError):
+        gm.ftp_recover({1: None}, [0, 3, L])                        # no replica of any kind
+    with pytest.raises(F.FtpError):
+        gm.ftp_recover({1: torch.empty(5, device="cuda")}, [0, 3, L])   # replica of the wrong size
+    with pytest.raises(F.FtpError):
+        gm.ftp_recover({1: None}, [0, 2, 4, L])                     # one failure leaves two stages
+    assert gm.ftp_get_partition() == before
+    gm.close()
+

@@ -101,3 +101,30 @@ def test_workspace_and_validation_without_gpu():
         F.ftp_workspace_bytes(bad, cfg)
     with pytest.raises(F.FtpError):
         F.ftp_workspace_bytes(ls, dict(cfg, batch=0))
+
+
+def test_recovery_plan_equals_oracle():
+    """ftp_recovery_plan (Sec. III-F) against the oracle's plan, unit by unit, over random partitions and every set
+    of up to three failed workers out of five; bad failure lists are refused."""
+    import itertools
+    rng = np.random.default_rng(9)
+    L, n_cur = 11, 5
+    code = {"local": F.SRC_LOCAL, "stage": F.SRC_STAGE, "replica": F.SRC_REPLICA, "central": F.SRC_CENTRAL}
+    for _ in range(40):
+        p_cur = [0] + sorted(rng.choice(np.arange(1, L), n_cur - 1, replace=False).tolist()) + [L]
+        for k in (1, 2, 3):
+            for failed in itertools.combinations(range(1, n_cur), k):
+                n_new = n_cur - k
+                p_new = [0] + sorted(rng.choice(np.arange(1, L), n_new - 1, replace=False).tolist()) + [L]
+                kind, index = F.ftp_recovery_plan(p_cur, list(failed), p_new)
+                for j, items in enumerate(oracle.recovery_sources(p_cur, list(failed), p_new)):
+                    for u, src in items:
+                        assert kind[u] == code[src[0]], (p_cur, failed, p_new, u)
+                        want = j if src[0] == "local" else (src[1] if len(src) > 1 else 0)
+                        assert index[u] == want, (p_cur, failed, p_new, u)
+    for bad in ([0], [5], [2, 2]):
+        with pytest.raises(F.FtpError):
+            F.ftp_recovery_plan([0, 2, 4, 6, 8, 11], bad, [0, 3, 6, 11] if len(bad) == 2 else [0, 3, 6, 8, 11])
+    with pytest.raises(F.FtpError):
+        F.ftp_recovery_plan([0, 2, 4, 6, 8, 11], [1], [0, 3, 6, 11])          # one failure leaves four stages, not three
+
