@@ -163,10 +163,13 @@ def run_reference(args, wl):
             "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
-def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host):
+def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=None):
     """Config 5: train `steps` iterations; after every `repartition`-th the stage capacities are redrawn from U[1,10] and the
     partition re-chosen (Eq. 4 on the profiled layer times); after every `snapshot`-th each stage's weights are copied to
     the next stage's replica buffer (last stage -> central) and every stage's to the central pinned-host buffer.
+    fail = (iteration, stage): after that iteration the stage is declared lost (a host-side event; Sec. III-F), the
+    survivors take over at the partition Eq. 4 gives for their capacities, the lost units reload from the replicas of
+    the last replication tick, and the stage rejoins at the next repartition.
     Returns (total ms, per-iteration ms list, log of partitions)."""
     import numpy as np
     import torch
@@ -181,6 +184,8 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host):
     central = torch.empty(2 * total, dtype=torch.float32).pin_memory()                             # chain tail + global copy (host)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     log = []
+    last_caps = list(wl["caps"])
+    replicated_at = None                 # partition under which the replicas were last written
     torch.cuda.synchronize()
     ev[0].record()
     for it in range(steps):
@@ -199,8 +204,24 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host):
                     m.ftp_snapshot_weights(s, central[total + off:total + off + n])    # chain: last stage to the central node
                 m.ftp_snapshot_weights(s, central[off:off + n])                        # global: every stage to the central node
                 off += n
+            replicated_at = tuple(pts)
+        if fail and it + 1 == fail[0] and fail[1] < len(m.ftp_get_partition()) - 1:
+            pts = m.ftp_get_partition()
+            caps = [c for s, c in enumerate(last_caps[:len(pts) - 1]) if s != fail[1]]
+            new_pts, bott = F.ftp_choose_partition(layer_times, caps)
+            t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+            t0.record()
+            nxt = fail[1] + 1
+            chain = replicas[nxt][:sum(sizes[pts[fail[1]]:pts[fail[1] + 1]])] if nxt < len(pts) - 1 else \
+                central[total + sum(sizes[:pts[fail[1]]]):total + sum(sizes[:pts[fail[1] + 1]])]
+            counts = m.ftp_recover({fail[1]: chain if replicated_at == tuple(pts) else None}, new_pts, central[:total] if replicated_at else None)
+            t1.record()
+            torch.cuda.synchronize()
+            log.append(dict(after_iteration=it + 1, failed_stage=fail[1], points=new_pts, from_stage_replica_central=list(counts),
+                            recovery_ms=round(t0.elapsed_time(t1), 4), virtual_bottleneck_ms=round(bott * 1e3, 4)))
         if (it + 1) % dyn["repartition"] == 0:
             caps = rng.uniform(1.0, 10.0, n_st).tolist()
+            last_caps = caps
             pts, bott = F.ftp_choose_partition(layer_times, caps)
             moved = m.ftp_set_partition(pts)
             log.append(dict(after_iteration=it + 1, capacities=[round(c, 3) for c in caps], points=pts, moved_units=moved,
@@ -222,6 +243,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
     ap.add_argument("--points", default=None, help="comma-separated partition points; skips the profile-and-optimise step")
     ap.add_argument("--graph", type=int, default=1, help="1: time CUDA-graph replays of the step (default); 0: eager launches")
+    ap.add_argument("--fail", default=None, help="cfg5 only, ITERATION:STAGE: that stage is lost after that iteration and recovered from the replicas")
     ap.add_argument("--lean", action="store_true", help="timed region only: no end-to-end leg, no kernel trace (profiling captures)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -311,7 +333,8 @@ def main():
         if dynamic:
             lt = (fwd_s + bwd_s).tolist()
             barrier()
-            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, args.steps, False)
+            fail = tuple(int(v) for v in args.fail.split(":")) if args.fail else None
+            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, args.steps, False, fail)
             barrier()
             ms = reps.max_over_ranks(ms)
             tick = lambda i, p: (i + 1) % p == 0
@@ -320,7 +343,7 @@ def main():
             rep = [t for i, t in enumerate(per_it) if tick(i, dynamic["repartition"])]
             med = lambda v: round(statistics.median(v), 4) if v else None
             dyn_info = dict(ms_plain_iteration=med(plain), ms_snapshot_iteration=med(snap), ms_repartition_iteration=med(rep),
-                            repartitions=plog[:10], snapshot_bytes_per_tick=int(3 * 4 * sum(m.ftp_unit_param_span(u)[1] + m.ftp_unit_state_span(u)[1] for u in range(m.L))))
+                            repartitions=plog[:12], snapshot_bytes_per_tick=int(3 * 4 * sum(m.ftp_unit_param_span(u)[1] + m.ftp_unit_state_span(u)[1] for u in range(m.L))))
         else:
             ms = timed(step_dev, args.steps)
     launches = m.ftp_launch_count() - n0
