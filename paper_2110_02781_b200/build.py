@@ -13,7 +13,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libftpipe.so")
 OBJ = os.path.join(HERE, "_build")
-SOURCES = ["partition.cpp", "model.cu", "gemm_f32.cu", "elem.cu", "gemm_tc.cu", "gemm_tc32.cu", "noalloc.cu"]
+SOURCES = ["partition.cpp", "model.cu", "gemm_f32.cu", "elem.cu", "gemm_tc.cu", "gemm_tc32.cu", "stem.cu", "noalloc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC,-Wall,-ffp-contract=off", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

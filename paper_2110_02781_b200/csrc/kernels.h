@@ -66,6 +66,17 @@ size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
 // dW[Mo][No] = X[R][Mo]^T dY[R][No], the fixed-order second pass over the reduction slices included
 bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
 
+// ---- first convolution of an image network (stem.cu): 3 x 3, pad 1, stride 1 or 2, 3 input channels, 32 or 64
+// output channels, no bias or activation.  w is [3][3][3][cout] in T (float masters, or the bf16 shadow).
+// false: shape not taken, nothing launched.
+bool stem_conv_supported(const ConvGeom& g);
+size_t stem_wgrad_scratch_floats(const ConvGeom& g);
+template <typename T>
+bool stem_conv_fwd(const T* x, const T* w, T* y, const ConvGeom& g, cudaStream_t st);
+// dw [3][3][3][cout] float; scratch: stem_wgrad_scratch_floats(g) floats (one partial per block, added in block order)
+template <typename T>
+bool stem_conv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, cudaStream_t st);
+
 // ---- streaming kernels (elem.cu); T = float or __nv_bfloat16, arithmetic in float ----------------
 // Column reductions view a (M, C) tensor as (M/f, C*f) so that narrow tensors still fill whole
 // 128-byte lines; `fold` picks f.  Partials are doubles: [chunks][2][C*f].

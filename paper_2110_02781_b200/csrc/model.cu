@@ -257,6 +257,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
         } else if (is_contraction(o.d.kind)) {
             finp = std::max(finp, fin_part_doubles(o.Co, 1)); finc = std::max(finc, fin_counter_count(o.Co, 1));
             red = std::max(red, std::max(conv_wgrad_scratch_floats(o.g), conv_gemm_scratch_floats(o.g)));
+            if (o.d.act == FTP_ACT_NONE && o.b_off < 0) red = std::max(red, stem_wgrad_scratch_floats(o.g));
             red = std::max(red, tc32_wgrad_scratch_floats(Mout, o.C, o.Co));
             red = std::max(red, std::max(tc32_gemm_scratch_floats((int)Mout, o.Co, o.C), tc32_gemm_scratch_floats((int)Mout, o.C, o.Co)));
             if (m.cfg.precision == FTP_BF16) red = std::max(red, std::max(tc_wgrad_scratch_floats(Mout, o.C, o.Co), tc_wgrad3x3_scratch_floats(Mout, o.C, o.Co)));
@@ -373,7 +374,8 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                                               m->tc_err, st, stats_req);
                     if (!tc) next_ps.entries = 0;
                     if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_FWD;
-                    if (!tc) conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
+                    const bool stem = !tc && o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_fwd<float>((const float*)in, ar.w + o.w_off, (float*)out, o.g, st);
+                    if (!tc && !stem) conv_fwd_f32((const float*)in, ar.w + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (float*)out, m->red_scratch, o.g, o.d.act, st);
                 } else if constexpr (!std::is_same<T, float>::value) {
                     if (o.d.kind == FTP_FC) {           // the classifier runs in float on a widened copy of its input
                         Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, o.in_elems * 2.0 + (o.out_elems + o.w_cnt) * 4.0, fl, 2);
@@ -386,6 +388,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                         if (!tc && is_3x3_op(o) && tc_conv3x3_supported(o.N, o.H, o.W, o.C, o.Co, in, ar.wbt + o.w_off, out, nullptr))
                             tc = tc_conv3x3((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, o.N, o.H, o.W, o.C, o.Co, 0, m->tc_err, st);
                         if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_FWD_BF16_SIMT;
+                        if (!tc && o.d.act == FTP_ACT_NONE && o.b_off < 0) tc = stem_conv_fwd<T>((const T*)in, ar.wb + o.w_off, (T*)out, o.g, st);
                         if (!tc) conv_fwd_bf16_simt((const T*)in, ar.wb + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (T*)out, o.g, o.d.act, st);
                     }
                 }
@@ -523,7 +526,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                       const bool tc = is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr) &&
                                       tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws);
                       if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
-                      if (!tc) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
+                      const bool stem = !tc && !widened && o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_wgrad<float>(x, d, gr + o.w_off, rs, o.g, ws);
+                      if (!tc && !stem) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
                       forked(i, d); }
                     if (gi) {
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
@@ -556,7 +560,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                       if (splits > 1) split_reduce_f32(rs, splits, o.w_cnt, gr + o.w_off, ws);
                       if (splits == 0) {
                           if (sc.slot) sc.slot->rec.kernel = K_CONV_WGRAD_BF16_SIMT;
-                          conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, rs, o.g, ws);
+                          const bool stem = o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_wgrad<T>((const T*)in, d, gr + o.w_off, rs, o.g, ws);
+                          if (!stem) conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, rs, o.g, ws);
                       }
                       forked(i, d); }
                     if (gi) {

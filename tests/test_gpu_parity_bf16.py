@@ -130,6 +130,8 @@ def test_mobilenet_bf16_split_equals_unsplit_bitwise():
 # ---- one layer at a time: every gradient at the max-abs tolerance ------------------------------------------
 LAYER_CASES = [  # kind, hw, cin, cout, k, stride, act, batch
     ("CONV2D", 16, 3, 32, 3, 2, 2, 8),        # MobileNetV2 stem (3 input channels, stride 2)
+    ("CONV2D", 15, 3, 32, 3, 2, 2, 3),        # the same on an odd map (15 -> 8), pixel count not a multiple of 32
+    ("CONV2D", 9, 3, 64, 3, 1, 1, 5),         # VGG stem (3 -> 64, stride 1), 405 pixels
     ("CONV2D", 16, 32, 96, 1, 1, 2, 16),      # pointwise expand
     ("CONV2D", 16, 96, 24, 1, 1, 0, 16),      # pointwise project (no activation)
     ("CONV2D", 7, 160, 960, 1, 1, 2, 8),      # late expand, odd map size

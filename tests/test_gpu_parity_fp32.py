@@ -202,6 +202,14 @@ def test_edge_shapes_batch_one_odd_channels():
         one_step_case((ls, cfg), 25, [0, 1, 2, 3])
 
 
+def test_first_convolution_kernels_on_ragged_maps():
+    """3 -> 32 and 3 -> 64 first convolutions take the dedicated kernels: odd map sizes, stride 1 and 2, pixel counts
+    that are not multiples of the 32-pixel chunks of the weight gradient."""
+    table = [(1, 8, 1, 1), (6, 16, 1, 2)]
+    for batch, hw, stem_c, cifar in ((3, 9, 32, True), (2, 11, 64, False), (5, 8, 32, False)):
+        one_step_case(synth.mobilenetv2(batch, hw, 5, 0, cifar, table, stem_c=stem_c, last_c=32), 27, [0, 2, 5])
+
+
 def test_conv1d_ragged_lengths():
     for batch, t, width in ((3, 50, 12), (1, 5, 4), (5, 131, 20)):
         one_step_case(synth.har_cnn(batch, 9, t, width, 6), 26, [0, 2, 5])
