@@ -47,6 +47,10 @@ def workload(name, batch=None):
         ls, cfg = synth.vgg16(b, 32, 10, 1)
         return dict(index=3, name=f"config 4: VGG-16-style 32x32x3 batch {b} bf16, 3 stages from the partition optimiser", layers=ls,
                     cfg=cfg, caps=[1.0, 1.0, 1.0], points=None)
+    if name == "cl8":
+        ls, cfg = synth.continual_mbv2(batch or 8)
+        return dict(index=5, name=f"continuous-learning shape (Sec. IV-F): MobileNetV2 28x28x1 batch {batch or 8} fp32, lr 0.00625, 3 stages at equal capacity",
+                    layers=ls, cfg=cfg, caps=[1.0, 1.0, 1.0], points=None)
     ls, cfg = synth.mobilenetv2(batch or 128, 32, 10, 0, True)
     return dict(index=1, name=f"config 2: MobileNetV2 32x32x3 batch {batch or 128} fp32, 3 stages at equal capacity", layers=ls,
                 cfg=cfg, caps=[1.0, 1.0, 1.0], points=None)
@@ -64,7 +68,7 @@ STEP_WORK = {"cfg2": (11.73e9 / 128, (63.1e9 + 4.5e9) / 128), "cfg3": (12.00e9 /
 # pass (profiles/ncu_tc32_kernels_cfg2_b128.md).  Valid only for the default batch and while the kernel source is the
 # one the counters were taken on: the entry carries the sha256 of that source file.
 NCU_TRAFFIC = {("cfg2", "tc_gemm_tf32x3_wgrad"): dict(bytes_per_step=1.038e9, source="paper_2110_02781_b200/csrc/gemm_tc32.cu",
-                                                     sha256="05a5819bd7ddc8f56e2b30af64a77cba0becc68bacda04293daf7a6e1b390be8")}
+                                                     sha256="2ff8697e2ab355217235afd74558155c659b954efed3f231d56f06b6a9a86f72")}
 
 
 def ncu_traffic(wl_key, kernel, default_batch):
@@ -139,7 +143,7 @@ def run_reference(args, wl):
     except Exception:
         cores = os.cpu_count() or 1
     ls, cfg = wl["layers"], dict(wl["cfg"])
-    sample_batch = min(cfg["batch"], {0: cfg["batch"], 1: 16, 2: 2, 3: 8, 4: 2}[wl["index"]])
+    sample_batch = min(cfg["batch"], {0: cfg["batch"], 1: 16, 2: 2, 3: 8, 4: 2, 5: cfg["batch"]}[wl["index"]])
     cfg["batch"] = sample_batch
     om = oracle.OracleModel(ls, cfg, synth.init_params(wl["index"], ls), synth.init_state(ls))
     L = om.L
@@ -185,6 +189,11 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     log = []
     last_caps = list(wl["caps"])
+    factors = rng.uniform(1.0, 10.0, n_st).tolist()              # slowdown factors of the simulated devices in the current window
+    closed_loop = not on_host
+    window = []
+    if closed_loop:
+        m.ftp_stage_timing_enable(True)
     replicated_at = None                 # partition under which the replicas were last written
     torch.cuda.synchronize()
     ev[0].record()
@@ -219,15 +228,32 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=
             torch.cuda.synchronize()
             log.append(dict(after_iteration=it + 1, failed_stage=fail[1], points=new_pts, from_stage_replica_central=list(counts),
                             recovery_ms=round(t0.elapsed_time(t1), 4), virtual_bottleneck_ms=round(bott * 1e3, 4)))
+        if closed_loop and (it + 1) % 10 == 0:                  # a worker reports its batch time now and then (Sec. III-B)
+            window.append(m.ftp_stage_times())
         if (it + 1) % dyn["repartition"] == 0:
-            caps = rng.uniform(1.0, 10.0, n_st).tolist()
-            last_caps = caps
+            n_now = len(m.ftp_get_partition()) - 1
+            reports = [w for w in window if len(w) == n_now]
+            if closed_loop and reports:
+                # Eq. 1-3 on what the workers reported over the window: reported time = device time of the stage x the
+                # slowdown factor its simulated device had; the central node's own layer times are the profile x its
+                # factor, so C_0 = 1 and C_i comes out near f_i / f_0.  A stage that rejoins has reported nothing yet.
+                mean = [sum(w[s] for w in reports) / len(reports) for s in range(n_now)]
+                central_times = [t * factors[0] for t in layer_times]
+                caps = F.ftp_estimate_capacity(central_times, m.ftp_get_partition(), [mean[s] * factors[s] for s in range(n_now)])
+                caps += [factors[s] / factors[0] for s in range(n_now, n_st)]
+            else:
+                caps = list(factors)
+            window = []
             pts, bott = F.ftp_choose_partition(layer_times, caps)
             moved = m.ftp_set_partition(pts)
-            log.append(dict(after_iteration=it + 1, capacities=[round(c, 3) for c in caps], points=pts, moved_units=moved,
-                            virtual_bottleneck_ms=round(bott * 1e3, 4)))
+            log.append(dict(after_iteration=it + 1, capacities=[round(c, 3) for c in caps], factors=[round(f, 3) for f in factors], points=pts,
+                            moved_units=moved, virtual_bottleneck_ms=round(bott * 1e3, 4)))
+            last_caps = list(caps)
+            factors = rng.uniform(1.0, 10.0, n_st).tolist()      # the simulated devices change speed for the next window
         ev[it + 1].record()
     torch.cuda.synchronize()
+    if closed_loop:
+        m.ftp_stage_timing_enable(False)
     per_it = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     return ev[0].elapsed_time(ev[steps]), per_it, log
 
@@ -238,7 +264,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None, help="timed steps (default 50; 500 for cfg5)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cl8"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
     ap.add_argument("--points", default=None, help="comma-separated partition points; skips the profile-and-optimise step")

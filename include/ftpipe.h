@@ -179,6 +179,15 @@ ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, in
 ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void* sample_in, const int32_t* labels,
                               double* fwd_s, double* bwd_s, int64_t* out_bytes, void* stream);
 
+/* Sec. III-B / III-D: every worker reports the execution time of its batches, from which the central
+ * node estimates capacities (Eq. 1).  With stage timing on, ftp_train_step brackets every stage's
+ * forward and backward with events (issued eagerly: not for steps replayed from a CUDA graph);
+ * ftp_stage_times waits for the last such step and returns forward + backward device seconds per
+ * stage of the partition it ran under (seconds: max_stages doubles; *n_stages: how many are set).
+ * The optimiser step is not included, as in ftp_profile_layers.  FTP_ESTATE if no step was timed. */
+ftp_status ftp_stage_timing_enable(ftp_model* m, int32_t on);
+ftp_status ftp_stage_times(ftp_model* m, double* seconds, int32_t* n_stages);
+
 /* Eq. 1-3: capacities[i] = stage_times[i] / sum of layer_times over stage i; [0] = 1.0. */
 ftp_status ftp_estimate_capacity(const double* layer_times, int32_t L, const int32_t* points, int32_t N,
                                  const double* stage_times, double* capacities);

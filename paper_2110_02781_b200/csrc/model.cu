@@ -660,16 +660,22 @@ ftp_status sgd_range(ftp_model* m, int a, int b, float lr, float* snap_dev, floa
 template <typename T>
 ftp_status train_step_t(ftp_model* m, const void* x, const int32_t* labels, float lr, cudaStream_t st) {
     const void* act = x;
+    const bool timing = m->stage_timing && (int)m->ev_sf.size() > m->n_stages;
+    if (timing) m->timed_stages = 0;
     for (int s = 0; s < m->n_stages; ++s) {
         const int a = m->points[s], b = m->points[s + 1];
+        if (timing) cudaEventRecord(m->ev_sf[s], st);
         ftp_status r = fwd_range<T>(m, a, b, act, nullptr, b == m->L ? labels : nullptr, b == m->L ? m->loss_dev : nullptr, st);
         if (r != FTP_OK) return r;
         act = m->cur_out[m->unit_last[b - 1]];
     }
+    if (timing) cudaEventRecord(m->ev_sf[m->n_stages], st);
     for (int s = m->n_stages - 1; s >= 0; --s) {
+        if (timing) cudaEventRecord(m->ev_sb[s + 1], st);
         ftp_status r = bwd_range<T>(m, m->points[s], m->points[s + 1], nullptr, nullptr, true, st);
         if (r != FTP_OK) return r;
     }
+    if (timing) { cudaEventRecord(m->ev_sb[0], st); m->timed_stages = m->n_stages; }
     for (int s = 0; s < m->n_stages; ++s) {
         ftp_status r = sgd_range(m, m->points[s], m->points[s + 1], lr, nullptr, nullptr, st);
         if (r != FTP_OK) return r;
@@ -750,6 +756,8 @@ extern "C" void ftp_destroy_model(ftp_model* m) {
     for (auto& t : m->tr) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
     for (auto e : m->ev_f) cudaEventDestroy(e);
     for (auto e : m->ev_b) cudaEventDestroy(e);
+    for (auto e : m->ev_sf) cudaEventDestroy(e);
+    for (auto e : m->ev_sb) cudaEventDestroy(e);
     for (auto e : m->ev_fork) cudaEventDestroy(e);
     for (auto e : m->ev_side) cudaEventDestroy(e);
     if (m->side) cudaStreamDestroy(m->side);
@@ -907,6 +915,31 @@ extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t*
         memcpy(&code, m->pinned + 1, 4);
         FTP_REQUIRE(code == 0, FTP_ETIMEOUT, "train_step: a bounded wait inside a tensor-core kernel ran out (code %d)", code);
     }
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_stage_timing_enable(ftp_model* m, int32_t on) {
+    FTP_REQUIRE(m, FTP_EINVAL, "stage_timing_enable: null model");
+    const size_t need = (size_t)m->cfg.max_stages + 1;
+    while (on && m->ev_sf.size() < need) { cudaEvent_t e; CUDA_OK(cudaEventCreate(&e)); m->ev_sf.push_back(e); }
+    while (on && m->ev_sb.size() < need) { cudaEvent_t e; CUDA_OK(cudaEventCreate(&e)); m->ev_sb.push_back(e); }
+    m->stage_timing = on != 0;
+    m->timed_stages = 0;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_stage_times(ftp_model* m, double* seconds, int32_t* n_stages) {
+    FTP_REQUIRE(m && seconds && n_stages, FTP_EINVAL, "stage_times: null argument");
+    FTP_REQUIRE(m->timed_stages > 0, FTP_ESTATE, "stage_times: no training step has run since stage timing was switched on");
+    const int n = m->timed_stages;
+    CUDA_OK(cudaEventSynchronize(m->ev_sb[0]));
+    for (int s = 0; s < n; ++s) {
+        float f = 0.f, b = 0.f;
+        CUDA_OK(cudaEventElapsedTime(&f, m->ev_sf[s], m->ev_sf[s + 1]));
+        CUDA_OK(cudaEventElapsedTime(&b, m->ev_sb[s + 1], m->ev_sb[s]));
+        seconds[s] = ((double)f + (double)b) * 1e-3;
+    }
+    *n_stages = n;
     return FTP_OK;
 }
 

@@ -84,6 +84,10 @@ struct ftp_model {
     std::vector<const void*> stage_in;            // act_in of the range starting at op i
     std::vector<void*> cur_out;                   // resolved output pointer of op i
     std::vector<char> fwd_done;
+    // per-stage timing of ftp_train_step (Sec. III-B: a worker reports the execution time of its batch)
+    bool stage_timing = false;
+    std::vector<cudaEvent_t> ev_sf, ev_sb;        // forward / backward boundaries, max_stages + 1 each
+    int timed_stages = 0;                         // stages of the last timed step (0: none yet)
     const int32_t* cur_labels;
     // trace
     bool trace;

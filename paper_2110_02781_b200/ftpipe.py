@@ -64,6 +64,8 @@ _SIGS = {
     "ftp_choose_partition": [_P(C.c_double), _i32, _P(C.c_double), _i32, _P(C.c_double), _P(C.c_double), _P(_i32),
                              _P(C.c_double)],
     "ftp_redistribution_plan": [_P(_i32), _i32, _P(_i32), _i32, _i32, _i32, _i32, _P(_i32), _P(_i32)],
+    "ftp_stage_timing_enable": [_vp, _i32],
+    "ftp_stage_times": [_vp, _P(C.c_double), _P(_i32)],
     "ftp_recovery_plan": [_P(_i32), _i32, _P(_i32), _i32, _P(_i32), _i32, _P(_i32), _P(_i32)],
     "ftp_recover": [_vp, _vp, _i32, _vp, _sz, _P(_i32), _i32, _P(_i32), _vp],
     "ftp_set_partition": [_vp, _P(_i32), _i32, _P(_i32), _vp],
@@ -283,6 +285,16 @@ class Model:
         _check(lib.ftp_train_step(self.h, _ptr(x), _ptr(labels), int(inputs_on_host), lr,
                                   C.byref(loss) if want_loss else None, _stream(stream)))
         return loss.value if want_loss else None
+
+    def ftp_stage_timing_enable(self, on):
+        _check(lib.ftp_stage_timing_enable(self.h, int(on)))
+
+    def ftp_stage_times(self):
+        """Forward + backward device seconds of every stage in the last timed ftp_train_step."""
+        t = (C.c_double * self.cfg["max_stages"])()
+        n = _i32()
+        _check(lib.ftp_stage_times(self.h, t, C.byref(n)))
+        return list(t[:n.value])
 
     def ftp_profile_layers(self, reps, sample_in, labels, stream=None):
         f, b = np.zeros(self.L), np.zeros(self.L)

@@ -62,12 +62,12 @@ def _inverted_residual(ls, unit, cin, cout, expand, stride):
 
 
 def mobilenetv2(batch, hw, n_classes, precision, cifar, table=None, stem_c=32, last_c=1280,
-                lr=0.01, momentum=0.9, weight_decay=4e-5):
+                lr=0.01, momentum=0.9, weight_decay=4e-5, in_c=3):
     """MobileNetV2, width 1.0.  `cifar` selects stride 1 for the stem and the 24-channel group."""
     if table is None:
         table = [(1, 16, 1, 1), (6, 24, 2, 1 if cifar else 2), (6, 32, 3, 2), (6, 64, 4, 2),
                  (6, 96, 3, 1), (6, 160, 3, 2), (6, 320, 1, 1)]
-    ls = [_L(0, "CONV2D", 3, stem_c, 3, 1 if cifar else 2, 1), _L(0, "BN", stem_c, stem_c, act="RELU6")]
+    ls = [_L(0, "CONV2D", in_c, stem_c, 3, 1 if cifar else 2, 1), _L(0, "BN", stem_c, stem_c, act="RELU6")]
     unit, c = 1, stem_c
     for t, cout, n, s in table:
         for i in range(n):
@@ -80,8 +80,14 @@ def mobilenetv2(batch, hw, n_classes, precision, cifar, table=None, stem_c=32, l
     ls.append(_L(unit, "GAP", last_c, last_c))
     ls.append(_L(unit, "FC", last_c, n_classes, 1, 1, 0, "NONE", 1))
     ls.append(_L(unit, "SOFTMAX_CE", n_classes, n_classes))
-    return ls, config(batch, 3, hw, hw, n_classes, precision, lr=lr, momentum=momentum,
+    return ls, config(batch, in_c, hw, hw, n_classes, precision, lr=lr, momentum=momentum,
                       weight_decay=weight_decay)
+
+
+def continual_mbv2(batch=8, hw=28, n_classes=10, precision=0):
+    """The continuous-learning shape of Sec. IV-F ("Continuous Learning Evaluation"): MobileNetV2 on 28 x 28 x 1 images at batch 8 with the learning rate
+    scaled to that batch (0.1 * 8 / 128 = 0.00625); strides as in the 32 x 32 variant (final map 4 x 4)."""
+    return mobilenetv2(batch, hw, n_classes, precision, True, lr=0.00625, in_c=1)
 
 
 def tiny_mbv2(batch=4, hw=8, n_classes=5, precision=0, momentum=0.9, weight_decay=4e-5):

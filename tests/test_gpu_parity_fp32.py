@@ -163,29 +163,41 @@ def test_full_size_mobilenet_cifar_batch_128():
     one_step_case(net, 1, [0, 7, 14, 20], params="safe", wgrad_tol=5e-3)
 
 
-def test_full_size_real_init_forward_and_split_invariance():
-    """Config 2 with its real (Kaiming) initialisation: the forward results, which are continuous in
-    the activation decisions, are held to 1e-4; with ~2e8 activations some lie within float32
-    rounding of a kink, so gradients are checked by what is unique there: split == unsplit bitwise."""
-    import oracle
-    ls, cfg = synth.mobilenetv2(128, 32, 10, 0, True)
-    om = make_oracle(ls, cfg, 1)
-    x, y = synth.make_batch(1, cfg)
+def real_init_case(net, idx, pts, lr):
+    """Real (Kaiming) initialisation at full size: the forward results, which are continuous in the activation
+    decisions, are held to 1e-4; with millions of activations some lie within float32 rounding of a kink, so
+    gradients are checked by what is unique there: split == unsplit bitwise."""
+    ls, cfg = net
+    om = make_oracle(ls, cfg, idx)
+    x, y = synth.make_batch(idx, cfg)
     om.forward(0, om.L, x, y)
-    ref, alt = make_gpu(ls, cfg, 1), make_gpu(ls, cfg, 1)
-    pts = [0, 7, 14, 20]
+    ref, alt = make_gpu(ls, cfg, idx), make_gpu(ls, cfg, idx)
     alt.ftp_set_partition(pts)
     xd, yd = to_dev(x), to_dev(y)
-    l0 = ref.ftp_train_step(xd, yd, 0.01)
-    l1, acts, _ = gpu_step_split(alt, pts, xd, yd, 0.01)
+    l0 = ref.ftp_train_step(xd, yd, lr)
+    l1, acts, _ = gpu_step_split(alt, pts, xd, yd, lr)
     assert l0 == l1 and abs(l0 - om.loss) <= TOL_FP32 * om.loss
     assert rel_err(ref.ftp_get_logits(), om.logits) <= TOL_FP32
-    for k, u in ((1, 6), (2, 13)):
+    for k in range(1, len(pts) - 1):
+        u = pts[k] - 1
         assert rel_err(acts[k].cpu().numpy(), om.out[max(i for i, l in enumerate(ls) if l.unit == u)]) <= TOL_FP32
     for u in range(ref.L):
         assert rel_err(ref.ftp_get_tensor(F.T_STATE, u), om.unit_state(u)) <= TOL_FP32
         for which in (F.T_WEIGHTS, F.T_GRADS, F.T_MOMENTUM):
             assert np.array_equal(ref.ftp_get_tensor(which, u), alt.ftp_get_tensor(which, u))
+    ref.close(); alt.close()
+
+
+def test_full_size_real_init_forward_and_split_invariance():
+    """Config 2 with its real initialisation, 3 stages."""
+    real_init_case(synth.mobilenetv2(128, 32, 10, 0, True), 1, [0, 7, 14, 20], 0.01)
+
+
+def test_continuous_learning_shape_batch_8():
+    """MobileNetV2 on 28 x 28 x 1 images at batch 8 (the continuous-learning set-up of Sec. IV-F), full network, 3 stages:
+    the small-batch regime in which every layer is a few tiles at most and the one-channel first convolution takes the
+    generic kernels."""
+    real_init_case(synth.continual_mbv2(), 6, [0, 7, 14, 20], 0.00625)
 
 
 def test_edge_shapes_batch_one_odd_channels():

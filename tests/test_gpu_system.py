@@ -259,3 +259,40 @@ def test_recover_refuses_what_it_cannot_restore():
     assert gm.ftp_get_partition() == before
     gm.close()
 
+
+def test_stage_times_feed_the_capacity_estimate():
+    """Sec. III-B / Eq. 1-3 in a closed loop: the per-stage times that ftp_train_step reports, scaled by simulated
+    slowdown factors, must give back those factors (relative to the central node) through ftp_estimate_capacity and
+    the profiled layer times, to within the noise of timing short kernels."""
+    import torch
+    ls, cfg = synth.mobilenetv2(32, 32, 10, 0, True)
+    gm = make_gpu(ls, dict(cfg, max_stages=4), 83)
+    x, y = synth.make_batch(83, cfg)
+    xd, yd = to_dev(x), to_dev(y)
+    pts = [0, 5, 10, 15, gm.L]
+    gm.ftp_set_partition(pts)
+    with pytest.raises(F.FtpError):
+        gm.ftp_stage_times()                                  # timing is off
+    fwd, bwd, _ = gm.ftp_profile_layers(5, xd, yd)
+    layer_times = (fwd + bwd).tolist()
+    gm.ftp_stage_timing_enable(True)
+    with pytest.raises(F.FtpError):
+        gm.ftp_stage_times()                                  # no step timed yet
+    for _ in range(3):
+        gm.ftp_train_step(xd, yd, 0.01, want_loss=False)
+    reports = []
+    for _ in range(5):
+        gm.ftp_train_step(xd, yd, 0.01, want_loss=False)
+        reports.append(gm.ftp_stage_times())
+    assert all(len(r) == 4 and min(r) > 0 for r in reports)
+    mean = np.mean(reports, axis=0)
+    factors = [2.0, 1.0, 8.0, 4.0]
+    caps = F.ftp_estimate_capacity([t * factors[0] for t in layer_times], pts, [m_ * f for m_, f in zip(mean, factors)])
+    assert caps[0] == 1.0
+    for c, f in zip(caps[1:], factors[1:]):
+        assert 0.5 * f / factors[0] <= c <= 2.0 * f / factors[0], (caps, factors)
+    gm.ftp_stage_timing_enable(False)
+    with pytest.raises(F.FtpError):
+        gm.ftp_stage_times()
+    gm.close()
+
