@@ -127,6 +127,59 @@ def test_mobilenet_bf16_split_equals_unsplit_bitwise():
             assert np.array_equal(a.ftp_get_tensor(which, u), b.ftp_get_tensor(which, u))
 
 
+def full_size_case(net, idx, pts):
+    """A benchmark network at (or near) its full size in the launch configuration the benchmark times.
+    (i) Every unit on its own, fed the oracle's input of that unit: output against the oracle at the bf16 tolerance,
+    element by element (what differs is single bf16 steps where float32 and exact accumulation round apart).
+    (ii) The chained network: loss and BN running statistics at the tolerance; the logits only loosely, because a
+    randomly initialised deep ReLU + BN network amplifies those single steps by about 1.7x per layer (measured on the
+    VGG: 1e-5 after the first unit, 2e-2 after the thirteenth, with every unit correct to 2e-4 in isolation).
+    (iii) The backward pass and update by what is unique at this size: the staged run equals the single-stage run
+    bit for bit."""
+    import torch
+    from oracle.model import round_bf16
+    ls, cfg = net
+    om = oracle.OracleModel(ls, cfg, synth.init_params(idx, ls), synth.init_state(ls))
+    x, y = synth.make_batch(idx, cfg)
+    x = round_bf16(x)
+    om.forward(0, om.L, x, y)
+    probe, ref, alt = F.Model(ls, cfg), F.Model(ls, cfg), F.Model(ls, cfg)
+    for m in (probe, ref, alt):
+        m.load_params(synth.init_params(idx, ls), synth.init_state(ls))
+    for u in range(probe.L - 1):
+        ops = [i for i, l in enumerate(ls) if l.unit == u]
+        unit_in = x if u == 0 else om.out[ops[0] - 1]
+        shp, _ = probe.ftp_unit_output_shape(u)
+        out = torch.empty(shp, dtype=torch.bfloat16, device="cuda")
+        probe.ftp_run_stage_forward(u, u + 1, dev_bf16(unit_in), out)
+        torch.cuda.synchronize()
+        assert rel_err(host(out), om.out[ops[-1]]) <= TOL_BF16, f"unit {u} on the oracle's input"
+        assert l2_err(host(out), om.out[ops[-1]]) <= 1e-3, f"unit {u} on the oracle's input (L2)"
+    probe.close()
+    alt.ftp_set_partition(pts)
+    xd, yd = dev_bf16(x), torch.from_numpy(y).cuda()
+    l0, l1 = ref.ftp_train_step(xd, yd, 0.01), alt.ftp_train_step(xd, yd, 0.01)
+    assert l0 == l1 and abs(l0 - om.loss) <= TOL_BF16 * max(abs(om.loss), 1.0)
+    assert l2_err(ref.ftp_get_logits(), om.logits) <= 5e-2
+    for u in range(ref.L):
+        assert rel_err(ref.ftp_get_tensor(F.T_STATE, u), om.unit_state(u)) <= TOL_BF16, f"running statistics of unit {u}"
+        for which in (F.T_WEIGHTS, F.T_GRADS, F.T_MOMENTUM):
+            assert np.array_equal(ref.ftp_get_tensor(which, u), alt.ftp_get_tensor(which, u)), f"unit {u}: the split changed a bit"
+    ref.close(); alt.close()
+
+
+def test_full_size_vgg16_batch_256():
+    """Config 4 as benchmarked: VGG-16-style, 32 x 32 x 3, batch 256, 3 stages."""
+    full_size_case(synth.vgg16(256, 32, 10, 1), 3, [0, 3, 8, 14])
+
+
+def test_mobilenet_224_full_resolution():
+    """Config 3's network at its full 224 x 224 resolution and 4 stages (every tile count and ragged edge of the
+    benchmark's launches per image), at batch 8 of 64 to keep the float64 oracle's memory in bounds."""
+    ls, cfg = synth.mobilenetv2(8, 224, 1000, 1, False)
+    full_size_case((ls, dict(cfg, max_stages=5)), 2, [0, 1, 3, 7, 20])
+
+
 # ---- one layer at a time: every gradient at the max-abs tolerance ------------------------------------------
 LAYER_CASES = [  # kind, hw, cin, cout, k, stride, act, batch
     ("CONV2D", 16, 3, 32, 3, 2, 2, 8),        # MobileNetV2 stem (3 input channels, stride 2)
