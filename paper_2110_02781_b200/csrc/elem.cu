@@ -112,9 +112,11 @@ inline unsigned flat_blocks(long long work, int threads) {
 // grid (column tiles of 32*V, row chunks); block (32, 8).  NS sums per column.
 // copies > 1 (then copies * C == 32 * V): the copies of a channel inside the column tile are added up as well, in copy
 // order, and the partial sums are laid out [chunk][NS][cols / copies].
+template <typename T, int V, int NS>
+__device__ __forceinline__ void fold_finish(float (&s)[NS][V], int cols, double* partial, int C, int copies);
+
 template <typename T, int V, int NS, typename F>
 __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chunk, double* partial, F body, int C = 0, int copies = 1) {
-    __shared__ float sh[NS][8][32 * V];
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     const int r0 = blockIdx.y * rows_per_chunk, r1 = min(rows, r0 + rows_per_chunk);
     float s[NS][V];
@@ -124,6 +126,37 @@ __device__ __forceinline__ void fold_reduce(int rows, int cols, int rows_per_chu
         for (int e = 0; e < V; ++e) s[a][e] = 0.f;
     if (col < cols)
         for (int r = r0 + threadIdx.y; r < r1; r += 8) body((long long)r * cols + col, col, s);
+    fold_finish<T, V, NS>(s, cols, partial, C, copies);
+}
+
+// The same reduction with the loads of two rows issued before either row is used: a thread that fetches 8 or 16
+// bytes per tensor and row has too few bytes in flight to cover the memory latency otherwise (Little's law: four
+// blocks of 256 threads per SM x 8 bytes x 2 tensors is 2.4 MB over the chip, a third of what 6.5 TB/s needs).
+// The rows are still added in the order r, r + 8, r + 16, ..., so the sums are bit-identical to fold_reduce's.
+template <typename T, int V, int NS, typename R, typename FL, typename FU>
+__device__ __forceinline__ void fold_reduce2(int rows, int cols, int rows_per_chunk, double* partial, FL load, FU use, int C = 0, int copies = 1) {
+    const int col = (blockIdx.x * 32 + threadIdx.x) * V;
+    const int r0 = blockIdx.y * rows_per_chunk, r1 = min(rows, r0 + rows_per_chunk);
+    float s[NS][V];
+#pragma unroll
+    for (int a = 0; a < NS; ++a)
+#pragma unroll
+        for (int e = 0; e < V; ++e) s[a][e] = 0.f;
+    if (col < cols)
+        for (int r = r0 + threadIdx.y; r < r1; r += 16) {
+            R a, b;
+            const bool two = r + 8 < r1;
+            load((long long)r * cols + col, a);
+            if (two) load((long long)(r + 8) * cols + col, b);
+            use(a, s);
+            if (two) use(b, s);
+        }
+    fold_finish<T, V, NS>(s, cols, partial, C, copies);
+}
+
+template <typename T, int V, int NS>
+__device__ __forceinline__ void fold_finish(float (&s)[NS][V], int cols, double* partial, int C, int copies) {
+    __shared__ float sh[NS][8][32 * V];
 #pragma unroll
     for (int a = 0; a < NS; ++a)
 #pragma unroll
@@ -345,17 +378,17 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
     float sc[V], sh[V], mu[V], ml[V], rs[V];
     if (col < cols) { const int c = col % C; ldtab<V>(scale + c, sc); ldtab<V>(shift + c, sh); ldtab<V>(mean + c, mu); ldtab<V>(mean_lo + c, ml); ldtab<V>(rstd + c, rs); }
-    fold_reduce<T, V, 2>(rows, cols, rpc, partial, [&](long long off, int, float (&s)[2][V]) {
-        float d[V], v[V];
-        ldv<V>(dz + off, d);
-        ldv<V>(y + off, v);
+    struct Row { float d[V], v[V]; };
+    fold_reduce2<T, V, 2, Row>(rows, cols, rpc, partial,
+        [&](long long off, Row& q) { ldv<V>(dz + off, q.d); ldv<V>(y + off, q.v); },
+        [&](const Row& q, float (&s)[2][V]) {
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-            const float g = act_pass(bn_z(v[e], mu[e], ml[e], sc[e], sh[e]), act) ? d[e] : 0.f;
-            s[0][e] += g;
-            s[1][e] = fmaf(g, ((v[e] - mu[e]) - ml[e]) * rs[e], s[1][e]);
-        }
-    }, C, copies);
+            for (int e = 0; e < V; ++e) {
+                const float g = act_pass(bn_z(q.v[e], mu[e], ml[e], sc[e], sh[e]), act) ? q.d[e] : 0.f;
+                s[0][e] += g;
+                s[1][e] = fmaf(g, ((q.v[e] - mu[e]) - ml[e]) * rs[e], s[1][e]);
+            }
+        }, C, copies);
 }
 
 __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double inv_M,
@@ -395,28 +428,35 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const T* __restrict__
     ldtab<V>(coef + c, ca); ldtab<V>(coef + C + c, bh); ldtab<V>(coef + 2 * C + c, bl);
     ldtab<V>(coef + 3 * C + c, ch); ldtab<V>(coef + 4 * C + c, cl);
     const int r0 = blockIdx.y * rpc, r1 = min(rows, r0 + rpc);
-    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
-        const long long off = (long long)r * cols + col;
-        float d[V], v[V], o[V];
-        ldv<V>(dz + off, d);
-        ldv<V>(y + off, v);
+    // two rows per trip, all their loads issued before the first use (see fold_reduce2)
+    for (int r = r0 + threadIdx.y; r < r1; r += 16) {
+        const bool two = r + 8 < r1;
+        const long long off[2] = {(long long)r * cols + col, (long long)(r + 8) * cols + col};
+        float d[2][V], v[2][V], a[2][V];
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-            const float cen = (v[e] - mu[e]) - ml[e];
-            const float g = act_pass(fmaf(cen, sc[e], sh[e]), act) ? d[e] : 0.f;
-            const float xh = cen * rs[e];
-            float t = (g - bh[e]) - bl[e];
-            t = fmaf(-xh, ch[e], t);
-            t = fmaf(-xh, cl[e], t);
-            o[e] = ca[e] * t;
-        }
-        if (addend) {
-            float a[V];
-            ldv<V>(addend + off, a);
+        for (int k = 0; k < 2; ++k)
+            if (k == 0 || two) {
+                ldv<V>(dz + off[k], d[k]);
+                ldv<V>(y + off[k], v[k]);
+                if (addend) ldv<V>(addend + off[k], a[k]);
+            }
 #pragma unroll
-            for (int e = 0; e < V; ++e) o[e] += a[e];
-        }
-        stv<V>(dy + off, o);
+        for (int k = 0; k < 2; ++k)
+            if (k == 0 || two) {
+                float o[V];
+#pragma unroll
+                for (int e = 0; e < V; ++e) {
+                    const float cen = (v[k][e] - mu[e]) - ml[e];
+                    const float g = act_pass(fmaf(cen, sc[e], sh[e]), act) ? d[k][e] : 0.f;
+                    const float xh = cen * rs[e];
+                    float t = (g - bh[e]) - bl[e];
+                    t = fmaf(-xh, ch[e], t);
+                    t = fmaf(-xh, cl[e], t);
+                    o[e] = ca[e] * t;
+                    if (addend) o[e] += a[k][e];
+                }
+                stv<V>(dy + off[k], o);
+            }
     }
 }
 
