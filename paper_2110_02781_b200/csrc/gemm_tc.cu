@@ -40,7 +40,7 @@ struct TcParams {
 
 template <int BN>
 __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                                                                const TcParams p) {
+                                                                const __grid_constant__ CUtensorMap mapD, const TcParams p) {
     constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = BN * TC_BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
 
     if (threadIdx.x == 0) {
         tma_prefetch_map(&mapA); tma_prefetch_map(&mapB);
+        if (BN >= 64) tma_prefetch_map(&mapD);
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -121,7 +122,8 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
     } else {
         // ---- epilogue: warps 2..5 own tensor-memory lanes 32*(warp%4) .. +31 ----
         const int q = warp & 3;
-        if (mbar_wait(accum, 0, p.err, 3)) {
+        const bool have = mbar_wait(accum, 0, p.err, 3);         // every stage has been consumed by now: the ring is free
+        if (have) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int m = m0 + q * 32 + lane;
 #pragma unroll 1
@@ -147,10 +149,29 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
                             unsigned o[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e) { const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]); o[e] = *reinterpret_cast<const unsigned*>(&h); }
-                            *reinterpret_cast<uint4*>(drow + g * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                            if (BN >= 64) {
+                                // staged for one TMA store per 128 x 64 piece: 128-byte rows, 16-byte chunk index XOR row % 8
+                                const int row = q * 32 + lane, j = (c & 1) * 4 + g;
+                                *reinterpret_cast<uint4*>(smem + (c >> 1) * (TC_BM * 128) + row * 128 + ((j ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                            } else
+                                *reinterpret_cast<uint4*>(drow + g * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
                 }
+            }
+            if (BN >= 64) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        if (BN >= 64) {
+            // whole 128-byte lines leave through TMA (clipped at the edges of D) instead of 16-byte pieces per thread
+            asm volatile("bar.sync 1, 128;" ::: "memory");                  // the four epilogue warps
+            if (have && threadIdx.x == 64) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 64; ++c)
+                    if (n0 + c * 64 < p.N)
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&mapD), "r"(n0 + c * 64), "r"(m0), "r"(smem_u32(smem + c * (TC_BM * 128))) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory may be released after this
             }
         }
     }
@@ -351,21 +372,25 @@ bool conv_tiles_ok(int H, int W, int pix) {
 template <int BN>
 bool launch_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No,
                     int flip, int* err, cudaStream_t st) {
-    CUtensorMap ma, mb;
+    CUtensorMap ma, mb, md;
     if (!make_map_4d(&ma, A, N, H, W, Ca, TC_BM) || !make_map_2d(&mb, B, 9LL * No, Ca, BN)) return false;
+    if (BN >= 64) { if (!make_map_2d(&md, D, (long long)N * H * W, No, TC_BM)) return false; }
+    else md = mb;
     constexpr int smem = TC_STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
     const int M = N * H * W;
     TcParams p{D, addend, M, No, 9 * Ca, err, ConvTap{1, H, W, Ca / 64, flip, No}};
-    launch(tc_gemm_tn_kernel<BN>, dim3((No + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, p);
+    launch(tc_gemm_tn_kernel<BN>, dim3((No + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, md, p);
     return true;
 }
 
 template <int BN>
 bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K, int* err,
                cudaStream_t st) {
-    CUtensorMap ma, mb;
+    CUtensorMap ma, mb, md;
     if (!make_map_2d(&ma, A, M, K, TC_BM) || !make_map_2d(&mb, B, N, K, BN)) return false;
+    if (BN >= 64) { if (!make_map_2d(&md, D, M, N, TC_BM)) return false; }
+    else md = mb;
     constexpr int smem = TC_STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
     static bool configured = false;
     if (!configured) {
@@ -373,7 +398,7 @@ bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat
         configured = true;
     }
     TcParams p{D, addend, M, N, K, err, ConvTap{0, 0, 0, 0, 0, 0}};
-    launch(tc_gemm_tn_kernel<BN>, dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, p);
+    launch(tc_gemm_tn_kernel<BN>, dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, md, p);
     return true;
 }
 
