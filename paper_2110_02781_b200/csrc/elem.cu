@@ -857,6 +857,79 @@ __global__ void __launch_bounds__(256) dw_wgrad_strip_kernel(const T* __restrict
     }
 }
 
+// The same weight gradient with three threads per strip, one per filter row (used for bf16 tensors, where it is
+// 20 % faster; float tensors are 10 % faster with the kernel above): a thread loads the four output gradients and the six inputs of its row once and feeds
+// its three taps from them.  (One thread per strip with all nine taps kept 36 accumulators and 109 registers: two
+// blocks per SM and a kernel that waited on its loads.)  Block: 8 channel vectors x 32 slots, slot = 3 * strip + row
+// for 10 strips, two slots idle; a block walks strips blockIdx.x * 10 + k, + gridDim.x * 10, ... and adds its slots
+// in slot order through shared memory.  partial[blockIdx.x][9][C] (float).
+constexpr int DW_WG_STRIPS = 10;
+template <typename T, int V>
+__global__ void __launch_bounds__(256) dw_wgrad_rows_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, int N, int H,
+                                                             int W, int C) {
+    grid_dep_sync();
+    __shared__ float sh[3][32][8 * V];
+    const int CV = C / V, cvl = threadIdx.x & 7, cv = blockIdx.y * 8 + cvl, slot = threadIdx.x >> 3;
+    const int c = cv * V;
+    const int k = slot / 3, rr = slot - 3 * k;              // strip within the block's group of ten, filter row
+    const int strips_w = (W + 3) >> 2;
+    const long long strips = (long long)N * H * strips_w;
+    float acc[3][V];
+#pragma unroll
+    for (int t = 0; t < 3; ++t)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
+    if (cv < CV && k < DW_WG_STRIPS) {
+        for (long long s = (long long)blockIdx.x * DW_WG_STRIPS + k; s < strips; s += (long long)gridDim.x * DW_WG_STRIPS) {
+            const int w0 = (int)(s % strips_w) * 4;
+            const long long R = s / strips_w;
+            const int h = (int)(R % H);
+            const int hi = h - 1 + rr;
+            if (hi < 0 || hi >= H) continue;
+            float d[4][V], in[6][V];
+            const T* row = x + ((R - h + hi) * W) * (long long)C + c;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (w0 + j < W) ldv<V>(dy + ((R * W) + w0 + j) * (long long)C + c, d[j]);
+                else {
+#pragma unroll
+                    for (int e = 0; e < V; ++e) d[j][e] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 6; ++j) {
+                const int wi = w0 - 1 + j;
+                if (wi >= 0 && wi < W) ldv<V>(row + (long long)wi * C, in[j]);
+                else {
+#pragma unroll
+                    for (int e = 0; e < V; ++e) in[j][e] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int ss = 0; ss < 3; ++ss)
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[ss][e] = fmaf(in[j + ss][e], d[j][e], acc[ss][e]);
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < 3; ++t)
+#pragma unroll
+        for (int e = 0; e < V; ++e) sh[t][slot][cvl * V + e] = acc[t][e];
+    __syncthreads();
+    for (int q = threadIdx.x; q < 9 * 8 * V; q += 256) {
+        const int tap = q / (8 * V), cc = q % (8 * V), gq = tap / 3, t = tap - 3 * gq;
+        const int gc = blockIdx.y * 8 * V + cc;
+        if (gc < C) {
+            float sum = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < DW_WG_STRIPS; ++kk) sum += sh[t][3 * kk + gq][cc];
+            partial[((long long)blockIdx.x * 9 + tap) * C + gc] = sum;
+        }
+    }
+}
+
 // dw[t][c] = sum over chunks and folded copies of partial[chunk][t][copy * C + c]; grid (ceil(C/32), G, 9)
 __global__ void dw_wgrad_finalize_kernel(const float* __restrict__ partial, int chunks, int f, int C, int cols, float* __restrict__ dw,
                                          const FinScratch fin) {
@@ -1337,11 +1410,12 @@ static FoldPlan plan_dw_wgrad(const ConvGeom& g, int elem_bytes) {
 }
 
 // strip kernel: number of blocks along the strips (each block walks strips with that stride)
-static inline int dw_wgrad_strip_blocks(const ConvGeom& g, int V) {
+static inline int dw_wgrad_strip_blocks(const ConvGeom& g, int V, bool rows_variant) {
     const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
     const int cgroups = (g.Cin / V + 7) / 8;
-    long long gx = (6LL * sm_count() + cgroups - 1) / cgroups;
-    const long long most = (strips + 31) / 32;
+    const int per_block = rows_variant ? DW_WG_STRIPS : 32;
+    long long gx = ((rows_variant ? 8LL : 6LL) * sm_count() + cgroups - 1) / cgroups;
+    const long long most = (strips + per_block - 1) / per_block;
     if (gx > most) gx = most;
     return (int)(gx < 1 ? 1 : gx);
 }
@@ -1349,8 +1423,7 @@ static inline int dw_wgrad_strip_blocks(const ConvGeom& g, int V) {
 size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
     const FoldPlan a = plan_dw_wgrad(g, 4), b = plan_dw_wgrad(g, 2);
     size_t n = std::max((size_t)a.chunks * 9 * a.cols, (size_t)b.chunks * 9 * b.cols);
-    if (g.Cin % 4 == 0) n = std::max(n, (size_t)dw_wgrad_strip_blocks(g, 4) * 9 * g.Cin);
-    if (g.Cin % 8 == 0) n = std::max(n, (size_t)dw_wgrad_strip_blocks(g, 8) * 9 * g.Cin);
+    if (g.Cin % 4 == 0) n = std::max(n, (size_t)std::max(dw_wgrad_strip_blocks(g, 4, false), dw_wgrad_strip_blocks(g, 4, true)) * 9 * g.Cin);
     return n;
 }
 
@@ -1360,8 +1433,10 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
     // four channels per thread for either type: with eight bf16 channels the nine accumulators would leave too few warps per SM
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy)) {
         constexpr int SV = 4;
-        const int gx = dw_wgrad_strip_blocks(g, SV);
-        launch(dw_wgrad_strip_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
+        constexpr bool rows_variant = sizeof(T) == 2;
+        const int gx = dw_wgrad_strip_blocks(g, SV, rows_variant);
+        if (rows_variant) launch(dw_wgrad_rows_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
+        else launch(dw_wgrad_strip_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
         if (gx <= DW_FIN_SMALL) {
             launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
             return;
