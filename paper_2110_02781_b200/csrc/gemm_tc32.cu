@@ -13,8 +13,8 @@
 //    MMAs (K = 8) of the stage; at the end warps 2-5 read the accumulator, stage it in shared memory and store
 //    it with TMA.
 //  * tc32_wgrad_kernel: both operands have the reduction as their slow dimension (activations and output
-//    gradients of the weight gradient); they land in a ring of source buffers and are transposed and split
-//    into K-major operand buffers by warps 2-5, the loads running ahead of conversion and MMAs.
+//    gradients of the weight gradient); the tensor core takes them as they land (MN-major operands), and the
+//    converter warps only add the lo parts.
 // Every wait is bounded; see gemm_tc.cu for the error protocol.
 #include "gemm_tc_common.cuh"
 
@@ -29,42 +29,6 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) { asm volatile("mbarri
 __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
                  ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// Transposing split.  src: nslabs slabs of [32 reduction rows][32 columns] floats as TMA wrote them (128-byte rows,
-// 16-byte chunk index XORed with row % 8).  hi / lo: K-major tiles [nslabs * 32 rows][32 reduction steps] in the
-// same swizzle.  A work item moves one output row's four consecutive reduction steps; the lanes of a warp take
-// 32 neighbouring columns of one source row, which is free of bank conflicts on both sides.  256 threads
-// cooperate: thread t always has column t % 32 and reduction steps 4 * (t / 32) .. + 3 of whatever slab it works
-// on, so its source and destination offsets inside a slab are computed once.
-struct TsplitLane { uint32_t s[4], d; };
-__device__ __forceinline__ TsplitLane tsplit_lane(int t) {
-    const int mn = t & 31, kq = (t >> 5) & 7;
-    TsplitLane l;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int k = kq * 4 + j;
-        l.s[j] = (uint32_t)(((mn & 3) << 2) + k * 128 + (((mn >> 2) ^ (k & 7)) << 4));
-    }
-    l.d = (uint32_t)(mn * 128 + ((kq ^ (mn & 7)) << 4));
-    return l;
-}
-__device__ __forceinline__ void transpose_split256(const uint8_t* src, uint8_t* hi, uint8_t* lo, int nslabs, const TsplitLane& l) {
-#pragma unroll 2
-    for (int sl = 0; sl < nslabs; ++sl) {
-        const uint8_t* s0 = src + sl * 4096;
-        float v[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) v[j] = *reinterpret_cast<const float*>(s0 + l.s[j]);
-        float4 h, q;
-        h.x = __uint_as_float(__float_as_uint(v[0]) & 0xffffe000u); q.x = v[0] - h.x;
-        h.y = __uint_as_float(__float_as_uint(v[1]) & 0xffffe000u); q.y = v[1] - h.y;
-        h.z = __uint_as_float(__float_as_uint(v[2]) & 0xffffe000u); q.z = v[2] - h.z;
-        h.w = __uint_as_float(__float_as_uint(v[3]) & 0xffffe000u); q.w = v[3] - h.w;
-        const uint32_t off = sl * 4096 + l.d;
-        *reinterpret_cast<float4*>(hi + off) = h;
-        *reinterpret_cast<float4*>(lo + off) = q;
-    }
 }
 
 // The tensor core reads only the upper 19 bits of a tf32 operand, so the tile as TMA delivered it already is the
@@ -276,49 +240,72 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
 }
 
 // Weight gradient: partials [slice][Mo][No] of X[R][Mo]^T dY[R][No].  Both operands have the reduction (rows) as
-// their slow dimension, so they land as slabs of 32 rows x 32 columns in a ring of source buffers; warps 2..5
-// transpose and split each source buffer into one of two operand buffers ([A hi][A lo][B hi][B lo]) and hand
-// the source buffer straight back to the loader, so that the loads run several reduction blocks ahead of the
-// conversion and the MMAs instead of waiting for them.
+// their slow dimension, so they are fed to the tensor core as they lie: a TMA box of 32 reduction rows x 32
+// columns with the 128-byte swizzle is four groups of 8 rows x 128 bytes, which is the MN-major operand layout of
+// the tensor core (one group per 8-deep MMA; 32-column slabs side by side, one slab = 4096 bytes apart).  A stage
+// is [A hi = as loaded][A lo][B hi = as loaded][B lo]; the converter warps only write the lo parts.
 template <int BN> struct Wg32Smem {
     static constexpr uint32_t A_BYTES = TC_BM * T32_BK * 4, B_BYTES = BN * T32_BK * 4;
-    static constexpr uint32_t SRC_BYTES = A_BYTES + B_BYTES, OP_BYTES = 2 * SRC_BYTES;
-    static constexpr int NOP = 2;
-    static constexpr int NSRC_FIT = (226 * 1024 - NOP * (int)OP_BYTES) / (int)SRC_BYTES;
-    static constexpr int NSRC = NSRC_FIT > 6 ? 6 : NSRC_FIT;
-    static constexpr int TOTAL = NOP * (int)OP_BYTES + NSRC * (int)SRC_BYTES + 1024;
+    static constexpr uint32_t STAGE_BYTES = 2 * (A_BYTES + B_BYTES);
+    static constexpr int NSTG_FIT = (226 * 1024) / (int)STAGE_BYTES;
+    static constexpr int NSTG = BN <= 64 ? 2 : (NSTG_FIT > 5 ? 5 : NSTG_FIT);
+    static constexpr int TOTAL = NSTG * (int)STAGE_BYTES + 1024;
 };
 
-// The conversion is the long pole of this kernel, so eight warps share it (two per scheduler hide each other's
-// shared-memory latency); four of them go on to the epilogue.
+// MN-major operand of 32-bit elements: 128-byte swizzle with 32-byte atoms (the 32-byte piece index of a 128-byte row is
+// XORed with row % 4), groups of 4 reduction rows 512 bytes apart, runs of 32 columns `slab_bytes` apart
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t slab_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);          // start address
+    d |= (uint64_t)(slab_bytes >> 4) << 16;          // leading byte offset: from one 128-byte run of columns to the next
+    d |= (uint64_t)(512 >> 4) << 32;                 // stride byte offset between 4-row groups of the reduction
+    d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+    d |= (uint64_t)1 << 61;                          // layout: 128-byte swizzle, 32-byte atoms
+    return d;
+}
+
+// as mma_block32, both operands MN-major: an 8-deep step of the reduction is one 1024-byte group further
+template <int BN>
+__device__ __forceinline__ void mma_block32_mn(uint32_t tmem, uint32_t a_hi, uint32_t a_lo, uint32_t b_hi, uint32_t b_lo, bool first) {
+    constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+    const uint64_t ah = umma_desc_mn_sw128(a_hi, 4096), al = umma_desc_mn_sw128(a_lo, 4096);
+    const uint64_t bh = umma_desc_mn_sw128(b_hi, 4096), bl = umma_desc_mn_sw128(b_lo, 4096);
+#pragma unroll
+    for (int k = 0; k < T32_BK / 8; ++k) {
+        const uint64_t o = (uint64_t)(k * (1024 >> 4));
+        umma_tf32(tmem, ah + o, bh + o, idesc, (!first || k > 0) ? 1u : 0u);
+        umma_tf32(tmem, ah + o, bl + o, idesc, 1u);
+        umma_tf32(tmem, al + o, bh + o, idesc, 1u);
+    }
+}
+
+// Eight warps write the lo parts (two per scheduler hide each other's shared-memory latency); four of them go on
+// to the epilogue.
 constexpr int WG32_CONV = 256, WG32_THREADS = 64 + WG32_CONV;
 
 template <int BN>
 __global__ void __launch_bounds__(WG32_THREADS) tc32_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                                                                 const __grid_constant__ CUtensorMap mapD, const T32Params p) {
     using L = Wg32Smem<BN>;
-    constexpr uint32_t A_BYTES = L::A_BYTES, B_BYTES = L::B_BYTES, SRC_BYTES = L::SRC_BYTES, OP_BYTES = L::OP_BYTES, SLAB = 32 * 32 * 4;
-    constexpr int NOP = L::NOP, NSRC = L::NSRC;
+    constexpr uint32_t A_BYTES = L::A_BYTES, B_BYTES = L::B_BYTES, STAGE_BYTES = L::STAGE_BYTES, SLAB = 32 * 32 * 4;
+    constexpr int NSTG = L::NSTG;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* srcs = smem + NOP * OP_BYTES;
-    __shared__ __align__(8) unsigned long long bars[2 * NSRC + 2 * NOP + 1];
+    __shared__ __align__(8) unsigned long long bars[3 * NSTG + 1];
     __shared__ uint32_t tmem_base;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * TC_BM, n0 = blockIdx.y * BN, split = blockIdx.z;
     const int kbeg = split * p.rows_per_split, kend = min(p.K, kbeg + p.rows_per_split);
     const int num_kb = (kend - kbeg + T32_BK - 1) / T32_BK;
-    // slabs wholly beyond the matrix are neither loaded nor converted (their rows of the hi / lo tiles are cleared once)
+    // slabs wholly beyond the matrix are neither loaded nor split (they are cleared once in every stage)
     const int slabsA = min(TC_BM / 32, (p.M - m0 + 31) / 32), slabsB = min(BN / 32, (p.N - n0 + 31) / 32);
     const uint32_t tx_bytes = (uint32_t)(slabsA + slabsB) * SLAB;
-    const uint32_t sfull0 = smem_u32(&bars[0]), sempty0 = smem_u32(&bars[NSRC]), ready0 = smem_u32(&bars[2 * NSRC]),
-                   oempty0 = smem_u32(&bars[2 * NSRC + NOP]), accum = smem_u32(&bars[2 * NSRC + 2 * NOP]);
+    const uint32_t full0 = smem_u32(&bars[0]), ready0 = smem_u32(&bars[NSTG]), empty0 = smem_u32(&bars[2 * NSTG]), accum = smem_u32(&bars[3 * NSTG]);
 
     if (threadIdx.x == 0) {
         tma_prefetch_map(&mapX); tma_prefetch_map(&mapY); tma_prefetch_map(&mapD);
-        for (int s = 0; s < NSRC; ++s) { mbar_init(sfull0 + 8 * s, 1); mbar_init(sempty0 + 8 * s, WG32_CONV); }
-        for (int s = 0; s < NOP; ++s) { mbar_init(ready0 + 8 * s, WG32_CONV); mbar_init(oempty0 + 8 * s, 1); }
+        for (int s = 0; s < NSTG; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(ready0 + 8 * s, WG32_CONV); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -336,20 +323,20 @@ __global__ void __launch_bounds__(WG32_THREADS) tc32_wgrad_kernel(const __grid_c
         if (lane == 0) {
             int issued = 0;
             for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % NSRC;
-                const uint32_t ph = (kb / NSRC) & 1;
-                if (kb >= NSRC && !mbar_wait(sempty0 + 8 * s, ph ^ 1, p.err, 11)) break;
-                const uint32_t sa = smem_u32(srcs + s * SRC_BYTES), sb = sa + A_BYTES;
+                const int s = kb % NSTG;
+                const uint32_t ph = (kb / NSTG) & 1;
+                if (kb >= NSTG && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 11)) break;     // the MMAs that read this stage are done
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + 2 * A_BYTES;
                 const int k = kbeg + kb * T32_BK;
-                mbar_expect_tx(sfull0 + 8 * s, tx_bytes);
-                for (int t = 0; t < slabsA; ++t) tma_load_2d(sa + t * SLAB, &mapX, m0 + 32 * t, k, sfull0 + 8 * s);
-                for (int t = 0; t < slabsB; ++t) tma_load_2d(sb + t * SLAB, &mapY, n0 + 32 * t, k, sfull0 + 8 * s);
+                mbar_expect_tx(full0 + 8 * s, tx_bytes);
+                for (int t = 0; t < slabsA; ++t) tma_load_2d(sa + t * SLAB, &mapX, m0 + 32 * t, k, full0 + 8 * s);
+                for (int t = 0; t < slabsB; ++t) tma_load_2d(sb + t * SLAB, &mapY, n0 + 32 * t, k, full0 + 8 * s);
                 issued = kb + 1;
             }
             if (*((volatile int*)p.err) != 0) {
-                for (int kb = max(0, issued - NSRC); kb < issued; ++kb) {
+                for (int kb = max(0, issued - NSTG); kb < issued; ++kb) {
                     const unsigned long long t0 = gtime();
-                    while (!mbar_test(sfull0 + 8 * (kb % NSRC), (kb / NSRC) & 1) && gtime() - t0 < 1000000ull) __nanosleep(128);
+                    while (!mbar_test(full0 + 8 * (kb % NSTG), (kb / NSTG) & 1) && gtime() - t0 < 1000000ull) __nanosleep(128);
                 }
             }
         }
@@ -357,43 +344,37 @@ __global__ void __launch_bounds__(WG32_THREADS) tc32_wgrad_kernel(const __grid_c
         if (lane == 0) {
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % NOP;
-                const uint32_t ph = (kb / NOP) & 1;
-                ok = mbar_wait(ready0 + 8 * s, ph, p.err, 12);                   // transposed, split and visible
+                const int s = kb % NSTG;
+                ok = mbar_wait(ready0 + 8 * s, (kb / NSTG) & 1, p.err, 12);            // landed, split and visible
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t sa = smem_u32(smem + s * OP_BYTES), sb = sa + 2 * A_BYTES;
-                mma_block32<BN>(tmem, sa, sa + A_BYTES, sb, sb + B_BYTES, kb == 0);
-                umma_commit(oempty0 + 8 * s);
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + 2 * A_BYTES;
+                mma_block32_mn<BN>(tmem, sa, sa + A_BYTES, sb, sb + B_BYTES, kb == 0);
+                umma_commit(empty0 + 8 * s);
             }
             if (ok) umma_commit(accum);
         }
     } else {
         const int t = threadIdx.x - 64;
-        static_assert(WG32_CONV == 256, "transpose_split256 assumes 256 converter threads");
-        const TsplitLane lane_off = tsplit_lane(t);
         bool ok = true;
         if (slabsA < TC_BM / 32 || slabsB < BN / 32) {
-            // clear the rows of the hi / lo tiles that no slab will ever fill
+            // clear the slabs that no load will ever fill, hi and lo, in every stage
             const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int s = 0; s < NOP; ++s) {
-                uint8_t* st = smem + s * OP_BYTES;
+            for (int s = 0; s < NSTG; ++s) {
+                uint8_t* st = smem + s * STAGE_BYTES;
                 for (int i = slabsA * SLAB + t * 16; i < (int)A_BYTES; i += WG32_CONV * 16) { *reinterpret_cast<float4*>(st + i) = z; *reinterpret_cast<float4*>(st + A_BYTES + i) = z; }
                 for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += WG32_CONV * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
             }
         }
         for (int kb = 0; kb < num_kb && ok; ++kb) {
-            const int ss = kb % NSRC, os = kb % NOP;
-            ok = mbar_wait(sfull0 + 8 * ss, (kb / NSRC) & 1, p.err, 13);
-            if (ok && kb >= NOP) ok = mbar_wait(oempty0 + 8 * os, ((kb / NOP) & 1) ^ 1, p.err, 15);   // the MMAs that read this operand buffer are done
+            const int s = kb % NSTG;
+            ok = mbar_wait(full0 + 8 * s, (kb / NSTG) & 1, p.err, 13);
             if (!ok) break;
-            const uint8_t* src = srcs + ss * SRC_BYTES;
-            uint8_t* st = smem + os * OP_BYTES;
-            transpose_split256(src, st, st + A_BYTES, slabsA, lane_off);
-            transpose_split256(src + A_BYTES, st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, lane_off);
+            uint8_t* st = smem + s * STAGE_BYTES;
+            split_tile(st, st + A_BYTES, slabsA * SLAB, t, WG32_CONV);
+            split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB * SLAB, t, WG32_CONV);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
-            mbar_arrive(ready0 + 8 * os);
-            mbar_arrive(sempty0 + 8 * ss);                                      // the loader may refill the source buffer
+            mbar_arrive(ready0 + 8 * s);
         }
         if (warp < 6) {                                                         // warps 2..5 own the four lane quarters of tensor memory
             const bool have = ok && (num_kb > 0 ? mbar_wait(accum, 0, p.err, 14) : true);
@@ -405,8 +386,8 @@ __global__ void __launch_bounds__(WG32_THREADS) tc32_wgrad_kernel(const __grid_c
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
 }
 
-// rows x cols float matrix, cols contiguous; box = 32 columns x box_rows rows, 128-byte swizzle, zero fill
-bool make_map_f32(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+// rows x cols float matrix, cols contiguous; box = 32 columns x box_rows rows, 128-byte swizzle (of 16-byte pieces unless told otherwise), zero fill
+bool make_map_f32(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -414,7 +395,7 @@ bool make_map_f32(CUtensorMap* map, const void* base, long long rows, long long 
     const cuuint32_t box[2] = {(cuuint32_t)T32_BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // output [S][rows][cols] floats; box = 32 columns x 128 rows x 1, 128-byte swizzle (stores clip at the edges)
@@ -442,7 +423,7 @@ bool launch32(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& m
 template <int BN>
 bool launch32_wgrad(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& md, const T32Params& p, dim3 grid, cudaStream_t st) {
     constexpr int smem = Wg32Smem<BN>::TOTAL;
-    static_assert(Wg32Smem<BN>::NSRC >= 2 && Wg32Smem<BN>::NOP * (int)Wg32Smem<BN>::OP_BYTES >= TC_BM * BN * 4, "shared-memory plan");
+    static_assert(Wg32Smem<BN>::NSTG >= 2 && Wg32Smem<BN>::NSTG * (int)Wg32Smem<BN>::STAGE_BYTES >= TC_BM * BN * 4, "shared-memory plan");
     if (cudaFuncSetAttribute(tc32_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
     launch(tc32_wgrad_kernel<BN>, grid, dim3(WG32_THREADS), smem, st, mx, my, md, p);
     return true;
@@ -463,7 +444,7 @@ Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
     const int m = w.swap ? No : Mo, n = w.swap ? Mo : No;
     w.BN = bn_for(n);
     const long long tiles = (long long)((m + TC_BM - 1) / TC_BM) * ((n + w.BN - 1) / w.BN);
-    long long S = (3LL * sm_count() + tiles - 1) / tiles;
+    long long S = (2LL * sm_count() + tiles - 1) / tiles;
     const long long maxS = (R + 255) / 256;
     long long cap = (2LL << 20) / ((long long)Mo * No);                     // partial sums cost traffic too: at most 2 Mi floats
     if (cap < 1) cap = 1;
@@ -550,6 +531,8 @@ struct G32Plan { int BN, S, rps; };
 G32Plan plan_gemm32(int M, int N, int K) {
     const int sms = sm_count(), mt = (M + TC_BM - 1) / TC_BM;
     int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
+    // 144, 192, 576 or 960 columns leave a 128-wide last tile mostly empty; 64-wide tiles fit them with less padding
+    if (BN == 128 && (N + 63) / 64 * 64 < (N + 127) / 128 * 128) BN = 64;
     while (BN > 32 && (long long)mt * ((N + BN - 1) / BN) < sms) BN >>= 1;
     const long long tiles = (long long)mt * ((N + BN - 1) / BN);
     const int nkb = (K + T32_BK - 1) / T32_BK;
@@ -621,7 +604,7 @@ bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long
     const int m = w.swap ? No : Mo, n = w.swap ? Mo : No;
     CUtensorMap mx, my, md;
     float* out = two_pass ? scratch : dW;
-    if (!make_map_f32(&mx, A, R, m, 32) || !make_map_f32(&my, B, R, n, 32) || !make_map_out(&md, out, w.S, m, n)) return false;
+    if (!make_map_f32(&mx, A, R, m, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) || !make_map_f32(&my, B, R, n, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) || !make_map_out(&md, out, w.S, m, n)) return false;
     T32Params p{out, nullptr, m, n, (int)R, w.rows_per_split, 0, err};
     const dim3 grid((m + TC_BM - 1) / TC_BM, (n + w.BN - 1) / w.BN, w.S);
     bool ok;
