@@ -214,6 +214,24 @@ def test_edge_shapes_batch_one_odd_channels():
         one_step_case((ls, cfg), 25, [0, 1, 2, 3])
 
 
+def test_pointwise_weight_gradients_on_ragged_slabs():
+    """1 x 1 convolutions whose weight gradients run on the tensor cores with both operands as they lie in memory:
+    channel counts that end inside a 32-column slab (40, 72, 136), on both sides of the 128-row tile (so the product
+    is taken both ways round), more than one tile (200 -> 160), and pixel counts (147, 50, 363) that end inside a
+    32-row block of the reduction."""
+    L = synth.Layer
+    K, A = synth.KIND, synth.ACT
+    for batch, hw, chans in ((3, 7, (40, 72, 24)), (2, 5, (136, 24, 136)), (3, 11, (200, 160, 8))):
+        c0, c1, c2 = chans
+        ls = [L(0, K["CONV2D"], 8, c0, 1, 1, 0, 0, 0, -1), L(0, K["BN"], c0, c0, 0, 1, 0, A["RELU6"], 0, -1),
+              L(1, K["CONV2D"], c0, c1, 1, 1, 0, 0, 0, -1), L(1, K["BN"], c1, c1, 0, 1, 0, A["RELU6"], 0, -1),
+              L(2, K["CONV2D"], c1, c2, 1, 1, 0, 0, 0, -1), L(2, K["BN"], c2, c2, 0, 1, 0, 0, 0, -1),
+              L(3, K["GAP"], c2, c2, 0, 1, 0, 0, 0, -1), L(3, K["FC"], c2, 5, 1, 1, 0, 0, 1, -1),
+              L(3, K["SOFTMAX_CE"], 5, 5, 0, 1, 0, 0, 0, -1)]
+        cfg = synth.config(batch, 8, hw, hw, 5, momentum=0.9, weight_decay=1e-4)
+        one_step_case((ls, cfg), 31, [0, 1, 3, 4])
+
+
 def test_first_convolution_kernels_on_ragged_maps():
     """3 -> 32 and 3 -> 64 first convolutions take the dedicated kernels: odd map sizes, stride 1 and 2, pixel counts
     that are not multiples of the 32-pixel chunks of the weight gradient."""
