@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
 struct TcWgPlan { int S, rows_per_split; };
 TcWgPlan plan_tc_wgrad(long long R, int Mo, int No) {
     const long long tiles = ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
-    long long S = (3LL * sm_count() + tiles - 1) / tiles;
+    long long S = (2LL * sm_count() + tiles - 1) / tiles;
     const long long maxS = (R + 511) / 512;                                 // at least 512 rows per split
     long long cap = (8LL << 20) / ((long long)Mo * No);                     // partials within 8 Mi floats
     if (cap < 1) cap = 1;
@@ -432,7 +432,7 @@ bool launch_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out
 
 TcWgPlan plan_tc_wgrad3x3(long long R, int Mo, int No) {
     const long long tiles = 9LL * ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
-    long long S = (3LL * sm_count() + tiles - 1) / tiles;
+    long long S = (2LL * sm_count() + tiles - 1) / tiles;
     const long long maxS = (R + 511) / 512;
     long long cap = (8LL << 20) / (9LL * Mo * No);
     if (cap < 1) cap = 1;
