@@ -68,7 +68,7 @@ STEP_WORK = {"cfg2": (11.73e9 / 128, (63.1e9 + 4.5e9) / 128), "cfg3": (12.00e9 /
 # pass (profiles/ncu_tc32_kernels_cfg2_b128.md).  Valid only for the default batch and while the kernel source is the
 # one the counters were taken on: the entry carries the sha256 of that source file.
 NCU_TRAFFIC = {("cfg2", "tc_gemm_tf32x3_wgrad"): dict(bytes_per_step=1.033e9, source="paper_2110_02781_b200/csrc/gemm_tc32.cu",
-                                                     sha256="3f09c7060b4dae22f251a33a6d0fe8b75c62d5d7b544a128a56ba08400c91469")}
+                                                     sha256="5ad3bd27eb66910b5a693747e616017454f81f9675fe7c86751d0b7a150bb82b")}
 
 
 def ncu_traffic(wl_key, kernel, default_batch):

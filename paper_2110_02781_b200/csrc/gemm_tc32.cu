@@ -524,8 +524,8 @@ __global__ void __launch_bounds__(256) slice_sum_kernel(const float4* __restrict
     out[i] = a;
 }
 
-// Tile width and reduction slices of a product D[M,N] over K.  With fewer tiles than SMs the tiles get narrower (not
-// below 64 columns: the MMAs of a 32-wide tile read the 128-row operand from shared memory for a quarter of the
+// Tile width and reduction slices of a product D[M,N] over K.  With fewer tiles than SMs the tiles get narrower (with
+// eight or more row tiles not below 64 columns: the MMAs of a 32-wide tile read the 128-row operand from shared memory for a quarter of the
 // output) and the reduction is cut into slices (each at least four 32-wide blocks), so that the late, small layers
 // still spread over the machine; the slices are summed in order by a second kernel.
 struct G32Plan { int BN, S, rps; };
@@ -534,7 +534,8 @@ G32Plan plan_gemm32(int M, int N, int K) {
     int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
     // 144, 192, 576 or 960 columns leave a 128-wide last tile mostly empty; 64-wide tiles fit them with less padding
     if (BN == 128 && (N + 63) / 64 * 64 < (N + 127) / 128 * 128) BN = 64;
-    while (BN > 64 && (long long)mt * ((N + BN - 1) / BN) < sms) BN >>= 1;
+    const int narrowest = mt >= 8 ? 64 : 32;     // a handful of row tiles: 32-wide tiles fill more SMs without a second pass
+    while (BN > narrowest && (long long)mt * ((N + BN - 1) / BN) < sms) BN >>= 1;
     const long long tiles = (long long)mt * ((N + BN - 1) / BN);
     const int nkb = (K + T32_BK - 1) / T32_BK;
     long long S = 1;
