@@ -58,17 +58,41 @@ def workload(name, batch=None):
 
 FALLBACK_BF16_TFLOPS = 1400.0            # sustained figure of the fallback measurement
 
-# Whole-step algorithmic work per sample: bytes of every tensor pass of the separate conv / BN forward / BN backward /
-# data-gradient / weight-gradient kernels counted once ((3 I + 11 O) elements per op), and dense + depthwise flops
-# (backward counted as twice the forward).  Keys: workload name -> (bytes per sample, flop per sample).
-STEP_WORK = {"cfg2": (11.73e9 / 128, (63.1e9 + 4.5e9) / 128), "cfg3": (12.00e9 / 64, (107.5e9 + 8.0e9) / 64),
-             "cfg5": (12.00e9 / 64, (107.5e9 + 8.0e9) / 64), "cfg4": (1.84e9 / 256, 481.1e9 / 256), "cfg1": (10e6 / 32, 1.08e9 / 32)}
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of all launches of a kernel class in one step, from one ncu
-# pass (profiles/ncu_tc32_kernels_cfg2_b128.md).  Valid only for the default batch and while the kernel source is the
-# one the counters were taken on: the entry carries the sha256 of that source file.
-NCU_TRAFFIC = {("cfg2", "tc_gemm_tf32x3_wgrad"): dict(bytes_per_step=1.033e9, source="paper_2110_02781_b200/csrc/gemm_tc32.cu",
-                                                     sha256="5ad3bd27eb66910b5a693747e616017454f81f9675fe7c86751d0b7a150bb82b")}
+def step_work(layers, cfg):
+    """Whole-step algorithmic work from the layer list at the configured batch.  Per contraction / depthwise op with I
+    input and O output elements: model A = every tensor pass of separate conv / BN forward / BN backward / data-gradient /
+    weight-gradient kernels counted once, (3 I + 11 O) elements; model B = batch-norm statistics from the producer and
+    both batch-norm apply passes folded into their neighbours, (3 I + 5 O) elements.  Flops: forward plus twice that for
+    the backward pass.  Returns (bytes A, bytes B, dense flop, depthwise flop)."""
+    import synth
+    K = synth.KIND
+    s = 2 if cfg["precision"] == 1 else 4
+    n, h, w, c = cfg["batch"], cfg["in_h"], cfg["in_w"], cfg["in_c"]
+    a = b = dense = dw = 0
+    for l in layers:
+        if l.kind in (K["CONV1D"], K["CONV2D"], K["FC"], K["DWCONV3x3"]):
+            kh, kw, ph, pw = (1, l.k, 0, l.pad) if l.kind == K["CONV1D"] else ((1, 1, 0, 0) if l.kind == K["FC"] else (l.k, l.k, l.pad, l.pad))
+            ho, wo = (h + 2 * ph - kh) // l.stride + 1, (w + 2 * pw - kw) // l.stride + 1
+            i_el, o_el = n * h * w * c, n * ho * wo * l.cout
+            a += (3 * i_el + 11 * o_el) * s
+            b += (3 * i_el + 5 * o_el) * s
+            if l.kind == K["DWCONV3x3"]:
+                dw += 3 * 18 * o_el
+            else:
+                dense += 3 * 2 * n * ho * wo * kh * kw * c * l.cout
+            h, w, c = ho, wo, l.cout
+        elif l.kind == K["MAXPOOL2"]:
+            h, w = h // 2, w // 2
+        elif l.kind == K["GAP"]:
+            h = w = 1
+    return a, b, dense, dw
+
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of all launches of a kernel class in one step of the default
+# workload, from one ncu pass.  An entry is valid only for the kernel source it was taken on (sha256 of the file) and is
+# added only together with a retaken pass; without a valid entry `traffic` is null.
+NCU_TRAFFIC = {}
 
 
 def ncu_traffic(wl_key, kernel, default_batch):
@@ -258,46 +282,14 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=
     return ev[0].elapsed_time(ev[steps]), per_it, log
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 50; 500 for cfg5)")
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cl8"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
-    ap.add_argument("--points", default=None, help="comma-separated partition points; skips the profile-and-optimise step")
-    ap.add_argument("--graph", type=int, default=1, help="1: time CUDA-graph replays of the step (default); 0: eager launches")
-    ap.add_argument("--fail", default=None, help="cfg5 only, ITERATION:STAGE: that stage is lost after that iteration and recovered from the replicas")
-    ap.add_argument("--lean", action="store_true", help="timed region only: no end-to-end leg, no kernel trace (profiling captures)")
-    args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    wl = workload(args.workload, args.batch)
-    if args.steps is None:
-        args.steps = 500 if args.workload == "cfg5" else 50
-
-    if args.impl == "reference":
-        if rank != 0:
-            return 0
-        args.warmup_ref = min(args.warmup, 1)
-        args.steps = min(args.steps, 3)
-        print(json.dumps(run_reference(args, wl)), flush=True)
-        return 0
-
-    import numpy as np
+def measure(args, wl_key, reps, steps, warmup, local_rank, replicas, batch=None, points=None, graph=1, fail=None, lean=False):
+    """Builds one workload, times `reps` blocks of `steps` steps on the device (median block), then the end-to-end
+    leg (host inputs copied in, loss read back, every step) and a per-launch event trace.  Returns the fields of a
+    bench line for that workload."""
     import torch
     import synth
     import paper_2110_02781_b200 as F
-
-    assert args.warmup >= 3, "at least 3 warm-up steps"
-    torch.cuda.set_device(local_rank)
-    from paper_2110_02781_b200.replicas import Replicas
-    reps = Replicas("nccl", torch.device("cuda", local_rank))
-    dist = reps.dist
-
+    wl = workload(wl_key, batch)
     ls, cfg = wl["layers"], wl["cfg"]
     m = F.Model(ls, cfg, f"cuda:{local_rank}")
     m.load_params(synth.init_params(wl["index"], ls), synth.init_state(ls))
@@ -308,37 +300,38 @@ def main():
     xh, yh = xt.pin_memory(), torch.from_numpy(y).pin_memory()
     lr = cfg["lr"]
 
-    # partition: profile -> equal capacities -> optimiser (or the split the workload fixes)
-    if args.points:
-        wl["points"] = [int(v) for v in args.points.split(",")]
+    # partition: profile -> capacities -> optimiser (or the split the workload fixes)
+    fwd_s = bwd_s = None
+    if points:
+        wl["points"] = list(points)
     else:
-        fwd_s, bwd_s, out_bytes = m.ftp_profile_layers(10, xd, yd)
+        fwd_s, bwd_s, _ = m.ftp_profile_layers(10, xd, yd)
     if wl["points"] is None:
-        points, bottleneck = F.ftp_choose_partition((fwd_s + bwd_s).tolist(), wl["caps"])
+        pts, _ = F.ftp_choose_partition((fwd_s + bwd_s).tolist(), wl["caps"])
     else:
-        points, bottleneck = wl["points"], None
-    m.ftp_set_partition(points)
+        pts = wl["points"]
+    m.ftp_set_partition(pts)
 
     def barrier():
-        reps.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
+    def timed(fn, n):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record()
-        for _ in range(steps):
+        for _ in range(n):
             fn()
         e1.record()
         barrier()
-        return reps.max_over_ranks(e0.elapsed_time(e1))
+        return replicas.max_over_ranks(e0.elapsed_time(e1))
 
     step_eager = lambda: m.ftp_train_step(xd, yd, lr, inputs_on_host=False, want_loss=False)
     step_dev = step_eager
     dynamic = wl.get("dynamic")
     if dynamic:
-        args.graph = 0                   # the partition changes during the run: launches are issued eagerly
-    if args.graph:
+        graph = 0                        # the partition changes during the run: launches are issued eagerly
+    if graph:
         # the launches of one step captured once on a side stream and replayed: same kernels, no per-launch CPU cost
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -346,23 +339,22 @@ def main():
             for _ in range(2):
                 step_eager()
         torch.cuda.current_stream().wait_stream(side)
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
             step_eager()
-        step_dev = graph.replay
+        step_dev = g.replay
     step_e2e = lambda: m.ftp_train_step(xh, yh, lr, inputs_on_host=True, want_loss=True)
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step_dev()
-    n0 = m.ftp_launch_count()
     dyn_info = None
+    blocks = []
     with ClockSampler(local_rank) as clk:
         if dynamic:
             lt = (fwd_s + bwd_s).tolist()
             barrier()
-            fail = tuple(int(v) for v in args.fail.split(":")) if args.fail else None
-            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, args.steps, False, fail)
+            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, steps, False, fail)
             barrier()
-            ms = reps.max_over_ranks(ms)
+            blocks = [replicas.max_over_ranks(ms)]
             tick = lambda i, p: (i + 1) % p == 0
             plain = [t for i, t in enumerate(per_it) if not tick(i, dynamic["snapshot"]) and not tick(i, dynamic["repartition"])]
             snap = [t for i, t in enumerate(per_it) if tick(i, dynamic["snapshot"]) and not tick(i, dynamic["repartition"])]
@@ -371,33 +363,37 @@ def main():
             dyn_info = dict(ms_plain_iteration=med(plain), ms_snapshot_iteration=med(snap), ms_repartition_iteration=med(rep),
                             repartitions=plog[:12], snapshot_bytes_per_tick=int(3 * 4 * sum(m.ftp_unit_param_span(u)[1] + m.ftp_unit_state_span(u)[1] for u in range(m.L))))
         else:
-            ms = timed(step_dev, args.steps)
-    launches = m.ftp_launch_count() - n0
-    if args.graph:                      # a replay re-issues the captured launches without passing through the counter
-        c0 = m.ftp_launch_count()
-        step_eager()
-        launches = (m.ftp_launch_count() - c0) * args.steps
-    if args.lean:
-        print(json.dumps({"lean": True, "ms_per_step": ms / args.steps, "gpu_launches": int(launches)}), flush=True)
-        return 0
+            blocks = [timed(step_dev, steps) for _ in range(reps)]
+    ms = statistics.median(blocks)
+    c0 = m.ftp_launch_count()
+    step_eager()                        # a replay re-issues the captured launches without passing through the counter
+    per_step = m.ftp_launch_count() - c0
+    out = {"workload": wl["name"], "index": wl["index"], "points": [int(p) for p in pts], "batch": cfg["batch"], "bf16": bf16, "steps": steps,
+           "ms_per_step": ms / steps, "value": replicas.job_throughput(cfg["batch"] * steps, ms),
+           "blocks_ms_per_step": {"median": ms / steps, "min": min(blocks) / steps, "max": max(blocks) / steps, "blocks": len(blocks)},
+           "clocks": clk.summary(), "launches_per_step": int(per_step), "gpu_launches": int(per_step * steps * len(blocks)),
+           "graph": bool(graph), "caps": wl["caps"], "dynamic": dyn_info}
+    if lean:
+        m.close()
+        return out
     for _ in range(3):
         step_e2e()
-    e2e_steps = args.steps
+    e2e_steps = steps
     if dynamic:
-        e2e_steps = max(dynamic["repartition"] * 2, args.steps // 5)
-        m.ftp_set_partition(points)
+        e2e_steps = max(dynamic["repartition"] * 2, steps // 5)
+        m.ftp_set_partition(pts)
         barrier()
         ms_e2e, _, _ = run_dynamic(m, F, wl, (fwd_s + bwd_s).tolist(), xd, yd, xh, yh, lr, e2e_steps, True)
         barrier()
-        ms_e2e = reps.max_over_ranks(ms_e2e)
-        m.ftp_set_partition(points)
+        ms_e2e = replicas.max_over_ranks(ms_e2e)
+        m.ftp_set_partition(pts)
     else:
-        ms_e2e = timed(step_e2e, args.steps)
-    batch = cfg["batch"]
-    value = reps.job_throughput(batch * args.steps, ms)
-    e2e = reps.job_throughput(batch * e2e_steps, ms_e2e)
+        ms_e2e = timed(step_e2e, steps)
+    out["e2e"] = {"value": replicas.job_throughput(cfg["batch"] * e2e_steps, ms_e2e), "unit": "samples/s",
+                  "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * 4), "d2h_bytes_per_step": 4,
+                  "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps}
 
-    # per-kernel roofline: one more step with every launch bracketed by events
+    # per-kernel roofline: three more steps with every launch bracketed by events
     m.ftp_trace_enable(True)
     for _ in range(3):
         step_eager()
@@ -413,14 +409,14 @@ def main():
     for name, k in sorted(by.items(), key=lambda kv: -kv[1]["ms"]):
         gbs = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
         tf = k["flops"] / (k["ms"] * 1e-3) / 1e12 if k["ms"] > 0 else 0.0
-        math_peak = tensor_peak if name.startswith("tc_") else FP32_ALU_PEAK_TFLOPS
+        math_peak = tensor_peak if name.startswith("tc_gemm_bf16") else FP32_ALU_PEAK_TFLOPS
         table[name] = dict(share=round(k["ms"] / total_ms, 4), launches_per_step=k["n"] // 3, ms_per_step=round(k["ms"] / 3, 4),
                            gbs=round(gbs, 1), tflops=round(tf, 2), frac_hbm=round(gbs / hbm_peak, 3),
                            frac_math=round(tf / math_peak, 3))
     dom = next(iter(table))
     d = table[dom]
     math_bound = d["frac_math"] > d["frac_hbm"]
-    tensor = dom.startswith("tc_")
+    tensor = dom.startswith("tc_gemm_bf16")
     roofline = {"kernel": dom, "bound": ("tensor" if tensor else "alu") if math_bound else "hbm",
                 "achieved": d["tflops"] if math_bound else d["gbs"],
                 "peak": (tensor_peak if tensor else round(FP32_ALU_PEAK_TFLOPS, 1)) if math_bound else hbm_peak,
@@ -428,36 +424,101 @@ def main():
                 "frac": d["frac_math"] if math_bound else d["frac_hbm"],
                 "peak_source": ((f"{peak_src} bf16 matmul, sustained" if tensor else "derived: 2 x 128 lanes x 148 SMs x 1.965 GHz")
                                 if math_bound else f"{peak_src} HBM copy"),
-                "traffic": ncu_traffic(args.workload, dom, args.batch is None), "share_of_step": d["share"],
+                "traffic": ncu_traffic(wl_key, dom, batch is None), "share_of_step": d["share"],
                 "note": "achieved = algorithmic bytes (or flops) of all launches of the kernel in a step / their CUDA-event time",
                 "kernels": table}
-    sw = STEP_WORK.get(args.workload)
-    if sw:
-        step_s = ms / args.steps * 1e-3
-        gbs = sw[0] * batch / step_s / 1e9
-        tfs = sw[1] * batch / step_s / 1e12
-        roofline["step"] = {"algorithmic_GB": round(sw[0] * batch / 1e9, 3), "GB/s": round(gbs, 1), "frac_hbm": round(gbs / hbm_peak, 3),
-                            "TFLOP/s": round(tfs, 2), "frac_tensor": round(tfs / tensor_peak, 3) if bf16 else None,
-                            "note": "whole step: algorithmic bytes (flops) of all kernels / device time of the timed steps"}
+    wa, wb, dense, dwf = step_work(ls, cfg)
+    step_s = ms / steps * 1e-3
+    tfs = (dense + dwf) / step_s / 1e12
+    roofline["step"] = {"algorithmic_GB_separate_passes": round(wa / 1e9, 3), "algorithmic_GB_fused_bn": round(wb / 1e9, 3),
+                        "frac_hbm_separate_passes": round(wa / step_s / 1e9 / hbm_peak, 3), "frac_hbm_fused_bn": round(wb / step_s / 1e9 / hbm_peak, 3),
+                        "TFLOP/s": round(tfs, 2), "frac_tensor": round(dense / step_s / 1e12 / tensor_peak, 3) if bf16 else None,
+                        "note": "whole step: algorithmic bytes of all kernels / device time of a step, against the count with separate "
+                                "batch-norm passes ((3I+11O) per convolution) and against the count with them folded into their neighbours ((3I+5O))"}
+    out["roofline"] = roofline
+    m.close()
+    return out
 
-    out = {"metric": "training samples/sec per partitioned step", "value": value, "unit": "samples/s", "n_gpus": world,
-           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-           "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
-           "config": {"workload": wl["name"], "points": points, "stages": len(points) - 1, "batch": batch,
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps per block (default 50; 500 for cfg5)")
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--reps", type=int, default=5, help="timed blocks of --steps steps; the median block is reported")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cl8"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short entries for the other workloads")
+    ap.add_argument("--batch", type=int, default=None, help="smaller batch of the same network (profiling captures only)")
+    ap.add_argument("--points", default=None, help="comma-separated partition points; skips the profile-and-optimise step")
+    ap.add_argument("--graph", type=int, default=1, help="1: time CUDA-graph replays of the step (default); 0: eager launches")
+    ap.add_argument("--fail", default=None, help="cfg5 only, ITERATION:STAGE: that stage is lost after that iteration and recovered from the replicas")
+    ap.add_argument("--lean", action="store_true", help="timed region only: no end-to-end leg, no kernel trace (profiling captures)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.steps is None:
+        args.steps = 500 if args.workload == "cfg5" else 50
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        args.warmup_ref = min(args.warmup, 1)
+        args.steps = min(args.steps, 3)
+        print(json.dumps(run_reference(args, workload(args.workload, args.batch))), flush=True)
+        return 0
+
+    import torch
+    assert args.warmup >= 3, "at least 3 warm-up steps"
+    torch.cuda.set_device(local_rank)
+    from paper_2110_02781_b200.replicas import Replicas
+    reps = Replicas("nccl", torch.device("cuda", local_rank))
+
+    points = [int(v) for v in args.points.split(",")] if args.points else None
+    fail = tuple(int(v) for v in args.fail.split(":")) if args.fail else None
+    r = measure(args, args.workload, args.reps, args.steps, args.warmup, local_rank, reps, args.batch, points, args.graph, fail, args.lean)
+    if args.lean:
+        if rank == 0:
+            print(json.dumps({"lean": True, "ms_per_step": r["ms_per_step"], "blocks_ms_per_step": r["blocks_ms_per_step"],
+                              "gpu_launches": r["gpu_launches"]}), flush=True)
+        reps.close()
+        return 0
+    bf16 = r["bf16"]
+    out = {"metric": "training samples/sec per partitioned step", "value": r["value"], "unit": "samples/s", "n_gpus": world,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if bf16 else "f32 (tf32x3 contractions)", "data": "synthetic",
+           "config": {"workload": r["workload"], "points": r["points"], "stages": len(r["points"]) - 1, "batch": r["batch"],
                       "parallelism": "replicas only" if world > 1 else "1 GPU, all stages resident",
                       "cache": "a step streams far more activation bytes than the 126 MB L2 holds",
-                      "capacities": wl["caps"],
-                      "launch": "cuda graph replay of ftp_train_step" if args.graph else "eager"},
-           "clocks": clk.summary(), "gpu_launches": int(launches),
-           "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * 4),
-                   "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps},
-           "roofline": roofline}
-    if dyn_info:
-        out["config"]["dynamic"] = dyn_info
+                      "capacities": r["caps"], "launch": "cuda graph replay of ftp_train_step" if r["graph"] else "eager",
+                      "timed": f"{r['blocks_ms_per_step']['blocks']} blocks of {args.steps} steps, median block reported",
+                      "blocks_ms_per_step": r["blocks_ms_per_step"], "launches_per_step": r["launches_per_step"]},
+           "clocks": r["clocks"], "gpu_launches": r["gpu_launches"], "e2e": r["e2e"], "roofline": r["roofline"]}
+    if r["dynamic"]:
+        out["config"]["dynamic"] = r["dynamic"]
+    if world == 1 and not args.no_configs:
+        # the other workloads, briefly: value, end-to-end value, the dominant kernel's fraction and the clocks seen, each
+        others = {}
+        for key in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cl8"):
+            if key == args.workload:
+                continue
+            q = measure(args, key, 3, 100 if key == "cfg5" else 20, 3, local_rank, reps)
+            rf = q["roofline"]
+            others[key] = {"workload": q["workload"], "value": round(q["value"], 1), "unit": "samples/s", "ms_per_step": round(q["ms_per_step"], 4),
+                           "blocks_ms_per_step": q["blocks_ms_per_step"], "points": q["points"], "launches_per_step": q["launches_per_step"],
+                           "e2e": {k: q["e2e"][k] for k in ("value", "h2d_bytes_per_step", "d2h_bytes_per_step", "ms_per_step")},
+                           "dtype": "bf16" if q["bf16"] else "f32 (tf32x3 contractions)",
+                           "dominant_kernel": {k: rf[k] for k in ("kernel", "bound", "achieved", "peak", "unit", "frac", "share_of_step")},
+                           "step": rf["step"], "clocks": q["clocks"]}
+            if q["dynamic"]:
+                others[key]["dynamic"] = {k: q["dynamic"][k] for k in ("ms_plain_iteration", "ms_snapshot_iteration", "ms_repartition_iteration")}
+        out["configs"] = others
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         a2 = argparse.Namespace(**vars(args))
         a2.warmup_ref, a2.steps = 0, 2
-        out["cpu_baseline"] = run_reference(a2, wl)["cpu_baseline"]
+        out["cpu_baseline"] = run_reference(a2, workload(args.workload, args.batch))["cpu_baseline"]
     if rank == 0:
         print(json.dumps(out), flush=True)
     reps.close()

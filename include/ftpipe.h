@@ -27,7 +27,15 @@
  *   - All GPU work is asynchronous on the given stream unless stated otherwise.
  *   - Errors: every call returns an ftp_status; arguments are validated before any launch
  *     and a failed call launches nothing.  ftp_last_error() gives the text for this thread.
- *     Kernels never trap or assert.
+ *     Kernels never trap or assert.  Every wait inside a tensor-core kernel is bounded; one that
+ *     runs out makes the kernel skip its stores, return, and leave a code in a device status
+ *     word.  Calls that synchronise (ftp_train_step with loss_host, ftp_profile_layers,
+ *     ftp_get_tensor / ftp_get_logits to a host buffer, ftp_check_device_status) read that word,
+ *     return FTP_ETIMEOUT when it is set and clear it; asynchronous calls queue a copy of it
+ *     behind their launches and the next call of the model that launches or reports
+ *     (run_stage, sgd_step, train_step, stage_times) returns FTP_ETIMEOUT before doing anything
+ *     once that copy shows a code, until ftp_check_device_status has cleared it.  Tensors
+ *     written between the failed wait and the report are invalid.
  */
 #ifndef FTPIPE_H
 #define FTPIPE_H
@@ -130,7 +138,8 @@ ftp_status ftp_get_tensor(const ftp_model* m, int32_t which, int32_t unit, float
  *   act_in  : device; the input batch (a == 0) or the boundary activation leaving unit a-1.
  *   act_out : device; receives the boundary activation leaving unit b-1; must be NULL when
  *             b == L (the last unit ends in the loss).
- *   labels  : device int32[batch], required iff b == L.
+ *   labels  : device int32[batch], required iff b == L.  Device-resident labels are not validated:
+ *             a label outside [0, n_classes) is treated as the nearest valid class.
  *   loss_out: device float[1], required iff b == L; mean softmax cross-entropy.
  * act_in and act_out must stay valid and unmodified until the backward pass of the same
  * range has completed (they are read again there; nothing is copied).  Updates the BN
@@ -162,12 +171,20 @@ ftp_status ftp_sgd_step(ftp_model* m, int32_t a, int32_t b, float lr, float* sna
 /* One synchronous training step over the current partition: forward through every stage,
  * backward through every stage, SGD on every stage; internal boundary buffers.
  *   x, labels   : the input batch and int32 labels; host (pinned or pageable) when
- *                 inputs_on_host != 0 -- they are then copied to the device inside the call --
- *                 else device.
+ *                 inputs_on_host != 0 -- they are then copied to the device inside the call, and a
+ *                 label outside [0, n_classes) is refused with FTP_ERANGE before anything is
+ *                 launched -- else device (labels then clamp as in ftp_run_stage_forward).
  *   loss_host   : if non-NULL (host float[1]) the loss is copied back and the call returns
  *                 after the step has completed; if NULL the call is fully asynchronous. */
 ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, int32_t inputs_on_host, float lr,
                           float* loss_host, void* stream);
+
+/* Waits for the stream, reads the device status word (see "Errors" above) and clears it:
+ * FTP_OK, or FTP_ETIMEOUT if a bounded device-side wait ran out since the last check. */
+ftp_status ftp_check_device_status(ftp_model* m, void* stream);
+/* Test hook: writes `code` into the device status word from the host, as a kernel whose wait ran
+ * out would (0 clears it).  No kernel is launched.  Synchronises the stream. */
+ftp_status ftp_debug_set_device_status(ftp_model* m, int32_t code, void* stream);
 
 /* ---- profile_layers(): Sec. III-B "model profiling" and Sec. III-D "execution profiling". */
 
@@ -262,6 +279,48 @@ ftp_status ftp_recover(ftp_model* m, const ftp_failed_stage* failed, int32_t n_f
                        size_t central_bytes, const int32_t* p_new, int32_t n_new, int32_t* counts /* 3 */,
                        void* stream);
 
+/* ---- training state of a node and the fault handler of the central node: Sec. III-B (Table I), Sec. III-F.
+ * Pure host functions; nothing on the device is involved.
+ *
+ * Table I: every node holds the committed forward id and the committed backward id (the latest batch
+ * that has completed forwarding / backwarding; both start at -1), the learning rate, the epoch and batch
+ * numbers, and `status` (0 normal, 1 fault recovery). */
+typedef struct {
+    int64_t committed_forward_id, committed_backward_id;
+    int32_t status;
+    float learning_rate;
+    int64_t epoch_number, batch_number;
+} ftp_train_state;
+ftp_status ftp_state_init(ftp_train_state* st, float learning_rate, int64_t epoch_number, int64_t batch_number);
+ftp_status ftp_state_forward_done(ftp_train_state* st, int64_t batch_id);
+ftp_status ftp_state_backward_done(ftp_train_state* st, int64_t batch_id);
+/* The central node's timer for batch_id ran out before its gradients came back.  *triggered = 1 and
+ * status becomes 1 if the handler was not running yet; 0 if it was (later timers do not start it again). */
+ftp_status ftp_state_timer_expired(ftp_train_state* st, int64_t batch_id, int32_t* triggered);
+/* *allowed = 0 while status is 1 for batches beyond the committed forward id: they were sent before the
+ * sub-models were rebuilt and are discarded. */
+ftp_status ftp_state_may_forward(const ftp_train_state* st, int64_t batch_id, int32_t* allowed);
+/* Last phase of the handler: both committed ids become batch_id (the batch whose gradients were not
+ * received), status returns to 0; *resume_from (nullable) = the batch to forward first, batch_id. */
+ftp_status ftp_state_reset(ftp_train_state* st, int64_t batch_id, int64_t* resume_from);
+
+/* The three outcomes of the handler's probe.  responses[n_workers]: how each worker of the list answered
+ * (worker 0 is the central node and answers normally).  All normal -> FTP_ACTION_RESTART_BATCH.  All answer
+ * and exactly one has restarted -> FTP_ACTION_RESEND_STATE, *restarted_worker = its index (it is sent the
+ * state variables and reloads its weights from the replica its neighbour keeps).  Otherwise ->
+ * FTP_ACTION_REDISTRIBUTE with failed[0 .. *n_failed) = the workers that were silent or, beside other
+ * faults, restarted (their weights are lost either way), ascending: the input of ftp_recovery_plan. */
+enum { FTP_PROBE_NORMAL = 0, FTP_PROBE_RESTARTED = 1, FTP_PROBE_SILENT = 2 };
+enum { FTP_ACTION_RESTART_BATCH = 0, FTP_ACTION_RESEND_STATE = 1, FTP_ACTION_REDISTRIBUTE = 2 };
+ftp_status ftp_classify_probe(const int32_t* responses, int32_t n_workers, int32_t* action, int32_t* failed /* n_workers */,
+                              int32_t* n_failed, int32_t* restarted_worker);
+
+/* Schedules (Sec. III-D, IV-B): 1 if, after the 0-indexed batch `it` has finished, the dynamic partition
+ * runs (after `first` batches, then whenever the count is a multiple of `period`; the paper uses 10 and
+ * 100) / a replication with the given period runs (chain 50, global 100 in the paper's runs). */
+int32_t ftp_is_repartition_iter(int64_t it, int64_t first, int64_t period);
+int32_t ftp_is_replication_iter(int64_t it, int64_t period);
+
 /* ---- snapshot_weights(stage, dst): Sec. III-E chain / global replication. ----------------- */
 
 /* Copy stage's replica -- per unit of the stage, in order: trainable weights then BN running
@@ -296,8 +355,12 @@ ftp_status ftp_launch_count(const ftp_model* m, int64_t* launches);
  * allocation would stall the device, or a host framework that owns all device memory.  The call
  * itself allocates nothing, on the host or on the device.
  *   - Shapes whose partials exceed the array are refused with FTP_ERANGE (use the model API).
- *   - The first call on a device looks the array's address up (the device must be current); make
- *     that first call outside any stream capture.
+ *   - The first call on a device looks the array's address up (the device must be current).  With
+ *     CUDA's lazy module loading that look-up is also what places the array on the device: an
+ *     implicit allocation that may synchronise the device.  So make that first call during set-up
+ *     -- any small shape will do -- before entering the region that must not allocate, and outside
+ *     any stream capture.  Later calls on that device only read a cached pointer (published
+ *     atomically, so concurrent first calls from several host threads are safe).
  *   - All calls on a device share the array: calls whose kernels may overlap on the GPU (different
  *     streams) race on it.  Nothing needs clearing between calls.
  * Asynchronous on the stream. */

@@ -6,7 +6,8 @@ shares no code with the CUDA library.
 
 Pin status (see tests/test_oracle_*.py):
   ops forward/backward, loss, SGD, stage split, capacity estimate, partition optimiser,
-  redistribution without failure, snapshot, schedules ........ pinned
+  redistribution without failure, snapshot, schedules, the state variables of Table I and the
+  three outcomes of the fault handler's probe (recovery.py) ........ pinned
   redistribution with a failed index (Algorithm 1, I_fail >= 0) and recovery sources after
   failures (Sec. III-F) ... parity unpinned beyond invariants, the prose rules of Sec. III-F and
   the agreement of the prose plan with Algorithm 1 (the worked figures are not available)
@@ -14,3 +15,4 @@ Pin status (see tests/test_oracle_*.py):
 from .ops import *          # noqa: F401,F403
 from .model import OracleModel   # noqa: F401
 from .partition import *    # noqa: F401,F403
+from . import recovery      # noqa: F401

@@ -23,7 +23,13 @@ def _newest(paths):
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(verbose=False, force=False):
+def build(verbose=False, force=False, timeline=False):
+    """timeline=True: the measurement variant (-DFTP_TIMELINE, see csrc/launch.cuh) as libftpipe_timeline.so; load it by
+    setting FTPIPE_LIB to its path."""
+    global OBJ, OUT
+    if timeline:
+        OBJ, OUT = os.path.join(HERE, "_build_timeline"), os.path.join(HERE, "libftpipe_timeline.so")
+        FLAGS.append("-DFTP_TIMELINE")
     os.makedirs(OBJ, exist_ok=True)
     srcs = SOURCES
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
@@ -59,4 +65,4 @@ def build(verbose=False, force=False):
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, timeline="--timeline" in sys.argv))

@@ -10,6 +10,7 @@
 #include <initializer_list>
 #include "kernels.h"
 #include "launch.cuh"
+#include "bn_math.cuh"
 
 namespace ftp {
 
@@ -55,6 +56,10 @@ template <int V> __device__ __forceinline__ void ldv(const __nv_bfloat16* p, flo
         o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
     } else { o[0] = __bfloat162float(*p); }
 }
+template <int V> __device__ __forceinline__ void ldplain(const float* p, float (&o)[V]) {       // coherent load of data the kernel also writes
+    if constexpr (V == 4) { const float4 v = *reinterpret_cast<const float4*>(p); o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w; }
+    else { o[0] = *p; }
+}
 template <int V> __device__ __forceinline__ void stv(float* p, const float (&v)[V]) {
     if constexpr (V == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
     else p[0] = v[0];
@@ -82,22 +87,19 @@ template <int V> __device__ __forceinline__ void ldtab(const float* p, float (&o
     }
 }
 
-__device__ __forceinline__ float act_f(float v, int act) {
-    if (act == 1) return fmaxf(v, 0.f);
-    if (act == 2) return fminf(fmaxf(v, 0.f), 6.f);
-    return v;
-}
-__device__ __forceinline__ bool act_pass(float z, int act) {      // derivative is 1 strictly inside the linear range
-    if (act == 1) return z > 0.f;
-    if (act == 2) return z > 0.f && z < 6.f;
-    return true;
-}
-
-// Normalised value: the mean is a two-float sum and is subtracted first, so that the result keeps
-// float accuracy relative to its own size even when the mean dwarfs the spread.
-__device__ __forceinline__ float bn_z(float y, float mh, float ml, float scale, float beta) {
-    return fmaf((y - mh) - ml, scale, beta);
-}
+// Per-thread constants of a batch norm applied on load to V consecutive channels (see BnXform)
+template <typename T, int V> struct XfRegs {
+    float sc[V], of[V];
+    float lo, hi;
+    __device__ __forceinline__ void load(const BnXform& x, int c) {
+        ldtab<V>(x.scale + c, sc); ldtab<V>(x.offset + c, of);
+        lo = x.lo; hi = x.hi;
+    }
+    __device__ __forceinline__ void apply(float (&v)[V]) const {
+#pragma unroll
+        for (int e = 0; e < V; ++e) v[e] = as_stored<T>(xf_z(v[e], sc[e], of[e], lo, hi));
+    }
+};
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 inline unsigned flat_blocks(long long work, int threads) {
@@ -313,7 +315,7 @@ __device__ __forceinline__ double rsqrt_f64(double v) {
 __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M, double inv_M, double unbias,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
                                    float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd,
-                                   const FinScratch fin) {
+                                   float* offset, const FinScratch fin) {
     grid_dep_sync();
     const int c = blockIdx.x * FIN_X + threadIdx.x;
     float ga = 0.f, be = 0.f, rm = 0.f, rv = 0.f;                    // fetched up front: their latency hides behind the sums
@@ -328,6 +330,7 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
         const double rs = rsqrt_f64(var + (double)eps);
         const float sc = (float)((double)ga * rs);
         scale[c] = sc;
+        offset[c] = (float)((double)be - mu * (double)sc);     // z = y * scale + offset, for readers that normalise as they load
         shift[c] = be;                            // z = (y - mean) * scale + beta, the mean kept as a two-float sum
         const float mh = (float)mu;
         mean[c] = mh;
@@ -523,13 +526,15 @@ __global__ void __launch_bounds__(256) act_bwd_kernel(const T* __restrict__ dout
 // The two gather kernels below map a block of 256 threads onto a tile of 64 output pixels (TW = 2^tws wide,
 // 64 / TW rows of the (image, row) index space) times 8 channel vectors, two pixels per thread, so that the
 // nine taps of neighbouring outputs hit the lines their neighbours just fetched.  grid (pixel tiles, ceil(CV / 8)).
-template <typename T, int V>
-__global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, ConvGeom g, int tws) {
+template <typename T, int V, bool XF>
+__global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, ConvGeom g, int tws, BnXform xf) {
     grid_dep_sync();
     const int CV = g.Cin / V;
     const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
     if (cv >= CV) return;
     const int c = cv * V;
+    XfRegs<T, V> xr;
+    if constexpr (XF) xr.load(xf, c);
     const int slot = threadIdx.x >> 3, TW = 1 << tws, half = 32 >> tws;
     const int tiles_w = (g.Wo + TW - 1) >> tws;
     const int tw_i = blockIdx.x % tiles_w, tr_i = blockIdx.x / tiles_w;
@@ -555,6 +560,7 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(const T* __restrict__ x, co
                 if (wi < 0 || wi >= g.W) continue;
                 float v[V], k[V];
                 ldv<V>(x + ((long long)(n * g.H + hi) * g.W + wi) * g.Cin + c, v);
+                if constexpr (XF) xr.apply(v);
                 ldtab<V>(w + (r * 3 + s) * g.Cin + c, k);
 #pragma unroll
                 for (int e = 0; e < V; ++e) acc[e] = fmaf(v[e], k[e], acc[e]);
@@ -624,13 +630,10 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(const T* __restrict__ dy,
 // 3 x 6 inputs they share, so every input vector is loaded once per row of taps instead of three times and
 // the six loads of a row are in flight together.  Block: 8 channel vectors x 32 strips; strips are numbered
 // row-major over (image, row, strip of 4 columns).
-template <typename T> __device__ __forceinline__ float as_stored(float v);
-template <> __device__ __forceinline__ float as_stored<float>(float v) { return v; }
-template <> __device__ __forceinline__ float as_stored<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
-
-template <typename T, int V, int FLIP, bool STATS>
+template <typename T, int V, int FLIP, bool STATS, bool XF>
 __device__ __forceinline__ void dw_strip_body(const T* __restrict__ x, const float* __restrict__ w, const T* __restrict__ addend, T* __restrict__ y,
-                                              int H, int W, int C, int c, long long strip, int strips_w, float (&su)[V], float (&sq)[V]) {
+                                              int H, int W, int C, int c, long long strip, int strips_w, float (&su)[V], float (&sq)[V],
+                                              const XfRegs<T, V>& xr) {
     const int w0 = (int)(strip % strips_w) * 4;
     const long long R = strip / strips_w;                 // image * H + row
     const int h = (int)(R % H);
@@ -648,8 +651,10 @@ __device__ __forceinline__ void dw_strip_body(const T* __restrict__ x, const flo
 #pragma unroll
         for (int j = 0; j < 6; ++j) {
             const int wi = w0 - 1 + j;
-            if (wi >= 0 && wi < W) ldv<V>(row + (long long)wi * C, in[j]);
-            else {
+            if (wi >= 0 && wi < W) {
+                ldv<V>(row + (long long)wi * C, in[j]);
+                if constexpr (XF) xr.apply(in[j]);
+            } else {
 #pragma unroll
                 for (int e = 0; e < V; ++e) in[j][e] = 0.f;
             }
@@ -684,9 +689,9 @@ __device__ __forceinline__ void dw_strip_body(const T* __restrict__ x, const flo
 
 // STATS: the block also leaves the column sums and sums of squares of the values it stored (as stored: rounded to T)
 // in stats[blockIdx.x][2][C], for the batch norm that follows.
-template <typename T, int V, int FLIP, int STATS>
+template <typename T, int V, int FLIP, int STATS, bool XF>
 __global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, const float* __restrict__ w, const T* __restrict__ addend,
-                                                       T* __restrict__ y, int N, int H, int W, int C, double* __restrict__ stats) {
+                                                       T* __restrict__ y, int N, int H, int W, int C, double* __restrict__ stats, BnXform xf) {
     grid_dep_sync();
     const int CV = C / V;
     const int cv = blockIdx.y * 8 + (threadIdx.x & 7);
@@ -694,12 +699,14 @@ __global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, 
     const int strips_w = (W + 3) >> 2;
     const long long strip = (long long)blockIdx.x * 32 + (threadIdx.x >> 3);
     const bool live = cv < CV && strip < (long long)N * H * strips_w;
+    XfRegs<T, V> xr;
+    if constexpr (XF) { if (cv < CV) xr.load(xf, c); }
     if constexpr (STATS) {
         __shared__ float shs[2][32][8 * V];
         float su[V], sq[V];
 #pragma unroll
         for (int e = 0; e < V; ++e) su[e] = sq[e] = 0.f;
-        if (live) dw_strip_body<T, V, FLIP, true>(x, w, addend, y, H, W, C, c, strip, strips_w, su, sq);
+        if (live) dw_strip_body<T, V, FLIP, true, XF>(x, w, addend, y, H, W, C, c, strip, strips_w, su, sq, xr);
 #pragma unroll
         for (int e = 0; e < V; ++e) { shs[0][threadIdx.x >> 3][(threadIdx.x & 7) * V + e] = su[e]; shs[1][threadIdx.x >> 3][(threadIdx.x & 7) * V + e] = sq[e]; }
         __syncthreads();
@@ -714,7 +721,7 @@ __global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, 
         }
     } else {
         float su[V], sq[V];
-        if (live) dw_strip_body<T, V, FLIP, false>(x, w, addend, y, H, W, C, c, strip, strips_w, su, sq);
+        if (live) dw_strip_body<T, V, FLIP, false, XF>(x, w, addend, y, H, W, C, c, strip, strips_w, su, sq, xr);
     }
 }
 
@@ -722,9 +729,9 @@ __global__ void __launch_bounds__(256) dw_strip_kernel(const T* __restrict__ x, 
 // A thread owns V folded columns (a fixed channel vector and a fixed pixel offset within each folded row)
 // and walks the rows of its chunk; the 9 taps are reduced over y three at a time through shared memory.
 // partial[chunk][9][cols] (float).
-template <typename T, int V>
+template <typename T, int V, bool XF>
 __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, ConvGeom g,
-                                                       int rows, int cols, int f, int rpc) {
+                                                       int rows, int cols, int f, int rpc, BnXform xf) {
     grid_dep_sync();
     __shared__ float sh[3][8][32 * V];
     const int col = (blockIdx.x * 32 + threadIdx.x) * V;
@@ -736,6 +743,8 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, 
         for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
     if (col < cols) {
         const int kf = col / g.Cin, c = col - kf * g.Cin;        // pixel offset inside a folded row, channel
+        XfRegs<T, V> xr;
+        if constexpr (XF) xr.load(xf, c);
         for (int r = r0 + threadIdx.y; r < r1; r += 8) {
             const long long pix = (long long)r * f + kf;
             const int wo = (int)(pix % g.Wo);
@@ -753,6 +762,7 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, 
                     if (wi < 0 || wi >= g.W) continue;
                     float v[V];
                     ldv<V>(x + ((long long)(n * g.H + hi) * g.W + wi) * g.Cin + c, v);
+                    if constexpr (XF) xr.apply(v);
 #pragma unroll
                     for (int e = 0; e < V; ++e) acc[rr * 3 + ss][e] = fmaf(v[e], d[e], acc[rr * 3 + ss][e]);
                 }
@@ -784,9 +794,9 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(const T* __restrict__ x, 
 // thread loads the four output gradients and the 3 x 6 inputs of a strip once and feeds all nine taps from them;
 // it walks strips blockIdx.x * 32 + slot, + gridDim.x * 32, ... with its nine accumulators in registers, and the
 // 32 strip slots of the block are added in slot order through shared memory.  partial[blockIdx.x][9][C] (float).
-template <typename T, int V>
+template <typename T, int V, bool XF>
 __global__ void __launch_bounds__(256) dw_wgrad_strip_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, int N, int H,
-                                                             int W, int C) {
+                                                             int W, int C, BnXform xf) {
     grid_dep_sync();
     __shared__ float sh[3][32][8 * V];
     const int CV = C / V, cvl = threadIdx.x & 7, cv = blockIdx.y * 8 + cvl, slot = threadIdx.x >> 3;
@@ -799,6 +809,8 @@ __global__ void __launch_bounds__(256) dw_wgrad_strip_kernel(const T* __restrict
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
     if (cv < CV) {
+        XfRegs<T, V> xr;
+        if constexpr (XF) xr.load(xf, c);
         for (long long s = (long long)blockIdx.x * 32 + slot; s < strips; s += (long long)gridDim.x * 32) {
             const int w0 = (int)(s % strips_w) * 4;
             const long long R = s / strips_w;
@@ -821,8 +833,10 @@ __global__ void __launch_bounds__(256) dw_wgrad_strip_kernel(const T* __restrict
 #pragma unroll
                 for (int j = 0; j < 6; ++j) {
                     const int wi = w0 - 1 + j;
-                    if (wi >= 0 && wi < W) ldv<V>(row + (long long)wi * C, in[j]);
-                    else {
+                    if (wi >= 0 && wi < W) {
+                        ldv<V>(row + (long long)wi * C, in[j]);
+                        if constexpr (XF) xr.apply(in[j]);
+                    } else {
 #pragma unroll
                         for (int e = 0; e < V; ++e) in[j][e] = 0.f;
                     }
@@ -864,9 +878,9 @@ __global__ void __launch_bounds__(256) dw_wgrad_strip_kernel(const T* __restrict
 // for 10 strips, two slots idle; a block walks strips blockIdx.x * 10 + k, + gridDim.x * 10, ... and adds its slots
 // in slot order through shared memory.  partial[blockIdx.x][9][C] (float).
 constexpr int DW_WG_STRIPS = 10;
-template <typename T, int V>
+template <typename T, int V, bool XF>
 __global__ void __launch_bounds__(256) dw_wgrad_rows_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial, int N, int H,
-                                                             int W, int C) {
+                                                             int W, int C, BnXform xf) {
     grid_dep_sync();
     __shared__ float sh[3][32][8 * V];
     const int CV = C / V, cvl = threadIdx.x & 7, cv = blockIdx.y * 8 + cvl, slot = threadIdx.x >> 3;
@@ -880,6 +894,8 @@ __global__ void __launch_bounds__(256) dw_wgrad_rows_kernel(const T* __restrict_
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[t][e] = 0.f;
     if (cv < CV && k < DW_WG_STRIPS) {
+        XfRegs<T, V> xr;
+        if constexpr (XF) xr.load(xf, c);
         for (long long s = (long long)blockIdx.x * DW_WG_STRIPS + k; s < strips; s += (long long)gridDim.x * DW_WG_STRIPS) {
             const int w0 = (int)(s % strips_w) * 4;
             const long long R = s / strips_w;
@@ -899,8 +915,10 @@ __global__ void __launch_bounds__(256) dw_wgrad_rows_kernel(const T* __restrict_
 #pragma unroll
             for (int j = 0; j < 6; ++j) {
                 const int wi = w0 - 1 + j;
-                if (wi >= 0 && wi < W) ldv<V>(row + (long long)wi * C, in[j]);
-                else {
+                if (wi >= 0 && wi < W) {
+                    ldv<V>(row + (long long)wi * C, in[j]);
+                    if constexpr (XF) xr.apply(in[j]);
+                } else {
 #pragma unroll
                     for (int e = 0; e < V; ++e) in[j][e] = 0.f;
                 }
@@ -963,6 +981,241 @@ __global__ void __launch_bounds__(256) dw_wgrad_finalize_small_kernel(const floa
 #pragma unroll
         for (int y = 0; y < 8; ++y) r += sh[y][threadIdx.x];
         dw[t * C + c] = (float)r;
+    }
+}
+
+// ---- stride-1 depthwise 3x3 on column strips, marching down the rows ---------------------------------------------
+// A thread owns four channels and a strip of four output columns and walks down RH rows of one image with the
+// three input rows of its window (3 x 6 vectors) in registers: every step loads one new row, so an input vector
+// is fetched (RH + 2) / RH * 1.5 times instead of 4.5 times, and a batch norm folded into the load (XF) is
+// evaluated once per fetch.  Block: 8 channel vectors x 32 slots; a slot is (image, row chunk, strip), numbered
+// row-major.  Per output the taps are added in the order of dw_strip_kernel, so both give the same bits.
+template <typename T>
+__device__ __forceinline__ void dw3_fetch_row(const T* __restrict__ img, int hi, int H, int W, int C, int w0, float (&r)[6][4]) {
+#pragma unroll
+    for (int j = 0; j < 6; ++j) {
+        const int wi = w0 - 1 + j;
+        if (hi >= 0 && hi < H && wi >= 0 && wi < W) ldv<4>(img + ((long long)hi * W + wi) * C, r[j]);
+        else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r[j][e] = 0.f;
+        }
+    }
+}
+// a fetched row becomes a window row: the batch norm of the tensor's producer, where one is folded in (padding stays zero)
+template <typename T, bool XF>
+__device__ __forceinline__ void dw3_take_row(const float (&raw)[6][4], int hi, int H, int W, int w0, float (&r)[6][4], const XfRegs<T, 4>& xr) {
+#pragma unroll
+    for (int j = 0; j < 6; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) r[j][e] = raw[j][e];
+        if constexpr (XF) {
+            const int wi = w0 - 1 + j;
+            if (hi >= 0 && hi < H && wi >= 0 && wi < W) xr.apply(r[j]);
+        }
+    }
+}
+template <typename T, bool XF>
+__device__ __forceinline__ void dw3_load_row(const T* __restrict__ img, int hi, int H, int W, int C, int w0, float (&r)[6][4], const XfRegs<T, 4>& xr) {
+    float raw[6][4];
+    dw3_fetch_row<T>(img, hi, H, W, C, w0, raw);
+    dw3_take_row<T, XF>(raw, hi, H, W, w0, r, xr);
+}
+
+template <typename T, bool XF, bool STATS>
+__global__ void __launch_bounds__(256, 2) dw3_fwd_rows_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int N, int H, int W,
+                                                              int C, int RH, int HC, double* __restrict__ stats, BnXform xf) {
+    grid_dep_sync();
+    __shared__ __align__(16) float wsm[9][32];
+    __shared__ float shs[STATS ? 2 : 1][32][33];
+    const int CV = C / 4, cvl = threadIdx.x & 7, slot = threadIdx.x >> 3, cv = blockIdx.y * 8 + cvl, c = cv * 4;
+    for (int i = threadIdx.x; i < 9 * 32; i += 256) {
+        const int tap = i >> 5, ch = blockIdx.y * 32 + (i & 31);
+        wsm[tap][i & 31] = ch < C ? w[tap * C + ch] : 0.f;
+    }
+    __syncthreads();
+    const int strips_w = (W + 3) >> 2;
+    const long long total = (long long)N * HC * strips_w;
+    float su[4] = {0.f, 0.f, 0.f, 0.f}, sq[4] = {0.f, 0.f, 0.f, 0.f};
+    for (long long gs = (long long)blockIdx.x * 32 + slot; cv < CV && gs < total; gs += (long long)gridDim.x * 32) {
+        const int sw = (int)(gs % strips_w);
+        const long long t = gs / strips_w;
+        const int hc = (int)(t % HC), n = (int)(t / HC);
+        const int w0 = sw * 4, h0 = hc * RH, h1 = min(H, h0 + RH);
+        XfRegs<T, 4> xr;
+        if constexpr (XF) xr.load(xf, c);
+        const T* img = x + (long long)n * H * W * C + c;
+        T* out = y + (long long)n * H * W * C + c;
+        float win[3][6][4], nxt[6][4];
+        dw3_load_row<T, XF>(img, h0 - 1, H, W, C, w0, win[0], xr);
+        dw3_load_row<T, XF>(img, h0, H, W, C, w0, win[1], xr);
+        dw3_fetch_row<T>(img, h0 + 1, H, W, C, w0, nxt);
+        for (int h = h0; h < h1; ++h) {
+            dw3_take_row<T, XF>(nxt, h + 1, H, W, w0, win[2], xr);
+            if (h + 1 < h1) dw3_fetch_row<T>(img, h + 2, H, W, C, w0, nxt);         // in flight while this row is computed
+            float acc[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
+#pragma unroll
+            for (int r = 0; r < 3; ++r)
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    const float4 kk = *reinterpret_cast<const float4*>(&wsm[r * 3 + s][cvl * 4]);
+                    const float k4[4] = {kk.x, kk.y, kk.z, kk.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[j][e] = fmaf(win[r][j + s][e], k4[e], acc[j][e]);
+                }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (w0 + j < W) {
+                    stv<4>(out + ((long long)h * W + w0 + j) * C, acc[j]);
+                    if constexpr (STATS) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { const float v = as_stored<T>(acc[j][e]); su[e] += v; sq[e] = fmaf(v, v, sq[e]); }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 6; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { win[0][j][e] = win[1][j][e]; win[1][j][e] = win[2][j][e]; }
+        }
+    }
+    if constexpr (STATS) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { shs[0][slot][cvl * 4 + e] = su[e]; shs[1][slot][cvl * 4 + e] = sq[e]; }
+        __syncthreads();
+        if (threadIdx.x < 64) {
+            const int a = threadIdx.x >> 5, ch = threadIdx.x & 31, gc = blockIdx.y * 32 + ch;
+            if (gc < C) {
+                double tsum = 0.0;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) tsum += (double)shs[a][q][ch];
+                stats[((long long)blockIdx.x * 2 + a) * C + gc] = tsum;
+            }
+        }
+    }
+}
+
+// Data gradient and weight gradient of the same convolution in one pass over dy: with the 3 x 6 window of output
+// gradients around its four pixels of a row in registers, a thread forms dx (the taps mirrored, added in the
+// order of dw_strip_kernel<FLIP = 1>) and adds x[pixel] * dy[pixel + offset] to the nine weight-gradient sums of its
+// four channels, which it carries down its rows.  At the end the 32 slots of a block are added in slot order:
+// partial[blockIdx.x][9][C] (float), summed over blocks by the finalize kernels.  dx may be NULL (no input gradient).
+template <typename T, bool XF>
+__global__ void __launch_bounds__(256) dw3_bwd_rows_kernel(const T* __restrict__ x, const T* __restrict__ dy, const float* __restrict__ w,
+                                                           const T* __restrict__ addend, T* __restrict__ dx, float* __restrict__ partial, int N, int H,
+                                                           int W, int C, int RH, int HC, BnXform xf) {
+    grid_dep_sync();
+    __shared__ __align__(16) float wsm[9][32];
+    __shared__ float sh[3][32][33];
+    const int CV = C / 4, cvl = threadIdx.x & 7, slot = threadIdx.x >> 3, cv = blockIdx.y * 8 + cvl, c = cv * 4;
+    for (int i = threadIdx.x; i < 9 * 32; i += 256) {
+        const int tap = i >> 5, ch = blockIdx.y * 32 + (i & 31);
+        wsm[tap][i & 31] = ch < C ? w[tap * C + ch] : 0.f;
+    }
+    __syncthreads();
+    const int strips_w = (W + 3) >> 2;
+    const long long total = (long long)N * HC * strips_w;
+    float dwa[9][4];
+#pragma unroll
+    for (int tap = 0; tap < 9; ++tap)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dwa[tap][e] = 0.f;
+    for (long long gs = (long long)blockIdx.x * 32 + slot; cv < CV && gs < total; gs += (long long)gridDim.x * 32) {
+        const int sw = (int)(gs % strips_w);
+        const long long t = gs / strips_w;
+        const int hc = (int)(t % HC), n = (int)(t / HC);
+        const int w0 = sw * 4, h0 = hc * RH, h1 = min(H, h0 + RH);
+        XfRegs<T, 4> xr, none;
+        if constexpr (XF) xr.load(xf, c);
+        const long long ioff = (long long)n * H * W * C + c;
+        const T* gimg = dy + ioff;
+        float win[3][6][4];
+        dw3_load_row<T, false>(gimg, h0 - 1, H, W, C, w0, win[0], none);
+        dw3_load_row<T, false>(gimg, h0, H, W, C, w0, win[1], none);
+        dw3_fetch_row<T>(gimg, h0 + 1, H, W, C, w0, win[2]);
+        float xnext[4][4];
+        auto fetch_x = [&](int h) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (w0 + j < W) ldv<4>(x + ioff + ((long long)h * W + w0 + j) * C, xnext[j]);
+                else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) xnext[j][e] = 0.f;
+                }
+            }
+        };
+        fetch_x(h0);
+        for (int h = h0; h < h1; ++h) {
+            float xv[4][4], acc[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { xv[j][e] = xnext[j][e]; acc[j][e] = 0.f; }
+                if constexpr (XF) { if (w0 + j < W) xr.apply(xv[j]); }
+            }
+            if (h + 1 < h1) fetch_x(h + 1);                      // lands while this row is computed
+#pragma unroll
+            for (int r = 0; r < 3; ++r)
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    const int tap = (2 - r) * 3 + (2 - s);
+                    const float4 kk = *reinterpret_cast<const float4*>(&wsm[tap][cvl * 4]);
+                    const float k4[4] = {kk.x, kk.y, kk.z, kk.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[j][e] = fmaf(win[r][j + s][e], k4[e], acc[j][e]);
+                            dwa[tap][e] = fmaf(xv[j][e], win[r][j + s][e], dwa[tap][e]);
+                        }
+                }
+            // the window moves down one row; the row after it is fetched now and lands while the next x row is awaited
+#pragma unroll
+            for (int j = 0; j < 6; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { win[0][j][e] = win[1][j][e]; win[1][j][e] = win[2][j][e]; }
+            if (h + 1 < h1) dw3_fetch_row<T>(gimg, h + 2, H, W, C, w0, win[2]);
+            if (dx) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (w0 + j < W) {
+                        const long long o = ioff + ((long long)h * W + w0 + j) * C;
+                        if (addend) {
+                            float a[4];
+                            ldv<4>(addend + o, a);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) acc[j][e] += a[e];
+                        }
+                        stv<4>(dx + o, acc[j]);
+                    }
+                }
+            }
+        }
+    }
+    // the nine sums of every channel over the block's 32 slots, three taps at a time, in slot order
+#pragma unroll
+    for (int gq = 0; gq < 3; ++gq) {
+        __syncthreads();
+#pragma unroll
+        for (int tq = 0; tq < 3; ++tq)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sh[tq][slot][cvl * 4 + e] = dwa[gq * 3 + tq][e];
+        __syncthreads();
+        if (threadIdx.x < 96) {
+            const int tq = threadIdx.x >> 5, ch = threadIdx.x & 31, gc = blockIdx.y * 32 + ch;
+            if (gc < C) {
+                float sum = 0.f;
+#pragma unroll 8
+                for (int q = 0; q < 32; ++q) sum += sh[tq][q][ch];
+                partial[((long long)blockIdx.x * 9 + gq * 3 + tq) * C + gc] = sum;
+            }
+        }
     }
 }
 
@@ -1109,20 +1362,37 @@ __global__ void loss_mean_kernel(const float* __restrict__ per_sample, int N, fl
 }
 
 // ---- SGD ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void sgd_one(float* w, const float* g, float* m, long long i, float lr, float mu, float wd, int first, __nv_bfloat16* shadow,
+                                        float* lo, float* snap_dev, float* snap_host) {
+    float wv = w[i], gv = fmaf(wd, wv, g[i]);
+    if (m) {
+        if (!first) gv = fmaf(mu, m[i], gv);
+        m[i] = gv;
+    }
+    wv = fmaf(-lr, gv, wv);
+    w[i] = wv;
+    if (lo) lo[i] = wv - __uint_as_float(__float_as_uint(wv) & 0xffffe000u);
+    if (snap_dev) snap_dev[i] = wv;
+    if (snap_host) snap_host[i] = wv;
+    if (shadow) shadow[i] = __float2bfloat16_rn(wv);
+}
+
+// nvec vectors of V parameters, then `tail` (< V) single parameters
 template <int V>
-__global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, long long nvec, float lr,
+__global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const float* __restrict__ g, float* __restrict__ m, long long nvec, int tail, float lr,
                                                   float mu, float wd, int first, __nv_bfloat16* __restrict__ shadow, float* __restrict__ lo,
                                                   float* __restrict__ snap_dev, float* __restrict__ snap_host) {
     grid_dep_sync();
+    if (blockIdx.x == 0 && (int)threadIdx.x < tail) sgd_one(w, g, m, nvec * V + threadIdx.x, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         float wv[V], gv[V], mv[V];
-        ldv<V>(w + i * V, wv);
+        ldplain<V>(w + i * V, wv);           // w and m are written below: plain loads, not the read-only path
         ldv<V>(g + i * V, gv);
 #pragma unroll
         for (int e = 0; e < V; ++e) gv[e] = fmaf(wd, wv[e], gv[e]);
         if (m) {
             if (!first) {
-                ldv<V>(m + i * V, mv);
+                ldplain<V>(m + i * V, mv);
 #pragma unroll
                 for (int e = 0; e < V; ++e) gv[e] = fmaf(mu, mv[e], gv[e]);
             }
@@ -1189,9 +1459,17 @@ __global__ void transpose_split_f32_kernel(const TransposeEntryDev* __restrict__
                                            float* __restrict__ wt, float* __restrict__ wtl) {
     grid_dep_sync();
     __shared__ float tile[32][33];
+    __shared__ int first_tile[256];
     const int t = tile_base + blockIdx.x;
+    const int tid = threadIdx.y * 32 + threadIdx.x;
     int e = 0;
-    while (e + 1 < n && table[e + 1].tile0 <= t) ++e;
+    if (n <= 256) {                     // the entries' first tiles, fetched by all threads at once instead of one after the other
+        if (tid < n) first_tile[tid] = table[tid].tile0;
+        __syncthreads();
+        while (e + 1 < n && first_tile[e + 1] <= t) ++e;
+    } else {
+        while (e + 1 < n && table[e + 1].tile0 <= t) ++e;
+    }
     const TransposeEntryDev en = table[e];
     const int local = t - en.tile0, tn = (en.N + 31) / 32;
     const int k0 = (local / tn) * 32, n0 = (local % tn) * 32;
@@ -1290,9 +1568,9 @@ PartialSums bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double*
 
 void bn_finalize(const PartialSums& ps, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
-                 float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st) {
+                 float* mean_lo, float* rstd, float* offset, const FinScratch& fin, cudaStream_t st) {
     launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp, (double)M,
-           1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0, gamma, beta, eps, momentum, run_mean, run_var, scale, shift, mean, mean_lo, rstd, fin);
+           1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0, gamma, beta, eps, momentum, run_mean, run_var, scale, shift, mean, mean_lo, rstd, offset, fin);
 }
 
 template <typename T>
@@ -1367,24 +1645,75 @@ void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int
 // log2 of the tile width: the largest power of two <= min(8, width)
 static inline int dw_tile_shift(int width) { return width >= 8 ? 3 : width >= 4 ? 2 : width >= 2 ? 1 : 0; }
 
+// Row chunks per image for the row-marching kernels.  A block walks groups of 32 slots (blockIdx.x, + gridDim.x, ...);
+// `resident_blocks` blocks are resident at once.  Longer walks re-load fewer halo rows, shorter ones balance the blocks better.
+struct Dw3Plan { int RH, HC; unsigned gx, gy; long long groups; };
+static Dw3Plan plan_dw3(const ConvGeom& g, int resident_blocks) {
+    const int strips_w = (g.W + 3) / 4, cgroups = (g.Cin / 4 + 7) / 8;
+    const long long slots_x = std::max(1, resident_blocks / cgroups);
+    auto groups = [&](int hc) { return ((long long)g.N * hc * strips_w + 31) / 32; };
+    // chunks of about eight rows: a quarter more rows loaded than computed, and enough groups that the blocks' shares differ little
+    int best = 1;
+    while ((g.H + best - 1) / best > 8) best *= 2;
+    (void)groups;
+    Dw3Plan p;
+    p.RH = (g.H + best - 1) / best;
+    p.HC = (g.H + p.RH - 1) / p.RH;
+    p.groups = groups(p.HC);
+    p.gx = (unsigned)std::min<long long>(p.groups, slots_x);
+    p.gy = (unsigned)cgroups;
+    return p;
+}
+// FTP_DW_ROWS: 0 never, 1 float tensors only (default: on bf16 tensors the two separate kernels, one of them on the
+// second stream, are faster), 2 always
+static bool dw_rows_enabled(size_t elem_bytes) {
+    static int on = -1;
+    if (on < 0) { const char* e = std::getenv("FTP_DW_ROWS"); on = e ? std::atoi(e) : 1; }
+    return on == 2 || (on == 1 && elem_bytes == 4);
+}
+
 template <typename T>
-void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st, const ColStatsReq* stats) {
+void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st, const ColStatsReq* stats, const BnXform* x_xform) {
     constexpr int V = VecOf<T>::N;
     const int tws = dw_tile_shift(g.Wo);
     const unsigned tiles = (unsigned)(((g.Wo + (1 << tws) - 1) >> tws) * (((long long)g.N * g.Ho + (64 >> tws) - 1) / (64 >> tws)));
     if (stats) stats->out->entries = 0;
-    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w)) {
+    const bool xf = x_xform != nullptr;
+    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f};
+    const bool xf_vec = !xf || (aligned16(xv.scale) && aligned16(xv.offset));
+    if (dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w) && xf_vec) {
+        const Dw3Plan pl = plan_dw3(g, 2 * sm_count());
+        const dim3 grid(pl.gx, pl.gy);
+        double* sp = stats ? stats->partial : nullptr;
+        if (stats) {
+            if (xf) launch(dw3_fwd_rows_kernel<T, true, true>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, sp, xv);
+            else launch(dw3_fwd_rows_kernel<T, false, true>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, sp, xv);
+            *stats->out = PartialSums{stats->partial, (int)grid.x, 1};
+        } else if (xf) launch(dw3_fwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, sp, xv);
+        else launch(dw3_fwd_rows_kernel<T, false, false>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, sp, xv);
+        return;
+    }
+    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w) && xf_vec) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
         const dim3 grid((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8);
         // four channels per thread for either type: eight lanes of a block then cover 32 channels, which every layer has
         if (stats) {
-            launch(dw_strip_kernel<T, 4, 0, 1>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, stats->partial);
+            if (xf) launch(dw_strip_kernel<T, 4, 0, 1, true>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, stats->partial, xv);
+            else launch(dw_strip_kernel<T, 4, 0, 1, false>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, stats->partial, xv);
             *stats->out = PartialSums{stats->partial, (int)grid.x, 1};
-        } else launch(dw_strip_kernel<T, 4, 0, 0>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, (double*)nullptr);
+        } else if (xf) launch(dw_strip_kernel<T, 4, 0, 0, true>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, (double*)nullptr, xv);
+        else launch(dw_strip_kernel<T, 4, 0, 0, false>, grid, dim3(256), 0, st, x, w, (const T*)nullptr, y, g.N, g.H, g.W, g.Cin, (double*)nullptr, xv);
         return;
     }
-    if (can_vec<T>(g.Cin, x, y) && aligned16(w)) launch(dw_fwd_kernel<T, V>, dim3(tiles, (g.Cin / V + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
-    else launch(dw_fwd_kernel<T, 1>, dim3(tiles, (g.Cin + 7) / 8), dim3(256), 0, st, x, w, y, g, tws);
+    if (can_vec<T>(g.Cin, x, y) && aligned16(w) && xf_vec) {
+        const dim3 grid(tiles, (g.Cin / V + 7) / 8);
+        if (xf) launch(dw_fwd_kernel<T, V, true>, grid, dim3(256), 0, st, x, w, y, g, tws, xv);
+        else launch(dw_fwd_kernel<T, V, false>, grid, dim3(256), 0, st, x, w, y, g, tws, xv);
+    } else {
+        const dim3 grid(tiles, (g.Cin + 7) / 8);
+        if (xf) launch(dw_fwd_kernel<T, 1, true>, grid, dim3(256), 0, st, x, w, y, g, tws, xv);
+        else launch(dw_fwd_kernel<T, 1, false>, grid, dim3(256), 0, st, x, w, y, g, tws, xv);
+    }
 }
 
 template <typename T>
@@ -1394,7 +1723,8 @@ void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const Con
     const unsigned tiles = (unsigned)(((g.W + (1 << tws) - 1) >> tws) * (((long long)g.N * g.H + (64 >> tws) - 1) / (64 >> tws)));
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
-        launch(dw_strip_kernel<T, 4, 1, 0>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin, (double*)nullptr);
+        launch(dw_strip_kernel<T, 4, 1, 0, false>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin, (double*)nullptr,
+               BnXform{nullptr, nullptr, 0.f, 0.f});
         return;
     }
     if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
@@ -1423,20 +1753,30 @@ static inline int dw_wgrad_strip_blocks(const ConvGeom& g, int V, bool rows_vari
 size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
     const FoldPlan a = plan_dw_wgrad(g, 4), b = plan_dw_wgrad(g, 2);
     size_t n = std::max((size_t)a.chunks * 9 * a.cols, (size_t)b.chunks * 9 * b.cols);
+    if (g.Cin % 4 == 0 && g.stride == 1) n = std::max(n, (size_t)plan_dw3(g, sm_count()).gx * 9 * g.Cin);
     if (g.Cin % 4 == 0) n = std::max(n, (size_t)std::max(dw_wgrad_strip_blocks(g, 4, false), dw_wgrad_strip_blocks(g, 4, true)) * 9 * g.Cin);
     return n;
 }
 
 template <typename T>
-void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st) {
+void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st, const BnXform* x_xform) {
     constexpr int V = VecOf<T>::N;
+    const bool xf = x_xform != nullptr;
+    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f};
+    const bool xf_vec = !xf || (aligned16(xv.scale) && aligned16(xv.offset));
     // four channels per thread for either type: with eight bf16 channels the nine accumulators would leave too few warps per SM
-    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy)) {
+    if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy) && xf_vec) {
         constexpr int SV = 4;
         constexpr bool rows_variant = sizeof(T) == 2;
         const int gx = dw_wgrad_strip_blocks(g, SV, rows_variant);
-        if (rows_variant) launch(dw_wgrad_rows_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
-        else launch(dw_wgrad_strip_kernel<T, SV>, dim3(gx, (g.Cin / SV + 7) / 8), dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin);
+        const dim3 grid(gx, (g.Cin / SV + 7) / 8);
+        if (rows_variant) {
+            if (xf) launch(dw_wgrad_rows_kernel<T, SV, true>, grid, dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin, xv);
+            else launch(dw_wgrad_rows_kernel<T, SV, false>, grid, dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin, xv);
+        } else {
+            if (xf) launch(dw_wgrad_strip_kernel<T, SV, true>, grid, dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin, xv);
+            else launch(dw_wgrad_strip_kernel<T, SV, false>, grid, dim3(256), 0, st, x, dy, scratch, g.N, g.H, g.W, g.Cin, xv);
+        }
         if (gx <= DW_FIN_SMALL) {
             launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
             return;
@@ -1448,12 +1788,37 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
     }
     FoldPlan fp = plan_dw_wgrad(g, (int)sizeof(T));
     const int rpc = fold_rpc(fp);
-    if (fp.vec == V && aligned16(x) && aligned16(dy))
-        launch(dw_wgrad_kernel<T, V>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
-    else
-        launch(dw_wgrad_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc);
+    if (fp.vec == V && aligned16(x) && aligned16(dy) && xf_vec) {
+        if (xf) launch(dw_wgrad_kernel<T, V, true>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc, xv);
+        else launch(dw_wgrad_kernel<T, V, false>, dim3(fold_grid(fp)), dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc, xv);
+    } else {
+        const dim3 grid((fp.cols + 31) / 32, fp.chunks);
+        if (xf) launch(dw_wgrad_kernel<T, 1, true>, grid, dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc, xv);
+        else launch(dw_wgrad_kernel<T, 1, false>, grid, dim3(32, 8), 0, st, x, dy, scratch, g, fp.rows, fp.cols, fp.f, rpc, xv);
+    }
     if (fp.chunks * fp.f <= DW_FIN_SMALL) launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw);
     else launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, fin_slices(fp), 9), dim3(FIN_X, FIN_Y), 0, st, scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
+}
+
+template <typename T>
+bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
+                      cudaStream_t st, const BnXform* x_xform) {
+    const bool xf = x_xform != nullptr;
+    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f};
+    const bool xf_vec = !xf || (aligned16(xv.scale) && aligned16(xv.offset));
+    if (!(dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy, addend, dx) && g.Cin % 4 == 0 && xf_vec)) return false;
+    const Dw3Plan pl = plan_dw3(g, sm_count());
+    const dim3 grid(pl.gx, pl.gy);
+    if (xf) launch(dw3_bwd_rows_kernel<T, true>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv);
+    else launch(dw3_bwd_rows_kernel<T, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv);
+    const int gx = (int)pl.gx;
+    if (gx <= DW_FIN_SMALL) launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
+    else {
+        int slices = gx / (4 * FIN_Y);
+        slices = slices < 1 ? 1 : (slices > FIN_GMAX ? FIN_GMAX : slices);
+        launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, slices, 9), dim3(FIN_X, FIN_Y), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw, fin);
+    }
+    return true;
 }
 
 template <typename T>
@@ -1495,9 +1860,9 @@ void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, 
 
 void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
                 __nv_bfloat16* shadow, float* lo, float* snap_dev, float* snap_host, cudaStream_t st) {
-    const bool v = n % 4 == 0 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(lo) && aligned16(snap_dev) && aligned16(snap_host);
-    if (v) launch(sgd_kernel<4>, dim3(flat_blocks(n / 4, 256)), dim3(256), 0, st, w, g, m, n / 4, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
-    else launch(sgd_kernel<1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, g, m, n, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
+    const bool v = n >= 4 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(lo) && aligned16(snap_dev) && aligned16(snap_host);
+    if (v) launch(sgd_kernel<4>, dim3(flat_blocks(n / 4, 256)), dim3(256), 0, st, w, g, m, n / 4, (int)(n % 4), lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
+    else launch(sgd_kernel<1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, g, m, n, 0, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
 }
 
 void tf32_lo(const float* w, float* lo, long long n, cudaStream_t st) {
@@ -1532,9 +1897,10 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
                                   const FinScratch&, cudaStream_t);                                                                           \
     template void act_fwd<T>(const T*, T*, long long, int, cudaStream_t);                                                   \
     template void act_bwd<T>(const T*, const T*, const T*, T*, long long, int, cudaStream_t);                               \
-    template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t, const ColStatsReq*);             \
+    template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t, const ColStatsReq*, const BnXform*); \
     template void dwconv_dgrad<T>(const T*, const float*, const T*, T*, const ConvGeom&, cudaStream_t);                     \
-    template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t);                       \
+    template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*); \
+    template bool dwconv_bwd_fused<T>(const T*, const T*, const float*, const T*, T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*); \
     template void maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);                                           \
     template void maxpool_bwd<T>(const T*, const T*, T*, int, int, int, int, cudaStream_t);                                 \
     template void gap_fwd<T>(const T*, T*, int, int, int, cudaStream_t);                                                    \

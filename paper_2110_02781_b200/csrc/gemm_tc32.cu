@@ -17,6 +17,7 @@
 //    converter warps only add the lo parts.
 // Every wait is bounded; see gemm_tc.cu for the error protocol.
 #include "gemm_tc_common.cuh"
+#include "bn_math.cuh"
 
 namespace ftp {
 using namespace tc;
@@ -46,6 +47,60 @@ __device__ __forceinline__ void split_tile(const uint8_t* hi, uint8_t* lo, int b
     }
 }
 
+__device__ __forceinline__ float tf32_lo_of(float v) { return v - __uint_as_float(__float_as_uint(v) & 0xffffe000u); }
+
+// Batch norm + activation on a float4 of four consecutive channels (constants in registers), zero where !keep
+struct Xf4 {
+    float4 sc, of;
+    __device__ __forceinline__ void load(const BnXform& x, int c, bool ok) {
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        sc = ok ? __ldg(reinterpret_cast<const float4*>(x.scale + c)) : z;
+        of = ok ? __ldg(reinterpret_cast<const float4*>(x.offset + c)) : z;
+    }
+    __device__ __forceinline__ float4 apply(float4 v, float lo, float hi, bool keep) const {
+        float4 o;
+        o.x = keep ? xf_z(v.x, sc.x, of.x, lo, hi) : 0.f;
+        o.y = keep ? xf_z(v.y, sc.y, of.y, lo, hi) : 0.f;
+        o.z = keep ? xf_z(v.z, sc.z, of.z, lo, hi) : 0.f;
+        o.w = keep ? xf_z(v.w, sc.w, of.w, lo, hi) : 0.f;
+        return o;
+    }
+};
+
+// A K-major 128 x 32 float tile (128-byte rows, 16-byte pieces XOR-swizzled with row % 8) whose values are the input
+// of a batch norm: 128 threads replace every value by its normalised, activated value (rows past `rows_valid` and
+// channels past the end of the reduction become zero, as padding must) and write the lo part.  Thread t owns the
+// physical piece t % 8 of rows t / 8 + 16 j, which is the same logical piece -- the same four channels -- in every row.
+__device__ __forceinline__ void xform_split_tile_k(uint8_t* hi, uint8_t* lo, int t, const Xf4& c, float zlo, float zhi, bool chan_ok, int rows_valid) {
+    const int row0 = t >> 3;
+    uint8_t* p = hi + row0 * 128 + (t & 7) * 16;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int row = row0 + 16 * j;
+        const float4 v = *reinterpret_cast<const float4*>(p + j * 2048);
+        const float4 z = c.apply(v, zlo, zhi, chan_ok && row < rows_valid);
+        *reinterpret_cast<float4*>(p + j * 2048) = z;
+        *reinterpret_cast<float4*>(p + j * 2048 + (lo - hi)) = make_float4(tf32_lo_of(z.x), tf32_lo_of(z.y), tf32_lo_of(z.z), tf32_lo_of(z.w));
+    }
+}
+
+// The same for an MN-major operand of the weight gradient: `slabs` slabs of 32 reduction rows x 32 channels (128-byte
+// rows, 32-byte pieces XOR-swizzled with row % 4), 256 threads.  Thread t owns the 16-byte piece t % 8 of row t / 8 in
+// every slab: channels 8 * ((t % 8 / 2) ^ (row % 4)) + 4 * (t % 2) of the slab, whose constants are c[slab].
+__device__ __forceinline__ void xform_split_slabs_mn(uint8_t* hi, uint8_t* lo, int slabs, int t, const Xf4 (&c)[4], const bool (&chan_ok)[4], float zlo,
+                                                     float zhi, bool row_ok) {
+#pragma unroll
+    for (int n = 0; n < 4; ++n) {
+        if (n < slabs) {
+            uint8_t* q = hi + n * 4096 + t * 16;
+            const float4 v = *reinterpret_cast<const float4*>(q);
+            const float4 z = c[n].apply(v, zlo, zhi, row_ok && chan_ok[n]);
+            *reinterpret_cast<float4*>(q) = z;
+            *reinterpret_cast<float4*>(q + (lo - hi)) = make_float4(tf32_lo_of(z.x), tf32_lo_of(z.y), tf32_lo_of(z.z), tf32_lo_of(z.w));
+        }
+    }
+}
+
 struct T32Params {
     float* D;              // output [S][M][N]: the result itself when S == 1, else partial sums over slices of the reduction
     const float* addend;   // gemm with S == 1 only, nullable
@@ -54,6 +109,8 @@ struct T32Params {
     int b_lo_given;        // gemm: the lo part of B comes from memory (mapBlo) instead of being computed per tile
     int* err;
     double* stats;         // gemm with S == 1 only, nullable: [row tiles][2][N] column sums and sums of squares of each output tile
+    BnXform xf;            // xf.scale != nullptr: a batch norm applied to one operand while its tiles are split (gemm: A; wgrad: see xf_operand)
+    int xf_operand;        // wgrad: 1 = the A operand is transformed, 2 = the B operand
 };
 
 // Epilogue shared by both kernels, run by warps 2..5: accumulator -> shared-memory tiles of 128 rows x 32 columns
@@ -220,13 +277,19 @@ __global__ void __launch_bounds__(TC_THREADS) tc32_kernel(const __grid_constant_
         // ---- warps 2..5: lo part of every landed stage, then the epilogue ----
         const int t = threadIdx.x - 64;
         bool ok = true;
+        const bool xf = p.xf.scale != nullptr;
+        const int xf_piece = (t & 7) ^ ((t >> 3) & 7);          // logical 16-byte piece (four channels) of this thread's pieces
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % STAGES;
             const uint32_t ph = (kb / STAGES) & 1;
+            Xf4 xc;
+            const int xch = kbeg + kb * T32_BK + 4 * xf_piece;
+            if (xf) xc.load(p.xf, xch, xch < p.K);               // fetched while the tile is still in flight
             ok = mbar_wait(full0 + 8 * s, ph, p.err, 13);
             if (!ok) break;
             uint8_t* st = smem + s * STAGE_BYTES;
-            split_tile(st, st + A_BYTES, A_BYTES, t, 128);
+            if (xf) xform_split_tile_k(st, st + A_BYTES, t, xc, p.xf.lo, p.xf.hi, xch < p.K, p.M - m0);
+            else split_tile(st, st + A_BYTES, A_BYTES, t, 128);
             if (!b_pre) split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, B_BYTES, t, 128);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
             mbar_arrive(ready0 + 8 * s);
@@ -366,13 +429,31 @@ __global__ void __launch_bounds__(WG32_THREADS) tc32_wgrad_kernel(const __grid_c
                 for (int i = slabsB * SLAB + t * 16; i < (int)B_BYTES; i += WG32_CONV * 16) { *reinterpret_cast<float4*>(st + 2 * A_BYTES + i) = z; *reinterpret_cast<float4*>(st + 2 * A_BYTES + B_BYTES + i) = z; }
             }
         }
+        // a batch norm applied to one operand as it is split: this thread's channels are the same in every block of the reduction
+        const int xop = p.xf.scale != nullptr ? p.xf_operand : 0;
+        Xf4 xc[4];
+        bool xok[4] = {false, false, false, false};
+        const int xrow = t >> 3;
+        if (xop) {
+            const int cw = 8 * (((t & 7) >> 1) ^ (xrow & 3)) + 4 * (t & 1);
+            const int o0 = xop == 1 ? m0 : n0, lim = xop == 1 ? p.M : p.N, nsl = xop == 1 ? slabsA : slabsB;
+#pragma unroll
+            for (int n = 0; n < 4; ++n) {
+                const int ch = o0 + 32 * n + cw;
+                xok[n] = n < nsl && ch < lim;
+                xc[n].load(p.xf, ch, xok[n]);
+            }
+        }
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % NSTG;
             ok = mbar_wait(full0 + 8 * s, (kb / NSTG) & 1, p.err, 13);
             if (!ok) break;
             uint8_t* st = smem + s * STAGE_BYTES;
-            split_tile(st, st + A_BYTES, slabsA * SLAB, t, WG32_CONV);
-            split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB * SLAB, t, WG32_CONV);
+            const bool row_ok = kbeg + kb * T32_BK + xrow < kend;
+            if (xop == 1) xform_split_slabs_mn(st, st + A_BYTES, slabsA, t, xc, xok, p.xf.lo, p.xf.hi, row_ok);
+            else split_tile(st, st + A_BYTES, slabsA * SLAB, t, WG32_CONV);
+            if (xop == 2) xform_split_slabs_mn(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB, t, xc, xok, p.xf.lo, p.xf.hi, row_ok);
+            else split_tile(st + 2 * A_BYTES, st + 2 * A_BYTES + B_BYTES, slabsB * SLAB, t, WG32_CONV);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic-proxy writes -> visible to the tensor cores
             mbar_arrive(ready0 + 8 * s);
         }
@@ -444,7 +525,9 @@ Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
     const int m = w.swap ? No : Mo, n = w.swap ? Mo : No;
     w.BN = bn_for(n);
     const long long tiles = (long long)((m + TC_BM - 1) / TC_BM) * ((n + w.BN - 1) / w.BN);
-    long long S = (2LL * sm_count() + tiles - 1) / tiles;
+    // as many blocks as the SMs hold at once (two per SM up to 64-wide tiles, one for 128-wide: see Wg32Smem), no second wave
+    const long long per_sm = w.BN <= 64 ? 2 : 1;
+    long long S = (per_sm * sm_count()) / tiles;
     const long long maxS = (R + 255) / 256;
     long long cap = (2LL << 20) / ((long long)Mo * No);                     // partial sums cost traffic too: at most 2 Mi floats
     if (cap < 1) cap = 1;
@@ -457,29 +540,37 @@ Wg32Plan plan_wgrad32(long long R, int Mo, int No) {
     return w;
 }
 
-// out[i][j] = sum_z partial[z][j][i] (partial slices are [cols][rows] = the transpose of out[rows][cols]); z in eight
-// interleaved runs combined in run order, as in the plain second pass
-__global__ void __launch_bounds__(256) slice_sum_transposed_kernel(const float* __restrict__ partial, int S, int rows, int cols, float* __restrict__ out) {
+// out[i][j] = sum_z partial[z][j][i]: the slices are [cols][rows] (the transpose of out[rows][cols]).  One block per
+// 32 x 32 tile of out: thread (x, y) reads element (j0 + y + 8 q, i0 + x) of the slices z = y', y' + 4, ... for q = 0..3
+// (reads run along the slices' contiguous dimension), the four runs of slices are added in run order, and the tile is
+// turned in shared memory so that the stores are contiguous too.  Block (32, 8, 4): z = slice run.
+__global__ void __launch_bounds__(1024) slice_sum_transposed_kernel(const float* __restrict__ partial, int S, int rows, int cols, float* __restrict__ out) {
     grid_dep_sync();
-    __shared__ float sh[8][33];
+    __shared__ float tile[4][32][33];
     const long long count = (long long)rows * cols;
-    const long long e = (long long)blockIdx.x * 32 + threadIdx.x;
-    float s0 = 0.f, s1 = 0.f;
-    if (e < count) {
-        const long long src = (e % cols) * rows + e / cols;
-        for (int z = threadIdx.y; z < S; z += 16) {
-            const float a = partial[(long long)z * count + src];
-            const float b = z + 8 < S ? partial[(long long)(z + 8) * count + src] : 0.f;
-            s0 += a; s1 += b;
+    const int i0 = blockIdx.x * 32, j0 = blockIdx.y * 32;            // out rows i0.., out columns j0..
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const int i = i0 + threadIdx.x;
+    for (int z = threadIdx.z; z < S; z += 4) {
+        const float* sl = partial + (long long)z * count;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int j = j0 + threadIdx.y + 8 * q;
+            if (j < cols && i < rows) acc[q] += sl[(long long)j * rows + i];
         }
     }
-    sh[threadIdx.y][threadIdx.x] = s0 + s1;
-    __syncthreads();
-    if (threadIdx.y == 0 && e < count) {
-        float s = 0.f;
 #pragma unroll
-        for (int y = 0; y < 8; ++y) s += sh[y][threadIdx.x];
-        out[e] = s;
+    for (int q = 0; q < 4; ++q) tile[threadIdx.z][threadIdx.y + 8 * q][threadIdx.x] = acc[q];
+    __syncthreads();
+    if (threadIdx.z == 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int io = i0 + threadIdx.y + 8 * q, jo = j0 + threadIdx.x;
+            if (io < rows && jo < cols) {
+                const int a = threadIdx.x, b = threadIdx.y + 8 * q;
+                out[(long long)io * cols + jo] = (tile[0][a][b] + tile[1][a][b]) + (tile[2][a][b] + tile[3][a][b]);
+            }
+        }
     }
 }
 
@@ -495,17 +586,23 @@ constexpr int max_stages32(int BN) {
     return n > 4 ? 4 : n;
 }
 
+// blocks of tc32_kernel<BN, stages> that an SM holds at once: shared memory (ring or the epilogue's staging tile,
+// whichever is larger), tensor-memory columns, threads
+static int resident32(int BN, int stages) {
+    const int ring = stages * 2 * (TC_BM * T32_BK * 4 + BN * T32_BK * 4), stage_out = TC_BM * BN * 4;
+    const int smem = (ring > stage_out ? ring : stage_out) + 1024 + 512;
+    int f = (227 * 1024) / smem;
+    f = std::min(f, 512 / BN);
+    f = std::min(f, 2048 / TC_THREADS);
+    return f < 1 ? 1 : f;
+}
+
 template <int BN>
-bool launch32_stages(int num_kb, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& md, const T32Params& p, dim3 grid,
+bool launch32_stages(int stages, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& md, const T32Params& p, dim3 grid,
                      cudaStream_t st) {
-    // Many tiles (memory-bound layers): one stage per CTA, so that several CTAs share an SM and hide each other's
-    // latencies.  Few tiles (late layers, long reductions): as deep a ring as shared memory holds instead.
     constexpr int MAXS = max_stages32(BN);
-    const long long tiles = (long long)grid.x * grid.y * grid.z;
-    int stages = tiles >= 4LL * sm_count() ? 1 : (tiles >= 2LL * sm_count() ? 2 : MAXS);
-    if (stages > num_kb) stages = num_kb < 1 ? 1 : num_kb;
     if (stages > MAXS) stages = MAXS;
-    if (stages == 1) return launch32<BN, 1>(ma, mb, ml, md, p, grid, st);
+    if (stages <= 1) return launch32<BN, 1>(ma, mb, ml, md, p, grid, st);
     if (stages == 2) return launch32<BN, 2>(ma, mb, ml, md, p, grid, st);
     if constexpr (MAXS >= 3) { if (stages == 3) return launch32<BN, 3>(ma, mb, ml, md, p, grid, st); }
     if constexpr (MAXS >= 4) { if (stages == 4) return launch32<BN, 4>(ma, mb, ml, md, p, grid, st); }
@@ -524,34 +621,45 @@ __global__ void __launch_bounds__(256) slice_sum_kernel(const float4* __restrict
     out[i] = a;
 }
 
-// Tile width and reduction slices of a product D[M,N] over K.  With fewer tiles than SMs the tiles get narrower (with
-// eight or more row tiles not below 64 columns: the MMAs of a 32-wide tile read the 128-row operand from shared memory for a quarter of the
-// output) and the reduction is cut into slices (each at least four 32-wide blocks), so that the late, small layers
-// still spread over the machine; the slices are summed in order by a second kernel.
-struct G32Plan { int BN, S, rps; };
+// Tile width, reduction slices and ring depth of a product D[M,N] over K, chosen together by a small cost model.
+// What it weighs: (i) blocks beyond what the SMs hold at once run as a second wave, so the number of blocks
+// (tiles x slices) is matched to the resident capacity, which the ring depth sets through shared memory; (ii) a
+// block's reduction is a serial chain (load, split, multiply) per 32-wide step unless the ring has two stages or
+// more; (iii) blocks sharing an SM share its shared-memory bandwidth; (iv) slices cost a second kernel that adds
+// them in order.  Times in microseconds, fitted to per-launch times measured on config 2.
+struct G32Plan { int BN, S, rps, stages; };
 G32Plan plan_gemm32(int M, int N, int K) {
-    const int sms = sm_count(), mt = (M + TC_BM - 1) / TC_BM;
-    int BN = N > 64 ? 128 : (N > 32 ? 64 : 32);
-    // 144, 192, 576 or 960 columns leave a 128-wide last tile mostly empty; 64-wide tiles fit them with less padding
-    if (BN == 128 && (N + 63) / 64 * 64 < (N + 127) / 128 * 128) BN = 64;
-    const int narrowest = mt >= 8 ? 64 : 32;     // a handful of row tiles: 32-wide tiles fill more SMs without a second pass
-    while (BN > narrowest && (long long)mt * ((N + BN - 1) / BN) < sms) BN >>= 1;
-    const long long tiles = (long long)mt * ((N + BN - 1) / BN);
-    const int nkb = (K + T32_BK - 1) / T32_BK;
-    long long S = 1;
-    if (tiles < sms && nkb >= 8) {
-        S = (2LL * sms + tiles - 1) / tiles;
-        if (S > nkb / 4) S = nkb / 4;
-        if (S > 8) S = 8;
-        const long long cap = (4LL << 20) / ((long long)M * N);
-        if (S > cap) S = cap;
-        if (S < 1) S = 1;
+    const int sms = sm_count(), mt = (M + TC_BM - 1) / TC_BM, nkb = (K + T32_BK - 1) / T32_BK;
+    // tile width: the widest that does not pad the columns more than a narrower one would (144, 192, 576 or 960 columns
+    // leave a 128-wide last tile mostly empty), narrower while the tiles are fewer than the SMs (with eight or more row
+    // tiles not below 64 columns: the MMAs of a 32-wide tile read the 128-row operand for a quarter of the output)
+    int BN0 = N > 64 ? 128 : (N > 32 ? 64 : 32);
+    if (BN0 == 128 && (N + 63) / 64 * 64 < (N + 127) / 128 * 128) BN0 = 64;
+    const int narrowest = mt >= 8 ? 64 : 32;
+    while (BN0 > narrowest && (long long)mt * ((N + BN0 - 1) / BN0) < sms) BN0 >>= 1;
+    G32Plan best{BN0, 1, nkb * T32_BK, 1};
+    double best_t = 1e30;
+    for (int BN = BN0; BN <= BN0; BN *= 2) {
+        const long long tiles = (long long)mt * ((N + BN - 1) / BN);
+        const double t0 = 3.0 + BN / 64.0, t_share = 0.3 + 0.1 * BN / 64.0;
+        const int maxst = max_stages32(BN);
+        for (int S = 1; S <= 8; ++S) {
+            const int kbps = (nkb + S - 1) / S, slices = (nkb + kbps - 1) / kbps;
+            if (slices != S || (S > 1 && kbps < 2)) continue;
+            if (S > 1 && (long long)S * M * N > (4LL << 20)) continue;      // partial sums cost traffic too
+            for (int st = 1; st <= maxst && st <= kbps; ++st) {
+                const int fit = resident32(BN, st);
+                const long long ctas = tiles * S, slots = (long long)sms * fit;
+                const long long waves = (ctas + slots - 1) / slots;
+                const double conc = (double)std::min<long long>(fit, (ctas + sms - 1) / sms);
+                const double chain = kbps * (st >= 2 ? 0.45 : 1.3), shared = conc * kbps * t_share;
+                double t = waves * (t0 + (chain > shared ? chain : shared));
+                if (S > 1) t += 2.5 + (double)(S + 1) * M * N * 4.0 / 3.0e6;
+                if (t < best_t - 1e-9) { best_t = t; best = G32Plan{BN, S, kbps * T32_BK, st}; }
+            }
+        }
     }
-    G32Plan g;
-    g.BN = BN;
-    g.rps = (int)((nkb + S - 1) / S) * T32_BK;
-    g.S = (K + g.rps - 1) / g.rps;
-    return g;
+    return best;
 }
 
 // D[M,N] = A[M,K] * B[N,K]^T (+ addend), float in and out, split-tf32 arithmetic; both operands with K contiguous.
@@ -559,22 +667,23 @@ G32Plan plan_gemm32(int M, int N, int K) {
 // to stats->partial, from the epilogue of the product kernel (one entry per 128-row tile) or from the kernel that adds
 // the reduction slices, and *stats->out describes them.
 bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err, cudaStream_t st,
-               const ColStatsReq* stats) {
+               const ColStatsReq* stats, const BnXform* a_xform) {
     G32Plan g = plan_gemm32(M, N, K);
-    if (g.S > 1 && !scratch) { g.S = 1; g.rps = (K + T32_BK - 1) / T32_BK * T32_BK; }
+    if (g.S > 1 && !scratch) { g.S = 1; g.rps = (K + T32_BK - 1) / T32_BK * T32_BK; g.stages = 4; }
     const int BN = g.BN;
     float* out = g.S > 1 ? scratch : D;
     CUtensorMap ma, mb, ml, md;
     if (!make_map_f32(&ma, A, M, K, TC_BM) || !make_map_out(&md, out, g.S, M, N) || !make_map_f32(&mb, B, N, K, BN)) return false;
     if (B_lo) { if (!make_map_f32(&ml, B_lo, N, K, BN)) return false; }
     else ml = mb;
-    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, B_lo ? 1 : 0, err, (stats && g.S == 1) ? stats->partial : nullptr};
+    T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, B_lo ? 1 : 0, err, (stats && g.S == 1) ? stats->partial : nullptr,
+                a_xform ? *a_xform : BnXform{nullptr, nullptr, 0.f, 0.f}, a_xform ? 1 : 0};
     const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM, g.S);
-    const int nkb = g.rps / T32_BK;
+    const int nkb = g.rps / T32_BK, stages = g.stages > nkb ? (nkb < 1 ? 1 : nkb) : g.stages;
     bool ok;
-    if (BN == 128) ok = launch32_stages<128>(nkb, ma, mb, ml, md, p, grid, st);
-    else if (BN == 64) ok = launch32_stages<64>(nkb, ma, mb, ml, md, p, grid, st);
-    else ok = launch32_stages<32>(nkb, ma, mb, ml, md, p, grid, st);
+    if (BN == 128) ok = launch32_stages<128>(stages, ma, mb, ml, md, p, grid, st);
+    else if (BN == 64) ok = launch32_stages<64>(stages, ma, mb, ml, md, p, grid, st);
+    else ok = launch32_stages<32>(stages, ma, mb, ml, md, p, grid, st);
     if (ok && stats) *stats->out = PartialSums{stats->partial, (int)grid.y, 1};
     if (ok && g.S > 1 && stats && !addend && slice_sum_stats(scratch, g.S, D, M, N, *stats->fold, stats->partial, stats->out, st)) return true;
     if (ok && g.S > 1) {
@@ -597,7 +706,7 @@ size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No) {
 }
 
 // dW[Mo][No] = X[R][Mo]^T * dY[R][No], second pass included; false: nothing launched
-bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st) {
+bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st, const BnXform* x_xform) {
     const Wg32Plan w = plan_wgrad32(R, Mo, No);
     const bool two_pass = w.S > 1 || w.swap;
     if (two_pass && !scratch) return false;
@@ -607,7 +716,8 @@ bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long
     CUtensorMap mx, my, md;
     float* out = two_pass ? scratch : dW;
     if (!make_map_f32(&mx, A, R, m, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) || !make_map_f32(&my, B, R, n, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) || !make_map_out(&md, out, w.S, m, n)) return false;
-    T32Params p{out, nullptr, m, n, (int)R, w.rows_per_split, 0, err};
+    T32Params p{out, nullptr, m, n, (int)R, w.rows_per_split, 0, err, nullptr,
+                x_xform ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f}, x_xform ? (w.swap ? 2 : 1) : 0};
     const dim3 grid((m + TC_BM - 1) / TC_BM, (n + w.BN - 1) / w.BN, w.S);
     bool ok;
     if (w.BN == 128) ok = launch32_wgrad<128>(mx, my, md, p, grid, st);
@@ -615,7 +725,7 @@ bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long
     else ok = launch32_wgrad<32>(mx, my, md, p, grid, st);
     if (!ok) return false;
     const long long count = (long long)Mo * No;
-    if (w.swap) launch(slice_sum_transposed_kernel, dim3((unsigned)((count + 31) / 32)), dim3(32, 8), 0, st, (const float*)scratch, w.S, Mo, No, dW);
+    if (w.swap) launch(slice_sum_transposed_kernel, dim3((Mo + 31) / 32, (No + 31) / 32), dim3(32, 8, 4), 0, st, (const float*)scratch, w.S, Mo, No, dW);
     else if (w.S > 1) split_reduce_f32(scratch, w.S, count, dW, st);
     return true;
 }

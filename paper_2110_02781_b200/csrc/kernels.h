@@ -7,6 +7,20 @@
 
 namespace ftp {
 
+// A consumer may be handed the input of a batch norm instead of its output: it then applies
+// z = min(max(y * scale + offset, lo), hi) to every element it loads (padding stays zero), so the normalised
+// tensor never exists in memory.  scale = gamma * rstd and offset = beta - mean * scale (formed in double by
+// bn_finalize) have one float per channel, 16-byte aligned; (lo, hi) = (-inf, inf), (0, inf) or (0, 6).
+struct BnXform {
+    const float* scale;
+    const float* offset;
+    float lo, hi;
+};
+inline BnXform make_xform(const float* scale, const float* offset, int act) {
+    const float inf = __builtin_huge_valf();
+    return BnXform{scale, offset, act == 0 ? -inf : 0.f, act == 2 ? 6.f : inf};
+}
+
 // Geometry of a (dense or depthwise) convolution.  Activations are (N, H, W, C).
 struct ConvGeom {
     int N, H, W, Cin;     // input
@@ -60,11 +74,14 @@ bool tc32_supported(int M, int N, int K, const void* A, const void* B, const voi
 size_t tc32_gemm_scratch_floats(int M, int N, int K);
 // B is [N][K]; B_lo (nullable): B - trunc_tf32(B) laid out like B, saves computing it per tile
 struct ColStatsReq;
+// a_xform (nullable): A holds the input of a batch norm that is applied to every tile as it is loaded
 bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* addend, float* D, float* scratch, int M, int N, int K, int* err,
-               cudaStream_t st, const ColStatsReq* stats = nullptr);
+               cudaStream_t st, const ColStatsReq* stats = nullptr, const BnXform* a_xform = nullptr);
 size_t tc32_wgrad_scratch_floats(long long R, int Mo, int No);
 // dW[Mo][No] = X[R][Mo]^T dY[R][No], the fixed-order second pass over the reduction slices included
-bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
+// x_xform (nullable): X holds the input of a batch norm that is applied as X is loaded
+bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st,
+                const BnXform* x_xform = nullptr);
 
 // ---- first convolution of an image network (stem.cu): 3 x 3, pad 1, stride 1 or 2, 3 input channels, 32 or 64
 // output channels, no bias or activation.  w is [3][3][3][cout] in T (float masters, or the bf16 shadow).
@@ -125,7 +142,7 @@ PartialSums bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double*
 // rstd; running statistics update (momentum, unbiased variance).  z = ((y - mean) - mean_lo) * scale + shift.
 void bn_finalize(const PartialSums& ps, long long M, int C, const float* gamma,
                  const float* beta, float eps, float momentum, float* run_mean, float* run_var, float* scale,
-                 float* shift, float* mean, float* mean_lo, float* rstd, const FinScratch& fin, cudaStream_t st);
+                 float* shift, float* mean, float* mean_lo, float* rstd, float* offset, const FinScratch& fin, cudaStream_t st);
 template <typename T>
 void bn_apply(const T* y, const T* residual, T* z, long long M, int C, const FoldPlan& fp, const float* scale, const float* shift,
               const float* mean, const float* mean_lo, int act, cudaStream_t st);
@@ -154,12 +171,19 @@ template <typename T>
 void act_bwd(const T* dout, const T* x, const T* addend, T* dx, long long n, int act, cudaStream_t st);
 
 template <typename T>
-void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st, const ColStatsReq* stats = nullptr);
+void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_t st, const ColStatsReq* stats = nullptr, const BnXform* x_xform = nullptr);
 template <typename T>
 void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const ConvGeom& g, cudaStream_t st);
 size_t dwconv_wgrad_scratch_floats(const ConvGeom& g);
 template <typename T>
-void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st);
+void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st,
+                  const BnXform* x_xform = nullptr);
+
+// Data gradient (+ addend) and weight gradient of a stride-1 depthwise convolution in one pass over dy (dx may be NULL).
+// scratch: dwconv_wgrad_scratch_floats(g) floats.  false: shape not taken, nothing launched.
+template <typename T>
+bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
+                      cudaStream_t st, const BnXform* x_xform = nullptr);
 
 template <typename T>
 void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);

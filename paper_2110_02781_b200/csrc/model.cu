@@ -56,6 +56,7 @@ struct Scope {
 };
 
 bool is_contraction(int kind) { return kind == FTP_CONV1D || kind == FTP_CONV2D || kind == FTP_FC; }
+bool is_pointwise_op(const Op& o);
 
 // ---- shapes, parameter offsets, validation ------------------------------------------------------
 ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cfg, ftp_model& m) {
@@ -166,6 +167,24 @@ ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cf
     // fuse "BN (no activation) -> residual add"
     for (int i = 0; i + 1 < n; ++i)
         if (m.ops[i + 1].d.kind == FTP_ADD_RESIDUAL) { m.ops[i].fused_add = true; m.ops[i + 1].skip = true; }
+    // A batch norm inside a unit whose only reader can normalise while it loads (a depthwise convolution, or a 1x1
+    // convolution on the split-tf32 tensor-core kernel) is never applied in memory: only its statistics and
+    // per-channel constants are computed, and forward and weight gradient of the reader work from the BN's input.
+    const char* fe = std::getenv("FTP_FUSE_BN");                      // bit 0: into depthwise readers, bit 1: into 1x1 readers; 0: every batch norm stores its output
+    const int fuse = fe ? std::atoi(fe) : 2;
+    const char* fm = std::getenv("FTP_FUSE_MAX_MB");                  // only batch norms whose output is at most this large (A/B measurements)
+    const double fuse_max_bytes = fm ? std::atof(fm) * 1e6 : 1e30;
+    for (int i = 0; fuse && i + 1 < n; ++i) {
+        Op& o = m.ops[i];
+        const Op& c = m.ops[i + 1];
+        if (o.d.kind != FTP_BN || o.fused_add || c.d.unit != o.d.unit) continue;
+        bool other_reader = false;
+        for (int j = i + 2; j < n; ++j) other_reader |= m.ops[j].d.kind == FTP_ADD_RESIDUAL && m.ops[j].d.residual_src == i;
+        if (other_reader || (double)o.out_elems * m.esize > fuse_max_bytes) continue;
+        void* const al = reinterpret_cast<void*>(256);
+        if (c.d.kind == FTP_DWCONV3x3) o.defer = (fuse & 1) != 0;
+        else if ((fuse & 2) && cfg->precision == FTP_FP32 && is_pointwise_op(c) && tc32_supported(c.N * c.Ho * c.Wo, c.Co, c.C, al, al, al, nullptr)) o.defer = true;
+    }
     return FTP_OK;
 }
 
@@ -202,8 +221,6 @@ ftp_status plan_gradients(ftp_model& m, int* n_slots) {
     *n_slots = (int)refc.size();
     return FTP_OK;
 }
-
-bool is_pointwise_op(const Op& o);
 
 // ---- memory layout inside the workspace --------------------------------------------------------------
 ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinned_total) {
@@ -243,14 +260,14 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     for (int i = 0; i < n; ++i) {
         Op& o = m.ops[i];
         const size_t obytes = (size_t)o.out_elems * (o.out_f32 ? 4 : es);
-        o.out = (o.fused_add) ? nullptr : bp.take(obytes);            // a fused BN writes into the add's buffer
+        o.out = (o.fused_add || o.defer) ? nullptr : bp.take(obytes);  // a fused BN writes into the add's buffer, a deferred one nowhere
         if (!o.out_f32 && i + 1 < n) max_act = std::max(max_act, obytes);
         const long long Mout = (long long)o.N * o.Ho * o.Wo;
         if (o.d.kind == FTP_BN) {
             const size_t stride = align_up((size_t)o.C * 4, 256) / 4;
-            float* t = (float*)bp.take((5 * stride + 5 * (size_t)o.C) * 4);
-            o.scale = t; o.shift = t + stride; o.mean = t + 2 * stride; o.mean_lo = t + 3 * stride; o.rstd = t + 4 * stride;
-            o.coef = t + 5 * stride;
+            float* t = (float*)bp.take((6 * stride + 5 * (size_t)o.C) * 4);
+            o.scale = t; o.shift = t + stride; o.mean = t + 2 * stride; o.mean_lo = t + 3 * stride; o.rstd = t + 4 * stride; o.offset = t + 5 * stride;
+            o.coef = t + 6 * stride;
             o.fold = make_fold(Mout, o.C, m.esize);
             foldd = std::max(foldd, std::max(fold_partial_doubles(o.fold), producer_partial_doubles(Mout, o.C)));
             finp = std::max(finp, fin_part_doubles(o.C, 1)); finc = std::max(finc, fin_counter_count(o.C, 1));
@@ -364,6 +381,10 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
         ColStatsReq req{m->fold_scratch, nullptr, &next_ps};
         const ColStatsReq* stats_req = nullptr;
         if (m->producer_stats && i + 1 <= last && m->ops[i + 1].d.kind == FTP_BN && o.d.kind != FTP_BN) { req.fold = &m->ops[i + 1].fold; stats_req = &req; }
+        // the input is what a deferred batch norm read: this op normalises as it loads
+        BnXform xfv{nullptr, nullptr, 0.f, 0.f};
+        const BnXform* xf = nullptr;
+        if (i > first && m->ops[i - 1].defer) { const Op& bn = m->ops[i - 1]; xfv = make_xform(bn.scale, bn.offset, bn.d.act); xf = &xfv; }
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
@@ -371,7 +392,8 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                     Scope sc(m, st, K_CONV_FWD_F32, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl);
                     const bool tc = is_pointwise_op(o) && o.d.kind != FTP_FC && tc32_supported((int)Mout, o.Co, o.C, in, ar.wt + o.w_off, out, nullptr) &&
                                     tc32_gemm((const float*)in, ar.wt + o.w_off, ar.wtl + o.w_off, nullptr, (float*)out, m->red_scratch, (int)Mout, o.Co, o.C,
-                                              m->tc_err, st, stats_req);
+                                              m->tc_err, st, stats_req, xf);
+                    FTP_REQUIRE(tc || !xf, FTP_ECUDA, "forward: op %d: the tensor-core product that applies the preceding batch norm could not be launched", i);
                     if (!tc) next_ps.entries = 0;
                     if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_FWD;
                     const bool stem = !tc && o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_fwd<float>((const float*)in, ar.w + o.w_off, (float*)out, o.g, st);
@@ -396,7 +418,7 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
             }
             case FTP_DWCONV3x3: {
                 Scope sc(m, st, K_DW_FWD, u, i, 0, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
-                dwconv_fwd<T>((const T*)in, ar.w + o.w_off, (T*)out, o.g, st, stats_req);
+                dwconv_fwd<T>((const T*)in, ar.w + o.w_off, (T*)out, o.g, st, stats_req, xf);
                 break;
             }
             case FTP_BN: {
@@ -410,7 +432,8 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                 if (o.fused_add) { const int s = m->ops[i + 1].d.residual_src; res = s < first ? act_in : m->cur_out[s]; }
                 { Scope sc(m, st, K_BN_FINALIZE, u, i, 0, ps.entries * 2.0 * o.C * 8.0, 0.0);
                   bn_finalize(ps, Mr, o.C, ar.w + o.w_off, ar.w + o.b_off, m->cfg.bn_eps, m->cfg.bn_momentum,
-                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, m->fin, st); }
+                              ar.run + o.rm_off, ar.run + o.rv_off, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.offset, m->fin, st); }
+                if (o.defer) { out = const_cast<void*>(in); break; }       // the next op applies it to what it loads
                 { Scope sc(m, st, K_BN_APPLY, u, i, 0, (o.in_elems * (res ? 3.0 : 2.0)) * es, 2.0 * o.in_elems);
                   bn_apply<T>((const T*)in, (const T*)res, (T*)out, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.d.act, st); }
                 break;
@@ -504,6 +527,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
         float* gr = m->grad;
         const long long Mout = (long long)o.N * o.Ho * o.Wo;
         if (gi) before_write(gi);
+        BnXform xfv{nullptr, nullptr, 0.f, 0.f};        // `in` is the input of a deferred batch norm: the weight gradient normalises as it loads
+        const BnXform* xf = nullptr;
+        if (i > first && m->ops[i - 1].defer) { const Op& bn = m->ops[i - 1]; xfv = make_xform(bn.scale, bn.offset, bn.d.act); xf = &xfv; }
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
@@ -524,7 +550,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                       const cudaStream_t ws = fork(i);
                       float* rs = ws == st ? m->red_scratch : m->red_side;
                       const bool tc = is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr) &&
-                                      tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws);
+                                      tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws, xf);
+                      FTP_REQUIRE(tc || !xf, FTP_ECUDA, "backward: op %d: the tensor-core weight gradient that applies the preceding batch norm could not be launched", i);
                       if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
                       const bool stem = !tc && !widened && o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_wgrad<float>(x, d, gr + o.w_off, rs, o.g, ws);
                       if (!tc && !stem) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
@@ -578,9 +605,13 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                 break;
             }
             case FTP_DWCONV3x3: {
+                if (gi && o.g.stride == 1) {          // one pass over dy gives the input gradient and the weight gradient
+                    Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 3.0 : 2.0) + o.out_elems) * es + 2.0 * o.w_cnt * 4.0, 36.0 * o.out_elems, 2);
+                    if (dwconv_bwd_fused<T>((const T*)in, (const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, gr + o.w_off, m->red_scratch, o.g, m->fin, st, xf)) break;
+                }
                 { Scope sc(m, st, K_DW_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems, 2);
                   const cudaStream_t ws = fork(i);
-                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, ws == st ? m->red_scratch : m->red_side, o.g, ws == st ? m->fin : m->fin_side, ws);
+                  dwconv_wgrad<T>((const T*)in, (const T*)go, gr + o.w_off, ws == st ? m->red_scratch : m->red_side, o.g, ws == st ? m->fin : m->fin_side, ws, xf);
                   forked(i, go); }
                 if (gi) {
                     Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems);
@@ -683,6 +714,37 @@ ftp_status train_step_t(ftp_model* m, const void* x, const int32_t* labels, floa
     return FTP_OK;
 }
 
+// The tensor-core kernels bound every wait; one that runs out leaves a code in the device word tc_err.  Every call
+// that launches such kernels queues a copy of that word into pinned memory behind its launches (no synchronisation),
+// and every later call looks at the copy first: a non-zero code is reported as FTP_ETIMEOUT from then on, until
+// ftp_check_device_status reads and clears the word.
+int pinned_status(const ftp_model* m) {
+    int code;
+    std::memcpy(&code, const_cast<const float*>(m->pinned) + 2, 4);
+    return code;
+}
+ftp_status pending_status(const ftp_model* m, const char* who) {
+    const int code = pinned_status(m);
+    FTP_REQUIRE(code == 0, FTP_ETIMEOUT, "%s: a bounded wait inside an earlier tensor-core kernel ran out (code %d): results since then are invalid; "
+                "ftp_check_device_status clears the condition", who, code);
+    return FTP_OK;
+}
+void queue_status(ftp_model* m, cudaStream_t st) { cudaMemcpyAsync(m->pinned + 2, m->tc_err, 4, cudaMemcpyDeviceToHost, st); }
+
+// Synchronising read of the device word; clears it when set.
+ftp_status read_device_status(ftp_model* m, cudaStream_t st, const char* who) {
+    CUDA_OK(cudaMemcpyAsync(m->pinned + 1, m->tc_err, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    int code;
+    std::memcpy(&code, m->pinned + 1, 4);
+    if (code == 0) code = pinned_status(m);
+    if (code == 0) return FTP_OK;
+    CUDA_OK(cudaMemsetAsync(m->tc_err, 0, 4, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    std::memset(m->pinned + 1, 0, 8);
+    return fail(FTP_ETIMEOUT, "%s: a bounded wait inside a tensor-core kernel ran out (code %d); the tensors written since are invalid, the condition is now cleared", who, code);
+}
+
 }  // namespace
 
 // ================================== C ABI ===========================================================
@@ -709,6 +771,7 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         s = fail(FTP_ENOMEM, "build_model: workspace too small (need %zu device and %zu pinned bytes)", need, pneed);
     if (s != FTP_OK) { delete m; return s; }
     m->pinned = (float*)pinned_ws; m->pinned_bytes = pinned_bytes;
+    std::memset(m->pinned, 0, 16);                            // loss, status words
     if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess || cudaMemset(m->fin_side.counters, 0, m->fin_counter_bytes) != cudaSuccess ||
         cudaMemset(m->tc_err, 0, 256) != cudaSuccess) {     // ticket counters start at zero
         const ftp_status e = fail(FTP_ECUDA, "build_model: clearing the ticket counters failed: %s", cudaGetErrorString(cudaGetLastError()));
@@ -846,33 +909,39 @@ extern "C" ftp_status ftp_get_tensor(const ftp_model* m, int32_t which, int32_t 
     FTP_REQUIRE(dst, FTP_EINVAL, "get_tensor: null destination");
     cudaStream_t st = (cudaStream_t)stream;
     CUDA_OK(cudaMemcpyAsync(dst, src, (size_t)count * 4, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
-    if (!dst_is_device) CUDA_OK(cudaStreamSynchronize(st));
+    if (!dst_is_device) return read_device_status(const_cast<ftp_model*>(m), st, "get_tensor");
     return FTP_OK;
 }
 
 extern "C" ftp_status ftp_run_stage_forward(ftp_model* m, int32_t a, int32_t b, const void* act_in, void* act_out, const int32_t* labels,
                                             float* loss_out, void* stream) {
     ftp_status s = check_range(m, a, b, "run_stage_forward");
+    if (s == FTP_OK) s = pending_status(m, "run_stage_forward");
     if (s != FTP_OK) return s;
     FTP_REQUIRE(act_in, FTP_EINVAL, "run_stage_forward: null act_in");
     FTP_REQUIRE(a16(act_in) && a16(act_out), FTP_ERANGE, "run_stage_forward: activation buffers must be 16-byte aligned");
     if (b == m->L) FTP_REQUIRE(labels && loss_out && !act_out, FTP_EINVAL, "run_stage_forward: the last stage needs labels and loss_out, and no act_out");
     else FTP_REQUIRE(act_out && !labels && !loss_out, FTP_EINVAL, "run_stage_forward: an inner stage needs act_out and takes no labels");
     cudaStream_t st = (cudaStream_t)stream;
-    return m->cfg.precision == FTP_FP32 ? fwd_range<float>(m, a, b, act_in, act_out, labels, loss_out, st)
-                                        : fwd_range<__nv_bfloat16>(m, a, b, act_in, act_out, labels, loss_out, st);
+    s = m->cfg.precision == FTP_FP32 ? fwd_range<float>(m, a, b, act_in, act_out, labels, loss_out, st)
+                                     : fwd_range<__nv_bfloat16>(m, a, b, act_in, act_out, labels, loss_out, st);
+    queue_status(m, st);
+    return s;
 }
 
 extern "C" ftp_status ftp_run_stage_backward(ftp_model* m, int32_t a, int32_t b, const void* grad_out, void* grad_in, void* stream) {
     ftp_status s = check_range(m, a, b, "run_stage_backward");
+    if (s == FTP_OK) s = pending_status(m, "run_stage_backward");
     if (s != FTP_OK) return s;
     if (b == m->L) FTP_REQUIRE(!grad_out, FTP_EINVAL, "run_stage_backward: the last stage takes no grad_out");
     else FTP_REQUIRE(grad_out, FTP_EINVAL, "run_stage_backward: an inner stage needs grad_out");
     FTP_REQUIRE(a == 0 || grad_in, FTP_EINVAL, "run_stage_backward: grad_in is required when a > 0");
     FTP_REQUIRE(a16(grad_out) && a16(grad_in), FTP_ERANGE, "run_stage_backward: gradient buffers must be 16-byte aligned");
     cudaStream_t st = (cudaStream_t)stream;
-    return m->cfg.precision == FTP_FP32 ? bwd_range<float>(m, a, b, grad_out, grad_in, false, st)
-                                        : bwd_range<__nv_bfloat16>(m, a, b, grad_out, grad_in, false, st);
+    s = m->cfg.precision == FTP_FP32 ? bwd_range<float>(m, a, b, grad_out, grad_in, false, st)
+                                     : bwd_range<__nv_bfloat16>(m, a, b, grad_out, grad_in, false, st);
+    queue_status(m, st);
+    return s;
 }
 
 extern "C" ftp_status ftp_get_logits(const ftp_model* m, float* dst, int32_t dst_is_device, void* stream) {
@@ -882,23 +951,32 @@ extern "C" ftp_status ftp_get_logits(const ftp_model* m, float* dst, int32_t dst
     cudaStream_t st = (cudaStream_t)stream;
     CUDA_OK(cudaMemcpyAsync(dst, m->cur_out[fc], (size_t)m->cfg.batch * m->cfg.n_classes * 4,
                             dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
-    if (!dst_is_device) CUDA_OK(cudaStreamSynchronize(st));
+    if (!dst_is_device) return read_device_status(const_cast<ftp_model*>(m), st, "get_logits");
     return FTP_OK;
 }
 
 extern "C" ftp_status ftp_sgd_step(ftp_model* m, int32_t a, int32_t b, float lr, float* snap_dev, float* snap_host, void* stream) {
     ftp_status s = check_range(m, a, b, "sgd_step");
+    if (s == FTP_OK) s = pending_status(m, "sgd_step");
     if (s != FTP_OK) return s;
-    return sgd_range(m, a, b, lr, snap_dev, snap_host, (cudaStream_t)stream);
+    s = sgd_range(m, a, b, lr, snap_dev, snap_host, (cudaStream_t)stream);
+    queue_status(m, (cudaStream_t)stream);
+    return s;
 }
 
 extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, int32_t inputs_on_host, float lr, float* loss_host,
                                      void* stream) {
     FTP_REQUIRE(m && x && labels, FTP_EINVAL, "train_step: null argument");
+    {
+        const ftp_status ps = pending_status(m, "train_step");
+        if (ps != FTP_OK) return ps;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     const void* xin = x;
     const int32_t* lab = labels;
     if (inputs_on_host) {
+        for (int i = 0; i < m->cfg.batch; ++i)
+            FTP_REQUIRE(labels[i] >= 0 && labels[i] < m->cfg.n_classes, FTP_ERANGE, "train_step: label %d of sample %d is outside [0, %d)", labels[i], i, m->cfg.n_classes);
         const size_t in_bytes = (size_t)m->cfg.batch * m->cfg.in_h * m->cfg.in_w * m->cfg.in_c * m->esize;
         CUDA_OK(cudaMemcpyAsync(m->input_dev, x, in_bytes, cudaMemcpyHostToDevice, st));
         CUDA_OK(cudaMemcpyAsync(m->labels_dev, labels, (size_t)m->cfg.batch * 4, cudaMemcpyHostToDevice, st));
@@ -908,13 +986,24 @@ extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t*
     if (s != FTP_OK) return s;
     if (loss_host) {
         CUDA_OK(cudaMemcpyAsync(m->pinned, m->loss_dev, 4, cudaMemcpyDeviceToHost, st));
-        CUDA_OK(cudaMemcpyAsync(m->pinned + 1, m->tc_err, 4, cudaMemcpyDeviceToHost, st));
-        CUDA_OK(cudaStreamSynchronize(st));
+        s = read_device_status(m, st, "train_step");
         *loss_host = m->pinned[0];
-        int code;
-        memcpy(&code, m->pinned + 1, 4);
-        FTP_REQUIRE(code == 0, FTP_ETIMEOUT, "train_step: a bounded wait inside a tensor-core kernel ran out (code %d)", code);
+        return s;
     }
+    queue_status(m, st);
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_check_device_status(ftp_model* m, void* stream) {
+    FTP_REQUIRE(m, FTP_EINVAL, "check_device_status: null model");
+    return read_device_status(m, (cudaStream_t)stream, "check_device_status");
+}
+
+extern "C" ftp_status ftp_debug_set_device_status(ftp_model* m, int32_t code, void* stream) {
+    FTP_REQUIRE(m, FTP_EINVAL, "debug_set_device_status: null model");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaMemcpyAsync(m->tc_err, &code, 4, cudaMemcpyHostToDevice, st));
+    CUDA_OK(cudaStreamSynchronize(st));
     return FTP_OK;
 }
 
@@ -933,6 +1022,10 @@ extern "C" ftp_status ftp_stage_times(ftp_model* m, double* seconds, int32_t* n_
     FTP_REQUIRE(m->timed_stages > 0, FTP_ESTATE, "stage_times: no training step has run since stage timing was switched on");
     const int n = m->timed_stages;
     CUDA_OK(cudaEventSynchronize(m->ev_sb[0]));
+    {
+        const ftp_status ps = pending_status(m, "stage_times");
+        if (ps != FTP_OK) return ps;
+    }
     for (int s = 0; s < n; ++s) {
         float f = 0.f, b = 0.f;
         CUDA_OK(cudaEventElapsedTime(&f, m->ev_sf[s], m->ev_sf[s + 1]));
@@ -948,6 +1041,10 @@ extern "C" ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void*
     FTP_REQUIRE(m && sample_in && labels && fwd_s && bwd_s && out_bytes, FTP_EINVAL, "profile_layers: null argument");
     FTP_REQUIRE(reps >= 1 && reps <= 1000, FTP_EINVAL, "profile_layers: reps must be in 1..1000");
     FTP_REQUIRE(a16(sample_in), FTP_ERANGE, "profile_layers: the sample batch must be 16-byte aligned");
+    {
+        const ftp_status ps = pending_status(m, "profile_layers");
+        if (ps != FTP_OK) return ps;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     const int L = m->L;
     while ((int)m->ev_f.size() < L + 1) { cudaEvent_t e; CUDA_OK(cudaEventCreate(&e)); m->ev_f.push_back(e); }
@@ -984,6 +1081,7 @@ extern "C" ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void*
             cudaMemcpyAsync(m->arena[m->owner[u]].run + m->unit_s_off[u], m->state_backup + m->unit_s_off[u], (size_t)m->unit_s_cnt[u] * 4,
                             cudaMemcpyDeviceToDevice, st);
     cudaStreamSynchronize(st);
+    if (s == FTP_OK) s = read_device_status(m, st, "profile_layers");
     if (s != FTP_OK) return s;
     for (int u = 0; u < L; ++u) {
         fwd_s[u] = f[u] / reps; bwd_s[u] = bk[u] / reps;
@@ -1190,6 +1288,47 @@ extern "C" ftp_status ftp_trace_read(ftp_model* m, ftp_trace_rec* out, int32_t m
     m->tr_used = 0;
     return FTP_OK;
 }
+
+#ifdef FTP_TIMELINE
+namespace ftp {
+static std::vector<void (*)(std::vector<unsigned long long>&, bool)>& tl_readers() {
+    static std::vector<void (*)(std::vector<unsigned long long>&, bool)> v;
+    return v;
+}
+void tl_register(void (*reader)(std::vector<unsigned long long>&, bool)) { tl_readers().push_back(reader); }
+static std::vector<const void*> g_tl_launched;
+void tl_note_launch(const void* kernel) { if (g_tl_launched.size() < (1u << 20)) g_tl_launched.push_back(kernel); }
+}  // namespace ftp
+// Measurement build only: the (mangled) names of the kernels launched since the last reset, one per line, in launch order.
+extern "C" int32_t ftp_debug_launch_names(char* buf, int32_t cap, int32_t reset) {
+    size_t used = 0;
+    int32_t n = 0;
+    for (const void* k : ftp::g_tl_launched) {
+        const char* name = nullptr;
+        if (cudaFuncGetName(&name, k) != cudaSuccess || !name) name = "?";
+        const size_t len = std::strlen(name);
+        if (used + len + 2 > (size_t)std::max(cap, 0)) break;
+        std::memcpy(buf + used, name, len);
+        used += len;
+        buf[used++] = '\n';
+        ++n;
+    }
+    if (cap > 0) buf[used < (size_t)cap ? used : (size_t)cap - 1] = 0;
+    if (reset) ftp::g_tl_launched.clear();
+    return n;
+}
+// Measurement build only: the start times (ns of the global timer) of all grids launched since the last reset, merged
+// over the translation units and sorted; synchronises the device.
+extern "C" int32_t ftp_debug_timeline(unsigned long long* out, int32_t max, int32_t reset) {
+    cudaDeviceSynchronize();
+    std::vector<unsigned long long> all;
+    for (auto r : ftp::tl_readers()) r(all, reset != 0);
+    std::sort(all.begin(), all.end());
+    const int32_t n = (int32_t)std::min<size_t>(all.size(), (size_t)std::max(max, 0));
+    for (int32_t i = 0; i < n; ++i) out[i] = all[i];
+    return (int32_t)all.size();
+}
+#endif
 
 extern "C" const char* ftp_kernel_name(int32_t kernel) { return kernel >= 0 && kernel < K_COUNT ? kKernelNames[kernel] : "?"; }
 

@@ -26,10 +26,11 @@ struct Op {
     long long rm_off, rv_off;  // BN running mean / variance in the state arena
     void* out;               // internal output buffer
     bool out_f32;            // output kept in float whatever the precision (logits, loss)
-    float *scale, *shift, *mean, *mean_lo, *rstd, *coef;   // BN per-channel tables
+    float *scale, *shift, *mean, *mean_lo, *rstd, *offset, *coef;   // BN per-channel tables
     FoldPlan fold;
     bool fused_add;          // BN whose normalised output goes straight through the following residual add
     bool skip;               // residual add folded into the preceding BN
+    bool defer;              // BN whose normalised output is never stored: the next op of the unit applies it to what it loads
     int gslot;               // slot holding the gradient w.r.t. this op's output (-1 none, -2 dlogits)
     int galias;              // op whose output-gradient buffer this op's output gradient shares
     int addend_of;           // when writing the gradient of this op's input, add the gradient buffer of that op's output

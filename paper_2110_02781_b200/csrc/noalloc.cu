@@ -7,6 +7,7 @@
 // gives it input and output buffers and nothing else, a process whose memory pool is owned by
 // another component).  For them the scratch lives in a fixed-size array in the library's own
 // device image; every GPU that loads the library carries it until the process exits.
+#include <atomic>
 #include <cstdint>
 #include "common.h"
 #include "kernels.h"
@@ -17,7 +18,7 @@ constexpr size_t kScratchFloats = size_t(1) << 21;          // 8 MiB: the stated
 static __device__ __align__(256) float g_wgrad_scratch[kScratchFloats];
 
 constexpr int kMaxDevices = 64;
-float* g_scratch_addr[kMaxDevices] = {};                    // device address of the array, per device
+std::atomic<float*> g_scratch_addr[kMaxDevices] = {};       // device address of the array, per device (every thread that looks it up gets the same value)
 
 // In host code the array's name is only a handle; the address a kernel may use has to be asked
 // for, once per device, with that device current.
@@ -26,13 +27,15 @@ ftp_status scratch_for_current_device(float** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return ftp::fail(FTP_ECUDA, "conv_wgrad_static: cudaGetDevice: %s", cudaGetErrorString(e));
     if (dev < 0 || dev >= kMaxDevices) return ftp::fail(FTP_ERANGE, "conv_wgrad_static: device index %d not supported", dev);
-    if (!g_scratch_addr[dev]) {
+    float* addr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!addr) {
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_wgrad_scratch);
         if (e != cudaSuccess || !p) return ftp::fail(FTP_ECUDA, "conv_wgrad_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
-        g_scratch_addr[dev] = static_cast<float*>(p);
+        addr = static_cast<float*>(p);
+        g_scratch_addr[dev].store(addr, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = addr;
     return FTP_OK;
 }
 
@@ -44,6 +47,9 @@ extern "C" ftp_status ftp_conv_wgrad_static(const float* x, const float* dy, flo
     FTP_REQUIRE(n >= 1 && h >= 1 && w >= 1 && cin >= 1 && cout >= 1 && k >= 1 && stride >= 1 && pad >= 0, FTP_EINVAL,
                 "conv_wgrad_static: sizes must be positive");
     FTP_REQUIRE(h + 2 * pad >= k && w + 2 * pad >= k, FTP_EINVAL, "conv_wgrad_static: kernel larger than the padded input");
+    // the kernels index the filter with int: k*k*cin (the reduction length) and k*k*cin*cout (the size of dw) must fit
+    FTP_REQUIRE((long long)k * k * cin < (1LL << 31) && (long long)k * k * cin * cout < (1LL << 31), FTP_ERANGE,
+                "conv_wgrad_static: filter too large (k*k*cin*cout must stay below 2^31)");
     ftp::ConvGeom g{n, h, w, cin, (h + 2 * pad - k) / stride + 1, (w + 2 * pad - k) / stride + 1, cout, k, k, stride, pad, pad};
     FTP_REQUIRE((long long)n * h * w * cin < (1LL << 31) && (long long)n * g.Ho * g.Wo * cout < (1LL << 31), FTP_ERANGE,
                 "conv_wgrad_static: tensor too large");

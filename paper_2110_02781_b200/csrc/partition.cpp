@@ -146,3 +146,82 @@ extern "C" ftp_status ftp_recovery_plan(const int32_t* p_cur, int32_t n_cur, con
     return FTP_OK;
 }
 
+
+// ---- training state of a node and the central node's fault handler (Sec. III-B Table I, Sec. III-F) -------------
+extern "C" ftp_status ftp_state_init(ftp_train_state* st, float learning_rate, int64_t epoch_number, int64_t batch_number) {
+    FTP_REQUIRE(st, FTP_EINVAL, "state_init: null state");
+    FTP_REQUIRE(epoch_number >= 0 && batch_number >= 0, FTP_EINVAL, "state_init: epoch and batch numbers must not be negative");
+    st->committed_forward_id = -1;
+    st->committed_backward_id = -1;
+    st->status = 0;
+    st->learning_rate = learning_rate;
+    st->epoch_number = epoch_number;
+    st->batch_number = batch_number;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_state_forward_done(ftp_train_state* st, int64_t batch_id) {
+    FTP_REQUIRE(st && batch_id >= 0, FTP_EINVAL, "state_forward_done: null state or negative batch id");
+    st->committed_forward_id = batch_id;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_state_backward_done(ftp_train_state* st, int64_t batch_id) {
+    FTP_REQUIRE(st && batch_id >= 0, FTP_EINVAL, "state_backward_done: null state or negative batch id");
+    st->committed_backward_id = batch_id;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_state_timer_expired(ftp_train_state* st, int64_t batch_id, int32_t* triggered) {
+    FTP_REQUIRE(st && triggered && batch_id >= 0, FTP_EINVAL, "state_timer_expired: null argument or negative batch id");
+    *triggered = st->status == 0 ? 1 : 0;          // later timers find the handler already running
+    st->status = 1;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_state_may_forward(const ftp_train_state* st, int64_t batch_id, int32_t* allowed) {
+    FTP_REQUIRE(st && allowed, FTP_EINVAL, "state_may_forward: null argument");
+    *allowed = (st->status == 0 || batch_id <= st->committed_forward_id) ? 1 : 0;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_state_reset(ftp_train_state* st, int64_t batch_id, int64_t* resume_from) {
+    FTP_REQUIRE(st && batch_id >= 0, FTP_EINVAL, "state_reset: null state or negative batch id");
+    st->committed_forward_id = batch_id;
+    st->committed_backward_id = batch_id;
+    st->status = 0;
+    if (resume_from) *resume_from = batch_id;
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_classify_probe(const int32_t* responses, int32_t n_workers, int32_t* action, int32_t* failed, int32_t* n_failed,
+                                         int32_t* restarted_worker) {
+    FTP_REQUIRE(responses && action && failed && n_failed && restarted_worker, FTP_EINVAL, "classify_probe: null argument");
+    FTP_REQUIRE(n_workers >= 1 && responses[0] == FTP_PROBE_NORMAL, FTP_EINVAL, "classify_probe: worker 0 is the central node and answers normally");
+    int32_t silent = 0, restarted = 0, last_restarted = -1;
+    for (int32_t i = 0; i < n_workers; ++i) {
+        FTP_REQUIRE(responses[i] >= FTP_PROBE_NORMAL && responses[i] <= FTP_PROBE_SILENT, FTP_EINVAL, "classify_probe: unknown response %d of worker %d", responses[i], i);
+        if (responses[i] == FTP_PROBE_SILENT) ++silent;
+        if (responses[i] == FTP_PROBE_RESTARTED) { ++restarted; last_restarted = i; }
+    }
+    *n_failed = 0;
+    *restarted_worker = -1;
+    if (silent == 0 && restarted == 0) { *action = FTP_ACTION_RESTART_BATCH; return FTP_OK; }
+    if (silent == 0 && restarted == 1) { *action = FTP_ACTION_RESEND_STATE; *restarted_worker = last_restarted; return FTP_OK; }
+    *action = FTP_ACTION_REDISTRIBUTE;
+    for (int32_t i = 0; i < n_workers; ++i)
+        if (responses[i] != FTP_PROBE_NORMAL) failed[(*n_failed)++] = i;
+    return FTP_OK;
+}
+
+// Sec. III-D: the dynamic partition runs after the first 10 batches and then every 100 batches.
+extern "C" int32_t ftp_is_repartition_iter(int64_t it, int64_t first, int64_t period) {
+    const int64_t done = it + 1;
+    if (first <= 0 || period <= 0 || done <= 0) return 0;
+    return (done == first || (done > first && done % period == 0)) ? 1 : 0;
+}
+
+// Sec. IV-B / IV-E: a replication runs when a batch whose 1-indexed count is a multiple of the period has finished.
+extern "C" int32_t ftp_is_replication_iter(int64_t it, int64_t period) {
+    return (period > 0 && it + 1 > 0 && (it + 1) % period == 0) ? 1 : 0;
+}

@@ -10,7 +10,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libftpipe.so")
+LIB_PATH = os.environ.get("FTPIPE_LIB") or os.path.join(_HERE, "libftpipe.so")       # FTPIPE_LIB: another build of the library (measurement variants)
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2110_02781_b200.build`")
 lib = C.CDLL(LIB_PATH)
@@ -35,6 +35,15 @@ class ModelCfg(C.Structure):
 class TraceRec(C.Structure):
     _fields_ = [("kernel", C.c_int32), ("unit", C.c_int32), ("op", C.c_int32), ("backward", C.c_int32),
                 ("ms", C.c_float), ("bytes", C.c_double), ("flops", C.c_double)]
+
+
+class TrainState(C.Structure):
+    _fields_ = [("committed_forward_id", C.c_int64), ("committed_backward_id", C.c_int64), ("status", C.c_int32),
+                ("learning_rate", C.c_float), ("epoch_number", C.c_int64), ("batch_number", C.c_int64)]
+
+
+PROBE_NORMAL, PROBE_RESTARTED, PROBE_SILENT = 0, 1, 2
+ACTION_RESTART_BATCH, ACTION_RESEND_STATE, ACTION_REDISTRIBUTE = 0, 1, 2
 
 
 class FtpError(RuntimeError):
@@ -71,6 +80,15 @@ _SIGS = {
     "ftp_set_partition": [_vp, _P(_i32), _i32, _P(_i32), _vp],
     "ftp_get_partition": [_vp, _P(_i32), _P(_i32)],
     "ftp_snapshot_weights": [_vp, _i32, _vp, _sz, _i32, _P(_sz), _vp],
+    "ftp_state_init": [_P(TrainState), _f32, _i64, _i64],
+    "ftp_state_forward_done": [_P(TrainState), _i64],
+    "ftp_state_backward_done": [_P(TrainState), _i64],
+    "ftp_state_timer_expired": [_P(TrainState), _i64, _P(_i32)],
+    "ftp_state_may_forward": [_P(TrainState), _i64, _P(_i32)],
+    "ftp_state_reset": [_P(TrainState), _i64, _P(_i64)],
+    "ftp_classify_probe": [_P(_i32), _i32, _P(_i32), _P(_i32), _P(_i32), _P(_i32)],
+    "ftp_check_device_status": [_vp, _vp],
+    "ftp_debug_set_device_status": [_vp, _i32, _vp],
     "ftp_trace_enable": [_vp, _i32],
     "ftp_trace_read": [_vp, _P(TraceRec), _i32, _P(_i32)],
     "ftp_launch_count": [_vp, _P(_i64)],
@@ -82,6 +100,8 @@ for _name, _args in _SIGS.items():
 lib.ftp_destroy_model.argtypes, lib.ftp_destroy_model.restype = [_vp], None
 lib.ftp_last_error.argtypes, lib.ftp_last_error.restype = [], C.c_char_p
 lib.ftp_kernel_name.argtypes, lib.ftp_kernel_name.restype = [_i32], C.c_char_p
+lib.ftp_is_repartition_iter.argtypes, lib.ftp_is_repartition_iter.restype = [_i64, _i64, _i64], _i32
+lib.ftp_is_replication_iter.argtypes, lib.ftp_is_replication_iter.restype = [_i64, _i64], _i32
 
 
 def _check(status):
@@ -184,6 +204,55 @@ def ftp_recovery_plan(p_cur, failed, p_new):
     return kind[:L].tolist(), index[:L].tolist()
 
 
+def ftp_state_init(learning_rate, epoch_number, batch_number):
+    st = TrainState()
+    _check(lib.ftp_state_init(C.byref(st), learning_rate, epoch_number, batch_number))
+    return st
+
+
+def ftp_state_forward_done(st, batch_id):
+    _check(lib.ftp_state_forward_done(C.byref(st), batch_id))
+
+
+def ftp_state_backward_done(st, batch_id):
+    _check(lib.ftp_state_backward_done(C.byref(st), batch_id))
+
+
+def ftp_state_timer_expired(st, batch_id):
+    t = _i32()
+    _check(lib.ftp_state_timer_expired(C.byref(st), batch_id, C.byref(t)))
+    return bool(t.value)
+
+
+def ftp_state_may_forward(st, batch_id):
+    a = _i32()
+    _check(lib.ftp_state_may_forward(C.byref(st), batch_id, C.byref(a)))
+    return bool(a.value)
+
+
+def ftp_state_reset(st, batch_id):
+    r = _i64()
+    _check(lib.ftp_state_reset(C.byref(st), batch_id, C.byref(r)))
+    return r.value
+
+
+def ftp_classify_probe(responses):
+    n = len(responses)
+    r = (_i32 * n)(*responses)
+    failed = (_i32 * n)()
+    action, nf, rw = _i32(), _i32(), _i32()
+    _check(lib.ftp_classify_probe(r, n, C.byref(action), failed, C.byref(nf), C.byref(rw)))
+    return action.value, list(failed[:nf.value]), (rw.value if rw.value >= 0 else None)
+
+
+def ftp_is_repartition_iter(it, first=10, period=100):
+    return bool(lib.ftp_is_repartition_iter(it, first, period))
+
+
+def ftp_is_replication_iter(it, period):
+    return bool(lib.ftp_is_replication_iter(it, period))
+
+
 def ftp_workspace_bytes(layers, cfg):
     d, p = _sz(), _sz()
     _check(lib.ftp_workspace_bytes(layer_array(layers), len(layers), C.byref(model_cfg(cfg)), C.byref(d), C.byref(p)))
@@ -194,7 +263,26 @@ def ftp_conv_wgrad_static(x, dy, dw, k, stride, pad, stream=None):
     """Weight gradient of a dense k x k convolution without any workspace argument, for callers that
     may not allocate device memory: x (n, h, w, cin), dy (n, ho, wo, cout) and dw (k, k, cin, cout)
     are float32 CUDA tensors the caller already owns.  See include/ftpipe.h for the limits."""
+    import torch
+    def bad(why):
+        raise FtpError(1, "conv_wgrad_static: " + why)
+    for name, t in (("x", x), ("dy", dy), ("dw", dw)):
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            bad(f"{name} must be a contiguous float32 CUDA tensor")
+        if t.device != x.device:
+            bad("x, dy and dw must live on one device")
+    if x.device.index != torch.cuda.current_device():
+        bad("the tensors' device must be the current device")
+    if x.dim() != 4 or dy.dim() != 4 or k < 1 or stride < 1 or pad < 0:
+        bad("x and dy must be 4-D (n, h, w, c); k, stride >= 1, pad >= 0")
     n, h, w, cin = x.shape
+    if h + 2 * pad < k or w + 2 * pad < k:
+        bad("kernel larger than the padded input")
+    ho, wo = (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1
+    if tuple(dy.shape[:3]) != (n, ho, wo):
+        bad(f"dy must be ({n}, {ho}, {wo}, cout), got {tuple(dy.shape)}")
+    if tuple(dw.shape) != (k, k, cin, dy.shape[3]):
+        bad(f"dw must be ({k}, {k}, {cin}, {dy.shape[3]}), got {tuple(dw.shape)}")
     _check(lib.ftp_conv_wgrad_static(_ptr(x), _ptr(dy), _ptr(dw), n, h, w, cin, dy.shape[3], k, stride, pad,
                                      _stream(stream)))
 
@@ -336,6 +424,12 @@ class Model:
         _check(lib.ftp_snapshot_weights(self.h, stage, _ptr(dst), dst.numel() * dst.element_size(),
                                         int(not dst.is_cuda), C.byref(w), _stream(stream)))
         return w.value
+
+    def ftp_check_device_status(self, stream=None):
+        _check(lib.ftp_check_device_status(self.h, _stream(stream)))
+
+    def ftp_debug_set_device_status(self, code, stream=None):
+        _check(lib.ftp_debug_set_device_status(self.h, int(code), _stream(stream)))
 
     def ftp_trace_enable(self, on):
         _check(lib.ftp_trace_enable(self.h, int(on)))

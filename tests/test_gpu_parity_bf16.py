@@ -236,3 +236,59 @@ def test_each_layer_kind_bf16(case):
         assert e <= TOL_BF16, f"{name}: {e:.3e}"
     assert rel_err(gm.ftp_get_tensor(F.T_STATE, 0), om.unit_state(0)) <= TOL_BF16
     gm.close()
+
+
+# ---- the bf16 path against the plain float64 definition (no rounding anywhere in the oracle) ------------------
+F64_NETS = {"tiny_mbv2": (lambda: synth.tiny_mbv2(precision=1), 66, "perturbed"),
+            "tiny_mbv2_b16_hw16": (lambda: synth.tiny_mbv2(batch=16, hw=16, precision=1), 67, "init"),
+            "tiny_vgg": (lambda: synth.tiny_vgg(batch=6, hw=4, precision=1), 68, "perturbed"),
+            "vgg_real_widths": (lambda: synth.vgg16(32, 8, 10, 1, plan=[64, 64, "M", 128, 128, "M", 128, "M"]), 69, "init")}
+
+
+@pytest.mark.parametrize("name", list(F64_NETS))
+def test_bf16_path_against_the_float64_oracle(name, record_property):
+    """One step of the bf16 device path from float32 master weights against the oracle with storage switched off:
+    every tensor float64, nothing rounded anywhere.  The stated bar (2e-2, max-abs relative) is asserted on what is
+    continuous in the stored values: the loss, the logits, the BN running statistics, the updated master weights.
+    Weight gradients are measured in the same norm and printed, not asserted at 2e-2: storing activations and
+    gradients with an 8-bit mantissa moves some pre-activations across a ReLU kink, and on these nets that alone puts
+    15-20 % between ANY bf16-storage run and the float64 one (the oracle's own bf16 mode, run beside it here, shows
+    the same figures).  What is asserted for them: the device is no further from float64 than bf16 storage itself is
+    (the oracle's bf16 mode against its float64 mode, plus the 2e-2 bar)."""
+    import torch
+    from oracle.model import round_bf16
+    net, idx, params = F64_NETS[name]
+    ls, cfg = net()
+    par = perturb(ls, idx) if params == "perturbed" else synth.init_params(idx, ls)
+    om = oracle.OracleModel(ls, cfg, par, synth.init_state(ls), storage="none")
+    oq = oracle.OracleModel(ls, cfg, par, synth.init_state(ls))
+    assert not om.quantised and oq.quantised
+    x, y = synth.make_batch(idx, cfg)
+    x = round_bf16(x)                                  # all three read the same (bf16-representable) batch
+    ref_loss = om.step([0, om.L], x, y, lr=0.01)
+    oq.step([0, oq.L], x, y, lr=0.01)
+    gm = F.Model(ls, cfg)
+    gm.load_params(par, synth.init_state(ls))
+    xd, yd = dev_bf16(x), torch.from_numpy(y).cuda()
+    loss = torch.zeros(1, device="cuda")
+    gm.ftp_run_stage_forward(0, gm.L, xd, None, yd, loss)
+    gm.ftp_run_stage_backward(0, gm.L)
+    torch.cuda.synchronize()
+    e_loss = abs(loss.item() - ref_loss) / max(abs(ref_loss), 1e-30)
+    e_logits = rel_err(gm.ftp_get_logits(), om.logits)
+    units = [u for u in range(gm.L) if om.unit_grads(u).size]
+    got = {u: gm.ftp_get_tensor(F.T_GRADS, u) for u in units}
+    e_dev = {u: (rel_err(got[u], om.unit_grads(u)), l2_err(got[u], om.unit_grads(u))) for u in units}
+    e_fmt = {u: (rel_err(oq.unit_grads(u), om.unit_grads(u)), l2_err(oq.unit_grads(u), om.unit_grads(u))) for u in units}
+    e_state = max(rel_err(gm.ftp_get_tensor(F.T_STATE, u), om.unit_state(u)) for u in range(gm.L))
+    gm.ftp_sgd_step(0, gm.L, 0.01)
+    e_w = max(rel_err(gm.ftp_get_tensor(F.T_WEIGHTS, u), om.unit_params(u)) for u in range(gm.L))
+    report = dict(loss=float(e_loss), logits=e_logits, state=e_state, weights=e_w,
+                  grad_maxabs_device={u: round(v[0], 4) for u, v in e_dev.items()}, grad_maxabs_bf16_storage={u: round(v[0], 4) for u, v in e_fmt.items()},
+                  grad_l2_device={u: round(v[1], 4) for u, v in e_dev.items()}, grad_l2_bf16_storage={u: round(v[1], 4) for u, v in e_fmt.items()})
+    print(f"\nbf16 device path vs float64 oracle, {name}: {report}")
+    record_property("bf16_vs_float64", str(report))
+    assert e_loss <= TOL_BF16 and e_logits <= TOL_BF16 and e_state <= TOL_BF16 and e_w <= TOL_BF16, report
+    for u in units:
+        assert e_dev[u][0] <= e_fmt[u][0] + TOL_BF16 and e_dev[u][1] <= e_fmt[u][1] + TOL_BF16, (u, report)
+    gm.close()

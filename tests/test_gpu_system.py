@@ -296,3 +296,43 @@ def test_stage_times_feed_the_capacity_estimate():
         gm.ftp_stage_times()
     gm.close()
 
+
+
+def test_device_status_word_is_reported_and_cleared():
+    """The status word that a tensor-core kernel sets when a bounded wait runs out, set here from the host
+    (no kernel is altered, no wait is made to expire, and no tensor-core kernel runs while it is set): the
+    synchronising routes return FTP_ETIMEOUT and clear it; an asynchronous call carries it to the host and
+    every later call refuses before launching; after the check training matches the oracle again."""
+    import torch
+    ls, cfg = synth.tiny_mbv2()
+    gm, om = make_gpu(ls, cfg, 36), make_oracle(ls, cfg, 36)
+    x, y = synth.make_batch(36, cfg)
+    xd, yd = to_dev(x), to_dev(y)
+    gm.ftp_check_device_status()                                            # clean model: no error
+    # synchronising routes read the word itself
+    for call in (lambda: gm.ftp_check_device_status(), lambda: gm.ftp_get_tensor(F.T_WEIGHTS, 0)):
+        gm.ftp_debug_set_device_status(12)
+        with pytest.raises(F.FtpError) as e:
+            call()
+        assert e.value.status == 6 and "12" in str(e.value)
+        gm.ftp_check_device_status()                                        # the failed call cleared it
+    # asynchronous route: the optimiser step (streaming kernels only) queues a copy of the word behind its launches
+    gm.ftp_debug_set_device_status(13)
+    loss = torch.zeros(1, device="cuda")
+    gm.ftp_sgd_step(0, 1, 0.0)
+    torch.cuda.synchronize()
+    before = gm.ftp_launch_count()
+    for call in (lambda: gm.ftp_run_stage_forward(0, gm.L, xd, None, yd, loss), lambda: gm.ftp_run_stage_backward(0, gm.L),
+                 lambda: gm.ftp_sgd_step(0, gm.L, 0.0), lambda: gm.ftp_train_step(xd, yd, 0.0, want_loss=False),
+                 lambda: gm.ftp_train_step(xd, yd, 0.0), lambda: gm.ftp_profile_layers(1, xd, yd)):
+        with pytest.raises(F.FtpError) as e:
+            call()
+        assert e.value.status == 6 and "13" in str(e.value)
+    assert gm.ftp_launch_count() == before                                   # refused before any launch
+    with pytest.raises(F.FtpError):
+        gm.ftp_check_device_status()                                        # reports once more and clears
+    gm.ftp_check_device_status()
+    got = gm.ftp_train_step(xd, yd, cfg["lr"])
+    ref = om.step([0, om.L], x, y)
+    assert abs(got - ref) <= TOL_FP32 * abs(ref)
+    gm.close()

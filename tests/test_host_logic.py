@@ -128,3 +128,43 @@ def test_recovery_plan_equals_oracle():
     with pytest.raises(F.FtpError):
         F.ftp_recovery_plan([0, 2, 4, 6, 8, 11], [1], [0, 3, 6, 11])          # one failure leaves four stages, not three
 
+
+
+def test_train_state_and_probe_match_the_oracle():
+    """The Table I state and the fault handler's decisions (Sec. III-F), library against oracle on random event
+    sequences and on every response pattern of up to five workers."""
+    import itertools
+    from oracle import recovery as R
+    rng = np.random.default_rng(11)
+    for trial in range(50):
+        lr, ep, nb = float(rng.uniform(0.001, 1.0)), int(rng.integers(1, 400)), int(rng.integers(1, 2000))
+        o, g = R.TrainState(lr, ep, nb), F.ftp_state_init(lr, ep, nb)
+        same = lambda: (o.committed_forward_id, o.committed_backward_id, o.status, ep, nb) == \
+            (g.committed_forward_id, g.committed_backward_id, g.status, g.epoch_number, g.batch_number)
+        assert same() and g.committed_forward_id == -1 and g.status == 0 and abs(g.learning_rate - lr) < 1e-6
+        for _ in range(60):
+            ev, b = int(rng.integers(0, 5)), int(rng.integers(0, 300))
+            if ev == 0:
+                o.forward_done(b); F.ftp_state_forward_done(g, b)
+            elif ev == 1:
+                o.backward_done(b); F.ftp_state_backward_done(g, b)
+            elif ev == 2:
+                assert o.timer_expired(b) == F.ftp_state_timer_expired(g, b)
+            elif ev == 3:
+                assert o.reset(b) == F.ftp_state_reset(g, b)
+            assert o.may_forward(b) == F.ftp_state_may_forward(g, b) and same()
+    for n in range(1, 6):
+        for rest in itertools.product((0, 1, 2), repeat=n - 1):
+            resp = [0] + list(rest)
+            assert F.ftp_classify_probe(resp) == R.classify_probe(resp)
+    with pytest.raises(F.FtpError):
+        F.ftp_classify_probe([2, 0])                      # the central node does not fail
+
+
+def test_schedule_helpers_match_the_oracle():
+    for it in range(-2, 1300):
+        assert F.ftp_is_repartition_iter(it) == oracle.is_repartition_iter(it) if it >= 0 else not F.ftp_is_repartition_iter(it)
+        for period in (20, 50, 100):
+            assert F.ftp_is_replication_iter(it, period) == (oracle.is_replication_iter(it, period) if it >= 0 else False)
+    assert [it + 1 for it in range(450) if F.ftp_is_repartition_iter(it)] == [10, 100, 200, 300, 400]
+    assert F.ftp_is_repartition_iter(6, 7, 5) and F.ftp_is_repartition_iter(9, 7, 5) and not F.ftp_is_repartition_iter(7, 7, 5)

@@ -196,3 +196,70 @@ def test_bf16_storage_mode(net):
     assert s.step([0, 1, q.L - 1, q.L], x, y) == lq
     for u in range(q.L):
         assert np.array_equal(s.unit_params(u), q.unit_params(u))
+
+
+# ---- where the bf16 storage mode rounds: one constructed input per rounding point, expected values by hand ----
+def _tail(unit, c, classes=2):
+    L, K = synth.Layer, synth.KIND
+    return [L(unit, K["GAP"], c, c, 0, 1, 0, 0, 0, -1), L(unit, K["FC"], c, classes, 1, 1, 0, 0, 1, -1),
+            L(unit, K["SOFTMAX_CE"], classes, classes, 0, 1, 0, 0, 0, -1)]
+
+
+def test_bf16_mode_rounds_a_convolution_output_to_nearest_even():
+    """1 x 1 convolution, one channel: x = 1.5, w = 1 + 2^-7 (both bf16 numbers).  The exact product
+    1.5 + 2^-7 + 2^-8 = 1.51171875 lies midway between the bf16 neighbours 1.5078125 (odd mantissa) and 1.515625 (even):
+    stored 1.515625.  With w = 1 + 2^-7 + 2^-9 in the master copy the weight is first used as bf16 (rounds to
+    1 + 2^-7): same stored output; the float64 mode keeps 1.5146484375."""
+    L, K = synth.Layer, synth.KIND
+    ls = [L(0, K["CONV2D"], 1, 1, 1, 1, 0, 0, 0, -1)] + _tail(1, 1)
+    cfg = synth.config(1, 1, 1, 1, 2, precision=1)
+    x = np.full((1, 1, 1, 1), 1.5)
+    for w, exact in ((1 + 2.0 ** -7, 1.51171875), (1 + 2.0 ** -7 + 2.0 ** -9, 1.5146484375)):
+        par = [[np.full((1, 1, 1, 1), w)], [], [np.zeros((1, 1, 1, 2)), np.zeros(2)], []]
+        q = oracle.OracleModel(ls, cfg, par, synth.init_state(ls))
+        assert q.forward(0, 1, x)[0, 0, 0, 0] == 1.515625
+        f = oracle.OracleModel(ls, cfg, par, synth.init_state(ls), storage="none")
+        assert f.forward(0, 1, x)[0, 0, 0, 0] == exact
+
+
+def _bn_add_net():
+    """[BN (no activation), residual add of the stage input] on a batch of four 1 x 1 x 1 samples x = (-a, a, -a, a),
+    a = 2^-10, eps = 0: mean 0, variance a^2, xhat = (-1, 1, -1, 1) exactly, gamma / sigma = 256 for gamma = 0.25."""
+    L, K = synth.Layer, synth.KIND
+    ls = [L(0, K["BN"], 1, 1, 0, 1, 0, 0, 0, -1), L(0, K["ADD_RESIDUAL"], 1, 1, 0, 1, 0, 0, 0, -1)] + _tail(1, 1)
+    cfg = synth.config(4, 1, 1, 1, 2, precision=1, bn_eps=0.0)
+    a = 2.0 ** -10
+    x = np.array([-a, a, -a, a]).reshape(4, 1, 1, 1)
+    return ls, cfg, x
+
+
+def test_bf16_mode_rounds_bn_plus_residual_once():
+    """gamma = 0.25, beta = 1.25439453125: z_0 = beta - gamma = 1 + 2^-8 + 2^-11, just above the tie between 1 and
+    1 + 2^-7.  Rounded once, after the add: z_0 + x_0 = 1 + 2^-8 - 2^-11 -> 1.0.  Rounding z first would give
+    1.0078125 - 2^-10 -> 1.0078125."""
+    ls, cfg, x = _bn_add_net()
+    par = [[np.array([0.25]), np.array([1.25439453125])], [], [], [np.zeros((1, 1, 1, 2)), np.zeros(2)], []]
+    q = oracle.OracleModel(ls, cfg, par, synth.init_state(ls))
+    out = q.forward(0, 1, x).reshape(-1)
+    assert out[0] == 1.0
+    from oracle.model import round_bf16
+    assert round_bf16(round_bf16(np.array([1.00439453125])) + x.reshape(-1)[:1])[0] == 1.0078125     # what "twice" would store
+    assert out[1] == round_bf16(np.array([1.50439453125 + 2.0 ** -10]))[0]
+
+
+def test_bf16_mode_rounds_a_gradient_with_two_contributions_after_the_sum():
+    """Same net; incoming gradient d = (0.6875, 0, 9 * 2^-12, 0) (bf16 numbers).  The stage input receives d through
+    the residual and 256 * (d - mean(d) - xhat * mean(d * xhat)) through the BN: for sample 0 that is
+    128 * (d_0 - d_2) = 87.71875.  Stored once, after the sum: 0.6875 + 87.71875 = 88.40625 -> 88.5.  Rounding the
+    BN contribution first (87.5) and then the sum (88.1875) would give 88.0."""
+    ls, cfg, x = _bn_add_net()
+    par = [[np.array([0.25]), np.array([1.0])], [], [], [np.zeros((1, 1, 1, 2)), np.zeros(2)], []]
+    q = oracle.OracleModel(ls, cfg, par, synth.init_state(ls))
+    q.forward(0, 1, x)
+    d = np.array([0.6875, 0.0, 9 * 2.0 ** -12, 0.0]).reshape(4, 1, 1, 1)
+    g = q.backward(0, 1, d).reshape(-1)
+    assert g[0] == 88.5
+    from oracle.model import round_bf16
+    assert round_bf16(np.array([0.6875 + round_bf16(np.array([87.71875]))[0]]))[0] == 88.0
+    # the BN's own parameter gradients are not stored in bf16: dgamma = sum d * xhat, dbeta = sum d, exactly
+    assert q.g[0][0][0] == -(0.6875 + 9 * 2.0 ** -12) and q.g[0][1][0] == 0.6875 + 9 * 2.0 ** -12

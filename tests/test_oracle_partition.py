@@ -187,3 +187,58 @@ def test_schedules_match_the_paper(golden_dir):
     glob = [it + 1 for it in range(210) if oracle.is_replication_iter(it, facts["global_period"])]
     assert chain == [50, 100, 150, 200] and glob == [100, 200]
     assert facts["both_replications_after_batch"] in chain and facts["both_replications_after_batch"] in glob
+
+
+def _facts(golden_dir):
+    facts = {}
+    for line in open(golden_dir + "/schedule_ticks.txt"):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            facts[k] = int(v)
+    return facts
+
+
+def test_state_variables_start_as_table_one_says(golden_dir):
+    """Sec. III-B, Table I: both committed ids are initialised as -1 and the status as 0."""
+    from oracle import recovery as R
+    facts = _facts(golden_dir)
+    st = R.TrainState(0.1, 300, 196)
+    assert st.committed_forward_id == facts["committed_id_init"] and st.committed_backward_id == facts["committed_id_init"]
+    assert st.status == facts["status_init"]
+    assert (st.learning_rate, st.epoch_number, st.batch_number) == (0.1, 300, 196)
+
+
+def test_fault_handler_state_follows_section_three_f():
+    """The worked case of Sec. IV-E in the words of Sec. III-F: the worker dies when batch 205 starts its backward
+    pass.  Batches up to 204 have gone all the way round, 205..207 have been forwarded into the pipeline.  The
+    timer of 205 triggers the handler once (status 1), later timers do not; batches beyond the committed forward
+    id are held back; the reset sets both ids to 205, the status to 0, and training resumes by forwarding 205."""
+    from oracle import recovery as R
+    st = R.TrainState(0.1, 1, 1000)
+    for b in range(208):
+        st.forward_done(b)
+        if b - 3 >= 0:
+            st.backward_done(b - 3)
+    assert (st.committed_forward_id, st.committed_backward_id, st.status) == (207, 204, 0)
+    assert st.may_forward(208)
+    assert st.timer_expired(205) is True and st.status == 1
+    assert st.timer_expired(206) is False and st.timer_expired(207) is False and st.status == 1
+    assert not st.may_forward(208) and st.may_forward(207)
+    assert st.reset(205) == 205
+    assert (st.committed_forward_id, st.committed_backward_id, st.status) == (205, 205, 0)
+    assert st.may_forward(206)
+
+
+def test_probe_outcomes_are_the_three_cases_of_the_paper():
+    from oracle import recovery as R
+    N, S, X = R.NORMAL, R.RESTARTED, R.SILENT
+    assert R.classify_probe([N, N, N, N]) == (R.RESTART_BATCH, [], None)              # all respond normally
+    assert R.classify_probe([N, N, S, N]) == (R.RESEND_STATE, [], 2)                  # one restarted at once
+    assert R.classify_probe([N, X, N, X]) == (R.REDISTRIBUTE, [1, 3], None)           # multiple workers silent
+    assert R.classify_probe([N, N, X, N]) == (R.REDISTRIBUTE, [2], None)              # one silent: Algorithm 1 with its index
+    assert R.classify_probe([N, S, X, N]) == (R.REDISTRIBUTE, [1, 2], None)           # a restart beside a failure: both lost their weights
+    # the failed list is what the recovery plan takes: survivors keep their order
+    action, failed, _ = R.classify_probe([N, X, N, X, N])
+    assert oracle.renew_worker_list([0, 1, 2, 3, 4], failed) == [0, 2, 4]
+    plan = oracle.recovery_sources([0, 2, 4, 6, 8, 10], failed, [0, 4, 7, 10])
+    assert [u for items in plan for u, _ in items] == list(range(10))

@@ -4,11 +4,12 @@ Some users of the library sit where device memory cannot be requested: inside a 
 section that an allocation would stall, or under a host that hands out buffers and keeps the
 allocator to itself.  ftp_conv_wgrad_static serves them with scratch built into the library.
 Here its result is compared with the weight gradient that ftp_run_stage_backward leaves in the
-gradient arena for the same convolution, on two calls in a row (the second after a call of a
-different shape has dirtied the shared scratch)."""
+gradient arena for the same convolution and with the oracle's, on two calls in a row (the second
+after a call of a different shape has dirtied the shared scratch)."""
 import numpy as np
 import pytest
 
+import oracle.ops
 import synth
 from helpers import TOL_FP32, rel_err, to_dev
 
@@ -49,6 +50,9 @@ def test_static_scratch_wgrad_matches_model_api_twice(n, h, cin, cout, k, stride
     torch.cuda.synchronize()
     first = dw.cpu().numpy().reshape(-1)
     assert rel_err(first, ref) <= TOL_FP32
+    _, want_dw, _ = oracle.ops.conv_bwd(x.cpu().numpy().astype(np.float64), np.zeros((k, k, cin, cout)), gout.cpu().numpy().astype(np.float64),
+                                        stride, pad, pad, False)
+    assert rel_err(first, want_dw.reshape(-1)) <= TOL_FP32
     # a call of another shape leaves its partial sums in the shared scratch
     x2, g2 = torch.randn(4, 8, 8, 16, device="cuda"), torch.randn(4, 8, 8, 8, device="cuda")
     dw2 = torch.empty(1, 1, 16, 8, device="cuda")
@@ -75,3 +79,16 @@ def test_static_scratch_refuses_shapes_beyond_its_size():
     with pytest.raises(F.FtpError) as e:
         F.ftp_conv_wgrad_static(xs, dys, dws, 3, 1, 1)        # 9*256*256 floats x several splits > 8 MiB
     assert "scratch" in str(e.value)
+
+
+def test_static_scratch_wrapper_refuses_wrong_shapes_and_types():
+    import torch
+    x = torch.zeros(2, 8, 8, 16, device="cuda")
+    dy = torch.zeros(2, 8, 8, 8, device="cuda")
+    dw = torch.zeros(1, 1, 16, 8, device="cuda")
+    F.ftp_conv_wgrad_static(x, dy, dw, 1, 1, 0)
+    for bad in ((x, dy[:, :4], dw), (x, dy, dw[:, :, :8]), (x.double(), dy, dw), (x, dy.cpu(), dw), (x, dy.permute(0, 2, 1, 3)[:, ::2], dw)):
+        with pytest.raises(F.FtpError):
+            F.ftp_conv_wgrad_static(*bad, 1, 1, 0)
+    with pytest.raises(F.FtpError):
+        F.ftp_conv_wgrad_static(x, dy, dw, 3, 1, 0)           # dy would have to be 6 x 6
