@@ -23,10 +23,10 @@ __device__ __forceinline__ float bn_z(float y, float mh, float ml, float scale, 
     return fmaf((y - mh) - ml, scale, beta);
 }
 
-// the same batch norm + activation in the form used by kernels that normalise what they load: one multiply-add with
-// offset = beta - mean * scale, then the clamp (lo, hi) of the activation
-__device__ __forceinline__ float xf_z(float y, float scale, float offset, float lo, float hi) {
-    return fminf(fmaxf(fmaf(y, scale, offset), lo), hi);
+// the same batch norm + activation in the form used by kernels that normalise what they load: the float part of the mean
+// is subtracted, its remainder is folded into offset = beta - mean_lo * scale, then the clamp (lo, hi) of the activation
+__device__ __forceinline__ float xf_z(float y, float mean, float scale, float offset, float lo, float hi) {
+    return fminf(fmaxf(fmaf(y - mean, scale, offset), lo), hi);
 }
 
 // a value as the tensor of element type T would hold it

@@ -89,15 +89,15 @@ template <int V> __device__ __forceinline__ void ldtab(const float* p, float (&o
 
 // Per-thread constants of a batch norm applied on load to V consecutive channels (see BnXform)
 template <typename T, int V> struct XfRegs {
-    float sc[V], of[V];
+    float mu[V], sc[V], of[V];
     float lo, hi;
     __device__ __forceinline__ void load(const BnXform& x, int c) {
-        ldtab<V>(x.scale + c, sc); ldtab<V>(x.offset + c, of);
+        ldtab<V>(x.mean + c, mu); ldtab<V>(x.scale + c, sc); ldtab<V>(x.offset + c, of);
         lo = x.lo; hi = x.hi;
     }
     __device__ __forceinline__ void apply(float (&v)[V]) const {
 #pragma unroll
-        for (int e = 0; e < V; ++e) v[e] = as_stored<T>(xf_z(v[e], sc[e], of[e], lo, hi));
+        for (int e = 0; e < V; ++e) v[e] = as_stored<T>(xf_z(v[e], mu[e], sc[e], of[e], lo, hi));
     }
 };
 
@@ -330,7 +330,7 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
         const double rs = rsqrt_f64(var + (double)eps);
         const float sc = (float)((double)ga * rs);
         scale[c] = sc;
-        offset[c] = (float)((double)be - mu * (double)sc);     // z = y * scale + offset, for readers that normalise as they load
+        offset[c] = (float)((double)be - (mu - (double)(float)mu) * (double)sc);     // z = (y - mean) * scale + offset, for readers that normalise as they load
         shift[c] = be;                            // z = (y - mean) * scale + beta, the mean kept as a two-float sum
         const float mh = (float)mu;
         mean[c] = mh;
@@ -1023,7 +1023,7 @@ __device__ __forceinline__ void dw3_load_row(const T* __restrict__ img, int hi, 
 }
 
 template <typename T, bool XF, bool STATS>
-__global__ void __launch_bounds__(256, 2) dw3_fwd_rows_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int N, int H, int W,
+__global__ void __launch_bounds__(256, XF ? 1 : 2) dw3_fwd_rows_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int N, int H, int W,
                                                               int C, int RH, int HC, double* __restrict__ stats, BnXform xf) {
     grid_dep_sync();
     __shared__ __align__(16) float wsm[9][32];
@@ -1652,10 +1652,11 @@ static Dw3Plan plan_dw3(const ConvGeom& g, int resident_blocks) {
     const int strips_w = (g.W + 3) / 4, cgroups = (g.Cin / 4 + 7) / 8;
     const long long slots_x = std::max(1, resident_blocks / cgroups);
     auto groups = [&](int hc) { return ((long long)g.N * hc * strips_w + 31) / 32; };
-    // chunks of about eight rows: a quarter more rows loaded than computed, and enough groups that the blocks' shares differ little
+    // chunks of at most eight rows (a quarter more rows loaded than computed, and groups enough that the blocks' shares
+    // differ little); shorter ones, down to two rows, while the blocks would not fill the machine (small maps: latency counts)
     int best = 1;
     while ((g.H + best - 1) / best > 8) best *= 2;
-    (void)groups;
+    while (groups(best) * cgroups < resident_blocks && (g.H + 2 * best - 1) / (2 * best) >= 2) best *= 2;
     Dw3Plan p;
     p.RH = (g.H + best - 1) / best;
     p.HC = (g.H + p.RH - 1) / p.RH;
@@ -1679,10 +1680,10 @@ void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_
     const unsigned tiles = (unsigned)(((g.Wo + (1 << tws) - 1) >> tws) * (((long long)g.N * g.Ho + (64 >> tws) - 1) / (64 >> tws)));
     if (stats) stats->out->entries = 0;
     const bool xf = x_xform != nullptr;
-    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f};
-    const bool xf_vec = !xf || (aligned16(xv.scale) && aligned16(xv.offset));
+    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f};
+    const bool xf_vec = !xf || (aligned16(xv.mean) && aligned16(xv.scale) && aligned16(xv.offset));
     if (dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w) && xf_vec) {
-        const Dw3Plan pl = plan_dw3(g, 2 * sm_count());
+        const Dw3Plan pl = plan_dw3(g, (xf ? 1 : 2) * sm_count());         // resident blocks per SM: see the kernel's launch bounds
         const dim3 grid(pl.gx, pl.gy);
         double* sp = stats ? stats->partial : nullptr;
         if (stats) {
@@ -1724,7 +1725,7 @@ void dwconv_dgrad(const T* dy, const float* w, const T* addend, T* dx, const Con
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
         const long long strips = (long long)g.N * g.H * ((g.W + 3) / 4);
         launch(dw_strip_kernel<T, 4, 1, 0, false>, dim3((unsigned)((strips + 31) / 32), (g.Cin / 4 + 7) / 8), dim3(256), 0, st, dy, w, addend, dx, g.N, g.H, g.W, g.Cin, (double*)nullptr,
-               BnXform{nullptr, nullptr, 0.f, 0.f});
+               BnXform{nullptr, nullptr, nullptr, 0.f, 0.f});
         return;
     }
     if (can_vec<T>(g.Cin, dy, addend, dx) && aligned16(w)) {
@@ -1762,8 +1763,8 @@ template <typename T>
 void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st, const BnXform* x_xform) {
     constexpr int V = VecOf<T>::N;
     const bool xf = x_xform != nullptr;
-    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f};
-    const bool xf_vec = !xf || (aligned16(xv.scale) && aligned16(xv.offset));
+    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f};
+    const bool xf_vec = !xf || (aligned16(xv.mean) && aligned16(xv.scale) && aligned16(xv.offset));
     // four channels per thread for either type: with eight bf16 channels the nine accumulators would leave too few warps per SM
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy) && xf_vec) {
         constexpr int SV = 4;
@@ -1804,8 +1805,8 @@ template <typename T>
 bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
                       cudaStream_t st, const BnXform* x_xform) {
     const bool xf = x_xform != nullptr;
-    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f};
-    const bool xf_vec = !xf || (aligned16(xv.scale) && aligned16(xv.offset));
+    const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f};
+    const bool xf_vec = !xf || (aligned16(xv.mean) && aligned16(xv.scale) && aligned16(xv.offset));
     if (!(dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy, addend, dx) && g.Cin % 4 == 0 && xf_vec)) return false;
     const Dw3Plan pl = plan_dw3(g, sm_count());
     const dim3 grid(pl.gx, pl.gy);

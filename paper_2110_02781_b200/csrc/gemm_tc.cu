@@ -9,6 +9,7 @@
 // own 32 lanes), add the optional addend, convert and store.  Every wait on an mbarrier is bounded: when it
 // runs out the kernel records a code in an error word, lets its own copies land, frees its tensor memory
 // and returns; the host reports FTP_ETIMEOUT.
+#include <algorithm>
 #include "gemm_tc_common.cuh"
 
 namespace ftp {
@@ -36,11 +37,16 @@ struct TcParams {
     int M, N, K;                   // K: reduction length (conv: 9 * channels)
     int* err;
     ConvTap conv;
+    float* partial;                // reduction cut into gridDim.z slices: partial sums [slice][M][N] (float) instead of D
+    int kb_per_slice;              // 64-wide reduction blocks per slice
 };
 
-template <int BN>
+// NSTG: depth of the operand ring.  A block's reduction advances one stage per (load latency / NSTG), so products with
+// one block per SM or fewer take a ring as deep as shared memory holds, products with several blocks per SM a short one.
+template <int BN, int NSTG>
 __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                                                                 const __grid_constant__ CUtensorMap mapD, const TcParams p) {
+    constexpr int TC_STAGES = NSTG;
     constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = BN * TC_BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -49,7 +55,10 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * TC_BM;
-    const int num_kb = (p.K + TC_BK - 1) / TC_BK;
+    const int all_kb = (p.K + TC_BK - 1) / TC_BK;
+    const bool sliced = p.partial != nullptr;
+    const int kb0 = sliced ? blockIdx.z * p.kb_per_slice : 0;
+    const int num_kb = sliced ? max(0, min(all_kb, kb0 + p.kb_per_slice) - kb0) : all_kb;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
 
     if (threadIdx.x == 0) {
@@ -78,12 +87,13 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
                 const uint32_t ph = (kb / TC_STAGES) & 1;
                 if (kb >= TC_STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 1)) break;
                 const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
+                const int gkb = kb0 + kb;                    // block of the whole reduction
                 mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
                 if (!p.conv.enabled) {
-                    tma_load_2d(sa, &mapA, kb * TC_BK, m0, full0 + 8 * s);
-                    tma_load_2d(sb, &mapB, kb * TC_BK, n0, full0 + 8 * s);
+                    tma_load_2d(sa, &mapA, gkb * TC_BK, m0, full0 + 8 * s);
+                    tma_load_2d(sb, &mapB, gkb * TC_BK, n0, full0 + 8 * s);
                 } else {
-                    const int tap = kb / p.conv.chunks, cc = kb - tap * p.conv.chunks, r = tap / 3, sx = tap - 3 * r;
+                    const int tap = gkb / p.conv.chunks, cc = gkb - tap * p.conv.chunks, r = tap / 3, sx = tap - 3 * r;
                     const int hw = p.conv.H * p.conv.W, img = m0 / hw, h0 = (m0 - img * hw) / p.conv.W;
                     const int dh = p.conv.flip ? 1 - r : r - 1, dw = p.conv.flip ? 1 - sx : sx - 1;
                     tma_load_4d(sa, &mapA, cc * 64, dw, h0 + dh, img, full0 + 8 * s);
@@ -122,15 +132,30 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
     } else {
         // ---- epilogue: warps 2..5 own tensor-memory lanes 32*(warp%4) .. +31 ----
         const int q = warp & 3;
-        const bool have = mbar_wait(accum, 0, p.err, 3);         // every stage has been consumed by now: the ring is free
+        const bool have = num_kb > 0 ? mbar_wait(accum, 0, p.err, 3) : true;         // every stage has been consumed by now: the ring is free
         if (have) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int m = m0 + q * 32 + lane;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+                if (num_kb > 0) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+                else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
                 const int nb = n0 + c * 32;
+                if (sliced) {                                        // float partial sums of this slice, added up by a second kernel
+                    if (m < p.M) {
+                        float* prow = p.partial + ((long long)blockIdx.z * p.M + m) * p.N + nb;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (nb + g * 4 < p.N)
+                                *reinterpret_cast<float4*>(prow + g * 4) = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
+                                                                                      __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                    }
+                    continue;
+                }
                 if (m < p.M) {
                     __nv_bfloat16* drow = p.D + (long long)m * p.N + nb;
                     const __nv_bfloat16* arow = p.addend ? p.addend + (long long)m * p.N + nb : nullptr;
@@ -159,12 +184,12 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_tn_kernel(const __grid_con
                     }
                 }
             }
-            if (BN >= 64) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (BN >= 64 && !sliced) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         if (BN >= 64) {
             // whole 128-byte lines leave through TMA (clipped at the edges of D) instead of 16-byte pieces per thread
             asm volatile("bar.sync 1, 128;" ::: "memory");                  // the four epilogue warps
-            if (have && threadIdx.x == 64) {
+            if (have && !sliced && threadIdx.x == 64) {
 #pragma unroll 1
                 for (int c = 0; c < BN / 64; ++c)
                     if (n0 + c * 64 < p.N)
@@ -369,37 +394,93 @@ bool conv_tiles_ok(int H, int W, int pix) {
     return bh % H == 0;            // several whole images per box
 }
 
+// Ring depth and reduction slices of a forward / data-gradient product with `tiles` output tiles and `nkb` 64-wide blocks
+// of the reduction.  At most one block per SM: the deepest ring (the reduction then advances at load latency / 6 per
+// block instead of / 3).  Far fewer blocks than SMs and a long reduction: cut it into slices (float partial sums,
+// added in order by a second kernel).
+struct TnPlan { int stages, S, kbps; };
+static TnPlan plan_tn(long long tiles, int nkb, long long out_elems) {
+    const int sms = sm_count();
+    TnPlan pl{tiles <= sms ? 6 : 3, 1, nkb};
+    if (tiles * 2 <= sms && nkb >= 16) {
+        long long S = sms / tiles;
+        if (S > nkb / 8) S = nkb / 8;
+        if (S > 8) S = 8;
+        const long long cap = (8LL << 20) / std::max<long long>(out_elems, 1);
+        if (S > cap) S = cap;
+        if (S > 1) {
+            pl.kbps = (int)((nkb + S - 1) / S);
+            pl.S = (nkb + pl.kbps - 1) / pl.kbps;
+        }
+    }
+    return pl;
+}
+
+// D = bf16(addend + sum over S float slices), slice order fixed
+__global__ void __launch_bounds__(256) slice_sum_bf16_kernel(const float4* __restrict__ part, int S, long long count4, const __nv_bfloat16* __restrict__ addend,
+                                                             __nv_bfloat16* __restrict__ out) {
+    grid_dep_sync();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count4) return;
+    float4 a = part[i];
+    for (int s = 1; s < S; ++s) { const float4 v = part[(long long)s * count4 + i]; a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+    if (addend) {
+        const uint2 q = *reinterpret_cast<const uint2*>(addend + i * 4);
+        a.x += __uint_as_float(q.x << 16); a.y += __uint_as_float(q.x & 0xffff0000u);
+        a.z += __uint_as_float(q.y << 16); a.w += __uint_as_float(q.y & 0xffff0000u);
+    }
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+    *reinterpret_cast<uint2*>(out + i * 4) = make_uint2(*reinterpret_cast<const unsigned*>(&lo), *reinterpret_cast<const unsigned*>(&hi));
+}
+
+template <int BN, int NSTG>
+bool launch_tn_kernel(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const TcParams& p, dim3 grid, cudaStream_t st) {
+    constexpr int smem = NSTG * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
+    static_assert(NSTG * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) >= TC_BM * BN * 2, "the epilogue stages its tile in the ring");
+    if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN, NSTG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    launch(tc_gemm_tn_kernel<BN, NSTG>, grid, dim3(TC_THREADS), smem, st, ma, mb, md, p);
+    return true;
+}
+
+// shared tail of the 1x1 and 3x3 launchers: plan, launch, second pass
 template <int BN>
-bool launch_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No,
-                    int flip, int* err, cudaStream_t st) {
+bool run_tn(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, TcParams p, float* scratch, cudaStream_t st) {
+    const long long tiles = (long long)((p.N + BN - 1) / BN) * ((p.M + TC_BM - 1) / TC_BM);
+    const int nkb = (p.K + TC_BK - 1) / TC_BK;
+    TnPlan pl = plan_tn(tiles, nkb, (long long)p.M * p.N);
+    if (!scratch || ((long long)p.M * p.N) % 4 != 0) { pl.S = 1; pl.kbps = nkb; }
+    const __nv_bfloat16* addend = p.addend;
+    if (pl.S > 1) { p.partial = scratch; p.kb_per_slice = pl.kbps; p.addend = nullptr; }
+    const dim3 grid((p.N + BN - 1) / BN, (p.M + TC_BM - 1) / TC_BM, pl.S);
+    const bool ok = pl.stages == 6 ? launch_tn_kernel<BN, 6>(ma, mb, md, p, grid, st) : launch_tn_kernel<BN, 3>(ma, mb, md, p, grid, st);
+    if (ok && pl.S > 1) {
+        const long long count4 = (long long)p.M * p.N / 4;
+        launch(slice_sum_bf16_kernel, dim3((unsigned)((count4 + 255) / 256)), dim3(256), 0, st, reinterpret_cast<const float4*>(scratch), pl.S, count4, addend, p.D);
+    }
+    return ok;
+}
+
+template <int BN>
+bool launch_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int N, int H, int W, int Ca,
+                    int No, int flip, int* err, cudaStream_t st) {
     CUtensorMap ma, mb, md;
     if (!make_map_4d(&ma, A, N, H, W, Ca, TC_BM) || !make_map_2d(&mb, B, 9LL * No, Ca, BN)) return false;
     if (BN >= 64) { if (!make_map_2d(&md, D, (long long)N * H * W, No, TC_BM)) return false; }
     else md = mb;
-    constexpr int smem = TC_STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
-    if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
     const int M = N * H * W;
-    TcParams p{D, addend, M, No, 9 * Ca, err, ConvTap{1, H, W, Ca / 64, flip, No}};
-    launch(tc_gemm_tn_kernel<BN>, dim3((No + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, md, p);
-    return true;
+    TcParams p{D, addend, M, No, 9 * Ca, err, ConvTap{1, H, W, Ca / 64, flip, No}, nullptr, 0};
+    return run_tn<BN>(ma, mb, md, p, scratch, st);
 }
 
 template <int BN>
-bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K, int* err,
+bool launch_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int M, int N, int K, int* err,
                cudaStream_t st) {
     CUtensorMap ma, mb, md;
     if (!make_map_2d(&ma, A, M, K, TC_BM) || !make_map_2d(&mb, B, N, K, BN)) return false;
     if (BN >= 64) { if (!make_map_2d(&md, D, M, N, TC_BM)) return false; }
     else md = mb;
-    constexpr int smem = TC_STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_tn_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-        configured = true;
-    }
-    TcParams p{D, addend, M, N, K, err, ConvTap{0, 0, 0, 0, 0, 0}};
-    launch(tc_gemm_tn_kernel<BN>, dim3((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM), dim3(TC_THREADS), smem, st, ma, mb, md, p);
-    return true;
+    TcParams p{D, addend, M, N, K, err, ConvTap{0, 0, 0, 0, 0, 0}, nullptr, 0};
+    return run_tn<BN>(ma, mb, md, p, scratch, st);
 }
 
 template <int BN>
@@ -456,11 +537,21 @@ bool tc_conv3x3_supported(int N, int H, int W, int Ca, int No, const void* A, co
 
 // 3x3, stride 1, pad 1.  Forward (flip 0): A = x (N,H,W,Ca), B = weights [9][No][Ca]; data gradient (flip 1): A = dy,
 // B = weights [9][No = cin][Ca = cout].  D (N,H,W,No) bf16.
-bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No, int flip,
-                int* err, cudaStream_t st) {
-    if (No > 64) return launch_conv3x3<128>(A, B, addend, D, N, H, W, Ca, No, flip, err, st);
-    if (No > 32) return launch_conv3x3<64>(A, B, addend, D, N, H, W, Ca, No, flip, err, st);
-    return launch_conv3x3<32>(A, B, addend, D, N, H, W, Ca, No, flip, err, st);
+bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int N, int H, int W, int Ca,
+                int No, int flip, int* err, cudaStream_t st) {
+    if (No > 64) return launch_conv3x3<128>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
+    if (No > 32) return launch_conv3x3<64>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
+    return launch_conv3x3<32>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
+}
+
+size_t tc_gemm_scratch_floats(int M, int N, int K) {
+    size_t most = 0;
+    for (int BN : {32, 64, 128}) {
+        const long long tiles = (long long)((N + BN - 1) / BN) * ((M + TC_BM - 1) / TC_BM);
+        const TnPlan pl = plan_tn(tiles, (K + TC_BK - 1) / TC_BK, (long long)M * N);
+        if (pl.S > 1) most = std::max(most, (size_t)pl.S * M * N);
+    }
+    return most;
 }
 
 size_t tc_wgrad3x3_scratch_floats(long long R, int Mo, int No) {
@@ -495,11 +586,11 @@ bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const 
     return M >= 1 && N % 8 == 0 && K % 8 == 0 && N >= 8 && K >= 8 && a16(A) && a16(B) && a16(D) && a16(addend) && encode_fn() != nullptr;
 }
 
-bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K, int* err,
+bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int M, int N, int K, int* err,
                 cudaStream_t st) {
-    if (N > 64) return launch_tn<128>(A, B, addend, D, M, N, K, err, st);
-    if (N > 32) return launch_tn<64>(A, B, addend, D, M, N, K, err, st);
-    return launch_tn<32>(A, B, addend, D, M, N, K, err, st);
+    if (N > 64) return launch_tn<128>(A, B, addend, D, scratch, M, N, K, err, st);
+    if (N > 32) return launch_tn<64>(A, B, addend, D, scratch, M, N, K, err, st);
+    return launch_tn<32>(A, B, addend, D, scratch, M, N, K, err, st);
 }
 
 }  // namespace ftp

@@ -16,6 +16,7 @@
 //    gradients of the weight gradient); the tensor core takes them as they land (MN-major operands), and the
 //    converter warps only add the lo parts.
 // Every wait is bounded; see gemm_tc.cu for the error protocol.
+#include <cstdlib>
 #include "gemm_tc_common.cuh"
 #include "bn_math.cuh"
 
@@ -51,18 +52,19 @@ __device__ __forceinline__ float tf32_lo_of(float v) { return v - __uint_as_floa
 
 // Batch norm + activation on a float4 of four consecutive channels (constants in registers), zero where !keep
 struct Xf4 {
-    float4 sc, of;
+    float4 mu, sc, of;
     __device__ __forceinline__ void load(const BnXform& x, int c, bool ok) {
         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        mu = ok ? __ldg(reinterpret_cast<const float4*>(x.mean + c)) : z;
         sc = ok ? __ldg(reinterpret_cast<const float4*>(x.scale + c)) : z;
         of = ok ? __ldg(reinterpret_cast<const float4*>(x.offset + c)) : z;
     }
     __device__ __forceinline__ float4 apply(float4 v, float lo, float hi, bool keep) const {
         float4 o;
-        o.x = keep ? xf_z(v.x, sc.x, of.x, lo, hi) : 0.f;
-        o.y = keep ? xf_z(v.y, sc.y, of.y, lo, hi) : 0.f;
-        o.z = keep ? xf_z(v.z, sc.z, of.z, lo, hi) : 0.f;
-        o.w = keep ? xf_z(v.w, sc.w, of.w, lo, hi) : 0.f;
+        o.x = keep ? xf_z(v.x, mu.x, sc.x, of.x, lo, hi) : 0.f;
+        o.y = keep ? xf_z(v.y, mu.y, sc.y, of.y, lo, hi) : 0.f;
+        o.z = keep ? xf_z(v.z, mu.z, sc.z, of.z, lo, hi) : 0.f;
+        o.w = keep ? xf_z(v.w, mu.w, sc.w, of.w, lo, hi) : 0.f;
         return o;
     }
 };
@@ -652,7 +654,9 @@ G32Plan plan_gemm32(int M, int N, int K) {
                 const long long ctas = tiles * S, slots = (long long)sms * fit;
                 const long long waves = (ctas + slots - 1) / slots;
                 const double conc = (double)std::min<long long>(fit, (ctas + sms - 1) / sms);
-                const double chain = kbps * (st >= 2 ? 0.45 : 1.3), shared = conc * kbps * t_share;
+                // a block's serial chain per 32-wide step: with a ring of `st` stages that many loads are in flight ahead of the split
+                static const double per_step[5] = {0.0, 1.6, 1.0, 0.7, 0.55};
+                const double chain = kbps * per_step[st], shared = conc * kbps * t_share;
                 double t = waves * (t0 + (chain > shared ? chain : shared));
                 if (S > 1) t += 2.5 + (double)(S + 1) * M * N * 4.0 / 3.0e6;
                 if (t < best_t - 1e-9) { best_t = t; best = G32Plan{BN, S, kbps * T32_BK, st}; }
@@ -677,7 +681,7 @@ bool tc32_gemm(const float* A, const float* B, const float* B_lo, const float* a
     if (B_lo) { if (!make_map_f32(&ml, B_lo, N, K, BN)) return false; }
     else ml = mb;
     T32Params p{out, g.S > 1 ? nullptr : addend, M, N, K, g.rps, B_lo ? 1 : 0, err, (stats && g.S == 1) ? stats->partial : nullptr,
-                a_xform ? *a_xform : BnXform{nullptr, nullptr, 0.f, 0.f}, a_xform ? 1 : 0};
+                a_xform ? *a_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f}, a_xform ? 1 : 0};
     const dim3 grid((N + BN - 1) / BN, (M + TC_BM - 1) / TC_BM, g.S);
     const int nkb = g.rps / T32_BK, stages = g.stages > nkb ? (nkb < 1 ? 1 : nkb) : g.stages;
     bool ok;
@@ -717,7 +721,7 @@ bool tc32_wgrad(const float* X, const float* dY, float* dW, float* scratch, long
     float* out = two_pass ? scratch : dW;
     if (!make_map_f32(&mx, A, R, m, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) || !make_map_f32(&my, B, R, n, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) || !make_map_out(&md, out, w.S, m, n)) return false;
     T32Params p{out, nullptr, m, n, (int)R, w.rows_per_split, 0, err, nullptr,
-                x_xform ? *x_xform : BnXform{nullptr, nullptr, 0.f, 0.f}, x_xform ? (w.swap ? 2 : 1) : 0};
+                x_xform ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f}, x_xform ? (w.swap ? 2 : 1) : 0};
     const dim3 grid((m + TC_BM - 1) / TC_BM, (n + w.BN - 1) / w.BN, w.S);
     bool ok;
     if (w.BN == 128) ok = launch32_wgrad<128>(mx, my, md, p, grid, st);

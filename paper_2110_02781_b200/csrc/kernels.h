@@ -8,17 +8,20 @@
 namespace ftp {
 
 // A consumer may be handed the input of a batch norm instead of its output: it then applies
-// z = min(max(y * scale + offset, lo), hi) to every element it loads (padding stays zero), so the normalised
-// tensor never exists in memory.  scale = gamma * rstd and offset = beta - mean * scale (formed in double by
-// bn_finalize) have one float per channel, 16-byte aligned; (lo, hi) = (-inf, inf), (0, inf) or (0, 6).
+// z = min(max((y - mean) * scale + offset, lo), hi) to every element it loads (padding stays zero), so the
+// normalised tensor never exists in memory.  mean is the float nearest the batch mean (subtracting it first keeps
+// float accuracy in channels whose spread is small beside their mean), scale = gamma * rstd, and offset = beta minus
+// the remainder of the mean times scale (formed in double by bn_finalize); one float per channel each, 16-byte
+// aligned; (lo, hi) = (-inf, inf), (0, inf) or (0, 6).
 struct BnXform {
+    const float* mean;
     const float* scale;
     const float* offset;
     float lo, hi;
 };
-inline BnXform make_xform(const float* scale, const float* offset, int act) {
+inline BnXform make_xform(const float* mean, const float* scale, const float* offset, int act) {
     const float inf = __builtin_huge_valf();
-    return BnXform{scale, offset, act == 0 ? -inf : 0.f, act == 2 ? 6.f : inf};
+    return BnXform{mean, scale, offset, act == 0 ? -inf : 0.f, act == 2 ? 6.f : inf};
 }
 
 // Geometry of a (dense or depthwise) convolution.  Activations are (N, H, W, C).
@@ -54,12 +57,14 @@ void conv_wgrad_bf16_simt(const __nv_bfloat16* x, const __nv_bfloat16* dy, float
 // contiguous.  tc_gemm_supported: channel counts multiples of 8, 16-byte aligned pointers, driver entry point found.
 // err: device int, stays 0 unless a bounded wait inside the kernel ran out.  Returns false if nothing was launched.
 bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
-bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int M, int N, int K,
+// scratch (nullable): tc_gemm_scratch_floats(M, N, K) floats; lets products with few tiles and a long reduction cut it into slices
+size_t tc_gemm_scratch_floats(int M, int N, int K);
+bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int M, int N, int K,
                 int* err, cudaStream_t st);
 // 3x3 / stride 1 / pad 1 convolutions on the same kernels through 4-D tensor maps (zero fill = padding).
 bool tc_conv3x3_supported(int N, int H, int W, int Ca, int No, const void* A, const void* B, const void* D, const void* addend);
-bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, int N, int H, int W, int Ca, int No,
-                int flip, int* err, cudaStream_t st);
+bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int N, int H, int W, int Ca,
+                int No, int flip, int* err, cudaStream_t st);          // scratch: tc_gemm_scratch_floats(N*H*W, No, 9*Ca) floats, nullable
 size_t tc_wgrad3x3_scratch_floats(long long R, int Mo, int No);
 int tc_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, int N, int H, int W, int Mo, int No, int* err,
                 cudaStream_t st);

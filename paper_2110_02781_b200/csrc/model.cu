@@ -170,8 +170,11 @@ ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cf
     // A batch norm inside a unit whose only reader can normalise while it loads (a depthwise convolution, or a 1x1
     // convolution on the split-tf32 tensor-core kernel) is never applied in memory: only its statistics and
     // per-channel constants are computed, and forward and weight gradient of the reader work from the BN's input.
-    const char* fe = std::getenv("FTP_FUSE_BN");                      // bit 0: into depthwise readers, bit 1: into 1x1 readers; 0: every batch norm stores its output
-    const int fuse = fe ? std::atoi(fe) : 2;
+    // FTP_FUSE_BN (A/B measurements): bit 0 = into depthwise readers, bit 1 = into 1x1 readers, 0 = every batch norm stores
+    // its output.  Default: both in float models; none in bf16 models, whose depthwise kernels are bound by instruction
+    // issue and lose more to the extra arithmetic per loaded element than the saved pass gives back.
+    const char* fe = std::getenv("FTP_FUSE_BN");
+    const int fuse = fe ? std::atoi(fe) : (cfg->precision == FTP_FP32 ? 3 : 0);
     const char* fm = std::getenv("FTP_FUSE_MAX_MB");                  // only batch norms whose output is at most this large (A/B measurements)
     const double fuse_max_bytes = fm ? std::atof(fm) * 1e6 : 1e30;
     for (int i = 0; fuse && i + 1 < n; ++i) {
@@ -277,7 +280,11 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             if (o.d.act == FTP_ACT_NONE && o.b_off < 0) red = std::max(red, stem_wgrad_scratch_floats(o.g));
             red = std::max(red, tc32_wgrad_scratch_floats(Mout, o.C, o.Co));
             red = std::max(red, std::max(tc32_gemm_scratch_floats((int)Mout, o.Co, o.C), tc32_gemm_scratch_floats((int)Mout, o.C, o.Co)));
-            if (m.cfg.precision == FTP_BF16) red = std::max(red, std::max(tc_wgrad_scratch_floats(Mout, o.C, o.Co), tc_wgrad3x3_scratch_floats(Mout, o.C, o.Co)));
+            if (m.cfg.precision == FTP_BF16) {
+                red = std::max(red, std::max(tc_wgrad_scratch_floats(Mout, o.C, o.Co), tc_wgrad3x3_scratch_floats(Mout, o.C, o.Co)));
+                const int kk = o.g.kh * o.g.kw;
+                red = std::max(red, std::max(tc_gemm_scratch_floats((int)Mout, o.Co, kk * o.C), tc_gemm_scratch_floats((int)Mout, o.C, kk * o.Co)));
+            }
             o.fold = make_fold(Mout, o.Co, o.out_f32 ? 4 : m.esize);
             if (o.d.act != FTP_ACT_NONE || o.d.has_bias) foldd = std::max(foldd, fold_partial_doubles(o.fold));
             if (o.d.act != FTP_ACT_NONE) dpre = std::max(dpre, obytes);
@@ -382,9 +389,9 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
         const ColStatsReq* stats_req = nullptr;
         if (m->producer_stats && i + 1 <= last && m->ops[i + 1].d.kind == FTP_BN && o.d.kind != FTP_BN) { req.fold = &m->ops[i + 1].fold; stats_req = &req; }
         // the input is what a deferred batch norm read: this op normalises as it loads
-        BnXform xfv{nullptr, nullptr, 0.f, 0.f};
+        BnXform xfv{nullptr, nullptr, nullptr, 0.f, 0.f};
         const BnXform* xf = nullptr;
-        if (i > first && m->ops[i - 1].defer) { const Op& bn = m->ops[i - 1]; xfv = make_xform(bn.scale, bn.offset, bn.d.act); xf = &xfv; }
+        if (i > first && m->ops[i - 1].defer) { const Op& bn = m->ops[i - 1]; xfv = make_xform(bn.mean, bn.scale, bn.offset, bn.d.act); xf = &xfv; }
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
@@ -406,9 +413,9 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
                     } else {
                         Scope sc(m, st, K_GEMM_BF16_FWD, u, i, 0, (o.in_elems + o.out_elems + o.w_cnt) * 2.0, fl);
                         bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, ar.wbt + o.w_off, out, nullptr) &&
-                                  tc_gemm_tn((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, (int)Mout, o.Co, o.C, m->tc_err, st);
+                                  tc_gemm_tn((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, m->red_scratch, (int)Mout, o.Co, o.C, m->tc_err, st);
                         if (!tc && is_3x3_op(o) && tc_conv3x3_supported(o.N, o.H, o.W, o.C, o.Co, in, ar.wbt + o.w_off, out, nullptr))
-                            tc = tc_conv3x3((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, o.N, o.H, o.W, o.C, o.Co, 0, m->tc_err, st);
+                            tc = tc_conv3x3((const T*)in, ar.wbt + o.w_off, nullptr, (T*)out, m->red_scratch, o.N, o.H, o.W, o.C, o.Co, 0, m->tc_err, st);
                         if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_FWD_BF16_SIMT;
                         if (!tc && o.d.act == FTP_ACT_NONE && o.b_off < 0) tc = stem_conv_fwd<T>((const T*)in, ar.wb + o.w_off, (T*)out, o.g, st);
                         if (!tc) conv_fwd_bf16_simt((const T*)in, ar.wb + o.w_off, o.b_off >= 0 ? ar.w + o.b_off : nullptr, (T*)out, o.g, o.d.act, st);
@@ -527,9 +534,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
         float* gr = m->grad;
         const long long Mout = (long long)o.N * o.Ho * o.Wo;
         if (gi) before_write(gi);
-        BnXform xfv{nullptr, nullptr, 0.f, 0.f};        // `in` is the input of a deferred batch norm: the weight gradient normalises as it loads
+        BnXform xfv{nullptr, nullptr, nullptr, 0.f, 0.f};        // `in` is the input of a deferred batch norm: the weight gradient normalises as it loads
         const BnXform* xf = nullptr;
-        if (i > first && m->ops[i - 1].defer) { const Op& bn = m->ops[i - 1]; xfv = make_xform(bn.scale, bn.offset, bn.d.act); xf = &xfv; }
+        if (i > first && m->ops[i - 1].defer) { const Op& bn = m->ops[i - 1]; xfv = make_xform(bn.mean, bn.scale, bn.offset, bn.d.act); xf = &xfv; }
         switch (o.d.kind) {
             case FTP_CONV1D: case FTP_CONV2D: case FTP_FC: {
                 const double fl = 2.0 * Mout * o.g.kh * o.g.kw * o.C * o.Co;
@@ -595,9 +602,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                         Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the canonical weight layout already has K = cout contiguous
                         bool tc = is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.C, o.Co, d, ar.wb + o.w_off, gi, addend) &&
-                                  tc_gemm_tn(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, (int)Mout, o.C, o.Co, m->tc_err, st);
+                                  tc_gemm_tn(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, m->red_scratch, (int)Mout, o.C, o.Co, m->tc_err, st);
                         if (!tc && is_3x3_op(o) && tc_conv3x3_supported(o.N, o.H, o.W, o.Co, o.C, d, ar.wb + o.w_off, gi, addend))
-                            tc = tc_conv3x3(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.N, o.H, o.W, o.Co, o.C, 1, m->tc_err, st);
+                            tc = tc_conv3x3(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, m->red_scratch, o.N, o.H, o.W, o.Co, o.C, 1, m->tc_err, st);
                         if (!tc && sc.slot) sc.slot->rec.kernel = K_CONV_DGRAD_BF16_SIMT;
                         if (!tc) conv_dgrad_bf16_simt(d, ar.wb + o.w_off, (const T*)addend, (T*)gi, o.g, st);
                     }

@@ -1,7 +1,7 @@
 """GPU tests of the fused routes: a batch norm that is applied by the op that reads it (never stored) against the
-same network with every batch norm stored by its own kernel.  The reader evaluates y * scale + offset with
-offset = beta - mean * scale formed in double, the stand-alone kernel ((y - mean) - mean_lo) * scale + beta: the two
-agree to float rounding, so losses, gradients, updated weights and running statistics must agree to a few 1e-6 in
+same network with every batch norm stored by its own kernel.  The reader evaluates (y - mean) * scale + offset with
+offset = beta - mean_lo * scale formed in double (mean_lo: the part of the mean that a float does not hold), the
+stand-alone kernel ((y - mean) - mean_lo) * scale + beta: the two agree to float rounding, so losses, gradients, updated weights and running statistics must agree to a few 1e-6 in
 float models; in bf16 models a value that rounds to the neighbouring bf16 number can flip an activation decision
 further on, so gradients are compared in the L2 norm there.  The oracle comparisons of the other files run on the
 default (fused) route."""
@@ -46,6 +46,29 @@ def _run(ls, cfg, idx, env, steps=2):
 # ragged on purpose: 3 x 10 x 10 = 300 rows (not a multiple of 128), 24 / 144 channels (reductions that end inside a
 # 32-wide block), a stride-2 block, a residual block
 RAGGED = dict(table=[(1, 16, 1, 1), (6, 24, 2, 1), (6, 40, 1, 2)], stem_c=32, last_c=64)
+
+
+def test_default_route_defers_batch_norms_in_float_models():
+    """The float default really takes the fused route: fewer launches per step than with every batch norm stored."""
+    ls, cfg = synth.tiny_mbv2()
+    counts = []
+    for env in ({}, {"FTP_FUSE_BN": "0"}):
+        old = os.environ.pop("FTP_FUSE_BN", None)
+        os.environ.update(env)
+        try:
+            gm = make_gpu(ls, cfg, 41)
+        finally:
+            os.environ.pop("FTP_FUSE_BN", None)
+            if old is not None:
+                os.environ["FTP_FUSE_BN"] = old
+        x, y = synth.make_batch(41, cfg)
+        xd, yd = to_dev(x), to_dev(y)
+        gm.ftp_train_step(xd, yd, 0.01)
+        n0 = gm.ftp_launch_count()
+        gm.ftp_train_step(xd, yd, 0.01)
+        counts.append(gm.ftp_launch_count() - n0)
+        gm.close()
+    assert counts[0] < counts[1], counts
 
 
 @pytest.mark.parametrize("precision", [0, 1])
