@@ -191,7 +191,7 @@ def run_reference(args, wl):
             "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
-def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=None):
+def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=None, out_bytes=None):
     """Config 5: train `steps` iterations; after every `repartition`-th the stage capacities are redrawn from U[1,10] and the
     partition re-chosen (Eq. 4 on the profiled layer times); after every `snapshot`-th each stage's weights are copied to
     the next stage's replica buffer (last stage -> central) and every stage's to the central pinned-host buffer.
@@ -216,6 +216,15 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=
     factors = rng.uniform(1.0, 10.0, n_st).tolist()              # slowdown factors of the simulated devices in the current window
     closed_loop = not on_host
     window = []
+    # Eq. 4-5 with the links this machine has: a boundary activation and its gradient cross a device-to-device copy
+    # (measured here, Sec. III-B); without the unit sizes the term is left out
+    link = None
+    if out_bytes is not None:
+        d2d, d2h = m.ftp_measure_bandwidth(central, min(64 << 20, central.numel() * 4), 5)
+        link = dict(out_bytes=[float(b) for b in out_bytes], d2d_GBps=round(d2d / 1e9, 1), d2h_GBps=round(d2h / 1e9, 1), bw=d2d)
+        log.append(dict(measured_link_bandwidth_GBps=dict(device_to_device=link["d2d_GBps"], device_to_pinned_host=link["d2h_GBps"])))
+    choose = lambda caps: F.ftp_choose_partition(layer_times, caps, link["out_bytes"] if link else None,
+                                                 [link["bw"]] * (len(caps) - 1) if link and len(caps) > 1 else None)
     if closed_loop:
         m.ftp_stage_timing_enable(True)
     replicated_at = None                 # partition under which the replicas were last written
@@ -241,7 +250,7 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=
         if fail and it + 1 == fail[0] and fail[1] < len(m.ftp_get_partition()) - 1:
             pts = m.ftp_get_partition()
             caps = [c for s, c in enumerate(last_caps[:len(pts) - 1]) if s != fail[1]]
-            new_pts, bott = F.ftp_choose_partition(layer_times, caps)
+            new_pts, bott = choose(caps)
             t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
             t0.record()
             nxt = fail[1] + 1
@@ -268,7 +277,7 @@ def run_dynamic(m, F, wl, layer_times, xd, yd, xh, yh, lr, steps, on_host, fail=
             else:
                 caps = list(factors)
             window = []
-            pts, bott = F.ftp_choose_partition(layer_times, caps)
+            pts, bott = choose(caps)
             moved = m.ftp_set_partition(pts)
             log.append(dict(after_iteration=it + 1, capacities=[round(c, 3) for c in caps], factors=[round(f, 3) for f in factors], points=pts,
                             moved_units=moved, virtual_bottleneck_ms=round(bott * 1e3, 4)))
@@ -301,11 +310,11 @@ def measure(args, wl_key, reps, steps, warmup, local_rank, replicas, batch=None,
     lr = cfg["lr"]
 
     # partition: profile -> capacities -> optimiser (or the split the workload fixes)
-    fwd_s = bwd_s = None
+    fwd_s = bwd_s = unit_bytes = None
     if points:
         wl["points"] = list(points)
     else:
-        fwd_s, bwd_s, _ = m.ftp_profile_layers(10, xd, yd)
+        fwd_s, bwd_s, unit_bytes = m.ftp_profile_layers(10, xd, yd)
     if wl["points"] is None:
         pts, _ = F.ftp_choose_partition((fwd_s + bwd_s).tolist(), wl["caps"])
     else:
@@ -352,7 +361,7 @@ def measure(args, wl_key, reps, steps, warmup, local_rank, replicas, batch=None,
         if dynamic:
             lt = (fwd_s + bwd_s).tolist()
             barrier()
-            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, steps, False, fail)
+            ms, per_it, plog = run_dynamic(m, F, wl, lt, xd, yd, xh, yh, lr, steps, False, fail, unit_bytes)
             barrier()
             blocks = [replicas.max_over_ranks(ms)]
             tick = lambda i, p: (i + 1) % p == 0

@@ -205,6 +205,15 @@ ftp_status ftp_profile_layers(ftp_model* m, int32_t reps, const void* sample_in,
 ftp_status ftp_stage_timing_enable(ftp_model* m, int32_t on);
 ftp_status ftp_stage_times(ftp_model* m, double* seconds, int32_t* n_stages);
 
+/* Sec. III-B "the i-th worker measures the bandwidth between itself and its next worker": the B_{i,i+1} of
+ * Eq. 5, as this machine has them.  Times `reps` copies of min(bytes, the model's scratch size) bytes with CUDA
+ * events: between two device buffers of the workspace (what a boundary activation or a chain replica crosses
+ * when stages share one GPU) and, if pinned_host is non-NULL (pinned host memory of at least `bytes` bytes),
+ * from the device to it (the path of the global replica to the central node).  Results in bytes per second;
+ * *d2h_bytes_per_s = 0 without a host buffer.  Synchronises the stream; call it between steps. */
+ftp_status ftp_measure_bandwidth(ftp_model* m, void* pinned_host, size_t bytes, int32_t reps, double* d2d_bytes_per_s,
+                                 double* d2h_bytes_per_s, void* stream);
+
 /* Eq. 1-3: capacities[i] = stage_times[i] / sum of layer_times over stage i; [0] = 1.0. */
 ftp_status ftp_estimate_capacity(const double* layer_times, int32_t L, const int32_t* points, int32_t N,
                                  const double* stage_times, double* capacities);

@@ -10,6 +10,8 @@
 // runs out the kernel records a code in an error word, lets its own copies land, frees its tensor memory
 // and returns; the host reports FTP_ETIMEOUT.
 #include <algorithm>
+#include <cstdlib>
+#include <cstring>
 #include "gemm_tc_common.cuh"
 
 namespace ftp {
@@ -416,6 +418,18 @@ static TnPlan plan_tn(long long tiles, int nkb, long long out_elems) {
     return pl;
 }
 
+// 128 x 256 tiles load a third less per multiply-add than 128 x 128 tiles (the products of the wide layers are bound
+// by the path from L2 to shared memory, not by the tensor pipe); taken when the output is at least 256 columns wide and
+// the wide tiles (times their reduction slices) still occupy most SMs.  FTP_TC_BN256=0 switches them off (A/B).
+static bool use_bn256(int M, int N, int K) {
+    static int on = -1;
+    if (on < 0) { const char* e = std::getenv("FTP_TC_BN256"); on = (e && std::strcmp(e, "0") == 0) ? 0 : 1; }
+    if (!on || N < 256) return false;
+    const long long tiles = (long long)((N + 255) / 256) * ((M + TC_BM - 1) / TC_BM);
+    const TnPlan pl = plan_tn(tiles, (K + TC_BK - 1) / TC_BK, (long long)M * N);
+    return tiles * pl.S >= sm_count() / 2;
+}
+
 // D = bf16(addend + sum over S float slices), slice order fixed
 __global__ void __launch_bounds__(256) slice_sum_bf16_kernel(const float4* __restrict__ part, int S, long long count4, const __nv_bfloat16* __restrict__ addend,
                                                              __nv_bfloat16* __restrict__ out) {
@@ -452,7 +466,9 @@ bool run_tn(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
     const __nv_bfloat16* addend = p.addend;
     if (pl.S > 1) { p.partial = scratch; p.kb_per_slice = pl.kbps; p.addend = nullptr; }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + TC_BM - 1) / TC_BM, pl.S);
-    const bool ok = pl.stages == 6 ? launch_tn_kernel<BN, 6>(ma, mb, md, p, grid, st) : launch_tn_kernel<BN, 3>(ma, mb, md, p, grid, st);
+    bool ok;
+    if constexpr (BN == 256) ok = launch_tn_kernel<BN, 4>(ma, mb, md, p, grid, st);              // 48 KB per stage: four fill the SM
+    else ok = pl.stages == 6 ? launch_tn_kernel<BN, 6>(ma, mb, md, p, grid, st) : launch_tn_kernel<BN, 3>(ma, mb, md, p, grid, st);
     if (ok && pl.S > 1) {
         const long long count4 = (long long)p.M * p.N / 4;
         launch(slice_sum_bf16_kernel, dim3((unsigned)((count4 + 255) / 256)), dim3(256), 0, st, reinterpret_cast<const float4*>(scratch), pl.S, count4, addend, p.D);
@@ -539,6 +555,7 @@ bool tc_conv3x3_supported(int N, int H, int W, int Ca, int No, const void* A, co
 // B = weights [9][No = cin][Ca = cout].  D (N,H,W,No) bf16.
 bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int N, int H, int W, int Ca,
                 int No, int flip, int* err, cudaStream_t st) {
+    if (use_bn256(N * H * W, No, 9 * Ca)) return launch_conv3x3<256>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
     if (No > 64) return launch_conv3x3<128>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
     if (No > 32) return launch_conv3x3<64>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
     return launch_conv3x3<32>(A, B, addend, D, scratch, N, H, W, Ca, No, flip, err, st);
@@ -546,7 +563,7 @@ bool tc_conv3x3(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloa
 
 size_t tc_gemm_scratch_floats(int M, int N, int K) {
     size_t most = 0;
-    for (int BN : {32, 64, 128}) {
+    for (int BN : {32, 64, 128, 256}) {
         const long long tiles = (long long)((N + BN - 1) / BN) * ((M + TC_BM - 1) / TC_BM);
         const TnPlan pl = plan_tn(tiles, (K + TC_BK - 1) / TC_BK, (long long)M * N);
         if (pl.S > 1) most = std::max(most, (size_t)pl.S * M * N);
@@ -588,6 +605,7 @@ bool tc_gemm_supported(int M, int N, int K, const void* A, const void* B, const 
 
 bool tc_gemm_tn(const __nv_bfloat16* A, const __nv_bfloat16* B, const __nv_bfloat16* addend, __nv_bfloat16* D, float* scratch, int M, int N, int K, int* err,
                 cudaStream_t st) {
+    if (use_bn256(M, N, K)) return launch_tn<256>(A, B, addend, D, scratch, M, N, K, err, st);
     if (N > 64) return launch_tn<128>(A, B, addend, D, scratch, M, N, K, err, st);
     if (N > 32) return launch_tn<64>(A, B, addend, D, scratch, M, N, K, err, st);
     return launch_tn<32>(A, B, addend, D, scratch, M, N, K, err, st);

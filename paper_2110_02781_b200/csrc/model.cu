@@ -1001,6 +1001,36 @@ extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t*
     return FTP_OK;
 }
 
+// Sec. III-B: every worker measures the bandwidth to its next worker (B_{i,i+1} of Eq. 5).  With all stages on one GPU
+// the "links" are copies inside device memory and, towards the central node's host copy, the path to pinned host memory.
+extern "C" ftp_status ftp_measure_bandwidth(ftp_model* m, void* pinned_host, size_t bytes, int32_t reps, double* d2d_bytes_per_s,
+                                            double* d2h_bytes_per_s, void* stream) {
+    FTP_REQUIRE(m && d2d_bytes_per_s && d2h_bytes_per_s, FTP_EINVAL, "measure_bandwidth: null argument");
+    FTP_REQUIRE(reps >= 1 && reps <= 1000 && bytes >= 4096, FTP_EINVAL, "measure_bandwidth: reps must be in 1..1000 and bytes at least 4096");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = std::min(bytes, m->red_floats * 4);          // the two reduction scratch areas are idle between steps
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    CUDA_OK(cudaEventCreate(&e0));
+    if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return fail(FTP_ECUDA, "measure_bandwidth: cudaEventCreate failed"); }
+    auto timed = [&](void* dst, const void* src, cudaMemcpyKind kind, double* out) -> ftp_status {
+        cudaError_t e = cudaMemcpyAsync(dst, src, n, kind, st);                    // warm-up
+        if (e == cudaSuccess) e = cudaEventRecord(e0, st);
+        for (int r = 0; r < reps && e == cudaSuccess; ++r) e = cudaMemcpyAsync(dst, src, n, kind, st);
+        if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+        if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+        if (e != cudaSuccess) return fail(FTP_ECUDA, "measure_bandwidth: %s", cudaGetErrorString(e));
+        *out = ms > 0.f ? (double)n * reps / (ms * 1e-3) : 0.0;
+        return FTP_OK;
+    };
+    ftp_status s = timed(m->red_side, m->red_scratch, cudaMemcpyDeviceToDevice, d2d_bytes_per_s);
+    *d2h_bytes_per_s = 0.0;
+    if (s == FTP_OK && pinned_host) s = timed(pinned_host, m->red_scratch, cudaMemcpyDeviceToHost, d2h_bytes_per_s);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    return s;
+}
+
 extern "C" ftp_status ftp_check_device_status(ftp_model* m, void* stream) {
     FTP_REQUIRE(m, FTP_EINVAL, "check_device_status: null model");
     return read_device_status(m, (cudaStream_t)stream, "check_device_status");

@@ -87,6 +87,7 @@ _SIGS = {
     "ftp_state_may_forward": [_P(TrainState), _i64, _P(_i32)],
     "ftp_state_reset": [_P(TrainState), _i64, _P(_i64)],
     "ftp_classify_probe": [_P(_i32), _i32, _P(_i32), _P(_i32), _P(_i32), _P(_i32)],
+    "ftp_measure_bandwidth": [_vp, _vp, _sz, _i32, _P(C.c_double), _P(C.c_double), _vp],
     "ftp_check_device_status": [_vp, _vp],
     "ftp_debug_set_device_status": [_vp, _i32, _vp],
     "ftp_trace_enable": [_vp, _i32],
@@ -424,6 +425,12 @@ class Model:
         _check(lib.ftp_snapshot_weights(self.h, stage, _ptr(dst), dst.numel() * dst.element_size(),
                                         int(not dst.is_cuda), C.byref(w), _stream(stream)))
         return w.value
+
+    def ftp_measure_bandwidth(self, pinned_host=None, nbytes=64 << 20, reps=5, stream=None):
+        """(device-to-device, device-to-pinned-host) copy bandwidth in bytes per second."""
+        a, b = C.c_double(), C.c_double()
+        _check(lib.ftp_measure_bandwidth(self.h, _ptr(pinned_host), nbytes, reps, C.byref(a), C.byref(b), _stream(stream)))
+        return a.value, b.value
 
     def ftp_check_device_status(self, stream=None):
         _check(lib.ftp_check_device_status(self.h, _stream(stream)))

@@ -336,3 +336,29 @@ def test_device_status_word_is_reported_and_cleared():
     ref = om.step([0, om.L], x, y)
     assert abs(got - ref) <= TOL_FP32 * abs(ref)
     gm.close()
+
+
+def test_measured_link_bandwidth_feeds_the_partition_choice():
+    """Sec. III-B / Eq. 4-5: the bandwidth between a worker and the next is measured (here: a device-to-device copy and
+    the path to pinned host memory, timed with CUDA events), and the partition optimiser takes D_j / B with those
+    numbers exactly as the oracle does."""
+    import torch
+    ls, cfg = synth.mobilenetv2(16, 32, 10, 0, True)
+    gm = make_gpu(ls, cfg, 37)
+    x, y = synth.make_batch(37, cfg)
+    f, b, ob = gm.ftp_profile_layers(3, to_dev(x), to_dev(y))
+    host = torch.empty(8 << 20, dtype=torch.uint8).pin_memory()
+    d2d, d2h = gm.ftp_measure_bandwidth(host, 8 << 20, 3)
+    assert 5e10 < d2d < 2e13 and 1e9 < d2h < 2e11, (d2d, d2h)          # device memory: tens of GB/s to TB/s; host link: GB/s
+    assert gm.ftp_measure_bandwidth(None, 1 << 20, 2)[1] == 0.0
+    with pytest.raises(F.FtpError):
+        gm.ftp_measure_bandwidth(host, 16, 1)
+    t = (f + b).tolist()
+    caps = [1.0, 2.0, 5.0, 10.0]
+    for bw in (d2d, d2h, 1e6):                                         # the last: a link slow enough that the term decides the cut
+        got = F.ftp_choose_partition(t, caps, ob.tolist(), [bw] * 3)
+        assert got == oracle.choose_partition(t, caps, [float(v) for v in ob], [bw] * 3)
+    slow, _ = F.ftp_choose_partition(t, caps, ob.tolist(), [1e6] * 3)
+    fast, _ = F.ftp_choose_partition(t, caps)
+    assert slow != fast
+    gm.close()
