@@ -330,6 +330,37 @@ ftp_status ftp_classify_probe(const int32_t* responses, int32_t n_workers, int32
 int32_t ftp_is_repartition_iter(int64_t it, int64_t first, int64_t period);
 int32_t ftp_is_replication_iter(int64_t it, int64_t period);
 
+/* ---- asynchronous pipeline training: Sec. III-C (1F1B, weight stashing, vertical sync, weight aggregation).
+ *
+ * The order of passes and the version numbers are pure host functions.  On the device a weight version of a
+ * stage is the set of parameter spans of its units inside one model object; several models built from the same
+ * layer list (each with a workspace of its own) hold the versions and the activations of the batches in flight,
+ * and the three calls below move and combine versions between them.  A driver (paper_2110_02781_b200/async_pipeline.py)
+ * strings them together with ftp_run_stage_forward / ftp_run_stage_backward. */
+
+/* 1F1B on `stage` of n_stages: the stage forwards min(n_stages - stage, n_batches) batches, then a backward and a
+ * forward pass alternate, then the remaining backward passes.  is_backward[e], batch[e] for e < 2 * n_batches. */
+ftp_status ftp_async_stage_order(int32_t n_stages, int32_t stage, int32_t n_batches, int32_t* is_backward, int32_t* batch);
+/* Version counter of a stage taken by itself (as on stage 0): starts at 0, every backward pass adds one; after the
+ * forward pass that follows every (k_interval * (n_stages - stage))-th update the n_stages - stage stashed versions
+ * are aggregated, which adds one more (no aggregation on the last stage, which has a single version).
+ * forward_version[b]: version batch b is forwarded (and, weight stashing, backwarded) with;
+ * version_after_backward[b]; aggregate_after_forward[b] = 1 where an aggregation follows F_b.  n_batches entries each. */
+ftp_status ftp_async_version_trace(int32_t n_stages, int32_t stage, int32_t n_batches, int32_t k_interval, int64_t* forward_version,
+                                   int64_t* version_after_backward, int32_t* aggregate_after_forward);
+
+/* Copy, for units [a, b), what `what` selects (a mask) from src to dst: float master weights (the copies the kernels
+ * read are rebuilt), momentum buffers, BN running statistics.  Both models must come from the same layer list.
+ * Device-to-device, asynchronous on the stream. */
+enum { FTP_SYNC_WEIGHTS = 1, FTP_SYNC_MOMENTUM = 2, FTP_SYNC_STATE = 4 };
+ftp_status ftp_sync_units(ftp_model* dst, const ftp_model* src, int32_t a, int32_t b, int32_t what, void* stream);
+/* ftp_sgd_step on dst's weights and momentum of units [a, b) with the gradients that the last backward pass of
+ * `grads` left in ITS gradient arena: the update of the latest weights by a gradient taken at stashed ones. */
+ftp_status ftp_sgd_step_from(ftp_model* dst, const ftp_model* grads, int32_t a, int32_t b, float lr, void* stream);
+/* Weight aggregation: for units [a, b), dst's master weights and BN running statistics become the arithmetic mean of
+ * those of srcs[0 .. n_src) (1..8 models, added in that order; dst may be one of them); momentum is left alone. */
+ftp_status ftp_aggregate_weights(ftp_model* dst, const ftp_model* const* srcs, int32_t n_src, int32_t a, int32_t b, void* stream);
+
 /* ---- snapshot_weights(stage, dst): Sec. III-E chain / global replication. ----------------- */
 
 /* Copy stage's replica -- per unit of the stage, in order: trainable weights then BN running

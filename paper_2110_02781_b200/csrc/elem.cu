@@ -1416,6 +1416,16 @@ __global__ void __launch_bounds__(256) sgd_kernel(float* __restrict__ w, const f
     }
 }
 
+__global__ void __launch_bounds__(256) mean_f32_kernel(MeanSources src, float* __restrict__ dst, long long count) {
+    grid_dep_sync();
+    const float inv = 1.f / (float)src.n;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x) {
+        float a = src.p[0][i];
+        for (int k = 1; k < src.n; ++k) a += src.p[k][i];
+        dst[i] = a * inv;
+    }
+}
+
 __global__ void f32_to_bf16_kernel(const float* __restrict__ s, __nv_bfloat16* __restrict__ d, long long n) {
     grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
@@ -1864,6 +1874,10 @@ void sgd_update(float* w, const float* g, float* m, long long n, float lr, float
     const bool v = n >= 4 && aligned16(w) && aligned16(g) && aligned16(m) && aligned16(lo) && aligned16(snap_dev) && aligned16(snap_host);
     if (v) launch(sgd_kernel<4>, dim3(flat_blocks(n / 4, 256)), dim3(256), 0, st, w, g, m, n / 4, (int)(n % 4), lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
     else launch(sgd_kernel<1>, dim3(flat_blocks(n, 256)), dim3(256), 0, st, w, g, m, n, 0, lr, mu, wd, first, shadow, lo, snap_dev, snap_host);
+}
+
+void mean_f32(const MeanSources& src, float* dst, long long count, cudaStream_t st) {
+    if (count > 0) launch(mean_f32_kernel, dim3(flat_blocks(count, 256)), dim3(256), 0, st, src, dst, count);
 }
 
 void tf32_lo(const float* w, float* lo, long long n, cudaStream_t st) {

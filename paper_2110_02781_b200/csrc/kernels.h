@@ -208,6 +208,9 @@ void softmax_ce(const float* logits, const int32_t* labels, int N, int classes, 
 // lo (nullable): receives w - trunc_tf32(w) of the updated weights.
 void sgd_update(float* w, const float* g, float* m, long long n, float lr, float mu, float wd, int first,
                 __nv_bfloat16* shadow, float* lo, float* snap_dev, float* snap_host, cudaStream_t st);
+// dst = arithmetic mean of n (1..8) arrays, added in the order given
+struct MeanSources { const float* p[8]; int n; };
+void mean_f32(const MeanSources& src, float* dst, long long count, cudaStream_t st);
 void tf32_lo(const float* w, float* lo, long long n, cudaStream_t st);                   // lo = w - trunc_tf32(w)
 // Batched transposition of float matrices: entry e describes a [K][N] matrix at w + w_off whose transpose goes to
 // wt + w_off ([N][K]) and the lo part of the transpose to wtl + w_off.  table: n + 1 device entries (the last one

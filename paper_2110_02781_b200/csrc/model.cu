@@ -1188,6 +1188,83 @@ extern "C" ftp_status ftp_set_partition(ftp_model* m, const int32_t* points, int
     return FTP_OK;
 }
 
+// ---- asynchronous pipeline training (Sec. III-C): weight versions live in models of the same architecture ----------
+static ftp_status same_architecture(const ftp_model* a, const ftp_model* b, const char* who) {
+    FTP_REQUIRE(a && b, FTP_EINVAL, "%s: null model", who);
+    FTP_REQUIRE(a->L == b->L && a->P == b->P && a->R == b->R && a->cfg.precision == b->cfg.precision && a->unit_p_off == b->unit_p_off &&
+                a->unit_s_off == b->unit_s_off, FTP_EINVAL, "%s: the models were not built from the same layer list", who);
+    return FTP_OK;
+}
+
+// after the float masters of units [a, b) changed: the copies the kernels read (bf16 shadow, tf32 lo part, transposes)
+static void refresh_derived(ftp_model* m, int a, int b, cudaStream_t st) {
+    for (int u = a; u < b; ++u) {
+        const Arena& ar = m->arena[m->owner[u]];
+        const long long po = m->unit_p_off[u], pc = m->unit_p_cnt[u];
+        if (!pc) continue;
+        if (ar.wb) f32_to_bf16(ar.w + po, ar.wb + po, pc, st);
+        if (ar.wl) tf32_lo(ar.w + po, ar.wl + po, pc, st);
+    }
+    refresh_transposed(m, a, b, st);
+}
+
+extern "C" ftp_status ftp_sync_units(ftp_model* dst, const ftp_model* src, int32_t a, int32_t b, int32_t what, void* stream) {
+    ftp_status s = same_architecture(dst, src, "sync_units");
+    if (s == FTP_OK) s = check_range(dst, a, b, "sync_units");
+    if (s != FTP_OK) return s;
+    FTP_REQUIRE(what > 0 && what < 8, FTP_EINVAL, "sync_units: `what` is a mask of FTP_SYNC_WEIGHTS, FTP_SYNC_MOMENTUM, FTP_SYNC_STATE");
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int u = a; u < b; ++u) {
+        const Arena& to = dst->arena[dst->owner[u]];
+        const Arena& from = src->arena[src->owner[u]];
+        const long long po = dst->unit_p_off[u], pc = dst->unit_p_cnt[u], so = dst->unit_s_off[u], sc_ = dst->unit_s_cnt[u];
+        if ((what & FTP_SYNC_WEIGHTS) && pc) CUDA_OK(cudaMemcpyAsync(to.w + po, from.w + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+        if ((what & FTP_SYNC_MOMENTUM) && pc) {
+            CUDA_OK(cudaMemcpyAsync(to.m + po, from.m + po, (size_t)pc * 4, cudaMemcpyDeviceToDevice, st));
+            dst->mom_init[u] = src->mom_init[u];
+        }
+        if ((what & FTP_SYNC_STATE) && sc_) CUDA_OK(cudaMemcpyAsync(to.run + so, from.run + so, (size_t)sc_ * 4, cudaMemcpyDeviceToDevice, st));
+    }
+    if (what & FTP_SYNC_WEIGHTS) refresh_derived(dst, a, b, st);
+    return check_launches("sync_units");
+}
+
+extern "C" ftp_status ftp_sgd_step_from(ftp_model* dst, const ftp_model* grads, int32_t a, int32_t b, float lr, void* stream) {
+    ftp_status s = same_architecture(dst, grads, "sgd_step_from");
+    if (s == FTP_OK) s = check_range(dst, a, b, "sgd_step_from");
+    if (s == FTP_OK) s = pending_status(dst, "sgd_step_from");
+    if (s != FTP_OK) return s;
+    float* own = dst->grad;
+    dst->grad = grads->grad;                               // the update reads the gradients the other model's backward pass left
+    s = sgd_range(dst, a, b, lr, nullptr, nullptr, (cudaStream_t)stream);
+    dst->grad = own;
+    return s;
+}
+
+extern "C" ftp_status ftp_aggregate_weights(ftp_model* dst, const ftp_model* const* srcs, int32_t n_src, int32_t a, int32_t b, void* stream) {
+    FTP_REQUIRE(dst && srcs, FTP_EINVAL, "aggregate_weights: null argument");
+    FTP_REQUIRE(n_src >= 1 && n_src <= 8, FTP_ERANGE, "aggregate_weights: 1 to 8 versions can be aggregated, not %d", n_src);
+    ftp_status s = check_range(dst, a, b, "aggregate_weights");
+    for (int k = 0; k < n_src && s == FTP_OK; ++k) s = same_architecture(dst, srcs[k], "aggregate_weights");
+    if (s != FTP_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int u = a; u < b; ++u) {
+        const Arena& to = dst->arena[dst->owner[u]];
+        MeanSources w{}, r{};
+        w.n = r.n = n_src;
+        for (int k = 0; k < n_src; ++k) {
+            const Arena& from = srcs[k]->arena[srcs[k]->owner[u]];
+            w.p[k] = from.w + dst->unit_p_off[u];
+            r.p[k] = from.run + dst->unit_s_off[u];
+        }
+        Scope sc(dst, st, K_SGD, u, -1, 2, (double)(dst->unit_p_cnt[u] + dst->unit_s_cnt[u]) * 4.0 * (n_src + 1), (double)(dst->unit_p_cnt[u] + dst->unit_s_cnt[u]) * n_src, 2);
+        mean_f32(w, to.w + dst->unit_p_off[u], dst->unit_p_cnt[u], st);
+        mean_f32(r, to.run + dst->unit_s_off[u], dst->unit_s_cnt[u], st);
+    }
+    refresh_derived(dst, a, b, st);
+    return check_launches("aggregate_weights");
+}
+
 extern "C" ftp_status ftp_get_partition(const ftp_model* m, int32_t* points, int32_t* n_stages) {
     FTP_REQUIRE(m && points && n_stages, FTP_EINVAL, "get_partition: null argument");
     for (int i = 0; i <= m->n_stages; ++i) points[i] = m->points[i];

@@ -2,6 +2,7 @@
 // and the weight-redistribution plan (Algorithm 1).  No GPU involved.
 #include <cstring>
 #include <limits>
+#include <algorithm>
 #include <vector>
 #include "common.h"
 
@@ -224,4 +225,49 @@ extern "C" int32_t ftp_is_repartition_iter(int64_t it, int64_t first, int64_t pe
 // Sec. IV-B / IV-E: a replication runs when a batch whose 1-indexed count is a multiple of the period has finished.
 extern "C" int32_t ftp_is_replication_iter(int64_t it, int64_t period) {
     return (period > 0 && it + 1 > 0 && (it + 1) % period == 0) ? 1 : 0;
+}
+
+// ---- asynchronous pipeline schedule (Sec. III-C): order of passes and weight-version numbers on one stage --------
+extern "C" ftp_status ftp_async_stage_order(int32_t n_stages, int32_t stage, int32_t n_batches, int32_t* is_backward, int32_t* batch) {
+    FTP_REQUIRE(is_backward && batch, FTP_EINVAL, "async_stage_order: null output");
+    FTP_REQUIRE(n_stages >= 1 && stage >= 0 && stage < n_stages && n_batches >= 0, FTP_EINVAL, "async_stage_order: need 0 <= stage < n_stages and n_batches >= 0");
+    const int32_t warm = std::min(n_stages - stage, n_batches);
+    int32_t k = 0, nf = warm, nb = 0;
+    for (int32_t b = 0; b < warm; ++b) { is_backward[k] = 0; batch[k++] = b; }
+    while (nb < n_batches) {
+        is_backward[k] = 1; batch[k++] = nb++;
+        if (nf < n_batches) { is_backward[k] = 0; batch[k++] = nf++; }
+    }
+    return FTP_OK;
+}
+
+extern "C" ftp_status ftp_async_version_trace(int32_t n_stages, int32_t stage, int32_t n_batches, int32_t k_interval, int64_t* forward_version,
+                                              int64_t* version_after_backward, int32_t* aggregate_after_forward) {
+    FTP_REQUIRE(forward_version && version_after_backward && aggregate_after_forward, FTP_EINVAL, "async_version_trace: null output");
+    FTP_REQUIRE(n_stages >= 1 && stage >= 0 && stage < n_stages && n_batches >= 0 && k_interval >= 1, FTP_EINVAL,
+                "async_version_trace: need 0 <= stage < n_stages, n_batches >= 0, k >= 1");
+    std::vector<int32_t> isb(2 * (size_t)n_batches + 1), bat(2 * (size_t)n_batches + 1);
+    ftp_status s = ftp_async_stage_order(n_stages, stage, n_batches, isb.data(), bat.data());
+    if (s != FTP_OK) return s;
+    const int64_t c = n_stages - stage;
+    int64_t ver = 0, updates = 0, done_at = 0, in_flight = 0;
+    for (int32_t b = 0; b < n_batches; ++b) aggregate_after_forward[b] = 0;
+    for (int32_t e = 0; e < 2 * n_batches; ++e) {
+        const int32_t b = bat[e];
+        if (!isb[e]) {
+            forward_version[b] = ver;
+            ++in_flight;
+            if (c > 1 && updates > 0 && updates % (k_interval * c) == 0 && updates != done_at && in_flight == c) {
+                ++ver;                                       // the n - i stashed versions are aggregated: one more version
+                done_at = updates;
+                aggregate_after_forward[b] = 1;
+            }
+        } else {
+            --in_flight;
+            ++ver;
+            ++updates;
+            version_after_backward[b] = ver;
+        }
+    }
+    return FTP_OK;
 }

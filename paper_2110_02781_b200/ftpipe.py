@@ -87,6 +87,11 @@ _SIGS = {
     "ftp_state_may_forward": [_P(TrainState), _i64, _P(_i32)],
     "ftp_state_reset": [_P(TrainState), _i64, _P(_i64)],
     "ftp_classify_probe": [_P(_i32), _i32, _P(_i32), _P(_i32), _P(_i32), _P(_i32)],
+    "ftp_async_stage_order": [_i32, _i32, _i32, _P(_i32), _P(_i32)],
+    "ftp_async_version_trace": [_i32, _i32, _i32, _i32, _P(_i64), _P(_i64), _P(_i32)],
+    "ftp_sync_units": [_vp, _vp, _i32, _i32, _i32, _vp],
+    "ftp_sgd_step_from": [_vp, _vp, _i32, _i32, _f32, _vp],
+    "ftp_aggregate_weights": [_vp, _P(_vp), _i32, _i32, _i32, _vp],
     "ftp_measure_bandwidth": [_vp, _vp, _sz, _i32, _P(C.c_double), _P(C.c_double), _vp],
     "ftp_check_device_status": [_vp, _vp],
     "ftp_debug_set_device_status": [_vp, _i32, _vp],
@@ -252,6 +257,34 @@ def ftp_is_repartition_iter(it, first=10, period=100):
 
 def ftp_is_replication_iter(it, period):
     return bool(lib.ftp_is_replication_iter(it, period))
+
+
+SYNC_WEIGHTS, SYNC_MOMENTUM, SYNC_STATE = 1, 2, 4
+
+
+def ftp_async_stage_order(n_stages, stage, n_batches):
+    isb, bat = (_i32 * (2 * n_batches + 1))(), (_i32 * (2 * n_batches + 1))()
+    _check(lib.ftp_async_stage_order(n_stages, stage, n_batches, isb, bat))
+    return [("B" if isb[e] else "F", bat[e]) for e in range(2 * n_batches)]
+
+
+def ftp_async_version_trace(n_stages, stage, n_batches, k=1):
+    fv, av, ag = (_i64 * max(n_batches, 1))(), (_i64 * max(n_batches, 1))(), (_i32 * max(n_batches, 1))()
+    _check(lib.ftp_async_version_trace(n_stages, stage, n_batches, k, fv, av, ag))
+    return list(fv[:n_batches]), list(av[:n_batches]), [b for b in range(n_batches) if ag[b]]
+
+
+def ftp_sync_units(dst, src, a, b, what, stream=None):
+    _check(lib.ftp_sync_units(dst.h, src.h, a, b, what, _stream(stream)))
+
+
+def ftp_sgd_step_from(dst, grads, a, b, lr, stream=None):
+    _check(lib.ftp_sgd_step_from(dst.h, grads.h, a, b, lr, _stream(stream)))
+
+
+def ftp_aggregate_weights(dst, srcs, a, b, stream=None):
+    arr = (_vp * len(srcs))(*[m.h for m in srcs])
+    _check(lib.ftp_aggregate_weights(dst.h, arr, len(srcs), a, b, _stream(stream)))
 
 
 def ftp_workspace_bytes(layers, cfg):
