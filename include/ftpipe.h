@@ -182,6 +182,11 @@ ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, in
 /* Waits for the stream, reads the device status word (see "Errors" above) and clears it:
  * FTP_OK, or FTP_ETIMEOUT if a bounded device-side wait ran out since the last check. */
 ftp_status ftp_check_device_status(ftp_model* m, void* stream);
+/* Memory-safety check (the workspace's stand-in for a memory checker): every buffer the model carves out of dev_ws is
+ * followed by a 256-byte guard zone holding a fixed pattern since ftp_build_model.  Waits for the stream, reads all
+ * zones back and returns FTP_ESTATE (text: which zone, at which workspace offset) if a kernel has written past the end
+ * of a buffer; *first_bad_offset (nullable) = that offset or -1, *n_guards (nullable) = zones checked. */
+ftp_status ftp_check_guards(ftp_model* m, int32_t* n_guards, int64_t* first_bad_offset, void* stream);
 /* Test hook: writes `code` into the device status word from the host, as a kernel whose wait ran
  * out would (0 clears it).  No kernel is launched.  Synchronises the stream. */
 ftp_status ftp_debug_set_device_status(ftp_model* m, int32_t code, void* stream);

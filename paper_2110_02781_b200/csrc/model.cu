@@ -16,13 +16,21 @@ static long long g_launches = 0;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Every buffer carved out of the workspace is followed by a 256-byte guard zone filled with a pattern when the model is
+// built; ftp_check_guards finds a kernel that wrote past the end of its buffer (the stand-in for a memory checker).
+constexpr size_t kGuardBytes = 256;
+constexpr unsigned char kGuardByte = 0xA5;
 struct Bump {
     char* base;
     size_t off;
+    std::vector<size_t>* guards;          // offsets of the guard zones (nullable)
     void* take(size_t bytes) {
         off = align_up(off, 256);
         void* p = base ? base + off : reinterpret_cast<void*>(off + 256);   // dry run: fake, never dereferenced
         off += bytes;
+        off = align_up(off, 256);
+        if (guards) guards->push_back(off);
+        off += kGuardBytes;
         return p;
     }
 };
@@ -227,7 +235,8 @@ ftp_status plan_gradients(ftp_model& m, int* n_slots) {
 
 // ---- memory layout inside the workspace --------------------------------------------------------------
 ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinned_total) {
-    Bump bp{dev_base, 0};
+    m.guards.clear();
+    Bump bp{dev_base, 0, &m.guards};
     const int n = (int)m.ops.size();
     const size_t es = (size_t)m.esize;
     m.arena.assign(m.cfg.max_stages, Arena{});
@@ -778,6 +787,13 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         s = fail(FTP_ENOMEM, "build_model: workspace too small (need %zu device and %zu pinned bytes)", need, pneed);
     if (s != FTP_OK) { delete m; return s; }
     m->pinned = (float*)pinned_ws; m->pinned_bytes = pinned_bytes;
+    m->ws_base = (char*)dev_ws;
+    for (size_t off : m->guards)
+        if (cudaMemset(m->ws_base + off, kGuardByte, kGuardBytes) != cudaSuccess) {
+            const ftp_status e = fail(FTP_ECUDA, "build_model: filling the guard zones failed: %s", cudaGetErrorString(cudaGetLastError()));
+            delete m;
+            return e;
+        }
     std::memset(m->pinned, 0, 16);                            // loss, status words
     if (cudaMemset(m->fin.counters, 0, m->fin_counter_bytes) != cudaSuccess || cudaMemset(m->fin_side.counters, 0, m->fin_counter_bytes) != cudaSuccess ||
         cudaMemset(m->tc_err, 0, 256) != cudaSuccess) {     // ticket counters start at zero
@@ -1029,6 +1045,25 @@ extern "C" ftp_status ftp_measure_bandwidth(ftp_model* m, void* pinned_host, siz
     if (s == FTP_OK && pinned_host) s = timed(pinned_host, m->red_scratch, cudaMemcpyDeviceToHost, d2h_bytes_per_s);
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     return s;
+}
+
+extern "C" ftp_status ftp_check_guards(ftp_model* m, int32_t* n_guards, int64_t* first_bad_offset, void* stream) {
+    FTP_REQUIRE(m, FTP_EINVAL, "check_guards: null model");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaStreamSynchronize(st));
+    if (n_guards) *n_guards = (int32_t)m->guards.size();
+    if (first_bad_offset) *first_bad_offset = -1;
+    unsigned char buf[kGuardBytes];
+    for (size_t k = 0; k < m->guards.size(); ++k) {
+        CUDA_OK(cudaMemcpy(buf, m->ws_base + m->guards[k], kGuardBytes, cudaMemcpyDeviceToHost));
+        for (size_t i = 0; i < kGuardBytes; ++i)
+            if (buf[i] != kGuardByte) {
+                if (first_bad_offset) *first_bad_offset = (int64_t)(m->guards[k] + i);
+                return fail(FTP_ESTATE, "check_guards: guard zone %zu of %zu was overwritten at workspace offset %zu: a kernel wrote past the end of the buffer before it",
+                            k, m->guards.size(), m->guards[k] + i);
+            }
+    }
+    return FTP_OK;
 }
 
 extern "C" ftp_status ftp_check_device_status(ftp_model* m, void* stream) {

@@ -81,6 +81,7 @@ struct ftp_model {
     float* fc_in; float* fc_din;                  // bf16 models: the classifier's input and input gradient widened to float
     float* dlogits; float* per_sample; float* loss_dev; int32_t* labels_dev; void* input_dev; float* state_backup;
     float* pinned; size_t pinned_bytes;
+    char* ws_base; std::vector<size_t> guards;    // device workspace and the offsets of its guard zones
     // run-time state of the last forward of each range
     std::vector<const void*> stage_in;            // act_in of the range starting at op i
     std::vector<void*> cur_out;                   // resolved output pointer of op i

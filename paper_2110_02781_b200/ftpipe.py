@@ -93,6 +93,7 @@ _SIGS = {
     "ftp_sgd_step_from": [_vp, _vp, _i32, _i32, _f32, _vp],
     "ftp_aggregate_weights": [_vp, _P(_vp), _i32, _i32, _i32, _vp],
     "ftp_measure_bandwidth": [_vp, _vp, _sz, _i32, _P(C.c_double), _P(C.c_double), _vp],
+    "ftp_check_guards": [_vp, _P(_i32), _P(_i64), _vp],
     "ftp_check_device_status": [_vp, _vp],
     "ftp_debug_set_device_status": [_vp, _i32, _vp],
     "ftp_trace_enable": [_vp, _i32],
@@ -464,6 +465,16 @@ class Model:
         a, b = C.c_double(), C.c_double()
         _check(lib.ftp_measure_bandwidth(self.h, _ptr(pinned_host), nbytes, reps, C.byref(a), C.byref(b), _stream(stream)))
         return a.value, b.value
+
+    def ftp_check_guards(self, stream=None):
+        """Number of guard zones checked; raises FtpError (with .bad_offset) if one was overwritten."""
+        n, bad = _i32(), _i64()
+        st = lib.ftp_check_guards(self.h, C.byref(n), C.byref(bad), _stream(stream))
+        if st != OK:
+            e = FtpError(st, lib.ftp_last_error().decode())
+            e.bad_offset = bad.value
+            raise e
+        return n.value
 
     def ftp_check_device_status(self, stream=None):
         _check(lib.ftp_check_device_status(self.h, _stream(stream)))

@@ -362,3 +362,47 @@ def test_measured_link_bandwidth_feeds_the_partition_choice():
     fast, _ = F.ftp_choose_partition(t, caps)
     assert slow != fast
     gm.close()
+
+
+def test_guard_zones_stay_intact_on_ragged_shapes_and_catch_a_planted_overwrite():
+    """Every buffer of the workspace ends in a guard zone.  After training steps on shapes with ragged tails (row counts
+    off the 128-row tiles, channel counts off the vector widths, odd maps) in both precisions every zone still holds its
+    pattern; a byte changed from the host inside one zone (no kernel misbehaves) is found and located."""
+    import torch
+    L, K, A = synth.Layer, synth.KIND, synth.ACT
+    odd = [L(0, K["CONV2D"], 3, 6, 3, 1, 1, 0, 0, -1), L(0, K["BN"], 6, 6, 0, 1, 0, A["RELU6"], 0, -1),
+           L(1, K["DWCONV3x3"], 6, 6, 3, 2, 1, 0, 0, -1), L(1, K["BN"], 6, 6, 0, 1, 0, A["RELU"], 0, -1),
+           L(1, K["CONV2D"], 6, 10, 1, 1, 0, A["RELU"], 1, -1), L(2, K["MAXPOOL2"], 10, 10, 2, 2, 0, 0, 0, -1),
+           L(2, K["GAP"], 10, 10, 0, 1, 0, 0, 0, -1), L(2, K["FC"], 10, 7, 1, 1, 0, 0, 1, -1), L(2, K["SOFTMAX_CE"], 7, 7, 0, 1, 0, 0, 0, -1)]
+    nets = [synth.mobilenetv2(3, 10, 7, 0, True, table=[(1, 16, 1, 1), (6, 24, 2, 1), (6, 40, 1, 2)], stem_c=32, last_c=64),
+            synth.mobilenetv2(3, 10, 7, 1, True, table=[(1, 16, 1, 1), (6, 24, 2, 1), (6, 40, 1, 2)], stem_c=32, last_c=64),
+            synth.mobilenetv2(5, 9, 5, 0, False, table=[(1, 8, 1, 1), (6, 16, 1, 2)], stem_c=32, last_c=32),
+            synth.tiny_vgg(batch=6, hw=4, precision=1), synth.har_cnn(5, 9, 131, 20, 6), (odd, synth.config(3, 3, 5, 5, 7, momentum=0.9))]
+    for ls, cfg in nets:
+        gm = make_gpu(ls, cfg, 38)
+        x, y = synth.make_batch(38, cfg)
+        xd = to_dev(x, torch.bfloat16 if cfg["precision"] == 1 else None)
+        yd = to_dev(y)
+        if gm.L >= 3:
+            gm.ftp_set_partition([0, 1, gm.L])
+        for _ in range(2):
+            gm.ftp_train_step(xd, yd, 0.01)
+        gm.ftp_profile_layers(1, xd, yd)
+        assert gm.ftp_check_guards() > 20
+        gm.close()
+    ls, cfg = synth.tiny_mbv2()
+    gm = make_gpu(ls, cfg, 38)
+    n = gm.ftp_check_guards()
+    base = (gm.dev_ws.data_ptr() + 255) // 256 * 256 - gm.dev_ws.data_ptr()
+    # find a guard zone from the host: the first 256-byte run of the pattern after the first buffer
+    ws = gm.dev_ws[base:base + (1 << 20)].cpu().numpy()
+    runs = np.flatnonzero((ws.reshape(-1, 256) == 0xA5).all(axis=1))
+    assert runs.size > 0
+    off = int(runs[0]) * 256 + 17
+    gm.dev_ws[base + off] = 0                                            # planted from the host
+    with pytest.raises(F.FtpError) as e:
+        gm.ftp_check_guards()
+    assert e.value.status == 5 and e.value.bad_offset == off
+    gm.dev_ws[base + off] = 0xA5
+    assert gm.ftp_check_guards() == n
+    gm.close()
