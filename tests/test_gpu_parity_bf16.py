@@ -292,3 +292,88 @@ def test_bf16_path_against_the_float64_oracle(name, record_property):
     for u in units:
         assert e_dev[u][0] <= e_fmt[u][0] + TOL_BF16 and e_dev[u][1] <= e_fmt[u][1] + TOL_BF16, (u, report)
     gm.close()
+
+
+# ---- config 4 at its full size, one unit at a time, backward included: every gradient at the max-abs tolerance ------
+def _vgg_units():
+    ls, cfg = synth.vgg16(256, 32, 10, 1)
+    return list(range(synth.num_units(ls) - 1))
+
+
+@pytest.mark.parametrize("u", _vgg_units())
+def test_full_size_vgg16_unit_forward_and_backward(u):
+    """Unit u of the VGG-16-style network at batch 256 ([3x3 convolution, BN + ReLU] and, where the group closes, the
+    2x2 max-pool), fed the input that unit has in the chained oracle run with the real initialisation, and a seeded
+    incoming gradient that is zero wherever the oracle's decision is within bf16 reach of flipping (a pre-activation
+    within 2e-2 of the ReLU kink, a pool window whose two largest values lie within 2e-2, a pool window that holds such
+    a pre-activation).  What is compared is then unique: output, input gradient, dW, dgamma, dbeta, running statistics,
+    each at 2e-2 max-abs."""
+    import torch
+    from oracle.model import round_bf16
+    ls, cfg = synth.vgg16(256, 32, 10, 1)
+    K = synth.KIND
+    ops = [i for i, l in enumerate(ls) if l.unit == u]
+    om = oracle.OracleModel(ls, cfg, synth.init_params(3, ls), synth.init_state(ls))
+    x, y = synth.make_batch(3, cfg)
+    act = round_bf16(x)
+    for v in range(u):                                        # the chained run up to this unit (forward only)
+        act = om.forward(v, v + 1, act)
+    out = om.forward(u, u + 1, act)
+    bn = next(i for i in ops if ls[i].kind == K["BN"])
+    amb = om.ambiguous_outputs(bn, 2e-2)
+    if ls[ops[-1]].kind == K["MAXPOOL2"]:
+        n, h, w, c = amb.shape
+        amb = amb.reshape(n, h // 2, 2, w // 2, 2, c).any(axis=(2, 4)) | om.ambiguous_outputs(ops[-1], 2e-2)
+    g = synth.rng_stream(71 + u, "misc")
+    gout = round_bf16(g.standard_normal(out.shape) / out[0].size)
+    gout[amb] = 0.0
+    dxref = om.backward(u, u + 1, gout)
+    gm = F.Model(ls, cfg)
+    gm.load_params(synth.init_params(3, ls), synth.init_state(ls))
+    xd, gd = dev_bf16(act), dev_bf16(gout)
+    yd = torch.empty(out.shape, dtype=torch.bfloat16, device="cuda")
+    dxd = torch.empty(act.shape, dtype=torch.bfloat16, device="cuda")
+    gm.ftp_run_stage_forward(u, u + 1, xd, yd)
+    gm.ftp_run_stage_backward(u, u + 1, gd, dxd)
+    torch.cuda.synchronize()
+    assert rel_err(host(yd), out) <= TOL_BF16
+    assert rel_err(host(dxd), dxref) <= TOL_BF16, f"input gradient: {rel_err(host(dxd), dxref):.3e}"
+    got, ref = gm.ftp_get_tensor(F.T_GRADS, u), om.unit_grads(u)
+    cout = ls[ops[0]].cout
+    nW = ref.size - 2 * cout
+    for name, sl in (("dW", slice(0, nW)), ("dgamma", slice(nW, nW + cout)), ("dbeta", slice(nW + cout, nW + 2 * cout))):
+        e = rel_err(got[sl], ref[sl])
+        assert e <= TOL_BF16, f"{name}: {e:.3e}"
+    assert rel_err(gm.ftp_get_tensor(F.T_STATE, u), om.unit_state(u)) <= TOL_BF16
+    gm.close()
+
+
+def test_mobilenet_224_batch_64_first_units():
+    """Config 3 at its full batch of 64: the first three units (first convolution, the expand-1 block, the first
+    stride-2 block at 112 x 112), one at a time to keep the float64 oracle's memory in bounds, each fed the oracle's
+    input of that unit: output and BN running statistics at the bf16 tolerance (max-abs) and 1e-3 in L2."""
+    import gc
+    import torch
+    from oracle.model import round_bf16
+    ls, cfg = synth.mobilenetv2(64, 224, 1000, 1, False)
+    om = oracle.OracleModel(ls, cfg, synth.init_params(2, ls), synth.init_state(ls))
+    gm = F.Model(ls, dict(cfg, max_stages=5))
+    gm.load_params(synth.init_params(2, ls), synth.init_state(ls))
+    x, _ = synth.make_batch(2, cfg)
+    act = round_bf16(x)
+    for u in range(3):
+        ref = om.forward(u, u + 1, act)
+        shp, _ = gm.ftp_unit_output_shape(u)
+        out = torch.empty(shp, dtype=torch.bfloat16, device="cuda")
+        xd = dev_bf16(act)
+        gm.ftp_run_stage_forward(u, u + 1, xd, out)
+        torch.cuda.synchronize()
+        got = host(out)
+        assert rel_err(got, ref) <= TOL_BF16, f"unit {u}"
+        assert l2_err(got, ref) <= 1e-3, f"unit {u} (L2)"
+        assert rel_err(gm.ftp_get_tensor(F.T_STATE, u), om.unit_state(u)) <= TOL_BF16, f"running statistics of unit {u}"
+        act = ref
+        om.out.clear(); om.saved.clear()
+        del got, out, xd
+        gc.collect()
+    gm.close()
