@@ -1106,13 +1106,20 @@ __global__ void __launch_bounds__(256, XF ? 1 : 2) dw3_fwd_rows_kernel(const T* 
 // order of dw_strip_kernel<FLIP = 1>) and adds x[pixel] * dy[pixel + offset] to the nine weight-gradient sums of its
 // four channels, which it carries down its rows.  At the end the 32 slots of a block are added in slot order:
 // partial[blockIdx.x][9][C] (float), summed over blocks by the finalize kernels.  dx may be NULL (no input gradient).
-template <typename T, bool XF>
+// BST (with XF): x is the input of the batch norm that precedes this convolution, so dx is the gradient with respect to
+// that batch norm's output: it is stored already masked by the batch norm's activation, and the block leaves the two sums
+// of the batch norm's backward pass (of g and of g * xhat, g as stored) in bstats[blockIdx.x][2][C] -- the separate
+// reduction pass over (dx, x) is not needed.
+template <typename T, bool XF, bool BST>
 __global__ void __launch_bounds__(256) dw3_bwd_rows_kernel(const T* __restrict__ x, const T* __restrict__ dy, const float* __restrict__ w,
                                                            const T* __restrict__ addend, T* __restrict__ dx, float* __restrict__ partial, int N, int H,
-                                                           int W, int C, int RH, int HC, BnXform xf) {
+                                                           int W, int C, int RH, int HC, BnXform xf, const float* __restrict__ rstd,
+                                                           double* __restrict__ bstats) {
+    static_assert(!BST || XF, "the backward sums need the batch norm's input");
     grid_dep_sync();
     __shared__ __align__(16) float wsm[9][32];
     __shared__ float sh[3][32][33];
+    float bs1[4] = {0.f, 0.f, 0.f, 0.f}, bs2[4] = {0.f, 0.f, 0.f, 0.f};
     const int CV = C / 4, cvl = threadIdx.x & 7, slot = threadIdx.x >> 3, cv = blockIdx.y * 8 + cvl, c = cv * 4;
     for (int i = threadIdx.x; i < 9 * 32; i += 256) {
         const int tap = i >> 5, ch = blockIdx.y * 32 + (i & 31);
@@ -1133,6 +1140,8 @@ __global__ void __launch_bounds__(256) dw3_bwd_rows_kernel(const T* __restrict__
         const int w0 = sw * 4, h0 = hc * RH, h1 = min(H, h0 + RH);
         XfRegs<T, 4> xr, none;
         if constexpr (XF) xr.load(xf, c);
+        float rs[4] = {0.f, 0.f, 0.f, 0.f};
+        if constexpr (BST) ldtab<4>(rstd + c, rs);
         const long long ioff = (long long)n * H * W * C + c;
         const T* gimg = dy + ioff;
         float win[3][6][4];
@@ -1152,12 +1161,26 @@ __global__ void __launch_bounds__(256) dw3_bwd_rows_kernel(const T* __restrict__
         };
         fetch_x(h0);
         for (int h = h0; h < h1; ++h) {
-            float xv[4][4], acc[4][4];
+            float xv[4][4], acc[4][4], xh[BST ? 4 : 1][4];
+            unsigned pass = 0u;                                  // bit 4 j + e: the activation lets the gradient through
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) { xv[j][e] = xnext[j][e]; acc[j][e] = 0.f; }
-                if constexpr (XF) { if (w0 + j < W) xr.apply(xv[j]); }
+                if constexpr (BST) {
+                    if (w0 + j < W) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float cen = xv[j][e] - xr.mu[e], z = fmaf(cen, xr.sc[e], xr.of[e]);
+                            xh[j][e] = cen * rs[e];
+                            if (z > xr.lo && z < xr.hi) pass |= 1u << (4 * j + e);
+                            xv[j][e] = as_stored<T>(fminf(fmaxf(z, xr.lo), xr.hi));
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) xh[j][e] = 0.f;
+                    }
+                } else if constexpr (XF) { if (w0 + j < W) xr.apply(xv[j]); }
             }
             if (h + 1 < h1) fetch_x(h + 1);                      // lands while this row is computed
 #pragma unroll
@@ -1192,9 +1215,34 @@ __global__ void __launch_bounds__(256) dw3_bwd_rows_kernel(const T* __restrict__
 #pragma unroll
                             for (int e = 0; e < 4; ++e) acc[j][e] += a[e];
                         }
+                        if constexpr (BST) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float gq = (pass >> (4 * j + e)) & 1u ? as_stored<T>(acc[j][e]) : 0.f;
+                                acc[j][e] = gq;
+                                bs1[e] += gq;
+                                bs2[e] = fmaf(gq, xh[j][e], bs2[e]);
+                            }
+                        }
                         stv<4>(dx + o, acc[j]);
                     }
                 }
+            }
+        }
+    }
+    if constexpr (BST) {
+        // the two sums of every channel over the block's 32 slots, in slot order, as doubles
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { sh[0][slot][cvl * 4 + e] = bs1[e]; sh[1][slot][cvl * 4 + e] = bs2[e]; }
+        __syncthreads();
+        if (threadIdx.x < 64) {
+            const int a = threadIdx.x >> 5, ch = threadIdx.x & 31, gc = blockIdx.y * 32 + ch;
+            if (gc < C) {
+                double tsum = 0.0;
+#pragma unroll 8
+                for (int q = 0; q < 32; ++q) tsum += (double)sh[a][q][ch];
+                bstats[((long long)blockIdx.x * 2 + a) * C + gc] = tsum;
             }
         }
     }
@@ -1811,17 +1859,26 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
     else launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, fin_slices(fp), 9), dim3(FIN_X, FIN_Y), 0, st, scratch, fp.chunks, fp.f, g.Cin, fp.cols, dw, fin);
 }
 
+size_t dwconv_bwd_stats_doubles(const ConvGeom& g) {
+    return g.Cin % 4 == 0 && g.stride == 1 ? (size_t)plan_dw3(g, sm_count()).gx * 2 * g.Cin : 0;
+}
+
 template <typename T>
 bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
-                      cudaStream_t st, const BnXform* x_xform) {
+                      cudaStream_t st, const BnXform* x_xform, const BnBwdSumsReq* sums) {
     const bool xf = x_xform != nullptr;
     const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f};
     const bool xf_vec = !xf || (aligned16(xv.mean) && aligned16(xv.scale) && aligned16(xv.offset));
     if (!(dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy, addend, dx) && g.Cin % 4 == 0 && xf_vec)) return false;
     const Dw3Plan pl = plan_dw3(g, sm_count());
     const dim3 grid(pl.gx, pl.gy);
-    if (xf) launch(dw3_bwd_rows_kernel<T, true>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv);
-    else launch(dw3_bwd_rows_kernel<T, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv);
+    if (sums) sums->out->entries = 0;
+    const bool bst = xf && sums && dx && aligned16(sums->rstd);
+    if (bst) {
+        launch(dw3_bwd_rows_kernel<T, true, true>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, sums->rstd, sums->partial);
+        *sums->out = PartialSums{sums->partial, (int)grid.x, 1};
+    } else if (xf) launch(dw3_bwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);
+    else launch(dw3_bwd_rows_kernel<T, false, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);
     const int gx = (int)pl.gx;
     if (gx <= DW_FIN_SMALL) launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
     else {
@@ -1915,7 +1972,7 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
     template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t, const ColStatsReq*, const BnXform*); \
     template void dwconv_dgrad<T>(const T*, const float*, const T*, T*, const ConvGeom&, cudaStream_t);                     \
     template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*); \
-    template bool dwconv_bwd_fused<T>(const T*, const T*, const float*, const T*, T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*); \
+    template bool dwconv_bwd_fused<T>(const T*, const T*, const float*, const T*, T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*, const BnBwdSumsReq*); \
     template void maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);                                           \
     template void maxpool_bwd<T>(const T*, const T*, T*, int, int, int, int, cudaStream_t);                                 \
     template void gap_fwd<T>(const T*, T*, int, int, int, cudaStream_t);                                                    \

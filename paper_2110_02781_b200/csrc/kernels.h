@@ -184,11 +184,23 @@ template <typename T>
 void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin, cudaStream_t st,
                   const BnXform* x_xform = nullptr);
 
+// A kernel that produces the gradient with respect to the OUTPUT of a batch norm whose input it reads anyway may take
+// over the first pass of that batch norm's backward: it stores the gradient masked by the activation and leaves the
+// sums of g and g * xhat as partial sums (layout as the forward statistics) for bn_bwd_finalize.  *out: what it wrote
+// (entries == 0: nothing; the separate reduction has to run).
+struct BnBwdSumsReq {
+    const float* rstd;       // per channel, 16-byte aligned
+    double* partial;         // room: see the producer's *_stats_doubles
+    PartialSums* out;
+};
 // Data gradient (+ addend) and weight gradient of a stride-1 depthwise convolution in one pass over dy (dx may be NULL).
 // scratch: dwconv_wgrad_scratch_floats(g) floats.  false: shape not taken, nothing launched.
+// sums (nullable, needs x_xform): x is the input of the batch norm before this convolution; see BnBwdSumsReq
+// (partial: dwconv_bwd_stats_doubles(g) doubles).
+size_t dwconv_bwd_stats_doubles(const ConvGeom& g);
 template <typename T>
 bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
-                      cudaStream_t st, const BnXform* x_xform = nullptr);
+                      cudaStream_t st, const BnXform* x_xform = nullptr, const BnBwdSumsReq* sums = nullptr);
 
 template <typename T>
 void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);

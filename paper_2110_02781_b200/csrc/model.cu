@@ -300,6 +300,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             if (o.d.kind == FTP_FC) fcin = std::max(fcin, (size_t)o.in_elems);
         } else if (o.d.kind == FTP_DWCONV3x3) {
             red = std::max(red, dwconv_wgrad_scratch_floats(o.g));
+            foldd = std::max(foldd, dwconv_bwd_stats_doubles(o.g));
             finp = std::max(finp, fin_part_doubles(o.C, 9)); finc = std::max(finc, fin_counter_count(o.C, 9));
         }
     }
@@ -528,6 +529,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
             if (pending[k].buf == buf) { cudaStreamWaitEvent(st, pending[k].done, 0); pending.erase(pending.begin() + k); }
             else ++k;
     };
+    PartialSums bwd_sums{nullptr, 0, 1};                     // sums of a batch norm's backward pass left by the kernel that produced its output gradient
+    int bwd_sums_for = -1;                                   // ... and the batch norm they belong to
     for (int i = last; i >= first; --i) {
         Op& o = m->ops[i];
         const int u = o.d.unit;
@@ -623,7 +626,15 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
             case FTP_DWCONV3x3: {
                 if (gi && o.g.stride == 1) {          // one pass over dy gives the input gradient and the weight gradient
                     Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 3.0 : 2.0) + o.out_elems) * es + 2.0 * o.w_cnt * 4.0, 36.0 * o.out_elems, 2);
-                    if (dwconv_bwd_fused<T>((const T*)in, (const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, gr + o.w_off, m->red_scratch, o.g, m->fin, st, xf)) break;
+                    // ... and, when the input is what a deferred batch norm read, the sums of that batch norm's backward pass
+                    bwd_sums.entries = 0;
+                    BnBwdSumsReq sreq{nullptr, m->fold_scratch, &bwd_sums};
+                    const BnBwdSumsReq* sums = nullptr;
+                    if (xf && m->bwd_sums_on) { sreq.rstd = m->ops[i - 1].rstd; sums = &sreq; }
+                    if (dwconv_bwd_fused<T>((const T*)in, (const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, gr + o.w_off, m->red_scratch, o.g, m->fin, st, xf, sums)) {
+                        bwd_sums_for = bwd_sums.entries > 0 ? i - 1 : -1;
+                        break;
+                    }
                 }
                 { Scope sc(m, st, K_DW_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * es + o.w_cnt * 4.0, 18.0 * o.out_elems, 2);
                   const cudaStream_t ws = fork(i);
@@ -638,13 +649,18 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
             case FTP_BN: {
                 const long long Mr = (long long)o.N * o.H * o.W;
                 PartialSums ps;
-                { Scope sc(m, st, K_BN_BWD_REDUCE, u, i, 1, 2.0 * o.in_elems * es, 8.0 * o.in_elems);
+                const bool premasked = bwd_sums_for == i;          // the producer of `go` masked it and left the sums
+                bwd_sums_for = -1;
+                if (premasked) ps = bwd_sums;
+                else {
+                  Scope sc(m, st, K_BN_BWD_REDUCE, u, i, 1, 2.0 * o.in_elems * es, 8.0 * o.in_elems);
                   ps = bn_bwd_reduce<T>((const T*)go, (const T*)in, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.d.act, m->fold_scratch, st); }
                 { Scope sc(m, st, K_BN_BWD_FINALIZE, u, i, 1, ps.entries * 2.0 * o.C * 8.0, 0.0);
                   bn_bwd_finalize(ps, Mr, o.C, ar.w + o.w_off, o.rstd, gr + o.w_off, gr + o.b_off, o.coef, m->fin, st); }
                 if (gi) {
                     Scope sc(m, st, K_BN_BWD_APPLY, u, i, 1, (addend ? 4.0 : 3.0) * o.in_elems * es, 8.0 * o.in_elems);
-                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef, o.d.act, st);
+                    bn_bwd_apply<T>((const T*)go, (const T*)in, (const T*)addend, (T*)gi, Mr, o.C, o.fold, o.scale, o.shift, o.mean, o.mean_lo, o.rstd, o.coef,
+                                    premasked ? FTP_ACT_NONE : o.d.act, st);
                 }
                 break;
             }
@@ -811,6 +827,8 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         m->overlap = !(e && std::strcmp(e, "0") == 0);
         const char* ps = std::getenv("FTP_PRODUCER_STATS");          // 0: batch-norm statistics always by their own kernel (A/B measurements)
         m->producer_stats = !(ps && std::strcmp(ps, "0") == 0);
+        const char* bs = std::getenv("FTP_BWD_SUMS");                // 0: the first pass of every batch-norm backward by its own kernel (A/B measurements)
+        m->bwd_sums_on = !(bs && std::strcmp(bs, "0") == 0);
         bool ok = cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking) == cudaSuccess;
         for (size_t i = 0; ok && i <= m->ops.size(); ++i) {
             cudaEvent_t a = nullptr, b = nullptr;

@@ -73,7 +73,7 @@ struct ftp_model {
     ftp::FinScratch fin; size_t fin_counter_bytes;
     // weight gradients run on a second stream beside the chain of input gradients; they have scratch of their own
     float* red_side; ftp::FinScratch fin_side;
-    cudaStream_t side; std::vector<cudaEvent_t> ev_fork, ev_side; bool overlap; bool producer_stats;
+    cudaStream_t side; std::vector<cudaEvent_t> ev_fork, ev_side; bool overlap; bool producer_stats; bool bwd_sums_on;
     std::vector<ftp::TransposeEntryDev> tp_host; std::vector<int> tp_first;   // tp_first[u]: first entry of unit u (L + 1 values)
     ftp::TransposeEntryDev* tp_dev;
     void* dpre; size_t dpre_bytes;
