@@ -418,21 +418,24 @@ def measure(args, wl_key, reps, steps, warmup, local_rank, replicas, batch=None,
     for name, k in sorted(by.items(), key=lambda kv: -kv[1]["ms"]):
         gbs = k["bytes"] / (k["ms"] * 1e-3) / 1e9 if k["ms"] > 0 else 0.0
         tf = k["flops"] / (k["ms"] * 1e-3) / 1e12 if k["ms"] > 0 else 0.0
-        math_peak = tensor_peak if name.startswith("tc_gemm_bf16") else FP32_ALU_PEAK_TFLOPS
+        # bf16 products: the measured bf16 matmul rate.  Split-tf32 products (three tf32 MMAs per float product): that rate x the
+        # nominal tf32 / bf16 ratio (1.1 / 2.25 PFLOP/s dense), a third of it per float product.  Everything else: the fp32 FMA rate.
+        math_peak = tensor_peak if name.startswith("tc_gemm_bf16") else (tensor_peak * (1.1 / 2.25) / 3.0 if name.startswith("tc_gemm_tf32x3") else FP32_ALU_PEAK_TFLOPS)
         table[name] = dict(share=round(k["ms"] / total_ms, 4), launches_per_step=k["n"] // 3, ms_per_step=round(k["ms"] / 3, 4),
                            gbs=round(gbs, 1), tflops=round(tf, 2), frac_hbm=round(gbs / hbm_peak, 3),
                            frac_math=round(tf / math_peak, 3))
     dom = next(iter(table))
     d = table[dom]
     math_bound = d["frac_math"] > d["frac_hbm"]
-    tensor = dom.startswith("tc_gemm_bf16")
+    tensor = dom.startswith("tc_gemm_")
+    tpeak = tensor_peak if dom.startswith("tc_gemm_bf16") else tensor_peak * (1.1 / 2.25) / 3.0
     roofline = {"kernel": dom, "bound": ("tensor" if tensor else "alu") if math_bound else "hbm",
                 "achieved": d["tflops"] if math_bound else d["gbs"],
-                "peak": (tensor_peak if tensor else round(FP32_ALU_PEAK_TFLOPS, 1)) if math_bound else hbm_peak,
+                "peak": (round(tpeak, 1) if tensor else round(FP32_ALU_PEAK_TFLOPS, 1)) if math_bound else hbm_peak,
                 "unit": "TFLOP/s" if math_bound else "GB/s",
                 "frac": d["frac_math"] if math_bound else d["frac_hbm"],
-                "peak_source": ((f"{peak_src} bf16 matmul, sustained" if tensor else "derived: 2 x 128 lanes x 148 SMs x 1.965 GHz")
-                                if math_bound else f"{peak_src} HBM copy"),
+                "peak_source": ((f"{peak_src} bf16 matmul, sustained" + ("" if dom.startswith("tc_gemm_bf16") else " x 1.1/2.25 (tf32) / 3 products")
+                                 if tensor else "derived: 2 x 128 lanes x 148 SMs x 1.965 GHz") if math_bound else f"{peak_src} HBM copy"),
                 "traffic": ncu_traffic(wl_key, dom, batch is None), "share_of_step": d["share"],
                 "note": "achieved = algorithmic bytes (or flops) of all launches of the kernel in a step / their CUDA-event time",
                 "kernels": table}
