@@ -1267,6 +1267,322 @@ __global__ void __launch_bounds__(256) dw3_bwd_rows_kernel(const T* __restrict__
     }
 }
 
+// ---- stride-2 depthwise 3x3 (pad 1) on column strips, marching down the output rows ------------------------------
+// A thread owns four channels and two neighbouring output columns (input columns 2 wo0 - 1 .. 2 wo0 + 3) and walks
+// down RH output rows of one image.  Output row ho reads input rows 2 ho - 1, 2 ho, 2 ho + 1; the thread takes the
+// input rows in order, one pair per step with the next pair in flight, and carries the contribution of row 2 ho + 1
+// to output row ho + 1 (filter row 0) in registers, so every input row is fetched once per strip.  Block and slot
+// numbering as in the stride-1 kernels above (a slot is (image, row chunk, strip of two output columns)).
+template <typename T>
+__device__ __forceinline__ void dws2_fetch_row(const T* __restrict__ img, int hi, int H, int W, int C, int wi0, float (&r)[5][4]) {
+#pragma unroll
+    for (int j = 0; j < 5; ++j) {
+        const int wi = wi0 + j;
+        if (hi >= 0 && hi < H && wi >= 0 && wi < W) ldv<4>(img + ((long long)hi * W + wi) * C, r[j]);
+        else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r[j][e] = 0.f;
+        }
+    }
+}
+template <typename T, bool XF>
+__device__ __forceinline__ void dws2_take_row(const float (&raw)[5][4], int hi, int H, int W, int wi0, float (&r)[5][4], const XfRegs<T, 4>& xr) {
+#pragma unroll
+    for (int j = 0; j < 5; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) r[j][e] = raw[j][e];
+        if constexpr (XF) {
+            const int wi = wi0 + j;
+            if (hi >= 0 && hi < H && wi >= 0 && wi < W) xr.apply(r[j]);
+        }
+    }
+}
+// acc[j] += sum over the three taps of filter row `fr` of z[2 j + s] * w[fr][s]
+__device__ __forceinline__ void dws2_row_taps(const float (&z)[5][4], const float (*wsm)[32], int fr, int cvl, float (&acc)[2][4]) {
+#pragma unroll
+    for (int s = 0; s < 3; ++s) {
+        const float4 kk = *reinterpret_cast<const float4*>(&wsm[fr * 3 + s][cvl * 4]);
+        const float k4[4] = {kk.x, kk.y, kk.z, kk.w};
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[j][e] = fmaf(z[2 * j + s][e], k4[e], acc[j][e]);
+    }
+}
+
+template <typename T, bool XF, bool STATS>
+__global__ void __launch_bounds__(256, 2) dw3s2_fwd_rows_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int N, int H, int W,
+                                                                int C, int Ho, int Wo, int RH, int HC, double* __restrict__ stats, BnXform xf) {
+    grid_dep_sync();
+    __shared__ __align__(16) float wsm[9][32];
+    __shared__ float shs[STATS ? 2 : 1][32][33];
+    const int CV = C / 4, cvl = threadIdx.x & 7, slot = threadIdx.x >> 3, cv = blockIdx.y * 8 + cvl, c = cv * 4;
+    for (int i = threadIdx.x; i < 9 * 32; i += 256) {
+        const int tap = i >> 5, ch = blockIdx.y * 32 + (i & 31);
+        wsm[tap][i & 31] = ch < C ? w[tap * C + ch] : 0.f;
+    }
+    __syncthreads();
+    const int strips_w = (Wo + 1) >> 1;
+    const long long total = (long long)N * HC * strips_w;
+    float su[4] = {0.f, 0.f, 0.f, 0.f}, sq[4] = {0.f, 0.f, 0.f, 0.f};
+    for (long long gs = (long long)blockIdx.x * 32 + slot; cv < CV && gs < total; gs += (long long)gridDim.x * 32) {
+        const int sw = (int)(gs % strips_w);
+        const long long t = gs / strips_w;
+        const int hc = (int)(t % HC), n = (int)(t / HC);
+        const int wo0 = sw * 2, wi0 = 2 * wo0 - 1, h0 = hc * RH, h1 = min(Ho, h0 + RH);
+        XfRegs<T, 4> xr;
+        if constexpr (XF) xr.load(xf, c);
+        const T* img = x + (long long)n * H * W * C + c;
+        T* out = y + (long long)n * Ho * Wo * C + c;
+        float ra[5][4], rb[5][4], z[5][4], acc[2][4], accn[2][4];
+        dws2_fetch_row<T>(img, 2 * h0 - 1, H, W, C, wi0, rb);
+        dws2_fetch_row<T>(img, 2 * h0, H, W, C, wi0, ra);
+        dws2_take_row<T, XF>(rb, 2 * h0 - 1, H, W, wi0, z, xr);
+        dws2_fetch_row<T>(img, 2 * h0 + 1, H, W, C, wi0, rb);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) accn[j][e] = 0.f;
+        dws2_row_taps(z, wsm, 0, cvl, accn);
+        for (int ho = h0; ho < h1; ++ho) {
+            const bool more = ho + 1 < h1;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { acc[j][e] = accn[j][e]; accn[j][e] = 0.f; }
+            dws2_take_row<T, XF>(ra, 2 * ho, H, W, wi0, z, xr);
+            if (more) dws2_fetch_row<T>(img, 2 * ho + 2, H, W, C, wi0, ra);            // in flight while these rows are computed
+            dws2_row_taps(z, wsm, 1, cvl, acc);
+            dws2_take_row<T, XF>(rb, 2 * ho + 1, H, W, wi0, z, xr);
+            if (more) dws2_fetch_row<T>(img, 2 * ho + 3, H, W, C, wi0, rb);
+            dws2_row_taps(z, wsm, 2, cvl, acc);
+            dws2_row_taps(z, wsm, 0, cvl, accn);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (wo0 + j < Wo) {
+                    stv<4>(out + ((long long)ho * Wo + wo0 + j) * C, acc[j]);
+                    if constexpr (STATS) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { const float v = as_stored<T>(acc[j][e]); su[e] += v; sq[e] = fmaf(v, v, sq[e]); }
+                    }
+                }
+            }
+        }
+    }
+    if constexpr (STATS) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { shs[0][slot][cvl * 4 + e] = su[e]; shs[1][slot][cvl * 4 + e] = sq[e]; }
+        __syncthreads();
+        if (threadIdx.x < 64) {
+            const int a = threadIdx.x >> 5, ch = threadIdx.x & 31, gc = blockIdx.y * 32 + ch;
+            if (gc < C) {
+                double tsum = 0.0;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) tsum += (double)shs[a][q][ch];
+                stats[((long long)blockIdx.x * 2 + a) * C + gc] = tsum;
+            }
+        }
+    }
+}
+
+// Backward of the same convolution in one pass.  For output row ho the thread holds dy of rows ho and ho + 1 (columns
+// wo0 .. wo0 + 2) and takes input rows 2 ho (even) and 2 ho + 1 (odd), columns 2 wo0 - 1 .. 2 wo0 + 3:
+//   weight gradient: row 2 ho meets filter row 1 with dy[ho]; row 2 ho + 1 meets filter row 2 with dy[ho] and filter
+//   row 0 with dy[ho + 1] -- so no input row is carried from step to step;
+//   data gradient of its four input columns 2 wo0 .. 2 wo0 + 3 in both rows: an even row or column receives the middle
+//   tap of one output, an odd one the two outer taps of two outputs.
+// partial[blockIdx.x][9][C], bstats[blockIdx.x][2][C] and the meaning of XF / BST are those of dw3_bwd_rows_kernel.
+template <typename T>
+__device__ __forceinline__ void dws2_fetch_dy(const T* __restrict__ gimg, int ho, int Ho, int Wo, int C, int wo0, float (&r)[3][4]) {
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        if (ho < Ho && wo0 + j < Wo) ldv<4>(gimg + ((long long)ho * Wo + wo0 + j) * C, r[j]);
+        else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r[j][e] = 0.f;
+        }
+    }
+}
+
+template <typename T, bool XF, bool BST>
+__global__ void __launch_bounds__(256) dw3s2_bwd_rows_kernel(const T* __restrict__ x, const T* __restrict__ dy, const float* __restrict__ w,
+                                                             const T* __restrict__ addend, T* __restrict__ dx, float* __restrict__ partial, int N, int H,
+                                                             int W, int C, int Ho, int Wo, int RH, int HC, BnXform xf, const float* __restrict__ rstd,
+                                                             double* __restrict__ bstats) {
+    static_assert(!BST || XF, "the backward sums need the batch norm's input");
+    grid_dep_sync();
+    __shared__ __align__(16) float wsm[9][32];
+    __shared__ float sh[3][32][33];
+    float bs1[4] = {0.f, 0.f, 0.f, 0.f}, bs2[4] = {0.f, 0.f, 0.f, 0.f};
+    const int CV = C / 4, cvl = threadIdx.x & 7, slot = threadIdx.x >> 3, cv = blockIdx.y * 8 + cvl, c = cv * 4;
+    for (int i = threadIdx.x; i < 9 * 32; i += 256) {
+        const int tap = i >> 5, ch = blockIdx.y * 32 + (i & 31);
+        wsm[tap][i & 31] = ch < C ? w[tap * C + ch] : 0.f;
+    }
+    __syncthreads();
+    const int strips_w = (Wo + 1) >> 1;
+    const long long total = (long long)N * HC * strips_w;
+    float dwa[9][4];
+#pragma unroll
+    for (int tap = 0; tap < 9; ++tap)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dwa[tap][e] = 0.f;
+    for (long long gs = (long long)blockIdx.x * 32 + slot; cv < CV && gs < total; gs += (long long)gridDim.x * 32) {
+        const int sw = (int)(gs % strips_w);
+        const long long t = gs / strips_w;
+        const int hc = (int)(t % HC), n = (int)(t / HC);
+        const int wo0 = sw * 2, wi0 = 2 * wo0 - 1, h0 = hc * RH, h1 = min(Ho, h0 + RH);
+        XfRegs<T, 4> xr;
+        if constexpr (XF) xr.load(xf, c);
+        float rs[4] = {0.f, 0.f, 0.f, 0.f};
+        if constexpr (BST) ldtab<4>(rstd + c, rs);
+        const long long ioff = (long long)n * H * W * C + c;
+        const T* ximg = x + ioff;
+        const T* gimg = dy + (long long)n * Ho * Wo * C + c;
+        float cur[3][4], nxt[3][4], ra[5][4], rb[5][4];
+        dws2_fetch_dy<T>(gimg, h0, Ho, Wo, C, wo0, cur);
+        dws2_fetch_dy<T>(gimg, h0 + 1, Ho, Wo, C, wo0, nxt);
+        dws2_fetch_row<T>(ximg, 2 * h0, H, W, C, wi0, ra);
+        dws2_fetch_row<T>(ximg, 2 * h0 + 1, H, W, C, wi0, rb);
+        for (int ho = h0; ho < h1; ++ho) {
+            const bool more = ho + 1 < h1;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int hi = 2 * ho + half;
+                float z[5][4], xh[BST ? 4 : 1][4], acc[4][4];
+                unsigned pass = 0u;                              // bit 4 q + e: the activation lets the gradient of column 2 wo0 + q through
+#pragma unroll
+                for (int j = 0; j < 5; ++j) {
+                    const int wi = wi0 + j;
+                    const bool in = hi < H && wi >= 0 && wi < W;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) z[j][e] = half ? rb[j][e] : ra[j][e];
+                    if constexpr (BST) {
+                        if (in) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float cen = z[j][e] - xr.mu[e], v = fmaf(cen, xr.sc[e], xr.of[e]);
+                                if (j > 0) {
+                                    xh[j > 0 ? j - 1 : 0][e] = cen * rs[e];
+                                    if (v > xr.lo && v < xr.hi) pass |= 1u << (4 * (j > 0 ? j - 1 : 0) + e);
+                                }
+                                z[j][e] = as_stored<T>(fminf(fmaxf(v, xr.lo), xr.hi));
+                            }
+                        } else if (j > 0) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) xh[j > 0 ? j - 1 : 0][e] = 0.f;
+                        }
+                    } else if constexpr (XF) { if (in) xr.apply(z[j]); }
+                }
+                // the row's buffer is free: the row two below lands while this one is used
+                if (more) { if (half) dws2_fetch_row<T>(ximg, hi + 2, H, W, C, wi0, rb); else dws2_fetch_row<T>(ximg, hi + 2, H, W, C, wi0, ra); }
+                // weight gradient
+#pragma unroll
+                for (int s = 0; s < 3; ++s)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (half) {
+                                dwa[6 + s][e] = fmaf(z[2 * j + s][e], cur[j][e], dwa[6 + s][e]);
+                                dwa[s][e] = fmaf(z[2 * j + s][e], nxt[j][e], dwa[s][e]);
+                            } else dwa[3 + s][e] = fmaf(z[2 * j + s][e], cur[j][e], dwa[3 + s][e]);
+                        }
+                if (dx && hi < H) {
+                    // data gradient of columns 2 wo0 + q, q = 0 .. 3
+                    auto tap4 = [&](int tap, float (&k4)[4]) {
+                        const float4 kk = *reinterpret_cast<const float4*>(&wsm[tap][cvl * 4]);
+                        k4[0] = kk.x; k4[1] = kk.y; k4[2] = kk.z; k4[3] = kk.w;
+                    };
+                    if (!half) {
+                        float k0[4], k1[4], k2[4];
+                        tap4(3, k0); tap4(4, k1); tap4(5, k2);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[0][e] = k1[e] * cur[0][e];
+                            acc[1][e] = fmaf(k2[e], cur[0][e], k0[e] * cur[1][e]);
+                            acc[2][e] = k1[e] * cur[1][e];
+                            acc[3][e] = fmaf(k2[e], cur[1][e], k0[e] * cur[2][e]);
+                        }
+                    } else {
+                        float t0[4], t1[4], t2[4], b0[4], b1[4], b2[4];
+                        tap4(0, t0); tap4(1, t1); tap4(2, t2); tap4(6, b0); tap4(7, b1); tap4(8, b2);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[0][e] = fmaf(b1[e], cur[0][e], t1[e] * nxt[0][e]);
+                            acc[1][e] = fmaf(b2[e], cur[0][e], fmaf(b0[e], cur[1][e], fmaf(t2[e], nxt[0][e], t0[e] * nxt[1][e])));
+                            acc[2][e] = fmaf(b1[e], cur[1][e], t1[e] * nxt[1][e]);
+                            acc[3][e] = fmaf(b2[e], cur[1][e], fmaf(b0[e], cur[2][e], fmaf(t2[e], nxt[1][e], t0[e] * nxt[2][e])));
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int wi = 2 * wo0 + q;
+                        if (wi < W) {
+                            const long long o = ioff + ((long long)hi * W + wi) * C;
+                            if (addend) {
+                                float a[4];
+                                ldv<4>(addend + o, a);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) acc[q][e] += a[e];
+                            }
+                            if constexpr (BST) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float gq = (pass >> (4 * q + e)) & 1u ? as_stored<T>(acc[q][e]) : 0.f;
+                                    acc[q][e] = gq;
+                                    bs1[e] += gq;
+                                    bs2[e] = fmaf(gq, xh[q][e], bs2[e]);
+                                }
+                            }
+                            stv<4>(dx + o, acc[q]);
+                        }
+                    }
+                }
+            }
+            // dy moves down one output row
+#pragma unroll
+            for (int j = 0; j < 3; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) cur[j][e] = nxt[j][e];
+            if (more) dws2_fetch_dy<T>(gimg, ho + 2, Ho, Wo, C, wo0, nxt);
+        }
+    }
+    if constexpr (BST) {
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { sh[0][slot][cvl * 4 + e] = bs1[e]; sh[1][slot][cvl * 4 + e] = bs2[e]; }
+        __syncthreads();
+        if (threadIdx.x < 64) {
+            const int a = threadIdx.x >> 5, ch = threadIdx.x & 31, gc = blockIdx.y * 32 + ch;
+            if (gc < C) {
+                double tsum = 0.0;
+#pragma unroll 8
+                for (int q = 0; q < 32; ++q) tsum += (double)sh[a][q][ch];
+                bstats[((long long)blockIdx.x * 2 + a) * C + gc] = tsum;
+            }
+        }
+    }
+#pragma unroll
+    for (int gq = 0; gq < 3; ++gq) {
+        __syncthreads();
+#pragma unroll
+        for (int tq = 0; tq < 3; ++tq)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sh[tq][slot][cvl * 4 + e] = dwa[gq * 3 + tq][e];
+        __syncthreads();
+        if (threadIdx.x < 96) {
+            const int tq = threadIdx.x >> 5, ch = threadIdx.x & 31, gc = blockIdx.y * 32 + ch;
+            if (gc < C) {
+                float sum = 0.f;
+#pragma unroll 8
+                for (int q = 0; q < 32; ++q) sum += sh[tq][q][ch];
+                partial[((long long)blockIdx.x * 9 + gq * 3 + tq) * C + gc] = sum;
+            }
+        }
+    }
+}
+
 // ---- pooling --------------------------------------------------------------------------------------
 template <typename T, int V>
 __global__ void __launch_bounds__(256) maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, int H, int W, int C, long long total) {
@@ -1723,6 +2039,31 @@ static Dw3Plan plan_dw3(const ConvGeom& g, int resident_blocks) {
     p.gy = (unsigned)cgroups;
     return p;
 }
+// The same for the stride-2 kernels: strips of two output columns, chunks of output rows.
+static Dw3Plan plan_dw3s2(const ConvGeom& g, int resident_blocks) {
+    const int strips_w = (g.Wo + 1) / 2, cgroups = (g.Cin / 4 + 7) / 8;
+    const long long slots_x = std::max(1, resident_blocks / cgroups);
+    auto groups = [&](int hc) { return ((long long)g.N * hc * strips_w + 31) / 32; };
+    int best = 1;
+    while ((g.Ho + best - 1) / best > 8) best *= 2;
+    while (groups(best) * cgroups < resident_blocks && (g.Ho + 2 * best - 1) / (2 * best) >= 2) best *= 2;
+    Dw3Plan p;
+    p.RH = (g.Ho + best - 1) / best;
+    p.HC = (g.Ho + p.RH - 1) / p.RH;
+    p.groups = groups(p.HC);
+    // a block leaves one entry of partial sums: no more blocks than the statistics buffers of a [M][C] tensor hold
+    const long long room = ((long long)g.N * g.Ho * g.Wo + 127) / 128;
+    p.gx = (unsigned)std::max<long long>(1, std::min(std::min<long long>(p.groups, slots_x), room));
+    p.gy = (unsigned)cgroups;
+    return p;
+}
+static bool dw_s2_shape(const ConvGeom& g) { return g.stride == 2 && g.ph == 1 && g.pw == 1 && g.kh == 3 && g.kw == 3 && g.Cin % 4 == 0; }
+// FTP_DW_ROWS2: the stride-2 row kernels: 0 never, 1 float tensors only, 2 always (default)
+static bool dw_rows2_enabled(size_t elem_bytes) {
+    static int on = -1;
+    if (on < 0) { const char* e = std::getenv("FTP_DW_ROWS2"); on = e ? std::atoi(e) : 2; }
+    return on == 2 || (on == 1 && elem_bytes == 4);
+}
 // FTP_DW_ROWS: 0 never, 1 float tensors only (default: on bf16 tensors the two separate kernels, one of them on the
 // second stream, are faster), 2 always
 static bool dw_rows_enabled(size_t elem_bytes) {
@@ -1750,6 +2091,18 @@ void dwconv_fwd(const T* x, const float* w, T* y, const ConvGeom& g, cudaStream_
             *stats->out = PartialSums{stats->partial, (int)grid.x, 1};
         } else if (xf) launch(dw3_fwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, sp, xv);
         else launch(dw3_fwd_rows_kernel<T, false, false>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, sp, xv);
+        return;
+    }
+    if (dw_rows2_enabled(sizeof(T)) && dw_s2_shape(g) && can_vec<T>(g.Cin, x, y) && aligned16(w) && xf_vec) {
+        const Dw3Plan pl = plan_dw3s2(g, 2 * sm_count());
+        const dim3 grid(pl.gx, pl.gy);
+        double* sp = stats ? stats->partial : nullptr;
+        if (stats) {
+            if (xf) launch(dw3s2_fwd_rows_kernel<T, true, true>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, sp, xv);
+            else launch(dw3s2_fwd_rows_kernel<T, false, true>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, sp, xv);
+            *stats->out = PartialSums{stats->partial, (int)grid.x, 1};
+        } else if (xf) launch(dw3s2_fwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, sp, xv);
+        else launch(dw3s2_fwd_rows_kernel<T, false, false>, grid, dim3(256), 0, st, x, w, y, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, sp, xv);
         return;
     }
     if (g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, y) && aligned16(w) && xf_vec) {
@@ -1813,6 +2166,7 @@ size_t dwconv_wgrad_scratch_floats(const ConvGeom& g) {
     const FoldPlan a = plan_dw_wgrad(g, 4), b = plan_dw_wgrad(g, 2);
     size_t n = std::max((size_t)a.chunks * 9 * a.cols, (size_t)b.chunks * 9 * b.cols);
     if (g.Cin % 4 == 0 && g.stride == 1) n = std::max(n, (size_t)plan_dw3(g, sm_count()).gx * 9 * g.Cin);
+    if (dw_s2_shape(g)) n = std::max(n, (size_t)plan_dw3s2(g, sm_count()).gx * 9 * g.Cin);
     if (g.Cin % 4 == 0) n = std::max(n, (size_t)std::max(dw_wgrad_strip_blocks(g, 4, false), dw_wgrad_strip_blocks(g, 4, true)) * 9 * g.Cin);
     return n;
 }
@@ -1860,6 +2214,7 @@ void dwconv_wgrad(const T* x, const T* dy, float* dw, float* scratch, const Conv
 }
 
 size_t dwconv_bwd_stats_doubles(const ConvGeom& g) {
+    if (dw_s2_shape(g)) return (size_t)plan_dw3s2(g, sm_count()).gx * 2 * g.Cin;
     return g.Cin % 4 == 0 && g.stride == 1 ? (size_t)plan_dw3(g, sm_count()).gx * 2 * g.Cin : 0;
 }
 
@@ -1869,12 +2224,20 @@ bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, 
     const bool xf = x_xform != nullptr;
     const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f};
     const bool xf_vec = !xf || (aligned16(xv.mean) && aligned16(xv.scale) && aligned16(xv.offset));
-    if (!(dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy, addend, dx) && g.Cin % 4 == 0 && xf_vec)) return false;
-    const Dw3Plan pl = plan_dw3(g, sm_count());
-    const dim3 grid(pl.gx, pl.gy);
     if (sums) sums->out->entries = 0;
     const bool bst = xf && sums && dx && aligned16(sums->rstd);
-    if (bst) {
+    const bool s2 = dw_rows2_enabled(sizeof(T)) && dw_s2_shape(g);
+    if (s2 && !(can_vec<T>(g.Cin, x, dy, addend, dx) && aligned16(w) && xf_vec)) return false;
+    if (!s2 && !(dw_rows_enabled(sizeof(T)) && g.stride == 1 && g.ph == 1 && g.pw == 1 && can_vec<T>(g.Cin, x, dy, addend, dx) && g.Cin % 4 == 0 && xf_vec)) return false;
+    const Dw3Plan pl = s2 ? plan_dw3s2(g, sm_count()) : plan_dw3(g, sm_count());
+    const dim3 grid(pl.gx, pl.gy);
+    if (s2) {
+        if (bst) {
+            launch(dw3s2_bwd_rows_kernel<T, true, true>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, xv, sums->rstd, sums->partial);
+            *sums->out = PartialSums{sums->partial, (int)grid.x, 1};
+        } else if (xf) launch(dw3s2_bwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);
+        else launch(dw3s2_bwd_rows_kernel<T, false, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, g.Ho, g.Wo, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);
+    } else if (bst) {
         launch(dw3_bwd_rows_kernel<T, true, true>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, sums->rstd, sums->partial);
         *sums->out = PartialSums{sums->partial, (int)grid.x, 1};
     } else if (xf) launch(dw3_bwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);

@@ -178,11 +178,12 @@ ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cf
     // A batch norm inside a unit whose only reader can normalise while it loads (a depthwise convolution, or a 1x1
     // convolution on the split-tf32 tensor-core kernel) is never applied in memory: only its statistics and
     // per-channel constants are computed, and forward and weight gradient of the reader work from the BN's input.
-    // FTP_FUSE_BN (A/B measurements): bit 0 = into depthwise readers, bit 1 = into 1x1 readers, 0 = every batch norm stores
-    // its output.  Default: both in float models; none in bf16 models, whose depthwise kernels are bound by instruction
-    // issue and lose more to the extra arithmetic per loaded element than the saved pass gives back.
+    // FTP_FUSE_BN (A/B measurements): bit 0 = into depthwise readers, bit 1 = into 1x1 readers, bit 2 = into stride-2
+    // depthwise readers only, 0 = every batch norm stores its output.  Default: bits 0 and 1 in float models; bit 2 in
+    // bf16 models, whose stride-1 depthwise kernels are bound by instruction issue and lose more to the extra arithmetic
+    // per loaded element than the saved pass gives back.
     const char* fe = std::getenv("FTP_FUSE_BN");
-    const int fuse = fe ? std::atoi(fe) : (cfg->precision == FTP_FP32 ? 3 : 0);
+    const int fuse = fe ? std::atoi(fe) : (cfg->precision == FTP_FP32 ? 3 : 4);
     const char* fm = std::getenv("FTP_FUSE_MAX_MB");                  // only batch norms whose output is at most this large (A/B measurements)
     const double fuse_max_bytes = fm ? std::atof(fm) * 1e6 : 1e30;
     for (int i = 0; fuse && i + 1 < n; ++i) {
@@ -193,7 +194,7 @@ ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cf
         for (int j = i + 2; j < n; ++j) other_reader |= m.ops[j].d.kind == FTP_ADD_RESIDUAL && m.ops[j].d.residual_src == i;
         if (other_reader || (double)o.out_elems * m.esize > fuse_max_bytes) continue;
         void* const al = reinterpret_cast<void*>(256);
-        if (c.d.kind == FTP_DWCONV3x3) o.defer = (fuse & 1) != 0;
+        if (c.d.kind == FTP_DWCONV3x3) o.defer = (fuse & 1) != 0 || ((fuse & 4) != 0 && c.g.stride == 2);
         else if ((fuse & 2) && cfg->precision == FTP_FP32 && is_pointwise_op(c) && tc32_supported(c.N * c.Ho * c.Wo, c.Co, c.C, al, al, al, nullptr)) o.defer = true;
     }
     return FTP_OK;
@@ -624,7 +625,7 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                 break;
             }
             case FTP_DWCONV3x3: {
-                if (gi && o.g.stride == 1) {          // one pass over dy gives the input gradient and the weight gradient
+                if (gi && (o.g.stride == 1 || o.g.stride == 2)) {   // one pass over dy gives the input gradient and the weight gradient
                     Scope sc(m, st, K_DW_DGRAD, u, i, 1, (o.in_elems * (addend ? 3.0 : 2.0) + o.out_elems) * es + 2.0 * o.w_cnt * 4.0, 36.0 * o.out_elems, 2);
                     // ... and, when the input is what a deferred batch norm read, the sums of that batch norm's backward pass
                     bwd_sums.entries = 0;
@@ -827,8 +828,11 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
         m->overlap = !(e && std::strcmp(e, "0") == 0);
         const char* ps = std::getenv("FTP_PRODUCER_STATS");          // 0: batch-norm statistics always by their own kernel (A/B measurements)
         m->producer_stats = !(ps && std::strcmp(ps, "0") == 0);
-        const char* bs = std::getenv("FTP_BWD_SUMS");                // 0: the first pass of every batch-norm backward by its own kernel (A/B measurements)
-        m->bwd_sums_on = !(bs && std::strcmp(bs, "0") == 0);
+        // FTP_BWD_SUMS: 0 = the first pass of every batch-norm backward by its own kernel, 1 = from the depthwise backward
+        // kernel where it can give them.  Default: 1 in float models, 0 in bf16 models (the kernel with the sums inside
+        // took longer there than the reduction pass it saves).
+        const char* bs = std::getenv("FTP_BWD_SUMS");
+        m->bwd_sums_on = bs ? std::strcmp(bs, "0") != 0 : m->cfg.precision == FTP_FP32;
         bool ok = cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking) == cudaSuccess;
         for (size_t i = 0; ok && i <= m->ops.size(); ++i) {
             cudaEvent_t a = nullptr, b = nullptr;
