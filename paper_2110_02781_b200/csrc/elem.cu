@@ -198,22 +198,26 @@ __device__ __forceinline__ void fold_finish(float (&s)[NS][V], int cols, double*
 constexpr int FIN_X = 8;
 constexpr int FIN_Y = 128;
 constexpr int FIN_GMAX = 16;
-template <typename PT, int NS>
+// FY: the block's extent in y, FIN_Y or FIN_Y_SMALL (few partial sums: a block of 1024 threads does not fit on an SM that
+// also holds blocks of a kernel of the second stream, and would wait for them to leave).
+constexpr int FIN_Y_SMALL = 32;
+template <typename PT, int NS, int FY = FIN_Y>
 __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int ns, int chunks, int f, int C, int cols, int c,
                                               const FinScratch fin, double (&out)[NS]) {
-    static_assert(FIN_X == 8 && FIN_Y == 128, "the reduction below is written for 8 x 128 threads");
-    __shared__ double red[NS][FIN_X * FIN_Y / 32][FIN_X];
+    static_assert(FIN_X == 8 && (FY == 128 || FY == 32), "the reduction below is written for 8 x 128 or 8 x 32 threads");
+    constexpr int WARPS = FIN_X * FY / 32;
+    __shared__ double red[NS][WARPS][FIN_X];
     __shared__ unsigned ticket;
     double t[NS];
 #pragma unroll
     for (int a = 0; a < NS; ++a) t[a] = 0.0;
     const int total = chunks * f, G = gridDim.y;
     const int per = (total + G - 1) / G, e0 = blockIdx.y * per, e1 = min(total, e0 + per);
-    for (int e = e0 + threadIdx.y; e < e1; e += 4 * FIN_Y) {
+    for (int e = e0 + threadIdx.y; e < e1; e += 4 * FY) {
         double v[NS][4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {                    // four independent loads in flight per sum
-            const int ee = e + u * FIN_Y;
+            const int ee = e + u * FY;
             const bool ok = ee < e1 && c < C;
             const int ch = ok ? ee / f : 0, k = ok ? ee - ch * f : 0;
 #pragma unroll
@@ -222,8 +226,8 @@ __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int 
 #pragma unroll
         for (int a = 0; a < NS; ++a) t[a] += (v[a][0] + v[a][1]) + (v[a][2] + v[a][3]);
     }
-    // fixed-shape sum over y: the four y of a warp by shuffles, the 32 warps through shared memory (eight per lane
-    // group of the first warp, in order), the four lane groups by shuffles again
+    // fixed-shape sum over y: the four y of a warp by shuffles, the warps through shared memory (a quarter of them per
+    // lane group of the first warp, in order), the four lane groups by shuffles again
     const int lane = (threadIdx.y * FIN_X + threadIdx.x) & 31, warp = (threadIdx.y * FIN_X + threadIdx.x) >> 5;
 #pragma unroll
     for (int a = 0; a < NS; ++a) {
@@ -241,7 +245,7 @@ __device__ __forceinline__ bool col_fold_sums(const PT* partial, int first, int 
         for (int a = 0; a < NS; ++a) {
             double v = 0.0;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) v += red[a][q * 8 + w][x];
+            for (int w = 0; w < WARPS / 4; ++w) v += red[a][q * (WARPS / 4) + w][x];
             v += __shfl_xor_sync(0xffffffffu, v, 8);
             v += __shfl_xor_sync(0xffffffffu, v, 16);
             out[a] = v;
@@ -312,7 +316,8 @@ __device__ __forceinline__ double rsqrt_f64(double v) {
     return r;
 }
 
-__global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M, double inv_M, double unbias,
+template <int FY>
+__global__ void __launch_bounds__(FIN_X * FY) bn_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double M, double inv_M, double unbias,
                                    const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float mom,
                                    float* run_mean, float* run_var, float* scale, float* shift, float* mean, float* mean_lo, float* rstd,
                                    float* offset, const FinScratch fin) {
@@ -321,7 +326,7 @@ __global__ void bn_finalize_kernel(const double* __restrict__ partial, int chunk
     float ga = 0.f, be = 0.f, rm = 0.f, rv = 0.f;                    // fetched up front: their latency hides behind the sums
     if (threadIdx.y == 0 && c < C) { ga = gamma[c]; be = beta[c]; rm = run_mean[c]; rv = run_var[c]; }
     double ss[2];
-    if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
+    if (!col_fold_sums<double, 2, FY>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
     if (threadIdx.y == 0 && c < C) {
         const double mu = s1 * inv_M;
@@ -394,7 +399,8 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_kernel(const T* __restrict_
         }, C, copies);
 }
 
-__global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double inv_M,
+template <int FY>
+__global__ void __launch_bounds__(FIN_X * FY) bn_bwd_finalize_kernel(const double* __restrict__ partial, int chunks, int f, int C, int cols, double inv_M,
                                        const float* __restrict__ gamma, const float* __restrict__ rstd, float* dgamma,
                                        float* dbeta, float* coef, const FinScratch fin) {
     grid_dep_sync();
@@ -402,7 +408,7 @@ __global__ void bn_bwd_finalize_kernel(const double* __restrict__ partial, int c
     float ga = 0.f, rs = 0.f;
     if (threadIdx.y == 0 && c < C) { ga = gamma[c]; rs = rstd[c]; }
     double ss[2];
-    if (!col_fold_sums<double, 2>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
+    if (!col_fold_sums<double, 2, FY>(partial, 0, 2, chunks, f, C, cols, c, fin, ss)) return;
     const double s1 = ss[0], s2 = ss[1];
     if (threadIdx.y == 0 && c < C) {
         dbeta[c] = (float)s1;
@@ -1899,6 +1905,8 @@ FoldPlan make_fold(long long M, int C, int elem_bytes) {
     return fp;
 }
 
+// up to this many partial sums per channel the second pass runs in blocks of FIN_X x FIN_Y_SMALL threads (one slice)
+constexpr int FIN_SMALL_ENTRIES = 8 * FIN_Y_SMALL;
 static inline int fin_slices_ps(const PartialSums& ps) {
     const int g = ps.entries / (4 * FIN_Y);
     return g < 1 ? 1 : (g > FIN_GMAX ? FIN_GMAX : g);
@@ -1943,8 +1951,12 @@ PartialSums bn_stats(const T* y, long long M, int C, const FoldPlan& fp, double*
 void bn_finalize(const PartialSums& ps, long long M, int C, const float* gamma, const float* beta,
                  float eps, float momentum, float* run_mean, float* run_var, float* scale, float* shift, float* mean,
                  float* mean_lo, float* rstd, float* offset, const FinScratch& fin, cudaStream_t st) {
-    launch(bn_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp, (double)M,
-           1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0, gamma, beta, eps, momentum, run_mean, run_var, scale, shift, mean, mean_lo, rstd, offset, fin);
+    if (ps.entries <= FIN_SMALL_ENTRIES)
+        launch(bn_finalize_kernel<FIN_Y_SMALL>, dim3((C + FIN_X - 1) / FIN_X, 1), dim3(FIN_X, FIN_Y_SMALL), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp, (double)M,
+               1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0, gamma, beta, eps, momentum, run_mean, run_var, scale, shift, mean, mean_lo, rstd, offset, fin);
+    else
+        launch(bn_finalize_kernel<FIN_Y>, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp, (double)M,
+               1.0 / (double)M, M > 1 ? (double)M / (double)(M - 1) : 1.0, gamma, beta, eps, momentum, run_mean, run_var, scale, shift, mean, mean_lo, rstd, offset, fin);
 }
 
 template <typename T>
@@ -1974,7 +1986,11 @@ PartialSums bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const Fol
 
 void bn_bwd_finalize(const PartialSums& ps, long long M, int C, const float* gamma, const float* rstd,
                      float* dgamma, float* dbeta, float* coef, const FinScratch& fin, cudaStream_t st) {
-    launch(bn_bwd_finalize_kernel, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp,
+    if (ps.entries <= FIN_SMALL_ENTRIES)
+        launch(bn_bwd_finalize_kernel<FIN_Y_SMALL>, dim3((C + FIN_X - 1) / FIN_X, 1), dim3(FIN_X, FIN_Y_SMALL), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp,
+           1.0 / (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
+    else
+        launch(bn_bwd_finalize_kernel<FIN_Y>, dim3((C + FIN_X - 1) / FIN_X, fin_slices_ps(ps)), dim3(FIN_X, FIN_Y), 0, st, ps.p, ps.entries / ps.fp, ps.fp, C, C * ps.fp,
            1.0 / (double)M, gamma, rstd, dgamma, dbeta, coef, fin);
 }
 

@@ -3,6 +3,7 @@
 // per-unit profile and the kernel trace.
 #include <algorithm>
 #include <cstdlib>
+#include <string>
 #include <cstring>
 #include <new>
 #include <type_traits>
@@ -206,7 +207,17 @@ ftp_status plan_gradients(ftp_model& m, int* n_slots) {
     std::vector<int> refc;               // per slot: readers still to come
     std::vector<int> freel;
     std::vector<int> pending(n + 1, -1); // pending[j+1]: op whose output-gradient buffer must be added into grad(out[j])
-    auto alloc = [&]() { if (!freel.empty()) { int s = freel.back(); freel.pop_back(); refc[s] = 1; return s; } refc.push_back(1); return (int)refc.size() - 1; };
+    // A freed slot is handed out again as late as possible (oldest first, and only once `spare` slots exist): the weight
+    // gradient that reads a gradient buffer runs on the second stream, and the main stream has to wait for it before the
+    // buffer is overwritten.  FTP_GRAD_SLOTS: the number of slots before any is reused (A/B measurements; at least the
+    // liveness minimum is always allocated).
+    const char* gs = std::getenv("FTP_GRAD_SLOTS");
+    const int spare = gs ? std::atoi(gs) : 16;
+    auto alloc = [&]() {
+        if (!freel.empty() && (int)refc.size() >= spare) { int s = freel.front(); freel.erase(freel.begin()); refc[s] = 1; return s; }
+        refc.push_back(1);
+        return (int)refc.size() - 1;
+    };
     auto release = [&](int s) { if (s >= 0 && --refc[s] == 0) freel.push_back(s); };
     for (int i = n - 1; i >= 0; --i) {
         Op& o = m.ops[i];
@@ -566,8 +577,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                                             o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                         if (dpre) d = dpre;
                     }
-                    { Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
-                      const cudaStream_t ws = fork(i);
+                    const cudaStream_t ws = fork(i);                 // forked here: the weight gradient depends on nothing after this point
+                    auto weight_gradient = [&]() -> ftp_status {
+                      Scope sc(m, st, K_CONV_WGRAD_F32, u, i, 1, (o.in_elems + o.out_elems + o.w_cnt) * 4.0, fl, 2);
                       float* rs = ws == st ? m->red_scratch : m->red_side;
                       const bool tc = is_pointwise_op(o) && tc32_supported((int)Mout, o.Co, o.C, x, d, gr + o.w_off, nullptr) &&
                                       tc32_wgrad(x, d, gr + o.w_off, rs, Mout, o.C, o.Co, m->tc_err, ws, xf);
@@ -575,7 +587,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                       if (tc && sc.slot) sc.slot->rec.kernel = K_TC32_WGRAD;
                       const bool stem = !tc && !widened && o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_wgrad<float>(x, d, gr + o.w_off, rs, o.g, ws);
                       if (!tc && !stem) conv_wgrad_f32(x, d, gr + o.w_off, rs, o.g, ws);
-                      forked(i, d); }
+                      forked(i, d);
+                      return FTP_OK; };
+                    { const ftp_status ws_s = weight_gradient(); if (ws_s != FTP_OK) return ws_s; }
                     if (gi) {
                         Scope sc(m, st, K_CONV_DGRAD_F32, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 4.0, fl, widened ? 2 : 1);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the weights as they lie are the K-major B operand
@@ -596,8 +610,9 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                                         o.b_off >= 0 ? gr + o.b_off : nullptr, m->fin, st);
                         if (dpre) d = dpre;
                     }
-                    { Scope sc(m, st, K_GEMM_BF16_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
-                      const cudaStream_t ws = fork(i);
+                    const cudaStream_t ws = fork(i);                 // forked here: the weight gradient depends on nothing after this point
+                    auto weight_gradient = [&]() {
+                      Scope sc(m, st, K_GEMM_BF16_WGRAD, u, i, 1, (o.in_elems + o.out_elems) * 2.0 + o.w_cnt * 4.0, fl, 2);
                       float* rs = ws == st ? m->red_scratch : m->red_side;
                       int splits = 0;
                       if (is_pointwise_op(o) && tc_gemm_supported((int)Mout, o.Co, o.C, in, d, gr + o.w_off, nullptr))
@@ -610,7 +625,8 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                           const bool stem = o.d.act == FTP_ACT_NONE && o.b_off < 0 && stem_conv_wgrad<T>((const T*)in, d, gr + o.w_off, rs, o.g, ws);
                           if (!stem) conv_wgrad_bf16_simt((const T*)in, d, gr + o.w_off, rs, o.g, ws);
                       }
-                      forked(i, d); }
+                      forked(i, d); };
+                    weight_gradient();
                     if (gi) {
                         Scope sc(m, st, K_GEMM_BF16_DGRAD, u, i, 1, (o.in_elems * (addend ? 2.0 : 1.0) + o.out_elems + o.w_cnt) * 2.0, fl);
                         // dx[M, cin] = dy[M, cout] * w[cin][cout]^T: the canonical weight layout already has K = cout contiguous
@@ -1467,17 +1483,25 @@ static std::vector<void (*)(std::vector<unsigned long long>&, bool)>& tl_readers
     return v;
 }
 void tl_register(void (*reader)(std::vector<unsigned long long>&, bool)) { tl_readers().push_back(reader); }
-static std::vector<const void*> g_tl_launched;
-void tl_note_launch(const void* kernel) { if (g_tl_launched.size() < (1u << 20)) g_tl_launched.push_back(kernel); }
+struct TlLaunch { const void* kernel; unsigned long long signature; const void* stream; };
+static std::vector<TlLaunch> g_tl_launched;
+void tl_note_launch(const void* kernel, unsigned long long signature, const void* stream) {
+    if (g_tl_launched.size() < (1u << 20)) g_tl_launched.push_back({kernel, signature, stream});
+}
 }  // namespace ftp
-// Measurement build only: the (mangled) names of the kernels launched since the last reset, one per line, in launch order.
+// Measurement build only: the kernels launched since the last reset, one per line in launch order: mangled name, tab,
+// signature of the grid (decimal), tab, stream (hex).
 extern "C" int32_t ftp_debug_launch_names(char* buf, int32_t cap, int32_t reset) {
     size_t used = 0;
     int32_t n = 0;
-    for (const void* k : ftp::g_tl_launched) {
-        const char* name = nullptr;
-        if (cudaFuncGetName(&name, k) != cudaSuccess || !name) name = "?";
-        const size_t len = std::strlen(name);
+    for (const ftp::TlLaunch& l : ftp::g_tl_launched) {
+        const char* fn = nullptr;
+        if (cudaFuncGetName(&fn, l.kernel) != cudaSuccess || !fn) fn = "?";
+        char tail[64];
+        std::snprintf(tail, sizeof tail, "\t%llu\t%p", l.signature, l.stream);
+        const std::string line = std::string(fn) + tail;
+        const char* name = line.c_str();
+        const size_t len = line.size();
         if (used + len + 2 > (size_t)std::max(cap, 0)) break;
         std::memcpy(buf + used, name, len);
         used += len;
@@ -1488,15 +1512,18 @@ extern "C" int32_t ftp_debug_launch_names(char* buf, int32_t cap, int32_t reset)
     if (reset) ftp::g_tl_launched.clear();
     return n;
 }
-// Measurement build only: the start times (ns of the global timer) of all grids launched since the last reset, merged
-// over the translation units and sorted; synchronises the device.
+// Measurement build only: the start time (ns of the global timer) and the signature of every grid launched since the last
+// reset, merged over the translation units and sorted by time: out[2 i] = time, out[2 i + 1] = signature, at most `max`
+// entries; returns the number of entries there are; synchronises the device.
 extern "C" int32_t ftp_debug_timeline(unsigned long long* out, int32_t max, int32_t reset) {
     cudaDeviceSynchronize();
-    std::vector<unsigned long long> all;
-    for (auto r : ftp::tl_readers()) r(all, reset != 0);
+    std::vector<unsigned long long> raw;
+    for (auto r : ftp::tl_readers()) r(raw, reset != 0);
+    std::vector<std::pair<unsigned long long, unsigned long long>> all(raw.size() / 2);
+    for (size_t i = 0; i < all.size(); ++i) all[i] = {raw[2 * i], raw[2 * i + 1]};
     std::sort(all.begin(), all.end());
     const int32_t n = (int32_t)std::min<size_t>(all.size(), (size_t)std::max(max, 0));
-    for (int32_t i = 0; i < n; ++i) out[i] = all[i];
+    for (int32_t i = 0; i < n; ++i) { out[2 * i] = all[i].first; out[2 * i + 1] = all[i].second; }
     return (int32_t)all.size();
 }
 #endif
