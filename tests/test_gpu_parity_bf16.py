@@ -100,6 +100,12 @@ def test_tiny_mobilenet_bf16_every_unit_a_stage():
     step_case((ls, cfg), 61, list(range(synth.num_units(ls) + 1)))
 
 
+def test_stride_two_depthwise_rows_on_odd_maps_bf16():
+    """The stride-2 depthwise kernels (with the batch norm in front of them folded in, the bf16 default) on 9 x 9 and 5 x 5 maps."""
+    net = synth.mobilenetv2(3, 9, 7, 1, True, table=[(1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 1, 2)], stem_c=32, last_c=64)
+    step_case(net, 29, [0, 2, 4, 7])
+
+
 def test_tiny_vgg_bf16_dense_3x3_and_maxpool():
     step_case(synth.tiny_vgg(batch=6, hw=4, precision=1), 62, [0, 1, 3])
 

@@ -214,6 +214,14 @@ def test_edge_shapes_batch_one_odd_channels():
         one_step_case((ls, cfg), 25, [0, 1, 2, 3])
 
 
+def test_stride_two_depthwise_rows_on_odd_maps():
+    """Stride-2 depthwise layers on 9 x 9 and 5 x 5 maps (outputs 5 x 5 and 3 x 3): the last input row and column have
+    no partner, the last output strip holds one column, and a thread's walk ends on an odd row; 144 and 192 channels
+    (the last channel group of a block is partly empty)."""
+    net = synth.mobilenetv2(3, 9, 7, 0, True, table=[(1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 1, 2)], stem_c=32, last_c=64)
+    one_step_case(net, 29, [0, 2, 4, 7], max_stages=4)
+
+
 def test_pointwise_weight_gradients_on_ragged_slabs():
     """1 x 1 convolutions whose weight gradients run on the tensor cores with both operands as they lie in memory:
     channel counts that end inside a 32-column slab (40, 72, 136), on both sides of the 128-row tile (so the product
