@@ -1808,24 +1808,6 @@ __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ s, float* _
         d[i] = __bfloat162float(s[i]);
 }
 
-// wt[n][k] = bf16(w[k][n]) through a 32 x 32 shared-memory tile
-__global__ void transpose_f32_to_bf16_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ wt, int K, int N) {
-    grid_dep_sync();
-    __shared__ float tile[32][33];
-    const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
-    w += (long long)blockIdx.z * K * N;
-    wt += (long long)blockIdx.z * K * N;
-    for (int r = threadIdx.y; r < 32; r += 8) {
-        const int k = k0 + r, n = n0 + threadIdx.x;
-        tile[r][threadIdx.x] = (k < K && n < N) ? w[(long long)k * N + n] : 0.f;
-    }
-    __syncthreads();
-    for (int r = threadIdx.y; r < 32; r += 8) {
-        const int n = n0 + r, k = k0 + threadIdx.x;
-        if (n < N && k < K) wt[(long long)n * K + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
-    }
-}
-
 __global__ void tf32_lo_kernel(const float* __restrict__ w, float* __restrict__ lo, long long n) {
     grid_dep_sync();
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
@@ -1866,6 +1848,39 @@ __global__ void transpose_split_f32_kernel(const TransposeEntryDev* __restrict__
             wt[en.w_off + (long long)c * en.K + k] = v;
             wtl[en.w_off + (long long)c * en.K + k] = v - __uint_as_float(__float_as_uint(v) & 0xffffe000u);
         }
+    }
+}
+
+// The bf16 models' counterpart: wt[tap][n][k] = bf16(w[tap][k][n]) for every matrix of the table in one launch (an entry's
+// `taps` matrices of K x N lie one after the other: 1 for a 1x1 convolution, 9 for a 3x3 one).
+__global__ void transpose_bf16_batched_kernel(const TransposeEntryDev* __restrict__ table, int n, int tile_base, const float* __restrict__ w,
+                                              __nv_bfloat16* __restrict__ wt) {
+    grid_dep_sync();
+    __shared__ float tile[32][33];
+    __shared__ int first_tile[256];
+    const int t = tile_base + blockIdx.x;
+    const int tid = threadIdx.y * 32 + threadIdx.x;
+    int e = 0;
+    if (n <= 256) {
+        if (tid < n) first_tile[tid] = table[tid].tile0;
+        __syncthreads();
+        while (e + 1 < n && first_tile[e + 1] <= t) ++e;
+    } else {
+        while (e + 1 < n && table[e + 1].tile0 <= t) ++e;
+    }
+    const TransposeEntryDev en = table[e];
+    const int tn = (en.N + 31) / 32, per_tap = ((en.K + 31) / 32) * tn;
+    const int local = t - en.tile0, tap = local / per_tap, in_tap = local - tap * per_tap;
+    const int k0 = (in_tap / tn) * 32, n0 = (in_tap % tn) * 32;
+    const long long base = en.w_off + (long long)tap * en.K * en.N;
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const int k = k0 + r, c = n0 + threadIdx.x;
+        tile[r][threadIdx.x] = (k < en.K && c < en.N) ? w[base + (long long)k * en.N + c] : 0.f;
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const int c = n0 + r, k = k0 + threadIdx.x;
+        if (c < en.N && k < en.K) wt[base + (long long)c * en.K + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
     }
 }
 
@@ -2324,8 +2339,8 @@ void transpose_split_f32(const TransposeEntryDev* table, int n, int tile_base, i
     if (tiles > 0) launch(transpose_split_f32_kernel, dim3(tiles), dim3(32, 8), 0, st, table, n, tile_base, w, wt, wtl);
 }
 
-void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st) {
-    launch(transpose_f32_to_bf16_kernel, dim3((N + 31) / 32, (K + 31) / 32, batch), dim3(32, 8), 0, st, w, wt, K, N);
+void transpose_bf16_batched(const TransposeEntryDev* table, int n, int tile_base, int tiles, const float* w, __nv_bfloat16* wt, cudaStream_t st) {
+    if (tiles > 0) launch(transpose_bf16_batched_kernel, dim3(tiles), dim3(32, 8), 0, st, table, n, tile_base, w, wt);
 }
 
 void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st) {

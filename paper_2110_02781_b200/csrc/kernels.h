@@ -71,7 +71,6 @@ int tc_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, floa
 size_t tc_wgrad_scratch_floats(long long R, int Mo, int No);
 int tc_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* dW, float* scratch, long long R, int Mo, int No, int* err, cudaStream_t st);
 void split_reduce_f32(const float* partial, int S, long long count, float* out, cudaStream_t st);   // out = sum over S partial arrays, in order
-void transpose_f32_to_bf16(const float* w, __nv_bfloat16* wt, int K, int N, int batch, cudaStream_t st);   // per matrix: wt[n][k] = bf16(w[k][n])
 
 // ---- float contractions on tensor cores with split-tf32 arithmetic (gemm_tc32.cu); same conventions as above ----
 bool tc32_supported(int M, int N, int K, const void* A, const void* B, const void* D, const void* addend);
@@ -227,8 +226,10 @@ void tf32_lo(const float* w, float* lo, long long n, cudaStream_t st);          
 // Batched transposition of float matrices: entry e describes a [K][N] matrix at w + w_off whose transpose goes to
 // wt + w_off ([N][K]) and the lo part of the transpose to wtl + w_off.  table: n + 1 device entries (the last one
 // closes the tile range); tiles = table[n].tile0 - table[0].tile0 blocks are launched.
-struct TransposeEntryDev { long long w_off; int K, N, tile0, pad; };
+struct TransposeEntryDev { long long w_off; int K, N, tile0, taps; };       // taps: matrices of K x N one after the other (bf16 models: 9 for a 3x3 convolution)
 void transpose_split_f32(const TransposeEntryDev* table, int n, int tile_base, int tiles, const float* w, float* wt, float* wtl, cudaStream_t st);
+// bf16 models: wt[tap][N][K] = bf16(w[tap][K][N]) for n table entries in one launch (tiles: 32 x 32 tiles of all their matrices)
+void transpose_bf16_batched(const TransposeEntryDev* table, int n, int tile_base, int tiles, const float* w, __nv_bfloat16* wt, cudaStream_t st);
 void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t st);
 void bf16_to_f32(const __nv_bfloat16* src, float* dst, long long n, cudaStream_t st);
 

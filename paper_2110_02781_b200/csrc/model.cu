@@ -66,6 +66,7 @@ struct Scope {
 
 bool is_contraction(int kind) { return kind == FTP_CONV1D || kind == FTP_CONV2D || kind == FTP_FC; }
 bool is_pointwise_op(const Op& o);
+bool is_3x3_op(const Op& o);
 
 // ---- shapes, parameter offsets, validation ------------------------------------------------------
 ftp_status plan_ops(const ftp_layer_desc* layers, int n, const ftp_model_cfg* cfg, ftp_model& m) {
@@ -270,12 +271,16 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             const Op& o = m.ops[i];
             while (u_next <= o.d.unit) m.tp_first[u_next++] = (int)m.tp_host.size();
             if (m.cfg.precision == FTP_FP32 && is_pointwise_op(o) && o.d.kind != FTP_FC) {
-                m.tp_host.push_back(TransposeEntryDev{o.w_off, o.C, o.Co, tile0, 0});
+                m.tp_host.push_back(TransposeEntryDev{o.w_off, o.C, o.Co, tile0, 1});
                 tile0 += ((o.C + 31) / 32) * ((o.Co + 31) / 32);
+            } else if (m.cfg.precision == FTP_BF16 && (is_pointwise_op(o) || is_3x3_op(o))) {
+                const int taps = o.g.kh * o.g.kw;
+                m.tp_host.push_back(TransposeEntryDev{o.w_off, o.C, o.Co, tile0, taps});
+                tile0 += taps * ((o.C + 31) / 32) * ((o.Co + 31) / 32);
             }
         }
         while (u_next <= m.L) m.tp_first[u_next++] = (int)m.tp_host.size();
-        m.tp_host.push_back(TransposeEntryDev{0, 0, 0, tile0, 0});
+        m.tp_host.push_back(TransposeEntryDev{0, 0, 0, tile0, 1});
         m.tp_dev = (TransposeEntryDev*)bp.take(m.tp_host.size() * sizeof(TransposeEntryDev));
     }
     m.grad = (float*)bp.take((size_t)m.P * 4);
@@ -355,26 +360,20 @@ bool is_3x3_op(const Op& o) {
     return o.d.kind == FTP_CONV2D && o.g.kh == 3 && o.g.kw == 3 && o.g.stride == 1 && o.g.ph == 1 && o.g.pw == 1 && o.d.act == FTP_ACT_NONE && o.b_off < 0;
 }
 
-// Rebuild the transposed copies of the 1x1-convolution matrices of units [a, b) from the float masters: bf16 models
-// one matrix at a time, float models in one batched launch per owning arena.
+// Rebuild the transposed copies of the convolution matrices of units [a, b) from the float masters: one batched launch
+// per owning arena (float models: the 1x1 matrices with their lo parts; bf16 models: the 1x1 and 3x3 matrices).
 void refresh_transposed(ftp_model* m, int a, int b, cudaStream_t st) {
-    if (m->cfg.precision == FTP_FP32) {
-        for (int u = a; u < b;) {
-            int v = u + 1;
-            while (v < b && m->owner[v] == m->owner[u]) ++v;
-            const Arena& ar = m->arena[m->owner[u]];
-            const int e0 = m->tp_first[u], e1 = m->tp_first[v];
-            if (e1 > e0)
-                transpose_split_f32(m->tp_dev + e0, e1 - e0, m->tp_host[e0].tile0, m->tp_host[e1].tile0 - m->tp_host[e0].tile0,
-                                    ar.w, ar.wt, ar.wtl, st);
-            u = v;
+    for (int u = a; u < b;) {
+        int v = u + 1;
+        while (v < b && m->owner[v] == m->owner[u]) ++v;
+        const Arena& ar = m->arena[m->owner[u]];
+        const int e0 = m->tp_first[u], e1 = m->tp_first[v];
+        if (e1 > e0) {
+            const int tiles = m->tp_host[e1].tile0 - m->tp_host[e0].tile0;
+            if (m->cfg.precision == FTP_FP32) transpose_split_f32(m->tp_dev + e0, e1 - e0, m->tp_host[e0].tile0, tiles, ar.w, ar.wt, ar.wtl, st);
+            else if (ar.wbt) transpose_bf16_batched(m->tp_dev + e0, e1 - e0, m->tp_host[e0].tile0, tiles, ar.w, ar.wbt, st);
         }
-        return;
-    }
-    for (int i = m->unit_first[a]; i <= m->unit_last[b - 1]; ++i) {
-        const Op& o = m->ops[i];
-        const Arena& ar = m->arena[m->owner[o.d.unit]];
-        if (ar.wbt && (is_pointwise_op(o) || is_3x3_op(o))) transpose_f32_to_bf16(ar.w + o.w_off, ar.wbt + o.w_off, o.C, o.Co, o.g.kh * o.g.kw, st);
+        u = v;
     }
 }
 
