@@ -175,7 +175,14 @@ ftp_status ftp_sgd_step(ftp_model* m, int32_t a, int32_t b, float lr, float* sna
  *                 label outside [0, n_classes) is refused with FTP_ERANGE before anything is
  *                 launched -- else device (labels then clamp as in ftp_run_stage_forward).
  *   loss_host   : if non-NULL (host float[1]) the loss is copied back and the call returns
- *                 after the step has completed; if NULL the call is fully asynchronous. */
+ *                 after the step has completed; if NULL the call is fully asynchronous.
+ * Under stream capture (the caller records the step into a CUDA graph): host inputs must be
+ * pinned -- their copies become nodes of the graph and read the same buffers at every replay, and
+ * the labels are checked at capture time only (at replay they clamp) -- and loss_host, if
+ * non-NULL, must be pinned too: the copy of the loss into it becomes the last node, nothing is
+ * synchronised, and the value is valid once a replay has completed.  Record after the model's
+ * first update: whether a unit's momentum buffer is initialised or accumulated is decided when
+ * the step is recorded, and so are lr and the partition. */
 ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t* labels, int32_t inputs_on_host, float lr,
                           float* loss_host, void* stream);
 

@@ -1904,7 +1904,11 @@ FoldPlan make_fold(long long M, int C, int elem_bytes) {
     fp.cols = C * fp.f;
     fp.rows = (int)(M / fp.f);
     const int coltiles = (fp.cols + 32 * fp.vec - 1) / (32 * fp.vec);
-    long long chunks = (4LL * sm_count() + coltiles - 1) / coltiles;
+    // blocks per SM: the float kernels with the most registers (bn_bwd_apply, 80) hold three blocks per SM, so a grid of
+    // four per SM runs a third of a second wave (config 2: 3.30 -> 3.27 ms per step with three); the bf16 kernels, which
+    // move half the bytes per thread, measured better with four (config 3: 5.06 against 5.09 ms)
+    const long long per_sm = elem_bytes == 4 ? 3 : 4;
+    long long chunks = (per_sm * sm_count() + coltiles - 1) / coltiles;
     const long long maxc = (fp.rows + 15) / 16;
     if (chunks > maxc) chunks = maxc;
     if (chunks < 1) chunks = 1;

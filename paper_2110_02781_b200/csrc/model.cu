@@ -1044,12 +1044,15 @@ extern "C" ftp_status ftp_train_step(ftp_model* m, const void* x, const int32_t*
     } else FTP_REQUIRE(a16(x), FTP_ERANGE, "train_step: the input batch must be 16-byte aligned");
     ftp_status s = m->cfg.precision == FTP_FP32 ? train_step_t<float>(m, xin, lab, lr, st) : train_step_t<__nv_bfloat16>(m, xin, lab, lr, st);
     if (s != FTP_OK) return s;
-    if (loss_host) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
+    if (loss_host && cap == cudaStreamCaptureStatusNone) {
         CUDA_OK(cudaMemcpyAsync(m->pinned, m->loss_dev, 4, cudaMemcpyDeviceToHost, st));
         s = read_device_status(m, st, "train_step");
         *loss_host = m->pinned[0];
         return s;
     }
+    if (loss_host) CUDA_OK(cudaMemcpyAsync(loss_host, m->loss_dev, 4, cudaMemcpyDeviceToHost, st));    // recorded into the caller's graph
     queue_status(m, st);
     return FTP_OK;
 }

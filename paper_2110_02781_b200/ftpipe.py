@@ -403,7 +403,15 @@ class Model:
     def ftp_sgd_step(self, a, b, lr, snap_dev=None, snap_host=None, stream=None):
         _check(lib.ftp_sgd_step(self.h, a, b, lr, _ptr(snap_dev), _ptr(snap_host), _stream(stream)))
 
-    def ftp_train_step(self, x, labels, lr, inputs_on_host=False, want_loss=True, stream=None):
+    def ftp_train_step(self, x, labels, lr, inputs_on_host=False, want_loss=True, stream=None, loss_pinned=None):
+        """loss_pinned: a pinned float32 host tensor of one element that receives the loss instead of the return value --
+        the form to use while the step is captured into a CUDA graph (the copy becomes a node of the graph)."""
+        if loss_pinned is not None:
+            if loss_pinned.is_cuda or not loss_pinned.is_pinned() or loss_pinned.numel() < 1 or loss_pinned.element_size() != 4:
+                raise ValueError("loss_pinned must be a pinned float32 host tensor")
+            _check(lib.ftp_train_step(self.h, _ptr(x), _ptr(labels), int(inputs_on_host), lr,
+                                      C.cast(loss_pinned.data_ptr(), _P(_f32)), _stream(stream)))
+            return None
         loss = _f32()
         _check(lib.ftp_train_step(self.h, _ptr(x), _ptr(labels), int(inputs_on_host), lr,
                                   C.byref(loss) if want_loss else None, _stream(stream)))

@@ -406,3 +406,42 @@ def test_guard_zones_stay_intact_on_ragged_shapes_and_catch_a_planted_overwrite(
     gm.dev_ws[base + off] = 0xA5
     assert gm.ftp_check_guards() == n
     gm.close()
+
+
+def test_train_step_captured_into_a_graph_with_host_inputs_equals_eager_calls():
+    """A step recorded into a CUDA graph with pinned host inputs and a pinned loss (the copies are nodes of the graph):
+    three replays with the host buffers refilled in between give bit for bit the losses and weights of three eager calls."""
+    import torch
+    ls, cfg = synth.tiny_mbv2()
+    batches = [synth.make_batch(70 + k, cfg) for k in range(3)]
+    first = synth.make_batch(69, cfg)
+    ref = make_gpu(ls, cfg, 70)
+    gm = make_gpu(ls, cfg, 70)
+    # one eager step on both before recording: whether a momentum buffer is initialised (a unit's first update) or
+    # accumulated is decided when the step is recorded, so a graph is recorded after the first update
+    for mdl in (ref, gm):
+        mdl.ftp_train_step(torch.from_numpy(first[0]).pin_memory(), torch.from_numpy(first[1]).pin_memory(), 0.01, inputs_on_host=True)
+    ref_losses = [ref.ftp_train_step(torch.from_numpy(x).pin_memory(), torch.from_numpy(y).pin_memory(), 0.01, inputs_on_host=True)
+                  for x, y in batches]
+    xh, yh = torch.from_numpy(batches[0][0].copy()).pin_memory(), torch.from_numpy(batches[0][1].copy()).pin_memory()
+    loss_pin = torch.zeros(1, dtype=torch.float32).pin_memory()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    state = [gm.ftp_get_tensor(F.T_WEIGHTS, u) for u in range(gm.L)]        # capture runs nothing: the weights stay as loaded
+    with torch.cuda.graph(g, stream=side):
+        gm.ftp_train_step(xh, yh, 0.01, inputs_on_host=True, loss_pinned=loss_pin)
+    for u in range(gm.L):
+        assert np.array_equal(gm.ftp_get_tensor(F.T_WEIGHTS, u), state[u])
+    losses = []
+    for x, y in batches:
+        xh.copy_(torch.from_numpy(x)); yh.copy_(torch.from_numpy(y))
+        g.replay()
+        torch.cuda.synchronize()
+        losses.append(float(loss_pin[0]))
+    assert losses == [float(np.float32(v)) for v in ref_losses]
+    for u in range(gm.L):
+        assert np.array_equal(gm.ftp_get_tensor(F.T_WEIGHTS, u), ref.ftp_get_tensor(F.T_WEIGHTS, u))
+    with pytest.raises(ValueError):
+        gm.ftp_train_step(xh, yh, 0.01, inputs_on_host=True, loss_pinned=torch.zeros(1))      # not pinned
+    gm.close(); ref.close()
