@@ -1658,7 +1658,18 @@ __global__ void __launch_bounds__(256) gap_fwd_kernel(const T* __restrict__ x, T
     float s[V];
 #pragma unroll
     for (int e = 0; e < V; ++e) s[e] = 0.f;
-    for (int p = 0; p < HW; ++p) {
+    // eight positions per trip: their loads are issued together, the additions keep the order of the positions
+    int p = 0;
+    for (; p + 8 <= HW; p += 8) {
+        float v[8][V];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) ldv<V>(x + (n * HW + p + u) * C + c, v[u]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int e = 0; e < V; ++e) s[e] += v[u][e];
+    }
+    for (; p < HW; ++p) {
         float v[V];
         ldv<V>(x + (n * HW + p) * C + c, v);
 #pragma unroll
