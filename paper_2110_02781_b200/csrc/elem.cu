@@ -2006,8 +2006,16 @@ PartialSums bn_bwd_reduce(const T* dz, const T* y, long long M, int C, const Fol
     constexpr int W = 4;      // columns per thread: four keep the per-channel constants of a thread at a register count that leaves four blocks per SM
     if (fp.vec == V && aligned16(dz) && aligned16(y) && aligned16(scale) && aligned16(shift) && aligned16(mean) && aligned16(mean_lo) && aligned16(rstd)) {
         const int copies = fp.fused ? fp.copies_bwd : 1;
-        launch(bn_bwd_reduce_kernel<T, W>, dim3(fold_grid_w(fp, W)), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial, copies);
-        return PartialSums{partial, fp.chunks * (fp.f / copies), fp.f / copies};
+        // the plan counts column tiles of V columns per thread; with W < V (bf16) there are V / W times as many, so the rows are
+        // cut into that many fewer chunks to keep the grid at the planned number of blocks (config 3: 5.050 -> 5.025 ms)
+        FoldPlan q = fp;
+        if (V > W) {
+            const int ch = std::max(1, fp.chunks * W / V);
+            const int rpc = (fp.rows + ch - 1) / ch;
+            q.chunks = (fp.rows + rpc - 1) / rpc;
+        }
+        launch(bn_bwd_reduce_kernel<T, W>, dim3(fold_grid_w(q, W)), dim3(32, 8), 0, st, dz, y, q.rows, q.cols, fold_rpc(q), C, scale, shift, mean, mean_lo, rstd, act, partial, copies);
+        return PartialSums{partial, q.chunks * (q.f / copies), q.f / copies};
     }
     // the scalar fallback keeps the plain partial layout
     launch(bn_bwd_reduce_kernel<T, 1>, dim3((fp.cols + 31) / 32, fp.chunks), dim3(32, 8), 0, st, dz, y, fp.rows, fp.cols, fold_rpc(fp), C, scale, shift, mean, mean_lo, rstd, act, partial, 1);
