@@ -199,6 +199,10 @@ LAYER_CASES = [  # kind, hw, cin, cout, k, stride, act, batch
     ("CONV2D", 16, 64, 64, 3, 1, 1, 8),       # VGG dense 3x3
     ("CONV2D", 8, 128, 256, 3, 1, 1, 8),
     ("CONV2D", 4, 512, 512, 3, 1, 1, 16),
+    # enough tiles for the persistent product (two or more per SM), a ragged last row tile and a last column tile of 16 columns
+    ("CONV2D", 56, 24, 144, 1, 1, 2, 7),
+    ("CONV2D", 28, 64, 96, 1, 1, 0, 50),
+    ("CONV2D", 28, 96, 64, 1, 1, 0, 50),      # 64-wide tiles, two reduction blocks
 ]
 
 
