@@ -431,6 +431,7 @@ struct TcWgParams {
     int rows_per_split;  // multiple of 64
     int* err;
     ConvTap conv;        // enabled: grid.z = splits * 9, X is read through a 4-D map shifted by the tap
+    int pair;            // conv with Mo <= 64: a block takes two taps, one per 64-row half of its tile (grid.z = splits * 5)
 };
 
 // out[z][i][j] = sum over rows r of split z of X[r][i] * dY[r][j].  Both operands are read as they lie in memory
@@ -446,8 +447,10 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int i0 = blockIdx.x * TC_BM, j0 = blockIdx.y * BN;
-    const int taps = p.conv.enabled ? 9 : 1;
-    const int split = blockIdx.z / taps, tap = blockIdx.z - split * taps;
+    // 64 input channels fill half of the 128-row tile: the other half then takes the next tap (rows 64.. = tap + 1)
+    const int taps = p.conv.enabled ? 9 : 1, groups = p.pair ? 5 : taps;
+    const int split = blockIdx.z / groups, grp = blockIdx.z - split * groups, tap = p.pair ? 2 * grp : grp;
+    const bool second = p.pair && tap + 1 < 9;
     const int rbeg = split * p.rows_per_split, rend = min(p.R, rbeg + p.rows_per_split);
     const int num_kb = (rend - rbeg + 63) / 64;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_STAGES]), accum = smem_u32(&bars[2 * TC_STAGES]);
@@ -477,7 +480,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
                 if (kb >= TC_STAGES && !mbar_wait(empty0 + 8 * s, ph ^ 1, p.err, 4)) break;
                 const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
                 const int r = rbeg + kb * 64;
-                mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+                mbar_expect_tx(full0 + 8 * s, (p.pair && !second) ? STAGE_BYTES - SLAB : STAGE_BYTES);
                 if (!p.conv.enabled) {
                     tma_load_2d(sa, &mapX, i0, r, full0 + 8 * s);
                     tma_load_2d(sa + SLAB, &mapX, i0 + 64, r, full0 + 8 * s);
@@ -485,7 +488,11 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
                     const int tr = tap / 3, ts = tap - 3 * tr;
                     const int hw = p.conv.H * p.conv.W, img = r / hw, h0 = (r - img * hw) / p.conv.W;
                     tma_load_4d(sa, &mapX, i0, ts - 1, h0 + tr - 1, img, full0 + 8 * s);
-                    tma_load_4d(sa + SLAB, &mapX, i0 + 64, ts - 1, h0 + tr - 1, img, full0 + 8 * s);
+                    if (!p.pair) tma_load_4d(sa + SLAB, &mapX, i0 + 64, ts - 1, h0 + tr - 1, img, full0 + 8 * s);
+                    else if (second) {
+                        const int tr2 = (tap + 1) / 3, ts2 = tap + 1 - 3 * tr2;
+                        tma_load_4d(sa + SLAB, &mapX, i0, ts2 - 1, h0 + tr2 - 1, img, full0 + 8 * s);
+                    }                                                // no second tap: rows 64.. of the tile are never stored
                 }
 #pragma unroll
                 for (int t = 0; t < BN / 64; ++t) tma_load_2d(sb + t * SLAB, &mapY, j0 + 64 * t, r, full0 + 8 * s);
@@ -522,8 +529,10 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
         const int q = warp & 3;
         if (num_kb > 0 ? mbar_wait(accum, 0, p.err, 6) : true) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int i = i0 + q * 32 + lane;
-            float* orow = p.out + (((long long)split * taps + tap) * p.Mo + i) * p.No;
+            const int row = q * 32 + lane;
+            const int i = p.pair ? (row & 63) : i0 + row, otap = p.pair ? tap + (row >> 6) : tap;
+            const bool row_ok = i < p.Mo && otap < taps;
+            float* orow = p.out + (((long long)split * taps + otap) * p.Mo + i) * p.No;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
@@ -533,7 +542,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
                     for (int e = 0; e < 32; ++e) r[e] = 0u;
                 }
                 const int jb = j0 + c * 32;
-                if (i < p.Mo) {
+                if (row_ok) {
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
                         if (jb + g * 4 < p.No)
@@ -549,6 +558,12 @@ __global__ void __launch_bounds__(TC_THREADS) tc_wgrad_kernel(const __grid_const
 }
 
 struct TcWgPlan { int S, rows_per_split; };
+// FTP_TC_WG_PAIR=0: one tap per block whatever the channel count (A/B measurements)
+static bool wgrad3x3_pairs_taps(int Mo) {
+    static int on = -1;
+    if (on < 0) { const char* e = std::getenv("FTP_TC_WG_PAIR"); on = (e && std::strcmp(e, "0") == 0) ? 0 : 1; }
+    return on != 0 && Mo <= 64;
+}
 TcWgPlan plan_tc_wgrad(long long R, int Mo, int No) {
     const long long tiles = ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
     long long S = (2LL * sm_count() + tiles - 1) / tiles;
@@ -741,7 +756,7 @@ bool launch_wgrad(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out, l
         if (cudaFuncSetAttribute(tc_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
         configured = true;
     }
-    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{0, 0, 0, 0, 0, 0}};
+    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{0, 0, 0, 0, 0, 0}, 0};
     launch(tc_wgrad_kernel<BN>, dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S), dim3(TC_THREADS), smem, st, mx, my, p);
     return true;
 }
@@ -754,13 +769,14 @@ bool launch_wgrad3x3(const __nv_bfloat16* X, const __nv_bfloat16* dY, float* out
     if (!make_map_4d(&mx, X, N, H, W, Mo, 64) || !make_map_2d(&my, dY, R, No, 64)) return false;
     constexpr int smem = TC_STAGES * (2 + BN / 64) * 64 * 64 * 2 + 1024;
     if (cudaFuncSetAttribute(tc_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{1, H, W, 0, 0, 0}};
-    launch(tc_wgrad_kernel<BN>, dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S * 9), dim3(TC_THREADS), smem, st, mx, my, p);
+    const int pair = wgrad3x3_pairs_taps(Mo) ? 1 : 0;
+    TcWgParams p{out, Mo, No, (int)R, w.rows_per_split, err, ConvTap{1, H, W, 0, 0, 0}, pair};
+    launch(tc_wgrad_kernel<BN>, dim3((Mo + TC_BM - 1) / TC_BM, (No + BN - 1) / BN, w.S * (pair ? 5 : 9)), dim3(TC_THREADS), smem, st, mx, my, p);
     return true;
 }
 
 TcWgPlan plan_tc_wgrad3x3(long long R, int Mo, int No) {
-    const long long tiles = 9LL * ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
+    const long long tiles = (wgrad3x3_pairs_taps(Mo) ? 5LL : 9LL) * ((Mo + TC_BM - 1) / TC_BM) * ((No + 127) / 128);
     long long S = (2LL * sm_count() + tiles - 1) / tiles;
     const long long maxS = (R + 511) / 512;
     long long cap = (8LL << 20) / (9LL * Mo * No);
