@@ -12,6 +12,7 @@ independent replica of the same workload ("replicas only"); value is the aggrega
 """
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -432,7 +433,14 @@ def measure(args, wl_key, reps, steps, warmup, local_rank, replicas, batch=None,
                   "h2d_bytes_per_step": int(xh.numel() * xh.element_size() + yh.numel() * 4), "d2h_bytes_per_step": 4,
                   "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps, "launch": "eager" if dynamic else e2e_launch}
 
-    # per-kernel roofline: three more steps with every launch bracketed by events
+    # per-kernel roofline: three more steps with every launch bracketed by events.  Eager launches are issued more
+    # slowly than the GPU runs them, and an event pair around a launch the GPU has to wait for would time the host
+    # (tensor-map encoding, the launch call), not the kernel: so untraced steps are queued first, enough of them that
+    # the host stays ahead of the device for the whole of the traced steps.
+    torch.cuda.synchronize()
+    lead = max(8, int(math.ceil(60.0 / max(ms / steps, 1e-3))))
+    for _ in range(min(lead, 400)):
+        step_eager()
     m.ftp_trace_enable(True)
     for _ in range(3):
         step_eager()
