@@ -499,7 +499,10 @@ ftp_status fwd_range(ftp_model* m, int a, int b, const void* act_in, void* act_o
 
 // ---- backward of a unit range -----------------------------------------------------------------------------
 template <typename T>
-ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* grad_in, bool internal, cudaStream_t st) {
+// defer_join (the training step): the caller's stream does not wait for the second stream at the end of this range -- the
+// backward pass of the next stage does not depend on this stage's weight gradients, only the update does -- and the
+// buffers those weight gradients still read stay listed in m->pending; the caller joins once (join_side) before the update.
+ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* grad_in, bool internal, cudaStream_t st, bool defer_join = false) {
     const int first = m->unit_first[a], last = m->unit_last[b - 1];
     const double es = (double)m->esize;
     for (int i = first; i <= last; ++i)
@@ -517,12 +520,16 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
     // overwrites the buffer that the weight gradient reads (and once at the end).  Per-unit timing and tracing keep
     // everything on one stream.
     const bool side_on = m->overlap && !m->unit_events && !m->trace;
-    struct Pending { const void* buf; cudaEvent_t done; };
-    std::vector<Pending> pending;
-    struct Join {                                            // the second stream always rejoins the caller's stream
-        ftp_model* m; cudaStream_t st; bool used;
-        ~Join() { if (used && cudaEventRecord(m->ev_side.back(), m->side) == cudaSuccess) cudaStreamWaitEvent(st, m->ev_side.back(), 0); }
-    } join{m, st, false};
+    std::vector<SidePending>& pending = m->pending;
+    struct Join {                                            // the second stream always rejoins the caller's stream, here or in join_side
+        ftp_model* m; cudaStream_t st; bool used, deferred;
+        ~Join() {
+            if (used && deferred) { m->side_unjoined = true; return; }
+            if ((used || m->side_unjoined) && cudaEventRecord(m->ev_side.back(), m->side) == cudaSuccess) cudaStreamWaitEvent(st, m->ev_side.back(), 0);
+            m->side_unjoined = false;
+            m->pending.clear();
+        }
+    } join{m, st, false, false};
     auto fork = [&](int i) -> cudaStream_t {                 // stream for the weight gradient of operation i
         if (!side_on) return st;
         cudaEventRecord(m->ev_fork[i], st);
@@ -703,13 +710,22 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
         }
     }
     if (m->unit_events) cudaEventRecord(m->ev_b[a], st);
-    return check_launches("backward");
+    const ftp_status launched = check_launches("backward");
+    join.deferred = defer_join && launched == FTP_OK;
+    return launched;
 }
 
 ftp_status check_range(const ftp_model* m, int a, int b, const char* who) {
     FTP_REQUIRE(m, FTP_EINVAL, "%s: null model", who);
     FTP_REQUIRE(a >= 0 && b <= m->L && a < b, FTP_EINVAL, "%s: need 0 <= a < b <= L (a=%d, b=%d, L=%d)", who, a, b, m->L);
     return FTP_OK;
+}
+
+// the caller's stream waits for everything the second stream was given by ranges that left without joining
+void join_side(ftp_model* m, cudaStream_t st) {
+    if (m->side_unjoined && cudaEventRecord(m->ev_side.back(), m->side) == cudaSuccess) cudaStreamWaitEvent(st, m->ev_side.back(), 0);
+    m->side_unjoined = false;
+    m->pending.clear();
 }
 
 ftp_status sgd_range(ftp_model* m, int a, int b, float lr, float* snap_dev, float* snap_host, cudaStream_t st) {
@@ -751,9 +767,11 @@ ftp_status train_step_t(ftp_model* m, const void* x, const int32_t* labels, floa
     if (timing) cudaEventRecord(m->ev_sf[m->n_stages], st);
     for (int s = m->n_stages - 1; s >= 0; --s) {
         if (timing) cudaEventRecord(m->ev_sb[s + 1], st);
-        ftp_status r = bwd_range<T>(m, m->points[s], m->points[s + 1], nullptr, nullptr, true, st);
-        if (r != FTP_OK) return r;
+        // stage timing wants each stage's weight gradients inside its own interval: those runs join per stage
+        ftp_status r = bwd_range<T>(m, m->points[s], m->points[s + 1], nullptr, nullptr, true, st, !timing && m->defer_join);
+        if (r != FTP_OK) { join_side(m, st); return r; }
     }
+    join_side(m, st);
     if (timing) { cudaEventRecord(m->ev_sb[0], st); m->timed_stages = m->n_stages; }
     for (int s = 0; s < m->n_stages; ++s) {
         ftp_status r = sgd_range(m, m->points[s], m->points[s + 1], lr, nullptr, nullptr, st);
@@ -841,6 +859,15 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
     {   // second stream and its fork / join events: one pair per operation, created here so that nothing is created inside a stream capture
         const char* e = std::getenv("FTP_OVERLAP");
         m->overlap = !(e && std::strcmp(e, "0") == 0);
+        {   // One join before the update instead of one per stage: measured 1.403 -> 1.377 ms on VGG-16 (few, long weight
+            // gradients), but 3.254 -> 3.280 ms and 4.97 -> 5.01 ms on the MobileNetV2 configurations, whose many short weight
+            // gradients then pile up beside the large early layers of the next stage.  Default: only for networks without
+            // depthwise convolutions; FTP_DEFER_JOIN=0 / 1 overrides.
+            bool has_dw = false;
+            for (const Op& o : m->ops) has_dw = has_dw || o.d.kind == FTP_DWCONV3x3;
+            const char* dj = std::getenv("FTP_DEFER_JOIN");
+            m->defer_join = dj ? std::strcmp(dj, "0") != 0 : !has_dw;
+        }
         const char* ps = std::getenv("FTP_PRODUCER_STATS");          // 0: batch-norm statistics always by their own kernel (A/B measurements)
         m->producer_stats = !(ps && std::strcmp(ps, "0") == 0);
         // FTP_BWD_SUMS: 0 = the first pass of every batch-norm backward by its own kernel, 1 = from the depthwise backward

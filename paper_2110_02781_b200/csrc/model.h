@@ -51,6 +51,8 @@ struct TraceSlot { cudaEvent_t e0, e1; ftp_trace_rec rec; };
 
 }  // namespace ftp
 
+struct SidePending { const void* buf; cudaEvent_t done; };
+
 struct ftp_model {
     ftp_model_cfg cfg;
     std::vector<ftp::Op> ops;
@@ -74,6 +76,9 @@ struct ftp_model {
     // weight gradients run on a second stream beside the chain of input gradients; they have scratch of their own
     float* red_side; ftp::FinScratch fin_side;
     cudaStream_t side; std::vector<cudaEvent_t> ev_fork, ev_side; bool overlap; bool producer_stats; bool bwd_sums_on;
+    std::vector<SidePending> pending;             // buffers that weight gradients on the second stream still read, with the event that ends the read
+    bool side_unjoined = false;                   // the second stream holds work the caller's stream has not waited for yet
+    bool defer_join = false;                      // the training step joins the second stream once, before the update, instead of after every stage
     std::vector<ftp::TransposeEntryDev> tp_host; std::vector<int> tp_first;   // tp_first[u]: first entry of unit u (L + 1 values)
     ftp::TransposeEntryDev* tp_dev;
     void* dpre; size_t dpre_bytes;
