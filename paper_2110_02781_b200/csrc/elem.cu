@@ -2274,7 +2274,7 @@ size_t dwconv_bwd_stats_doubles(const ConvGeom& g) {
 
 template <typename T>
 bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
-                      cudaStream_t st, const BnXform* x_xform, const BnBwdSumsReq* sums) {
+                      cudaStream_t st, const BnXform* x_xform, const BnBwdSumsReq* sums, cudaStream_t fin_st, cudaEvent_t fin_fork) {
     const bool xf = x_xform != nullptr;
     const BnXform xv = xf ? *x_xform : BnXform{nullptr, nullptr, nullptr, 0.f, 0.f};
     const bool xf_vec = !xf || (aligned16(xv.mean) && aligned16(xv.scale) && aligned16(xv.offset));
@@ -2297,11 +2297,14 @@ bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, 
     } else if (xf) launch(dw3_bwd_rows_kernel<T, true, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);
     else launch(dw3_bwd_rows_kernel<T, false, false>, grid, dim3(256), 0, st, x, dy, w, addend, dx, scratch, g.N, g.H, g.W, g.Cin, pl.RH, pl.HC, xv, (const float*)nullptr, (double*)nullptr);
     const int gx = (int)pl.gx;
-    if (gx <= DW_FIN_SMALL) launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
+    // the sums over the blocks' weight-gradient partials feed only the update: the caller may give them another stream
+    if (fin_st == nullptr) fin_st = st;
+    if (fin_st != st) { cudaEventRecord(fin_fork, st); cudaStreamWaitEvent(fin_st, fin_fork, 0); }
+    if (gx <= DW_FIN_SMALL) launch(dw_wgrad_finalize_small_kernel, dim3((g.Cin + 31) / 32, 9), dim3(32, 8), 0, fin_st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw);
     else {
         int slices = gx / (4 * FIN_Y);
         slices = slices < 1 ? 1 : (slices > FIN_GMAX ? FIN_GMAX : slices);
-        launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, slices, 9), dim3(FIN_X, FIN_Y), 0, st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw, fin);
+        launch(dw_wgrad_finalize_kernel, dim3((g.Cin + FIN_X - 1) / FIN_X, slices, 9), dim3(FIN_X, FIN_Y), 0, fin_st, (const float*)scratch, gx, 1, g.Cin, g.Cin, dw, fin);
     }
     return true;
 }
@@ -2389,7 +2392,7 @@ void f32_to_bf16(const float* src, __nv_bfloat16* dst, long long n, cudaStream_t
     template void dwconv_fwd<T>(const T*, const float*, T*, const ConvGeom&, cudaStream_t, const ColStatsReq*, const BnXform*); \
     template void dwconv_dgrad<T>(const T*, const float*, const T*, T*, const ConvGeom&, cudaStream_t);                     \
     template void dwconv_wgrad<T>(const T*, const T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*); \
-    template bool dwconv_bwd_fused<T>(const T*, const T*, const float*, const T*, T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*, const BnBwdSumsReq*); \
+    template bool dwconv_bwd_fused<T>(const T*, const T*, const float*, const T*, T*, float*, float*, const ConvGeom&, const FinScratch&, cudaStream_t, const BnXform*, const BnBwdSumsReq*, cudaStream_t, cudaEvent_t); \
     template void maxpool_fwd<T>(const T*, T*, int, int, int, int, cudaStream_t);                                           \
     template void maxpool_bwd<T>(const T*, const T*, T*, int, int, int, int, cudaStream_t);                                 \
     template void gap_fwd<T>(const T*, T*, int, int, int, cudaStream_t);                                                    \

@@ -199,7 +199,10 @@ struct BnBwdSumsReq {
 size_t dwconv_bwd_stats_doubles(const ConvGeom& g);
 template <typename T>
 bool dwconv_bwd_fused(const T* x, const T* dy, const float* w, const T* addend, T* dx, float* dw, float* scratch, const ConvGeom& g, const FinScratch& fin,
-                      cudaStream_t st, const BnXform* x_xform = nullptr, const BnBwdSumsReq* sums = nullptr);
+                      cudaStream_t st, const BnXform* x_xform = nullptr, const BnBwdSumsReq* sums = nullptr, cudaStream_t fin_st = nullptr,
+                      cudaEvent_t fin_fork = nullptr);
+// fin_st (with fin_fork, an event of the caller): the kernel that adds the blocks' weight-gradient partials runs on that stream, after
+// the main kernel (fin then belongs to that stream, and scratch must stay untouched until it has run)
 
 template <typename T>
 void maxpool_fwd(const T* x, T* y, int N, int H, int W, int C, cudaStream_t st);

@@ -285,7 +285,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     }
     m.grad = (float*)bp.take((size_t)m.P * 4);
     m.state_backup = (float*)bp.take((size_t)std::max<long long>(m.R, 1) * 4);
-    size_t max_act = 0, red = 0, foldd = 0, dpre = 0, finp = 64, finc = 1, fcin = 64;
+    size_t max_act = 0, red = 0, dwp = 0, foldd = 0, dpre = 0, finp = 64, finc = 1, fcin = 64;
     for (int i = 0; i < n; ++i) {
         Op& o = m.ops[i];
         const size_t obytes = (size_t)o.out_elems * (o.out_f32 ? 4 : es);
@@ -317,6 +317,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
             if (o.d.kind == FTP_FC) fcin = std::max(fcin, (size_t)o.in_elems);
         } else if (o.d.kind == FTP_DWCONV3x3) {
             red = std::max(red, dwconv_wgrad_scratch_floats(o.g));
+            dwp = std::max(dwp, dwconv_wgrad_scratch_floats(o.g));
             foldd = std::max(foldd, dwconv_bwd_stats_doubles(o.g));
             finp = std::max(finp, fin_part_doubles(o.C, 9)); finc = std::max(finc, fin_counter_count(o.C, 9));
         }
@@ -329,6 +330,7 @@ ftp_status layout(ftp_model& m, char* dev_base, size_t* dev_total, size_t* pinne
     for (auto& p : m.slots) p = bp.take(m.slot_bytes);
     m.red_floats = std::max<size_t>(red, 64); m.red_scratch = (float*)bp.take(m.red_floats * 4);
     m.red_side = (float*)bp.take(m.red_floats * 4);
+    for (int k = 0; k < 4; ++k) m.dw_part[k] = (float*)bp.take(std::max<size_t>(dwp, 64) * 4);
     m.fold_doubles = std::max<size_t>(foldd, 64); m.fold_scratch = (double*)bp.take(m.fold_doubles * 8);
     m.dpre_bytes = std::max<size_t>(dpre, 256); m.dpre = bp.take(m.dpre_bytes);
     m.tc_err = (int*)bp.take(256);
@@ -654,7 +656,13 @@ ftp_status bwd_range(ftp_model* m, int a, int b, const void* grad_out, void* gra
                     BnBwdSumsReq sreq{nullptr, m->fold_scratch, &bwd_sums};
                     const BnBwdSumsReq* sums = nullptr;
                     if (xf && m->bwd_sums_on) { sreq.rstd = m->ops[i - 1].rstd; sums = &sreq; }
-                    if (dwconv_bwd_fused<T>((const T*)in, (const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, gr + o.w_off, m->red_scratch, o.g, m->fin, st, xf, sums)) {
+                    // the second pass over the blocks' weight-gradient partials feeds only the update: second stream, its own buffers in turn
+                    const bool fin_side = side_on && m->dw_fin_side;
+                    float* part = m->red_scratch;
+                    if (fin_side) { part = m->dw_part[m->dw_rot]; m->dw_rot = (m->dw_rot + 1) % 4; before_write(part); }
+                    if (dwconv_bwd_fused<T>((const T*)in, (const T*)go, ar.w + o.w_off, (const T*)addend, (T*)gi, gr + o.w_off, part, o.g, fin_side ? m->fin_side : m->fin,
+                                            st, xf, sums, fin_side ? m->side : st, m->ev_fork[i])) {
+                        if (fin_side) { join.used = true; forked(i, part); }
                         bwd_sums_for = bwd_sums.entries > 0 ? i - 1 : -1;
                         break;
                     }
@@ -865,6 +873,8 @@ extern "C" ftp_status ftp_build_model(const ftp_layer_desc* layers, int32_t n, c
             // depthwise convolutions; FTP_DEFER_JOIN=0 / 1 overrides.
             bool has_dw = false;
             for (const Op& o : m->ops) has_dw = has_dw || o.d.kind == FTP_DWCONV3x3;
+            const char* df = std::getenv("FTP_DW_FIN_SIDE");
+            m->dw_fin_side = !(df && std::strcmp(df, "0") == 0);
             const char* dj = std::getenv("FTP_DEFER_JOIN");
             m->defer_join = dj ? std::strcmp(dj, "0") != 0 : !has_dw;
         }

@@ -76,6 +76,7 @@ struct ftp_model {
     // weight gradients run on a second stream beside the chain of input gradients; they have scratch of their own
     float* red_side; ftp::FinScratch fin_side;
     cudaStream_t side; std::vector<cudaEvent_t> ev_fork, ev_side; bool overlap; bool producer_stats; bool bwd_sums_on;
+    float* dw_part[4]; int dw_rot = 0; bool dw_fin_side = true;   // partial sums of the fused depthwise backward kernels, in turn: their second pass runs on the second stream
     std::vector<SidePending> pending;             // buffers that weight gradients on the second stream still read, with the event that ends the read
     bool side_unjoined = false;                   // the second stream holds work the caller's stream has not waited for yet
     bool defer_join = false;                      // the training step joins the second stream once, before the update, instead of after every stage
