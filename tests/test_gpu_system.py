@@ -445,3 +445,55 @@ def test_train_step_captured_into_a_graph_with_host_inputs_equals_eager_calls():
     with pytest.raises(ValueError):
         gm.ftp_train_step(xh, yh, 0.01, inputs_on_host=True, loss_pinned=torch.zeros(1))      # not pinned
     gm.close(); ref.close()
+
+
+def _three_steps(net, idx, points, env):
+    """Weights and losses after three training steps of a model built under the given environment switches."""
+    import os
+    import torch
+    ls, cfg = net
+    old = {k: os.environ.get(k) for k in env}
+    os.environ.update(env)
+    try:
+        m = make_gpu(ls, cfg, idx)            # the switches are read when the model is built
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+    m.ftp_set_partition(points)
+    bf16 = cfg["precision"] == 1
+    losses = []
+    for it in range(3):
+        x, y = synth.make_batch(idx, cfg, it)
+        xt = torch.from_numpy(x).to(torch.bfloat16) if bf16 else torch.from_numpy(x)
+        losses.append(m.ftp_train_step(xt.cuda(), torch.from_numpy(y).cuda(), 0.01))
+    w = [m.ftp_get_tensor(F.T_WEIGHTS, u) for u in range(m.L)]
+    m.close()
+    return losses, w
+
+
+def test_one_join_before_the_update_changes_no_bit():
+    """Networks without depthwise convolutions let the weight-gradient stream run on across the stages of a training
+    step and join it once, before the update; with the join after every stage the same step gives the same bits
+    (bf16 VGG groups at their real widths, three stages, 64-channel layers on the paired-tap weight gradient)."""
+    net = synth.vgg16(32, 8, 10, 1, plan=[64, 64, "M", 128, 128, "M", 128, "M"])
+    a = _three_steps(net, 63, [0, 2, 4, 6], {"FTP_DEFER_JOIN": "1"})
+    b = _three_steps(net, 63, [0, 2, 4, 6], {"FTP_DEFER_JOIN": "0"})
+    assert a[0] == b[0]
+    assert all(np.array_equal(p, q) for p, q in zip(a[1], b[1]))
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_depthwise_partial_sums_on_the_second_stream_change_no_bit(precision):
+    """The kernel that adds the per-block weight-gradient partials of the fused depthwise backward kernels runs on the
+    second stream from buffers handed out in turn; on the main stream it gives the same bits (and so does the join taken
+    once before the update, which these networks do not use by default)."""
+    ls, cfg = synth.tiny_mbv2(precision=precision)
+    pts = [0, 2, 4, synth.num_units(ls)]
+    a = _three_steps((ls, cfg), 71, pts, {"FTP_DW_FIN_SIDE": "1"})
+    b = _three_steps((ls, cfg), 71, pts, {"FTP_DW_FIN_SIDE": "0"})
+    c = _three_steps((ls, cfg), 71, pts, {"FTP_DW_FIN_SIDE": "1", "FTP_DEFER_JOIN": "1"})
+    assert a[0] == b[0] == c[0]
+    assert all(np.array_equal(p, q) and np.array_equal(p, r) for p, q, r in zip(a[1], b[1], c[1]))
